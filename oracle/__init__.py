@@ -1,0 +1,250 @@
+"""ctypes front end of the CPU oracle (oracle/disco_oracle.cpp).
+
+TEST INFRASTRUCTURE ONLY: imported by tests/, by the smoke check and by the
+benchmark's CPU-baseline leg.  The CUDA library and its Python binding never
+import this package, and this package never imports them.
+
+Arrays are numpy.  bf16 tensors are passed as uint16 bit patterns
+(``torch_tensor.view(torch.uint16).numpy()``).  All floating-point results are
+float64.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+from dataclasses import dataclass
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "disco_oracle.cpp")
+_LIB = os.path.join(_HERE, "liboracle.so")
+
+K_TOP = 10  # Eq. 2 footnote: k = 10 in all of the paper's experiments
+
+
+def build(force: bool = False) -> str:
+    """Compile liboracle.so with the host C++ compiler (no CUDA involved)."""
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        cmd = ["g++", "-O2", "-std=c++17", "-fPIC", "-shared", "-pthread", "-o", _LIB, _SRC]
+        subprocess.run(cmd, check=True)
+    return _LIB
+
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    global _lib
+    if _lib is None:
+        _lib = ctypes.CDLL(build())
+    return _lib
+
+
+def hardware_threads() -> int:
+    return int(lib().oracle_hardware_threads())
+
+
+# --------------------------------------------------------------------------- helpers
+def _p(a, ctype):
+    if a is None:
+        return None
+    return a.ctypes.data_as(ctypes.POINTER(ctype))
+
+
+def _u16(a) -> np.ndarray:
+    a = np.ascontiguousarray(a)
+    if a.dtype != np.uint16:
+        raise TypeError("bf16 data must be passed as uint16 bit patterns")
+    return a
+
+
+def _check(rc: int, what: str) -> None:
+    if rc != 0:
+        raise ValueError(f"{what}: oracle rejected its arguments (rc={rc})")
+
+
+# --------------------------------------------------------------------------- steps
+def project(W: np.ndarray, H: np.ndarray, nthreads: int = 1) -> np.ndarray:
+    """z[r, v] = sum_j W[v, j] H[r, j] in float64; W [V,d], H [R,d] (bf16 bits)."""
+    W, H = _u16(W), _u16(H)
+    V, d = W.shape
+    R = H.shape[0]
+    assert H.shape[1] == d
+    z = np.empty((R, V), dtype=np.float64)
+    _check(lib().oracle_project(_p(W, ctypes.c_uint16), _p(H, ctypes.c_uint16), V, d, R,
+                                _p(z, ctypes.c_double), nthreads), "project")
+    return z
+
+
+def argmax(z: np.ndarray):
+    """(lowest index of the maximum, gap between the two largest values)."""
+    z = np.ascontiguousarray(z, dtype=np.float64)
+    best = ctypes.c_int32()
+    gap = ctypes.c_double()
+    _check(lib().oracle_argmax(_p(z, ctypes.c_double), z.shape[0], ctypes.byref(best),
+                               ctypes.byref(gap)), "argmax")
+    return int(best.value), float(gap.value)
+
+
+def softmax(z: np.ndarray) -> np.ndarray:
+    z = np.ascontiguousarray(z, dtype=np.float64)
+    y = np.empty_like(z)
+    _check(lib().oracle_softmax(_p(z, ctypes.c_double), z.shape[0], _p(y, ctypes.c_double)),
+           "softmax")
+    return y
+
+
+def topk(y: np.ndarray, k: int = K_TOP):
+    y = np.ascontiguousarray(y, dtype=np.float64)
+    vals = np.empty(k, dtype=np.float64)
+    ids = np.empty(k, dtype=np.int32)
+    _check(lib().oracle_topk(_p(y, ctypes.c_double), y.shape[0], k, _p(vals, ctypes.c_double),
+                             _p(ids, ctypes.c_int32)), "topk")
+    return vals, ids
+
+
+def entropy(y: np.ndarray) -> float:
+    y = np.ascontiguousarray(y, dtype=np.float64)
+    e = ctypes.c_double()
+    _check(lib().oracle_entropy(_p(y, ctypes.c_double), y.shape[0], ctypes.byref(e)), "entropy")
+    return float(e.value)
+
+
+def features(y: np.ndarray, pos: int, k: int = K_TOP) -> np.ndarray:
+    y = np.ascontiguousarray(y, dtype=np.float64)
+    x = np.empty(k + 2, dtype=np.float64)
+    _check(lib().oracle_features(_p(y, ctypes.c_double), y.shape[0], k, int(pos),
+                                 _p(x, ctypes.c_double)), "features")
+    return x
+
+
+@dataclass
+class Classifier:
+    """Parameters of the 2-layer halt classifier: nfeat -> H (ReLU) -> 1 (logistic)."""
+    W1: np.ndarray  # [H, nfeat] float32
+    b1: np.ndarray  # [H]
+    w2: np.ndarray  # [H]
+    b2: np.ndarray  # [1]
+
+    def __post_init__(self):
+        self.W1 = np.ascontiguousarray(self.W1, dtype=np.float32)
+        self.b1 = np.ascontiguousarray(self.b1, dtype=np.float32)
+        self.w2 = np.ascontiguousarray(self.w2, dtype=np.float32)
+        self.b2 = np.ascontiguousarray(self.b2, dtype=np.float32).reshape(1)
+
+    @property
+    def H(self) -> int:
+        return int(self.W1.shape[0])
+
+
+def classifier(x: np.ndarray, clf: Classifier) -> float:
+    x = np.ascontiguousarray(x, dtype=np.float64)
+    C = ctypes.c_double()
+    assert clf.W1.shape[1] == x.shape[0]
+    _check(lib().oracle_classifier(_p(x, ctypes.c_double), x.shape[0], _p(clf.W1, ctypes.c_float),
+                                   _p(clf.b1, ctypes.c_float), _p(clf.w2, ctypes.c_float),
+                                   _p(clf.b2, ctypes.c_float), clf.H, ctypes.byref(C)),
+           "classifier")
+    return float(C.value)
+
+
+def accept_prefix(draft, target):
+    draft = np.ascontiguousarray(draft, dtype=np.int32)
+    target = np.ascontiguousarray(target, dtype=np.int32)
+    SL = draft.shape[0]
+    assert target.shape[0] == SL + 1
+    n = ctypes.c_int32()
+    bonus = ctypes.c_int32()
+    _check(lib().oracle_accept_prefix(_p(draft, ctypes.c_int32) if SL else None,
+                                      _p(target, ctypes.c_int32), SL, ctypes.byref(n),
+                                      ctypes.byref(bonus)), "accept_prefix")
+    return int(n.value), int(bonus.value)
+
+
+# --------------------------------------------------------------------------- whole calls
+@dataclass
+class DraftStepResult:
+    token: np.ndarray      # [B] int32
+    conf: np.ndarray       # [B] float64
+    halt: np.ndarray       # [B] uint8
+    feats: np.ndarray      # [B, k+2] float64
+    gap: np.ndarray        # [B] float64, top-2 logit gap
+    topk_ids: np.ndarray   # [B, k] int32
+    probs: np.ndarray | None  # [B, V] float64
+
+
+def draft_step(W_D, h_D, pos, n_drafted, clf: Classifier, tau: float, sl_max: int,
+               active=None, want_probs: bool = False, k: int = K_TOP,
+               nthreads: int = 1) -> DraftStepResult:
+    W_D, h_D = _u16(W_D), _u16(h_D)
+    V, d = W_D.shape
+    B = h_D.shape[0]
+    pos = np.ascontiguousarray(pos, dtype=np.int32)
+    n_drafted = np.ascontiguousarray(n_drafted, dtype=np.int32)
+    act = None if active is None else np.ascontiguousarray(active, dtype=np.uint8)
+    token = np.full(B, -1, dtype=np.int32)
+    conf = np.full(B, np.nan)
+    halt = np.full(B, 255, dtype=np.uint8)
+    feats = np.full((B, k + 2), np.nan)
+    gap = np.full(B, np.nan)
+    ids = np.full((B, k), -1, dtype=np.int32)
+    probs = np.full((B, V), np.nan) if want_probs else None
+    _check(lib().oracle_draft_step(
+        _p(W_D, ctypes.c_uint16), _p(h_D, ctypes.c_uint16), V, d, B,
+        _p(pos, ctypes.c_int32), _p(n_drafted, ctypes.c_int32), _p(act, ctypes.c_uint8),
+        _p(clf.W1, ctypes.c_float), _p(clf.b1, ctypes.c_float), _p(clf.w2, ctypes.c_float),
+        _p(clf.b2, ctypes.c_float), clf.H, k, ctypes.c_float(tau), int(sl_max),
+        _p(token, ctypes.c_int32), _p(conf, ctypes.c_double), _p(halt, ctypes.c_uint8),
+        _p(feats, ctypes.c_double), _p(probs, ctypes.c_double), _p(gap, ctypes.c_double),
+        _p(ids, ctypes.c_int32), nthreads), "draft_step")
+    return DraftStepResult(token, conf, halt, feats, gap, ids, probs)
+
+
+@dataclass
+class VerifyResult:
+    n_accept: np.ndarray    # [B] int32
+    bonus: np.ndarray       # [B] int32
+    target_ids: np.ndarray  # [R] int32
+    gap: np.ndarray         # [R] float64, top-2 logit gap per row
+
+
+def verify_ragged(W_T, H_T, draft_ids, row_off, nthreads: int = 1) -> VerifyResult:
+    W_T, H_T = _u16(W_T), _u16(H_T)
+    V, d = W_T.shape
+    row_off = np.ascontiguousarray(row_off, dtype=np.int32)
+    B = row_off.shape[0] - 1
+    R = int(row_off[-1]) if B >= 0 else 0
+    assert H_T.shape[0] == R
+    draft_ids = np.ascontiguousarray(draft_ids, dtype=np.int32)
+    assert draft_ids.shape[0] == R - B
+    n = np.full(B, -1, dtype=np.int32)
+    bonus = np.full(B, -1, dtype=np.int32)
+    tid = np.full(R, -1, dtype=np.int32)
+    gap = np.full(R, np.nan)
+    _check(lib().oracle_verify_ragged(
+        _p(W_T, ctypes.c_uint16), _p(H_T, ctypes.c_uint16), V, d,
+        _p(draft_ids, ctypes.c_int32) if draft_ids.size else None, _p(row_off, ctypes.c_int32), B,
+        _p(n, ctypes.c_int32), _p(bonus, ctypes.c_int32), _p(tid, ctypes.c_int32),
+        _p(gap, ctypes.c_double), nthreads), "verify_ragged")
+    return VerifyResult(n, bonus, tid, gap)
+
+
+def verify(W_T, H_T, draft_ids, B: int, SL: int, nthreads: int = 1) -> VerifyResult:
+    W_T, H_T = _u16(W_T), _u16(H_T)
+    V, d = W_T.shape
+    R = B * (SL + 1)
+    assert H_T.shape[0] == R
+    draft_ids = np.ascontiguousarray(draft_ids, dtype=np.int32)
+    assert draft_ids.shape[0] == B * SL
+    n = np.full(B, -1, dtype=np.int32)
+    bonus = np.full(B, -1, dtype=np.int32)
+    tid = np.full(R, -1, dtype=np.int32)
+    gap = np.full(R, np.nan)
+    _check(lib().oracle_verify(
+        _p(W_T, ctypes.c_uint16), _p(H_T, ctypes.c_uint16), V, d,
+        _p(draft_ids, ctypes.c_int32) if draft_ids.size else None, B, SL,
+        _p(n, ctypes.c_int32), _p(bonus, ctypes.c_int32), _p(tid, ctypes.c_int32),
+        _p(gap, ctypes.c_double), nthreads), "verify")
+    return VerifyResult(n, bonus, tid, gap)

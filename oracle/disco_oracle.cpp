@@ -1,0 +1,265 @@
+// CPU oracle for the DISCO per-iteration logit tails (arXiv 2405.04304).
+//
+// TEST INFRASTRUCTURE ONLY.  This file is the slow, plain definition that the
+// CUDA library is checked against.  It is compiled into liboracle.so and may be
+// loaded only by the test-suite, by the smoke check and by the benchmark's CPU
+// baseline leg.  The product library never links, loads or calls it, and the
+// two share no source.
+//
+// Every function writes out the definition it cites, one step after another,
+// in double precision, with the full probability vector materialised.  Nothing
+// is blocked, fused or reordered.  Host pointers everywhere; bf16 values arrive
+// as raw 16-bit patterns (the upper half of an IEEE binary32).
+//
+// Pins (tests that fix each function to something other than itself) are in
+// tests/test_oracle_pins.py.  Unpinned: nothing in this file.  (Behaviour of a
+// *trained* classifier, its tuned threshold and SL_max are not reproduced at
+// all: the paper prints neither weights nor values.)
+
+#include <algorithm>
+#include <cmath>
+#include <cstdint>
+#include <cstring>
+#include <limits>
+#include <thread>
+#include <vector>
+
+namespace {
+
+// bf16 -> double.  Exact: bf16 is the top 16 bits of a binary32.
+inline double bf16_value(uint16_t bits) {
+    uint32_t u = static_cast<uint32_t>(bits) << 16;
+    float f;
+    std::memcpy(&f, &u, sizeof f);
+    return static_cast<double>(f);
+}
+
+constexpr int ORACLE_OK = 0;
+constexpr int ORACLE_BAD_ARG = -1;
+
+}  // namespace
+
+extern "C" {
+
+// LM-head projection (Sec. 3: the "probability vector of the draft model" is
+// the soft-max of these logits; Sec. 2: the target scores all SL+1 positions in
+// one pass).   z[r,v] = sum_{j=0}^{d-1} W[v,j] * H[r,j],  j ascending, double.
+// W is [V,d] row-major, H is [R,d] row-major, z is [R,V] row-major.
+// nthreads > 1 splits the vocabulary rows between threads; every z[r,v] is
+// still the same single ascending sum, so the result does not depend on it.
+int oracle_project(const uint16_t* W, const uint16_t* H, int V, int d, int R,
+                   double* z, int nthreads) {
+    if (!W || !H || !z || V <= 0 || d <= 0 || R < 0) return ORACLE_BAD_ARG;
+    auto slab = [&](int v0, int v1) {
+        for (int r = 0; r < R; ++r)
+            for (int v = v0; v < v1; ++v) {
+                double acc = 0.0;
+                for (int j = 0; j < d; ++j)
+                    acc += bf16_value(W[(size_t)v * d + j]) * bf16_value(H[(size_t)r * d + j]);
+                z[(size_t)r * V + v] = acc;
+            }
+    };
+    if (nthreads <= 1) {
+        slab(0, V);
+    } else {
+        std::vector<std::thread> pool;
+        for (int t = 0; t < nthreads; ++t) {
+            int v0 = (int)((long long)V * t / nthreads);
+            int v1 = (int)((long long)V * (t + 1) / nthreads);
+            pool.emplace_back(slab, v0, v1);
+        }
+        for (auto& th : pool) th.join();
+    }
+    return ORACLE_OK;
+}
+
+// Greedy token (temperature 0, Sec. 4 "greedy decoding"): the smallest index
+// attaining the maximum.  *gap receives the distance between the largest and
+// the second largest logit (0 on an exact tie, +inf when V == 1); the tests use
+// it to find positions where fp32 and fp64 may legitimately disagree.
+int oracle_argmax(const double* z, int V, int32_t* best, double* gap) {
+    if (!z || !best || V <= 0) return ORACLE_BAD_ARG;
+    int b = 0;
+    for (int v = 1; v < V; ++v)
+        if (z[v] > z[b]) b = v;
+    double second = -std::numeric_limits<double>::infinity();
+    for (int v = 0; v < V; ++v)
+        if (v != b && z[v] > second) second = z[v];
+    *best = b;
+    if (gap) *gap = (V == 1) ? std::numeric_limits<double>::infinity() : z[b] - second;
+    return ORACLE_OK;
+}
+
+// Soft-max at temperature 1 of the raw logits (Sec. 3, y^D_i):
+// y_v = exp(z_v - m) / sum_u exp(z_u - m),  m = max_u z_u.
+int oracle_softmax(const double* z, int V, double* y) {
+    if (!z || !y || V <= 0) return ORACLE_BAD_ARG;
+    double m = z[0];
+    for (int v = 1; v < V; ++v) m = std::max(m, z[v]);
+    double denom = 0.0;
+    for (int v = 0; v < V; ++v) denom += std::exp(z[v] - m);
+    for (int v = 0; v < V; ++v) y[v] = std::exp(z[v] - m) / denom;
+    return ORACLE_OK;
+}
+
+// Top_k of Eq. 2: the k largest probabilities, descending.  Equal values keep
+// the lower index first.  If V < k the tail is padded with value 0, index -1.
+int oracle_topk(const double* y, int V, int k, double* vals, int32_t* ids) {
+    if (!y || !vals || V <= 0 || k <= 0) return ORACLE_BAD_ARG;
+    std::vector<int32_t> order(V);
+    for (int v = 0; v < V; ++v) order[v] = v;
+    std::stable_sort(order.begin(), order.end(),
+                     [&](int32_t a, int32_t b) { return y[a] > y[b]; });
+    for (int i = 0; i < k; ++i) {
+        if (i < V) {
+            vals[i] = y[order[i]];
+            if (ids) ids[i] = order[i];
+        } else {
+            vals[i] = 0.0;
+            if (ids) ids[i] = -1;
+        }
+    }
+    return ORACLE_OK;
+}
+
+// Ent of Eq. 2: Shannon entropy of the whole vector, natural logarithm;
+// a zero probability contributes nothing.
+int oracle_entropy(const double* y, int V, double* ent) {
+    if (!y || !ent || V <= 0) return ORACLE_BAD_ARG;
+    double e = 0.0;
+    for (int v = 0; v < V; ++v)
+        if (y[v] > 0.0) e -= y[v] * std::log(y[v]);
+    *ent = e;
+    return ORACLE_OK;
+}
+
+// Feature vector of Eq. 2:  x = Concat(Top_k(y), Ent(y), i)  ->  k + 2 numbers.
+int oracle_features(const double* y, int V, int k, int32_t pos, double* x) {
+    if (!x) return ORACLE_BAD_ARG;
+    int rc = oracle_topk(y, V, k, x, nullptr);
+    if (rc) return rc;
+    rc = oracle_entropy(y, V, &x[k]);
+    if (rc) return rc;
+    x[k + 1] = static_cast<double>(pos);
+    return ORACLE_OK;
+}
+
+// FFN of Eq. 2, read as the "shallow 2-layer FFN" of Sec. 4: two linear layers
+// nfeat -> H -> 1 with a ReLU between them and a logistic output, so that C is
+// a likelihood in (0,1) of the draft token being accepted (Sec. 1).
+// W1 is [H,nfeat] row-major.
+int oracle_classifier(const double* x, int nfeat, const float* W1, const float* b1,
+                      const float* w2, const float* b2, int H, double* C) {
+    if (!x || !W1 || !b1 || !w2 || !b2 || !C || H <= 0 || nfeat <= 0) return ORACLE_BAD_ARG;
+    double s = static_cast<double>(b2[0]);
+    for (int j = 0; j < H; ++j) {
+        double a = static_cast<double>(b1[j]);
+        for (int i = 0; i < nfeat; ++i) a += static_cast<double>(W1[(size_t)j * nfeat + i]) * x[i];
+        if (a < 0.0) a = 0.0;
+        s += static_cast<double>(w2[j]) * a;
+    }
+    *C = 1.0 / (1.0 + std::exp(-s));
+    return ORACLE_OK;
+}
+
+// One draft step for B independent sequences (Sec. 3): project, soft-max,
+// greedy token, features, classifier, then the stopping rule
+//     halt = (C < tau)  or  (n_drafted >= SL_max).
+// C == tau continues.  The comparison is taken on C rounded to binary32, the
+// precision in which the library holds C and tau.  Sequences with active[b]==0
+// are skipped and their outputs left untouched.
+// Outputs (any may be null except token): token[B], conf[B], halt[B],
+// feats[B,k+2], probs[B,V], gap[B] (top-2 logit gap), topk_ids[B,k].
+int oracle_draft_step(const uint16_t* W_D, const uint16_t* h_D, int V, int d, int B,
+                      const int32_t* pos, const int32_t* n_drafted, const uint8_t* active,
+                      const float* W1, const float* b1, const float* w2, const float* b2, int H,
+                      int k, float tau, int sl_max,
+                      int32_t* token, double* conf, uint8_t* halt, double* feats,
+                      double* probs, double* gap, int32_t* topk_ids, int nthreads) {
+    if (!W_D || !h_D || !pos || !n_drafted || !token || V <= 0 || d <= 0 || B < 0 || k <= 0)
+        return ORACLE_BAD_ARG;
+    std::vector<double> z(V), y(V), x(k + 2);
+    for (int b = 0; b < B; ++b) {
+        if (active && !active[b]) continue;
+        int rc = oracle_project(W_D, h_D + (size_t)b * d, V, d, 1, z.data(), nthreads);
+        if (rc) return rc;
+        rc = oracle_argmax(z.data(), V, &token[b], gap ? &gap[b] : nullptr);
+        if (rc) return rc;
+        rc = oracle_softmax(z.data(), V, y.data());
+        if (rc) return rc;
+        rc = oracle_features(y.data(), V, k, pos[b], x.data());
+        if (rc) return rc;
+        if (topk_ids) {
+            std::vector<double> tmp(k);
+            oracle_topk(y.data(), V, k, tmp.data(), topk_ids + (size_t)b * k);
+        }
+        double C = 0.0;
+        rc = oracle_classifier(x.data(), k + 2, W1, b1, w2, b2, H, &C);
+        if (rc) return rc;
+        if (conf) conf[b] = C;
+        if (halt) halt[b] = (static_cast<float>(C) < tau) || (n_drafted[b] >= sl_max) ? 1 : 0;
+        if (feats) std::copy(x.begin(), x.end(), feats + (size_t)b * (k + 2));
+        if (probs) std::copy(y.begin(), y.end(), probs + (size_t)b * V);
+    }
+    return ORACLE_OK;
+}
+
+// Acceptance at temperature 0 (Sec. 3, rejection sampling "with zero
+// temperature"; Fig. 1): draft token j+1 is accepted iff it equals the target's
+// greedy token at row j and every earlier draft token was accepted.
+//   n = |longest matching prefix|,  bonus = target token at row n.
+int oracle_accept_prefix(const int32_t* draft, const int32_t* target, int SL,
+                         int32_t* n_accept, int32_t* bonus) {
+    if (SL < 0 || !target || !n_accept || !bonus || (SL > 0 && !draft)) return ORACLE_BAD_ARG;
+    int n = 0;
+    while (n < SL && draft[n] == target[n]) ++n;
+    *n_accept = n;
+    *bonus = target[n];
+    return ORACLE_OK;
+}
+
+// Verification tail for B sequences with ragged look-ahead (Sec. 2, Sec. 3).
+// Sequence b owns rows row_off[b] .. row_off[b+1]-1 of H_T (SL_b + 1 rows) and
+// draft ids draft_ids[row_off[b]-b .. row_off[b+1]-b-2] (SL_b of them).
+// target_ids[R] and gap[R] are optional.
+int oracle_verify_ragged(const uint16_t* W_T, const uint16_t* H_T, int V, int d,
+                         const int32_t* draft_ids, const int32_t* row_off, int B,
+                         int32_t* n_accept, int32_t* bonus, int32_t* target_ids, double* gap,
+                         int nthreads) {
+    if (!W_T || !H_T || !row_off || !n_accept || !bonus || V <= 0 || d <= 0 || B < 0)
+        return ORACLE_BAD_ARG;
+    std::vector<double> z(V);
+    for (int b = 0; b < B; ++b) {
+        int r0 = row_off[b], r1 = row_off[b + 1];
+        int SL = r1 - r0 - 1;
+        if (SL < 0) return ORACLE_BAD_ARG;
+        std::vector<int32_t> a(SL + 1);
+        for (int r = r0; r < r1; ++r) {
+            int rc = oracle_project(W_T, H_T + (size_t)r * d, V, d, 1, z.data(), nthreads);
+            if (rc) return rc;
+            rc = oracle_argmax(z.data(), V, &a[r - r0], gap ? &gap[r] : nullptr);
+            if (rc) return rc;
+            if (target_ids) target_ids[r] = a[r - r0];
+        }
+        int rc = oracle_accept_prefix(draft_ids ? draft_ids + (r0 - b) : nullptr, a.data(), SL,
+                                      &n_accept[b], &bonus[b]);
+        if (rc) return rc;
+    }
+    return ORACLE_OK;
+}
+
+// Uniform look-ahead: every sequence has SL draft tokens and SL+1 rows.
+int oracle_verify(const uint16_t* W_T, const uint16_t* H_T, int V, int d,
+                  const int32_t* draft_ids, int B, int SL,
+                  int32_t* n_accept, int32_t* bonus, int32_t* target_ids, double* gap,
+                  int nthreads) {
+    if (B < 0 || SL < 0) return ORACLE_BAD_ARG;
+    std::vector<int32_t> off(B + 1);
+    for (int b = 0; b <= B; ++b) off[b] = b * (SL + 1);
+    return oracle_verify_ragged(W_T, H_T, V, d, draft_ids, off.data(), B, n_accept, bonus,
+                                target_ids, gap, nthreads);
+}
+
+int oracle_hardware_threads() { return (int)std::thread::hardware_concurrency(); }
+
+}  // extern "C"

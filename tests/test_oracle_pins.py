@@ -1,0 +1,368 @@
+"""Pins of the CPU oracle: each oracle function is fixed to something other than itself
+(closed forms, textbook special cases, brute force with independent code, values the paper prints).
+"""
+import math
+import os
+import struct
+
+import numpy as np
+import pytest
+import torch
+
+from paper_2405_04304_b200 import inputs
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def bits_of(t: torch.Tensor) -> np.ndarray:
+    return inputs.bf16_bits(t.to(torch.bfloat16))
+
+
+def py_bf16(bits: int) -> float:
+    """Decode one bf16 pattern with the struct module (independent of the oracle's decoder)."""
+    return struct.unpack("<f", struct.pack("<I", int(bits) << 16))[0]
+
+
+# ------------------------------------------------------------------ projection
+def test_project_brute_force_python_loops(oracle):
+    rng = np.random.default_rng(5)
+    V, d, R = 37, 19, 3   # all different: a transposed operand or swapped extent cannot pass
+    W = bits_of(torch.from_numpy(rng.normal(size=(V, d)).astype(np.float32)))
+    H = bits_of(torch.from_numpy(rng.normal(size=(R, d)).astype(np.float32)))
+    z = oracle.project(W, H)
+    assert z.shape == (R, V)
+    for r in range(R):
+        for v in range(V):
+            ref = math.fsum(py_bf16(W[v, j]) * py_bf16(H[r, j]) for j in range(d))
+            assert abs(z[r, v] - ref) < 1e-12
+
+
+def test_project_unit_vector_selects_column(oracle):
+    V, d = 33, 24
+    Wt = torch.randn(V, d, generator=torch.Generator().manual_seed(1)).to(torch.bfloat16)
+    for j in (0, 7, d - 1):
+        h = torch.zeros(1, d)
+        h[0, j] = 1.0
+        z = oracle.project(bits_of(Wt), bits_of(h))
+        np.testing.assert_array_equal(z[0], Wt[:, j].double().numpy())
+
+
+def test_project_one_hot_rows_copy_hidden(oracle):
+    d = 16
+    Wt = torch.eye(d)                       # V = d, row v is e_v
+    h = torch.randn(2, d, generator=torch.Generator().manual_seed(2)).to(torch.bfloat16)
+    z = oracle.project(bits_of(Wt), bits_of(h))
+    np.testing.assert_array_equal(z, h.double().numpy())
+
+
+def test_project_matches_numpy_matmul_and_threads(oracle):
+    g = torch.Generator().manual_seed(3)
+    Wt = (torch.randn(200, 72, generator=g) * 0.02).to(torch.bfloat16)
+    Ht = torch.randn(5, 72, generator=g).to(torch.bfloat16)
+    z1 = oracle.project(bits_of(Wt), bits_of(Ht), nthreads=1)
+    z4 = oracle.project(bits_of(Wt), bits_of(Ht), nthreads=4)
+    np.testing.assert_array_equal(z1, z4)          # threads split rows, never a sum
+    ref = Ht.double().numpy() @ Wt.double().numpy().T
+    np.testing.assert_allclose(z1, ref, rtol=0, atol=1e-13)
+
+
+# ------------------------------------------------------------------ argmax
+def test_argmax_lowest_index_on_ties_and_gap(oracle):
+    assert oracle.argmax(np.array([1.0, 3.0, 3.0, 2.0])) == (1, 0.0)
+    best, gap = oracle.argmax(np.array([0.5, -1.0, 4.0, 3.25]))
+    assert best == 2 and gap == 0.75
+    best, gap = oracle.argmax(np.array([7.0]))
+    assert best == 0 and math.isinf(gap)
+    assert oracle.argmax(np.zeros(9))[0] == 0
+
+
+# ------------------------------------------------------------------ soft-max
+def test_softmax_sums_to_one_and_matches_scipy(oracle):
+    from scipy.special import softmax as sp_softmax
+    rng = np.random.default_rng(0)
+    for V in (1, 2, 10, 1000):
+        z = rng.normal(scale=3.0, size=V)
+        y = oracle.softmax(z)
+        assert abs(y.sum() - 1.0) < 1e-12
+        np.testing.assert_allclose(y, sp_softmax(z), rtol=1e-12, atol=0)
+
+
+def test_softmax_shift_invariance_and_large_logits(oracle):
+    z = np.array([1000.0, 999.0, 998.0])
+    y = oracle.softmax(z)
+    e = np.exp([0.0, -1.0, -2.0])
+    np.testing.assert_allclose(y, e / e.sum(), rtol=1e-14)
+    np.testing.assert_allclose(oracle.softmax(z - 1000.0), y, rtol=1e-14)
+
+
+def test_zero_hidden_state_gives_uniform(oracle):
+    V, d = 50, 8
+    W = bits_of(torch.randn(V, d, generator=torch.Generator().manual_seed(4)))
+    z = oracle.project(W, bits_of(torch.zeros(1, d)))[0]
+    y = oracle.softmax(z)
+    np.testing.assert_allclose(y, np.full(V, 1.0 / V), rtol=1e-15)
+    assert abs(oracle.entropy(y) - math.log(V)) < 1e-12
+    assert oracle.argmax(z)[0] == 0
+
+
+# ------------------------------------------------------------------ top-k
+def test_topk_equals_full_sort(oracle):
+    rng = np.random.default_rng(1)
+    y = rng.dirichlet(np.ones(64))
+    vals, ids = oracle.topk(y, 10)
+    order = sorted(range(64), key=lambda v: (-y[v], v))[:10]
+    assert list(ids) == order
+    np.testing.assert_array_equal(vals, y[order])
+    assert all(vals[i] >= vals[i + 1] for i in range(9))
+    assert vals.sum() <= 1.0 + 1e-15
+
+
+def test_topk_ties_keep_lowest_index_and_padding(oracle):
+    y = np.array([0.1, 0.3, 0.3, 0.1, 0.2])
+    vals, ids = oracle.topk(y, 10)
+    assert list(ids[:5]) == [1, 2, 4, 0, 3]
+    assert list(ids[5:]) == [-1] * 5
+    np.testing.assert_array_equal(vals, [0.3, 0.3, 0.2, 0.1, 0.1, 0, 0, 0, 0, 0])
+
+
+def test_top0_is_one_over_Z(oracle):
+    rng = np.random.default_rng(2)
+    z = rng.normal(size=300)
+    y = oracle.softmax(z)
+    vals, ids = oracle.topk(y, 10)
+    assert ids[0] == oracle.argmax(z)[0]
+    assert abs(vals[0] - 1.0 / np.exp(z - z.max()).sum()) < 1e-15
+
+
+# ------------------------------------------------------------------ entropy
+def test_entropy_two_level_closed_form(oracle):
+    V = 1000
+    for L in (0.0, 1.0, 5.0, 12.0):
+        z = np.zeros(V)
+        z[123] = L
+        y = oracle.softmax(z)
+        p = math.exp(L) / (math.exp(L) + V - 1)
+        ref = -p * math.log(p) - (1 - p) * math.log((1 - p) / (V - 1))
+        assert abs(oracle.entropy(y) - ref) < 1e-12
+
+
+def test_entropy_bounds_zero_terms_and_scipy(oracle):
+    from scipy.stats import entropy as sp_entropy
+    assert oracle.entropy(np.array([1.0, 0.0, 0.0])) == 0.0
+    rng = np.random.default_rng(3)
+    y = rng.dirichlet(np.ones(200) * 0.3)
+    e = oracle.entropy(y)
+    assert 0.0 <= e <= math.log(200)
+    assert abs(e - sp_entropy(y)) < 1e-12          # natural logarithm
+
+
+def test_planted_peak_drives_top0_to_one(oracle):
+    V, d = 64, 32
+    g = torch.Generator().manual_seed(6)
+    Wt = (torch.randn(V, d, generator=g) * 0.1).to(torch.bfloat16)
+    h = (Wt[17].float() * 400.0).to(torch.bfloat16).view(1, d)
+    z = oracle.project(bits_of(Wt), bits_of(h))[0]
+    y = oracle.softmax(z)
+    x = oracle.features(y, pos=3)
+    assert oracle.argmax(z)[0] == 17
+    assert x[0] > 0.999 and x[10] < 0.02
+
+
+# ------------------------------------------------------------------ features
+def test_feature_layout(oracle):
+    rng = np.random.default_rng(4)
+    y = rng.dirichlet(np.ones(40))
+    x = oracle.features(y, pos=77)
+    assert x.shape == (12,)
+    np.testing.assert_array_equal(x[:10], np.sort(y)[::-1][:10])
+    assert abs(x[10] + float((y * np.log(y)).sum())) < 1e-13
+    assert x[11] == 77.0
+
+
+# ------------------------------------------------------------------ classifier
+def _clf(oracle, W1, b1, w2, b2):
+    return oracle.Classifier(np.array(W1, np.float32), np.array(b1, np.float32),
+                             np.array(w2, np.float32), np.array([b2], np.float32))
+
+
+def test_classifier_zero_head_gives_half(oracle):
+    rng = np.random.default_rng(5)
+    clf = _clf(oracle, rng.normal(size=(8, 12)), rng.normal(size=8), np.zeros(8), 0.0)
+    assert oracle.classifier(rng.normal(size=12), clf) == 0.5
+
+
+def test_classifier_hand_computed(oracle):
+    # two hidden units on three features: a = relu([x0 - x2 + 0.5, -x1 + 0.25]) ; s = 2 a0 - 3 a1 + 0.125
+    clf = _clf(oracle, [[1, 0, -1], [0, -1, 0]], [0.5, 0.25], [2, -3], 0.125)
+    x = np.array([0.75, 0.5, 0.25])              # a = [1.0, relu(-0.25) = 0]
+    assert abs(oracle.classifier(x, clf) - 1 / (1 + math.exp(-2.125))) < 1e-15
+    x = np.array([0.0, -0.75, 1.0])              # a = [relu(-0.5) = 0, 1.0] ; s = -2.875
+    assert abs(oracle.classifier(x, clf) - 1 / (1 + math.exp(2.875))) < 1e-15
+
+
+def test_classifier_relu_is_not_identity(oracle):
+    clf = _clf(oracle, [[1.0]], [0.0], [1.0], 0.0)
+    assert oracle.classifier(np.array([-5.0]), clf) == 0.5            # clipped to 0
+    assert abs(oracle.classifier(np.array([2.0]), clf) - 1 / (1 + math.exp(-2.0))) < 1e-15
+
+
+# ------------------------------------------------------------------ whole draft step
+def _small_problem(seed, V=50, d=16, B=3, H=8):
+    g = torch.Generator().manual_seed(seed)
+    W = (torch.randn(V, d, generator=g) * 0.5).to(torch.bfloat16)
+    h = torch.randn(B, d, generator=g).to(torch.bfloat16)
+    W1, b1, w2, b2 = inputs.classifier_params(H, seed + 100)
+    return W, h, (W1.numpy(), b1.numpy(), w2.numpy(), b2.numpy())
+
+
+def test_draft_step_against_independent_numpy_pipeline(oracle):
+    from scipy.special import softmax as sp_softmax
+    W, h, (W1, b1, w2, b2) = _small_problem(11)
+    clf = oracle.Classifier(W1, b1, w2, b2)
+    pos = np.array([1, 5, 9], np.int32)
+    nd = np.array([1, 2, 3], np.int32)
+    res = oracle.draft_step(bits_of(W), bits_of(h), pos, nd, clf, tau=0.5, sl_max=4, want_probs=True)
+    z = h.double().numpy() @ W.double().numpy().T
+    y = sp_softmax(z, axis=1)
+    for b in range(3):
+        assert res.token[b] == int(np.argmax(z[b]))
+        np.testing.assert_allclose(res.probs[b], y[b], rtol=1e-12)
+        x = np.concatenate([np.sort(y[b])[::-1][:10], [-(y[b] * np.log(y[b])).sum()], [float(pos[b])]])
+        np.testing.assert_allclose(res.feats[b], x, rtol=1e-12)
+        a = np.maximum(W1.astype(np.float64) @ x + b1, 0.0)
+        C = 1.0 / (1.0 + math.exp(-(float(w2.astype(np.float64) @ a) + float(b2[0]))))
+        assert abs(res.conf[b] - C) < 1e-14
+        assert res.halt[b] == int(np.float32(C) < np.float32(0.5) or nd[b] >= 4)
+
+
+def test_threshold_rule_static_sl_special_cases(oracle):
+    W, h, (W1, b1, w2, b2) = _small_problem(12)
+    clf = oracle.Classifier(W1, b1, w2, b2)
+    pos = np.arange(1, 4, dtype=np.int32)
+    # tau <= 0 never halts before the cap: static SL = SL_max (Sec. 3)
+    for nd, expect in ((1, 0), (4, 0), (5, 1), (6, 1)):
+        r = oracle.draft_step(bits_of(W), bits_of(h), pos, np.full(3, nd, np.int32), clf, 0.0, 5)
+        assert list(r.halt) == [expect] * 3
+    # tau > 1 halts after the first token
+    r = oracle.draft_step(bits_of(W), bits_of(h), pos, np.ones(3, np.int32), clf, 1.5, 5)
+    assert list(r.halt) == [1, 1, 1]
+    # C == tau continues: zero output layer gives C = 0.5 exactly
+    flat = oracle.Classifier(W1, b1, np.zeros_like(w2), np.zeros(1, np.float32))
+    r = oracle.draft_step(bits_of(W), bits_of(h), pos, np.ones(3, np.int32), flat, 0.5, 5)
+    assert list(r.conf) == [0.5] * 3 and list(r.halt) == [0, 0, 0]
+    r = oracle.draft_step(bits_of(W), bits_of(h), pos, np.ones(3, np.int32), flat, 0.5000001, 5)
+    assert list(r.halt) == [1, 1, 1]
+
+
+def test_halt_is_monotone_in_tau(oracle):
+    W, h, (W1, b1, w2, b2) = _small_problem(13, B=3)
+    clf = oracle.Classifier(W1, b1, w2, b2)
+    pos = np.array([2, 3, 4], np.int32)
+    nd = np.ones(3, np.int32)
+    halts = [oracle.draft_step(bits_of(W), bits_of(h), pos, nd, clf, tau, 9).halt for tau in (0.3, 0.5, 0.7)]
+    assert np.all(halts[0] <= halts[1]) and np.all(halts[1] <= halts[2])
+
+
+def test_inactive_sequences_untouched(oracle):
+    W, h, (W1, b1, w2, b2) = _small_problem(14)
+    clf = oracle.Classifier(W1, b1, w2, b2)
+    pos = np.ones(3, np.int32)
+    r = oracle.draft_step(bits_of(W), bits_of(h), pos, pos, clf, 0.5, 5, active=np.array([1, 0, 1], np.uint8))
+    assert r.token[1] == -1 and r.halt[1] == 255 and np.isnan(r.conf[1])
+    assert r.token[0] >= 0 and r.token[2] >= 0
+
+
+# ------------------------------------------------------------------ verification
+def _golden_pairs(name):
+    rows = []
+    with open(os.path.join(GOLDEN, name)) as f:
+        for line in f:
+            line = line.strip()
+            if line and not line.startswith("#"):
+                rows.append(line.split())
+    return rows
+
+
+def test_fig1_worked_example(oracle):
+    g = dict((k, int(v)) for k, v in _golden_pairs("fig1_iteration.txt"))
+    SL = g["SL"]
+    target = np.array([11, 12, 13, 14, 15, 16], np.int32)        # SL + 1 target tokens
+    draft = target[:SL].copy()
+    draft[g["accepted"]] = 99                                     # t4 wrong
+    draft[g["accepted"] + 1] = 98                                 # t5 wrong
+    n, bonus = oracle.accept_prefix(draft, target)
+    assert n == g["accepted"] and n + 1 == g["emitted"]
+    assert bonus == target[n]
+
+
+def test_prefix_rule_special_cases(oracle):
+    target = np.array([5, 6, 7, 8, 9, 10], np.int32)
+    assert oracle.accept_prefix(target[:5], target) == (5, 10)             # all accepted -> row SL
+    bad_first = np.array([0, 6, 7, 8, 9], np.int32)
+    assert oracle.accept_prefix(bad_first, target) == (0, 5)               # later matches do not count
+    hole = np.array([5, 6, 7, 0, 9], np.int32)
+    assert oracle.accept_prefix(hole, target) == (3, 8)
+    assert oracle.accept_prefix(np.zeros(0, np.int32), target[:1]) == (0, 5)   # SL = 0: plain target step
+
+
+def test_verify_draft_equal_to_argmax_accepts_all(oracle):
+    g = torch.Generator().manual_seed(21)
+    V, d, SL = 64, 24, 4
+    W = (torch.randn(V, d, generator=g)).to(torch.bfloat16)
+    H = torch.randn(SL + 1, d, generator=g).to(torch.bfloat16)
+    z = H.double().numpy() @ W.double().numpy().T
+    a = np.argmax(z, axis=1).astype(np.int32)
+    r = oracle.verify(bits_of(W), bits_of(H), a[:SL], B=1, SL=SL)
+    assert r.n_accept[0] == SL and r.bonus[0] == a[SL]
+    np.testing.assert_array_equal(r.target_ids, a)
+    srt = np.sort(z, axis=1)
+    np.testing.assert_allclose(r.gap, srt[:, -1] - srt[:, -2], atol=1e-12)
+    wrong = a[:SL].copy()
+    wrong[0] = (wrong[0] + 1) % V
+    r = oracle.verify(bits_of(W), bits_of(H), wrong, B=1, SL=SL)
+    assert r.n_accept[0] == 0 and r.bonus[0] == a[0]
+
+
+def test_ragged_equals_loop_of_single_calls_and_row_permutation(oracle):
+    g = torch.Generator().manual_seed(22)
+    V, d = 48, 16
+    W = torch.randn(V, d, generator=g).to(torch.bfloat16)
+    sl = torch.tensor([3, 0, 5, 1], dtype=torch.int32)
+    off = inputs.row_offsets(sl).numpy()
+    R = int(off[-1])
+    H = torch.randn(R, d, generator=g).to(torch.bfloat16)
+    a = np.argmax(H.double().numpy() @ W.double().numpy().T, axis=1).astype(np.int32)
+    draft = np.concatenate([a[off[b]:off[b + 1] - 1] for b in range(4)]).astype(np.int32)
+    draft[1] = (draft[1] + 7) % V                       # sequence 0: second token wrong
+    rag = oracle.verify_ragged(bits_of(W), bits_of(H), draft, off)
+    assert np.all(rag.n_accept >= 0) and np.all(rag.n_accept <= sl.numpy())
+    assert list(rag.n_accept) == [1, 0, 5, 1]
+    for b in range(4):
+        one = oracle.verify(bits_of(W), bits_of(H[off[b]:off[b + 1]]), draft[off[b] - b: off[b + 1] - b - 1],
+                            B=1, SL=int(sl[b]))
+        assert one.n_accept[0] == rag.n_accept[b] and one.bonus[0] == rag.bonus[b]
+    perm = torch.randperm(V, generator=g)
+    inv = torch.empty_like(perm)
+    inv[perm] = torch.arange(V)
+    ragp = oracle.verify_ragged(bits_of(W[perm]), bits_of(H), inv.numpy()[draft].astype(np.int32), off)
+    np.testing.assert_array_equal(ragp.n_accept, rag.n_accept)
+    np.testing.assert_array_equal(perm.numpy()[ragp.bonus], rag.bonus)
+    np.testing.assert_array_equal(perm.numpy()[ragp.target_ids], rag.target_ids)
+
+
+def test_eq1_numerator_golden_and_sample_mean(oracle):
+    for alpha, gamma, expected in _golden_pairs("eq1_expected_tokens.txt"):
+        alpha, gamma, expected = float(alpha), int(gamma), float(expected)
+        closed = (1 - alpha ** (gamma + 1)) / (1 - alpha)
+        assert abs(closed - expected) < 1e-5
+    # i.i.d. corruption with probability p per position: acceptance rate 1 - p (1 - 1/V)
+    V, SL, p, N = 32000, 5, 0.2, 20000
+    rng = np.random.default_rng(7)
+    target = rng.integers(0, V, size=(N, SL + 1)).astype(np.int32)
+    flat = inputs.corrupt_ids(torch.from_numpy(target[:, :SL].copy()), p, V, seed=9).numpy()
+    emitted = np.array([oracle.accept_prefix(flat[i], target[i])[0] + 1 for i in range(N)])
+    alpha = 1 - p * (1 - 1 / V)
+    mean = (1 - alpha ** (SL + 1)) / (1 - alpha)
+    sigma = emitted.std() / math.sqrt(N)
+    assert abs(emitted.mean() - mean) < 3 * sigma + 1e-9
+    assert abs(mean - 3.68928) < 1e-3              # Eq. 1 numerator at alpha = 0.8, gamma = 5
