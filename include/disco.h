@@ -1,0 +1,171 @@
+/*
+ * disco.h - C ABI of the B200 (sm_100a) logit tails of DISCO speculative decoding
+ * (Mamou et al., "Dynamic Speculation Lookahead Accelerates Speculative Decoding of
+ * Large Language Models", arXiv 2405.04304).
+ *
+ * Two operations, each one enqueue of hand-written CUDA kernels on the caller's stream:
+ *
+ *   draft step   (Sec. 3, Eq. 2)  LM-head projection of one draft hidden state per sequence,
+ *                soft-max statistics, greedy token, the features Concat(Top_k(y), Ent(y), i)
+ *                with k = 10, the 2-layer halt classifier C_i = FFN(features) and the
+ *                stopping rule  halt = (C_i < tau) or (n_drafted >= SL_max).
+ *   verification (Sec. 2, Fig. 1; Sec. 3 "rejection sampling ... with zero temperature")
+ *                LM-head projection of the SL+1 target hidden states, greedy token per
+ *                position, longest accepted draft prefix, next ("bonus") token.
+ *
+ * Conventions
+ *   - Every function returns DISCO_OK (0) or a negative DISCO_ERR_* code.  Nothing throws or
+ *     aborts.  Argument errors are detected on the host before anything is enqueued.
+ *   - Unless a parameter says "host", data pointers are DEVICE pointers owned by the caller,
+ *     16-byte aligned, and must stay valid until the stream has run the call.
+ *   - bf16 matrices are row-major with the hidden dimension contiguous; hidden widths are
+ *     multiples of 8.
+ *   - The library owns only the opaque context: scratch for cross-block reductions, a device
+ *     status word, and staging for the *_host entry points.  A context serves one stream at a
+ *     time; calls on the same context must not overlap on the GPU.
+ *   - No call synchronises the host except disco_create, disco_destroy,
+ *     disco_last_device_status and the *_host entry points.
+ *   - Kernels never trap or spin without bound: a condition they detect (inconsistent
+ *     row offsets, a wait that ran out) is recorded in the device status word.
+ */
+#ifndef DISCO_H_
+#define DISCO_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define DISCO_TOPK 10                 /* k of Top_k in Eq. 2 (footnote: k = 10 in all experiments) */
+#define DISCO_NFEAT (DISCO_TOPK + 2)  /* top-k probabilities, entropy, position */
+#define DISCO_MAX_CLF_HIDDEN 256
+
+enum {
+    DISCO_OK = 0,
+    DISCO_ERR_INVALID_ARG = -1,       /* null / misaligned pointer, size out of range */
+    DISCO_ERR_UNSUPPORTED_SHAPE = -2, /* shape outside what the kernels handle */
+    DISCO_ERR_WORKSPACE = -3,         /* batch or row count beyond what the context was created for */
+    DISCO_ERR_CUDA = -4,              /* a CUDA runtime call failed */
+    DISCO_ERR_TIMEOUT = -5            /* a bounded device-side wait ran out (device status word only) */
+};
+
+typedef struct disco_ctx disco_ctx;
+
+/* Halt classifier of Eq. 2, read as the "shallow 2-layer FFN" of Sec. 4:
+ *   C = sigmoid(w2 . relu(W1 x + b1) + b2),  x = the DISCO_NFEAT features.
+ * The struct itself lives on the host; the four pointers are device fp32 arrays
+ * (4-byte alignment is enough).  1 <= H <= DISCO_MAX_CLF_HIDDEN. */
+typedef struct {
+    const float* W1; /* [H, DISCO_NFEAT] row-major */
+    const float* b1; /* [H] */
+    const float* w2; /* [H] */
+    const float* b2; /* [1] */
+    int H;
+} disco_clf;
+
+/* Create a context on the current CUDA device for LM heads of V rows, draft hidden width
+ * d_draft and target hidden width d_target, at most max_batch sequences per draft step and
+ * at most max_rows (sum over sequences of SL+1) rows per verification.  k must be DISCO_TOPK;
+ * clf_hidden is the largest classifier width that will be used.  Allocates device scratch
+ * (host-synchronising).  *out is set only on success. */
+int disco_create(disco_ctx** out, int V, int d_draft, int d_target, int max_batch, int max_rows,
+                 int k, int clf_hidden);
+
+/* Free everything the context owns.  The caller must have synchronised the stream(s) it used. */
+int disco_destroy(disco_ctx* ctx);
+
+/* Static, human-readable text for a return code. */
+const char* disco_strerror(int code);
+
+/* Host-synchronising: copy the device status word (DISCO_OK or the first DISCO_ERR_* a kernel
+ * recorded since the last query) to *out and clear it.  Meant for tests and debugging. */
+int disco_last_device_status(disco_ctx* ctx, int* out);
+
+/* Number of kernels the library has launched through this context since creation. */
+int disco_launch_count(disco_ctx* ctx, long long* out);
+
+/* Kernel selection (tuning and tests): which = 0 automatic (default), 1 force the CUDA-core
+ * streaming kernels, 2 force the tcgen05 kernels where the shape allows them. */
+int disco_set_kernel_path(disco_ctx* ctx, int which);
+
+/*
+ * One draft step for B sequences (Sec. 3, Eq. 2).  B = 1 is the single-sequence call.
+ *   W_D        bf16 [V, d_draft]   draft LM head
+ *   h_D        bf16 [B, d_draft]   last draft hidden state of each sequence
+ *   pos        int32 [B]           feature i: position of the token being drafted, counted from
+ *                                  the start of generation (App. D); used as (float) pos
+ *   n_drafted  int32 [B]           draft tokens of this iteration including this one (>= 1)
+ *   active     uint8 [B] or NULL   0 = skip the sequence: none of its outputs is written
+ *   clf        host struct         classifier parameters (device arrays)
+ *   tau        threshold; halt iff C < tau (C == tau continues) or n_drafted >= sl_max
+ * Outputs
+ *   token      int32 [B]           greedy draft token: lowest index attaining the largest logit
+ *   conf       float [B]           C
+ *   halt       uint8 [B]           1 = stop drafting and hand over to the target
+ *   feats      float [B, DISCO_NFEAT] or NULL   the feature vector (top-10 probabilities
+ *                                  descending, entropy in nats, (float) pos)
+ *   probs      float [B, V] or NULL   the full soft-max vector; test/debug only (costs a second
+ *                                  pass over [B, V] floats)
+ * Logits are accumulated in fp32 from bf16 inputs and never written to memory (unless probs).
+ */
+int disco_draft_step(disco_ctx* ctx, const void* W_D, const void* h_D, int B,
+                     const int32_t* pos, const int32_t* n_drafted, const uint8_t* active,
+                     const disco_clf* clf, float tau, int sl_max,
+                     int32_t* token, float* conf, uint8_t* halt, float* feats, float* probs,
+                     void* stream);
+
+/*
+ * Verification with the same look-ahead SL for all B sequences (Sec. 2; Fig. 1).
+ *   W_T        bf16 [V, d_target]          target LM head
+ *   H_T        bf16 [B*(SL+1), d_target]   row b*(SL+1)+j is the target hidden state whose
+ *                                          next-token prediction is compared with draft token
+ *                                          j+1 of sequence b; row SL predicts the token after
+ *                                          the last draft token
+ *   draft_ids  int32 [B*SL]                (may be NULL when SL == 0)
+ * Outputs
+ *   n_accept   int32 [B]    length of the longest prefix with draft_ids[b,j] == target token j
+ *   bonus      int32 [B]    target token at row n_accept (always emitted after the prefix)
+ *   target_ids int32 [B*(SL+1)] or NULL   greedy target token of every row
+ * SL = 0 is a plain target step: n_accept = 0, bonus = the target token.
+ */
+int disco_verify(disco_ctx* ctx, const void* W_T, const void* H_T, const int32_t* draft_ids,
+                 int B, int SL, int32_t* n_accept, int32_t* bonus, int32_t* target_ids,
+                 void* stream);
+
+/*
+ * Verification with a per-sequence look-ahead (the SL chosen by the halt classifier differs
+ * between sequences).  Sequence b owns rows row_off[b] .. row_off[b+1]-1 of H_T (SL_b + 1 rows)
+ * and the SL_b draft ids starting at draft_ids[row_off[b] - b].
+ *   H_T        bf16 [R, d_target],  R = row_off[B] (passed by value; the host does not read row_off)
+ *   draft_ids  int32 [R - B]
+ *   row_off    int32 [B + 1], device, increasing by at least 1, row_off[0] = 0
+ * If the kernel finds row_off inconsistent with R it records DISCO_ERR_INVALID_ARG in the
+ * device status word and writes -1 to n_accept and bonus of the offending sequences.
+ */
+int disco_verify_ragged(disco_ctx* ctx, const void* W_T, const void* H_T, const int32_t* draft_ids,
+                        const int32_t* row_off, int B, int R,
+                        int32_t* n_accept, int32_t* bonus, int32_t* target_ids, void* stream);
+
+/*
+ * The same two operations for a caller whose per-step data lives in HOST memory (pinned memory
+ * makes the copies asynchronous).  The LM heads and classifier parameters stay on the device;
+ * the hidden states, integer inputs and every output are host pointers.  Each call copies its
+ * inputs to staging owned by the context, runs the kernels, copies the results back and
+ * synchronises the stream before returning.  feats / target_ids may be NULL.
+ */
+int disco_draft_step_host(disco_ctx* ctx, const void* W_D /*device*/, const void* h_D_host, int B,
+                          const int32_t* pos_host, const int32_t* n_drafted_host,
+                          const uint8_t* active_host /*or NULL*/, const disco_clf* clf /*device arrays*/,
+                          float tau, int sl_max, int32_t* token_host, float* conf_host,
+                          uint8_t* halt_host, float* feats_host, void* stream);
+
+int disco_verify_ragged_host(disco_ctx* ctx, const void* W_T /*device*/, const void* H_T_host,
+                             const int32_t* draft_ids_host, const int32_t* row_off_host, int B, int R,
+                             int32_t* n_accept_host, int32_t* bonus_host, int32_t* target_ids_host,
+                             void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* DISCO_H_ */

@@ -1,0 +1,262 @@
+// Shared device helpers of the DISCO logit-tail kernels: PTX wrappers (mbarrier, bulk copy),
+// ordered keys for deterministic arg-max, online soft-max state, warp-resident top-10 lists.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "disco.h"
+
+namespace disco {
+
+constexpr int kTopK = DISCO_TOPK;
+constexpr int kNFeat = DISCO_NFEAT;
+constexpr unsigned kFullMask = 0xffffffffu;
+constexpr int kNoIndex = 0x7fffffff;
+
+// Bounded-wait budget: a barrier wait gives up after this many clock ticks (about 0.2 s).
+constexpr long long kWaitBudgetClocks = 400000000ll;
+
+// ------------------------------------------------------------------------------------------
+// status word
+// ------------------------------------------------------------------------------------------
+__device__ __forceinline__ void record_status(int* status, int code) {
+    if (status) atomicCAS(status, 0, code);
+}
+
+// ------------------------------------------------------------------------------------------
+// shared-memory barriers and bulk (TMA-unit) copies
+// ------------------------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_addr(const void* p) {
+    return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
+
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_addr(bar)), "r"(count));
+}
+
+__device__ __forceinline__ void fence_mbar_init() {
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+}
+
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_addr(bar)) : "memory");
+}
+
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint64_t* bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_addr(bar)),
+                 "r"(bytes)
+                 : "memory");
+}
+
+__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(smem_addr(bar)), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+
+// Wait for the phase with the given parity to complete.  Never spins without bound: after
+// kWaitBudgetClocks it records DISCO_ERR_TIMEOUT and returns false; the caller carries on
+// (its results are then meaningless, but every later wait is bounded in the same way).
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, int* status) {
+    if (mbar_try_wait(bar, parity)) return true;
+    const long long t0 = clock64();
+    for (;;) {
+#pragma unroll 1
+        for (int i = 0; i < 256; ++i)
+            if (mbar_try_wait(bar, parity)) return true;
+        if (clock64() - t0 > kWaitBudgetClocks) {
+            record_status(status, DISCO_ERR_TIMEOUT);
+            return false;
+        }
+    }
+}
+
+// Contiguous global -> shared copy by the TMA unit; completion is counted in bytes on `bar`.
+// Both addresses 16-byte aligned, bytes a multiple of 16.
+__device__ __forceinline__ void bulk_g2s(void* dst_smem, const void* src_gmem, uint32_t bytes,
+                                         uint64_t* bar) {
+    asm volatile(
+        "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+            smem_addr(dst_smem)),
+        "l"(src_gmem), "r"(bytes), "r"(smem_addr(bar))
+        : "memory");
+}
+
+__device__ __forceinline__ void named_barrier_sync(int id, int nthreads) {
+    asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(nthreads) : "memory");
+}
+
+// 4-byte asynchronous copy global -> shared (classifier parameters)
+__device__ __forceinline__ void cp_async4(void* dst_smem, const void* src) {
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(smem_addr(dst_smem)), "l"(src)
+                 : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_all;" ::: "memory"); }
+
+// ------------------------------------------------------------------------------------------
+// numerics
+// ------------------------------------------------------------------------------------------
+#define DISCO_NEG_INF (-__int_as_float(0x7f800000))
+
+// Monotone map float -> uint32 (larger float, larger key); -0 must have been folded into +0.
+__device__ __forceinline__ uint32_t ordered_bits(float x) {
+    uint32_t u = __float_as_uint(x);
+    return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+__device__ __forceinline__ float from_ordered_bits(uint32_t k) {
+    uint32_t u = (k & 0x80000000u) ? (k & 0x7fffffffu) : ~k;
+    return __uint_as_float(u);
+}
+// 64-bit key whose maximum is "largest value, then lowest index".  Key 0 means "nothing yet".
+__device__ __forceinline__ unsigned long long argmax_key(float x, int idx) {
+    return (static_cast<unsigned long long>(ordered_bits(x)) << 32) |
+           static_cast<unsigned long long>(0xffffffffu - static_cast<uint32_t>(idx));
+}
+__device__ __forceinline__ int key_index(unsigned long long key) {
+    return static_cast<int>(0xffffffffu - static_cast<uint32_t>(key & 0xffffffffull));
+}
+
+__device__ __forceinline__ void unpack_bf16x8(const uint4& q, float (&f)[8]) {
+    f[0] = __uint_as_float(q.x << 16);
+    f[1] = __uint_as_float(q.x & 0xffff0000u);
+    f[2] = __uint_as_float(q.y << 16);
+    f[3] = __uint_as_float(q.y & 0xffff0000u);
+    f[4] = __uint_as_float(q.z << 16);
+    f[5] = __uint_as_float(q.z & 0xffff0000u);
+    f[6] = __uint_as_float(q.w << 16);
+    f[7] = __uint_as_float(q.w & 0xffff0000u);
+}
+
+// Soft-max statistics of a set of logits z_i:  m = max, Z = sum e^{z_i-m}, S = sum e^{z_i-m}(z_i-m).
+// Entropy = ln Z - S/Z;  probability of logit z = e^{z-m}/Z.
+struct SoftmaxState {
+    float m, Z, S;
+    __device__ __forceinline__ void init() {
+        m = DISCO_NEG_INF;
+        Z = 0.f;
+        S = 0.f;
+    }
+    __device__ __forceinline__ void push(float z) {
+        if (z > m) {
+            if (Z > 0.f) {
+                const float dm = m - z;
+                const float e = __expf(dm);
+                S = e * (S + dm * Z);
+                Z = Z * e + 1.f;
+            } else {
+                Z = 1.f;
+                S = 0.f;
+            }
+            m = z;
+        } else {
+            const float t = z - m;
+            const float e = __expf(t);
+            Z += e;
+            S = fmaf(e, t, S);
+        }
+    }
+    __device__ __forceinline__ void merge(float m2, float Z2, float S2) {
+        if (!(Z2 > 0.f)) return;
+        if (!(Z > 0.f)) {
+            m = m2;
+            Z = Z2;
+            S = S2;
+            return;
+        }
+        const float M = fmaxf(m, m2);
+        const float d1 = m - M, d2 = m2 - M;
+        const float e1 = __expf(d1), e2 = __expf(d2);
+        S = e1 * (S + d1 * Z) + e2 * (S2 + d2 * Z2);
+        Z = Z * e1 + Z2 * e2;
+        m = M;
+    }
+};
+
+// Butterfly merge of one SoftmaxState per lane; every lane ends with the merged state.
+__device__ __forceinline__ void warp_merge_softmax(SoftmaxState& st) {
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) {
+        const float m2 = __shfl_xor_sync(kFullMask, st.m, off);
+        const float Z2 = __shfl_xor_sync(kFullMask, st.Z, off);
+        const float S2 = __shfl_xor_sync(kFullMask, st.S, off);
+        st.merge(m2, Z2, S2);
+    }
+}
+
+// A descending top-10 list kept by one warp: lane l < 10 holds entry l.  Values offered must be
+// warp-uniform.  An offered value equal to a stored one goes behind it, so offering candidates in
+// ascending index order keeps "lowest index first" among equals.
+struct WarpTop10 {
+    float v;
+    int i;
+    float floor_v;  // warp-uniform copy of entry 9's value
+    __device__ __forceinline__ void init() {
+        v = DISCO_NEG_INF;
+        i = kNoIndex;
+        floor_v = DISCO_NEG_INF;
+    }
+    __device__ __forceinline__ void insert(float z, int idx, int lane) {
+        const unsigned ahead = __ballot_sync(kFullMask, lane < kTopK && v >= z);
+        const int p = __popc(ahead);
+        const float up_v = __shfl_up_sync(kFullMask, v, 1);
+        const int up_i = __shfl_up_sync(kFullMask, i, 1);
+        if (lane > p) {
+            v = up_v;
+            i = up_i;
+        } else if (lane == p) {
+            v = z;
+            i = idx;
+        }
+        floor_v = __shfl_sync(kFullMask, v, kTopK - 1);
+    }
+    __device__ __forceinline__ void offer(float z, int idx, int lane) {
+        if (z > floor_v) insert(z, idx, lane);
+    }
+};
+
+// Select the 10 best of the 32*E candidates a warp holds in registers (E slots per lane), ordered
+// by (value descending, index ascending).  Empty slots are (-inf, kNoIndex).  The slots are
+// consumed.  Result: lane r < 10 returns entry r, other lanes (-inf, kNoIndex).
+template <int E>
+__device__ __forceinline__ void warp_select_top10(float (&v)[E], int (&id)[E], int lane, float& out_v,
+                                                  int& out_i) {
+    out_v = DISCO_NEG_INF;
+    out_i = kNoIndex;
+#pragma unroll 1
+    for (int r = 0; r < kTopK; ++r) {
+        float bv = v[0];
+        int bi = id[0];
+#pragma unroll
+        for (int e = 1; e < E; ++e) {
+            const bool better = (v[e] > bv) || (v[e] == bv && id[e] < bi);
+            bv = better ? v[e] : bv;
+            bi = better ? id[e] : bi;
+        }
+        const uint32_t mine = ordered_bits(bv);
+        const uint32_t best = __reduce_max_sync(kFullMask, mine);
+        const int cand_i = (mine == best) ? bi : kNoIndex;
+        const int win_i = __reduce_min_sync(kFullMask, cand_i);
+        if (lane == r) {
+            out_v = from_ordered_bits(best);
+            out_i = win_i;
+        }
+        if (cand_i == win_i && win_i != kNoIndex) {  // this lane owns the winner: retire it
+#pragma unroll
+            for (int e = 0; e < E; ++e)
+                if (id[e] == win_i) {
+                    v[e] = DISCO_NEG_INF;
+                    id[e] = kNoIndex;
+                }
+        }
+    }
+}
+
+}  // namespace disco
