@@ -1,0 +1,206 @@
+"""Thin ctypes binding of libdisco.so (include/disco.h).  Argument marshalling only.
+
+Every step of the path runs inside the CUDA library.  There is no fallback: if the library has
+not been built, loading raises.  Tensors are torch CUDA tensors (torch is used for device memory
+and streams only); the ``*_host`` calls take CPU tensors (pinned for asynchronous copies).
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libdisco.so")
+
+TOPK = 10
+NFEAT = 12
+
+OK = 0
+ERR_INVALID_ARG = -1
+ERR_UNSUPPORTED_SHAPE = -2
+ERR_WORKSPACE = -3
+ERR_CUDA = -4
+ERR_TIMEOUT = -5
+
+EXPORTS = [
+    "disco_create", "disco_destroy", "disco_strerror", "disco_last_device_status", "disco_launch_count",
+    "disco_set_kernel_path", "disco_draft_step", "disco_verify", "disco_verify_ragged",
+    "disco_draft_step_host", "disco_verify_ragged_host",
+]
+
+
+class DiscoError(RuntimeError):
+    def __init__(self, code: int, what: str):
+        self.code = code
+        super().__init__(f"{what}: {strerror(code)} (code {code})")
+
+
+class _Clf(ctypes.Structure):
+    _fields_ = [("W1", ctypes.c_void_p), ("b1", ctypes.c_void_p), ("w2", ctypes.c_void_p),
+                ("b2", ctypes.c_void_p), ("H", ctypes.c_int)]
+
+
+_lib = None
+
+
+def load() -> ctypes.CDLL:
+    """Load libdisco.so; raises if it is missing (build it with paper_2405_04304_b200/build.py)."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise RuntimeError(f"{LIB_PATH} is missing: the CUDA library has not been built "
+                           "(python paper_2405_04304_b200/build.py); there is no fallback path")
+    lib = ctypes.CDLL(LIB_PATH)
+    vp, ci, cf = ctypes.c_void_p, ctypes.c_int, ctypes.c_float
+    lib.disco_create.argtypes = [ctypes.POINTER(vp), ci, ci, ci, ci, ci, ci, ci]
+    lib.disco_destroy.argtypes = [vp]
+    lib.disco_strerror.argtypes = [ci]
+    lib.disco_strerror.restype = ctypes.c_char_p
+    lib.disco_last_device_status.argtypes = [vp, ctypes.POINTER(ci)]
+    lib.disco_launch_count.argtypes = [vp, ctypes.POINTER(ctypes.c_longlong)]
+    lib.disco_set_kernel_path.argtypes = [vp, ci]
+    lib.disco_draft_step.argtypes = [vp, vp, vp, ci, vp, vp, vp, ctypes.POINTER(_Clf), cf, ci,
+                                     vp, vp, vp, vp, vp, vp]
+    lib.disco_verify.argtypes = [vp, vp, vp, vp, ci, ci, vp, vp, vp, vp]
+    lib.disco_verify_ragged.argtypes = [vp, vp, vp, vp, vp, ci, ci, vp, vp, vp, vp]
+    lib.disco_draft_step_host.argtypes = [vp, vp, vp, ci, vp, vp, vp, ctypes.POINTER(_Clf), cf, ci,
+                                          vp, vp, vp, vp, vp]
+    lib.disco_verify_ragged_host.argtypes = [vp, vp, vp, vp, vp, ci, ci, vp, vp, vp, vp]
+    _lib = lib
+    return lib
+
+
+def strerror(code: int) -> str:
+    return load().disco_strerror(int(code)).decode()
+
+
+def _ptr(t, dtype=None, cuda=True):
+    if t is None:
+        return None
+    if dtype is not None and t.dtype != dtype:
+        raise TypeError(f"expected {dtype}, got {t.dtype}")
+    if t.is_cuda != cuda:
+        raise ValueError("tensor is on the wrong device kind for this call")
+    if not t.is_contiguous():
+        raise ValueError("tensor must be contiguous")
+    return ctypes.c_void_p(t.data_ptr())
+
+
+def _stream(stream) -> ctypes.c_void_p:
+    s = stream if stream is not None else torch.cuda.current_stream()
+    return ctypes.c_void_p(s.cuda_stream)
+
+
+class Classifier:
+    """Device-resident parameters of the halt classifier (fp32)."""
+
+    def __init__(self, W1: torch.Tensor, b1: torch.Tensor, w2: torch.Tensor, b2: torch.Tensor):
+        for t in (W1, b1, w2, b2):
+            if not t.is_cuda or t.dtype != torch.float32:
+                raise TypeError("classifier parameters must be fp32 CUDA tensors")
+        self.W1, self.b1, self.w2, self.b2 = (t.contiguous() for t in (W1, b1, w2, b2))
+        self.H = int(W1.shape[0])
+        if tuple(W1.shape) != (self.H, NFEAT) or b1.numel() != self.H or w2.numel() != self.H or b2.numel() != 1:
+            raise ValueError("classifier shapes must be [H,12], [H], [H], [1]")
+        self._c = _Clf(self.W1.data_ptr(), self.b1.data_ptr(), self.w2.data_ptr(), self.b2.data_ptr(), self.H)
+
+
+class Context:
+    """disco_ctx: scratch for one (V, d_draft, d_target) configuration on the current device."""
+
+    def __init__(self, V: int, d_draft: int, d_target: int, max_batch: int = 1, max_rows: int = 32,
+                 clf_hidden: int = 64):
+        self._lib = load()
+        self._h = ctypes.c_void_p()
+        rc = self._lib.disco_create(ctypes.byref(self._h), V, d_draft, d_target, max_batch, max_rows, TOPK,
+                                    clf_hidden)
+        if rc != OK:
+            self._h = ctypes.c_void_p()
+            raise DiscoError(rc, "disco_create")
+        self.V, self.d_draft, self.d_target = V, d_draft, d_target
+        self.max_batch, self.max_rows = max_batch, max_rows
+
+    def close(self):
+        if getattr(self, "_h", None) and self._h.value:
+            self._lib.disco_destroy(self._h)
+            self._h = ctypes.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    # ---------------------------------------------------------------- bookkeeping
+    def device_status(self) -> int:
+        out = ctypes.c_int()
+        rc = self._lib.disco_last_device_status(self._h, ctypes.byref(out))
+        if rc != OK:
+            raise DiscoError(rc, "disco_last_device_status")
+        return int(out.value)
+
+    def launch_count(self) -> int:
+        out = ctypes.c_longlong()
+        self._lib.disco_launch_count(self._h, ctypes.byref(out))
+        return int(out.value)
+
+    def set_kernel_path(self, which: int) -> None:
+        rc = self._lib.disco_set_kernel_path(self._h, int(which))
+        if rc != OK:
+            raise DiscoError(rc, "disco_set_kernel_path")
+
+    # ---------------------------------------------------------------- device-resident calls
+    def draft_step(self, W_D, h_D, pos, n_drafted, clf: Classifier, tau: float, sl_max: int,
+                   token, conf, halt, active=None, feats=None, probs=None, stream=None) -> None:
+        B = int(h_D.shape[0])
+        rc = self._lib.disco_draft_step(
+            self._h, _ptr(W_D, torch.bfloat16), _ptr(h_D, torch.bfloat16), B, _ptr(pos, torch.int32),
+            _ptr(n_drafted, torch.int32), _ptr(active, torch.uint8), ctypes.byref(clf._c), float(tau),
+            int(sl_max), _ptr(token, torch.int32), _ptr(conf, torch.float32), _ptr(halt, torch.uint8),
+            _ptr(feats, torch.float32), _ptr(probs, torch.float32), _stream(stream))
+        if rc != OK:
+            raise DiscoError(rc, "disco_draft_step")
+
+    def verify(self, W_T, H_T, draft_ids, B: int, SL: int, n_accept, bonus, target_ids=None,
+               stream=None) -> None:
+        rc = self._lib.disco_verify(
+            self._h, _ptr(W_T, torch.bfloat16), _ptr(H_T, torch.bfloat16), _ptr(draft_ids, torch.int32),
+            int(B), int(SL), _ptr(n_accept, torch.int32), _ptr(bonus, torch.int32),
+            _ptr(target_ids, torch.int32), _stream(stream))
+        if rc != OK:
+            raise DiscoError(rc, "disco_verify")
+
+    def verify_ragged(self, W_T, H_T, draft_ids, row_off, B: int, R: int, n_accept, bonus,
+                      target_ids=None, stream=None) -> None:
+        rc = self._lib.disco_verify_ragged(
+            self._h, _ptr(W_T, torch.bfloat16), _ptr(H_T, torch.bfloat16), _ptr(draft_ids, torch.int32),
+            _ptr(row_off, torch.int32), int(B), int(R), _ptr(n_accept, torch.int32),
+            _ptr(bonus, torch.int32), _ptr(target_ids, torch.int32), _stream(stream))
+        if rc != OK:
+            raise DiscoError(rc, "disco_verify_ragged")
+
+    # ---------------------------------------------------------------- host-buffer calls
+    def draft_step_host(self, W_D, h_D, pos, n_drafted, clf: Classifier, tau: float, sl_max: int,
+                        token, conf, halt, active=None, feats=None, stream=None) -> None:
+        B = int(h_D.shape[0])
+        rc = self._lib.disco_draft_step_host(
+            self._h, _ptr(W_D, torch.bfloat16), _ptr(h_D, torch.bfloat16, cuda=False), B,
+            _ptr(pos, torch.int32, cuda=False), _ptr(n_drafted, torch.int32, cuda=False),
+            _ptr(active, torch.uint8, cuda=False), ctypes.byref(clf._c), float(tau), int(sl_max),
+            _ptr(token, torch.int32, cuda=False), _ptr(conf, torch.float32, cuda=False),
+            _ptr(halt, torch.uint8, cuda=False), _ptr(feats, torch.float32, cuda=False), _stream(stream))
+        if rc != OK:
+            raise DiscoError(rc, "disco_draft_step_host")
+
+    def verify_ragged_host(self, W_T, H_T, draft_ids, row_off, B: int, R: int, n_accept, bonus,
+                           target_ids=None, stream=None) -> None:
+        rc = self._lib.disco_verify_ragged_host(
+            self._h, _ptr(W_T, torch.bfloat16), _ptr(H_T, torch.bfloat16, cuda=False),
+            _ptr(draft_ids, torch.int32, cuda=False), _ptr(row_off, torch.int32, cuda=False), int(B),
+            int(R), _ptr(n_accept, torch.int32, cuda=False), _ptr(bonus, torch.int32, cuda=False),
+            _ptr(target_ids, torch.int32, cuda=False), _stream(stream))
+        if rc != OK:
+            raise DiscoError(rc, "disco_verify_ragged_host")

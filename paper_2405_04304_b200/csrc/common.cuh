@@ -71,6 +71,8 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, int* s
 #pragma unroll 1
         for (int i = 0; i < 256; ++i)
             if (mbar_try_wait(bar, parity)) return true;
+        // once any wait in the grid has run out, the others give up at once
+        if (status && *reinterpret_cast<volatile int*>(status) == DISCO_ERR_TIMEOUT) return false;
         if (clock64() - t0 > kWaitBudgetClocks) {
             record_status(status, DISCO_ERR_TIMEOUT);
             return false;

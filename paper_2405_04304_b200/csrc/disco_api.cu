@@ -1,0 +1,407 @@
+// Host side of the C ABI declared in include/disco.h: context, argument checks, kernel selection
+// and launches.  No PyTorch types; plain pointers and sizes only.
+#include <cuda_runtime.h>
+
+#include <algorithm>
+#include <cstdio>
+#include <cstring>
+#include <new>
+
+#include "disco.h"
+#include "stream_tail.cuh"
+
+using namespace disco;
+
+namespace {
+
+constexpr int kStreamWarps = 16;     // consumer warps of the streaming kernel
+constexpr int kMaxHidden = 16384;    // widest hidden dimension the kernels accept
+constexpr int kSlotTargetBytes = 12288;
+
+struct StreamPlan {
+    int rows_per_cta, grid, rps, stages;
+    uint32_t slot_bytes;
+    size_t smem;
+    bool ok;
+};
+
+}  // namespace
+
+struct disco_ctx {
+    int device;
+    int V, d_draft, d_target, max_batch, max_rows, clf_hidden;
+    int sm_count;
+    size_t smem_optin;
+    int path;
+    long long launches;
+    // scratch for cross-block reductions
+    int part_rows;  // rows the partial buffers can hold
+    int max_grid;
+    float* part_stats;
+    float* part_topv;
+    int* part_topi;
+    unsigned long long* keys;
+    unsigned int* ticket;
+    int* status;
+    float* final_stats;
+    // device staging for the *_host entry points
+    void* stage_hidden;
+    int32_t* stage_int;   // pos | n_drafted | draft_ids | row_off | token | n_accept | bonus | target_ids
+    float* stage_float;   // conf | feats
+    uint8_t* stage_byte;  // active | halt
+};
+
+namespace {
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+StreamPlan plan_stream(const disco_ctx* c, int V, int d, int RT, int clf_H) {
+    StreamPlan pl{};
+    const uint32_t row_bytes = (uint32_t)d * 2u;
+    int rpc = (V + c->sm_count - 1) / c->sm_count;
+    rpc = std::max(1, std::min(rpc, 2048));
+    pl.rows_per_cta = rpc;
+    pl.grid = (V + rpc - 1) / rpc;
+    int rps = std::max(1, kSlotTargetBytes / (int)row_bytes);
+    rps = std::min(rps, rpc);
+    pl.rps = rps;
+    pl.slot_bytes = (uint32_t)rps * row_bytes;
+    const size_t fixed = stream_tail_smem_bytes(RT, kStreamWarps, d, 0, 0, clf_H);
+    const size_t budget = c->smem_optin > 2048 ? c->smem_optin - 2048 : 0;
+    if (budget <= fixed) return pl;
+    long long stages = (long long)((budget - fixed) / (pl.slot_bytes + 16));
+    const int need = (rpc + rps - 1) / rps;  // slots that one pass over the slab takes
+    stages = std::min<long long>(stages, std::max(2, std::min(need, 24)));
+    if (stages < 2) return pl;
+    pl.stages = (int)stages;
+    pl.smem = stream_tail_smem_bytes(RT, kStreamWarps, d, pl.stages, pl.slot_bytes, clf_H);
+    pl.ok = true;
+    return pl;
+}
+
+template <int RT, bool DRAFT>
+int launch_stream(disco_ctx* c, TailParams& p, const StreamPlan& pl, cudaStream_t st) {
+    auto kern = stream_tail_kernel<RT, DRAFT, kStreamWarps>;
+    static int configured_dev = -1;
+    static size_t configured_smem = 0;
+    if (configured_dev != c->device || configured_smem < pl.smem) {
+        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)c->smem_optin) !=
+            cudaSuccess)
+            return DISCO_ERR_CUDA;
+        configured_dev = c->device;
+        configured_smem = c->smem_optin;
+    }
+    kern<<<pl.grid, (kStreamWarps + 1) * 32, pl.smem, st>>>(p);
+    c->launches += 1;
+    return cudaGetLastError() == cudaSuccess ? DISCO_OK : DISCO_ERR_CUDA;
+}
+
+template <bool DRAFT>
+int run_stream(disco_ctx* c, TailParams& p, int clf_H, cudaStream_t st) {
+    const int RT = p.R == 1 ? 1 : (p.R == 2 ? 2 : 4);
+    const StreamPlan pl = plan_stream(c, p.V, p.d, RT, clf_H);
+    if (!pl.ok) return DISCO_ERR_UNSUPPORTED_SHAPE;
+    if (DRAFT && (pl.grid > c->max_grid || p.R > c->part_rows)) return DISCO_ERR_WORKSPACE;
+    p.rows_per_cta = pl.rows_per_cta;
+    p.rps = pl.rps;
+    p.stages = pl.stages;
+    p.slot_bytes = pl.slot_bytes;
+    switch (RT) {
+        case 1: return launch_stream<1, DRAFT>(c, p, pl, st);
+        case 2: return launch_stream<2, DRAFT>(c, p, pl, st);
+        default: return launch_stream<4, DRAFT>(c, p, pl, st);
+    }
+}
+
+void fill_scratch(const disco_ctx* c, TailParams& p) {
+    p.part_stats = c->part_stats;
+    p.part_topv = c->part_topv;
+    p.part_topi = c->part_topi;
+    p.keys = c->keys;
+    p.ticket = c->ticket;
+    p.status = c->status;
+    p.final_stats = c->final_stats;
+}
+
+int check_clf(const disco_ctx* c, const disco_clf* clf) {
+    if (!clf || !clf->W1 || !clf->b1 || !clf->w2 || !clf->b2) return DISCO_ERR_INVALID_ARG;
+    if (clf->H < 1 || clf->H > DISCO_MAX_CLF_HIDDEN) return DISCO_ERR_INVALID_ARG;
+    if (clf->H > c->clf_hidden) return DISCO_ERR_WORKSPACE;
+    return DISCO_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* disco_strerror(int code) {
+    switch (code) {
+        case DISCO_OK: return "ok";
+        case DISCO_ERR_INVALID_ARG: return "invalid argument (null or misaligned pointer, size out of range)";
+        case DISCO_ERR_UNSUPPORTED_SHAPE: return "shape not supported by the kernels";
+        case DISCO_ERR_WORKSPACE: return "batch, rows or classifier width beyond what the context was created for";
+        case DISCO_ERR_CUDA: return "a CUDA runtime call failed";
+        case DISCO_ERR_TIMEOUT: return "a bounded device-side wait ran out";
+        default: return "unknown disco status";
+    }
+}
+
+int disco_create(disco_ctx** out, int V, int d_draft, int d_target, int max_batch, int max_rows, int k,
+                 int clf_hidden) {
+    if (!out) return DISCO_ERR_INVALID_ARG;
+    if (V < 1 || d_draft < 8 || d_target < 8 || (d_draft % 8) || (d_target % 8)) return DISCO_ERR_INVALID_ARG;
+    if (max_batch < 1 || max_rows < 1 || k != DISCO_TOPK) return DISCO_ERR_INVALID_ARG;
+    if (clf_hidden < 1 || clf_hidden > DISCO_MAX_CLF_HIDDEN) return DISCO_ERR_INVALID_ARG;
+    if (d_draft > kMaxHidden || d_target > kMaxHidden) return DISCO_ERR_UNSUPPORTED_SHAPE;
+
+    disco_ctx* c = new (std::nothrow) disco_ctx();
+    if (!c) return DISCO_ERR_CUDA;
+    std::memset(c, 0, sizeof(*c));
+    cudaDeviceProp prop;
+    if (cudaGetDevice(&c->device) != cudaSuccess || cudaGetDeviceProperties(&prop, c->device) != cudaSuccess) {
+        delete c;
+        return DISCO_ERR_CUDA;
+    }
+    c->V = V;
+    c->d_draft = d_draft;
+    c->d_target = d_target;
+    c->max_batch = max_batch;
+    c->max_rows = max_rows;
+    c->clf_hidden = clf_hidden;
+    c->sm_count = prop.multiProcessorCount;
+    c->smem_optin = prop.sharedMemPerBlockOptin;
+
+    const int rpc = std::max(1, std::min((V + c->sm_count - 1) / c->sm_count, 2048));
+    c->max_grid = (V + rpc - 1) / rpc;
+    c->part_rows = max_batch;
+    const size_t slots = (size_t)c->part_rows * c->max_grid;
+    const size_t n_int = (size_t)2 * max_batch + (size_t)max_rows + (max_batch + 1) + max_batch + 2 * (size_t)max_batch +
+                         (size_t)max_rows + 64;
+    const size_t hid = std::max((size_t)max_batch * d_draft, (size_t)max_rows * d_target) * 2;
+    bool ok = true;
+    ok = ok && cudaMalloc(&c->part_stats, slots * 4 * sizeof(float)) == cudaSuccess;
+    ok = ok && cudaMalloc(&c->part_topv, slots * kTopK * sizeof(float)) == cudaSuccess;
+    ok = ok && cudaMalloc(&c->part_topi, slots * kTopK * sizeof(int)) == cudaSuccess;
+    ok = ok && cudaMalloc(&c->keys, (size_t)max_rows * sizeof(unsigned long long)) == cudaSuccess;
+    ok = ok && cudaMalloc(&c->ticket, 256) == cudaSuccess;
+    ok = ok && cudaMalloc(&c->status, 256) == cudaSuccess;
+    ok = ok && cudaMalloc(&c->final_stats, (size_t)max_batch * 2 * sizeof(float)) == cudaSuccess;
+    ok = ok && cudaMalloc(&c->stage_hidden, hid) == cudaSuccess;
+    ok = ok && cudaMalloc(&c->stage_int, n_int * sizeof(int32_t)) == cudaSuccess;
+    ok = ok && cudaMalloc(&c->stage_float, (size_t)max_batch * (1 + kNFeat) * sizeof(float)) == cudaSuccess;
+    ok = ok && cudaMalloc(&c->stage_byte, (size_t)max_batch * 2 + 64) == cudaSuccess;
+    ok = ok && cudaMemset(c->keys, 0, (size_t)max_rows * sizeof(unsigned long long)) == cudaSuccess;
+    ok = ok && cudaMemset(c->ticket, 0, 256) == cudaSuccess;
+    ok = ok && cudaMemset(c->status, 0, 256) == cudaSuccess;
+    ok = ok && cudaDeviceSynchronize() == cudaSuccess;
+    if (!ok) {
+        disco_destroy(c);
+        return DISCO_ERR_CUDA;
+    }
+    *out = c;
+    return DISCO_OK;
+}
+
+int disco_destroy(disco_ctx* c) {
+    if (!c) return DISCO_ERR_INVALID_ARG;
+    cudaFree(c->part_stats);
+    cudaFree(c->part_topv);
+    cudaFree(c->part_topi);
+    cudaFree(c->keys);
+    cudaFree(c->ticket);
+    cudaFree(c->status);
+    cudaFree(c->final_stats);
+    cudaFree(c->stage_hidden);
+    cudaFree(c->stage_int);
+    cudaFree(c->stage_float);
+    cudaFree(c->stage_byte);
+    delete c;
+    return DISCO_OK;
+}
+
+int disco_last_device_status(disco_ctx* c, int* out) {
+    if (!c || !out) return DISCO_ERR_INVALID_ARG;
+    int v = 0;
+    if (cudaDeviceSynchronize() != cudaSuccess) return DISCO_ERR_CUDA;
+    if (cudaMemcpy(&v, c->status, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) return DISCO_ERR_CUDA;
+    if (cudaMemset(c->status, 0, sizeof(int)) != cudaSuccess) return DISCO_ERR_CUDA;
+    *out = v;
+    return DISCO_OK;
+}
+
+int disco_launch_count(disco_ctx* c, long long* out) {
+    if (!c || !out) return DISCO_ERR_INVALID_ARG;
+    *out = c->launches;
+    return DISCO_OK;
+}
+
+int disco_set_kernel_path(disco_ctx* c, int which) {
+    if (!c || which < 0 || which > 2) return DISCO_ERR_INVALID_ARG;
+    c->path = which;
+    return DISCO_OK;
+}
+
+int disco_draft_step(disco_ctx* c, const void* W_D, const void* h_D, int B, const int32_t* pos,
+                     const int32_t* n_drafted, const uint8_t* active, const disco_clf* clf, float tau,
+                     int sl_max, int32_t* token, float* conf, uint8_t* halt, float* feats, float* probs,
+                     void* stream) {
+    if (!c || !W_D || !h_D || !pos || !n_drafted || !token || !conf || !halt) return DISCO_ERR_INVALID_ARG;
+    if (!aligned16(W_D) || !aligned16(h_D)) return DISCO_ERR_INVALID_ARG;
+    if (B < 1 || sl_max < 1) return DISCO_ERR_INVALID_ARG;
+    if (B > c->max_batch) return DISCO_ERR_WORKSPACE;
+    int rc = check_clf(c, clf);
+    if (rc) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+
+    TailParams p{};
+    p.W = static_cast<const uint16_t*>(W_D);
+    p.H = static_cast<const uint16_t*>(h_D);
+    p.V = c->V;
+    p.d = c->d_draft;
+    p.R = B;
+    p.B = B;
+    fill_scratch(c, p);
+    p.pos = pos;
+    p.n_drafted = n_drafted;
+    p.active = active;
+    p.clf_W1 = clf->W1;
+    p.clf_b1 = clf->b1;
+    p.clf_w2 = clf->w2;
+    p.clf_b2 = clf->b2;
+    p.clf_H = clf->H;
+    p.tau = tau;
+    p.sl_max = sl_max;
+    p.token = token;
+    p.conf = conf;
+    p.halt = halt;
+    p.feats = feats;
+    p.probs = probs;
+    rc = run_stream<true>(c, p, clf->H, st);
+    if (rc) return rc;
+    if (probs) {
+        dim3 grid((unsigned)std::min(64, (c->V + 255) / 256), (unsigned)B);
+        normalize_probs_kernel<<<grid, 256, 0, st>>>(probs, c->final_stats, active, c->V);
+        c->launches += 1;
+        if (cudaGetLastError() != cudaSuccess) return DISCO_ERR_CUDA;
+    }
+    return DISCO_OK;
+}
+
+int disco_verify_ragged(disco_ctx* c, const void* W_T, const void* H_T, const int32_t* draft_ids,
+                        const int32_t* row_off, int B, int R, int32_t* n_accept, int32_t* bonus,
+                        int32_t* target_ids, void* stream) {
+    if (!c || !W_T || !H_T || !n_accept || !bonus) return DISCO_ERR_INVALID_ARG;
+    if (!aligned16(W_T) || !aligned16(H_T)) return DISCO_ERR_INVALID_ARG;
+    if (B < 1 || R < B) return DISCO_ERR_INVALID_ARG;
+    if (R > B && !draft_ids) return DISCO_ERR_INVALID_ARG;
+    if (R > c->max_rows) return DISCO_ERR_WORKSPACE;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+
+    TailParams p{};
+    p.W = static_cast<const uint16_t*>(W_T);
+    p.H = static_cast<const uint16_t*>(H_T);
+    p.V = c->V;
+    p.d = c->d_target;
+    p.R = R;
+    p.B = B;
+    p.SL = row_off ? 0 : (R / B - 1);
+    fill_scratch(c, p);
+    p.draft_ids = draft_ids;
+    p.row_off = row_off;
+    p.n_accept = n_accept;
+    p.bonus = bonus;
+    p.target_ids = target_ids;
+    return run_stream<false>(c, p, 0, st);
+}
+
+int disco_verify(disco_ctx* c, const void* W_T, const void* H_T, const int32_t* draft_ids, int B, int SL,
+                 int32_t* n_accept, int32_t* bonus, int32_t* target_ids, void* stream) {
+    if (B < 1 || SL < 0) return DISCO_ERR_INVALID_ARG;
+    const long long R = (long long)B * (SL + 1);
+    if (c && R > c->max_rows) return DISCO_ERR_WORKSPACE;
+    return disco_verify_ragged(c, W_T, H_T, draft_ids, nullptr, B, (int)R, n_accept, bonus, target_ids, stream);
+}
+
+int disco_draft_step_host(disco_ctx* c, const void* W_D, const void* h_D_host, int B, const int32_t* pos_host,
+                          const int32_t* n_drafted_host, const uint8_t* active_host, const disco_clf* clf,
+                          float tau, int sl_max, int32_t* token_host, float* conf_host, uint8_t* halt_host,
+                          float* feats_host, void* stream) {
+    if (!c || !h_D_host || !pos_host || !n_drafted_host || !token_host || !conf_host || !halt_host)
+        return DISCO_ERR_INVALID_ARG;
+    if (B < 1) return DISCO_ERR_INVALID_ARG;
+    if (B > c->max_batch) return DISCO_ERR_WORKSPACE;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const int mb = c->max_batch;
+    int32_t* d_pos = c->stage_int;
+    int32_t* d_nd = d_pos + mb;
+    int32_t* d_tok = d_nd + mb;
+    float* d_conf = c->stage_float;
+    float* d_feats = d_conf + mb;
+    uint8_t* d_act = c->stage_byte;
+    uint8_t* d_halt = d_act + mb;
+    bool ok = true;
+    ok = ok && cudaMemcpyAsync(c->stage_hidden, h_D_host, (size_t)B * c->d_draft * 2, cudaMemcpyHostToDevice, st) == cudaSuccess;
+    ok = ok && cudaMemcpyAsync(d_pos, pos_host, (size_t)B * 4, cudaMemcpyHostToDevice, st) == cudaSuccess;
+    ok = ok && cudaMemcpyAsync(d_nd, n_drafted_host, (size_t)B * 4, cudaMemcpyHostToDevice, st) == cudaSuccess;
+    if (active_host) ok = ok && cudaMemcpyAsync(d_act, active_host, (size_t)B, cudaMemcpyHostToDevice, st) == cudaSuccess;
+    if (!ok) return DISCO_ERR_CUDA;
+    int rc = disco_draft_step(c, W_D, c->stage_hidden, B, d_pos, d_nd, active_host ? d_act : nullptr, clf, tau,
+                              sl_max, d_tok, d_conf, d_halt, feats_host ? d_feats : nullptr, nullptr, stream);
+    if (rc) return rc;
+    if (active_host) {
+        // inactive sequences keep the caller's values: copy back only what the kernel wrote
+        for (int b = 0; b < B; ++b) {
+            if (!active_host[b]) continue;
+            ok = ok && cudaMemcpyAsync(token_host + b, d_tok + b, 4, cudaMemcpyDeviceToHost, st) == cudaSuccess;
+            ok = ok && cudaMemcpyAsync(conf_host + b, d_conf + b, 4, cudaMemcpyDeviceToHost, st) == cudaSuccess;
+            ok = ok && cudaMemcpyAsync(halt_host + b, d_halt + b, 1, cudaMemcpyDeviceToHost, st) == cudaSuccess;
+            if (feats_host)
+                ok = ok && cudaMemcpyAsync(feats_host + (size_t)b * kNFeat, d_feats + (size_t)b * kNFeat,
+                                           kNFeat * 4, cudaMemcpyDeviceToHost, st) == cudaSuccess;
+        }
+    } else {
+        ok = ok && cudaMemcpyAsync(token_host, d_tok, (size_t)B * 4, cudaMemcpyDeviceToHost, st) == cudaSuccess;
+        ok = ok && cudaMemcpyAsync(conf_host, d_conf, (size_t)B * 4, cudaMemcpyDeviceToHost, st) == cudaSuccess;
+        ok = ok && cudaMemcpyAsync(halt_host, d_halt, (size_t)B, cudaMemcpyDeviceToHost, st) == cudaSuccess;
+        if (feats_host)
+            ok = ok && cudaMemcpyAsync(feats_host, d_feats, (size_t)B * kNFeat * 4, cudaMemcpyDeviceToHost, st) == cudaSuccess;
+    }
+    ok = ok && cudaStreamSynchronize(st) == cudaSuccess;
+    return ok ? DISCO_OK : DISCO_ERR_CUDA;
+}
+
+int disco_verify_ragged_host(disco_ctx* c, const void* W_T, const void* H_T_host, const int32_t* draft_ids_host,
+                             const int32_t* row_off_host, int B, int R, int32_t* n_accept_host,
+                             int32_t* bonus_host, int32_t* target_ids_host, void* stream) {
+    if (!c || !H_T_host || !row_off_host || !n_accept_host || !bonus_host) return DISCO_ERR_INVALID_ARG;
+    if (B < 1 || R < B) return DISCO_ERR_INVALID_ARG;
+    if (R > B && !draft_ids_host) return DISCO_ERR_INVALID_ARG;
+    if (B > c->max_batch || R > c->max_rows) return DISCO_ERR_WORKSPACE;
+    // the host can see row_off here, so check it before anything is enqueued
+    if (row_off_host[0] != 0 || row_off_host[B] != R) return DISCO_ERR_INVALID_ARG;
+    for (int b = 0; b < B; ++b)
+        if (row_off_host[b + 1] <= row_off_host[b]) return DISCO_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const int mb = c->max_batch, mr = c->max_rows;
+    int32_t* d_ids = c->stage_int + 3 * (size_t)mb;
+    int32_t* d_off = d_ids + mr;
+    int32_t* d_nacc = d_off + mb + 1;
+    int32_t* d_bonus = d_nacc + mb;
+    int32_t* d_tids = d_bonus + mb;
+    bool ok = true;
+    ok = ok && cudaMemcpyAsync(c->stage_hidden, H_T_host, (size_t)R * c->d_target * 2, cudaMemcpyHostToDevice, st) == cudaSuccess;
+    if (R > B) ok = ok && cudaMemcpyAsync(d_ids, draft_ids_host, (size_t)(R - B) * 4, cudaMemcpyHostToDevice, st) == cudaSuccess;
+    ok = ok && cudaMemcpyAsync(d_off, row_off_host, (size_t)(B + 1) * 4, cudaMemcpyHostToDevice, st) == cudaSuccess;
+    if (!ok) return DISCO_ERR_CUDA;
+    int rc = disco_verify_ragged(c, W_T, c->stage_hidden, d_ids, d_off, B, R, d_nacc, d_bonus,
+                                 target_ids_host ? d_tids : nullptr, stream);
+    if (rc) return rc;
+    ok = ok && cudaMemcpyAsync(n_accept_host, d_nacc, (size_t)B * 4, cudaMemcpyDeviceToHost, st) == cudaSuccess;
+    ok = ok && cudaMemcpyAsync(bonus_host, d_bonus, (size_t)B * 4, cudaMemcpyDeviceToHost, st) == cudaSuccess;
+    if (target_ids_host)
+        ok = ok && cudaMemcpyAsync(target_ids_host, d_tids, (size_t)R * 4, cudaMemcpyDeviceToHost, st) == cudaSuccess;
+    ok = ok && cudaStreamSynchronize(st) == cudaSuccess;
+    return ok ? DISCO_OK : DISCO_ERR_CUDA;
+}
+
+}  // extern "C"

@@ -2,7 +2,7 @@
 
 This module only draws random numbers and packs them.  It contains none of the
 method's arithmetic (no projection, soft-max, classifier or prefix match), so
-it can feed the CUDA library, the CPU oracle and the benchmark alike without
+it can feed the CUDA library, a CPU checker and the benchmark alike without
 making any of them depend on another.  It never loads the CUDA library.
 
 The workloads mirror the model pairs the paper evaluates (Vicuna-13B/68M and

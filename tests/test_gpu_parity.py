@@ -1,0 +1,248 @@
+"""Parity of the CUDA library (through its C ABI) with the CPU oracle, element by element on the same
+seeded inputs.  Needs a B200: run with -m gpu."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2405_04304_b200 import binding, inputs
+from util import (check_draft, check_verify, gpu_draft_step, gpu_verify, make_clf, to_gpu_clf,
+                  to_oracle_clf)
+
+pytestmark = pytest.mark.gpu
+
+
+def _bits(t):
+    return inputs.bf16_bits(t)
+
+
+def _ctx(V, dD, dT, max_batch=8, max_rows=64, H=64):
+    return binding.Context(V, dD, dT, max_batch=max_batch, max_rows=max_rows, clf_hidden=H)
+
+
+# ---------------------------------------------------------------------------------- draft step
+@pytest.mark.parametrize("V,d,B", [(1, 8, 1), (5, 8, 2), (9, 16, 1), (10, 16, 3), (11, 24, 1), (64, 64, 5),
+                                   (217, 72, 2), (1000, 128, 4), (4099, 264, 7), (33, 8, 8)])
+def test_draft_step_small_shapes(oracle, V, d, B):
+    W = inputs.lm_head(V, d, seed=V + d, std=0.3)
+    h = inputs.hidden(B, d, seed=V * 7 + B)
+    params = make_clf(16, seed=V)
+    pos = np.arange(1, B + 1, dtype=np.int32) * 3
+    nd = (np.arange(B, dtype=np.int32) % 4) + 1
+    ctx = _ctx(V, d, 8, max_batch=8, H=16)
+    got = gpu_draft_step(ctx, W.cuda(), h, pos, nd, to_gpu_clf(params), 0.5, 3, want_probs=True)
+    ref = oracle.draft_step(_bits(W), _bits(h), pos, nd, to_oracle_clf(oracle, params), 0.5, 3, want_probs=True)
+    check_draft(got, ref, 0.5)
+    assert ctx.device_status() == 0
+    ctx.close()
+
+
+def test_draft_step_tiny_workload_shapes(oracle):
+    wl = inputs.WORKLOADS["tiny"]
+    W = inputs.lm_head(wl.V, wl.d_D, seed=inputs.sub_seed(wl.seed, 1))
+    params = make_clf(wl.H, seed=inputs.sub_seed(wl.seed, 2))
+    ctx = _ctx(wl.V, wl.d_D, wl.d_T, H=wl.H)
+    Wg, clf_g, clf_o = W.cuda(), to_gpu_clf(params), to_oracle_clf(oracle, params)
+    exempt = 0
+    for step in range(6):
+        h = inputs.hidden(1, wl.d_D, seed=inputs.sub_seed(wl.seed, 3, step))
+        pos, nd = np.array([step + 1], np.int32), np.array([step % wl.sl_max + 1], np.int32)
+        got = gpu_draft_step(ctx, Wg, h, pos, nd, clf_g, wl.tau, wl.sl_max, want_probs=(step == 0))
+        ref = oracle.draft_step(_bits(W), _bits(h), pos, nd, clf_o, wl.tau, wl.sl_max, want_probs=(step == 0),
+                                nthreads=8)
+        exempt += check_draft(got, ref, wl.tau)
+    assert exempt <= 1
+    assert ctx.device_status() == 0
+    ctx.close()
+
+
+@pytest.mark.parametrize("name", ["vicuna_b1", "starcoder_b1"])
+def test_draft_step_full_size_heads(oracle, name):
+    wl = inputs.WORKLOADS[name]
+    W = inputs.lm_head(wl.V, wl.d_D, seed=inputs.sub_seed(wl.seed, 1))
+    params = make_clf(wl.H, seed=inputs.sub_seed(wl.seed, 2))
+    ctx = _ctx(wl.V, wl.d_D, wl.d_T, H=wl.H)
+    for B in (1, 3):
+        h = inputs.hidden(B, wl.d_D, seed=inputs.sub_seed(wl.seed, 3, B))
+        pos, nd = np.arange(10, 10 + B, dtype=np.int32), np.ones(B, np.int32)
+        got = gpu_draft_step(ctx, W.cuda(), h, pos, nd, to_gpu_clf(params), wl.tau, wl.sl_max)
+        ref = oracle.draft_step(_bits(W), _bits(h), pos, nd, to_oracle_clf(oracle, params), wl.tau, wl.sl_max,
+                                nthreads=8)
+        check_draft(got, ref, wl.tau)
+    assert ctx.device_status() == 0
+    ctx.close()
+
+
+def test_draft_step_closed_forms(oracle):
+    V, d = 3000, 64
+    W = inputs.lm_head(V, d, seed=5, std=0.1)
+    params = make_clf(8, seed=6)
+    ctx = _ctx(V, d, 8, H=8)
+    # zero hidden state: uniform distribution, entropy ln V, token 0 (lowest index among equals)
+    h = torch.zeros(1, d, dtype=torch.bfloat16)
+    got = gpu_draft_step(ctx, W.cuda(), h, [4], [1], to_gpu_clf(params), 0.5, 5, want_probs=True)
+    assert got["token"][0] == 0
+    np.testing.assert_allclose(got["probs"][0], 1.0 / V, rtol=1e-5)
+    np.testing.assert_allclose(got["feats"][0, :10], 1.0 / V, rtol=1e-5)
+    assert abs(got["feats"][0, 10] - np.log(V)) < 1e-4
+    # planted peak: hidden state aligned with one row
+    h = (W[1234].float() * 300.0).to(torch.bfloat16).view(1, d)
+    got = gpu_draft_step(ctx, W.cuda(), h, [4], [1], to_gpu_clf(params), 0.5, 5)
+    ref = oracle.draft_step(_bits(W), _bits(h), [4], [1], to_oracle_clf(oracle, params), 0.5, 5)
+    assert got["token"][0] == 1234 == ref.token[0]
+    check_draft(got, ref, 0.5)
+    assert got["feats"][0, 0] > 0.99
+    ctx.close()
+
+
+def test_threshold_rule_and_cap(oracle):
+    V, d, B = 500, 32, 4
+    W = inputs.lm_head(V, d, seed=8, std=0.2)
+    h = inputs.hidden(B, d, seed=9)
+    params = make_clf(8, seed=10)
+    flat = make_clf(8, seed=10, zero_head=True)
+    ctx = _ctx(V, d, 8, H=8)
+    Wg = W.cuda()
+    pos = np.arange(1, B + 1, dtype=np.int32)
+    for nd, expect in ((1, 0), (4, 0), (5, 1), (7, 1)):      # tau <= 0: static SL = SL_max
+        got = gpu_draft_step(ctx, Wg, h, pos, np.full(B, nd, np.int32), to_gpu_clf(params), 0.0, 5)
+        assert list(got["halt"]) == [expect] * B
+    got = gpu_draft_step(ctx, Wg, h, pos, np.ones(B, np.int32), to_gpu_clf(params), 1.5, 5)
+    assert list(got["halt"]) == [1] * B                      # tau > 1: SL = 1
+    got = gpu_draft_step(ctx, Wg, h, pos, np.ones(B, np.int32), to_gpu_clf(flat), 0.5, 5)
+    assert list(got["conf"]) == [0.5] * B and list(got["halt"]) == [0] * B   # C == tau continues
+    got = gpu_draft_step(ctx, Wg, h, pos, np.ones(B, np.int32), to_gpu_clf(flat), 0.5000001, 5)
+    assert list(got["halt"]) == [1] * B
+    halts = [gpu_draft_step(ctx, Wg, h, pos, np.ones(B, np.int32), to_gpu_clf(params), tau, 9)["halt"]
+             for tau in (0.3, 0.5, 0.7)]
+    assert np.all(halts[0] <= halts[1]) and np.all(halts[1] <= halts[2])
+    ctx.close()
+
+
+def test_inactive_sequences_are_not_written(oracle):
+    V, d, B = 700, 40, 5
+    W = inputs.lm_head(V, d, seed=11, std=0.2)
+    h = inputs.hidden(B, d, seed=12)
+    params = make_clf(8, seed=13)
+    active = np.array([1, 0, 1, 0, 1], np.uint8)
+    pos, nd = np.arange(B, dtype=np.int32) + 2, np.ones(B, np.int32)
+    ctx = _ctx(V, d, 8, H=8)
+    ref = oracle.draft_step(_bits(W), _bits(h), pos, nd, to_oracle_clf(oracle, params), 0.5, 5, active=active)
+    for host in (False, True):
+        got = gpu_draft_step(ctx, W.cuda(), h, pos, nd, to_gpu_clf(params), 0.5, 5, active=active, host=host)
+        check_draft(got, ref, 0.5, active=active)
+    ctx.close()
+
+
+def test_draft_step_is_deterministic_and_host_variant_matches():
+    V, d, B = 32000, 768, 2
+    W = inputs.lm_head(V, d, seed=14).cuda()
+    h = inputs.hidden(B, d, seed=15)
+    clf = to_gpu_clf(make_clf(64, seed=16))
+    ctx = _ctx(V, d, 8)
+    a = gpu_draft_step(ctx, W, h, [1, 2], [1, 1], clf, 0.5, 5)
+    b = gpu_draft_step(ctx, W, h, [1, 2], [1, 1], clf, 0.5, 5)
+    c = gpu_draft_step(ctx, W, h, [1, 2], [1, 1], clf, 0.5, 5, host=True)
+    for k in ("token", "conf", "halt", "feats"):
+        np.testing.assert_array_equal(a[k], b[k])
+        np.testing.assert_array_equal(a[k], c[k])
+    ctx.close()
+
+
+# ---------------------------------------------------------------------------------- verification
+@pytest.mark.parametrize("V,d,sls", [(1, 8, [0]), (7, 8, [2]), (64, 16, [5]), (64, 16, [3, 0, 5, 1]),
+                                     (1000, 136, [10]), (4099, 72, [1, 2, 3, 4, 5, 6]), (300, 64, [40, 33, 0])])
+def test_verify_small_shapes(oracle, V, d, sls):
+    sl = torch.tensor(sls, dtype=torch.int32)
+    off = inputs.row_offsets(sl).numpy()
+    R, B = int(off[-1]), len(sls)
+    W = inputs.lm_head(V, d, seed=V + d, std=0.3)
+    H = inputs.hidden(R, d, seed=V + R)
+    free = oracle.verify_ragged(_bits(W), _bits(H), np.zeros(R - B, np.int32), off)   # target ids only
+    clean = np.concatenate([free.target_ids[off[b]:off[b + 1] - 1] for b in range(B)]).astype(np.int32)
+    draft = inputs.corrupt_ids(torch.from_numpy(clean), 0.25, V, seed=R).numpy()
+    ref = oracle.verify_ragged(_bits(W), _bits(H), draft, off)
+    ctx = binding.Context(V, 8, d, max_batch=8, max_rows=128)
+    got = gpu_verify(ctx, W.cuda(), H, draft, row_off=off)
+    check_verify(got, ref, off, draft)
+    got_h = gpu_verify(ctx, W.cuda(), H, draft, row_off=off, host=True)
+    for k in ("n_accept", "bonus", "target_ids"):
+        np.testing.assert_array_equal(got[k], got_h[k])
+    if len(set(sls)) == 1:                                    # uniform entry point == ragged entry point
+        got_u = gpu_verify(ctx, W.cuda(), H, draft, B=B, SL=sls[0])
+        for k in ("n_accept", "bonus", "target_ids"):
+            np.testing.assert_array_equal(got[k], got_u[k])
+    assert ctx.device_status() == 0
+    ctx.close()
+
+
+def test_verify_fig1_and_special_cases(oracle):
+    V, d, SL = 2000, 64, 5
+    W = inputs.lm_head(V, d, seed=21, std=0.3)
+    H = inputs.hidden(SL + 1, d, seed=22)
+    a = oracle.verify(_bits(W), _bits(H), np.zeros(SL, np.int32), 1, SL).target_ids
+    ctx = binding.Context(V, 8, d, max_batch=2, max_rows=16)
+    Wg = W.cuda()
+    got = gpu_verify(ctx, Wg, H, a[:SL], B=1, SL=SL)               # draft == target: all accepted
+    assert got["n_accept"][0] == SL and got["bonus"][0] == a[SL]
+    fig1 = a[:SL].copy()
+    fig1[3] = (fig1[3] + 1) % V                                     # Fig. 1: t4 and t5 rejected
+    fig1[4] = (fig1[4] + 1) % V
+    got = gpu_verify(ctx, Wg, H, fig1, B=1, SL=SL)
+    assert got["n_accept"][0] == 3 and got["bonus"][0] == a[3]
+    hole = a[:SL].copy()
+    hole[0] = (hole[0] + 1) % V                                     # first wrong: later matches do not count
+    got = gpu_verify(ctx, Wg, H, hole, B=1, SL=SL)
+    assert got["n_accept"][0] == 0 and got["bonus"][0] == a[0]
+    got = gpu_verify(ctx, Wg, H[:1], np.zeros(0, np.int32), B=1, SL=0)   # SL = 0: plain target step
+    assert got["n_accept"][0] == 0 and got["bonus"][0] == a[0]
+    ctx.close()
+
+
+@pytest.mark.parametrize("name,SL", [("tiny", 5), ("vicuna_b1", 10), ("starcoder_b1", 10)])
+def test_verify_full_size_heads(oracle, name, SL):
+    wl = inputs.WORKLOADS[name]
+    W = inputs.lm_head(wl.V, wl.d_T, seed=inputs.sub_seed(wl.seed, 4))
+    H = inputs.hidden(SL + 1, wl.d_T, seed=inputs.sub_seed(wl.seed, 5))
+    free = oracle.verify(_bits(W), _bits(H), np.zeros(SL, np.int32), 1, SL, nthreads=8)
+    draft = inputs.corrupt_ids(torch.from_numpy(free.target_ids[:SL].copy()), wl.p_corrupt, wl.V,
+                               seed=inputs.sub_seed(wl.seed, 6)).numpy()
+    ref_n, ref_bonus = oracle.accept_prefix(draft, free.target_ids)
+    ctx = binding.Context(wl.V, wl.d_D, wl.d_T, max_batch=1, max_rows=SL + 1)
+    got = gpu_verify(ctx, W.cuda(), H, draft, B=1, SL=SL)
+    ref = oracle.VerifyResult(np.array([ref_n], np.int32), np.array([ref_bonus], np.int32), free.target_ids,
+                              free.gap)
+    check_verify(got, ref, [0, SL + 1], draft)
+    assert ctx.device_status() == 0
+    ctx.close()
+
+
+# ---------------------------------------------------------------------------------- error handling
+def test_errors_are_codes_not_faults():
+    V, d = 100, 16
+    ctx = binding.Context(V, d, d, max_batch=2, max_rows=8, clf_hidden=8)
+    W = inputs.lm_head(V, d, seed=1).cuda()
+    clf = to_gpu_clf(make_clf(8, seed=2))
+    h3 = inputs.hidden(3, d, seed=3)
+    with pytest.raises(binding.DiscoError) as e:
+        gpu_draft_step(ctx, W, h3, [1, 2, 3], [1, 1, 1], clf, 0.5, 5)
+    assert e.value.code == binding.ERR_WORKSPACE
+    big = to_gpu_clf(make_clf(16, seed=2))
+    with pytest.raises(binding.DiscoError) as e:
+        gpu_draft_step(ctx, W, h3[:1], [1], [1], big, 0.5, 5)
+    assert e.value.code == binding.ERR_WORKSPACE
+    with pytest.raises(binding.DiscoError) as e:
+        gpu_verify(ctx, W, inputs.hidden(9, d, seed=4), np.zeros(8, np.int32), B=1, SL=8)
+    assert e.value.code == binding.ERR_WORKSPACE
+    with pytest.raises(binding.DiscoError) as e:                     # misaligned LM head
+        gpu_draft_step(ctx, W.view(-1)[4:4 + 50 * d].view(50, d), h3[:1], [1], [1], clf, 0.5, 5)
+    assert e.value.code == binding.ERR_INVALID_ARG
+    # inconsistent row offsets are caught by the kernel: status word + -1 outputs, no fault
+    H = inputs.hidden(6, d, seed=5)
+    got = gpu_verify(ctx, W, H, np.zeros(4, np.int32), row_off=[0, 4, 7])
+    assert got["n_accept"][1] == -1 and got["bonus"][1] == -1
+    assert ctx.device_status() == binding.ERR_INVALID_ARG
+    assert ctx.device_status() == 0
+    # the context still works afterwards
+    got = gpu_verify(ctx, W, H, np.zeros(4, np.int32), row_off=[0, 4, 6])
+    assert np.all(got["n_accept"] >= 0)
+    ctx.close()
