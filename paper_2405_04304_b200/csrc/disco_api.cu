@@ -4,6 +4,7 @@
 
 #include <algorithm>
 #include <cstdio>
+#include <cstdlib>
 #include <cstring>
 #include <new>
 
@@ -16,7 +17,7 @@ namespace {
 
 constexpr int kStreamWarps = 16;     // consumer warps of the streaming kernel
 constexpr int kMaxHidden = 16384;    // widest hidden dimension the kernels accept
-constexpr int kSlotTargetBytes = 12288;
+constexpr int kSlotTargetBytes = 6144;
 
 struct StreamPlan {
     int rows_per_cta, grid, rps, stages;
@@ -53,6 +54,14 @@ struct disco_ctx {
 
 namespace {
 
+// With DISCO_DEBUG set in the environment, failed CUDA runtime calls are reported on stderr.
+inline bool cuda_ok(cudaError_t e, const char* what) {
+    if (e == cudaSuccess) return true;
+    static const bool verbose = std::getenv("DISCO_DEBUG") != nullptr;
+    if (verbose) std::fprintf(stderr, "[disco] %s: %s\n", what, cudaGetErrorString(e));
+    return false;
+}
+
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 StreamPlan plan_stream(const disco_ctx* c, int V, int d, int RT, int clf_H) {
@@ -70,8 +79,8 @@ StreamPlan plan_stream(const disco_ctx* c, int V, int d, int RT, int clf_H) {
     const size_t budget = c->smem_optin > 2048 ? c->smem_optin - 2048 : 0;
     if (budget <= fixed) return pl;
     long long stages = (long long)((budget - fixed) / (pl.slot_bytes + 16));
-    const int need = (rpc + rps - 1) / rps;  // slots that one pass over the slab takes
-    stages = std::min<long long>(stages, std::max(2, std::min(need, 24)));
+    stages = std::min<long long>(stages, 2 * kStreamWarps);
+    if (stages > kStreamWarps) stages -= stages % kStreamWarps;  // slots are dealt round-robin to the warps
     if (stages < 2) return pl;
     pl.stages = (int)stages;
     pl.smem = stream_tail_smem_bytes(RT, kStreamWarps, d, pl.stages, pl.slot_bytes, clf_H);
@@ -83,17 +92,20 @@ template <int RT, bool DRAFT>
 int launch_stream(disco_ctx* c, TailParams& p, const StreamPlan& pl, cudaStream_t st) {
     auto kern = stream_tail_kernel<RT, DRAFT, kStreamWarps>;
     static int configured_dev = -1;
-    static size_t configured_smem = 0;
-    if (configured_dev != c->device || configured_smem < pl.smem) {
-        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)c->smem_optin) !=
-            cudaSuccess)
+    static size_t dyn_limit = 0;
+    if (configured_dev != c->device) {
+        cudaFuncAttributes fa;
+        if (!cuda_ok(cudaFuncGetAttributes(&fa, kern), "cudaFuncGetAttributes")) return DISCO_ERR_CUDA;
+        dyn_limit = c->smem_optin - fa.sharedSizeBytes;
+        if (!cuda_ok(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn_limit),
+                     "cudaFuncSetAttribute"))
             return DISCO_ERR_CUDA;
         configured_dev = c->device;
-        configured_smem = c->smem_optin;
     }
+    if (pl.smem > dyn_limit) return DISCO_ERR_UNSUPPORTED_SHAPE;
     kern<<<pl.grid, (kStreamWarps + 1) * 32, pl.smem, st>>>(p);
     c->launches += 1;
-    return cudaGetLastError() == cudaSuccess ? DISCO_OK : DISCO_ERR_CUDA;
+    return cuda_ok(cudaGetLastError(), "stream_tail_kernel launch") ? DISCO_OK : DISCO_ERR_CUDA;
 }
 
 template <bool DRAFT>

@@ -273,7 +273,7 @@ __global__ void __launch_bounds__((NW + 1) * 32, 1) stream_tail_kernel(const __g
     if (tid == 0) {
         for (int s = 0; s < p.stages; ++s) {
             mbar_init(&full[s], 1);
-            mbar_init(&empty[s], p.rps);
+            mbar_init(&empty[s], 1);
         }
         fence_mbar_init();
     }
@@ -334,54 +334,54 @@ __global__ void __launch_bounds__((NW + 1) * 32, 1) stream_tail_kernel(const __g
             best_i[r] = kNoIndex;
         }
 
-        for (int g = warp; g < nrows; g += NW) {
-            const int fill = chunk * nslots + g / p.rps;
-            const int s = fill % p.stages;
-            const int it = fill / p.stages;
-            mbar_wait(&full[s], it & 1, p.status);
-            const uint4* wrow = reinterpret_cast<const uint4*>(ring + (size_t)s * p.slot_bytes +
-                                                              (size_t)(g % p.rps) * row_bytes);
-            float acc[RT];
+        // Each ring slot belongs to one warp (slot s -> warp s % NW), so a warp meets every phase
+        // of the barriers it waits on, in order: parity waits can never alias an older phase.
+        const int f_begin = chunk * nslots;
+        for (int f = f_begin; f < f_begin + nslots; ++f) {
+            const int s = f % p.stages;
+            if ((s % NW) != warp) continue;
+            mbar_wait(&full[s], (f / p.stages) & 1, p.status);
+            const int r0 = (f - f_begin) * p.rps;
+            const int nr = min(p.rps, nrows - r0);
+            for (int j = 0; j < nr; ++j) {
+                const uint4* wrow = reinterpret_cast<const uint4*>(ring + (size_t)s * p.slot_bytes +
+                                                                  (size_t)j * row_bytes);
+                float acc[RT];
 #pragma unroll
-            for (int r = 0; r < RT; ++r) acc[r] = 0.f;
+                for (int r = 0; r < RT; ++r) acc[r] = 0.f;
 #pragma unroll 4
-            for (int c = lane; c < n16; c += 32) {
-                float wf[8];
-                unpack_bf16x8(wrow[c], wf);
+                for (int c = lane; c < n16; c += 32) {
+                    float wf[8];
+                    unpack_bf16x8(wrow[c], wf);
+#pragma unroll
+                    for (int r = 0; r < RT; ++r) {
+                        float hf[8];
+                        unpack_bf16x8(reinterpret_cast<const uint4*>(htile + (size_t)r * row_bytes)[c], hf);
+#pragma unroll
+                        for (int k = 0; k < 8; ++k) acc[r] = fmaf(wf[k], hf[k], acc[r]);
+                    }
+                }
+                const int v = v0 + r0 + j;
 #pragma unroll
                 for (int r = 0; r < RT; ++r) {
-                    float hf[8];
-                    unpack_bf16x8(reinterpret_cast<const uint4*>(htile + (size_t)r * row_bytes)[c], hf);
 #pragma unroll
-                    for (int k = 0; k < 8; ++k) acc[r] = fmaf(wf[k], hf[k], acc[r]);
-                }
-            }
-            __syncwarp();
-            if (lane == 0) {  // this row of the slot is consumed
-                mbar_arrive(&empty[s]);
-                if (g == nrows - 1) {  // a short last slot still needs rps arrivals
-                    const int missing = nslots * p.rps - nrows;
-                    for (int k = 0; k < missing; ++k) mbar_arrive(&empty[s]);
-                }
-            }
-#pragma unroll
-            for (int r = 0; r < RT; ++r) {
-#pragma unroll
-                for (int off = 16; off > 0; off >>= 1) acc[r] += __shfl_xor_sync(kFullMask, acc[r], off);
-                const float z = __fadd_rn(acc[r], 0.f);  // folds -0 into +0
-                const int v = v0 + g;
-                if (DRAFT) {
-                    st[r].push(z);
-                    top[r].offer(z, v, lane);
-                    if (p.probs && lane == 0 && chunk * RT + r < p.R)
-                        p.probs[(size_t)(chunk * RT + r) * p.V + v] = z;
-                } else {
-                    if (z > best_v[r]) {
-                        best_v[r] = z;
-                        best_i[r] = v;
+                    for (int off = 16; off > 0; off >>= 1) acc[r] += __shfl_xor_sync(kFullMask, acc[r], off);
+                    const float z = __fadd_rn(acc[r], 0.f);  // folds -0 into +0
+                    if (DRAFT) {
+                        st[r].push(z);
+                        top[r].offer(z, v, lane);
+                        if (p.probs && lane == 0 && chunk * RT + r < p.R)
+                            p.probs[(size_t)(chunk * RT + r) * p.V + v] = z;
+                    } else {
+                        if (z > best_v[r]) {
+                            best_v[r] = z;
+                            best_i[r] = v;
+                        }
                     }
                 }
             }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&empty[s]);  // the slot may be refilled
         }
 
         // ---- merge the NW warps of this CTA, publish the CTA's partial for each hidden row ----
