@@ -14,8 +14,8 @@ constexpr int kNFeat = DISCO_NFEAT;
 constexpr unsigned kFullMask = 0xffffffffu;
 constexpr int kNoIndex = 0x7fffffff;
 
-// Bounded-wait budget: a barrier wait gives up after this many clock ticks (about 0.2 s).
-constexpr long long kWaitBudgetClocks = 400000000ll;
+// Bounded-wait budget: a barrier wait gives up after this many clock ticks (about 0.05 s).
+constexpr long long kWaitBudgetClocks = 100000000ll;
 
 // ------------------------------------------------------------------------------------------
 // status word
@@ -68,11 +68,11 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, int* s
     if (mbar_try_wait(bar, parity)) return true;
     const long long t0 = clock64();
     for (;;) {
-#pragma unroll 1
-        for (int i = 0; i < 256; ++i)
-            if (mbar_try_wait(bar, parity)) return true;
-        // once any wait in the grid has run out, the others give up at once
+        // once any wait in the grid has run out, all others give up at once
         if (status && *reinterpret_cast<volatile int*>(status) == DISCO_ERR_TIMEOUT) return false;
+#pragma unroll 1
+        for (int i = 0; i < 64; ++i)
+            if (mbar_try_wait(bar, parity)) return true;
         if (clock64() - t0 > kWaitBudgetClocks) {
             record_status(status, DISCO_ERR_TIMEOUT);
             return false;

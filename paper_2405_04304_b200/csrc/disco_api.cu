@@ -10,6 +10,7 @@
 
 #include "disco.h"
 #include "stream_tail.cuh"
+#include "umma_tail.cuh"
 
 using namespace disco;
 
@@ -45,6 +46,9 @@ struct disco_ctx {
     unsigned int* ticket;
     int* status;
     float* final_stats;
+    unsigned long long* part_key;  // tcgen05 draft path: arg-max key per partial
+    int part_slots;                // partials per row the buffers can hold
+    void* encode_tiled;            // cuTensorMapEncodeTiled, resolved through the runtime
     // device staging for the *_host entry points
     void* stage_hidden;
     int32_t* stage_int;   // pos | n_drafted | draft_ids | row_off | token | n_accept | bonus | target_ids
@@ -88,9 +92,9 @@ StreamPlan plan_stream(const disco_ctx* c, int V, int d, int RT, int clf_H) {
     return pl;
 }
 
-template <int RT, bool DRAFT>
+template <int RT, bool DRAFT, int KC>
 int launch_stream(disco_ctx* c, TailParams& p, const StreamPlan& pl, cudaStream_t st) {
-    auto kern = stream_tail_kernel<RT, DRAFT, kStreamWarps>;
+    auto kern = stream_tail_kernel<RT, DRAFT, kStreamWarps, KC>;
     static int configured_dev = -1;
     static size_t dyn_limit = 0;
     if (configured_dev != c->device) {
@@ -119,10 +123,77 @@ int run_stream(disco_ctx* c, TailParams& p, int clf_H, cudaStream_t st) {
     p.stages = pl.stages;
     p.slot_bytes = pl.slot_bytes;
     switch (RT) {
-        case 1: return launch_stream<1, DRAFT>(c, p, pl, st);
-        case 2: return launch_stream<2, DRAFT>(c, p, pl, st);
-        default: return launch_stream<4, DRAFT>(c, p, pl, st);
+        case 1:  // one hidden row: the warp can hold its share of h in registers (32 * 8 * KC values)
+            if (p.d <= 768) return launch_stream<1, DRAFT, 3>(c, p, pl, st);
+            if (p.d <= 1024) return launch_stream<1, DRAFT, 4>(c, p, pl, st);
+            return launch_stream<1, DRAFT, 0>(c, p, pl, st);
+        case 2: return launch_stream<2, DRAFT, 0>(c, p, pl, st);
+        default: return launch_stream<4, DRAFT, 0>(c, p, pl, st);
     }
+}
+
+
+// ------------------------------------------------------------------------------------------------
+// tcgen05 path
+// ------------------------------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+// bf16 [rows, d] row-major, boxes of box_rows x 64 elements, 128-byte swizzle, zero fill out of bounds
+bool encode_bf16_2d(const disco_ctx* c, CUtensorMap* map, const void* base, int rows, int d, int box_rows) {
+    if (!c->encode_tiled) return false;
+    const cuuint64_t gdim[2] = {(cuuint64_t)d, (cuuint64_t)rows};
+    const cuuint64_t gstride[1] = {(cuuint64_t)d * 2};
+    const cuuint32_t box[2] = {(cuuint32_t)kUmmaBK, (cuuint32_t)box_rows};
+    const cuuint32_t estride[2] = {1, 1};
+    const CUresult r = reinterpret_cast<EncodeTiledFn>(c->encode_tiled)(
+        map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), gdim, gstride, box, estride,
+        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS;
+}
+
+bool umma_possible(const disco_ctx* c, int R) {
+    const int MT = (R + 127) / 128;
+    return c->encode_tiled != nullptr && MT <= c->sm_count;
+}
+
+// Launch the tcgen05 kernel for R hidden rows of width d against the LM head W [V, d].
+template <bool DRAFT>
+int launch_umma(disco_ctx* c, const void* W, const void* H, int d, int R, float* probs, int* n_partials,
+                cudaStream_t st) {
+    UmmaParams p{};
+    p.V = c->V;
+    p.d = d;
+    p.R = R;
+    p.MT = (R + 127) / 128;
+    p.CN = c->sm_count / p.MT;
+    p.G16 = (c->V + 15) / 16;
+    p.TPC = std::max(1, (p.G16 + 16 * p.CN - 1) / (16 * p.CN));
+    p.a_rows = p.MT > 1 ? 128 : std::max(8, (R + 7) / 8 * 8);
+    p.status = c->status;
+    p.keys = c->keys;
+    p.part_stats = c->part_stats;
+    p.part_topv = c->part_topv;
+    p.part_key = c->part_key;
+    p.probs = probs;
+    if (DRAFT && (2 * p.CN > c->part_slots || R > c->part_rows)) return DISCO_ERR_WORKSPACE;
+    if (n_partials) *n_partials = 2 * p.CN;
+    CUtensorMap tmap_W, tmap_H;
+    if (!encode_bf16_2d(c, &tmap_W, W, c->V, d, 16) || !encode_bf16_2d(c, &tmap_H, H, R, d, p.a_rows))
+        return DISCO_ERR_CUDA;
+    auto kern = umma_tail_kernel<DRAFT>;
+    static int configured_dev = -1;
+    if (configured_dev != c->device) {
+        if (!cuda_ok(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kUmmaSmemBytes),
+                     "cudaFuncSetAttribute(umma)"))
+            return DISCO_ERR_CUDA;
+        configured_dev = c->device;
+    }
+    kern<<<p.MT * p.CN, kUmmaThreads, kUmmaSmemBytes, st>>>(tmap_W, tmap_H, p);
+    c->launches += 1;
+    return cuda_ok(cudaGetLastError(), "umma_tail_kernel launch") ? DISCO_OK : DISCO_ERR_CUDA;
 }
 
 void fill_scratch(const disco_ctx* c, TailParams& p) {
@@ -186,7 +257,15 @@ int disco_create(disco_ctx** out, int V, int d_draft, int d_target, int max_batc
     const int rpc = std::max(1, std::min((V + c->sm_count - 1) / c->sm_count, 2048));
     c->max_grid = (V + rpc - 1) / rpc;
     c->part_rows = max_batch;
-    const size_t slots = (size_t)c->part_rows * c->max_grid;
+    c->part_slots = std::max(c->max_grid, 2 * c->sm_count);
+    const size_t slots = (size_t)c->part_rows * c->part_slots;
+    {
+        cudaDriverEntryPointQueryResult qres;
+        void* fn = nullptr;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) == cudaSuccess &&
+            qres == cudaDriverEntryPointSuccess)
+            c->encode_tiled = fn;
+    }
     const size_t n_int = (size_t)2 * max_batch + (size_t)max_rows + (max_batch + 1) + max_batch + 2 * (size_t)max_batch +
                          (size_t)max_rows + 64;
     const size_t hid = std::max((size_t)max_batch * d_draft, (size_t)max_rows * d_target) * 2;
@@ -195,6 +274,7 @@ int disco_create(disco_ctx** out, int V, int d_draft, int d_target, int max_batc
     ok = ok && cudaMalloc(&c->part_topv, slots * kTopK * sizeof(float)) == cudaSuccess;
     ok = ok && cudaMalloc(&c->part_topi, slots * kTopK * sizeof(int)) == cudaSuccess;
     ok = ok && cudaMalloc(&c->keys, (size_t)max_rows * sizeof(unsigned long long)) == cudaSuccess;
+    ok = ok && cudaMalloc(&c->part_key, slots * sizeof(unsigned long long)) == cudaSuccess;
     ok = ok && cudaMalloc(&c->ticket, 256) == cudaSuccess;
     ok = ok && cudaMalloc(&c->status, 256) == cudaSuccess;
     ok = ok && cudaMalloc(&c->final_stats, (size_t)max_batch * 2 * sizeof(float)) == cudaSuccess;
@@ -220,6 +300,7 @@ int disco_destroy(disco_ctx* c) {
     cudaFree(c->part_topv);
     cudaFree(c->part_topi);
     cudaFree(c->keys);
+    cudaFree(c->part_key);
     cudaFree(c->ticket);
     cudaFree(c->status);
     cudaFree(c->final_stats);
@@ -288,8 +369,41 @@ int disco_draft_step(disco_ctx* c, const void* W_D, const void* h_D, int B, cons
     p.halt = halt;
     p.feats = feats;
     p.probs = probs;
-    rc = run_stream<true>(c, p, clf->H, st);
-    if (rc) return rc;
+    const bool use_umma = umma_possible(c, B) && (c->path == 2 || (c->path == 0 && B >= 2));
+    if (use_umma) {
+        int np = 0;
+        rc = launch_umma<true>(c, W_D, h_D, c->d_draft, B, probs, &np, st);
+        if (rc) return rc;
+        DraftFinalParams f{};
+        f.part_stats = c->part_stats;
+        f.part_topv = c->part_topv;
+        f.part_key = c->part_key;
+        f.B = B;
+        f.NP = np;
+        f.pos = pos;
+        f.n_drafted = n_drafted;
+        f.active = active;
+        f.clf_W1 = clf->W1;
+        f.clf_b1 = clf->b1;
+        f.clf_w2 = clf->w2;
+        f.clf_b2 = clf->b2;
+        f.clf_H = clf->H;
+        f.tau = tau;
+        f.sl_max = sl_max;
+        f.token = token;
+        f.conf = conf;
+        f.halt = halt;
+        f.feats = feats;
+        f.final_stats = c->final_stats;
+        const int nclf = clf->H * (kNFeat + 2) + 1;
+        const size_t fsmem = (size_t)(((nclf + 3) & ~3) + kDraftFinalWarps * 16) * sizeof(float);
+        draft_finalize_kernel<<<(B + kDraftFinalWarps - 1) / kDraftFinalWarps, kDraftFinalWarps * 32, fsmem, st>>>(f);
+        c->launches += 1;
+        if (!cuda_ok(cudaGetLastError(), "draft_finalize_kernel launch")) return DISCO_ERR_CUDA;
+    } else {
+        rc = run_stream<true>(c, p, clf->H, st);
+        if (rc) return rc;
+    }
     if (probs) {
         dim3 grid((unsigned)std::min(64, (c->V + 255) / 256), (unsigned)B);
         normalize_probs_kernel<<<grid, 256, 0, st>>>(probs, c->final_stats, active, c->V);
@@ -323,7 +437,25 @@ int disco_verify_ragged(disco_ctx* c, const void* W_T, const void* H_T, const in
     p.n_accept = n_accept;
     p.bonus = bonus;
     p.target_ids = target_ids;
-    return run_stream<false>(c, p, 0, st);
+    const bool use_umma = umma_possible(c, R) && (c->path == 2 || (c->path == 0 && R >= 2));
+    if (!use_umma) return run_stream<false>(c, p, 0, st);
+    int rc = launch_umma<false>(c, W_T, H_T, c->d_target, R, nullptr, nullptr, st);
+    if (rc) return rc;
+    VerifyFinalParams f{};
+    f.keys = c->keys;
+    f.draft_ids = draft_ids;
+    f.row_off = row_off;
+    f.B = B;
+    f.SL = p.SL;
+    f.R = R;
+    f.n_accept = n_accept;
+    f.bonus = bonus;
+    f.target_ids = target_ids;
+    f.status = c->status;
+    f.ticket = c->ticket + 16;
+    verify_finalize_kernel<<<(B + 3) / 4, 128, 0, st>>>(f);
+    c->launches += 1;
+    return cuda_ok(cudaGetLastError(), "verify_finalize_kernel launch") ? DISCO_OK : DISCO_ERR_CUDA;
 }
 
 int disco_verify(disco_ctx* c, const void* W_T, const void* H_T, const int32_t* draft_ids, int B, int SL,

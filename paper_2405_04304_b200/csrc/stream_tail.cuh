@@ -5,9 +5,10 @@
 //
 //   * one CTA per slab of consecutive vocabulary rows; a producer warp streams the slab through a
 //     ring of shared-memory slots with bulk (TMA-unit) copies signalled on mbarriers;
-//   * consumer warps take one vocabulary row each: 128-bit shared loads, fp32 FMAs, shuffle
-//     reduction; the logit is warp-uniform and goes straight into the warp's online soft-max
-//     state and its top-10 list (draft step) or its running arg-max (verification);
+//   * each ring slot is owned by one consumer warp, which works on up to four vocabulary rows at
+//     once: 128-bit shared loads, fp32 FMAs, shuffle reduction; the logits are warp-uniform and
+//     go straight into the warp's online soft-max state and its top-10 list (draft step) or its
+//     running arg-max (verification);
 //   * per-CTA partials go to scratch; the last CTA to take a ticket merges them and runs the
 //     fused epilogue (features + halt classifier + stopping rule, or prefix match + bonus token).
 //
@@ -111,21 +112,40 @@ __device__ void finalize_draft_row(const TailParams& p, int b, int grid, float* 
     const int c1 = min(grid, c0 + cpw);
     const size_t base = (size_t)b * grid;
 
+    // issue every global load this warp needs before any of the arithmetic
+    const float fpos = static_cast<float>(p.pos[b]);
+    const int n_drafted = p.n_drafted[b];
+    const int ncand = (c1 - c0) * kTopK;
+    const float* tv = p.part_topv + (base + c0) * kTopK;
+    const int* ti = p.part_topi + (base + c0) * kTopK;
+    float4 q0 = make_float4(DISCO_NEG_INF, 0.f, 0.f, 0.f);
+    if (c0 + lane < c1) q0 = __ldcg(reinterpret_cast<const float4*>(p.part_stats) + base + c0 + lane);
+    float v0[5];
+    int id0[5];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+        const int e = j * 32 + lane;
+        const bool ok = e < ncand;
+        v0[j] = ok ? __ldcg(tv + e) : DISCO_NEG_INF;
+        id0[j] = ok ? __ldcg(ti + e) : kNoIndex;
+    }
+    v0[4] = DISCO_NEG_INF;
+    id0[4] = kNoIndex;
+
     // stage A: this warp reduces its share of the CTAs
     SoftmaxState st;
     st.init();
-    for (int c = c0 + lane; c < c1; c += 32) {
+    st.merge(q0.x, q0.y, q0.z);
+    for (int c = c0 + lane + 32; c < c1; c += 32) {
         const float4 q = __ldcg(reinterpret_cast<const float4*>(p.part_stats) + base + c);
         st.merge(q.x, q.y, q.z);
     }
     warp_merge_softmax(st);
 
-    float run_v = DISCO_NEG_INF;
-    int run_i = kNoIndex;
-    const int ncand = (c1 - c0) * kTopK;
-    const float* tv = p.part_topv + (base + c0) * kTopK;
-    const int* ti = p.part_topi + (base + c0) * kTopK;
-    for (int e0 = 0; e0 < ncand; e0 += 32 * 4) {
+    float run_v;
+    int run_i;
+    warp_select_top10<5>(v0, id0, lane, run_v, run_i);
+    for (int e0 = 32 * 4; e0 < ncand; e0 += 32 * 4) {
         float v[5];
         int id[5];
 #pragma unroll
@@ -177,14 +197,13 @@ __device__ void finalize_draft_row(const TailParams& p, int b, int grid, float* 
         const float inv_Z = 1.f / g.Z;
         const float prob = (lane < kTopK && top_i != kNoIndex) ? expf(top_v - g.m) * inv_Z : 0.f;
         const float ent = logf(g.Z) - g.S * inv_Z;
-        const float fpos = static_cast<float>(p.pos[b]);
         const float x = lane < kTopK ? prob : (lane == kTopK ? ent : (lane == kTopK + 1 ? fpos : 0.f));
         const float C = warp_halt_classifier(x, feat_s, clf_s, p.clf_H, lane);
         const int tok = __shfl_sync(kFullMask, top_i, 0);
         if (lane == 0) {
             p.token[b] = tok;
             p.conf[b] = C;
-            p.halt[b] = ((C < p.tau) || (p.n_drafted[b] >= p.sl_max)) ? 1 : 0;
+            p.halt[b] = ((C < p.tau) || (n_drafted >= p.sl_max)) ? 1 : 0;
             p.final_stats[2 * b] = g.m;
             p.final_stats[2 * b + 1] = g.Z;
         }
@@ -246,7 +265,7 @@ __device__ __forceinline__ void verify_one_sequence(const unsigned long long* ke
 // ---------------------------------------------------------------------------------------------
 // the streaming kernel
 // ---------------------------------------------------------------------------------------------
-template <int RT, bool DRAFT, int NW>
+template <int RT, bool DRAFT, int NW, int KC>
 __global__ void __launch_bounds__((NW + 1) * 32, 1) stream_tail_kernel(const __grid_constant__ TailParams p) {
     extern __shared__ __align__(128) uint8_t smem_raw[];
     constexpr int BAR_THREADS = NW * 32;
@@ -284,15 +303,18 @@ __global__ void __launch_bounds__((NW + 1) * 32, 1) stream_tail_kernel(const __g
         if (lane == 0) {
             const int total = nchunks * nslots;
             const uint16_t* slab = p.W + (size_t)v0 * p.d;
+            int st = 0, round = 0, slot = 0;
             for (int fill = 0; fill < total; ++fill) {
-                const int s = fill % p.stages;
-                const int it = fill / p.stages;
-                if (it > 0) mbar_wait(&empty[s], (it - 1) & 1, p.status);
-                const int slot = fill % nslots;
+                if (round > 0) mbar_wait(&empty[st], (round - 1) & 1, p.status);
                 const int r0 = slot * p.rps;
                 const uint32_t bytes = (uint32_t)min(p.rps, nrows - r0) * row_bytes;
-                mbar_arrive_expect_tx(&full[s], bytes);
-                bulk_g2s(ring + (size_t)s * p.slot_bytes, slab + (size_t)r0 * p.d, bytes, &full[s]);
+                mbar_arrive_expect_tx(&full[st], bytes);
+                bulk_g2s(ring + (size_t)st * p.slot_bytes, slab + (size_t)r0 * p.d, bytes, &full[st]);
+                if (++st == p.stages) {
+                    st = 0;
+                    ++round;
+                }
+                if (++slot == nslots) slot = 0;
             }
         }
         return;
@@ -334,54 +356,102 @@ __global__ void __launch_bounds__((NW + 1) * 32, 1) stream_tail_kernel(const __g
             best_i[r] = kNoIndex;
         }
 
+        // With one hidden row and a narrow head the warp keeps its share of h in registers.
+        float hreg[KC > 0 ? KC : 1][8];
+        if (KC > 0) {
+#pragma unroll
+            for (int k = 0; k < (KC > 0 ? KC : 1); ++k) {
+                const int c = lane + 32 * k;
+                uint4 q = make_uint4(0, 0, 0, 0);
+                if (c < n16) q = reinterpret_cast<const uint4*>(htile)[c];
+                unpack_bf16x8(q, hreg[k]);
+            }
+        }
+
         // Each ring slot belongs to one warp (slot s -> warp s % NW), so a warp meets every phase
         // of the barriers it waits on, in order: parity waits can never alias an older phase.
-        const int f_begin = chunk * nslots;
-        for (int f = f_begin; f < f_begin + nslots; ++f) {
-            const int s = f % p.stages;
-            if ((s % NW) != warp) continue;
-            mbar_wait(&full[s], (f / p.stages) & 1, p.status);
-            const int r0 = (f - f_begin) * p.rps;
-            const int nr = min(p.rps, nrows - r0);
-            for (int j = 0; j < nr; ++j) {
-                const uint4* wrow = reinterpret_cast<const uint4*>(ring + (size_t)s * p.slot_bytes +
-                                                                  (size_t)j * row_bytes);
-                float acc[RT];
+        // Fill f of the stream lands in slot f % stages during round f / stages.
+        constexpr int G = 4 / RT;  // vocabulary rows a warp works on at once
+        const int f_begin = chunk * nslots, f_end = f_begin + nslots;
+        const int round_end = (f_end + p.stages - 1) / p.stages;
+        for (int round = f_begin / p.stages; round < round_end; ++round) {
+            for (int s = warp; s < p.stages; s += NW) {
+                const int f = round * p.stages + s;
+                if (f < f_begin || f >= f_end) continue;
+                mbar_wait(&full[s], round & 1, p.status);
+                const int r0 = (f - f_begin) * p.rps;
+                const int nr = min(p.rps, nrows - r0);
+                const uint8_t* slot_base = ring + (size_t)s * p.slot_bytes;
+                for (int j0 = 0; j0 < nr; j0 += G) {
+                    const uint4* wrow[G];
 #pragma unroll
-                for (int r = 0; r < RT; ++r) acc[r] = 0.f;
-#pragma unroll 4
-                for (int c = lane; c < n16; c += 32) {
-                    float wf[8];
-                    unpack_bf16x8(wrow[c], wf);
+                    for (int g = 0; g < G; ++g)
+                        wrow[g] = reinterpret_cast<const uint4*>(slot_base + (size_t)min(j0 + g, nr - 1) * row_bytes);
+                    float acc[G][RT];
 #pragma unroll
-                    for (int r = 0; r < RT; ++r) {
-                        float hf[8];
-                        unpack_bf16x8(reinterpret_cast<const uint4*>(htile + (size_t)r * row_bytes)[c], hf);
+                    for (int g = 0; g < G; ++g)
 #pragma unroll
-                        for (int k = 0; k < 8; ++k) acc[r] = fmaf(wf[k], hf[k], acc[r]);
-                    }
-                }
-                const int v = v0 + r0 + j;
+                        for (int r = 0; r < RT; ++r) acc[g][r] = 0.f;
+                    if (KC > 0) {
 #pragma unroll
-                for (int r = 0; r < RT; ++r) {
+                        for (int k = 0; k < (KC > 0 ? KC : 1); ++k) {
+                            const int c = min(lane + 32 * k, n16 - 1);  // past the row: h is zero there
 #pragma unroll
-                    for (int off = 16; off > 0; off >>= 1) acc[r] += __shfl_xor_sync(kFullMask, acc[r], off);
-                    const float z = __fadd_rn(acc[r], 0.f);  // folds -0 into +0
-                    if (DRAFT) {
-                        st[r].push(z);
-                        top[r].offer(z, v, lane);
-                        if (p.probs && lane == 0 && chunk * RT + r < p.R)
-                            p.probs[(size_t)(chunk * RT + r) * p.V + v] = z;
+                            for (int g = 0; g < G; ++g) {
+                                float wf[8];
+                                unpack_bf16x8(wrow[g][c], wf);
+#pragma unroll
+                                for (int e = 0; e < 8; ++e) acc[g][0] = fmaf(wf[e], hreg[k][e], acc[g][0]);
+                            }
+                        }
                     } else {
-                        if (z > best_v[r]) {
-                            best_v[r] = z;
-                            best_i[r] = v;
+#pragma unroll 2
+                        for (int c = lane; c < n16; c += 32) {
+                            float hf[RT][8];
+#pragma unroll
+                            for (int r = 0; r < RT; ++r)
+                                unpack_bf16x8(reinterpret_cast<const uint4*>(htile + (size_t)r * row_bytes)[c], hf[r]);
+#pragma unroll
+                            for (int g = 0; g < G; ++g) {
+                                float wf[8];
+                                unpack_bf16x8(wrow[g][c], wf);
+#pragma unroll
+                                for (int r = 0; r < RT; ++r)
+#pragma unroll
+                                    for (int e = 0; e < 8; ++e) acc[g][r] = fmaf(wf[e], hf[r][e], acc[g][r]);
+                            }
+                        }
+                    }
+#pragma unroll
+                    for (int off = 16; off > 0; off >>= 1)
+#pragma unroll
+                        for (int g = 0; g < G; ++g)
+#pragma unroll
+                            for (int r = 0; r < RT; ++r) acc[g][r] += __shfl_xor_sync(kFullMask, acc[g][r], off);
+#pragma unroll
+                    for (int g = 0; g < G; ++g) {
+                        if (j0 + g >= nr) break;
+                        const int v = v0 + r0 + j0 + g;
+#pragma unroll
+                        for (int r = 0; r < RT; ++r) {
+                            const float z = __fadd_rn(acc[g][r], 0.f);  // folds -0 into +0
+                            if (DRAFT) {
+                                st[r].push(z);
+                                top[r].offer(z, v, lane);
+                                if (p.probs && lane == 0 && chunk * RT + r < p.R)
+                                    p.probs[(size_t)(chunk * RT + r) * p.V + v] = z;
+                            } else {
+                                if (z > best_v[r]) {
+                                    best_v[r] = z;
+                                    best_i[r] = v;
+                                }
+                            }
                         }
                     }
                 }
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&empty[s]);  // the slot may be refilled
             }
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&empty[s]);  // the slot may be refilled
         }
 
         // ---- merge the NW warps of this CTA, publish the CTA's partial for each hidden row ----

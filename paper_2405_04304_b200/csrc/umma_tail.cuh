@@ -1,0 +1,490 @@
+// Tensor-core (tcgen05) kernel for the logit tails when several hidden rows share one pass over the
+// LM head: single-sequence verification (SL+1 rows), batched verification, batched draft steps.
+//
+//   D[r, v] = sum_k H[r, k] * W[v, k]      r on the 128 TMEM lanes, v on the TMEM columns
+//
+//   * warp 0   producer: TMA tiles of H (A operand, up to 128 rows x 64 k) and of W (B operand, up to
+//              256 vocabulary rows x 64 k, fetched as 16-row boxes so that a slab can end on any
+//              16-row boundary), 128-byte swizzle, through a ring of shared-memory stages;
+//   * warp 1   issues tcgen05.mma (M = 128, N = rows of the vocabulary tile, K = 16 per instruction),
+//              accumulating in one of two 256-column TMEM buffers; tcgen05.commit frees the stage;
+//   * warps 2+ epilogue: tcgen05.ld 32 columns at a time; every thread owns one hidden row and walks
+//              over the vocabulary columns, so the running arg-max (verification) or the running
+//              soft-max statistics and top-10 values (draft step) live in its registers: no shuffles,
+//              and the logits never leave the chip.  Two warps share each TMEM lane quadrant and
+//              split the columns.
+//
+// A CTA keeps one tile of hidden rows (m_tile) and walks over a contiguous range of vocabulary
+// tiles; CTAs that share a vocabulary tile run side by side, so the LM head crosses HBM once and is
+// shared through L2.  Results leave the CTA as one atomicMax per row (verification) or one partial
+// per row (draft step); small separate kernels finish the job.
+#pragma once
+
+#include <cuda.h>
+
+#include "common.cuh"
+#include "stream_tail.cuh"  // verify_one_sequence, warp_halt_classifier
+
+namespace disco {
+
+constexpr int kUmmaStages = 4;
+constexpr int kUmmaBK = 64;               // k elements per stage (one 128-byte swizzle span)
+constexpr int kUmmaATileBytes = 128 * 128;  // 128 rows x 128 B
+constexpr int kUmmaBTileBytes = 256 * 128;  // 256 rows x 128 B
+constexpr int kUmmaEpiWarps = 8;
+constexpr int kUmmaThreads = (2 + kUmmaEpiWarps) * 32;
+constexpr int kUmmaSmemBytes = kUmmaStages * (kUmmaATileBytes + kUmmaBTileBytes) + 1024 /*align*/ + 256;
+
+struct UmmaParams {
+    int V, d, R;
+    int MT;      // tiles of 128 hidden rows
+    int CN;      // CTAs per m_tile (grid = MT * CN)
+    int TPC;     // vocabulary tiles per CTA
+    int G16;     // 16-row groups of the vocabulary: ceil(V / 16)
+    int a_rows;  // rows of the H box (multiple of 8, <= 128)
+    int* status;
+    // verification
+    unsigned long long* keys;  // [R]
+    // draft step
+    float* part_stats;  // [R][CN][4]  (m, Z, S, -)
+    float* part_topv;   // [R][CN][10] top-10 logits, descending
+    unsigned long long* part_key;  // [R][CN] arg-max key
+    float* probs;       // optional [R][V]: raw logits are written here
+};
+
+// ---------------------------------------------------------------------------------------------
+// PTX wrappers
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ void tma_load_2d(void* dst_smem, const CUtensorMap* tmap, int c0, int c1, uint64_t* bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(
+            smem_addr(dst_smem)),
+        "l"(tmap), "r"(c0), "r"(c1), "r"(smem_addr(bar))
+        : "memory");
+}
+__device__ __forceinline__ void prefetch_tensormap(const CUtensorMap* tmap) {
+    asm volatile("prefetch.tensormap [%0];" ::"l"(tmap) : "memory");
+}
+__device__ __forceinline__ void tmem_alloc(uint32_t* dst_smem, uint32_t ncols) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_addr(dst_smem)),
+                 "r"(ncols)
+                 : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish() {
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols) {
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint64_t* bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_addr(bar))
+                 : "memory");
+}
+__device__ __forceinline__ void tc_mma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                            uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(d_tmem),
+        "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+// 32 lanes x 32 consecutive fp32 columns -> 32 registers per thread
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
+    uint32_t r[32];
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+          "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+          "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr)
+        : "memory");
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+    for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+}
+
+// Shared-memory matrix descriptor: K-major tile, 128-byte swizzle, 8-row groups 1024 bytes apart.
+__device__ __forceinline__ uint64_t umma_smem_desc(const void* tile) {
+    uint64_t desc = 0;
+    desc |= static_cast<uint64_t>((smem_addr(tile) & 0x3ffffu) >> 4);  // start address
+    desc |= static_cast<uint64_t>(1) << 16;                            // leading byte offset (unused with swizzle)
+    desc |= static_cast<uint64_t>(1024 >> 4) << 32;                    // stride byte offset
+    desc |= static_cast<uint64_t>(1) << 46;                            // descriptor version
+    desc |= static_cast<uint64_t>(2) << 61;                            // 128-byte swizzle
+    return desc;
+}
+// Instruction descriptor: bf16 x bf16 -> fp32, both operands K-major, M = 128, N = n.
+__device__ __forceinline__ uint32_t umma_idesc(int n) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | (static_cast<uint32_t>(n >> 3) << 17) | ((128u >> 4) << 24);
+}
+
+// Vocabulary tile t of NT covers the 16-row groups [g0, g1).
+__device__ __forceinline__ void tile_groups(int t, int NT, int G16, int& g0, int& g1) {
+    g0 = static_cast<int>(static_cast<long long>(t) * G16 / NT);
+    g1 = static_cast<int>(static_cast<long long>(t + 1) * G16 / NT);
+}
+
+// Ten largest values seen so far, descending, in registers.
+struct RegTop10 {
+    float t[kTopK];
+    __device__ __forceinline__ void init() {
+#pragma unroll
+        for (int k = 0; k < kTopK; ++k) t[k] = DISCO_NEG_INF;
+    }
+    __device__ __forceinline__ void push(float z) {
+        float carry = z;
+#pragma unroll
+        for (int k = 0; k < kTopK; ++k) {
+            const float hi = fmaxf(t[k], carry);
+            carry = fminf(t[k], carry);
+            t[k] = hi;
+        }
+    }
+};
+
+// ---------------------------------------------------------------------------------------------
+// main kernel
+// ---------------------------------------------------------------------------------------------
+template <bool DRAFT>
+__global__ void __launch_bounds__(kUmmaThreads, 1)
+umma_tail_kernel(const __grid_constant__ CUtensorMap tmap_W, const __grid_constant__ CUtensorMap tmap_H,
+                 const UmmaParams p) {
+    extern __shared__ uint8_t smem_dyn[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~uintptr_t(1023));
+    uint8_t* a_tiles = smem;
+    uint8_t* b_tiles = smem + kUmmaStages * kUmmaATileBytes;
+    uint64_t* full = reinterpret_cast<uint64_t*>(b_tiles + kUmmaStages * kUmmaBTileBytes);
+    uint64_t* empty = full + kUmmaStages;
+    uint64_t* tmem_full = empty + kUmmaStages;
+    uint64_t* tmem_empty = tmem_full + 2;
+    uint32_t* tmem_base_s = reinterpret_cast<uint32_t*>(tmem_empty + 2);
+
+    const int warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31;
+    const int m_tile = blockIdx.x % p.MT;
+    const int nslot = blockIdx.x / p.MT;
+    const int NT = p.CN * p.TPC;
+    const int KB = (p.d + kUmmaBK - 1) / kUmmaBK;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kUmmaStages; ++s) {
+            mbar_init(&full[s], 1);
+            mbar_init(&empty[s], 1);
+        }
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(&tmem_full[b], 1);
+            mbar_init(&tmem_empty[b], kUmmaEpiWarps);
+        }
+        fence_mbar_init();
+        prefetch_tensormap(&tmap_W);
+        prefetch_tensormap(&tmap_H);
+    }
+    if (warp == 1) {
+        tmem_alloc(tmem_base_s, 512);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_base_s;
+
+    if (warp == 0) {
+        // ------------------------------ producer ------------------------------
+        if (lane == 0) {
+            int stage = 0, phase = 0;
+            for (int i = 0; i < p.TPC; ++i) {
+                int g0, g1;
+                tile_groups(nslot * p.TPC + i, NT, p.G16, g0, g1);
+                if (g1 <= g0) continue;
+                const uint32_t bytes = (uint32_t)(p.a_rows + (g1 - g0) * 16) * 128u;
+                for (int kb = 0; kb < KB; ++kb) {
+                    mbar_wait(&empty[stage], phase ^ 1, p.status);
+                    mbar_arrive_expect_tx(&full[stage], bytes);
+                    tma_load_2d(a_tiles + stage * kUmmaATileBytes, &tmap_H, kb * kUmmaBK, m_tile * 128, &full[stage]);
+                    uint8_t* b_dst = b_tiles + stage * kUmmaBTileBytes;
+                    for (int g = g0; g < g1; ++g)
+                        tma_load_2d(b_dst + (g - g0) * 2048, &tmap_W, kb * kUmmaBK, g * 16, &full[stage]);
+                    if (++stage == kUmmaStages) {
+                        stage = 0;
+                        phase ^= 1;
+                    }
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------ MMA issuer ------------------------------
+        if (lane == 0) {
+            int stage = 0, phase = 0, it = 0;
+            for (int i = 0; i < p.TPC; ++i) {
+                int g0, g1;
+                tile_groups(nslot * p.TPC + i, NT, p.G16, g0, g1);
+                if (g1 <= g0) continue;
+                const int buf = it & 1;
+                mbar_wait(&tmem_empty[buf], ((it >> 1) & 1) ^ 1, p.status);
+                tc_fence_after();
+                const uint32_t idesc = umma_idesc((g1 - g0) * 16);
+                const uint32_t d_tmem = tmem_base + buf * 256;
+                for (int kb = 0; kb < KB; ++kb) {
+                    mbar_wait(&full[stage], phase, p.status);
+                    tc_fence_after();
+                    const uint64_t a_desc = umma_smem_desc(a_tiles + stage * kUmmaATileBytes);
+                    const uint64_t b_desc = umma_smem_desc(b_tiles + stage * kUmmaBTileBytes);
+#pragma unroll
+                    for (int k = 0; k < kUmmaBK / 16; ++k)  // 16 k-elements = 32 bytes = 2 descriptor units
+                        tc_mma_bf16(d_tmem, a_desc + 2 * k, b_desc + 2 * k, idesc, (kb | k) != 0);
+                    tc_commit(&empty[stage]);
+                    if (++stage == kUmmaStages) {
+                        stage = 0;
+                        phase ^= 1;
+                    }
+                }
+                tc_commit(&tmem_full[buf]);
+                ++it;
+            }
+        }
+    } else {
+        // ------------------------------ epilogue ------------------------------
+        const int ew = warp - 2;            // 0 .. kUmmaEpiWarps-1
+        const int quad = warp & 3;          // TMEM lane quadrant this warp may read
+        const int half = ew >> 2;           // which share of the columns (two warps per quadrant)
+        const int row = m_tile * 128 + quad * 32 + lane;
+        const bool warp_has_rows = (m_tile * 128 + quad * 32) < p.R;
+        const bool valid = row < p.R;
+
+        float best_v = DISCO_NEG_INF;
+        int best_i = kNoIndex;
+        SoftmaxState st;
+        st.init();
+        RegTop10 top;
+        top.init();
+
+        int it = 0;
+        for (int i = 0; i < p.TPC; ++i) {
+            int g0, g1;
+            tile_groups(nslot * p.TPC + i, NT, p.G16, g0, g1);
+            if (g1 <= g0) continue;
+            const int buf = it & 1;
+            mbar_wait(&tmem_full[buf], (it >> 1) & 1, p.status);
+            tc_fence_after();
+            const int v0 = g0 * 16;
+            const int ncols = min((g1 - g0) * 16, p.V - v0);  // columns past V hold zero-filled rows
+            if (warp_has_rows) {
+                const int nchunks = (ncols + 31) >> 5;
+                const int c_lo = (half == 0) ? 0 : (nchunks + 1) / 2;
+                const int c_hi = (half == 0) ? (nchunks + 1) / 2 : nchunks;
+                for (int c = c_lo; c < c_hi; ++c) {
+                    float z[32];
+                    tmem_ld32(tmem_base + buf * 256 + c * 32 + (static_cast<uint32_t>(quad * 32) << 16), z);
+                    const int cbase = c * 32;
+                    if (DRAFT) {
+                        float cmax = DISCO_NEG_INF;
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) {
+                            z[j] = (cbase + j < ncols) ? __fadd_rn(z[j], 0.f) : DISCO_NEG_INF;
+                            cmax = fmaxf(cmax, z[j]);
+                        }
+                        if (cmax > st.m) {  // move the reference maximum first, then add the chunk
+                            if (st.Z > 0.f) {
+                                const float dm = st.m - cmax;
+                                const float e = __expf(dm);
+                                st.S = e * (st.S + dm * st.Z);
+                                st.Z *= e;
+                            }
+                            st.m = cmax;
+                        }
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) {
+                            const float t = z[j] - st.m;       // -inf for masked columns: e = 0
+                            const float e = __expf(t);
+                            st.Z += e;
+                            st.S = (cbase + j < ncols) ? fmaf(e, t, st.S) : st.S;
+                            top.push(z[j]);
+                            if (z[j] > best_v) {
+                                best_v = z[j];
+                                best_i = v0 + cbase + j;
+                            }
+                        }
+                        if (p.probs && valid) {
+#pragma unroll
+                            for (int j = 0; j < 32; ++j)
+                                if (cbase + j < ncols) p.probs[(size_t)row * p.V + v0 + cbase + j] = z[j];
+                        }
+                    } else {
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) {
+                            const float zz = __fadd_rn(z[j], 0.f);
+                            if (cbase + j < ncols && zz > best_v) {
+                                best_v = zz;
+                                best_i = v0 + cbase + j;
+                            }
+                        }
+                    }
+                }
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&tmem_empty[buf]);
+            ++it;
+        }
+
+        // one result per hidden row and CTA
+        if (DRAFT) {
+            if (valid) {
+                const size_t slot = ((size_t)row * p.CN + nslot) * 2 + half;
+                reinterpret_cast<float4*>(p.part_stats)[slot] = make_float4(st.m, st.Z, st.S, 0.f);
+#pragma unroll
+                for (int k = 0; k < kTopK; ++k) p.part_topv[slot * kTopK + k] = top.t[k];
+                p.part_key[slot] = best_i != kNoIndex ? argmax_key(best_v, best_i) : 0ull;
+            }
+        } else {
+            if (valid && best_i != kNoIndex) atomicMax(p.keys + row, argmax_key(best_v, best_i));
+        }
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc(tmem_base, 512);
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// finishing kernels
+// ---------------------------------------------------------------------------------------------
+
+// Verification: one warp per sequence decodes the arg-max keys, matches the prefix and picks the
+// bonus token.  The last CTA to finish clears the keys for the next call.
+struct VerifyFinalParams {
+    unsigned long long* keys;
+    const int32_t* draft_ids;
+    const int32_t* row_off;
+    int B, SL, R;
+    int32_t* n_accept;
+    int32_t* bonus;
+    int32_t* target_ids;
+    int* status;
+    unsigned int* ticket;
+};
+
+// Draft step: one warp per sequence merges the per-CTA partials, forms the features of Eq. 2 and
+// runs the halt classifier and the stopping rule.
+struct DraftFinalParams {
+    const float* part_stats;
+    const float* part_topv;
+    const unsigned long long* part_key;
+    int B, NP;  // partials per sequence
+    const int32_t* pos;
+    const int32_t* n_drafted;
+    const uint8_t* active;
+    const float* clf_W1;
+    const float* clf_b1;
+    const float* clf_w2;
+    const float* clf_b2;
+    int clf_H;
+    float tau;
+    int sl_max;
+    int32_t* token;
+    float* conf;
+    uint8_t* halt;
+    float* feats;
+    float* final_stats;
+};
+
+__global__ void __launch_bounds__(128) verify_finalize_kernel(const VerifyFinalParams p) {
+    __shared__ int s_last;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int b = blockIdx.x * (blockDim.x >> 5) + warp;
+    if (b < p.B)
+        verify_one_sequence(p.keys, p.draft_ids, p.row_off, p.B, p.SL, p.R, b, p.n_accept, p.bonus, p.target_ids,
+                            p.status, lane);
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        __threadfence();
+        s_last = atomicAdd(p.ticket, 1u) == gridDim.x - 1;
+    }
+    __syncthreads();
+    if (!s_last) return;
+    __threadfence();
+    for (int r = threadIdx.x; r < p.R; r += blockDim.x) p.keys[r] = 0ull;  // every reader is done
+    if (threadIdx.x == 0) *p.ticket = 0u;
+}
+
+constexpr int kDraftFinalWarps = 4;
+
+__global__ void __launch_bounds__(kDraftFinalWarps * 32) draft_finalize_kernel(const DraftFinalParams p) {
+    extern __shared__ float clf_s[];  // W1 | b1 | w2 | b2, then 16 feature words per warp
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int Hc = p.clf_H;
+    const int n1 = Hc * kNFeat;
+    const int nclf = n1 + 2 * Hc + 1;
+    for (int i = threadIdx.x; i < nclf; i += blockDim.x)
+        clf_s[i] = i < n1 ? p.clf_W1[i]
+                          : (i < n1 + Hc ? p.clf_b1[i - n1] : (i < n1 + 2 * Hc ? p.clf_w2[i - n1 - Hc] : p.clf_b2[0]));
+    __syncthreads();
+    float* feat_s = clf_s + ((nclf + 3) & ~3) + warp * 16;
+
+    const int b = blockIdx.x * kDraftFinalWarps + warp;
+    if (b >= p.B) return;
+    if (p.active && !p.active[b]) return;
+    const float fpos = static_cast<float>(p.pos[b]);
+    const int n_drafted = p.n_drafted[b];
+    const size_t base = (size_t)b * p.NP;
+
+    SoftmaxState st;
+    st.init();
+    unsigned long long key = 0ull;
+    RegTop10 top;
+    top.init();
+    for (int c = lane; c < p.NP; c += 32) {
+        const float4 q = __ldcg(reinterpret_cast<const float4*>(p.part_stats) + base + c);
+        st.merge(q.x, q.y, q.z);
+        const unsigned long long k2 = __ldcg(p.part_key + base + c);
+        key = k2 > key ? k2 : key;
+        if (q.y > 0.f) {
+            const float* lv = p.part_topv + (base + c) * kTopK;
+#pragma unroll 1
+            for (int k = 0; k < kTopK; ++k) {  // the list is descending: stop at the first value that cannot enter
+                const float v = __ldcg(lv + k);
+                if (!(v > top.t[kTopK - 1])) break;
+                top.push(v);
+            }
+        }
+    }
+    warp_merge_softmax(st);
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) {
+        const unsigned long long k2 = __shfl_xor_sync(kFullMask, key, off);
+        key = k2 > key ? k2 : key;
+        float other[kTopK];
+#pragma unroll
+        for (int k = 0; k < kTopK; ++k) other[k] = __shfl_xor_sync(kFullMask, top.t[k], off);
+#pragma unroll
+        for (int k = 0; k < kTopK; ++k) top.push(other[k]);
+    }
+    // every lane now holds the merged state; lane k < 10 takes the k-th largest logit
+    float mine = DISCO_NEG_INF;
+#pragma unroll
+    for (int k = 0; k < kTopK; ++k) mine = (lane == k) ? top.t[k] : mine;
+    const float inv_Z = 1.f / st.Z;
+    const float prob = (lane < kTopK && mine > DISCO_NEG_INF) ? expf(mine - st.m) * inv_Z : 0.f;
+    const float ent = logf(st.Z) - st.S * inv_Z;
+    const float x = lane < kTopK ? prob : (lane == kTopK ? ent : (lane == kTopK + 1 ? fpos : 0.f));
+    const float C = warp_halt_classifier(x, feat_s, clf_s, Hc, lane);
+    if (lane == 0) {
+        p.token[b] = key_index(key);
+        p.conf[b] = C;
+        p.halt[b] = ((C < p.tau) || (n_drafted >= p.sl_max)) ? 1 : 0;
+        p.final_stats[2 * b] = st.m;
+        p.final_stats[2 * b + 1] = st.Z;
+    }
+    if (p.feats && lane < kNFeat) p.feats[(size_t)b * kNFeat + lane] = x;
+}
+
+}  // namespace disco

@@ -246,3 +246,55 @@ def test_errors_are_codes_not_faults():
     got = gpu_verify(ctx, W, H, np.zeros(4, np.int32), row_off=[0, 4, 6])
     assert np.all(got["n_accept"] >= 0)
     ctx.close()
+
+
+# ---------------------------------------------------------------------------------- both kernel families
+@pytest.mark.parametrize("path", [1, 2])
+@pytest.mark.parametrize("V,d,B", [(50, 16, 1), (1000, 72, 3), (4099, 264, 7), (5000, 768, 64), (3000, 128, 130)])
+def test_draft_step_on_each_kernel_path(oracle, path, V, d, B):
+    if path == 1 and B > 16:
+        pytest.skip("the CUDA-core kernel is only meant for a handful of rows")
+    W = inputs.lm_head(V, d, seed=3 * V + d, std=0.2)
+    h = inputs.hidden(B, d, seed=V + 11 * B)
+    params = make_clf(32, seed=B)
+    pos = (np.arange(B, dtype=np.int32) * 7) % 50 + 1
+    nd = (np.arange(B, dtype=np.int32) % 5) + 1
+    active = None if B < 5 else (np.arange(B) % 3 != 1).astype(np.uint8)
+    ctx = _ctx(V, d, 8, max_batch=B, H=32)
+    ctx.set_kernel_path(path)
+    got = gpu_draft_step(ctx, W.cuda(), h, pos, nd, to_gpu_clf(params), 0.5, 4, active=active,
+                         want_probs=(B <= 7))
+    ref = oracle.draft_step(_bits(W), _bits(h), pos, nd, to_oracle_clf(oracle, params), 0.5, 4, active=active,
+                            want_probs=(B <= 7), nthreads=8)
+    check_draft(got, ref, 0.5, active=active)
+    assert ctx.device_status() == 0
+    ctx.close()
+
+
+@pytest.mark.parametrize("path", [1, 2])
+@pytest.mark.parametrize("V,d,sls", [(7, 8, [0]), (64, 16, [5]), (1000, 136, [10]), (4099, 72, [1, 2, 3, 4, 5, 6]),
+                                     (2000, 5120, [10]), (3000, 128, [16] * 9 + [3, 0, 7]), (600, 64, [9] * 40)])
+def test_verify_on_each_kernel_path(oracle, path, V, d, sls):
+    sl = torch.tensor(sls, dtype=torch.int32)
+    off = inputs.row_offsets(sl).numpy()
+    R, B = int(off[-1]), len(sls)
+    if path == 1 and R > 64:
+        pytest.skip("the CUDA-core kernel is only meant for a handful of rows")
+    W = inputs.lm_head(V, d, seed=V + 2 * d, std=0.3)
+    H = inputs.hidden(R, d, seed=V + 3 * R)
+    free = oracle.verify_ragged(_bits(W), _bits(H), np.zeros(R - B, np.int32), off, nthreads=8)
+    clean = np.concatenate([free.target_ids[off[b]:off[b + 1] - 1] for b in range(B)]).astype(np.int32)
+    draft = inputs.corrupt_ids(torch.from_numpy(clean), 0.2, V, seed=R).numpy()
+    n_b = [oracle.accept_prefix(draft[off[b] - b: off[b + 1] - b - 1], free.target_ids[off[b]:off[b + 1]])
+           for b in range(B)]
+    ref = oracle.VerifyResult(np.array([x[0] for x in n_b], np.int32), np.array([x[1] for x in n_b], np.int32),
+                              free.target_ids, free.gap)
+    ctx = binding.Context(V, 8, d, max_batch=B, max_rows=R)
+    ctx.set_kernel_path(path)
+    got = gpu_verify(ctx, W.cuda(), H, draft, row_off=off)
+    check_verify(got, ref, off, draft)
+    got2 = gpu_verify(ctx, W.cuda(), H, draft, row_off=off)          # scratch is clean for the next call
+    for k in ("n_accept", "bonus", "target_ids"):
+        np.testing.assert_array_equal(got[k], got2[k])
+    assert ctx.device_status() == 0
+    ctx.close()
