@@ -261,4 +261,23 @@ __device__ __forceinline__ void warp_select_top10(float (&v)[E], int (&id)[E], i
     }
 }
 
+// Every lane holds a descending list l[0..9] (values only, -inf = empty).  Lane k < 10 returns the k-th
+// largest of all 320 values; the lists are consumed.  Equal values are interchangeable here.
+__device__ __forceinline__ float warp_select_sorted(float (&l)[kTopK], int lane) {
+    float out = DISCO_NEG_INF;
+#pragma unroll 1
+    for (int r = 0; r < kTopK; ++r) {
+        const uint32_t mine = ordered_bits(l[0]);
+        const uint32_t best = __reduce_max_sync(kFullMask, mine);
+        const unsigned who = __ballot_sync(kFullMask, mine == best);
+        if (lane == r) out = from_ordered_bits(best);
+        if (lane == __ffs(who) - 1) {  // the owner of the winner moves its list up by one
+#pragma unroll
+            for (int k = 0; k + 1 < kTopK; ++k) l[k] = l[k + 1];
+            l[kTopK - 1] = DISCO_NEG_INF;
+        }
+    }
+    return out;
+}
+
 }  // namespace disco

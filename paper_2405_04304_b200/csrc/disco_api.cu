@@ -46,7 +46,7 @@ struct disco_ctx {
     unsigned int* ticket;
     int* status;
     float* final_stats;
-    unsigned long long* part_key;  // tcgen05 draft path: arg-max key per partial
+    void* part_rec;                // tcgen05 draft path: 64-byte partial records
     int part_slots;                // partials per row the buffers can hold
     void* encode_tiled;            // cuTensorMapEncodeTiled, resolved through the runtime
     // device staging for the *_host entry points
@@ -169,19 +169,18 @@ int launch_umma(disco_ctx* c, const void* W, const void* H, int d, int R, float*
     p.R = R;
     p.MT = (R + 127) / 128;
     p.CN = c->sm_count / p.MT;
-    p.G16 = (c->V + 15) / 16;
-    p.TPC = std::max(1, (p.G16 + 16 * p.CN - 1) / (16 * p.CN));
+    p.TPC = std::max(1, (c->V + 256 * p.CN - 1) / (256 * p.CN));
+    p.TR = (c->V + p.CN * p.TPC - 1) / (p.CN * p.TPC);
+    p.TRN = std::max(16, (p.TR + 15) / 16 * 16);
     p.a_rows = p.MT > 1 ? 128 : std::max(8, (R + 7) / 8 * 8);
     p.status = c->status;
     p.keys = c->keys;
-    p.part_stats = c->part_stats;
-    p.part_topv = c->part_topv;
-    p.part_key = c->part_key;
+    p.part_rec = reinterpret_cast<float4*>(c->part_rec);
     p.probs = probs;
-    if (DRAFT && (2 * p.CN > c->part_slots || R > c->part_rows)) return DISCO_ERR_WORKSPACE;
-    if (n_partials) *n_partials = 2 * p.CN;
+    if (DRAFT && (p.CN > c->part_slots || R > c->part_rows)) return DISCO_ERR_WORKSPACE;
+    if (n_partials) *n_partials = p.CN;
     CUtensorMap tmap_W, tmap_H;
-    if (!encode_bf16_2d(c, &tmap_W, W, c->V, d, 16) || !encode_bf16_2d(c, &tmap_H, H, R, d, p.a_rows))
+    if (!encode_bf16_2d(c, &tmap_W, W, c->V, d, p.TRN) || !encode_bf16_2d(c, &tmap_H, H, R, d, p.a_rows))
         return DISCO_ERR_CUDA;
     auto kern = umma_tail_kernel<DRAFT>;
     static int configured_dev = -1;
@@ -274,7 +273,7 @@ int disco_create(disco_ctx** out, int V, int d_draft, int d_target, int max_batc
     ok = ok && cudaMalloc(&c->part_topv, slots * kTopK * sizeof(float)) == cudaSuccess;
     ok = ok && cudaMalloc(&c->part_topi, slots * kTopK * sizeof(int)) == cudaSuccess;
     ok = ok && cudaMalloc(&c->keys, (size_t)max_rows * sizeof(unsigned long long)) == cudaSuccess;
-    ok = ok && cudaMalloc(&c->part_key, slots * sizeof(unsigned long long)) == cudaSuccess;
+    ok = ok && cudaMalloc(&c->part_rec, slots * 64) == cudaSuccess;
     ok = ok && cudaMalloc(&c->ticket, 256) == cudaSuccess;
     ok = ok && cudaMalloc(&c->status, 256) == cudaSuccess;
     ok = ok && cudaMalloc(&c->final_stats, (size_t)max_batch * 2 * sizeof(float)) == cudaSuccess;
@@ -300,7 +299,7 @@ int disco_destroy(disco_ctx* c) {
     cudaFree(c->part_topv);
     cudaFree(c->part_topi);
     cudaFree(c->keys);
-    cudaFree(c->part_key);
+    cudaFree(c->part_rec);
     cudaFree(c->ticket);
     cudaFree(c->status);
     cudaFree(c->final_stats);
@@ -375,9 +374,7 @@ int disco_draft_step(disco_ctx* c, const void* W_D, const void* h_D, int B, cons
         rc = launch_umma<true>(c, W_D, h_D, c->d_draft, B, probs, &np, st);
         if (rc) return rc;
         DraftFinalParams f{};
-        f.part_stats = c->part_stats;
-        f.part_topv = c->part_topv;
-        f.part_key = c->part_key;
+        f.part_rec = reinterpret_cast<const float4*>(c->part_rec);
         f.B = B;
         f.NP = np;
         f.pos = pos;
@@ -395,9 +392,7 @@ int disco_draft_step(disco_ctx* c, const void* W_D, const void* h_D, int B, cons
         f.halt = halt;
         f.feats = feats;
         f.final_stats = c->final_stats;
-        const int nclf = clf->H * (kNFeat + 2) + 1;
-        const size_t fsmem = (size_t)(((nclf + 3) & ~3) + kDraftFinalWarps * 16) * sizeof(float);
-        draft_finalize_kernel<<<(B + kDraftFinalWarps - 1) / kDraftFinalWarps, kDraftFinalWarps * 32, fsmem, st>>>(f);
+        draft_finalize_kernel<<<B, kDraftFinalWarps * 32, 0, st>>>(f);
         c->launches += 1;
         if (!cuda_ok(cudaGetLastError(), "draft_finalize_kernel launch")) return DISCO_ERR_CUDA;
     } else {

@@ -78,16 +78,13 @@ inline size_t stream_tail_smem_bytes(int RT, int NW, int d, int stages, uint32_t
 // fused epilogues run by the last CTA
 // ---------------------------------------------------------------------------------------------
 
-// Classifier and stopping rule (Eq. 2) by one warp.  x (lane < 12) is the feature of that lane;
-// feat_s is 16 words of shared scratch; clf_s holds W1 | b1 | w2 | b2 in shared memory.
-__device__ __forceinline__ float warp_halt_classifier(float x, float* feat_s, const float* clf_s, int Hc,
-                                                      int lane) {
+// Halt classifier of Eq. 2 by one warp: C = sigmoid(w2 . relu(W1 x + b1) + b2).  x (lane < 12) is the
+// feature held by that lane; feat_s is 16 words of shared scratch owned by the warp.
+__device__ __forceinline__ float warp_halt_classifier(float x, float* feat_s, const float* W1, const float* b1,
+                                                      const float* w2, const float* b2p, int Hc, int lane) {
     if (lane < kNFeat) feat_s[lane] = x;
     __syncwarp();
-    const float* W1 = clf_s;
-    const float* b1 = W1 + Hc * kNFeat;
-    const float* w2 = b1 + Hc;
-    const float b2 = w2[Hc];
+    const float b2 = b2p[0];
     float acc = 0.f;
     for (int j = lane; j < Hc; j += 32) {
         float a = b1[j];
@@ -198,7 +195,8 @@ __device__ void finalize_draft_row(const TailParams& p, int b, int grid, float* 
         const float prob = (lane < kTopK && top_i != kNoIndex) ? expf(top_v - g.m) * inv_Z : 0.f;
         const float ent = logf(g.Z) - g.S * inv_Z;
         const float x = lane < kTopK ? prob : (lane == kTopK ? ent : (lane == kTopK + 1 ? fpos : 0.f));
-        const float C = warp_halt_classifier(x, feat_s, clf_s, p.clf_H, lane);
+        const float C = warp_halt_classifier(x, feat_s, clf_s, clf_s + p.clf_H * kNFeat, clf_s + p.clf_H * (kNFeat + 1),
+                                             clf_s + p.clf_H * (kNFeat + 2), p.clf_H, lane);
         const int tok = __shfl_sync(kFullMask, top_i, 0);
         if (lane == 0) {
             p.token[b] = tok;

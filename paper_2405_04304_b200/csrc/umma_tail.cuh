@@ -3,9 +3,9 @@
 //
 //   D[r, v] = sum_k H[r, k] * W[v, k]      r on the 128 TMEM lanes, v on the TMEM columns
 //
-//   * warp 0   producer: TMA tiles of H (A operand, up to 128 rows x 64 k) and of W (B operand, up to
-//              256 vocabulary rows x 64 k, fetched as 16-row boxes so that a slab can end on any
-//              16-row boundary), 128-byte swizzle, through a ring of shared-memory stages;
+//   * warp 0   producer: one TMA box of H (A operand, up to 128 rows x 64 k) and one of W (B operand, up
+//              to 256 vocabulary rows x 64 k) per stage, 128-byte swizzle, through a ring of
+//              shared-memory stages;
 //   * warp 1   issues tcgen05.mma (M = 128, N = rows of the vocabulary tile, K = 16 per instruction),
 //              accumulating in one of two 256-column TMEM buffers; tcgen05.commit frees the stage;
 //   * warps 2+ epilogue: tcgen05.ld 32 columns at a time; every thread owns one hidden row and walks
@@ -33,22 +33,23 @@ constexpr int kUmmaATileBytes = 128 * 128;  // 128 rows x 128 B
 constexpr int kUmmaBTileBytes = 256 * 128;  // 256 rows x 128 B
 constexpr int kUmmaEpiWarps = 8;
 constexpr int kUmmaThreads = (2 + kUmmaEpiWarps) * 32;
-constexpr int kUmmaSmemBytes = kUmmaStages * (kUmmaATileBytes + kUmmaBTileBytes) + 1024 /*align*/ + 256;
+constexpr int kUmmaXchBytes = 128 * 16 * 4;  // one 64-byte record per hidden row of the tile
+constexpr int kUmmaSmemBytes =
+    kUmmaStages * (kUmmaATileBytes + kUmmaBTileBytes) + 1024 /*align*/ + 256 /*barriers*/ + kUmmaXchBytes;
 
 struct UmmaParams {
     int V, d, R;
     int MT;      // tiles of 128 hidden rows
     int CN;      // CTAs per m_tile (grid = MT * CN)
     int TPC;     // vocabulary tiles per CTA
-    int G16;     // 16-row groups of the vocabulary: ceil(V / 16)
+    int TR;      // vocabulary rows per tile; the MMA and the TMA box use TRN = TR rounded up to 16
+    int TRN;
     int a_rows;  // rows of the H box (multiple of 8, <= 128)
     int* status;
     // verification
     unsigned long long* keys;  // [R]
     // draft step
-    float* part_stats;  // [R][CN][4]  (m, Z, S, -)
-    float* part_topv;   // [R][CN][10] top-10 logits, descending
-    unsigned long long* part_key;  // [R][CN] arg-max key
+    float4* part_rec;   // [R][CN] records of 64 bytes: (m, Z, S, -), top-10 logits descending, arg-max key
     float* probs;       // optional [R][V]: raw logits are written here
 };
 
@@ -124,12 +125,8 @@ __device__ __forceinline__ uint32_t umma_idesc(int n) {
     return (1u << 4) | (1u << 7) | (1u << 10) | (static_cast<uint32_t>(n >> 3) << 17) | ((128u >> 4) << 24);
 }
 
-// Vocabulary tile t of NT covers the 16-row groups [g0, g1).
-__device__ __forceinline__ void tile_groups(int t, int NT, int G16, int& g0, int& g1) {
-    g0 = static_cast<int>(static_cast<long long>(t) * G16 / NT);
-    g1 = static_cast<int>(static_cast<long long>(t + 1) * G16 / NT);
-}
-
+// Vocabulary tile t covers rows [t * TR, min(V, (t + 1) * TR)).  The TMA box and the MMA take TRN >= TR
+// rows; the extra rows (the next tile's first rows, or zero fill past V) land in columns the epilogue skips.
 // Ten largest values seen so far, descending, in registers.
 struct RegTop10 {
     float t[kTopK];
@@ -164,12 +161,12 @@ umma_tail_kernel(const __grid_constant__ CUtensorMap tmap_W, const __grid_consta
     uint64_t* tmem_full = empty + kUmmaStages;
     uint64_t* tmem_empty = tmem_full + 2;
     uint32_t* tmem_base_s = reinterpret_cast<uint32_t*>(tmem_empty + 2);
+    float4* xch = reinterpret_cast<float4*>(reinterpret_cast<uint8_t*>(full) + 256);
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
     const int m_tile = blockIdx.x % p.MT;
     const int nslot = blockIdx.x / p.MT;
-    const int NT = p.CN * p.TPC;
     const int KB = (p.d + kUmmaBK - 1) / kUmmaBK;
 
     if (threadIdx.x == 0) {
@@ -198,18 +195,15 @@ umma_tail_kernel(const __grid_constant__ CUtensorMap tmap_W, const __grid_consta
         // ------------------------------ producer ------------------------------
         if (lane == 0) {
             int stage = 0, phase = 0;
+            const uint32_t bytes = (uint32_t)(p.a_rows + p.TRN) * 128u;
             for (int i = 0; i < p.TPC; ++i) {
-                int g0, g1;
-                tile_groups(nslot * p.TPC + i, NT, p.G16, g0, g1);
-                if (g1 <= g0) continue;
-                const uint32_t bytes = (uint32_t)(p.a_rows + (g1 - g0) * 16) * 128u;
+                const int v0 = (nslot * p.TPC + i) * p.TR;
+                if (v0 >= p.V) break;
                 for (int kb = 0; kb < KB; ++kb) {
                     mbar_wait(&empty[stage], phase ^ 1, p.status);
                     mbar_arrive_expect_tx(&full[stage], bytes);
                     tma_load_2d(a_tiles + stage * kUmmaATileBytes, &tmap_H, kb * kUmmaBK, m_tile * 128, &full[stage]);
-                    uint8_t* b_dst = b_tiles + stage * kUmmaBTileBytes;
-                    for (int g = g0; g < g1; ++g)
-                        tma_load_2d(b_dst + (g - g0) * 2048, &tmap_W, kb * kUmmaBK, g * 16, &full[stage]);
+                    tma_load_2d(b_tiles + stage * kUmmaBTileBytes, &tmap_W, kb * kUmmaBK, v0, &full[stage]);
                     if (++stage == kUmmaStages) {
                         stage = 0;
                         phase ^= 1;
@@ -221,14 +215,12 @@ umma_tail_kernel(const __grid_constant__ CUtensorMap tmap_W, const __grid_consta
         // ------------------------------ MMA issuer ------------------------------
         if (lane == 0) {
             int stage = 0, phase = 0, it = 0;
+            const uint32_t idesc = umma_idesc(p.TRN);
             for (int i = 0; i < p.TPC; ++i) {
-                int g0, g1;
-                tile_groups(nslot * p.TPC + i, NT, p.G16, g0, g1);
-                if (g1 <= g0) continue;
+                if ((nslot * p.TPC + i) * p.TR >= p.V) break;
                 const int buf = it & 1;
                 mbar_wait(&tmem_empty[buf], ((it >> 1) & 1) ^ 1, p.status);
                 tc_fence_after();
-                const uint32_t idesc = umma_idesc((g1 - g0) * 16);
                 const uint32_t d_tmem = tmem_base + buf * 256;
                 for (int kb = 0; kb < KB; ++kb) {
                     mbar_wait(&full[stage], phase, p.status);
@@ -266,14 +258,12 @@ umma_tail_kernel(const __grid_constant__ CUtensorMap tmap_W, const __grid_consta
 
         int it = 0;
         for (int i = 0; i < p.TPC; ++i) {
-            int g0, g1;
-            tile_groups(nslot * p.TPC + i, NT, p.G16, g0, g1);
-            if (g1 <= g0) continue;
+            const int v0 = (nslot * p.TPC + i) * p.TR;
+            if (v0 >= p.V) break;
             const int buf = it & 1;
             mbar_wait(&tmem_full[buf], (it >> 1) & 1, p.status);
             tc_fence_after();
-            const int v0 = g0 * 16;
-            const int ncols = min((g1 - g0) * 16, p.V - v0);  // columns past V hold zero-filled rows
+            const int ncols = min(p.TR, p.V - v0);  // further columns belong to the next tile or lie past V
             if (warp_has_rows) {
                 const int nchunks = (ncols + 31) >> 5;
                 const int c_lo = (half == 0) ? 0 : (nchunks + 1) / 2;
@@ -335,12 +325,33 @@ umma_tail_kernel(const __grid_constant__ CUtensorMap tmap_W, const __grid_consta
 
         // one result per hidden row and CTA
         if (DRAFT) {
-            if (valid) {
-                const size_t slot = ((size_t)row * p.CN + nslot) * 2 + half;
-                reinterpret_cast<float4*>(p.part_stats)[slot] = make_float4(st.m, st.Z, st.S, 0.f);
+            // the two warps of a quadrant hold the same rows: the second hands its state to the first
+            unsigned long long key = best_i != kNoIndex ? argmax_key(best_v, best_i) : 0ull;
+            float4* mine = xch + (quad * 32 + lane) * 4;
+            if (half == 1) {
+                mine[0] = make_float4(st.m, st.Z, st.S, 0.f);
+                mine[1] = make_float4(top.t[0], top.t[1], top.t[2], top.t[3]);
+                mine[2] = make_float4(top.t[4], top.t[5], top.t[6], top.t[7]);
+                mine[3] = make_float4(top.t[8], top.t[9], __uint_as_float((uint32_t)(key & 0xffffffffull)),
+                                      __uint_as_float((uint32_t)(key >> 32)));
+            }
+            named_barrier_sync(2, kUmmaEpiWarps * 32);
+            if (half == 0 && valid) {
+                const float4 q = mine[0], a = mine[1], bq = mine[2], cq = mine[3];
+                st.merge(q.x, q.y, q.z);
+                const unsigned long long k2 =
+                    (static_cast<unsigned long long>(__float_as_uint(cq.w)) << 32) | __float_as_uint(cq.z);
+                key = k2 > key ? k2 : key;
+                const float lv[kTopK] = {a.x, a.y, a.z, a.w, bq.x, bq.y, bq.z, bq.w, cq.x, cq.y};
 #pragma unroll
-                for (int k = 0; k < kTopK; ++k) p.part_topv[slot * kTopK + k] = top.t[k];
-                p.part_key[slot] = best_i != kNoIndex ? argmax_key(best_v, best_i) : 0ull;
+                for (int k = 0; k < kTopK; ++k)
+                    if (lv[k] > top.t[kTopK - 1]) top.push(lv[k]);
+                float4* rec = p.part_rec + ((size_t)row * p.CN + nslot) * 4;
+                rec[0] = make_float4(st.m, st.Z, st.S, 0.f);
+                rec[1] = make_float4(top.t[0], top.t[1], top.t[2], top.t[3]);
+                rec[2] = make_float4(top.t[4], top.t[5], top.t[6], top.t[7]);
+                rec[3] = make_float4(top.t[8], top.t[9], __uint_as_float((uint32_t)(key & 0xffffffffull)),
+                                     __uint_as_float((uint32_t)(key >> 32)));
             }
         } else {
             if (valid && best_i != kNoIndex) atomicMax(p.keys + row, argmax_key(best_v, best_i));
@@ -376,10 +387,8 @@ struct VerifyFinalParams {
 // Draft step: one warp per sequence merges the per-CTA partials, forms the features of Eq. 2 and
 // runs the halt classifier and the stopping rule.
 struct DraftFinalParams {
-    const float* part_stats;
-    const float* part_topv;
-    const unsigned long long* part_key;
-    int B, NP;  // partials per sequence
+    const float4* part_rec;
+    int B, NP;  // partial records per sequence
     const int32_t* pos;
     const int32_t* n_drafted;
     const uint8_t* active;
@@ -416,25 +425,16 @@ __global__ void __launch_bounds__(128) verify_finalize_kernel(const VerifyFinalP
     if (threadIdx.x == 0) *p.ticket = 0u;
 }
 
-constexpr int kDraftFinalWarps = 4;
+constexpr int kDraftFinalWarps = 8;
 
+// One CTA per sequence: every lane takes one partial record (more only if there are over 256 of them),
+// the warps reduce to one sorted list each, warp 0 finishes.
 __global__ void __launch_bounds__(kDraftFinalWarps * 32) draft_finalize_kernel(const DraftFinalParams p) {
-    extern __shared__ float clf_s[];  // W1 | b1 | w2 | b2, then 16 feature words per warp
+    __shared__ float4 wres[kDraftFinalWarps][4];
+    __shared__ float feat_s[16];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int Hc = p.clf_H;
-    const int n1 = Hc * kNFeat;
-    const int nclf = n1 + 2 * Hc + 1;
-    for (int i = threadIdx.x; i < nclf; i += blockDim.x)
-        clf_s[i] = i < n1 ? p.clf_W1[i]
-                          : (i < n1 + Hc ? p.clf_b1[i - n1] : (i < n1 + 2 * Hc ? p.clf_w2[i - n1 - Hc] : p.clf_b2[0]));
-    __syncthreads();
-    float* feat_s = clf_s + ((nclf + 3) & ~3) + warp * 16;
-
-    const int b = blockIdx.x * kDraftFinalWarps + warp;
-    if (b >= p.B) return;
+    const int b = blockIdx.x;
     if (p.active && !p.active[b]) return;
-    const float fpos = static_cast<float>(p.pos[b]);
-    const int n_drafted = p.n_drafted[b];
     const size_t base = (size_t)b * p.NP;
 
     SoftmaxState st;
@@ -442,19 +442,22 @@ __global__ void __launch_bounds__(kDraftFinalWarps * 32) draft_finalize_kernel(c
     unsigned long long key = 0ull;
     RegTop10 top;
     top.init();
-    for (int c = lane; c < p.NP; c += 32) {
-        const float4 q = __ldcg(reinterpret_cast<const float4*>(p.part_stats) + base + c);
+    for (int c = threadIdx.x; c < p.NP; c += kDraftFinalWarps * 32) {
+        const float4* rec = p.part_rec + (base + c) * 4;
+        const float4 q = __ldcg(rec), a = __ldcg(rec + 1), bq = __ldcg(rec + 2), cq = __ldcg(rec + 3);
+        if (!(q.y > 0.f)) continue;  // that CTA had no columns
         st.merge(q.x, q.y, q.z);
-        const unsigned long long k2 = __ldcg(p.part_key + base + c);
+        const unsigned long long k2 =
+            (static_cast<unsigned long long>(__float_as_uint(cq.w)) << 32) | __float_as_uint(cq.z);
         key = k2 > key ? k2 : key;
-        if (q.y > 0.f) {
-            const float* lv = p.part_topv + (base + c) * kTopK;
-#pragma unroll 1
-            for (int k = 0; k < kTopK; ++k) {  // the list is descending: stop at the first value that cannot enter
-                const float v = __ldcg(lv + k);
-                if (!(v > top.t[kTopK - 1])) break;
-                top.push(v);
-            }
+        const float lv[kTopK] = {a.x, a.y, a.z, a.w, bq.x, bq.y, bq.z, bq.w, cq.x, cq.y};
+        if (c < kDraftFinalWarps * 32) {
+#pragma unroll
+            for (int k = 0; k < kTopK; ++k) top.t[k] = lv[k];  // first record: already sorted
+        } else {
+#pragma unroll
+            for (int k = 0; k < kTopK; ++k)
+                if (lv[k] > top.t[kTopK - 1]) top.push(lv[k]);
         }
     }
     warp_merge_softmax(st);
@@ -462,25 +465,47 @@ __global__ void __launch_bounds__(kDraftFinalWarps * 32) draft_finalize_kernel(c
     for (int off = 16; off > 0; off >>= 1) {
         const unsigned long long k2 = __shfl_xor_sync(kFullMask, key, off);
         key = k2 > key ? k2 : key;
-        float other[kTopK];
-#pragma unroll
-        for (int k = 0; k < kTopK; ++k) other[k] = __shfl_xor_sync(kFullMask, top.t[k], off);
-#pragma unroll
-        for (int k = 0; k < kTopK; ++k) top.push(other[k]);
     }
-    // every lane now holds the merged state; lane k < 10 takes the k-th largest logit
-    float mine = DISCO_NEG_INF;
+    const float sel = warp_select_sorted(top.t, lane);  // lane k < 10: k-th largest logit of this warp's records
+    float* wr = reinterpret_cast<float*>(&wres[warp][0]);
+    if (lane == 0) {
+        wr[0] = st.m;
+        wr[1] = st.Z;
+        wr[2] = st.S;
+        wr[14] = __uint_as_float((uint32_t)(key & 0xffffffffull));
+        wr[15] = __uint_as_float((uint32_t)(key >> 32));
+    }
+    if (lane < kTopK) wr[4 + lane] = sel;
+    __syncthreads();
+    if (warp != 0) return;
+
+    st.init();
+    key = 0ull;
+    top.init();
+    if (lane < kDraftFinalWarps) {
+        const float* o = reinterpret_cast<const float*>(&wres[lane][0]);
+        st.merge(o[0], o[1], o[2]);
+        key = (static_cast<unsigned long long>(__float_as_uint(o[15])) << 32) | __float_as_uint(o[14]);
 #pragma unroll
-    for (int k = 0; k < kTopK; ++k) mine = (lane == k) ? top.t[k] : mine;
+        for (int k = 0; k < kTopK; ++k) top.t[k] = o[4 + k];
+    }
+    warp_merge_softmax(st);
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) {
+        const unsigned long long k2 = __shfl_xor_sync(kFullMask, key, off);
+        key = k2 > key ? k2 : key;
+    }
+    const float mine = warp_select_sorted(top.t, lane);
     const float inv_Z = 1.f / st.Z;
     const float prob = (lane < kTopK && mine > DISCO_NEG_INF) ? expf(mine - st.m) * inv_Z : 0.f;
     const float ent = logf(st.Z) - st.S * inv_Z;
+    const float fpos = static_cast<float>(p.pos[b]);
     const float x = lane < kTopK ? prob : (lane == kTopK ? ent : (lane == kTopK + 1 ? fpos : 0.f));
-    const float C = warp_halt_classifier(x, feat_s, clf_s, Hc, lane);
+    const float C = warp_halt_classifier(x, feat_s, p.clf_W1, p.clf_b1, p.clf_w2, p.clf_b2, p.clf_H, lane);
     if (lane == 0) {
         p.token[b] = key_index(key);
         p.conf[b] = C;
-        p.halt[b] = ((C < p.tau) || (n_drafted >= p.sl_max)) ? 1 : 0;
+        p.halt[b] = ((C < p.tau) || (p.n_drafted[b] >= p.sl_max)) ? 1 : 0;
         p.final_stats[2 * b] = st.m;
         p.final_stats[2 * b + 1] = st.Z;
     }
