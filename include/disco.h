@@ -47,7 +47,8 @@ enum {
     DISCO_ERR_UNSUPPORTED_SHAPE = -2, /* shape outside what the kernels handle */
     DISCO_ERR_WORKSPACE = -3,         /* batch or row count beyond what the context was created for */
     DISCO_ERR_CUDA = -4,              /* a CUDA runtime call failed */
-    DISCO_ERR_TIMEOUT = -5            /* a bounded device-side wait ran out (device status word only) */
+    DISCO_ERR_TIMEOUT = -5,           /* a bounded device-side wait ran out (device status word only) */
+    DISCO_ERR_STATIC_LIMIT = -6       /* size beyond the fixed scratch of disco_draft_step_static */
 };
 
 typedef struct disco_ctx disco_ctx;
@@ -164,6 +165,38 @@ int disco_verify_ragged_host(disco_ctx* ctx, const void* W_T /*device*/, const v
                              const int32_t* draft_ids_host, const int32_t* row_off_host, int B, int R,
                              int32_t* n_accept_host, int32_t* bonus_host, int32_t* target_ids_host,
                              void* stream);
+
+/*
+ * Draft step without any allocation.  (The paper has no counterpart: this is a packaging variant of
+ * disco_draft_step, not another operation.)
+ *
+ * Who needs it: hosts that must not allocate device memory - a serving process whose GPU memory is
+ * owned and capped by another component that hands this library no allocator, or a decode loop that
+ * cannot take the device-wide synchronisation a cudaMalloc may bring.  disco_create allocates its
+ * scratch with cudaMalloc, so those hosts cannot have a context.  This entry point needs none: the
+ * scratch for the cross-block reduction lives in a fixed array inside the library image
+ * (about 385 KB of device memory on every GPU that loads the library, held until the process exits),
+ * and the call itself uses no cudaMalloc, cudaFree or allocating library routine.
+ *
+ * Arguments and results are those of disco_draft_step (same layouts, device pointers owned by the
+ * caller; there is no probs output), with the LM-head shape passed by value since there is no context.
+ * Limits, checked before anything is enqueued: B <= DISCO_STATIC_MAX_BATCH and at most
+ * DISCO_STATIC_MAX_GRID vocabulary slabs (V up to about two million rows); beyond them the call
+ * returns DISCO_ERR_STATIC_LIMIT and does nothing.
+ *
+ * The first call on each device resolves the array's device address and raises the kernel's
+ * shared-memory limit (with that device current); make that first call before any stream capture.
+ * All calls on a device share the one array: it keeps the previous call's contents (the call clears
+ * the words that must start at zero), and two calls that overlap on the GPU - different streams, or a
+ * context-free call racing another - corrupt each other's results.  Issue them on one stream, or
+ * otherwise one after the other.  Kernel-detected conditions are not reported by this entry point.
+ */
+#define DISCO_STATIC_MAX_BATCH 4
+#define DISCO_STATIC_MAX_GRID 1024
+int disco_draft_step_static(int V, int d_draft, const void* W_D, const void* h_D, int B,
+                            const int32_t* pos, const int32_t* n_drafted, const uint8_t* active,
+                            const disco_clf* clf, float tau, int sl_max,
+                            int32_t* token, float* conf, uint8_t* halt, float* feats, void* stream);
 
 #ifdef __cplusplus
 }

@@ -23,11 +23,13 @@ ERR_UNSUPPORTED_SHAPE = -2
 ERR_WORKSPACE = -3
 ERR_CUDA = -4
 ERR_TIMEOUT = -5
+ERR_STATIC_LIMIT = -6
+STATIC_MAX_BATCH = 4
 
 EXPORTS = [
     "disco_create", "disco_destroy", "disco_strerror", "disco_last_device_status", "disco_launch_count",
     "disco_set_kernel_path", "disco_draft_step", "disco_verify", "disco_verify_ragged",
-    "disco_draft_step_host", "disco_verify_ragged_host",
+    "disco_draft_step_host", "disco_verify_ragged_host", "disco_draft_step_static",
 ]
 
 
@@ -69,6 +71,8 @@ def load() -> ctypes.CDLL:
     lib.disco_draft_step_host.argtypes = [vp, vp, vp, ci, vp, vp, vp, ctypes.POINTER(_Clf), cf, ci,
                                           vp, vp, vp, vp, vp]
     lib.disco_verify_ragged_host.argtypes = [vp, vp, vp, vp, vp, ci, ci, vp, vp, vp, vp]
+    lib.disco_draft_step_static.argtypes = [ci, ci, vp, vp, ci, vp, vp, vp, ctypes.POINTER(_Clf), cf, ci,
+                                            vp, vp, vp, vp, vp]
     _lib = lib
     return lib
 
@@ -106,6 +110,25 @@ class Classifier:
         if tuple(W1.shape) != (self.H, NFEAT) or b1.numel() != self.H or w2.numel() != self.H or b2.numel() != 1:
             raise ValueError("classifier shapes must be [H,12], [H], [H], [1]")
         self._c = _Clf(self.W1.data_ptr(), self.b1.data_ptr(), self.w2.data_ptr(), self.b2.data_ptr(), self.H)
+
+
+def draft_step_static(W_D, h_D, pos, n_drafted, clf: "Classifier", tau: float, sl_max: int, token, conf, halt,
+                      active=None, feats=None, stream=None) -> None:
+    """disco_draft_step_static: the draft step for hosts that may not allocate device memory.
+
+    Needs no Context (creating one calls cudaMalloc).  The cross-block scratch is a fixed array inside
+    libdisco.so, shared by every call on the device, so calls must not overlap on the GPU.  At most
+    STATIC_MAX_BATCH sequences; larger requests raise DiscoError(ERR_STATIC_LIMIT).  The first call on a
+    device also does the one-time set-up and should come before any stream capture."""
+    V, d = int(W_D.shape[0]), int(W_D.shape[1])
+    B = int(h_D.shape[0])
+    rc = load().disco_draft_step_static(
+        V, d, _ptr(W_D, torch.bfloat16), _ptr(h_D, torch.bfloat16), B, _ptr(pos, torch.int32),
+        _ptr(n_drafted, torch.int32), _ptr(active, torch.uint8), ctypes.byref(clf._c), float(tau), int(sl_max),
+        _ptr(token, torch.int32), _ptr(conf, torch.float32), _ptr(halt, torch.uint8), _ptr(feats, torch.float32),
+        _stream(stream))
+    if rc != OK:
+        raise DiscoError(rc, "disco_draft_step_static")
 
 
 class Context:

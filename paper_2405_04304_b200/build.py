@@ -9,7 +9,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 _ROOT = os.path.dirname(_HERE)
 CSRC = os.path.join(_HERE, "csrc")
 LIB = os.path.join(_HERE, "libdisco.so")
-SOURCES = ["disco_api.cu"]
+SOURCES = ["disco_api.cu", "disco_static.cu"]
 
 
 def _newest_source_mtime() -> float:

@@ -224,6 +224,7 @@ const char* disco_strerror(int code) {
         case DISCO_ERR_WORKSPACE: return "batch, rows or classifier width beyond what the context was created for";
         case DISCO_ERR_CUDA: return "a CUDA runtime call failed";
         case DISCO_ERR_TIMEOUT: return "a bounded device-side wait ran out";
+        case DISCO_ERR_STATIC_LIMIT: return "size beyond the fixed scratch of the allocation-free entry point";
         default: return "unknown disco status";
     }
 }
