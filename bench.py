@@ -34,12 +34,13 @@ L2_BYTES = 126 * 1024 * 1024
 
 
 def measured_peaks():
+    """(HBM GB/s, sustained bf16 TFLOP/s, 'measured' | 'fallback')."""
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
         with open(path) as f:
             j = json.load(f)
-        return float(j["hbm_gbs"]), "measured"
-    return 6650.0, "fallback"
+        return float(j["hbm_gbs"]), float(j.get("bf16_tflops_sustained", 1400.0)), "measured"
+    return 6650.0, 1400.0, "fallback"
 
 
 # ------------------------------------------------------------------------------------------ clocks
@@ -162,24 +163,13 @@ def pack_iteration(data: Data, it: int, sl: np.ndarray):
 
 
 # ------------------------------------------------------------------------------------------ our arm
-def run_ours(args, rank: int, world: int):
-    from paper_2405_04304_b200 import binding, build
-    build.build()
-    dev_index = int(os.environ.get("LOCAL_RANK", 0))
-    torch.cuda.set_device(dev_index)
-    device = f"cuda:{dev_index}"
-    wl = inputs.WORKLOADS[args.workload]
-    K, Wm = args.steps, args.warmup
-    T = Wm + K
-    data = Data(wl, T, wl.seed + 1000 * rank, device)
-    B, S = wl.B, wl.sl_max
-    max_rows = B * (S + 1)
-    ctx = binding.Context(wl.V, wl.d_D, wl.d_T, max_batch=B, max_rows=max_rows, clf_hidden=wl.H)
-    clf = binding.Classifier(*(t.to(device) for t in data.clf_params))
-    stream = torch.cuda.Stream()
-    hbm_peak, peak_kind = measured_peaks()
+def device_pass(ctx, data: Data, clf, wl, tau: float, Wm: int, K: int, stream, world: int, device, sampler=None):
+    """Closed loop once (discovery + warm-up), then the same launches captured in CUDA graphs and timed.
 
-    # ---------------- discovery: the closed loop, host reads the halt flags (also the warm-up) ---------
+    Returns the time of the K timed iterations, the times of graphs holding only their draft-step or
+    only their verification launches, and the closed-loop trace."""
+    B, S = wl.B, wl.sl_max
+    T = Wm + K
     token = torch.zeros((T, S, B), dtype=torch.int32, device=device)
     conf = torch.zeros((T, S, B), dtype=torch.float32, device=device)
     halt = torch.zeros((T, S, B), dtype=torch.uint8, device=device)
@@ -193,6 +183,7 @@ def run_ours(args, rank: int, world: int):
     emitted = np.zeros(B, dtype=np.int64)
     packed = []
     rot = 0
+    # ---------------- discovery: the closed loop, the host reads the halt flags ----------------
     with torch.cuda.stream(stream):
         for it in range(T):
             d = data.idx(it)
@@ -203,7 +194,7 @@ def run_ours(args, rank: int, world: int):
                 act_all[it, j] = torch.from_numpy(active)
                 pos_d = pos_all[it, j].to(device, non_blocking=False)
                 act_d = act_all[it, j].to(device)
-                ctx.draft_step(data.W_D[rot % data.n_rot], data.h_D[d, j], pos_d, nd_all[j], clf, wl.tau, S,
+                ctx.draft_step(data.W_D[rot % data.n_rot], data.h_D[d, j], pos_d, nd_all[j], clf, tau, S,
                                token[it, j], conf[it, j], halt[it, j], active=act_d, stream=stream)
                 rot += 1
                 stream.synchronize()
@@ -240,7 +231,7 @@ def run_ours(args, rank: int, world: int):
             d = data.idx(it)
             if which in ("all", "draft"):
                 for j in range(int(steps_all[it])):
-                    ctx.draft_step(data.W_D[r % data.n_rot], data.h_D[d, j], pos_dev[it, j], nd_all[j], clf, wl.tau,
+                    ctx.draft_step(data.W_D[r % data.n_rot], data.h_D[d, j], pos_dev[it, j], nd_all[j], clf, tau,
                                    S, token[it, j], conf[it, j], halt[it, j], active=act_dev[it, j])
                     r += 1
             if which in ("all", "verify"):
@@ -259,7 +250,7 @@ def run_ours(args, rank: int, world: int):
         launches[which] = ctx.launch_count() - c0
         graphs[which] = g
 
-    def time_graph(g, sampler=None):
+    def time_graph(g, smp=None):
         with torch.cuda.stream(stream):
             g.replay()                               # untimed replay (graph upload, caches, clocks)
             stream.synchronize()
@@ -267,20 +258,19 @@ def run_ours(args, rank: int, world: int):
                 torch.distributed.barrier()
             torch.cuda.synchronize()
             e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            if sampler is not None:
-                sampler.__enter__()
+            if smp is not None:
+                smp.__enter__()
             e0.record(stream)
             g.replay()
             e1.record(stream)
             stream.synchronize()
             torch.cuda.synchronize()
-            if sampler is not None:
-                sampler.__exit__()
+            if smp is not None:
+                smp.__exit__()
             if world > 1:
                 torch.distributed.barrier()
         return e0.elapsed_time(e1) * 1e-3
 
-    sampler = ClockSampler(dev_index)
     t_all = time_graph(graphs["all"], sampler)
     # results of the replay must be those of the closed loop
     same = (torch.equal(token[Wm:], ref_token[Wm:]) and torch.equal(halt[Wm:], ref_halt[Wm:]) and
@@ -289,25 +279,72 @@ def run_ours(args, rank: int, world: int):
         raise RuntimeError("graph replay did not reproduce the closed-loop results")
     t_draft = time_graph(graphs["draft"])
     t_verify = time_graph(graphs["verify"])
-
+    del graphs
     n_draft = int(steps_all[Wm:].sum())
     rows_total = int(sum(packed[it][3] for it in timed))
-    draft_bytes = n_draft * (wl.V * wl.d_D * 2 + B * wl.d_D * 2)
-    verify_bytes = K * wl.V * wl.d_T * 2 + rows_total * wl.d_T * 2
-    roof_verify = {"kernel": "verification tail", "bound": "hbm", "achieved": verify_bytes / t_verify / 1e9,
+    return {"t_all": t_all, "t_draft": t_draft, "t_verify": t_verify, "n_draft": n_draft, "rows_total": rows_total,
+            "sl_all": sl_all, "n_acc": ref_nacc.cpu().numpy(), "launches": launches["all"]}
+
+
+def rooflines(wl, K: int, res: dict, hbm_peak: float, tensor_peak: float, peak_kind: str):
+    """Achieved algorithmic GB/s (or, beyond the machine balance, TFLOP/s) of the two kernels against the
+    measured peaks.  Returns (dominant kernel, other kernel)."""
+    draft_bytes = res["n_draft"] * (wl.V * wl.d_D * 2 + wl.B * wl.d_D * 2)
+    verify_bytes = K * wl.V * wl.d_T * 2 + res["rows_total"] * wl.d_T * 2
+    verify_flops = 2.0 * res["rows_total"] * wl.V * wl.d_T
+    roof_verify = {"kernel": "verification tail", "bound": "hbm", "achieved": verify_bytes / res["t_verify"] / 1e9,
                    "peak": hbm_peak, "peak_kind": peak_kind, "unit": "GB/s", "launches": K,
-                   "avg_launch_us": t_verify / K * 1e6, "traffic": None}
-    roof_draft = {"kernel": "draft-step tail", "bound": "hbm", "achieved": draft_bytes / t_draft / 1e9,
-                  "peak": hbm_peak, "peak_kind": peak_kind, "unit": "GB/s", "launches": n_draft,
-                  "avg_launch_us": t_draft / max(n_draft, 1) * 1e6, "traffic": None}
+                   "avg_launch_us": res["t_verify"] / K * 1e6, "traffic": None,
+                   "tensor_tflops": verify_flops / res["t_verify"] / 1e12}
+    roof_draft = {"kernel": "draft-step tail", "bound": "hbm", "achieved": draft_bytes / res["t_draft"] / 1e9,
+                  "peak": hbm_peak, "peak_kind": peak_kind, "unit": "GB/s", "launches": res["n_draft"],
+                  "avg_launch_us": res["t_draft"] / max(res["n_draft"], 1) * 1e6, "traffic": None}
     for r in (roof_verify, roof_draft):
         r["frac"] = r["achieved"] / r["peak"]
         r["frac_of_nominal_8TBs"] = r["achieved"] / 8000.0
-    dominant, other = (roof_verify, roof_draft) if t_verify >= t_draft else (roof_draft, roof_verify)
+    if res["rows_total"] / K > tensor_peak * 1e12 / (hbm_peak * 1e9):   # rows per call beyond the machine balance
+        roof_verify.update({"bound": "tensor", "hbm_gbs": roof_verify["achieved"],
+                            "achieved": roof_verify["tensor_tflops"], "peak": tensor_peak, "unit": "TFLOP/s",
+                            "frac": roof_verify["tensor_tflops"] / tensor_peak})
+        roof_verify.pop("frac_of_nominal_8TBs")
+    return (roof_verify, roof_draft) if res["t_verify"] >= res["t_draft"] else (roof_draft, roof_verify)
+
+
+def run_ours(args, rank: int, world: int):
+    from paper_2405_04304_b200 import binding, build
+    build.build()
+    dev_index = int(os.environ.get("LOCAL_RANK", 0))
+    torch.cuda.set_device(dev_index)
+    device = f"cuda:{dev_index}"
+    wl = inputs.WORKLOADS[args.workload]
+    K, Wm = args.steps, args.warmup
+    T = Wm + K
+    data = Data(wl, T, wl.seed + 1000 * rank, device)
+    B, S = wl.B, wl.sl_max
+    max_rows = B * (S + 1)
+    ctx = binding.Context(wl.V, wl.d_D, wl.d_T, max_batch=B, max_rows=max_rows, clf_hidden=wl.H)
+    clf = binding.Classifier(*(t.to(device) for t in data.clf_params))
+    stream = torch.cuda.Stream()
+    hbm_peak, tensor_peak, peak_kind = measured_peaks()
+
+    sampler = ClockSampler(dev_index)
+    res = device_pass(ctx, data, clf, wl, wl.tau, Wm, K, stream, world, device, sampler)
+    dominant, other = rooflines(wl, K, res, hbm_peak, tensor_peak, peak_kind)
+    t_all = res["t_all"]
+
+    # the same workload with the classifier overruled: tau = 0 never halts before SL_max (static SL)
+    static = None
+    if data.forced_sl is None and not args.no_static:
+        Ks = min(K, 256)
+        rs = device_pass(ctx, data, clf, wl, 0.0, Wm, Ks, stream, world, device)
+        sd, so = rooflines(wl, Ks, rs, hbm_peak, tensor_peak, peak_kind)
+        static = {"value": Ks * world / rs["t_all"], "unit": UNIT, "steps": Ks,
+                  "mean_sl": float(rs["sl_all"][Wm:].mean()), "ms_per_step": rs["t_all"] / Ks * 1e3,
+                  "roofline": sd, "roofline_other_kernel": so}
 
     # ---------------- end to end: host buffers through the *_host entry points, closed loop ----------
     e2e = run_e2e(ctx, data, clf, wl, Wm, K, stream, world)
-    e2e["matches"] = all(np.array_equal(sl, sl_all[it]) and np.array_equal(na, ref_nacc[it].cpu().numpy())
+    e2e["matches"] = all(np.array_equal(sl, res["sl_all"][it]) and np.array_equal(na, res["n_acc"][it])
                          for it, (sl, na) in enumerate(e2e["trace"]))
 
     if world > 1:
@@ -321,16 +358,18 @@ def run_ours(args, rank: int, world: int):
         "dtype": "bf16 inputs, fp32 accumulate", "data": "synthetic (seeded Gaussian LM heads and hidden states)",
         "config": {"workload": wl.name, "V": wl.V, "d_draft": wl.d_D, "d_target": wl.d_T, "batch": B,
                    "sl_max": S, "tau": wl.tau, "clf_hidden": wl.H, "p_corrupt": wl.p_corrupt,
-                   "sl_source": wl.sl_mode, "mean_sl": float(sl_all[Wm:].mean()),
-                   "mean_accepted": float(ref_nacc[Wm:].float().mean()),
-                   "draft_steps_per_iteration": n_draft / K, "replicas": world,
+                   "sl_source": wl.sl_mode, "mean_sl": float(res["sl_all"][Wm:].mean()),
+                   "mean_accepted": float(res["n_acc"][Wm:].mean()),
+                   "draft_steps_per_iteration": res["n_draft"] / K, "replicas": world,
                    "l2": f"draft LM head rotates through {data.n_rot} copies (> 2x L2); the target LM head alone "
                          "exceeds L2", "launch": "CUDA graph of the K iterations' kernels"},
         "roofline": dominant, "roofline_other_kernel": other,
         "e2e": {"value": K * world / e2e["seconds"], "unit": UNIT, "h2d_bytes_per_step": e2e["h2d"] / K,
                 "d2h_bytes_per_step": e2e["d2h"] / K, "matches_device_run": e2e["matches"]},
-        "gpu_launches": launches["all"], "clocks": sampler.summary(),
+        "gpu_launches": res["launches"], "clocks": sampler.summary(),
     }
+    if static is not None:
+        out["static_sl_max"] = static
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         out["cpu_baseline"] = cpu_baseline(data, wl, budget_s=args.cpu_seconds)
     ctx.close()
@@ -510,6 +549,7 @@ def main():
     ap.add_argument("--cpu-seconds", type=float, default=15.0)
     ap.add_argument("--reference-seconds", type=float, default=120.0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-static", action="store_true", help="skip the extra pass with SL forced to SL_max")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
     rank = int(os.environ.get("RANK", 0))
