@@ -175,7 +175,7 @@ int disco_verify_ragged_host(disco_ctx* ctx, const void* W_T /*device*/, const v
  * cannot take the device-wide synchronisation a cudaMalloc may bring.  disco_create allocates its
  * scratch with cudaMalloc, so those hosts cannot have a context.  This entry point needs none: the
  * scratch for the cross-block reduction lives in a fixed array inside the library image
- * (about 385 KB of device memory on every GPU that loads the library, held until the process exits),
+ * (about 256 KB of device memory on every GPU that loads the library, held until the process exits),
  * and the call itself uses no cudaMalloc, cudaFree or allocating library routine.
  *
  * Arguments and results are those of disco_draft_step (same layouts, device pointers owned by the

@@ -193,73 +193,44 @@ __device__ __forceinline__ void warp_merge_softmax(SoftmaxState& st) {
     }
 }
 
-// A descending top-10 list kept by one warp: lane l < 10 holds entry l.  Values offered must be
-// warp-uniform.  An offered value equal to a stored one goes behind it, so offering candidates in
-// ascending index order keeps "lowest index first" among equals.
-struct WarpTop10 {
+// The ten largest values offered so far, kept by one warp: lane l < 10 holds the l-th largest.
+// Offered values must be warp-uniform.
+struct WarpTopV {
     float v;
-    int i;
-    float floor_v;  // warp-uniform copy of entry 9's value
+    float floor_v;  // warp-uniform copy of entry 9
     __device__ __forceinline__ void init() {
         v = DISCO_NEG_INF;
-        i = kNoIndex;
         floor_v = DISCO_NEG_INF;
     }
-    __device__ __forceinline__ void insert(float z, int idx, int lane) {
-        const unsigned ahead = __ballot_sync(kFullMask, lane < kTopK && v >= z);
-        const int p = __popc(ahead);
-        const float up_v = __shfl_up_sync(kFullMask, v, 1);
-        const int up_i = __shfl_up_sync(kFullMask, i, 1);
-        if (lane > p) {
-            v = up_v;
-            i = up_i;
-        } else if (lane == p) {
-            v = z;
-            i = idx;
+    __device__ __forceinline__ void offer(float z, int lane) {
+        if (z > floor_v) {
+            const unsigned ahead = __ballot_sync(kFullMask, lane < kTopK && v >= z);
+            const int p = __popc(ahead);
+            const float up_v = __shfl_up_sync(kFullMask, v, 1);
+            if (lane > p) v = up_v;
+            else if (lane == p) v = z;
+            floor_v = __shfl_sync(kFullMask, v, kTopK - 1);
         }
-        floor_v = __shfl_sync(kFullMask, v, kTopK - 1);
-    }
-    __device__ __forceinline__ void offer(float z, int idx, int lane) {
-        if (z > floor_v) insert(z, idx, lane);
     }
 };
 
-// Select the 10 best of the 32*E candidates a warp holds in registers (E slots per lane), ordered
-// by (value descending, index ascending).  Empty slots are (-inf, kNoIndex).  The slots are
-// consumed.  Result: lane r < 10 returns entry r, other lanes (-inf, kNoIndex).
-template <int E>
-__device__ __forceinline__ void warp_select_top10(float (&v)[E], int (&id)[E], int lane, float& out_v,
-                                                  int& out_i) {
-    out_v = DISCO_NEG_INF;
-    out_i = kNoIndex;
-#pragma unroll 1
-    for (int r = 0; r < kTopK; ++r) {
-        float bv = v[0];
-        int bi = id[0];
+// Ten largest values seen so far, descending, in the registers of one thread.
+struct RegTop10 {
+    float t[kTopK];
+    __device__ __forceinline__ void init() {
 #pragma unroll
-        for (int e = 1; e < E; ++e) {
-            const bool better = (v[e] > bv) || (v[e] == bv && id[e] < bi);
-            bv = better ? v[e] : bv;
-            bi = better ? id[e] : bi;
-        }
-        const uint32_t mine = ordered_bits(bv);
-        const uint32_t best = __reduce_max_sync(kFullMask, mine);
-        const int cand_i = (mine == best) ? bi : kNoIndex;
-        const int win_i = __reduce_min_sync(kFullMask, cand_i);
-        if (lane == r) {
-            out_v = from_ordered_bits(best);
-            out_i = win_i;
-        }
-        if (cand_i == win_i && win_i != kNoIndex) {  // this lane owns the winner: retire it
+        for (int k = 0; k < kTopK; ++k) t[k] = DISCO_NEG_INF;
+    }
+    __device__ __forceinline__ void push(float z) {
+        float carry = z;
 #pragma unroll
-            for (int e = 0; e < E; ++e)
-                if (id[e] == win_i) {
-                    v[e] = DISCO_NEG_INF;
-                    id[e] = kNoIndex;
-                }
+        for (int k = 0; k < kTopK; ++k) {
+            const float hi = fmaxf(t[k], carry);
+            carry = fminf(t[k], carry);
+            t[k] = hi;
         }
     }
-}
+};
 
 // Every lane holds a descending list l[0..9] (values only, -inf = empty).  Lane k < 10 returns the k-th
 // largest of all 320 values; the lists are consumed.  Equal values are interchangeable here.

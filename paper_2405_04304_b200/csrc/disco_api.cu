@@ -39,14 +39,11 @@ struct disco_ctx {
     // scratch for cross-block reductions
     int part_rows;  // rows the partial buffers can hold
     int max_grid;
-    float* part_stats;
-    float* part_topv;
-    int* part_topi;
     unsigned long long* keys;
     unsigned int* ticket;
     int* status;
     float* final_stats;
-    void* part_rec;                // tcgen05 draft path: 64-byte partial records
+    void* part_rec;                // draft step: 64-byte partial records, [sequence][CTA]
     int part_slots;                // partials per row the buffers can hold
     void* encode_tiled;            // cuTensorMapEncodeTiled, resolved through the runtime
     // device staging for the *_host entry points
@@ -196,9 +193,7 @@ int launch_umma(disco_ctx* c, const void* W, const void* H, int d, int R, float*
 }
 
 void fill_scratch(const disco_ctx* c, TailParams& p) {
-    p.part_stats = c->part_stats;
-    p.part_topv = c->part_topv;
-    p.part_topi = c->part_topi;
+    p.part_rec = reinterpret_cast<float4*>(c->part_rec);
     p.keys = c->keys;
     p.ticket = c->ticket;
     p.status = c->status;
@@ -270,9 +265,6 @@ int disco_create(disco_ctx** out, int V, int d_draft, int d_target, int max_batc
                          (size_t)max_rows + 64;
     const size_t hid = std::max((size_t)max_batch * d_draft, (size_t)max_rows * d_target) * 2;
     bool ok = true;
-    ok = ok && cudaMalloc(&c->part_stats, slots * 4 * sizeof(float)) == cudaSuccess;
-    ok = ok && cudaMalloc(&c->part_topv, slots * kTopK * sizeof(float)) == cudaSuccess;
-    ok = ok && cudaMalloc(&c->part_topi, slots * kTopK * sizeof(int)) == cudaSuccess;
     ok = ok && cudaMalloc(&c->keys, (size_t)max_rows * sizeof(unsigned long long)) == cudaSuccess;
     ok = ok && cudaMalloc(&c->part_rec, slots * 64) == cudaSuccess;
     ok = ok && cudaMalloc(&c->ticket, 256) == cudaSuccess;
@@ -296,9 +288,6 @@ int disco_create(disco_ctx** out, int V, int d_draft, int d_target, int max_batc
 
 int disco_destroy(disco_ctx* c) {
     if (!c) return DISCO_ERR_INVALID_ARG;
-    cudaFree(c->part_stats);
-    cudaFree(c->part_topv);
-    cudaFree(c->part_topi);
     cudaFree(c->keys);
     cudaFree(c->part_rec);
     cudaFree(c->ticket);

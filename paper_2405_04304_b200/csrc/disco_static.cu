@@ -25,9 +25,8 @@ constexpr int kWarps = 16;
 constexpr int kMaxB = DISCO_STATIC_MAX_BATCH;
 constexpr int kMaxGrid = DISCO_STATIC_MAX_GRID;
 constexpr size_t kHeadBytes = 256;  // ticket @0, status @64, final (m, Z) per sequence @128
-constexpr size_t kStatsBytes = (size_t)kMaxB * kMaxGrid * 16;
-constexpr size_t kTopBytes = (size_t)kMaxB * kMaxGrid * kTopK * 4;
-constexpr size_t kScratchBytes = kHeadBytes + kStatsBytes + 2 * kTopBytes;
+constexpr size_t kRecordBytes = (size_t)kMaxB * kMaxGrid * 64;  // one 64-byte partial record per (sequence, CTA)
+constexpr size_t kScratchBytes = kHeadBytes + kRecordBytes;
 
 // The scratch itself.  In host code this name is only a handle for cudaGetSymbolAddress; it is NOT a
 // device address and must never be handed to a kernel as one.
@@ -135,9 +134,7 @@ extern "C" int disco_draft_step_static(int V, int d_draft, const void* W_D, cons
     p.ticket = reinterpret_cast<unsigned int*>(s.scratch);
     p.status = reinterpret_cast<int*>(s.scratch + 64);
     p.final_stats = reinterpret_cast<float*>(s.scratch + 128);
-    p.part_stats = reinterpret_cast<float*>(s.scratch + kHeadBytes);
-    p.part_topv = reinterpret_cast<float*>(s.scratch + kHeadBytes + kStatsBytes);
-    p.part_topi = reinterpret_cast<int*>(s.scratch + kHeadBytes + kStatsBytes + kTopBytes);
+    p.part_rec = reinterpret_cast<float4*>(s.scratch + kHeadBytes);
     p.keys = nullptr;
     p.pos = pos;
     p.n_drafted = n_drafted;

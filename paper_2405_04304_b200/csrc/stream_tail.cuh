@@ -7,10 +7,14 @@
 //     ring of shared-memory slots with bulk (TMA-unit) copies signalled on mbarriers;
 //   * each ring slot is owned by one consumer warp, which works on up to four vocabulary rows at
 //     once: 128-bit shared loads, fp32 FMAs, shuffle reduction; the logits are warp-uniform and
-//     go straight into the warp's online soft-max state and its top-10 list (draft step) or its
-//     running arg-max (verification);
-//   * per-CTA partials go to scratch; the last CTA to take a ticket merges them and runs the
-//     fused epilogue (features + halt classifier + stopping rule, or prefix match + bonus token).
+//     go straight into the warp's online soft-max state, its top-10 values and its running arg-max;
+//   * per-CTA partials (64-byte records) go to scratch; the last CTA to take a ticket merges them
+//     and runs the fused epilogue (features + halt classifier + stopping rule, or prefix match +
+//     bonus token).
+//
+// The LM head is never written by this library, so the kernel starts streaming it before it waits
+// (griddepcontrol.wait) for the preceding kernel of the stream; everything that kernel may have
+// produced (hidden states, scratch) is touched only after the wait.
 //
 // More than RT hidden rows are handled by passing over the slab again (correct for any R, but
 // the tcgen05 kernel is the one meant for many rows).
@@ -30,9 +34,7 @@ struct TailParams {
     int stages;          // ring depth
     uint32_t slot_bytes; // rps * d * 2
     // scratch (context-owned)
-    float* part_stats;   // [R][grid][4]   (m, Z, S, -)
-    float* part_topv;    // [R][grid][10]
-    int* part_topi;      // [R][grid][10]
+    float4* part_rec;          // [R][grid] records: (m, Z, S, -), top-10 logits descending, arg-max key
     unsigned long long* keys;  // [R] packed arg-max keys, zero between calls
     unsigned int* ticket;      // zero between calls
     int* status;
@@ -62,20 +64,81 @@ struct TailParams {
     int32_t* target_ids;
 };
 
-constexpr int kWarpStateWords = 24;  // m, Z, S, pad, 10 values, 10 indices
+constexpr int kRecordWords = 16;  // one partial record: m, Z, S, -, 10 logits, key (2 words)
 
 inline size_t stream_tail_smem_bytes(int RT, int NW, int d, int stages, uint32_t slot_bytes, int clf_H) {
     size_t b = (size_t)stages * slot_bytes;           // ring
     b += (size_t)RT * d * 2;                          // hidden tile
     b += (size_t)stages * 16;                         // full/empty barriers
-    b += (size_t)NW * RT * kWarpStateWords * 4;       // warp states / finalize staging
+    b += (size_t)NW * RT * kRecordWords * 4;          // warp records / finalize staging
     b += 64 * 4;                                      // features
     b += ((size_t)clf_H * (kNFeat + 2) + 4) * 4;      // classifier parameters
     return b + 128;
 }
 
 // ---------------------------------------------------------------------------------------------
-// fused epilogues run by the last CTA
+// partial records
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ unsigned long long key_from_words(float lo, float hi) {
+    return (static_cast<unsigned long long>(__float_as_uint(hi)) << 32) | __float_as_uint(lo);
+}
+
+// Merge records [c0, c1) of one sequence into a single one; all lanes return the merged statistics
+// and key, lane k < 10 returns the k-th largest logit in sel.  Works from global or shared memory.
+template <bool GLOBAL>
+__device__ __forceinline__ void warp_merge_records(const float4* rec, int c0, int c1, int lane, SoftmaxState& st,
+                                                   unsigned long long& key, float& sel) {
+    st.init();
+    key = 0ull;
+    RegTop10 top;
+    top.init();
+    for (int c = c0 + lane; c < c1; c += 32) {
+        const float4* r = rec + (size_t)c * 4;
+        float4 q, a, bq, cq;
+        if (GLOBAL) {
+            q = __ldcg(r), a = __ldcg(r + 1), bq = __ldcg(r + 2), cq = __ldcg(r + 3);
+        } else {
+            q = r[0], a = r[1], bq = r[2], cq = r[3];
+        }
+        if (!(q.y > 0.f)) continue;  // empty record
+        st.merge(q.x, q.y, q.z);
+        const unsigned long long k2 = key_from_words(cq.z, cq.w);
+        key = k2 > key ? k2 : key;
+        const float lv[kTopK] = {a.x, a.y, a.z, a.w, bq.x, bq.y, bq.z, bq.w, cq.x, cq.y};
+        if (c < c0 + 32) {
+#pragma unroll
+            for (int k = 0; k < kTopK; ++k) top.t[k] = lv[k];  // first record of this lane: already sorted
+        } else {
+#pragma unroll
+            for (int k = 0; k < kTopK; ++k)
+                if (lv[k] > top.t[kTopK - 1]) top.push(lv[k]);
+        }
+    }
+    warp_merge_softmax(st);
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) {
+        const unsigned long long k2 = __shfl_xor_sync(kFullMask, key, off);
+        key = k2 > key ? k2 : key;
+    }
+    sel = warp_select_sorted(top.t, lane);
+}
+
+// Lane 0 holds (m, Z, S, key); lane k < 10 holds the k-th logit: write them as one record.
+__device__ __forceinline__ void warp_store_record(float* rec, const SoftmaxState& st, unsigned long long key, float sel,
+                                                  int lane) {
+    if (lane == 0) {
+        rec[0] = st.m;
+        rec[1] = st.Z;
+        rec[2] = st.S;
+        rec[3] = 0.f;
+        rec[14] = __uint_as_float(static_cast<uint32_t>(key & 0xffffffffull));
+        rec[15] = __uint_as_float(static_cast<uint32_t>(key >> 32));
+    }
+    if (lane < kTopK) rec[4 + lane] = sel;
+}
+
+// ---------------------------------------------------------------------------------------------
+// fused epilogues
 // ---------------------------------------------------------------------------------------------
 
 // Halt classifier of Eq. 2 by one warp: C = sigmoid(w2 . relu(W1 x + b1) + b2).  x (lane < 12) is the
@@ -98,114 +161,56 @@ __device__ __forceinline__ float warp_halt_classifier(float x, float* feat_s, co
     return 1.f / (1.f + expf(-(acc + b2)));
 }
 
-// Draft step, sequence b: merge the per-CTA partials, form the features of Eq. 2, run the
-// classifier and the stopping rule.  Called by all NW consumer warps of the last CTA.
+// Features of Eq. 2 from merged statistics, then classifier and stopping rule; one warp.
+// sel: lane k < 10 holds the k-th largest logit.
+struct DraftOutputs {
+    int32_t* token;
+    float* conf;
+    uint8_t* halt;
+    float* feats;
+    float* final_stats;
+};
+__device__ __forceinline__ void warp_draft_epilogue(const SoftmaxState& st, unsigned long long key, float sel, float fpos,
+                                                    int n_drafted, float tau, int sl_max, float* feat_s, const float* W1,
+                                                    const float* b1, const float* w2, const float* b2, int Hc, int b,
+                                                    const DraftOutputs& o, int lane) {
+    const float inv_Z = 1.f / st.Z;
+    const float prob = (lane < kTopK && sel > DISCO_NEG_INF) ? expf(sel - st.m) * inv_Z : 0.f;
+    const float ent = logf(st.Z) - st.S * inv_Z;
+    const float x = lane < kTopK ? prob : (lane == kTopK ? ent : (lane == kTopK + 1 ? fpos : 0.f));
+    const float C = warp_halt_classifier(x, feat_s, W1, b1, w2, b2, Hc, lane);
+    if (lane == 0) {
+        o.token[b] = key_index(key);
+        o.conf[b] = C;
+        o.halt[b] = ((C < tau) || (n_drafted >= sl_max)) ? 1 : 0;
+        o.final_stats[2 * b] = st.m;
+        o.final_stats[2 * b + 1] = st.Z;
+    }
+    if (o.feats && lane < kNFeat) o.feats[(size_t)b * kNFeat + lane] = x;
+}
+
+// Draft step, sequence b, in the last CTA: NW warps reduce the per-CTA records in two levels.
 template <int NW>
-__device__ void finalize_draft_row(const TailParams& p, int b, int grid, float* stage /*NW*24 words*/,
-                                   float* feat_s, const float* clf_s, int warp, int lane) {
+__device__ void finalize_draft_row(const TailParams& p, int b, int grid, float* stage /*NW records*/, float* feat_s,
+                                   const float* clf_s, int warp, int lane) {
     constexpr int BAR_THREADS = NW * 32;
+    const float fpos = static_cast<float>(p.pos[b]);  // issued early: hidden behind the merge
+    const int n_drafted = p.n_drafted[b];
     const int cpw = (grid + NW - 1) / NW;  // CTAs per warp
     const int c0 = min(grid, warp * cpw);
     const int c1 = min(grid, c0 + cpw);
-    const size_t base = (size_t)b * grid;
-
-    // issue every global load this warp needs before any of the arithmetic
-    const float fpos = static_cast<float>(p.pos[b]);
-    const int n_drafted = p.n_drafted[b];
-    const int ncand = (c1 - c0) * kTopK;
-    const float* tv = p.part_topv + (base + c0) * kTopK;
-    const int* ti = p.part_topi + (base + c0) * kTopK;
-    float4 q0 = make_float4(DISCO_NEG_INF, 0.f, 0.f, 0.f);
-    if (c0 + lane < c1) q0 = __ldcg(reinterpret_cast<const float4*>(p.part_stats) + base + c0 + lane);
-    float v0[5];
-    int id0[5];
-#pragma unroll
-    for (int j = 0; j < 4; ++j) {
-        const int e = j * 32 + lane;
-        const bool ok = e < ncand;
-        v0[j] = ok ? __ldcg(tv + e) : DISCO_NEG_INF;
-        id0[j] = ok ? __ldcg(ti + e) : kNoIndex;
-    }
-    v0[4] = DISCO_NEG_INF;
-    id0[4] = kNoIndex;
-
-    // stage A: this warp reduces its share of the CTAs
     SoftmaxState st;
-    st.init();
-    st.merge(q0.x, q0.y, q0.z);
-    for (int c = c0 + lane + 32; c < c1; c += 32) {
-        const float4 q = __ldcg(reinterpret_cast<const float4*>(p.part_stats) + base + c);
-        st.merge(q.x, q.y, q.z);
-    }
-    warp_merge_softmax(st);
-
-    float run_v;
-    int run_i;
-    warp_select_top10<5>(v0, id0, lane, run_v, run_i);
-    for (int e0 = 32 * 4; e0 < ncand; e0 += 32 * 4) {
-        float v[5];
-        int id[5];
-#pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            const int e = e0 + j * 32 + lane;
-            const bool ok = e < ncand;
-            v[j] = ok ? __ldcg(tv + e) : DISCO_NEG_INF;
-            id[j] = ok ? __ldcg(ti + e) : kNoIndex;
-        }
-        v[4] = run_v;
-        id[4] = run_i;
-        warp_select_top10<5>(v, id, lane, run_v, run_i);
-    }
-    float* mine = stage + warp * kWarpStateWords;
-    if (lane == 0) {
-        mine[0] = st.m;
-        mine[1] = st.Z;
-        mine[2] = st.S;
-    }
-    if (lane < kTopK) {
-        mine[4 + lane] = run_v;
-        reinterpret_cast<int*>(mine)[4 + kTopK + lane] = run_i;
-    }
+    unsigned long long key;
+    float sel;
+    warp_merge_records<true>(p.part_rec + (size_t)b * grid * 4, c0, c1, lane, st, key, sel);
+    warp_store_record(stage + warp * kRecordWords, st, key, sel, lane);
     named_barrier_sync(1, BAR_THREADS);
-
-    // stage B: warp 0 merges the NW warp results and runs the epilogue
     if (warp == 0) {
-        SoftmaxState g;
-        g.init();
-        for (int w = lane; w < NW; w += 32)
-            g.merge(stage[w * kWarpStateWords], stage[w * kWarpStateWords + 1], stage[w * kWarpStateWords + 2]);
-        warp_merge_softmax(g);
-        constexpr int E = (NW * kTopK + 31) / 32;
-        float v[E];
-        int id[E];
-#pragma unroll
-        for (int j = 0; j < E; ++j) {
-            const int e = j * 32 + lane;
-            const bool ok = e < NW * kTopK;
-            const int w = ok ? e / kTopK : 0, k = ok ? e % kTopK : 0;
-            v[j] = ok ? stage[w * kWarpStateWords + 4 + k] : DISCO_NEG_INF;
-            id[j] = ok ? reinterpret_cast<const int*>(stage)[w * kWarpStateWords + 4 + kTopK + k] : kNoIndex;
-        }
-        float top_v;
-        int top_i;
-        warp_select_top10<E>(v, id, lane, top_v, top_i);
-
-        // features: top-10 probabilities, entropy, position
-        const float inv_Z = 1.f / g.Z;
-        const float prob = (lane < kTopK && top_i != kNoIndex) ? expf(top_v - g.m) * inv_Z : 0.f;
-        const float ent = logf(g.Z) - g.S * inv_Z;
-        const float x = lane < kTopK ? prob : (lane == kTopK ? ent : (lane == kTopK + 1 ? fpos : 0.f));
-        const float C = warp_halt_classifier(x, feat_s, clf_s, clf_s + p.clf_H * kNFeat, clf_s + p.clf_H * (kNFeat + 1),
-                                             clf_s + p.clf_H * (kNFeat + 2), p.clf_H, lane);
-        const int tok = __shfl_sync(kFullMask, top_i, 0);
-        if (lane == 0) {
-            p.token[b] = tok;
-            p.conf[b] = C;
-            p.halt[b] = ((C < p.tau) || (n_drafted >= p.sl_max)) ? 1 : 0;
-            p.final_stats[2 * b] = g.m;
-            p.final_stats[2 * b + 1] = g.Z;
-        }
-        if (p.feats && lane < kNFeat) p.feats[(size_t)b * kNFeat + lane] = x;
+        warp_merge_records<false>(reinterpret_cast<const float4*>(stage), 0, NW, lane, st, key, sel);
+        const int Hc = p.clf_H;
+        const DraftOutputs o{p.token, p.conf, p.halt, p.feats, p.final_stats};
+        warp_draft_epilogue(st, key, sel, fpos, n_drafted, p.tau, p.sl_max, feat_s, clf_s, clf_s + Hc * kNFeat,
+                            clf_s + Hc * (kNFeat + 1), clf_s + Hc * (kNFeat + 2), Hc, b, o, lane);
     }
     named_barrier_sync(1, BAR_THREADS);
 }
@@ -277,8 +282,8 @@ __global__ void __launch_bounds__((NW + 1) * 32, 1) stream_tail_kernel(const __g
     uint8_t* htile = ring + (size_t)p.stages * p.slot_bytes;
     uint64_t* full = reinterpret_cast<uint64_t*>(htile + (size_t)RT * row_bytes);
     uint64_t* empty = full + p.stages;
-    float* wstate = reinterpret_cast<float*>(empty + p.stages);
-    float* feat_s = wstate + NW * RT * kWarpStateWords;
+    float* wstate = reinterpret_cast<float*>(empty + p.stages);  // 16-byte aligned
+    float* feat_s = wstate + NW * RT * kRecordWords;
     float* clf_s = feat_s + 64;
     __shared__ int s_is_last;
 
@@ -286,6 +291,9 @@ __global__ void __launch_bounds__((NW + 1) * 32, 1) stream_tail_kernel(const __g
     const int nrows = min(p.V, v0 + p.rows_per_cta) - v0;
     const int nslots = (nrows + p.rps - 1) / p.rps;
     const int nchunks = (p.R + RT - 1) / RT;
+
+    // the next kernel of the stream may start its own prologue now
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
     if (tid == 0) {
         for (int s = 0; s < p.stages; ++s) {
@@ -330,6 +338,10 @@ __global__ void __launch_bounds__((NW + 1) * 32, 1) stream_tail_kernel(const __g
         }
         cp_async_commit();
     }
+    // from here on the kernel reads the hidden states and writes scratch and outputs: the preceding
+    // kernel of the stream must have finished
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+
     const int n16 = (int)(row_bytes >> 4);  // 16-byte pieces per row
     for (int chunk = 0; chunk < nchunks; ++chunk) {
         named_barrier_sync(1, BAR_THREADS);  // previous chunk's readers of the hidden tile are done
@@ -343,7 +355,7 @@ __global__ void __launch_bounds__((NW + 1) * 32, 1) stream_tail_kernel(const __g
         named_barrier_sync(1, BAR_THREADS);
 
         SoftmaxState st[RT];
-        WarpTop10 top[RT];
+        WarpTopV top[RT];
         float best_v[RT];
         int best_i[RT];
 #pragma unroll
@@ -433,16 +445,15 @@ __global__ void __launch_bounds__((NW + 1) * 32, 1) stream_tail_kernel(const __g
 #pragma unroll
                         for (int r = 0; r < RT; ++r) {
                             const float z = __fadd_rn(acc[g][r], 0.f);  // folds -0 into +0
+                            if (z > best_v[r]) {  // rows arrive in ascending order: the lowest index wins ties
+                                best_v[r] = z;
+                                best_i[r] = v;
+                            }
                             if (DRAFT) {
                                 st[r].push(z);
-                                top[r].offer(z, v, lane);
+                                top[r].offer(z, lane);
                                 if (p.probs && lane == 0 && chunk * RT + r < p.R)
                                     p.probs[(size_t)(chunk * RT + r) * p.V + v] = z;
-                            } else {
-                                if (z > best_v[r]) {
-                                    best_v[r] = z;
-                                    best_i[r] = v;
-                                }
                             }
                         }
                     }
@@ -452,53 +463,42 @@ __global__ void __launch_bounds__((NW + 1) * 32, 1) stream_tail_kernel(const __g
             }
         }
 
-        // ---- merge the NW warps of this CTA, publish the CTA's partial for each hidden row ----
+        // ---- merge the NW warps of this CTA, publish the CTA's result for each hidden row ----
         if (DRAFT) {
 #pragma unroll
             for (int r = 0; r < RT; ++r) {
-                float* mine = wstate + (warp * RT + r) * kWarpStateWords;
-                if (lane == 0) {
-                    mine[0] = st[r].m;
-                    mine[1] = st[r].Z;
-                    mine[2] = st[r].S;
-                }
-                if (lane < kTopK) {
-                    mine[4 + lane] = top[r].v;
-                    reinterpret_cast<int*>(mine)[4 + kTopK + lane] = top[r].i;
-                }
+                const unsigned long long key = best_i[r] != kNoIndex ? argmax_key(best_v[r], best_i[r]) : 0ull;
+                warp_store_record(wstate + (warp * RT + r) * kRecordWords, st[r], key, top[r].v, lane);
             }
             named_barrier_sync(1, BAR_THREADS);
             for (int r = warp; r < RT; r += NW) {
                 const int row = chunk * RT + r;
                 if (row >= p.R) continue;
+                // the records of hidden row r sit RT records apart; lane w < NW takes warp w's
                 SoftmaxState g;
                 g.init();
-                for (int w = lane; w < NW; w += 32) {
-                    const float* o = wstate + (w * RT + r) * kWarpStateWords;
-                    g.merge(o[0], o[1], o[2]);
+                unsigned long long key = 0ull;
+                float l[kTopK];
+#pragma unroll
+                for (int k = 0; k < kTopK; ++k) l[k] = DISCO_NEG_INF;
+                if (lane < NW) {
+                    const float* o = wstate + (lane * RT + r) * kRecordWords;
+                    if (o[1] > 0.f) {
+                        g.merge(o[0], o[1], o[2]);
+                        key = key_from_words(o[14], o[15]);
+#pragma unroll
+                        for (int k = 0; k < kTopK; ++k) l[k] = o[4 + k];
+                    }
                 }
                 warp_merge_softmax(g);
-                constexpr int E = (NW * kTopK + 31) / 32;
-                float v[E];
-                int id[E];
 #pragma unroll
-                for (int j = 0; j < E; ++j) {
-                    const int e = j * 32 + lane;
-                    const bool ok = e < NW * kTopK;
-                    const int w = ok ? e / kTopK : 0, k = ok ? e % kTopK : 0;
-                    const float* o = wstate + (w * RT + r) * kWarpStateWords;
-                    v[j] = ok ? o[4 + k] : DISCO_NEG_INF;
-                    id[j] = ok ? reinterpret_cast<const int*>(o)[4 + kTopK + k] : kNoIndex;
+                for (int off = 16; off > 0; off >>= 1) {
+                    const unsigned long long k2 = __shfl_xor_sync(kFullMask, key, off);
+                    key = k2 > key ? k2 : key;
                 }
-                float tv;
-                int ti;
-                warp_select_top10<E>(v, id, lane, tv, ti);
-                const size_t slot = (size_t)row * grid + blockIdx.x;
-                if (lane == 0) reinterpret_cast<float4*>(p.part_stats)[slot] = make_float4(g.m, g.Z, g.S, 0.f);
-                if (lane < kTopK) {
-                    p.part_topv[slot * kTopK + lane] = tv;
-                    p.part_topi[slot * kTopK + lane] = ti;
-                }
+                const float sel = warp_select_sorted(l, lane);
+                warp_store_record(reinterpret_cast<float*>(p.part_rec + ((size_t)row * grid + blockIdx.x) * 4), g, key,
+                                  sel, lane);
             }
         } else {
             unsigned long long* keys_s = reinterpret_cast<unsigned long long*>(wstate);

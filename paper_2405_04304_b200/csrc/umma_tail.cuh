@@ -127,24 +127,6 @@ __device__ __forceinline__ uint32_t umma_idesc(int n) {
 
 // Vocabulary tile t covers rows [t * TR, min(V, (t + 1) * TR)).  The TMA box and the MMA take TRN >= TR
 // rows; the extra rows (the next tile's first rows, or zero fill past V) land in columns the epilogue skips.
-// Ten largest values seen so far, descending, in registers.
-struct RegTop10 {
-    float t[kTopK];
-    __device__ __forceinline__ void init() {
-#pragma unroll
-        for (int k = 0; k < kTopK; ++k) t[k] = DISCO_NEG_INF;
-    }
-    __device__ __forceinline__ void push(float z) {
-        float carry = z;
-#pragma unroll
-        for (int k = 0; k < kTopK; ++k) {
-            const float hi = fmaxf(t[k], carry);
-            carry = fminf(t[k], carry);
-            t[k] = hi;
-        }
-    }
-};
-
 // ---------------------------------------------------------------------------------------------
 // main kernel
 // ---------------------------------------------------------------------------------------------
