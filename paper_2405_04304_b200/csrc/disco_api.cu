@@ -35,6 +35,7 @@ struct disco_ctx {
     int sm_count;
     size_t smem_optin;
     int path;
+    int pdl;  // launch the streaming kernel with programmatic stream serialization (DISCO_PDL=0 turns it off)
     long long launches;
     // scratch for cross-block reductions
     int part_rows;  // rows the partial buffers can hold
@@ -104,9 +105,22 @@ int launch_stream(disco_ctx* c, TailParams& p, const StreamPlan& pl, cudaStream_
         configured_dev = c->device;
     }
     if (pl.smem > dyn_limit) return DISCO_ERR_UNSUPPORTED_SHAPE;
-    kern<<<pl.grid, (kStreamWarps + 1) * 32, pl.smem, st>>>(p);
+    // Programmatic dependent launch: the kernel may start while the preceding kernel of the stream is
+    // still in its tail; it streams the LM head (never written by this library) and waits with
+    // griddepcontrol.wait before it touches anything else.
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3((unsigned)pl.grid);
+    cfg.blockDim = dim3((kStreamWarps + 1) * 32);
+    cfg.dynamicSmemBytes = pl.smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = c->pdl ? 1 : 0;
+    const cudaError_t e = cudaLaunchKernelEx(&cfg, kern, p);
     c->launches += 1;
-    return cuda_ok(cudaGetLastError(), "stream_tail_kernel launch") ? DISCO_OK : DISCO_ERR_CUDA;
+    return cuda_ok(e, "stream_tail_kernel launch") ? DISCO_OK : DISCO_ERR_CUDA;
 }
 
 template <bool DRAFT>
@@ -246,6 +260,10 @@ int disco_create(disco_ctx** out, int V, int d_draft, int d_target, int max_batc
     c->max_batch = max_batch;
     c->max_rows = max_rows;
     c->clf_hidden = clf_hidden;
+    {
+        const char* e = std::getenv("DISCO_PDL");
+        c->pdl = !(e && e[0] == '0');
+    }
     c->sm_count = prop.multiProcessorCount;
     c->smem_optin = prop.sharedMemPerBlockOptin;
 
