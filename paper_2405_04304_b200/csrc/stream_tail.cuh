@@ -70,7 +70,7 @@ inline size_t stream_tail_smem_bytes(int RT, int NW, int d, int stages, uint32_t
     size_t b = (size_t)stages * slot_bytes;           // ring
     b += (size_t)RT * d * 2;                          // hidden tile
     b += (size_t)stages * 16;                         // full/empty barriers
-    b += (size_t)NW * RT * kRecordWords * 4;          // warp records / finalize staging
+    b += (size_t)(NW * RT + 1) * kRecordWords * 4;    // warp records / finalize staging (+ carry)
     b += 64 * 4;                                      // features
     b += ((size_t)clf_H * (kNFeat + 2) + 4) * 4;      // classifier parameters
     return b + 128;
@@ -83,44 +83,45 @@ __device__ __forceinline__ unsigned long long key_from_words(float lo, float hi)
     return (static_cast<unsigned long long>(__float_as_uint(hi)) << 32) | __float_as_uint(lo);
 }
 
-// Merge records [c0, c1) of one sequence into a single one; all lanes return the merged statistics
-// and key, lane k < 10 returns the k-th largest logit in sel.  Works from global or shared memory.
-template <bool GLOBAL>
-__device__ __forceinline__ void warp_merge_records(const float4* rec, int c0, int c1, int lane, SoftmaxState& st,
-                                                   unsigned long long& key, float& sel) {
+// Merge up to 32 partial records (lane i takes record i, `stride` words apart) into one: every lane
+// returns the merged statistics and arg-max key, lane k < 10 the k-th largest logit.  The records may
+// live in shared or in global memory (volatile reads, so values written by other CTAs are fetched from
+// L2).  Deliberately small and not inlined: it runs a few times per launch, and every call after the
+// first finds its instructions in the instruction cache.
+static __device__ __noinline__ void warp_merge_records(const volatile float* recs, int n, int stride, SoftmaxState& st,
+                                                unsigned long long& key, float& sel) {
+    const int lane = threadIdx.x & 31;
+    const volatile float* mine = recs + (size_t)lane * stride;
     st.init();
     key = 0ull;
-    RegTop10 top;
-    top.init();
-    for (int c = c0 + lane; c < c1; c += 32) {
-        const float4* r = rec + (size_t)c * 4;
-        float4 q, a, bq, cq;
-        if (GLOBAL) {
-            q = __ldcg(r), a = __ldcg(r + 1), bq = __ldcg(r + 2), cq = __ldcg(r + 3);
-        } else {
-            q = r[0], a = r[1], bq = r[2], cq = r[3];
-        }
-        if (!(q.y > 0.f)) continue;  // empty record
-        st.merge(q.x, q.y, q.z);
-        const unsigned long long k2 = key_from_words(cq.z, cq.w);
-        key = k2 > key ? k2 : key;
-        const float lv[kTopK] = {a.x, a.y, a.z, a.w, bq.x, bq.y, bq.z, bq.w, cq.x, cq.y};
-        if (c < c0 + 32) {
-#pragma unroll
-            for (int k = 0; k < kTopK; ++k) top.t[k] = lv[k];  // first record of this lane: already sorted
-        } else {
-#pragma unroll
-            for (int k = 0; k < kTopK; ++k)
-                if (lv[k] > top.t[kTopK - 1]) top.push(lv[k]);
-        }
+    const bool have = lane < n && mine[1] > 0.f;
+    if (have) {
+        st.m = mine[0];
+        st.Z = mine[1];
+        st.S = mine[2];
+        key = key_from_words(mine[14], mine[15]);
     }
-    warp_merge_softmax(st);
-#pragma unroll
+#pragma unroll 1
     for (int off = 16; off > 0; off >>= 1) {
+        const float m2 = __shfl_xor_sync(kFullMask, st.m, off);
+        const float Z2 = __shfl_xor_sync(kFullMask, st.Z, off);
+        const float S2 = __shfl_xor_sync(kFullMask, st.S, off);
         const unsigned long long k2 = __shfl_xor_sync(kFullMask, key, off);
+        st.merge(m2, Z2, S2);
         key = k2 > key ? k2 : key;
     }
-    sel = warp_select_sorted(top.t, lane);
+    // each record's list is descending: ten rounds over the list heads
+    int head = 0;
+    sel = DISCO_NEG_INF;
+#pragma unroll 1
+    for (int r = 0; r < kTopK; ++r) {
+        const float hv = (have && head < kTopK) ? mine[4 + head] : DISCO_NEG_INF;
+        const uint32_t bits = ordered_bits(hv);
+        const uint32_t best = __reduce_max_sync(kFullMask, bits);
+        const unsigned who = __ballot_sync(kFullMask, bits == best);
+        if (lane == r) sel = from_ordered_bits(best);
+        if (lane == __ffs(who) - 1) ++head;
+    }
 }
 
 // Lane 0 holds (m, Z, S, key); lane k < 10 holds the k-th logit: write them as one record.
@@ -189,24 +190,31 @@ __device__ __forceinline__ void warp_draft_epilogue(const SoftmaxState& st, unsi
     if (o.feats && lane < kNFeat) o.feats[(size_t)b * kNFeat + lane] = x;
 }
 
-// Draft step, sequence b, in the last CTA: NW warps reduce the per-CTA records in two levels.
+// Draft step, sequence b, in the last CTA: the NW warps reduce the per-CTA records 32 at a time, warp 0
+// merges their results (plus the carry of an earlier block when there are more than 32 * NW records).
 template <int NW>
-__device__ void finalize_draft_row(const TailParams& p, int b, int grid, float* stage /*NW records*/, float* feat_s,
-                                   const float* clf_s, int warp, int lane) {
+__device__ void finalize_draft_row(const TailParams& p, int b, int grid, float* stage /*(NW + 1) records*/,
+                                   float* feat_s, const float* clf_s, int warp, int lane) {
     constexpr int BAR_THREADS = NW * 32;
     const float fpos = static_cast<float>(p.pos[b]);  // issued early: hidden behind the merge
     const int n_drafted = p.n_drafted[b];
-    const int cpw = (grid + NW - 1) / NW;  // CTAs per warp
-    const int c0 = min(grid, warp * cpw);
-    const int c1 = min(grid, c0 + cpw);
+    const float* recs = reinterpret_cast<const float*>(p.part_rec + (size_t)b * grid * 4);
     SoftmaxState st;
     unsigned long long key;
     float sel;
-    warp_merge_records<true>(p.part_rec + (size_t)b * grid * 4, c0, c1, lane, st, key, sel);
-    warp_store_record(stage + warp * kRecordWords, st, key, sel, lane);
-    named_barrier_sync(1, BAR_THREADS);
+    for (int base = 0; base < grid; base += 32 * NW) {
+        const int c0 = base + warp * 32;
+        const int n = max(0, min(32, grid - c0));
+        warp_merge_records(recs + (size_t)c0 * kRecordWords, n, kRecordWords, st, key, sel);
+        warp_store_record(stage + warp * kRecordWords, st, key, sel, lane);
+        named_barrier_sync(1, BAR_THREADS);
+        if (warp == 0) {
+            warp_merge_records(stage, base == 0 ? NW : NW + 1, kRecordWords, st, key, sel);
+            if (base + 32 * NW < grid) warp_store_record(stage + NW * kRecordWords, st, key, sel, lane);  // carry
+        }
+        named_barrier_sync(1, BAR_THREADS);
+    }
     if (warp == 0) {
-        warp_merge_records<false>(reinterpret_cast<const float4*>(stage), 0, NW, lane, st, key, sel);
         const int Hc = p.clf_H;
         const DraftOutputs o{p.token, p.conf, p.halt, p.feats, p.final_stats};
         warp_draft_epilogue(st, key, sel, fpos, n_drafted, p.tau, p.sl_max, feat_s, clf_s, clf_s + Hc * kNFeat,
@@ -283,7 +291,7 @@ __global__ void __launch_bounds__((NW + 1) * 32, 1) stream_tail_kernel(const __g
     uint64_t* full = reinterpret_cast<uint64_t*>(htile + (size_t)RT * row_bytes);
     uint64_t* empty = full + p.stages;
     float* wstate = reinterpret_cast<float*>(empty + p.stages);  // 16-byte aligned
-    float* feat_s = wstate + NW * RT * kRecordWords;
+    float* feat_s = wstate + (NW * RT + 1) * kRecordWords;
     float* clf_s = feat_s + 64;
     __shared__ int s_is_last;
 
@@ -476,27 +484,9 @@ __global__ void __launch_bounds__((NW + 1) * 32, 1) stream_tail_kernel(const __g
                 if (row >= p.R) continue;
                 // the records of hidden row r sit RT records apart; lane w < NW takes warp w's
                 SoftmaxState g;
-                g.init();
-                unsigned long long key = 0ull;
-                float l[kTopK];
-#pragma unroll
-                for (int k = 0; k < kTopK; ++k) l[k] = DISCO_NEG_INF;
-                if (lane < NW) {
-                    const float* o = wstate + (lane * RT + r) * kRecordWords;
-                    if (o[1] > 0.f) {
-                        g.merge(o[0], o[1], o[2]);
-                        key = key_from_words(o[14], o[15]);
-#pragma unroll
-                        for (int k = 0; k < kTopK; ++k) l[k] = o[4 + k];
-                    }
-                }
-                warp_merge_softmax(g);
-#pragma unroll
-                for (int off = 16; off > 0; off >>= 1) {
-                    const unsigned long long k2 = __shfl_xor_sync(kFullMask, key, off);
-                    key = k2 > key ? k2 : key;
-                }
-                const float sel = warp_select_sorted(l, lane);
+                unsigned long long key;
+                float sel;
+                warp_merge_records(wstate + r * kRecordWords, NW, RT * kRecordWords, g, key, sel);
                 warp_store_record(reinterpret_cast<float*>(p.part_rec + ((size_t)row * grid + blockIdx.x) * 4), g, key,
                                   sel, lane);
             }

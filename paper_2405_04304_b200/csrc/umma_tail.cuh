@@ -409,89 +409,38 @@ __global__ void __launch_bounds__(128) verify_finalize_kernel(const VerifyFinalP
 
 constexpr int kDraftFinalWarps = 8;
 
-// One CTA per sequence: every lane takes one partial record (more only if there are over 256 of them),
-// the warps reduce to one sorted list each, warp 0 finishes.
+// One CTA per sequence: the warps reduce the per-CTA records 32 at a time, warp 0 merges their results
+// and runs the epilogue.
 __global__ void __launch_bounds__(kDraftFinalWarps * 32) draft_finalize_kernel(const DraftFinalParams p) {
-    __shared__ float4 wres[kDraftFinalWarps][4];
+    __shared__ __align__(16) float stage[(kDraftFinalWarps + 1) * kRecordWords];
     __shared__ float feat_s[16];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int b = blockIdx.x;
     if (p.active && !p.active[b]) return;
-    const size_t base = (size_t)b * p.NP;
-
-    SoftmaxState st;
-    st.init();
-    unsigned long long key = 0ull;
-    RegTop10 top;
-    top.init();
-    for (int c = threadIdx.x; c < p.NP; c += kDraftFinalWarps * 32) {
-        const float4* rec = p.part_rec + (base + c) * 4;
-        const float4 q = __ldcg(rec), a = __ldcg(rec + 1), bq = __ldcg(rec + 2), cq = __ldcg(rec + 3);
-        if (!(q.y > 0.f)) continue;  // that CTA had no columns
-        st.merge(q.x, q.y, q.z);
-        const unsigned long long k2 =
-            (static_cast<unsigned long long>(__float_as_uint(cq.w)) << 32) | __float_as_uint(cq.z);
-        key = k2 > key ? k2 : key;
-        const float lv[kTopK] = {a.x, a.y, a.z, a.w, bq.x, bq.y, bq.z, bq.w, cq.x, cq.y};
-        if (c < kDraftFinalWarps * 32) {
-#pragma unroll
-            for (int k = 0; k < kTopK; ++k) top.t[k] = lv[k];  // first record: already sorted
-        } else {
-#pragma unroll
-            for (int k = 0; k < kTopK; ++k)
-                if (lv[k] > top.t[kTopK - 1]) top.push(lv[k]);
-        }
-    }
-    warp_merge_softmax(st);
-#pragma unroll
-    for (int off = 16; off > 0; off >>= 1) {
-        const unsigned long long k2 = __shfl_xor_sync(kFullMask, key, off);
-        key = k2 > key ? k2 : key;
-    }
-    const float sel = warp_select_sorted(top.t, lane);  // lane k < 10: k-th largest logit of this warp's records
-    float* wr = reinterpret_cast<float*>(&wres[warp][0]);
-    if (lane == 0) {
-        wr[0] = st.m;
-        wr[1] = st.Z;
-        wr[2] = st.S;
-        wr[14] = __uint_as_float((uint32_t)(key & 0xffffffffull));
-        wr[15] = __uint_as_float((uint32_t)(key >> 32));
-    }
-    if (lane < kTopK) wr[4 + lane] = sel;
-    __syncthreads();
-    if (warp != 0) return;
-
-    st.init();
-    key = 0ull;
-    top.init();
-    if (lane < kDraftFinalWarps) {
-        const float* o = reinterpret_cast<const float*>(&wres[lane][0]);
-        st.merge(o[0], o[1], o[2]);
-        key = (static_cast<unsigned long long>(__float_as_uint(o[15])) << 32) | __float_as_uint(o[14]);
-#pragma unroll
-        for (int k = 0; k < kTopK; ++k) top.t[k] = o[4 + k];
-    }
-    warp_merge_softmax(st);
-#pragma unroll
-    for (int off = 16; off > 0; off >>= 1) {
-        const unsigned long long k2 = __shfl_xor_sync(kFullMask, key, off);
-        key = k2 > key ? k2 : key;
-    }
-    const float mine = warp_select_sorted(top.t, lane);
-    const float inv_Z = 1.f / st.Z;
-    const float prob = (lane < kTopK && mine > DISCO_NEG_INF) ? expf(mine - st.m) * inv_Z : 0.f;
-    const float ent = logf(st.Z) - st.S * inv_Z;
     const float fpos = static_cast<float>(p.pos[b]);
-    const float x = lane < kTopK ? prob : (lane == kTopK ? ent : (lane == kTopK + 1 ? fpos : 0.f));
-    const float C = warp_halt_classifier(x, feat_s, p.clf_W1, p.clf_b1, p.clf_w2, p.clf_b2, p.clf_H, lane);
-    if (lane == 0) {
-        p.token[b] = key_index(key);
-        p.conf[b] = C;
-        p.halt[b] = ((C < p.tau) || (p.n_drafted[b] >= p.sl_max)) ? 1 : 0;
-        p.final_stats[2 * b] = st.m;
-        p.final_stats[2 * b + 1] = st.Z;
+    const int n_drafted = p.n_drafted[b];
+    const float* recs = reinterpret_cast<const float*>(p.part_rec + (size_t)b * p.NP * 4);
+    SoftmaxState st;
+    unsigned long long key;
+    float sel;
+    for (int base = 0; base < p.NP; base += 32 * kDraftFinalWarps) {
+        const int c0 = base + warp * 32;
+        const int n = max(0, min(32, p.NP - c0));
+        warp_merge_records(recs + (size_t)c0 * kRecordWords, n, kRecordWords, st, key, sel);
+        warp_store_record(stage + warp * kRecordWords, st, key, sel, lane);
+        __syncthreads();
+        if (warp == 0) {
+            warp_merge_records(stage, base == 0 ? kDraftFinalWarps : kDraftFinalWarps + 1, kRecordWords, st, key, sel);
+            if (base + 32 * kDraftFinalWarps < p.NP)
+                warp_store_record(stage + kDraftFinalWarps * kRecordWords, st, key, sel, lane);
+        }
+        __syncthreads();
     }
-    if (p.feats && lane < kNFeat) p.feats[(size_t)b * kNFeat + lane] = x;
+    if (warp == 0) {
+        const DraftOutputs o{p.token, p.conf, p.halt, p.feats, p.final_stats};
+        warp_draft_epilogue(st, key, sel, fpos, n_drafted, p.tau, p.sl_max, feat_s, p.clf_W1, p.clf_b1, p.clf_w2,
+                            p.clf_b2, p.clf_H, b, o, lane);
+    }
 }
 
 }  // namespace disco
