@@ -83,46 +83,89 @@ __device__ __forceinline__ unsigned long long key_from_words(float lo, float hi)
     return (static_cast<unsigned long long>(__float_as_uint(hi)) << 32) | __float_as_uint(lo);
 }
 
-// Merge up to 32 partial records (lane i takes record i, `stride` words apart) into one: every lane
-// returns the merged statistics and arg-max key, lane k < 10 the k-th largest logit.  The records may
-// live in shared or in global memory (volatile reads, so values written by other CTAs are fetched from
-// L2).  Deliberately small and not inlined: it runs a few times per launch, and every call after the
-// first finds its instructions in the instruction cache.
-static __device__ __noinline__ void warp_merge_records(const volatile float* recs, int n, int stride, SoftmaxState& st,
-                                                unsigned long long& key, float& sel) {
-    const int lane = threadIdx.x & 31;
-    const volatile float* mine = recs + (size_t)lane * stride;
-    st.init();
-    key = 0ull;
-    const bool have = lane < n && mine[1] > 0.f;
-    if (have) {
-        st.m = mine[0];
-        st.Z = mine[1];
-        st.S = mine[2];
-        key = key_from_words(mine[14], mine[15]);
+// One partial record held by a lane: statistics, arg-max key and a descending list of 16 values
+// (the ten logits of the record, then -inf).
+struct LaneRecord {
+    float m, Z, S;
+    unsigned long long key;
+    float l[16];
+    __device__ __forceinline__ void clear() {
+        m = DISCO_NEG_INF;
+        Z = 0.f;
+        S = 0.f;
+        key = 0ull;
+#pragma unroll
+        for (int k = 0; k < 16; ++k) l[k] = DISCO_NEG_INF;
+    }
+    __device__ __forceinline__ void set(const float4& q, const float4& a, const float4& b, const float4& c) {
+        clear();
+        if (q.y > 0.f) {
+            m = q.x, Z = q.y, S = q.z;
+            key = key_from_words(c.z, c.w);
+            l[0] = a.x, l[1] = a.y, l[2] = a.z, l[3] = a.w, l[4] = b.x, l[5] = b.y, l[6] = b.z, l[7] = b.w;
+            l[8] = c.x, l[9] = c.y;
+        }
+    }
+};
+
+// Reduce the records held by the lanes of a warp (lanes without one hold a cleared record).  Afterwards
+// the low lanes hold the merged statistics, the largest key and, in l[0..9], the ten largest logits.
+//   * statistics: one integer max-reduction for the reference maximum, one exponential per lane, then
+//     shuffle sums (much shorter than a butterfly of pairwise merges);
+//   * lists: a bitonic merge network across lanes: max(a[i], partner[15 - i]) keeps the 16 largest of
+//     two descending lists as a bitonic sequence, four compare-exchange stages sort it again.
+// `levels` = ceil(log2(number of lanes that may hold a record)); at least four levels run, so that
+// lanes 0..15 always end up with the result (lanes 0..11 are the ones that use it).
+__device__ __forceinline__ void warp_reduce_records(LaneRecord& r, int levels) {
+    levels = max(levels, 4);
+    const uint32_t mbits = __reduce_max_sync(kFullMask, ordered_bits(r.m));
+    const float M = from_ordered_bits(mbits);
+    float Zc = 0.f, Sc = 0.f;
+    if (r.Z > 0.f) {
+        const float dm = r.m - M;
+        const float e = __expf(dm);
+        Zc = r.Z * e;
+        Sc = e * (r.S + dm * r.Z);
     }
 #pragma unroll 1
-    for (int off = 16; off > 0; off >>= 1) {
-        const float m2 = __shfl_xor_sync(kFullMask, st.m, off);
-        const float Z2 = __shfl_xor_sync(kFullMask, st.Z, off);
-        const float S2 = __shfl_xor_sync(kFullMask, st.S, off);
-        const unsigned long long k2 = __shfl_xor_sync(kFullMask, key, off);
-        st.merge(m2, Z2, S2);
-        key = k2 > key ? k2 : key;
+    for (int lv = 0; lv < levels; ++lv) {
+        const int off = 1 << lv;
+        Zc += __shfl_xor_sync(kFullMask, Zc, off);
+        Sc += __shfl_xor_sync(kFullMask, Sc, off);
+        const unsigned long long k2 = __shfl_xor_sync(kFullMask, r.key, off);
+        r.key = k2 > r.key ? k2 : r.key;
+        float o[16];
+#pragma unroll
+        for (int i = 0; i < 16; ++i) o[i] = __shfl_xor_sync(kFullMask, r.l[15 - i], off);
+#pragma unroll
+        for (int i = 0; i < 16; ++i) r.l[i] = fmaxf(r.l[i], o[i]);
+#pragma unroll
+        for (int stride = 8; stride > 0; stride >>= 1) {
+#pragma unroll
+            for (int i = 0; i < 16; ++i) {
+                if ((i & stride) == 0) {
+                    const float hi = fmaxf(r.l[i], r.l[i + stride]);
+                    const float lo = fminf(r.l[i], r.l[i + stride]);
+                    r.l[i] = hi;
+                    r.l[i + stride] = lo;
+                }
+            }
+        }
     }
-    // each record's list is descending: ten rounds over the list heads
-    int head = 0;
-    sel = DISCO_NEG_INF;
-#pragma unroll 1
-    for (int r = 0; r < kTopK; ++r) {
-        const float hv = (have && head < kTopK) ? mine[4 + head] : DISCO_NEG_INF;
-        const uint32_t bits = ordered_bits(hv);
-        const uint32_t best = __reduce_max_sync(kFullMask, bits);
-        const unsigned who = __ballot_sync(kFullMask, bits == best);
-        if (lane == r) sel = from_ordered_bits(best);
-        if (lane == __ffs(who) - 1) ++head;
-    }
+    r.m = M;
+    r.Z = Zc;
+    r.S = Sc;
 }
+
+// The k-th largest logit for lane k < 10 (others: -inf) out of a reduced record.
+__device__ __forceinline__ float lane_pick(const LaneRecord& r, int lane) {
+    float sel = DISCO_NEG_INF;
+#pragma unroll
+    for (int k = 0; k < kTopK; ++k) sel = (lane == k) ? r.l[k] : sel;
+    return sel;
+}
+
+__device__ __forceinline__ int ceil_log2(int n) { return n <= 1 ? 0 : 32 - __clz(n - 1); }
 
 // Lane 0 holds (m, Z, S, key); lane k < 10 holds the k-th logit: write them as one record.
 __device__ __forceinline__ void warp_store_record(float* rec, const SoftmaxState& st, unsigned long long key, float sel,
@@ -136,6 +179,12 @@ __device__ __forceinline__ void warp_store_record(float* rec, const SoftmaxState
         rec[15] = __uint_as_float(static_cast<uint32_t>(key >> 32));
     }
     if (lane < kTopK) rec[4 + lane] = sel;
+}
+
+__device__ __forceinline__ void warp_store_record(float* rec, const LaneRecord& r, int lane) {
+    SoftmaxState st;
+    st.m = r.m, st.Z = r.Z, st.S = r.S;
+    warp_store_record(rec, st, r.key, lane_pick(r, lane), lane);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -198,27 +247,36 @@ __device__ void finalize_draft_row(const TailParams& p, int b, int grid, float* 
     constexpr int BAR_THREADS = NW * 32;
     const float fpos = static_cast<float>(p.pos[b]);  // issued early: hidden behind the merge
     const int n_drafted = p.n_drafted[b];
-    const float* recs = reinterpret_cast<const float*>(p.part_rec + (size_t)b * grid * 4);
-    SoftmaxState st;
-    unsigned long long key;
-    float sel;
+    const float4* recs = p.part_rec + (size_t)b * grid * 4;
+    LaneRecord r;
     for (int base = 0; base < grid; base += 32 * NW) {
-        const int c0 = base + warp * 32;
-        const int n = max(0, min(32, grid - c0));
-        warp_merge_records(recs + (size_t)c0 * kRecordWords, n, kRecordWords, st, key, sel);
-        warp_store_record(stage + warp * kRecordWords, st, key, sel, lane);
+        const int c = base + warp * 32 + lane;
+        r.clear();
+        if (c < grid) {  // one L2 round trip per lane: the four quarters of its record
+            const float4* src = recs + (size_t)c * 4;
+            const float4 q0 = __ldcg(src), q1 = __ldcg(src + 1), q2 = __ldcg(src + 2), q3 = __ldcg(src + 3);
+            r.set(q0, q1, q2, q3);
+        }
+        warp_reduce_records(r, 5);
+        warp_store_record(stage + warp * kRecordWords, r, lane);
         named_barrier_sync(1, BAR_THREADS);
         if (warp == 0) {
-            warp_merge_records(stage, base == 0 ? NW : NW + 1, kRecordWords, st, key, sel);
-            if (base + 32 * NW < grid) warp_store_record(stage + NW * kRecordWords, st, key, sel, lane);  // carry
+            const int n = base == 0 ? NW : NW + 1;
+            const float4* sr = reinterpret_cast<const float4*>(stage) + lane * 4;
+            r.clear();
+            if (lane < n) r.set(sr[0], sr[1], sr[2], sr[3]);
+            warp_reduce_records(r, ceil_log2(n));
+            if (base + 32 * NW < grid) warp_store_record(stage + NW * kRecordWords, r, lane);  // carry
         }
         named_barrier_sync(1, BAR_THREADS);
     }
     if (warp == 0) {
         const int Hc = p.clf_H;
+        SoftmaxState st;
+        st.m = r.m, st.Z = r.Z, st.S = r.S;
         const DraftOutputs o{p.token, p.conf, p.halt, p.feats, p.final_stats};
-        warp_draft_epilogue(st, key, sel, fpos, n_drafted, p.tau, p.sl_max, feat_s, clf_s, clf_s + Hc * kNFeat,
-                            clf_s + Hc * (kNFeat + 1), clf_s + Hc * (kNFeat + 2), Hc, b, o, lane);
+        warp_draft_epilogue(st, r.key, lane_pick(r, lane), fpos, n_drafted, p.tau, p.sl_max, feat_s, clf_s,
+                            clf_s + Hc * kNFeat, clf_s + Hc * (kNFeat + 1), clf_s + Hc * (kNFeat + 2), Hc, b, o, lane);
     }
     named_barrier_sync(1, BAR_THREADS);
 }
@@ -483,12 +541,14 @@ __global__ void __launch_bounds__((NW + 1) * 32, 1) stream_tail_kernel(const __g
                 const int row = chunk * RT + r;
                 if (row >= p.R) continue;
                 // the records of hidden row r sit RT records apart; lane w < NW takes warp w's
-                SoftmaxState g;
-                unsigned long long key;
-                float sel;
-                warp_merge_records(wstate + r * kRecordWords, NW, RT * kRecordWords, g, key, sel);
-                warp_store_record(reinterpret_cast<float*>(p.part_rec + ((size_t)row * grid + blockIdx.x) * 4), g, key,
-                                  sel, lane);
+                LaneRecord rec;
+                rec.clear();
+                if (lane < NW) {
+                    const float4* sr = reinterpret_cast<const float4*>(wstate + (lane * RT + r) * kRecordWords);
+                    rec.set(sr[0], sr[1], sr[2], sr[3]);
+                }
+                warp_reduce_records(rec, ceil_log2(NW));
+                warp_store_record(reinterpret_cast<float*>(p.part_rec + ((size_t)row * grid + blockIdx.x) * 4), rec, lane);
             }
         } else {
             unsigned long long* keys_s = reinterpret_cast<unsigned long long*>(wstate);

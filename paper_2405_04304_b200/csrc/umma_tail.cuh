@@ -419,27 +419,35 @@ __global__ void __launch_bounds__(kDraftFinalWarps * 32) draft_finalize_kernel(c
     if (p.active && !p.active[b]) return;
     const float fpos = static_cast<float>(p.pos[b]);
     const int n_drafted = p.n_drafted[b];
-    const float* recs = reinterpret_cast<const float*>(p.part_rec + (size_t)b * p.NP * 4);
-    SoftmaxState st;
-    unsigned long long key;
-    float sel;
+    const float4* recs = p.part_rec + (size_t)b * p.NP * 4;
+    LaneRecord r;
     for (int base = 0; base < p.NP; base += 32 * kDraftFinalWarps) {
-        const int c0 = base + warp * 32;
-        const int n = max(0, min(32, p.NP - c0));
-        warp_merge_records(recs + (size_t)c0 * kRecordWords, n, kRecordWords, st, key, sel);
-        warp_store_record(stage + warp * kRecordWords, st, key, sel, lane);
+        const int c = base + warp * 32 + lane;
+        r.clear();
+        if (c < p.NP) {
+            const float4* src = recs + (size_t)c * 4;
+            const float4 q0 = __ldcg(src), q1 = __ldcg(src + 1), q2 = __ldcg(src + 2), q3 = __ldcg(src + 3);
+            r.set(q0, q1, q2, q3);
+        }
+        warp_reduce_records(r, 5);
+        warp_store_record(stage + warp * kRecordWords, r, lane);
         __syncthreads();
         if (warp == 0) {
-            warp_merge_records(stage, base == 0 ? kDraftFinalWarps : kDraftFinalWarps + 1, kRecordWords, st, key, sel);
-            if (base + 32 * kDraftFinalWarps < p.NP)
-                warp_store_record(stage + kDraftFinalWarps * kRecordWords, st, key, sel, lane);
+            const int n = base == 0 ? kDraftFinalWarps : kDraftFinalWarps + 1;
+            const float4* sr = reinterpret_cast<const float4*>(stage) + lane * 4;
+            r.clear();
+            if (lane < n) r.set(sr[0], sr[1], sr[2], sr[3]);
+            warp_reduce_records(r, ceil_log2(n));
+            if (base + 32 * kDraftFinalWarps < p.NP) warp_store_record(stage + kDraftFinalWarps * kRecordWords, r, lane);
         }
         __syncthreads();
     }
     if (warp == 0) {
+        SoftmaxState st;
+        st.m = r.m, st.Z = r.Z, st.S = r.S;
         const DraftOutputs o{p.token, p.conf, p.halt, p.feats, p.final_stats};
-        warp_draft_epilogue(st, key, sel, fpos, n_drafted, p.tau, p.sl_max, feat_s, p.clf_W1, p.clf_b1, p.clf_w2,
-                            p.clf_b2, p.clf_H, b, o, lane);
+        warp_draft_epilogue(st, r.key, lane_pick(r, lane), fpos, n_drafted, p.tau, p.sl_max, feat_s, p.clf_W1, p.clf_b1,
+                            p.clf_w2, p.clf_b2, p.clf_H, b, o, lane);
     }
 }
 
