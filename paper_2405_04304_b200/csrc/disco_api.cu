@@ -173,8 +173,9 @@ bool umma_possible(const disco_ctx* c, int R) {
 // Launch the tcgen05 kernel for R hidden rows of width d against the LM head W [V, d].
 template <bool DRAFT>
 int launch_umma(disco_ctx* c, const void* W, const void* H, int d, int R, float* probs, int* n_partials,
-                cudaStream_t st) {
+                const UmmaParams* fused, cudaStream_t st) {
     UmmaParams p{};
+    if (fused) p = *fused;  // verification finished by the main kernel's last CTA
     p.V = c->V;
     p.d = d;
     p.R = R;
@@ -201,9 +202,19 @@ int launch_umma(disco_ctx* c, const void* W, const void* H, int d, int R, float*
             return DISCO_ERR_CUDA;
         configured_dev = c->device;
     }
-    kern<<<p.MT * p.CN, kUmmaThreads, kUmmaSmemBytes, st>>>(tmap_W, tmap_H, p);
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3((unsigned)(p.MT * p.CN));
+    cfg.blockDim = dim3(kUmmaThreads);
+    cfg.dynamicSmemBytes = kUmmaSmemBytes;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = c->pdl ? 1 : 0;
+    const cudaError_t e = cudaLaunchKernelEx(&cfg, kern, tmap_W, tmap_H, p);
     c->launches += 1;
-    return cuda_ok(cudaGetLastError(), "umma_tail_kernel launch") ? DISCO_OK : DISCO_ERR_CUDA;
+    return cuda_ok(e, "umma_tail_kernel launch") ? DISCO_OK : DISCO_ERR_CUDA;
 }
 
 void fill_scratch(const disco_ctx* c, TailParams& p) {
@@ -379,7 +390,7 @@ int disco_draft_step(disco_ctx* c, const void* W_D, const void* h_D, int B, cons
     const bool use_umma = umma_possible(c, B) && (c->path == 2 || (c->path == 0 && B >= 2));
     if (use_umma) {
         int np = 0;
-        rc = launch_umma<true>(c, W_D, h_D, c->d_draft, B, probs, &np, st);
+        rc = launch_umma<true>(c, W_D, h_D, c->d_draft, B, probs, &np, nullptr, st);
         if (rc) return rc;
         DraftFinalParams f{};
         f.part_rec = reinterpret_cast<const float4*>(c->part_rec);
@@ -442,7 +453,20 @@ int disco_verify_ragged(disco_ctx* c, const void* W_T, const void* H_T, const in
     p.target_ids = target_ids;
     const bool use_umma = umma_possible(c, R) && (c->path == 2 || (c->path == 0 && R >= 2));
     if (!use_umma) return run_stream<false>(c, p, 0, st);
-    int rc = launch_umma<false>(c, W_T, H_T, c->d_target, R, nullptr, nullptr, st);
+    if (B <= 16) {  // few sequences: the last CTA of the main kernel finishes the job, no second launch
+        UmmaParams fp{};
+        fp.fuse_final = 1;
+        fp.ticket = c->ticket + 32;
+        fp.draft_ids = draft_ids;
+        fp.row_off = row_off;
+        fp.B = B;
+        fp.SL = p.SL;
+        fp.n_accept = n_accept;
+        fp.bonus = bonus;
+        fp.target_ids = target_ids;
+        return launch_umma<false>(c, W_T, H_T, c->d_target, R, nullptr, nullptr, &fp, st);
+    }
+    int rc = launch_umma<false>(c, W_T, H_T, c->d_target, R, nullptr, nullptr, nullptr, st);
     if (rc) return rc;
     VerifyFinalParams f{};
     f.keys = c->keys;

@@ -51,6 +51,15 @@ struct UmmaParams {
     // draft step
     float4* part_rec;   // [R][CN] records of 64 bytes: (m, Z, S, -), top-10 logits descending, arg-max key
     float* probs;       // optional [R][V]: raw logits are written here
+    // verification finished inside this kernel by the last CTA (few sequences only)
+    int fuse_final;
+    unsigned int* ticket;
+    const int32_t* draft_ids;
+    const int32_t* row_off;
+    int B, SL;
+    int32_t* n_accept;
+    int32_t* bonus;
+    int32_t* target_ids;
 };
 
 // ---------------------------------------------------------------------------------------------
@@ -145,6 +154,10 @@ umma_tail_kernel(const __grid_constant__ CUtensorMap tmap_W, const __grid_consta
     uint32_t* tmem_base_s = reinterpret_cast<uint32_t*>(tmem_empty + 2);
     float4* xch = reinterpret_cast<float4*>(reinterpret_cast<uint8_t*>(full) + 256);
 
+    // the next kernel of the stream may begin its prologue; this one touches what its predecessor may
+    // have written (hidden states, scratch) only after griddepcontrol.wait
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
     const int m_tile = blockIdx.x % p.MT;
@@ -178,14 +191,31 @@ umma_tail_kernel(const __grid_constant__ CUtensorMap tmap_W, const __grid_consta
         if (lane == 0) {
             int stage = 0, phase = 0;
             const uint32_t bytes = (uint32_t)(p.a_rows + p.TRN) * 128u;
+            // The LM head is never written by this library: its first tiles are requested before the
+            // dependency wait, the hidden-state tiles of the same stages right after it.
+            int pre = 0;
+            {
+                const int v0 = nslot * p.TPC * p.TR;
+                if (v0 < p.V) {
+                    pre = min(kUmmaStages, KB);
+                    for (int kb = 0; kb < pre; ++kb) {
+                        mbar_arrive_expect_tx(&full[kb], bytes);
+                        tma_load_2d(b_tiles + kb * kUmmaBTileBytes, &tmap_W, kb * kUmmaBK, v0, &full[kb]);
+                    }
+                }
+            }
+            asm volatile("griddepcontrol.wait;" ::: "memory");
+            int n = 0;
             for (int i = 0; i < p.TPC; ++i) {
                 const int v0 = (nslot * p.TPC + i) * p.TR;
                 if (v0 >= p.V) break;
-                for (int kb = 0; kb < KB; ++kb) {
-                    mbar_wait(&empty[stage], phase ^ 1, p.status);
-                    mbar_arrive_expect_tx(&full[stage], bytes);
+                for (int kb = 0; kb < KB; ++kb, ++n) {
+                    if (n >= pre) {
+                        mbar_wait(&empty[stage], phase ^ 1, p.status);
+                        mbar_arrive_expect_tx(&full[stage], bytes);
+                        tma_load_2d(b_tiles + stage * kUmmaBTileBytes, &tmap_W, kb * kUmmaBK, v0, &full[stage]);
+                    }
                     tma_load_2d(a_tiles + stage * kUmmaATileBytes, &tmap_H, kb * kUmmaBK, m_tile * 128, &full[stage]);
-                    tma_load_2d(b_tiles + stage * kUmmaBTileBytes, &tmap_W, kb * kUmmaBK, v0, &full[stage]);
                     if (++stage == kUmmaStages) {
                         stage = 0;
                         phase ^= 1;
@@ -224,6 +254,7 @@ umma_tail_kernel(const __grid_constant__ CUtensorMap tmap_W, const __grid_consta
         }
     } else {
         // ------------------------------ epilogue ------------------------------
+        asm volatile("griddepcontrol.wait;" ::: "memory");  // scratch and outputs belong to the predecessor until now
         const int ew = warp - 2;            // 0 .. kUmmaEpiWarps-1
         const int quad = warp & 3;          // TMEM lane quadrant this warp may read
         const int half = ew >> 2;           // which share of the columns (two warps per quadrant)
@@ -337,6 +368,23 @@ umma_tail_kernel(const __grid_constant__ CUtensorMap tmap_W, const __grid_consta
             }
         } else {
             if (valid && best_i != kNoIndex) atomicMax(p.keys + row, argmax_key(best_v, best_i));
+            if (p.fuse_final) {
+                // ticket: the last CTA to get here matches the prefixes and clears the keys
+                __shared__ int s_last;
+                __threadfence();
+                named_barrier_sync(2, kUmmaEpiWarps * 32);
+                if (ew == 0 && lane == 0) s_last = atomicAdd(p.ticket, 1u) == gridDim.x - 1;
+                named_barrier_sync(2, kUmmaEpiWarps * 32);
+                if (s_last) {
+                    __threadfence();
+                    for (int b = ew; b < p.B; b += kUmmaEpiWarps)
+                        verify_one_sequence(p.keys, p.draft_ids, p.row_off, p.B, p.SL, p.R, b, p.n_accept, p.bonus,
+                                            p.target_ids, p.status, lane);
+                    named_barrier_sync(2, kUmmaEpiWarps * 32);
+                    for (int r = ew * 32 + lane; r < p.R; r += kUmmaEpiWarps * 32) p.keys[r] = 0ull;
+                    if (ew == 0 && lane == 0) *p.ticket = 0u;
+                }
+            }
         }
     }
 
