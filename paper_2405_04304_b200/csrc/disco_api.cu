@@ -64,6 +64,11 @@ inline bool cuda_ok(cudaError_t e, const char* what) {
     return false;
 }
 
+inline int getenv_int(const char* name, int dflt) {
+    const char* e = std::getenv(name);
+    return e ? std::atoi(e) : dflt;
+}
+
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 StreamPlan plan_stream(const disco_ctx* c, int V, int d, int RT, int clf_H) {
@@ -181,10 +186,19 @@ int launch_umma(disco_ctx* c, const void* W, const void* H, int d, int R, float*
     p.R = R;
     p.MT = (R + 127) / 128;
     p.CN = c->sm_count / p.MT;
-    p.TPC = std::max(1, (c->V + 256 * p.CN - 1) / (256 * p.CN));
+    // Vocabulary rows per tile: up to 256 for verification (its epilogue is a compare per logit); the
+    // draft step's epilogue is heavy (soft-max, top-10), so it gets several small tiles per CTA and
+    // the epilogue of one tile runs under the loads of the next.
+    const int tile_target = DRAFT ? (getenv_int("DISCO_DRAFT_TILE", 64)) : 256;
+    p.TPC = std::max(1, (c->V + tile_target * p.CN - 1) / (tile_target * p.CN));
     p.TR = (c->V + p.CN * p.TPC - 1) / (p.CN * p.TPC);
     p.TRN = std::max(16, (p.TR + 15) / 16 * 16);
     p.a_rows = p.MT > 1 ? 128 : std::max(8, (R + 7) / 8 * 8);
+    // The A stage holds a_rows rows.  The MMA still reads 128 rows from its start: what lies behind the
+    // tile (other stages of the ring, always inside it) only feeds accumulator lanes nobody reads.
+    p.a_bytes = (p.a_rows * 128 + 1023) / 1024 * 1024;
+    p.b_bytes = (p.TRN * 128 + 1023) / 1024 * 1024;
+    p.stages = std::max(2, std::min(kUmmaMaxStages, kUmmaRingBytes / (p.a_bytes + p.b_bytes)));
     p.status = c->status;
     p.keys = c->keys;
     p.part_rec = reinterpret_cast<float4*>(c->part_rec);

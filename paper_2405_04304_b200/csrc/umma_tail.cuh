@@ -27,15 +27,14 @@
 
 namespace disco {
 
-constexpr int kUmmaStages = 4;
+constexpr int kUmmaMaxStages = 16;
 constexpr int kUmmaBK = 64;               // k elements per stage (one 128-byte swizzle span)
-constexpr int kUmmaATileBytes = 128 * 128;  // 128 rows x 128 B
-constexpr int kUmmaBTileBytes = 256 * 128;  // 256 rows x 128 B
+constexpr int kUmmaRingBytes = 192 * 1024;  // shared memory for the operand stages
 constexpr int kUmmaEpiWarps = 8;
 constexpr int kUmmaThreads = (2 + kUmmaEpiWarps) * 32;
 constexpr int kUmmaXchBytes = 128 * 16 * 4;  // one 64-byte record per hidden row of the tile
 constexpr int kUmmaSmemBytes =
-    kUmmaStages * (kUmmaATileBytes + kUmmaBTileBytes) + 1024 /*align*/ + 256 /*barriers*/ + kUmmaXchBytes;
+    kUmmaRingBytes + 1024 /*align*/ + 512 /*barriers*/ + kUmmaXchBytes;
 
 struct UmmaParams {
     int V, d, R;
@@ -45,6 +44,8 @@ struct UmmaParams {
     int TR;      // vocabulary rows per tile; the MMA and the TMA box use TRN = TR rounded up to 16
     int TRN;
     int a_rows;  // rows of the H box (multiple of 8, <= 128)
+    int stages;  // ring depth (<= kUmmaMaxStages); stage s holds an A tile of a_bytes and a B tile of b_bytes
+    int a_bytes, b_bytes;  // multiples of 1024
     int* status;
     // verification
     unsigned long long* keys;  // [R]
@@ -146,13 +147,13 @@ umma_tail_kernel(const __grid_constant__ CUtensorMap tmap_W, const __grid_consta
     extern __shared__ uint8_t smem_dyn[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~uintptr_t(1023));
     uint8_t* a_tiles = smem;
-    uint8_t* b_tiles = smem + kUmmaStages * kUmmaATileBytes;
-    uint64_t* full = reinterpret_cast<uint64_t*>(b_tiles + kUmmaStages * kUmmaBTileBytes);
-    uint64_t* empty = full + kUmmaStages;
-    uint64_t* tmem_full = empty + kUmmaStages;
+    uint8_t* b_tiles = smem + p.stages * p.a_bytes;
+    uint64_t* full = reinterpret_cast<uint64_t*>(smem + kUmmaRingBytes);
+    uint64_t* empty = full + kUmmaMaxStages;
+    uint64_t* tmem_full = empty + kUmmaMaxStages;
     uint64_t* tmem_empty = tmem_full + 2;
     uint32_t* tmem_base_s = reinterpret_cast<uint32_t*>(tmem_empty + 2);
-    float4* xch = reinterpret_cast<float4*>(reinterpret_cast<uint8_t*>(full) + 256);
+    float4* xch = reinterpret_cast<float4*>(reinterpret_cast<uint8_t*>(full) + 512);
 
     // the next kernel of the stream may begin its prologue; this one touches what its predecessor may
     // have written (hidden states, scratch) only after griddepcontrol.wait
@@ -165,7 +166,7 @@ umma_tail_kernel(const __grid_constant__ CUtensorMap tmap_W, const __grid_consta
     const int KB = (p.d + kUmmaBK - 1) / kUmmaBK;
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < kUmmaStages; ++s) {
+        for (int s = 0; s < p.stages; ++s) {
             mbar_init(&full[s], 1);
             mbar_init(&empty[s], 1);
         }
@@ -197,10 +198,10 @@ umma_tail_kernel(const __grid_constant__ CUtensorMap tmap_W, const __grid_consta
             {
                 const int v0 = nslot * p.TPC * p.TR;
                 if (v0 < p.V) {
-                    pre = min(kUmmaStages, KB);
+                    pre = min(p.stages, KB);
                     for (int kb = 0; kb < pre; ++kb) {
                         mbar_arrive_expect_tx(&full[kb], bytes);
-                        tma_load_2d(b_tiles + kb * kUmmaBTileBytes, &tmap_W, kb * kUmmaBK, v0, &full[kb]);
+                        tma_load_2d(b_tiles + kb * p.b_bytes, &tmap_W, kb * kUmmaBK, v0, &full[kb]);
                     }
                 }
             }
@@ -213,10 +214,10 @@ umma_tail_kernel(const __grid_constant__ CUtensorMap tmap_W, const __grid_consta
                     if (n >= pre) {
                         mbar_wait(&empty[stage], phase ^ 1, p.status);
                         mbar_arrive_expect_tx(&full[stage], bytes);
-                        tma_load_2d(b_tiles + stage * kUmmaBTileBytes, &tmap_W, kb * kUmmaBK, v0, &full[stage]);
+                        tma_load_2d(b_tiles + stage * p.b_bytes, &tmap_W, kb * kUmmaBK, v0, &full[stage]);
                     }
-                    tma_load_2d(a_tiles + stage * kUmmaATileBytes, &tmap_H, kb * kUmmaBK, m_tile * 128, &full[stage]);
-                    if (++stage == kUmmaStages) {
+                    tma_load_2d(a_tiles + stage * p.a_bytes, &tmap_H, kb * kUmmaBK, m_tile * 128, &full[stage]);
+                    if (++stage == p.stages) {
                         stage = 0;
                         phase ^= 1;
                     }
@@ -237,13 +238,13 @@ umma_tail_kernel(const __grid_constant__ CUtensorMap tmap_W, const __grid_consta
                 for (int kb = 0; kb < KB; ++kb) {
                     mbar_wait(&full[stage], phase, p.status);
                     tc_fence_after();
-                    const uint64_t a_desc = umma_smem_desc(a_tiles + stage * kUmmaATileBytes);
-                    const uint64_t b_desc = umma_smem_desc(b_tiles + stage * kUmmaBTileBytes);
+                    const uint64_t a_desc = umma_smem_desc(a_tiles + stage * p.a_bytes);
+                    const uint64_t b_desc = umma_smem_desc(b_tiles + stage * p.b_bytes);
 #pragma unroll
                     for (int k = 0; k < kUmmaBK / 16; ++k)  // 16 k-elements = 32 bytes = 2 descriptor units
                         tc_mma_bf16(d_tmem, a_desc + 2 * k, b_desc + 2 * k, idesc, (kb | k) != 0);
                     tc_commit(&empty[stage]);
-                    if (++stage == kUmmaStages) {
+                    if (++stage == p.stages) {
                         stage = 0;
                         phase ^= 1;
                     }
