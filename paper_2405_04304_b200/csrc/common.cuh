@@ -193,26 +193,59 @@ __device__ __forceinline__ void warp_merge_softmax(SoftmaxState& st) {
     }
 }
 
-// The ten largest values offered so far, kept by one warp: lane l < 10 holds the l-th largest.
-// Offered values must be warp-uniform.
-struct WarpTopV {
-    float v;
-    float floor_v;  // warp-uniform copy of entry 9
-    __device__ __forceinline__ void init() {
-        v = DISCO_NEG_INF;
-        floor_v = DISCO_NEG_INF;
+// A block of up to 32 logits of one hidden row, one per lane (lanes >= n hold -inf), folded into the
+// warp's running state in one go: soft-max statistics by an integer max-reduction, one exponential per
+// lane and shuffle sums; arg-max by a ballot (lanes hold ascending vocabulary indices, so the lowest
+// lane wins ties); top-10 by rank counting (every candidate counts how many others beat it and writes
+// itself to that position).  top_v: lane k < 10 holds the k-th largest value so far.  scratch: 10
+// floats of shared memory owned by the warp.
+__device__ __forceinline__ void warp_fold_block(float val, int idx, int n, int lane, SoftmaxState& st, float& best_v,
+                                                int& best_i, float& top_v, float* scratch) {
+    const uint32_t bits = ordered_bits(val);
+    const uint32_t mbits = __reduce_max_sync(kFullMask, bits);
+    const float M = from_ordered_bits(mbits);
+    // arg-max of the block
+    const int lead = __ffs(__ballot_sync(kFullMask, bits == mbits)) - 1;
+    const int lead_idx = __shfl_sync(kFullMask, idx, lead);
+    if (M > best_v) {
+        best_v = M;
+        best_i = lead_idx;
     }
-    __device__ __forceinline__ void offer(float z, int lane) {
-        if (z > floor_v) {
-            const unsigned ahead = __ballot_sync(kFullMask, lane < kTopK && v >= z);
-            const int p = __popc(ahead);
-            const float up_v = __shfl_up_sync(kFullMask, v, 1);
-            if (lane > p) v = up_v;
-            else if (lane == p) v = z;
-            floor_v = __shfl_sync(kFullMask, v, kTopK - 1);
-        }
+    // statistics of the block, then merged into the running state
+    float e = 0.f, et = 0.f;
+    if (lane < n) {
+        const float t = val - M;
+        e = __expf(t);
+        et = e * t;
     }
-};
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) {
+        e += __shfl_xor_sync(kFullMask, e, off);
+        et += __shfl_xor_sync(kFullMask, et, off);
+    }
+    st.merge(M, e, et);
+    // ranks among the block's candidates and the ten values kept so far (which win ties)
+    const float old_v = top_v;  // lanes >= 10 hold -inf
+    int rank_new = 0, rank_old = lane;
+#pragma unroll 8
+    for (int k = 0; k < 32; ++k) {
+        const float vk = __shfl_sync(kFullMask, val, k);
+        rank_new += (vk > val) || (vk == val && k < lane);
+        rank_old += vk > old_v;
+    }
+#pragma unroll
+    for (int k = 0; k < kTopK; ++k) {
+        const float ok = __shfl_sync(kFullMask, old_v, k);
+        rank_new += ok >= val;
+    }
+    if (lane < kTopK) scratch[lane] = DISCO_NEG_INF;  // positions nobody claims stay empty
+    __syncwarp();
+    if (lane < n && rank_new < kTopK) scratch[rank_new] = val;
+    if (lane < kTopK && old_v > DISCO_NEG_INF && rank_old < kTopK) scratch[rank_old] = old_v;
+    __syncwarp();
+    top_v = lane < kTopK ? scratch[lane] : DISCO_NEG_INF;
+    __syncwarp();
+}
 
 // Ten largest values seen so far, descending, in the registers of one thread.
 struct RegTop10 {

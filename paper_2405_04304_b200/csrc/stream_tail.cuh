@@ -420,17 +420,22 @@ __global__ void __launch_bounds__((NW + 1) * 32, 1) stream_tail_kernel(const __g
         }
         named_barrier_sync(1, BAR_THREADS);
 
+        // Running state of this warp per hidden row, and the block of logits not folded into it yet:
+        // the warp-uniform logit of the cnt-th vocabulary row this warp meets is parked in lane cnt % 32.
         SoftmaxState st[RT];
-        WarpTopV top[RT];
-        float best_v[RT];
+        float top_v[RT], best_v[RT], blk_v[RT];
         int best_i[RT];
+        int blk_idx = 0, cnt = 0;
 #pragma unroll
         for (int r = 0; r < RT; ++r) {
             st[r].init();
-            top[r].init();
+            top_v[r] = DISCO_NEG_INF;
             best_v[r] = DISCO_NEG_INF;
             best_i[r] = kNoIndex;
+            blk_v[r] = DISCO_NEG_INF;
         }
+        // scratch for the rank scatter: the warp's record slots (written for good only after the loop)
+        float* fold_scratch = wstate + (warp * RT) * kRecordWords + 4;
 
         // With one hidden row and a narrow head the warp keeps its share of h in registers.
         float hreg[KC > 0 ? KC : 1][8];
@@ -508,18 +513,21 @@ __global__ void __launch_bounds__((NW + 1) * 32, 1) stream_tail_kernel(const __g
                     for (int g = 0; g < G; ++g) {
                         if (j0 + g >= nr) break;
                         const int v = v0 + r0 + j0 + g;
+                        const bool mine = lane == (cnt & 31);
+                        if (mine) blk_idx = v;
 #pragma unroll
                         for (int r = 0; r < RT; ++r) {
                             const float z = __fadd_rn(acc[g][r], 0.f);  // folds -0 into +0
-                            if (z > best_v[r]) {  // rows arrive in ascending order: the lowest index wins ties
-                                best_v[r] = z;
-                                best_i[r] = v;
-                            }
-                            if (DRAFT) {
-                                st[r].push(z);
-                                top[r].offer(z, lane);
-                                if (p.probs && lane == 0 && chunk * RT + r < p.R)
-                                    p.probs[(size_t)(chunk * RT + r) * p.V + v] = z;
+                            if (mine) blk_v[r] = z;
+                            if (DRAFT && p.probs && lane == 0 && chunk * RT + r < p.R)
+                                p.probs[(size_t)(chunk * RT + r) * p.V + v] = z;
+                        }
+                        if ((++cnt & 31) == 0) {  // 32 logits parked: fold them
+#pragma unroll
+                            for (int r = 0; r < RT; ++r) {
+                                warp_fold_block(blk_v[r], blk_idx, 32, lane, st[r], best_v[r], best_i[r], top_v[r],
+                                                fold_scratch + r * kRecordWords);
+                                blk_v[r] = DISCO_NEG_INF;
                             }
                         }
                     }
@@ -529,12 +537,19 @@ __global__ void __launch_bounds__((NW + 1) * 32, 1) stream_tail_kernel(const __g
             }
         }
 
+        if (cnt & 31) {  // the last, partial block
+#pragma unroll
+            for (int r = 0; r < RT; ++r)
+                warp_fold_block(blk_v[r], blk_idx, cnt & 31, lane, st[r], best_v[r], best_i[r], top_v[r],
+                                fold_scratch + r * kRecordWords);
+        }
+
         // ---- merge the NW warps of this CTA, publish the CTA's result for each hidden row ----
         if (DRAFT) {
 #pragma unroll
             for (int r = 0; r < RT; ++r) {
                 const unsigned long long key = best_i[r] != kNoIndex ? argmax_key(best_v[r], best_i[r]) : 0ull;
-                warp_store_record(wstate + (warp * RT + r) * kRecordWords, st[r], key, top[r].v, lane);
+                warp_store_record(wstate + (warp * RT + r) * kRecordWords, st[r], key, top_v[r], lane);
             }
             named_barrier_sync(1, BAR_THREADS);
             for (int r = warp; r < RT; r += NW) {
