@@ -298,3 +298,79 @@ def test_verify_on_each_kernel_path(oracle, path, V, d, sls):
         np.testing.assert_array_equal(got[k], got2[k])
     assert ctx.device_status() == 0
     ctx.close()
+
+
+# ---------------------------------------------------------------------------------- full-size batched workloads
+def _prefix_rule(draft, target_rows):
+    n = 0
+    while n < len(draft) and draft[n] == target_rows[n]:
+        n += 1
+    return n, target_rows[n]
+
+
+@pytest.mark.parametrize("name,n_sample", [("vicuna_b64", 48), ("starcoder_b256", 32)])
+def test_batched_verification_at_full_size(oracle, name, n_sample):
+    """The launch configuration bench.py times (ragged rows over the whole LM head).  The oracle projects a
+    sample of rows one by one; every sequence is checked against the prefix rule applied to the ids the
+    library itself reported."""
+    wl = inputs.WORKLOADS[name]
+    B, S = wl.B, wl.sl_max
+    if wl.sl_mode == "uniform":
+        sl = inputs.uniform_sl(B, 1, S, inputs.sub_seed(wl.seed, 8))
+    else:
+        sl = torch.full((B,), S, dtype=torch.int32)
+    off = inputs.row_offsets(sl).numpy()
+    R = int(off[-1])
+    W = inputs.lm_head(wl.V, wl.d_T, seed=inputs.sub_seed(wl.seed, 2))
+    H = inputs.hidden(R, wl.d_T, seed=inputs.sub_seed(wl.seed, 5))
+    rng = np.random.default_rng(wl.seed)
+    draft = rng.integers(0, wl.V, size=R - B).astype(np.int32)
+    rows = np.sort(rng.choice(R, size=n_sample, replace=False))
+    z = oracle.project(_bits(W), _bits(H[torch.from_numpy(rows)]), nthreads=16)
+    want = [oracle.argmax(z[i]) for i in range(n_sample)]
+    # make some sampled rows "accepted": the draft id at that position equals the oracle's target id
+    row_seq = np.searchsorted(off, rows, side="right") - 1
+    for (r, b), (tok, gap) in zip(zip(rows, row_seq), want):
+        j = r - off[b]
+        if j < sl[b]:
+            draft[off[b] - b + j] = tok
+    ctx = binding.Context(wl.V, wl.d_D, wl.d_T, max_batch=B, max_rows=R)
+    Wg = W.cuda()
+    got = gpu_verify(ctx, Wg, H, draft, row_off=off)
+    assert ctx.device_status() == 0
+    tid = got["target_ids"]
+    exempt = 0
+    for r, (tok, gap) in zip(rows, want):
+        if gap < 1e-3:
+            exempt += 1
+            continue
+        assert tid[r] == tok, f"row {r}: target id {tid[r]} != oracle {tok}"
+    assert exempt <= 2
+    assert np.all((tid >= 0) & (tid < wl.V))
+    for b in range(B):
+        n, bonus = _prefix_rule(draft[off[b] - b: off[b + 1] - b - 1], tid[off[b]:off[b + 1]])
+        assert got["n_accept"][b] == n and got["bonus"][b] == bonus
+    got2 = gpu_verify(ctx, Wg, H, draft, row_off=off)            # deterministic, scratch left clean
+    for k in ("n_accept", "bonus", "target_ids"):
+        np.testing.assert_array_equal(got[k], got2[k])
+    ctx.close()
+
+
+@pytest.mark.parametrize("name", ["vicuna_b64", "starcoder_b256"])
+def test_batched_draft_step_at_full_size(oracle, name):
+    wl = inputs.WORKLOADS[name]
+    B = wl.B
+    W = inputs.lm_head(wl.V, wl.d_D, seed=inputs.sub_seed(wl.seed, 1))
+    h = inputs.hidden(B, wl.d_D, seed=inputs.sub_seed(wl.seed, 4))
+    params = make_clf(wl.H, seed=inputs.sub_seed(wl.seed, 3))
+    pos = (np.arange(B, dtype=np.int32) * 13) % 97 + 1
+    nd = (np.arange(B, dtype=np.int32) % wl.sl_max) + 1
+    active = (np.arange(B) % 5 != 2).astype(np.uint8)
+    ctx = _ctx(wl.V, wl.d_D, wl.d_T, max_batch=B, H=wl.H)
+    got = gpu_draft_step(ctx, W.cuda(), h, pos, nd, to_gpu_clf(params), wl.tau, wl.sl_max, active=active)
+    ref = oracle.draft_step(_bits(W), _bits(h), pos, nd, to_oracle_clf(oracle, params), wl.tau, wl.sl_max,
+                            active=active, nthreads=16)
+    exempt = check_draft(got, ref, wl.tau, active=active)
+    assert exempt <= max(2, B // 50)
+    assert ctx.device_status() == 0
+    ctx.close()
