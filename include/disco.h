@@ -87,7 +87,8 @@ int disco_last_device_status(disco_ctx* ctx, int* out);
 int disco_launch_count(disco_ctx* ctx, long long* out);
 
 /* Kernel selection (tuning and tests): which = 0 automatic (default), 1 force the CUDA-core
- * streaming kernels, 2 force the tcgen05 kernels where the shape allows them. */
+ * streaming kernels, 2 force the tcgen05 kernels with the hidden rows on the TMEM lanes, 3 prefer the
+ * tcgen05 kernel with the vocabulary on the TMEM lanes (draft step, up to 16 sequences). */
 int disco_set_kernel_path(disco_ctx* ctx, int which);
 
 /*

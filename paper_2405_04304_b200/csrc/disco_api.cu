@@ -11,6 +11,7 @@
 #include "disco.h"
 #include "stream_tail.cuh"
 #include "umma_tail.cuh"
+#include "umma_gemv.cuh"
 
 using namespace disco;
 
@@ -231,6 +232,57 @@ int launch_umma(disco_ctx* c, const void* W, const void* H, int d, int R, float*
     return cuda_ok(e, "umma_tail_kernel launch") ? DISCO_OK : DISCO_ERR_CUDA;
 }
 
+
+// Launch the tensor-core GEMV-shaped draft step (1..16 sequences).
+template <int RK>
+int launch_gemv_rk(disco_ctx* c, GemvParams& g, const CUtensorMap& mW, const CUtensorMap& mWt, const CUtensorMap& mH,
+                   cudaStream_t st) {
+    auto kern = umma_gemv_draft_kernel<RK>;
+    const size_t smem = gemv_smem_bytes(RK, g.t.clf_H);
+    static int configured_dev = -1;
+    static size_t configured_smem = 0;
+    if (configured_dev != c->device || configured_smem < smem) {
+        if (!cuda_ok(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem),
+                     "cudaFuncSetAttribute(gemv)"))
+            return DISCO_ERR_CUDA;
+        configured_dev = c->device;
+        configured_smem = smem;
+    }
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3((unsigned)c->sm_count);
+    cfg.blockDim = dim3(kGemvThreads);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = c->pdl ? 1 : 0;
+    const cudaError_t e = cudaLaunchKernelEx(&cfg, kern, mW, mWt, mH, g);
+    c->launches += 1;
+    return cuda_ok(e, "umma_gemv_draft_kernel launch") ? DISCO_OK : DISCO_ERR_CUDA;
+}
+
+int launch_gemv(disco_ctx* c, const TailParams& t, cudaStream_t st) {
+    GemvParams g{};
+    g.t = t;
+    const int grid = c->sm_count;
+    if (grid > c->part_slots || t.R > c->part_rows) return DISCO_ERR_WORKSPACE;
+    g.TR = (t.V + grid - 1) / grid;
+    g.tiles = (g.TR + 127) / 128;
+    g.tail_rows = std::max(8, (g.TR - 128 * (g.tiles - 1) + 7) / 8 * 8);
+    g.h_rows = t.R <= 8 ? 8 : 16;
+    CUtensorMap mW, mWt, mH;
+    if (!encode_bf16_2d(c, &mW, t.W, t.V, t.d, 128) || !encode_bf16_2d(c, &mWt, t.W, t.V, t.d, g.tail_rows) ||
+        !encode_bf16_2d(c, &mH, t.H, t.R, t.d, g.h_rows))
+        return DISCO_ERR_CUDA;
+    if (t.R == 1) return launch_gemv_rk<1>(c, g, mW, mWt, mH, st);
+    if (t.R == 2) return launch_gemv_rk<2>(c, g, mW, mWt, mH, st);
+    if (t.R <= 4) return launch_gemv_rk<4>(c, g, mW, mWt, mH, st);
+    if (t.R <= 8) return launch_gemv_rk<8>(c, g, mW, mWt, mH, st);
+    return launch_gemv_rk<16>(c, g, mW, mWt, mH, st);
+}
+
 void fill_scratch(const disco_ctx* c, TailParams& p) {
     p.part_rec = reinterpret_cast<float4*>(c->part_rec);
     p.keys = c->keys;
@@ -361,7 +413,7 @@ int disco_launch_count(disco_ctx* c, long long* out) {
 }
 
 int disco_set_kernel_path(disco_ctx* c, int which) {
-    if (!c || which < 0 || which > 2) return DISCO_ERR_INVALID_ARG;
+    if (!c || which < 0 || which > 3) return DISCO_ERR_INVALID_ARG;
     c->path = which;
     return DISCO_OK;
 }
@@ -401,8 +453,12 @@ int disco_draft_step(disco_ctx* c, const void* W_D, const void* h_D, int B, cons
     p.halt = halt;
     p.feats = feats;
     p.probs = probs;
-    const bool use_umma = umma_possible(c, B) && (c->path == 2 || (c->path == 0 && B >= 2));
-    if (use_umma) {
+    const bool use_gemv = c->encode_tiled != nullptr && B <= kGemvMaxRows && (c->path == 3 || c->path == 0);
+    const bool use_umma = !use_gemv && umma_possible(c, B) && (c->path == 2 || c->path == 0 || c->path == 3);
+    if (use_gemv) {
+        rc = launch_gemv(c, p, st);
+        if (rc) return rc;
+    } else if (use_umma) {
         int np = 0;
         rc = launch_umma<true>(c, W_D, h_D, c->d_draft, B, probs, &np, nullptr, st);
         if (rc) return rc;

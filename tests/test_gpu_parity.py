@@ -249,11 +249,14 @@ def test_errors_are_codes_not_faults():
 
 
 # ---------------------------------------------------------------------------------- both kernel families
-@pytest.mark.parametrize("path", [1, 2])
-@pytest.mark.parametrize("V,d,B", [(50, 16, 1), (1000, 72, 3), (4099, 264, 7), (5000, 768, 64), (3000, 128, 130)])
+@pytest.mark.parametrize("path", [1, 2, 3])
+@pytest.mark.parametrize("V,d,B", [(50, 16, 1), (1000, 72, 3), (4099, 264, 7), (32000, 768, 1), (20011, 320, 16),
+                                   (5000, 768, 64), (3000, 128, 130)])
 def test_draft_step_on_each_kernel_path(oracle, path, V, d, B):
     if path == 1 and B > 16:
         pytest.skip("the CUDA-core kernel is only meant for a handful of rows")
+    if path == 3 and B > 16:
+        pytest.skip("the vocabulary-on-lanes kernel takes at most 16 sequences")
     W = inputs.lm_head(V, d, seed=3 * V + d, std=0.2)
     h = inputs.hidden(B, d, seed=V + 11 * B)
     params = make_clf(32, seed=B)
