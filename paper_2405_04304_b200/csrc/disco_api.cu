@@ -481,7 +481,7 @@ int disco_draft_step(disco_ctx* c, const void* W_D, const void* h_D, int B, cons
         f.halt = halt;
         f.feats = feats;
         f.final_stats = c->final_stats;
-        draft_finalize_kernel<<<B, kDraftFinalWarps * 32, 0, st>>>(f);
+        draft_finalize_kernel<<<(B + kDraftFinalWarps - 1) / kDraftFinalWarps, kDraftFinalWarps * 32, 0, st>>>(f);
         c->launches += 1;
         if (!cuda_ok(cudaGetLastError(), "draft_finalize_kernel launch")) return DISCO_ERR_CUDA;
     } else {

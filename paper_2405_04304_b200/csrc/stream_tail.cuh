@@ -71,7 +71,7 @@ inline size_t stream_tail_smem_bytes(int RT, int NW, int d, int stages, uint32_t
     b += (size_t)RT * d * 2;                          // hidden tile
     b += (size_t)stages * 16;                         // full/empty barriers
     b += (size_t)(NW * RT + 1) * kRecordWords * 4;    // warp records / finalize staging (+ carry)
-    b += 64 * 4;                                      // features
+    b += (size_t)NW * 16 * 4;                         // features, 16 words per warp
     b += ((size_t)clf_H * (kNFeat + 2) + 4) * 4;      // classifier parameters
     return b + 128;
 }
@@ -104,6 +104,30 @@ struct LaneRecord {
             key = key_from_words(c.z, c.w);
             l[0] = a.x, l[1] = a.y, l[2] = a.z, l[3] = a.w, l[4] = b.x, l[5] = b.y, l[6] = b.z, l[7] = b.w;
             l[8] = c.x, l[9] = c.y;
+        }
+    }
+    // Fold another record into this one, inside the lane: statistics, key, and the two descending
+    // lists merged by a bitonic network (max(a[i], b[15 - i]) holds the 16 largest as a bitonic sequence).
+    __device__ __forceinline__ void absorb(const LaneRecord& o) {
+        if (!(o.Z > 0.f)) return;
+        SoftmaxState st;
+        st.m = m, st.Z = Z, st.S = S;
+        st.merge(o.m, o.Z, o.S);
+        m = st.m, Z = st.Z, S = st.S;
+        key = o.key > key ? o.key : key;
+#pragma unroll
+        for (int i = 0; i < 16; ++i) l[i] = fmaxf(l[i], o.l[15 - i]);
+#pragma unroll
+        for (int stride = 8; stride > 0; stride >>= 1) {
+#pragma unroll
+            for (int i = 0; i < 16; ++i) {
+                if ((i & stride) == 0) {
+                    const float hi = fmaxf(l[i], l[i + stride]);
+                    const float lo = fminf(l[i], l[i + stride]);
+                    l[i] = hi;
+                    l[i + stride] = lo;
+                }
+            }
         }
     }
 };
@@ -239,46 +263,44 @@ __device__ __forceinline__ void warp_draft_epilogue(const SoftmaxState& st, unsi
     if (o.feats && lane < kNFeat) o.feats[(size_t)b * kNFeat + lane] = x;
 }
 
-// Draft step, sequence b, in the last CTA: the NW warps reduce the per-CTA records 32 at a time, warp 0
-// merges their results (plus the carry of an earlier block when there are more than 32 * NW records).
-template <int NW>
-__device__ void finalize_draft_row(const TailParams& p, int b, int grid, float* stage /*(NW + 1) records*/,
-                                   float* feat_s, const float* clf_s, int warp, int lane) {
-    constexpr int BAR_THREADS = NW * 32;
+// Draft step, sequence b, in the last CTA, by ONE warp (the warps take different sequences): every lane
+// fetches its share of the per-CTA records (four per L2 round trip) and folds them lane-locally, one
+// cross-lane reduction merges the lanes, then features, classifier and stopping rule.
+// feat16: 16 words of shared memory owned by the calling warp.
+__device__ __forceinline__ void finalize_draft_seq(const TailParams& p, int b, int grid, float* feat16, const float* clf_s,
+                                                   int lane) {
     const float fpos = static_cast<float>(p.pos[b]);  // issued early: hidden behind the merge
     const int n_drafted = p.n_drafted[b];
     const float4* recs = p.part_rec + (size_t)b * grid * 4;
     LaneRecord r;
-    for (int base = 0; base < grid; base += 32 * NW) {
-        const int c = base + warp * 32 + lane;
-        r.clear();
-        if (c < grid) {  // one L2 round trip per lane: the four quarters of its record
-            const float4* src = recs + (size_t)c * 4;
-            const float4 q0 = __ldcg(src), q1 = __ldcg(src + 1), q2 = __ldcg(src + 2), q3 = __ldcg(src + 3);
-            r.set(q0, q1, q2, q3);
+    r.clear();
+#pragma unroll 1
+    for (int c0 = 0; c0 < grid; c0 += 128) {
+        float4 q[4][4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const int c = c0 + j * 32 + lane;
+            if (c < grid) {
+                const float4* src = recs + (size_t)c * 4;
+                q[j][0] = __ldcg(src), q[j][1] = __ldcg(src + 1), q[j][2] = __ldcg(src + 2), q[j][3] = __ldcg(src + 3);
+            } else {
+                q[j][0] = make_float4(0.f, 0.f, 0.f, 0.f);  // Z = 0: empty
+            }
         }
-        warp_reduce_records(r, 5);
-        warp_store_record(stage + warp * kRecordWords, r, lane);
-        named_barrier_sync(1, BAR_THREADS);
-        if (warp == 0) {
-            const int n = base == 0 ? NW : NW + 1;
-            const float4* sr = reinterpret_cast<const float4*>(stage) + lane * 4;
-            r.clear();
-            if (lane < n) r.set(sr[0], sr[1], sr[2], sr[3]);
-            warp_reduce_records(r, ceil_log2(n));
-            if (base + 32 * NW < grid) warp_store_record(stage + NW * kRecordWords, r, lane);  // carry
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            LaneRecord o;
+            o.set(q[j][0], q[j][1], q[j][2], q[j][3]);
+            r.absorb(o);
         }
-        named_barrier_sync(1, BAR_THREADS);
     }
-    if (warp == 0) {
-        const int Hc = p.clf_H;
-        SoftmaxState st;
-        st.m = r.m, st.Z = r.Z, st.S = r.S;
-        const DraftOutputs o{p.token, p.conf, p.halt, p.feats, p.final_stats};
-        warp_draft_epilogue(st, r.key, lane_pick(r, lane), fpos, n_drafted, p.tau, p.sl_max, feat_s, clf_s,
-                            clf_s + Hc * kNFeat, clf_s + Hc * (kNFeat + 1), clf_s + Hc * (kNFeat + 2), Hc, b, o, lane);
-    }
-    named_barrier_sync(1, BAR_THREADS);
+    warp_reduce_records(r, 5);
+    const int Hc = p.clf_H;
+    SoftmaxState st;
+    st.m = r.m, st.Z = r.Z, st.S = r.S;
+    const DraftOutputs o{p.token, p.conf, p.halt, p.feats, p.final_stats};
+    warp_draft_epilogue(st, r.key, lane_pick(r, lane), fpos, n_drafted, p.tau, p.sl_max, feat16, clf_s, clf_s + Hc * kNFeat,
+                        clf_s + Hc * (kNFeat + 1), clf_s + Hc * (kNFeat + 2), Hc, b, o, lane);
 }
 
 // Verification: decode the arg-max keys, match the draft prefix, pick the bonus token.
@@ -350,7 +372,7 @@ __global__ void __launch_bounds__((NW + 1) * 32, 1) stream_tail_kernel(const __g
     uint64_t* empty = full + p.stages;
     float* wstate = reinterpret_cast<float*>(empty + p.stages);  // 16-byte aligned
     float* feat_s = wstate + (NW * RT + 1) * kRecordWords;
-    float* clf_s = feat_s + 64;
+    float* clf_s = feat_s + NW * 16;
     __shared__ int s_is_last;
 
     const int v0 = blockIdx.x * p.rows_per_cta;
@@ -594,10 +616,11 @@ __global__ void __launch_bounds__((NW + 1) * 32, 1) stream_tail_kernel(const __g
 
     if (DRAFT) {
         named_barrier_sync(1, BAR_THREADS);
-        for (int b = 0; b < p.R; ++b) {
+        for (int b = warp; b < p.R; b += NW) {
             if (p.active && !p.active[b]) continue;
-            finalize_draft_row<NW>(p, b, grid, wstate, feat_s, clf_s, warp, lane);
+            finalize_draft_seq(p, b, grid, feat_s + warp * 16, clf_s, lane);
         }
+        named_barrier_sync(1, BAR_THREADS);
     } else {
         for (int b = warp; b < p.B; b += NW)
             verify_one_sequence(p.keys, p.draft_ids, p.row_off, p.B, p.SL, p.R, b, p.n_accept, p.bonus,

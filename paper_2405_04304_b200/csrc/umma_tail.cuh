@@ -456,48 +456,46 @@ __global__ void __launch_bounds__(128) verify_finalize_kernel(const VerifyFinalP
     if (threadIdx.x == 0) *p.ticket = 0u;
 }
 
-constexpr int kDraftFinalWarps = 8;
+constexpr int kDraftFinalWarps = 4;
 
-// One CTA per sequence: the warps reduce the per-CTA records 32 at a time, warp 0 merges their results
-// and runs the epilogue.
+// One warp per sequence: reduce the per-CTA records and run the epilogue.
 __global__ void __launch_bounds__(kDraftFinalWarps * 32) draft_finalize_kernel(const DraftFinalParams p) {
-    __shared__ __align__(16) float stage[(kDraftFinalWarps + 1) * kRecordWords];
-    __shared__ float feat_s[16];
+    __shared__ float feat_s[kDraftFinalWarps * 16];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int b = blockIdx.x;
+    const int b = blockIdx.x * kDraftFinalWarps + warp;
+    if (b >= p.B) return;
     if (p.active && !p.active[b]) return;
     const float fpos = static_cast<float>(p.pos[b]);
     const int n_drafted = p.n_drafted[b];
     const float4* recs = p.part_rec + (size_t)b * p.NP * 4;
     LaneRecord r;
-    for (int base = 0; base < p.NP; base += 32 * kDraftFinalWarps) {
-        const int c = base + warp * 32 + lane;
-        r.clear();
-        if (c < p.NP) {
-            const float4* src = recs + (size_t)c * 4;
-            const float4 q0 = __ldcg(src), q1 = __ldcg(src + 1), q2 = __ldcg(src + 2), q3 = __ldcg(src + 3);
-            r.set(q0, q1, q2, q3);
+    r.clear();
+#pragma unroll 1
+    for (int c0 = 0; c0 < p.NP; c0 += 128) {
+        float4 q[4][4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const int c = c0 + j * 32 + lane;
+            if (c < p.NP) {
+                const float4* src = recs + (size_t)c * 4;
+                q[j][0] = __ldcg(src), q[j][1] = __ldcg(src + 1), q[j][2] = __ldcg(src + 2), q[j][3] = __ldcg(src + 3);
+            } else {
+                q[j][0] = make_float4(0.f, 0.f, 0.f, 0.f);
+            }
         }
-        warp_reduce_records(r, 5);
-        warp_store_record(stage + warp * kRecordWords, r, lane);
-        __syncthreads();
-        if (warp == 0) {
-            const int n = base == 0 ? kDraftFinalWarps : kDraftFinalWarps + 1;
-            const float4* sr = reinterpret_cast<const float4*>(stage) + lane * 4;
-            r.clear();
-            if (lane < n) r.set(sr[0], sr[1], sr[2], sr[3]);
-            warp_reduce_records(r, ceil_log2(n));
-            if (base + 32 * kDraftFinalWarps < p.NP) warp_store_record(stage + kDraftFinalWarps * kRecordWords, r, lane);
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            LaneRecord o;
+            o.set(q[j][0], q[j][1], q[j][2], q[j][3]);
+            r.absorb(o);
         }
-        __syncthreads();
     }
-    if (warp == 0) {
-        SoftmaxState st;
-        st.m = r.m, st.Z = r.Z, st.S = r.S;
-        const DraftOutputs o{p.token, p.conf, p.halt, p.feats, p.final_stats};
-        warp_draft_epilogue(st, r.key, lane_pick(r, lane), fpos, n_drafted, p.tau, p.sl_max, feat_s, p.clf_W1, p.clf_b1,
-                            p.clf_w2, p.clf_b2, p.clf_H, b, o, lane);
-    }
+    warp_reduce_records(r, 5);
+    SoftmaxState st;
+    st.m = r.m, st.Z = r.Z, st.S = r.S;
+    const DraftOutputs o{p.token, p.conf, p.halt, p.feats, p.final_stats};
+    warp_draft_epilogue(st, r.key, lane_pick(r, lane), fpos, n_drafted, p.tau, p.sl_max, feat_s + warp * 16, p.clf_W1,
+                        p.clf_b1, p.clf_w2, p.clf_b2, p.clf_H, b, o, lane);
 }
 
 }  // namespace disco
