@@ -43,6 +43,27 @@ def measured_peaks():
     return 6650.0, 1400.0, "fallback"
 
 
+# ------------------------------------------------------------------------------------------ ranks
+def max_over_ranks(values, device="cpu"):
+    """Element-wise maximum of a list of floats over all ranks (identity without a process group).
+    Every rank times its own replica; the job is as slow as its slowest replica."""
+    if not (torch.distributed.is_available() and torch.distributed.is_initialized()):
+        return [float(v) for v in values]
+    t = torch.tensor([float(v) for v in values], dtype=torch.float64, device=device)
+    torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
+    return [float(v) for v in t.cpu()]
+
+
+def replica_seed(workload_seed: int, rank: int) -> int:
+    """Each rank runs an independent replica of the workload on its own seeded inputs."""
+    return workload_seed + 1000 * rank
+
+
+def whole_job_value(steps_per_rank: int, world: int, seconds: float) -> float:
+    """Iterations per second of the whole job: all replicas' steps over the slowest replica's time."""
+    return steps_per_rank * world / seconds
+
+
 # ------------------------------------------------------------------------------------------ clocks
 class ClockSampler:
     """Polls SM clock and throttle reasons through NVML while the timed region runs (read-only)."""
@@ -319,7 +340,7 @@ def run_ours(args, rank: int, world: int):
     wl = inputs.WORKLOADS[args.workload]
     K, Wm = args.steps, args.warmup
     T = Wm + K
-    data = Data(wl, T, wl.seed + 1000 * rank, device)
+    data = Data(wl, T, replica_seed(wl.seed, rank), device)
     B, S = wl.B, wl.sl_max
     max_rows = B * (S + 1)
     ctx = binding.Context(wl.V, wl.d_D, wl.d_T, max_batch=B, max_rows=max_rows, clf_hidden=wl.H)
@@ -347,13 +368,10 @@ def run_ours(args, rank: int, world: int):
     e2e["matches"] = all(np.array_equal(sl, res["sl_all"][it]) and np.array_equal(na, res["n_acc"][it])
                          for it, (sl, na) in enumerate(e2e["trace"]))
 
-    if world > 1:
-        tt = torch.tensor([t_all, e2e["seconds"]], dtype=torch.float64, device=device)
-        torch.distributed.all_reduce(tt, op=torch.distributed.ReduceOp.MAX)
-        t_all, e2e["seconds"] = float(tt[0]), float(tt[1])
+    t_all, e2e["seconds"] = max_over_ranks([t_all, e2e["seconds"]], device)
 
     out = {
-        "metric": METRIC, "value": K * world / t_all, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": Wm,
+        "metric": METRIC, "value": whole_job_value(K, world, t_all), "unit": UNIT, "n_gpus": world, "steps": K, "warmup": Wm,
         "ms_per_step": t_all / K * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "bf16 inputs, fp32 accumulate", "data": "synthetic (seeded Gaussian LM heads and hidden states)",
         "config": {"workload": wl.name, "V": wl.V, "d_draft": wl.d_D, "d_target": wl.d_T, "batch": B,
@@ -364,7 +382,7 @@ def run_ours(args, rank: int, world: int):
                    "l2": f"draft LM head rotates through {data.n_rot} copies (> 2x L2); the target LM head alone "
                          "exceeds L2", "launch": "CUDA graph of the K iterations' kernels"},
         "roofline": dominant, "roofline_other_kernel": other,
-        "e2e": {"value": K * world / e2e["seconds"], "unit": UNIT, "h2d_bytes_per_step": e2e["h2d"] / K,
+        "e2e": {"value": whole_job_value(K, world, e2e["seconds"]), "unit": UNIT, "h2d_bytes_per_step": e2e["h2d"] / K,
                 "d2h_bytes_per_step": e2e["d2h"] / K, "matches_device_run": e2e["matches"]},
         "gpu_launches": res["launches"], "clocks": sampler.summary(),
     }
