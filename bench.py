@@ -43,6 +43,34 @@ def measured_peaks():
     return 6650.0, 1400.0, "fallback"
 
 
+# ------------------------------------------------------------------------------------------ ncu traffic
+# dram__bytes_read.sum + dram__bytes_write.sum per launch, from the ncu captures summarised under
+# profiles/.  Valid only for the kernel sources they were taken on: reported as null once csrc/ changes.
+NCU_TRAFFIC = {
+    "sources": "5b234849681c402d",
+    "bytes_per_launch": {
+        ("vicuna_b1", "verification tail"): 327.77e6 + 3.72e6,
+        ("vicuna_b1", "draft-step tail"): 49.22e6 + 0.01e6,
+    },
+}
+
+
+def kernel_sources_hash() -> str:
+    import glob
+    import hashlib
+    h = hashlib.sha256()
+    for f in sorted(glob.glob(os.path.join(ROOT, "paper_2405_04304_b200", "csrc", "*"))):
+        with open(f, "rb") as fh:
+            h.update(fh.read())
+    return h.hexdigest()[:16]
+
+
+def ncu_traffic(workload: str, kernel: str):
+    if kernel_sources_hash() != NCU_TRAFFIC["sources"]:
+        return None
+    return NCU_TRAFFIC["bytes_per_launch"].get((workload, kernel))
+
+
 # ------------------------------------------------------------------------------------------ ranks
 def max_over_ranks(values, device="cpu"):
     """Element-wise maximum of a list of floats over all ranks (identity without a process group).
@@ -321,6 +349,7 @@ def rooflines(wl, K: int, res: dict, hbm_peak: float, tensor_peak: float, peak_k
                   "peak": hbm_peak, "peak_kind": peak_kind, "unit": "GB/s", "launches": res["n_draft"],
                   "avg_launch_us": res["t_draft"] / max(res["n_draft"], 1) * 1e6, "traffic": None}
     for r in (roof_verify, roof_draft):
+        r["traffic"] = ncu_traffic(wl.name, r["kernel"])
         r["frac"] = r["achieved"] / r["peak"]
         r["frac_of_nominal_8TBs"] = r["achieved"] / 8000.0
     if res["rows_total"] / K > tensor_peak * 1e12 / (hbm_peak * 1e9):   # rows per call beyond the machine balance
