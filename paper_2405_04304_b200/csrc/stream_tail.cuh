@@ -138,10 +138,9 @@ struct LaneRecord {
 //     shuffle sums (much shorter than a butterfly of pairwise merges);
 //   * lists: a bitonic merge network across lanes: max(a[i], partner[15 - i]) keeps the 16 largest of
 //     two descending lists as a bitonic sequence, four compare-exchange stages sort it again.
-// `levels` = ceil(log2(number of lanes that may hold a record)); at least four levels run, so that
-// lanes 0..15 always end up with the result (lanes 0..11 are the ones that use it).
+// `levels` = ceil(log2(number of lanes that may hold a record)): lanes 0 .. 2^levels - 1 end up with the
+// result (lane 0 always does).
 __device__ __forceinline__ void warp_reduce_records(LaneRecord& r, int levels) {
-    levels = max(levels, 4);
     const uint32_t mbits = __reduce_max_sync(kFullMask, ordered_bits(r.m));
     const float M = from_ordered_bits(mbits);
     float Zc = 0.f, Sc = 0.f;
@@ -205,10 +204,17 @@ __device__ __forceinline__ void warp_store_record(float* rec, const SoftmaxState
     if (lane < kTopK) rec[4 + lane] = sel;
 }
 
+// Store the reduced record that lane 0 holds (the other lanes may hold partial results).
 __device__ __forceinline__ void warp_store_record(float* rec, const LaneRecord& r, int lane) {
+    float sel = DISCO_NEG_INF;
+#pragma unroll
+    for (int k = 0; k < kTopK; ++k) {
+        const float v = __shfl_sync(kFullMask, r.l[k], 0);
+        sel = (lane == k) ? v : sel;
+    }
     SoftmaxState st;
     st.m = r.m, st.Z = r.Z, st.S = r.S;
-    warp_store_record(rec, st, r.key, lane_pick(r, lane), lane);
+    warp_store_record(rec, st, r.key, sel, lane);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -249,8 +255,8 @@ __device__ __forceinline__ void warp_draft_epilogue(const SoftmaxState& st, unsi
                                                     const float* b1, const float* w2, const float* b2, int Hc, int b,
                                                     const DraftOutputs& o, int lane) {
     const float inv_Z = 1.f / st.Z;
-    const float prob = (lane < kTopK && sel > DISCO_NEG_INF) ? expf(sel - st.m) * inv_Z : 0.f;
-    const float ent = logf(st.Z) - st.S * inv_Z;
+    const float prob = (lane < kTopK && sel > DISCO_NEG_INF) ? __expf(sel - st.m) * inv_Z : 0.f;
+    const float ent = __logf(st.Z) - st.S * inv_Z;
     const float x = lane < kTopK ? prob : (lane == kTopK ? ent : (lane == kTopK + 1 ? fpos : 0.f));
     const float C = warp_halt_classifier(x, feat_s, W1, b1, w2, b2, Hc, lane);
     if (lane == 0) {
@@ -274,11 +280,12 @@ __device__ __forceinline__ void finalize_draft_seq(const TailParams& p, int b, i
     const float4* recs = p.part_rec + (size_t)b * grid * 4;
     LaneRecord r;
     r.clear();
+    constexpr int kPerLane = 5;  // 160 records per L2 round trip: one round trip for a grid of 148 CTAs
 #pragma unroll 1
-    for (int c0 = 0; c0 < grid; c0 += 128) {
-        float4 q[4][4];
+    for (int c0 = 0; c0 < grid; c0 += 32 * kPerLane) {
+        float4 q[kPerLane][4];
 #pragma unroll
-        for (int j = 0; j < 4; ++j) {
+        for (int j = 0; j < kPerLane; ++j) {
             const int c = c0 + j * 32 + lane;
             if (c < grid) {
                 const float4* src = recs + (size_t)c * 4;
@@ -288,7 +295,7 @@ __device__ __forceinline__ void finalize_draft_seq(const TailParams& p, int b, i
             }
         }
 #pragma unroll
-        for (int j = 0; j < 4; ++j) {
+        for (int j = 0; j < kPerLane; ++j) {
             LaneRecord o;
             o.set(q[j][0], q[j][1], q[j][2], q[j][3]);
             r.absorb(o);

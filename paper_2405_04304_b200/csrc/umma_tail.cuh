@@ -470,11 +470,12 @@ __global__ void __launch_bounds__(kDraftFinalWarps * 32) draft_finalize_kernel(c
     const float4* recs = p.part_rec + (size_t)b * p.NP * 4;
     LaneRecord r;
     r.clear();
+    constexpr int kPerLane = 5;  // 160 records per L2 round trip
 #pragma unroll 1
-    for (int c0 = 0; c0 < p.NP; c0 += 128) {
-        float4 q[4][4];
+    for (int c0 = 0; c0 < p.NP; c0 += 32 * kPerLane) {
+        float4 q[kPerLane][4];
 #pragma unroll
-        for (int j = 0; j < 4; ++j) {
+        for (int j = 0; j < kPerLane; ++j) {
             const int c = c0 + j * 32 + lane;
             if (c < p.NP) {
                 const float4* src = recs + (size_t)c * 4;
@@ -484,7 +485,7 @@ __global__ void __launch_bounds__(kDraftFinalWarps * 32) draft_finalize_kernel(c
             }
         }
 #pragma unroll
-        for (int j = 0; j < 4; ++j) {
+        for (int j = 0; j < kPerLane; ++j) {
             LaneRecord o;
             o.set(q[j][0], q[j][1], q[j][2], q[j][3]);
             r.absorb(o);
