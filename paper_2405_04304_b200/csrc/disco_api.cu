@@ -453,10 +453,11 @@ int disco_draft_step(disco_ctx* c, const void* W_D, const void* h_D, int B, cons
     p.halt = halt;
     p.feats = feats;
     p.probs = probs;
-    // Measured on B200 (Vicuna head): one sequence is fastest on the CUDA-core streaming kernel, 2..6 on
-    // the tensor-core kernel with the vocabulary on the lanes, more on the one with the hidden rows on the lanes.
+    // Measured on B200 (Vicuna head): up to 6 sequences are fastest on the tensor-core kernel with the
+    // vocabulary on the TMEM lanes, more on the one with the hidden rows on the lanes; the CUDA-core
+    // streaming kernel is within 10 % for one sequence and serves as the path without tensor maps.
     const bool gemv_ok = c->encode_tiled != nullptr && B <= kGemvMaxRows;
-    const bool use_gemv = gemv_ok && (c->path == 3 || (c->path == 0 && B >= 2 && B <= 6));
+    const bool use_gemv = gemv_ok && (c->path == 3 || (c->path == 0 && B <= 6));
     const bool use_umma = !use_gemv && umma_possible(c, B) && (c->path == 2 || c->path == 3 || (c->path == 0 && B >= 2));
     if (use_gemv) {
         rc = launch_gemv(c, p, st);
