@@ -373,6 +373,7 @@ def run_ours(args, rank: int, world: int):
     B, S = wl.B, wl.sl_max
     max_rows = B * (S + 1)
     ctx = binding.Context(wl.V, wl.d_D, wl.d_T, max_batch=B, max_rows=max_rows, clf_hidden=wl.H)
+    ctx.set_kernel_path(args.kernel_path)
     clf = binding.Classifier(*(t.to(device) for t in data.clf_params))
     stream = torch.cuda.Stream()
     hbm_peak, tensor_peak, peak_kind = measured_peaks()
@@ -595,6 +596,7 @@ def main():
     ap.add_argument("--workload", default="vicuna_b1", choices=sorted(inputs.WORKLOADS))
     ap.add_argument("--cpu-seconds", type=float, default=15.0)
     ap.add_argument("--reference-seconds", type=float, default=120.0)
+    ap.add_argument("--kernel-path", type=int, default=0, help="0 automatic; 1..3 force a kernel family (tuning)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-static", action="store_true", help="skip the extra pass with SL forced to SL_max")
     args = ap.parse_args()
