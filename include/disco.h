@@ -118,6 +118,23 @@ int disco_draft_step(disco_ctx* ctx, const void* W_D, const void* h_D, int B,
                      void* stream);
 
 /*
+ * Draft step with the rule-based stopping test of App. F ("ppl SL-opt") in place of the classifier:
+ * the confidence in the tokens drafted so far in this iteration is their perplexity,
+ *     ppl_n = exp( -(1/n) * sum_{j <= n} ln y^D_j(t_j) ),
+ * lower meaning more confident; drafting stops when ppl_n > ppl_max or n_drafted >= sl_max.
+ * With greedy drafting t_j attains the largest logit, so -ln y^D_j(t_j) = ln Z_j (Z_j = sum exp(z - max z)).
+ *   nll_sum    float [B], device, in/out: the sum of -ln y over the tokens drafted earlier in this
+ *              iteration (0 before the first one); the call adds this token's term (active sequences only)
+ *   n_drafted  int32 [B]  draft tokens of this iteration including this one (>= 1)
+ * Outputs: token [B], ppl [B] (the perplexity including this token), halt [B].
+ * Other arguments as in disco_draft_step.
+ */
+int disco_draft_step_ppl(disco_ctx* ctx, const void* W_D, const void* h_D, int B,
+                         const int32_t* n_drafted, const uint8_t* active, float* nll_sum,
+                         float ppl_max, int sl_max, int32_t* token, float* ppl, uint8_t* halt,
+                         void* stream);
+
+/*
  * Verification with the same look-ahead SL for all B sequences (Sec. 2; Fig. 1).
  *   W_T        bf16 [V, d_target]          target LM head
  *   H_T        bf16 [B*(SL+1), d_target]   row b*(SL+1)+j is the target hidden state whose

@@ -202,6 +202,26 @@ def draft_step(W_D, h_D, pos, n_drafted, clf: Classifier, tau: float, sl_max: in
     return DraftStepResult(token, conf, halt, feats, gap, ids, probs)
 
 
+def draft_step_ppl(W_D, h_D, n_drafted, nll_sum, ppl_max: float, sl_max: int, active=None, nthreads: int = 1):
+    """Perplexity stopping rule (App. F).  Returns (token, ppl, halt, gap, new nll_sum)."""
+    W_D, h_D = _u16(W_D), _u16(h_D)
+    V, d = W_D.shape
+    B = h_D.shape[0]
+    n_drafted = np.ascontiguousarray(n_drafted, dtype=np.int32)
+    nll = np.array(nll_sum, dtype=np.float64).copy()
+    act = None if active is None else np.ascontiguousarray(active, dtype=np.uint8)
+    token = np.full(B, -1, dtype=np.int32)
+    ppl = np.full(B, np.nan)
+    halt = np.full(B, 255, dtype=np.uint8)
+    gap = np.full(B, np.nan)
+    _check(lib().oracle_draft_step_ppl(
+        _p(W_D, ctypes.c_uint16), _p(h_D, ctypes.c_uint16), V, d, B, _p(n_drafted, ctypes.c_int32),
+        _p(act, ctypes.c_uint8), _p(nll, ctypes.c_double), ctypes.c_float(ppl_max), int(sl_max),
+        _p(token, ctypes.c_int32), _p(ppl, ctypes.c_double), _p(halt, ctypes.c_uint8), _p(gap, ctypes.c_double),
+        nthreads), "draft_step_ppl")
+    return token, ppl, halt, gap, nll
+
+
 @dataclass
 class VerifyResult:
     n_accept: np.ndarray    # [B] int32

@@ -204,6 +204,33 @@ int oracle_draft_step(const uint16_t* W_D, const uint16_t* h_D, int V, int d, in
     return ORACLE_OK;
 }
 
+// Rule-based stopping test of App. F ("ppl SL-opt"): the confidence in the tokens drafted so far in
+// this iteration is their perplexity  ppl_n = exp(-(1/n) sum_{j<=n} ln y_j(t_j)),  lower = more
+// confident;  halt = (ppl_n > ppl_max) or (n_drafted >= SL_max).  nll_sum[b] carries the sum over the
+// earlier tokens of the iteration and receives this token's term.  The comparison is taken on ppl
+// rounded to binary32 (the library's precision).
+int oracle_draft_step_ppl(const uint16_t* W_D, const uint16_t* h_D, int V, int d, int B,
+                          const int32_t* n_drafted, const uint8_t* active, double* nll_sum, float ppl_max,
+                          int sl_max, int32_t* token, double* ppl, uint8_t* halt, double* gap, int nthreads) {
+    if (!W_D || !h_D || !n_drafted || !nll_sum || !token || V <= 0 || d <= 0 || B < 0) return ORACLE_BAD_ARG;
+    std::vector<double> z(V), y(V);
+    for (int b = 0; b < B; ++b) {
+        if (active && !active[b]) continue;
+        if (n_drafted[b] < 1) return ORACLE_BAD_ARG;
+        int rc = oracle_project(W_D, h_D + (size_t)b * d, V, d, 1, z.data(), nthreads);
+        if (rc) return rc;
+        rc = oracle_argmax(z.data(), V, &token[b], gap ? &gap[b] : nullptr);
+        if (rc) return rc;
+        rc = oracle_softmax(z.data(), V, y.data());
+        if (rc) return rc;
+        nll_sum[b] += -std::log(y[token[b]]);
+        const double perp = std::exp(nll_sum[b] / n_drafted[b]);
+        if (ppl) ppl[b] = perp;
+        if (halt) halt[b] = (static_cast<float>(perp) > ppl_max) || (n_drafted[b] >= sl_max) ? 1 : 0;
+    }
+    return ORACLE_OK;
+}
+
 // Acceptance at temperature 0 (Sec. 3, rejection sampling "with zero
 // temperature"; Fig. 1): draft token j+1 is accepted iff it equals the target's
 // greedy token at row j and every earlier draft token was accepted.

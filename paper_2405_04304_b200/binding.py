@@ -29,7 +29,7 @@ STATIC_MAX_BATCH = 4
 EXPORTS = [
     "disco_create", "disco_destroy", "disco_strerror", "disco_last_device_status", "disco_launch_count",
     "disco_set_kernel_path", "disco_draft_step", "disco_verify", "disco_verify_ragged",
-    "disco_draft_step_host", "disco_verify_ragged_host", "disco_draft_step_static",
+    "disco_draft_step_host", "disco_verify_ragged_host", "disco_draft_step_static", "disco_draft_step_ppl",
 ]
 
 
@@ -66,6 +66,7 @@ def load() -> ctypes.CDLL:
     lib.disco_set_kernel_path.argtypes = [vp, ci]
     lib.disco_draft_step.argtypes = [vp, vp, vp, ci, vp, vp, vp, ctypes.POINTER(_Clf), cf, ci,
                                      vp, vp, vp, vp, vp, vp]
+    lib.disco_draft_step_ppl.argtypes = [vp, vp, vp, ci, vp, vp, vp, cf, ci, vp, vp, vp, vp]
     lib.disco_verify.argtypes = [vp, vp, vp, vp, ci, ci, vp, vp, vp, vp]
     lib.disco_verify_ragged.argtypes = [vp, vp, vp, vp, vp, ci, ci, vp, vp, vp, vp]
     lib.disco_draft_step_host.argtypes = [vp, vp, vp, ci, vp, vp, vp, ctypes.POINTER(_Clf), cf, ci,
@@ -186,6 +187,16 @@ class Context:
             _ptr(feats, torch.float32), _ptr(probs, torch.float32), _stream(stream))
         if rc != OK:
             raise DiscoError(rc, "disco_draft_step")
+
+    def draft_step_ppl(self, W_D, h_D, n_drafted, nll_sum, ppl_max: float, sl_max: int, token, ppl, halt,
+                       active=None, stream=None) -> None:
+        B = int(h_D.shape[0])
+        rc = self._lib.disco_draft_step_ppl(
+            self._h, _ptr(W_D, torch.bfloat16), _ptr(h_D, torch.bfloat16), B, _ptr(n_drafted, torch.int32),
+            _ptr(active, torch.uint8), _ptr(nll_sum, torch.float32), float(ppl_max), int(sl_max),
+            _ptr(token, torch.int32), _ptr(ppl, torch.float32), _ptr(halt, torch.uint8), _stream(stream))
+        if rc != OK:
+            raise DiscoError(rc, "disco_draft_step_ppl")
 
     def verify(self, W_T, H_T, draft_ids, B: int, SL: int, n_accept, bonus, target_ids=None,
                stream=None) -> None:

@@ -418,16 +418,27 @@ int disco_set_kernel_path(disco_ctx* c, int which) {
     return DISCO_OK;
 }
 
-int disco_draft_step(disco_ctx* c, const void* W_D, const void* h_D, int B, const int32_t* pos,
-                     const int32_t* n_drafted, const uint8_t* active, const disco_clf* clf, float tau,
-                     int sl_max, int32_t* token, float* conf, uint8_t* halt, float* feats, float* probs,
-                     void* stream) {
+}  // extern "C"
+
+namespace {
+// Shared body of the two draft-step entry points.  nll_sum != null selects the perplexity rule (no
+// classifier; tau is the perplexity bound).
+int draft_step_common(disco_ctx* c, const void* W_D, const void* h_D, int B, const int32_t* pos,
+                      const int32_t* n_drafted, const uint8_t* active, const disco_clf* clf, float tau,
+                      int sl_max, int32_t* token, float* conf, uint8_t* halt, float* feats, float* probs,
+                      float* nll_sum, void* stream) {
     if (!c || !W_D || !h_D || !pos || !n_drafted || !token || !conf || !halt) return DISCO_ERR_INVALID_ARG;
     if (!aligned16(W_D) || !aligned16(h_D)) return DISCO_ERR_INVALID_ARG;
     if (B < 1 || sl_max < 1) return DISCO_ERR_INVALID_ARG;
     if (B > c->max_batch) return DISCO_ERR_WORKSPACE;
-    int rc = check_clf(c, clf);
-    if (rc) return rc;
+    static const disco_clf no_clf = {nullptr, nullptr, nullptr, nullptr, 0};
+    int rc = DISCO_OK;
+    if (nll_sum) {
+        clf = &no_clf;
+    } else {
+        rc = check_clf(c, clf);
+        if (rc) return rc;
+    }
     cudaStream_t st = static_cast<cudaStream_t>(stream);
 
     TailParams p{};
@@ -453,6 +464,7 @@ int disco_draft_step(disco_ctx* c, const void* W_D, const void* h_D, int B, cons
     p.halt = halt;
     p.feats = feats;
     p.probs = probs;
+    p.nll_sum = nll_sum;
     // Measured on B200 (Vicuna head): up to 6 sequences are fastest on the tensor-core kernel with the
     // vocabulary on the TMEM lanes, more on the one with the hidden rows on the lanes; the CUDA-core
     // streaming kernel is within 10 % for one sequence and serves as the path without tensor maps.
@@ -485,6 +497,7 @@ int disco_draft_step(disco_ctx* c, const void* W_D, const void* h_D, int B, cons
         f.halt = halt;
         f.feats = feats;
         f.final_stats = c->final_stats;
+        f.nll_sum = nll_sum;
         draft_finalize_kernel<<<(B + kDraftFinalWarps - 1) / kDraftFinalWarps, kDraftFinalWarps * 32, 0, st>>>(f);
         c->launches += 1;
         if (!cuda_ok(cudaGetLastError(), "draft_finalize_kernel launch")) return DISCO_ERR_CUDA;
@@ -499,6 +512,26 @@ int disco_draft_step(disco_ctx* c, const void* W_D, const void* h_D, int B, cons
         if (cudaGetLastError() != cudaSuccess) return DISCO_ERR_CUDA;
     }
     return DISCO_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int disco_draft_step(disco_ctx* c, const void* W_D, const void* h_D, int B, const int32_t* pos,
+                     const int32_t* n_drafted, const uint8_t* active, const disco_clf* clf, float tau,
+                     int sl_max, int32_t* token, float* conf, uint8_t* halt, float* feats, float* probs,
+                     void* stream) {
+    return draft_step_common(c, W_D, h_D, B, pos, n_drafted, active, clf, tau, sl_max, token, conf, halt, feats,
+                             probs, nullptr, stream);
+}
+
+int disco_draft_step_ppl(disco_ctx* c, const void* W_D, const void* h_D, int B, const int32_t* n_drafted,
+                         const uint8_t* active, float* nll_sum, float ppl_max, int sl_max, int32_t* token,
+                         float* ppl, uint8_t* halt, void* stream) {
+    if (!nll_sum) return DISCO_ERR_INVALID_ARG;
+    return draft_step_common(c, W_D, h_D, B, n_drafted, n_drafted, active, nullptr, ppl_max, sl_max, token, ppl,
+                             halt, nullptr, nullptr, nll_sum, stream);
 }
 
 int disco_verify_ragged(disco_ctx* c, const void* W_T, const void* H_T, const int32_t* draft_ids,

@@ -55,6 +55,7 @@ struct TailParams {
     uint8_t* halt;
     float* feats;
     float* probs;
+    float* nll_sum;      // non-null: perplexity rule instead of the classifier (tau is then the perplexity bound)
     // verification
     const int32_t* draft_ids;
     const int32_t* row_off;  // null: uniform SL
@@ -249,11 +250,28 @@ struct DraftOutputs {
     uint8_t* halt;
     float* feats;
     float* final_stats;
+    float* nll_sum;  // non-null: perplexity rule (App. F) instead of the classifier
 };
 __device__ __forceinline__ void warp_draft_epilogue(const SoftmaxState& st, unsigned long long key, float sel, float fpos,
                                                     int n_drafted, float tau, int sl_max, float* feat_s, const float* W1,
                                                     const float* b1, const float* w2, const float* b2, int Hc, int b,
                                                     const DraftOutputs& o, int lane) {
+    if (o.nll_sum) {
+        // Perplexity rule: the greedy token attains the largest logit, so -ln y(token) = ln Z.  The caller
+        // keeps the running sum over the tokens drafted in this iteration; halt when the perplexity of
+        // that run exceeds the bound (here passed in tau) or the cap is reached.
+        if (lane == 0) {
+            const float nll = o.nll_sum[b] + logf(st.Z);
+            const float ppl = expf(nll / static_cast<float>(n_drafted));
+            o.nll_sum[b] = nll;
+            o.token[b] = key_index(key);
+            o.conf[b] = ppl;
+            o.halt[b] = ((ppl > tau) || (n_drafted >= sl_max)) ? 1 : 0;
+            o.final_stats[2 * b] = st.m;
+            o.final_stats[2 * b + 1] = st.Z;
+        }
+        return;
+    }
     const float inv_Z = 1.f / st.Z;
     const float prob = (lane < kTopK && sel > DISCO_NEG_INF) ? __expf(sel - st.m) * inv_Z : 0.f;
     const float ent = __logf(st.Z) - st.S * inv_Z;
@@ -305,7 +323,7 @@ __device__ __forceinline__ void finalize_draft_seq(const TailParams& p, int b, i
     const int Hc = p.clf_H;
     SoftmaxState st;
     st.m = r.m, st.Z = r.Z, st.S = r.S;
-    const DraftOutputs o{p.token, p.conf, p.halt, p.feats, p.final_stats};
+    const DraftOutputs o{p.token, p.conf, p.halt, p.feats, p.final_stats, p.nll_sum};
     warp_draft_epilogue(st, r.key, lane_pick(r, lane), fpos, n_drafted, p.tau, p.sl_max, feat16, clf_s, clf_s + Hc * kNFeat,
                         clf_s + Hc * (kNFeat + 1), clf_s + Hc * (kNFeat + 2), Hc, b, o, lane);
 }
@@ -422,7 +440,7 @@ __global__ void __launch_bounds__((NW + 1) * 32, 1) stream_tail_kernel(const __g
     }
 
     // -------------------- consumers --------------------
-    if (DRAFT) {  // classifier parameters -> shared, asynchronously; only the last CTA reads them
+    if (DRAFT && p.clf_H > 0) {  // classifier parameters -> shared, asynchronously; only the last CTA reads them
         const int Hc = p.clf_H;
         const int n1 = Hc * kNFeat;
         for (int i = tid; i < n1 + 2 * Hc + 1; i += BAR_THREADS) {

@@ -178,7 +178,7 @@ umma_gemv_draft_kernel(const __grid_constant__ CUtensorMap tmap_W, const __grid_
         const int ew = warp - 2;    // 0..3: role in the reductions
         const int quad = warp & 3;  // TMEM lane quadrant this warp may read
         const int tid = ew * 32 + lane;
-        {  // classifier parameters -> shared, asynchronously; only the last CTA reads them
+        if (p.clf_H > 0) {  // classifier parameters -> shared, asynchronously; only the last CTA reads them
             const int Hc = p.clf_H;
             const int n1 = Hc * kNFeat;
             for (int i = tid; i < n1 + 2 * Hc + 1; i += BAR_THREADS) {

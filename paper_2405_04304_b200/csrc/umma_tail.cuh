@@ -435,6 +435,7 @@ struct DraftFinalParams {
     uint8_t* halt;
     float* feats;
     float* final_stats;
+    float* nll_sum;
 };
 
 __global__ void __launch_bounds__(128) verify_finalize_kernel(const VerifyFinalParams p) {
@@ -494,7 +495,7 @@ __global__ void __launch_bounds__(kDraftFinalWarps * 32) draft_finalize_kernel(c
     warp_reduce_records(r, 5);
     SoftmaxState st;
     st.m = r.m, st.Z = r.Z, st.S = r.S;
-    const DraftOutputs o{p.token, p.conf, p.halt, p.feats, p.final_stats};
+    const DraftOutputs o{p.token, p.conf, p.halt, p.feats, p.final_stats, p.nll_sum};
     warp_draft_epilogue(st, r.key, lane_pick(r, lane), fpos, n_drafted, p.tau, p.sl_max, feat_s + warp * 16, p.clf_W1,
                         p.clf_b1, p.clf_w2, p.clf_b2, p.clf_H, b, o, lane);
 }

@@ -377,3 +377,43 @@ def test_batched_draft_step_at_full_size(oracle, name):
     assert exempt <= max(2, B // 50)
     assert ctx.device_status() == 0
     ctx.close()
+
+
+# ---------------------------------------------------------------------------------- perplexity stopping rule
+@pytest.mark.parametrize("path", [0, 1, 2, 3])
+@pytest.mark.parametrize("V,d,B", [(700, 40, 1), (4099, 264, 5), (32000, 768, 1), (5000, 128, 40)])
+def test_draft_step_with_perplexity_rule(oracle, path, V, d, B):
+    if (path == 1 or path == 3) and B > 16:
+        pytest.skip("kernel family not meant for this many sequences")
+    W = inputs.lm_head(V, d, seed=V + d, std=0.3)
+    ctx = _ctx(V, d, 8, max_batch=B)
+    ctx.set_kernel_path(path)
+    Wg = W.cuda()
+    active = None if B < 3 else (np.arange(B) % 4 != 1).astype(np.uint8)
+    nll_ref = np.zeros(B)
+    nll_gpu = torch.zeros(B, dtype=torch.float32, device="cuda")
+    bound = float(np.exp(0.6 * np.log(V)))
+    for n in (1, 2, 3):                                        # three consecutive draft steps of one iteration
+        h = inputs.hidden(B, d, seed=V + 17 * n)
+        nd = np.full(B, n, np.int32)
+        tok_r, ppl_r, halt_r, gap_r, nll_ref = oracle.draft_step_ppl(_bits(W), _bits(h), nd, nll_ref, bound, 3,
+                                                                       active=active, nthreads=8)
+        token = torch.full((B,), -7, dtype=torch.int32, device="cuda")
+        ppl = torch.full((B,), -7.0, dtype=torch.float32, device="cuda")
+        halt = torch.full((B,), 77, dtype=torch.uint8, device="cuda")
+        ctx.draft_step_ppl(Wg, h.cuda(), torch.from_numpy(nd).cuda(), nll_gpu, bound, 3, token, ppl, halt,
+                           active=None if active is None else torch.from_numpy(active).cuda())
+        torch.cuda.synchronize()
+        token, ppl, halt = token.cpu().numpy(), ppl.cpu().numpy(), halt.cpu().numpy()
+        for b in range(B):
+            if active is not None and not active[b]:
+                assert token[b] == -7 and halt[b] == 77 and ppl[b] == -7.0
+                continue
+            if gap_r[b] >= 1e-3:
+                assert token[b] == tok_r[b]
+            assert abs(ppl[b] - ppl_r[b]) <= 2e-3 * ppl_r[b]   # relative: a perplexity is not bounded by 1
+            if abs(ppl_r[b] - bound) > 2e-3 * bound:
+                assert halt[b] == halt_r[b]
+        np.testing.assert_allclose(nll_gpu.cpu().numpy(), nll_ref, rtol=1e-4, atol=1e-4)
+    assert ctx.device_status() == 0
+    ctx.close()

@@ -366,3 +366,50 @@ def test_eq1_numerator_golden_and_sample_mean(oracle):
     sigma = emitted.std() / math.sqrt(N)
     assert abs(emitted.mean() - mean) < 3 * sigma + 1e-9
     assert abs(mean - 3.68928) < 1e-3              # Eq. 1 numerator at alpha = 0.8, gamma = 5
+
+
+# ------------------------------------------------------------------ perplexity stopping rule (App. F)
+def test_ppl_rule_uniform_distribution_has_perplexity_V(oracle):
+    V, d = 50, 8
+    W = bits_of(torch.randn(V, d, generator=torch.Generator().manual_seed(31)))
+    h0 = bits_of(torch.zeros(1, d))
+    nll = np.zeros(1)
+    for n in (1, 2, 3):                       # every token of a uniform model costs ln V: perplexity V at any length
+        tok, ppl, halt, gap, nll = oracle.draft_step_ppl(W, h0, [n], nll, ppl_max=V + 1.0, sl_max=10)
+        assert tok[0] == 0 and abs(ppl[0] - V) < 1e-9 and halt[0] == 0
+        assert abs(nll[0] - n * math.log(V)) < 1e-12
+    tok, ppl, halt, gap, _ = oracle.draft_step_ppl(W, h0, [1], np.zeros(1), ppl_max=V - 1.0, sl_max=10)
+    assert halt[0] == 1                       # perplexity above the bound: stop drafting
+    tok, ppl, halt, gap, _ = oracle.draft_step_ppl(W, h0, [10], np.zeros(1), ppl_max=1e9, sl_max=10)
+    assert halt[0] == 1                       # the cap still applies
+
+
+def test_ppl_rule_is_geometric_mean_of_inverse_token_probabilities(oracle):
+    from scipy.special import softmax as sp_softmax
+    g = torch.Generator().manual_seed(32)
+    V, d = 40, 12
+    Wt = torch.randn(V, d, generator=g).to(torch.bfloat16)
+    hs = torch.randn(3, d, generator=g).to(torch.bfloat16)
+    nll = np.zeros(1)
+    inv = []
+    for n in range(1, 4):
+        h = hs[n - 1:n]
+        tok, ppl, halt, gap, nll = oracle.draft_step_ppl(bits_of(Wt), bits_of(h), [n], nll, 1e9, 10)
+        y = sp_softmax(h.double().numpy() @ Wt.double().numpy().T, axis=1)[0]
+        assert tok[0] == int(np.argmax(y))
+        inv.append(1.0 / y.max())
+        assert abs(ppl[0] - float(np.prod(inv)) ** (1.0 / n)) < 1e-9 * ppl[0]
+    # a confident (peaked) step pulls the perplexity towards 1
+    peaked = (Wt[5].float() * 50).to(torch.bfloat16).view(1, d)
+    _, ppl1, _, _, _ = oracle.draft_step_ppl(bits_of(Wt), bits_of(peaked), [1], np.zeros(1), 1e9, 10)
+    assert 1.0 <= ppl1[0] < 1.001
+
+
+def test_ppl_rule_halts_monotonically_in_the_bound_and_skips_inactive(oracle):
+    W, h, _ = _small_problem(33, B=3)
+    nd = np.array([1, 2, 3], np.int32)
+    halts = [oracle.draft_step_ppl(bits_of(W), bits_of(h), nd, np.zeros(3), bound, 9)[2] for bound in (40.0, 20.0, 5.0)]
+    assert np.all(halts[0] <= halts[1]) and np.all(halts[1] <= halts[2])
+    tok, ppl, halt, gap, nll = oracle.draft_step_ppl(bits_of(W), bits_of(h), nd, np.full(3, 0.25), 20.0, 9,
+                                                     active=np.array([1, 0, 1], np.uint8))
+    assert tok[1] == -1 and halt[1] == 255 and nll[1] == 0.25 and nll[0] > 0.25
