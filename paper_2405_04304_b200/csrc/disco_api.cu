@@ -178,8 +178,8 @@ bool umma_possible(const disco_ctx* c, int R) {
 
 // Launch the tcgen05 kernel for R hidden rows of width d against the LM head W [V, d].
 template <bool DRAFT>
-int launch_umma(disco_ctx* c, const void* W, const void* H, int d, int R, float* probs, int* n_partials,
-                const UmmaParams* fused, cudaStream_t st) {
+int launch_umma(disco_ctx* c, const void* W, const void* H, int d, int R, float* probs,
+                const DraftFinalParams* draft_final, const UmmaParams* fused, cudaStream_t st) {
     UmmaParams p{};
     if (fused) p = *fused;  // verification finished by the main kernel's last CTA
     p.V = c->V;
@@ -195,9 +195,15 @@ int launch_umma(disco_ctx* c, const void* W, const void* H, int d, int R, float*
     p.TR = (c->V + p.CN * p.TPC - 1) / (p.CN * p.TPC);
     p.TRN = std::max(16, (p.TR + 15) / 16 * 16);
     p.a_rows = p.MT > 1 ? 128 : std::max(8, (R + 7) / 8 * 8);
-    // The A stage holds a_rows rows.  The MMA still reads 128 rows from its start: what lies behind the
-    // tile (other stages of the ring, always inside it) only feeds accumulator lanes nobody reads.
-    p.a_bytes = (p.a_rows * 128 + 1023) / 1024 * 1024;
+    // Draft step with few rows: copies of the rows fill the other TMEM lane quadrants, so that the
+    // epilogue (heavy there) runs on every warp scheduler.  Verification's epilogue is a compare per
+    // logit and keeps the smaller stage instead.
+    p.rep = (DRAFT && R <= 64) ? (R <= 32 ? 4 : 2) : 1;
+    p.rows_pad = 128 / p.rep;
+    // The A stage holds a_rows rows (rep copies, rows_pad rows apart).  The MMA still reads 128 rows from
+    // its start: what lies behind the tile (other stages of the ring, always inside it) or between the
+    // copies only feeds accumulator lanes nobody reads.
+    p.a_bytes = p.rep > 1 ? 128 * 128 : (p.a_rows * 128 + 1023) / 1024 * 1024;
     p.b_bytes = (p.TRN * 128 + 1023) / 1024 * 1024;
     p.stages = std::max(2, std::min(kUmmaMaxStages, kUmmaRingBytes / (p.a_bytes + p.b_bytes)));
     p.status = c->status;
@@ -205,7 +211,6 @@ int launch_umma(disco_ctx* c, const void* W, const void* H, int d, int R, float*
     p.part_rec = reinterpret_cast<float4*>(c->part_rec);
     p.probs = probs;
     if (DRAFT && (p.CN > c->part_slots || R > c->part_rows)) return DISCO_ERR_WORKSPACE;
-    if (n_partials) *n_partials = p.CN;
     CUtensorMap tmap_W, tmap_H;
     if (!encode_bf16_2d(c, &tmap_W, W, c->V, d, p.TRN) || !encode_bf16_2d(c, &tmap_H, H, R, d, p.a_rows))
         return DISCO_ERR_CUDA;
@@ -222,12 +227,24 @@ int launch_umma(disco_ctx* c, const void* W, const void* H, int d, int R, float*
     cfg.blockDim = dim3(kUmmaThreads);
     cfg.dynamicSmemBytes = kUmmaSmemBytes;
     cfg.stream = st;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    // The draft step's second phase waits for every CTA of the grid: a cooperative launch makes the
+    // driver refuse the launch unless all of them can be resident at once.
+    cudaLaunchAttribute attr[2];
+    int na = 0;
+    if (DRAFT) {
+        attr[na].id = cudaLaunchAttributeCooperative;
+        attr[na].val.cooperative = 1;
+        ++na;
+    }
+    if (c->pdl) {
+        attr[na].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[na].val.programmaticStreamSerializationAllowed = 1;
+        ++na;
+    }
     cfg.attrs = attr;
-    cfg.numAttrs = c->pdl ? 1 : 0;
-    const cudaError_t e = cudaLaunchKernelEx(&cfg, kern, tmap_W, tmap_H, p);
+    cfg.numAttrs = na;
+    const DraftFinalParams f = draft_final ? *draft_final : DraftFinalParams{};
+    const cudaError_t e = cudaLaunchKernelEx(&cfg, kern, tmap_W, tmap_H, p, f);
     c->launches += 1;
     return cuda_ok(e, "umma_tail_kernel launch") ? DISCO_OK : DISCO_ERR_CUDA;
 }
@@ -475,13 +492,8 @@ int draft_step_common(disco_ctx* c, const void* W_D, const void* h_D, int B, con
         rc = launch_gemv(c, p, st);
         if (rc) return rc;
     } else if (use_umma) {
-        int np = 0;
-        rc = launch_umma<true>(c, W_D, h_D, c->d_draft, B, probs, &np, nullptr, st);
-        if (rc) return rc;
         DraftFinalParams f{};
-        f.part_rec = reinterpret_cast<const float4*>(c->part_rec);
         f.B = B;
-        f.NP = np;
         f.pos = pos;
         f.n_drafted = n_drafted;
         f.active = active;
@@ -498,9 +510,9 @@ int draft_step_common(disco_ctx* c, const void* W_D, const void* h_D, int B, con
         f.feats = feats;
         f.final_stats = c->final_stats;
         f.nll_sum = nll_sum;
-        draft_finalize_kernel<<<(B + kDraftFinalWarps - 1) / kDraftFinalWarps, kDraftFinalWarps * 32, 0, st>>>(f);
-        c->launches += 1;
-        if (!cuda_ok(cudaGetLastError(), "draft_finalize_kernel launch")) return DISCO_ERR_CUDA;
+        f.ticket = c->ticket + 48;
+        rc = launch_umma<true>(c, W_D, h_D, c->d_draft, B, probs, &f, nullptr, st);
+        if (rc) return rc;
     } else {
         rc = run_stream<true>(c, p, clf->H, st);
         if (rc) return rc;

@@ -32,7 +32,7 @@ constexpr int kUmmaBK = 64;               // k elements per stage (one 128-byte 
 constexpr int kUmmaRingBytes = 192 * 1024;  // shared memory for the operand stages
 constexpr int kUmmaEpiWarps = 8;
 constexpr int kUmmaThreads = (2 + kUmmaEpiWarps) * 32;
-constexpr int kUmmaXchBytes = 128 * 16 * 4;  // one 64-byte record per hidden row of the tile
+constexpr int kUmmaXchBytes = 14 * 1024;  // 64-byte records handed between the warps that share a hidden row
 constexpr int kUmmaSmemBytes =
     kUmmaRingBytes + 1024 /*align*/ + 512 /*barriers*/ + kUmmaXchBytes;
 
@@ -44,6 +44,10 @@ struct UmmaParams {
     int TR;      // vocabulary rows per tile; the MMA and the TMA box use TRN = TR rounded up to 16
     int TRN;
     int a_rows;  // rows of the H box (multiple of 8, <= 128)
+    // Draft step with at most 64 hidden rows: the H box is loaded `rep` times per stage, rows_pad rows
+    // apart, so every TMEM lane quadrant holds a copy of each row and all epilogue warps share the columns.
+    int rep;       // 1, 2 or 4
+    int rows_pad;  // 128 / rep
     int stages;  // ring depth (<= kUmmaMaxStages); stage s holds an A tile of a_bytes and a B tile of b_bytes
     int a_bytes, b_bytes;  // multiples of 1024
     int* status;
@@ -135,6 +139,73 @@ __device__ __forceinline__ uint32_t umma_idesc(int n) {
     return (1u << 4) | (1u << 7) | (1u << 10) | (static_cast<uint32_t>(n >> 3) << 17) | ((128u >> 4) << 24);
 }
 
+// Draft step, second phase: one warp per sequence merges the per-CTA partial records, forms the
+// features of Eq. 2 and runs the halt classifier and the stopping rule.
+struct DraftFinalParams {
+    int B;
+    const int32_t* pos;
+    const int32_t* n_drafted;
+    const uint8_t* active;
+    const float* clf_W1;
+    const float* clf_b1;
+    const float* clf_w2;
+    const float* clf_b2;
+    int clf_H;
+    float tau;
+    int sl_max;
+    int32_t* token;
+    float* conf;
+    uint8_t* halt;
+    float* feats;
+    float* final_stats;
+    float* nll_sum;
+    unsigned int* ticket;  // [0] CTAs whose records are published, [1] finishing warps that are done
+};
+
+__device__ __forceinline__ unsigned int load_acquire(const unsigned int* p) {
+    unsigned int v;
+    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+
+// One warp finishes sequence b from its NP partial records.
+__device__ __forceinline__ void umma_finish_sequence(const DraftFinalParams& p, const float4* part_rec, int NP, int b,
+                                                     float* feat16, int lane) {
+    if (p.active && !p.active[b]) return;
+    const float fpos = static_cast<float>(p.pos[b]);
+    const int n_drafted = p.n_drafted[b];
+    const float4* recs = part_rec + (size_t)b * NP * 4;
+    LaneRecord r;
+    r.clear();
+    constexpr int kPerLane = 5;  // 160 records per L2 round trip
+#pragma unroll 1
+    for (int c0 = 0; c0 < NP; c0 += 32 * kPerLane) {
+        float4 q[kPerLane][4];
+#pragma unroll
+        for (int j = 0; j < kPerLane; ++j) {
+            const int c = c0 + j * 32 + lane;
+            if (c < NP) {
+                const float4* src = recs + (size_t)c * 4;
+                q[j][0] = __ldcg(src), q[j][1] = __ldcg(src + 1), q[j][2] = __ldcg(src + 2), q[j][3] = __ldcg(src + 3);
+            } else {
+                q[j][0] = make_float4(0.f, 0.f, 0.f, 0.f);
+            }
+        }
+#pragma unroll
+        for (int j = 0; j < kPerLane; ++j) {
+            LaneRecord o;
+            o.set(q[j][0], q[j][1], q[j][2], q[j][3]);
+            r.absorb(o);
+        }
+    }
+    warp_reduce_records(r, 5);
+    SoftmaxState st;
+    st.m = r.m, st.Z = r.Z, st.S = r.S;
+    const DraftOutputs o{p.token, p.conf, p.halt, p.feats, p.final_stats, p.nll_sum};
+    warp_draft_epilogue(st, r.key, lane_pick(r, lane), fpos, n_drafted, p.tau, p.sl_max, feat16, p.clf_W1, p.clf_b1,
+                        p.clf_w2, p.clf_b2, p.clf_H, b, o, lane);
+}
+
 // Vocabulary tile t covers rows [t * TR, min(V, (t + 1) * TR)).  The TMA box and the MMA take TRN >= TR
 // rows; the extra rows (the next tile's first rows, or zero fill past V) land in columns the epilogue skips.
 // ---------------------------------------------------------------------------------------------
@@ -143,7 +214,7 @@ __device__ __forceinline__ uint32_t umma_idesc(int n) {
 template <bool DRAFT>
 __global__ void __launch_bounds__(kUmmaThreads, 1)
 umma_tail_kernel(const __grid_constant__ CUtensorMap tmap_W, const __grid_constant__ CUtensorMap tmap_H,
-                 const UmmaParams p) {
+                 const UmmaParams p, const DraftFinalParams f) {
     extern __shared__ uint8_t smem_dyn[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~uintptr_t(1023));
     uint8_t* a_tiles = smem;
@@ -191,7 +262,7 @@ umma_tail_kernel(const __grid_constant__ CUtensorMap tmap_W, const __grid_consta
         // ------------------------------ producer ------------------------------
         if (lane == 0) {
             int stage = 0, phase = 0;
-            const uint32_t bytes = (uint32_t)(p.a_rows + p.TRN) * 128u;
+            const uint32_t bytes = (uint32_t)(p.rep * p.a_rows + p.TRN) * 128u;
             // The LM head is never written by this library: its first tiles are requested before the
             // dependency wait, the hidden-state tiles of the same stages right after it.
             int pre = 0;
@@ -216,7 +287,9 @@ umma_tail_kernel(const __grid_constant__ CUtensorMap tmap_W, const __grid_consta
                         mbar_arrive_expect_tx(&full[stage], bytes);
                         tma_load_2d(b_tiles + stage * p.b_bytes, &tmap_W, kb * kUmmaBK, v0, &full[stage]);
                     }
-                    tma_load_2d(a_tiles + stage * p.a_bytes, &tmap_H, kb * kUmmaBK, m_tile * 128, &full[stage]);
+                    for (int c = 0; c < p.rep; ++c)
+                        tma_load_2d(a_tiles + stage * p.a_bytes + c * p.rows_pad * 128, &tmap_H, kb * kUmmaBK,
+                                    m_tile * 128, &full[stage]);
                     if (++stage == p.stages) {
                         stage = 0;
                         phase ^= 1;
@@ -258,9 +331,13 @@ umma_tail_kernel(const __grid_constant__ CUtensorMap tmap_W, const __grid_consta
         asm volatile("griddepcontrol.wait;" ::: "memory");  // scratch and outputs belong to the predecessor until now
         const int ew = warp - 2;            // 0 .. kUmmaEpiWarps-1
         const int quad = warp & 3;          // TMEM lane quadrant this warp may read
-        const int half = ew >> 2;           // which share of the columns (two warps per quadrant)
-        const int row = m_tile * 128 + quad * 32 + lane;
-        const bool warp_has_rows = (m_tile * 128 + quad * 32) < p.R;
+        // The warps that hold the same hidden rows (two per quadrant, times the copies of the rows in
+        // other quadrants) split the columns of a tile into `nshare` shares.
+        const int tile_row = (quad * 32) % p.rows_pad + lane;     // row within this tile of hidden rows
+        const int share = (ew >> 2) * p.rep + (quad * 32) / p.rows_pad;
+        const int nshare = 2 * p.rep;
+        const int row = m_tile * 128 + tile_row;
+        const bool warp_has_rows = (m_tile * 128 + (quad * 32) % p.rows_pad) < p.R;
         const bool valid = row < p.R;
 
         float best_v = DISCO_NEG_INF;
@@ -280,8 +357,8 @@ umma_tail_kernel(const __grid_constant__ CUtensorMap tmap_W, const __grid_consta
             const int ncols = min(p.TR, p.V - v0);  // further columns belong to the next tile or lie past V
             if (warp_has_rows) {
                 const int nchunks = (ncols + 31) >> 5;
-                const int c_lo = (half == 0) ? 0 : (nchunks + 1) / 2;
-                const int c_hi = (half == 0) ? (nchunks + 1) / 2 : nchunks;
+                const int c_lo = (nchunks * share + nshare - 1) / nshare;
+                const int c_hi = (nchunks * (share + 1) + nshare - 1) / nshare;
                 for (int c = c_lo; c < c_hi; ++c) {
                     float z[32];
                     tmem_ld32(tmem_base + buf * 256 + c * 32 + (static_cast<uint32_t>(quad * 32) << 16), z);
@@ -339,10 +416,10 @@ umma_tail_kernel(const __grid_constant__ CUtensorMap tmap_W, const __grid_consta
 
         // one result per hidden row and CTA
         if (DRAFT) {
-            // the two warps of a quadrant hold the same rows: the second hands its state to the first
+            // the warps that hold the same rows hand their state to the one with share 0
             unsigned long long key = best_i != kNoIndex ? argmax_key(best_v, best_i) : 0ull;
-            float4* mine = xch + (quad * 32 + lane) * 4;
-            if (half == 1) {
+            if (share != 0) {
+                float4* mine = xch + ((share - 1) * p.rows_pad + tile_row) * 4;
                 mine[0] = make_float4(st.m, st.Z, st.S, 0.f);
                 mine[1] = make_float4(top.t[0], top.t[1], top.t[2], top.t[3]);
                 mine[2] = make_float4(top.t[4], top.t[5], top.t[6], top.t[7]);
@@ -350,22 +427,60 @@ umma_tail_kernel(const __grid_constant__ CUtensorMap tmap_W, const __grid_consta
                                       __uint_as_float((uint32_t)(key >> 32)));
             }
             named_barrier_sync(2, kUmmaEpiWarps * 32);
-            if (half == 0 && valid) {
-                const float4 q = mine[0], a = mine[1], bq = mine[2], cq = mine[3];
-                st.merge(q.x, q.y, q.z);
-                const unsigned long long k2 =
-                    (static_cast<unsigned long long>(__float_as_uint(cq.w)) << 32) | __float_as_uint(cq.z);
-                key = k2 > key ? k2 : key;
-                const float lv[kTopK] = {a.x, a.y, a.z, a.w, bq.x, bq.y, bq.z, bq.w, cq.x, cq.y};
+            if (share == 0 && valid) {
+                for (int o = 0; o < nshare - 1; ++o) {
+                    const float4* theirs = xch + (o * p.rows_pad + tile_row) * 4;
+                    const float4 q = theirs[0], a = theirs[1], bq = theirs[2], cq = theirs[3];
+                    st.merge(q.x, q.y, q.z);   // a share without columns has Z = 0 and changes nothing
+                    const unsigned long long k2 =
+                        (static_cast<unsigned long long>(__float_as_uint(cq.w)) << 32) | __float_as_uint(cq.z);
+                    key = k2 > key ? k2 : key;
+                    const float lv[kTopK] = {a.x, a.y, a.z, a.w, bq.x, bq.y, bq.z, bq.w, cq.x, cq.y};
 #pragma unroll
-                for (int k = 0; k < kTopK; ++k)
-                    if (lv[k] > top.t[kTopK - 1]) top.push(lv[k]);
+                    for (int k = 0; k < kTopK; ++k)
+                        if (lv[k] > top.t[kTopK - 1]) top.push(lv[k]);
+                }
                 float4* rec = p.part_rec + ((size_t)row * p.CN + nslot) * 4;
                 rec[0] = make_float4(st.m, st.Z, st.S, 0.f);
                 rec[1] = make_float4(top.t[0], top.t[1], top.t[2], top.t[3]);
                 rec[2] = make_float4(top.t[4], top.t[5], top.t[6], top.t[7]);
                 rec[3] = make_float4(top.t[8], top.t[9], __uint_as_float((uint32_t)(key & 0xffffffffull)),
                                      __uint_as_float((uint32_t)(key >> 32)));
+            }
+            // Second phase inside the same (cooperative) launch: every CTA publishes its records and
+            // counts itself in; the sequences are then shared out, one warp each, over the CTAs, and a
+            // warp starts once all CTAs are counted.  The wait is bounded like every other one.
+            __threadfence();
+            named_barrier_sync(2, kUmmaEpiWarps * 32);
+            if (ew == 0 && lane == 0) atomicAdd(f.ticket, 1u);
+            const int first = ew * (int)gridDim.x + (int)blockIdx.x;
+            if (first < f.B) {
+                bool ok = true;
+                if (lane == 0) {
+                    const long long t0 = clock64();
+                    while (load_acquire(f.ticket) < gridDim.x) {
+                        if (*reinterpret_cast<volatile int*>(p.status) == DISCO_ERR_TIMEOUT ||
+                            clock64() - t0 > kWaitBudgetClocks) {
+                            record_status(p.status, DISCO_ERR_TIMEOUT);
+                            ok = false;
+                            break;
+                        }
+                        __nanosleep(64);
+                    }
+                }
+                ok = __shfl_sync(kFullMask, ok, 0);
+                __threadfence();
+                if (ok) {
+                    float* feat16 = reinterpret_cast<float*>(xch) + ew * 16;  // the exchange area is free again
+                    for (int b = first; b < f.B; b += kUmmaEpiWarps * (int)gridDim.x)
+                        umma_finish_sequence(f, p.part_rec, p.CN, b, feat16, lane);
+                }
+                // the last finishing warp of the grid puts the counters back to zero for the next call
+                const unsigned int nwarps = (unsigned int)min(f.B, kUmmaEpiWarps * (int)gridDim.x);
+                if (lane == 0 && atomicAdd(f.ticket + 1, 1u) == nwarps - 1) {
+                    f.ticket[0] = 0u;
+                    f.ticket[1] = 0u;
+                }
             }
         } else {
             if (valid && best_i != kNoIndex) atomicMax(p.keys + row, argmax_key(best_v, best_i));
@@ -415,29 +530,6 @@ struct VerifyFinalParams {
     unsigned int* ticket;
 };
 
-// Draft step: one warp per sequence merges the per-CTA partials, forms the features of Eq. 2 and
-// runs the halt classifier and the stopping rule.
-struct DraftFinalParams {
-    const float4* part_rec;
-    int B, NP;  // partial records per sequence
-    const int32_t* pos;
-    const int32_t* n_drafted;
-    const uint8_t* active;
-    const float* clf_W1;
-    const float* clf_b1;
-    const float* clf_w2;
-    const float* clf_b2;
-    int clf_H;
-    float tau;
-    int sl_max;
-    int32_t* token;
-    float* conf;
-    uint8_t* halt;
-    float* feats;
-    float* final_stats;
-    float* nll_sum;
-};
-
 __global__ void __launch_bounds__(128) verify_finalize_kernel(const VerifyFinalParams p) {
     __shared__ int s_last;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -455,49 +547,6 @@ __global__ void __launch_bounds__(128) verify_finalize_kernel(const VerifyFinalP
     __threadfence();
     for (int r = threadIdx.x; r < p.R; r += blockDim.x) p.keys[r] = 0ull;  // every reader is done
     if (threadIdx.x == 0) *p.ticket = 0u;
-}
-
-constexpr int kDraftFinalWarps = 4;
-
-// One warp per sequence: reduce the per-CTA records and run the epilogue.
-__global__ void __launch_bounds__(kDraftFinalWarps * 32) draft_finalize_kernel(const DraftFinalParams p) {
-    __shared__ float feat_s[kDraftFinalWarps * 16];
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int b = blockIdx.x * kDraftFinalWarps + warp;
-    if (b >= p.B) return;
-    if (p.active && !p.active[b]) return;
-    const float fpos = static_cast<float>(p.pos[b]);
-    const int n_drafted = p.n_drafted[b];
-    const float4* recs = p.part_rec + (size_t)b * p.NP * 4;
-    LaneRecord r;
-    r.clear();
-    constexpr int kPerLane = 5;  // 160 records per L2 round trip
-#pragma unroll 1
-    for (int c0 = 0; c0 < p.NP; c0 += 32 * kPerLane) {
-        float4 q[kPerLane][4];
-#pragma unroll
-        for (int j = 0; j < kPerLane; ++j) {
-            const int c = c0 + j * 32 + lane;
-            if (c < p.NP) {
-                const float4* src = recs + (size_t)c * 4;
-                q[j][0] = __ldcg(src), q[j][1] = __ldcg(src + 1), q[j][2] = __ldcg(src + 2), q[j][3] = __ldcg(src + 3);
-            } else {
-                q[j][0] = make_float4(0.f, 0.f, 0.f, 0.f);
-            }
-        }
-#pragma unroll
-        for (int j = 0; j < kPerLane; ++j) {
-            LaneRecord o;
-            o.set(q[j][0], q[j][1], q[j][2], q[j][3]);
-            r.absorb(o);
-        }
-    }
-    warp_reduce_records(r, 5);
-    SoftmaxState st;
-    st.m = r.m, st.Z = r.Z, st.S = r.S;
-    const DraftOutputs o{p.token, p.conf, p.halt, p.feats, p.final_stats, p.nll_sum};
-    warp_draft_epilogue(st, r.key, lane_pick(r, lane), fpos, n_drafted, p.tau, p.sl_max, feat_s + warp * 16, p.clf_W1,
-                        p.clf_b1, p.clf_w2, p.clf_b2, p.clf_H, b, o, lane);
 }
 
 }  // namespace disco
