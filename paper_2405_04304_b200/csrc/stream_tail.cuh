@@ -66,13 +66,17 @@ struct TailParams {
 };
 
 constexpr int kRecordWords = 16;  // one partial record: m, Z, S, -, 10 logits, key (2 words)
+// Shared scratch owned by one warp in the second phase: 16 words for the features of Eq. 2, then the
+// candidate list of warp_merge_partials (counter, 64 candidates, 10 results).
+constexpr int kWarpScratchWords = 112;
+constexpr int kMergeCandidates = 64;
 
 inline size_t stream_tail_smem_bytes(int RT, int NW, int d, int stages, uint32_t slot_bytes, int clf_H) {
     size_t b = (size_t)stages * slot_bytes;           // ring
     b += (size_t)RT * d * 2;                          // hidden tile
     b += (size_t)stages * 16;                         // full/empty barriers
     b += (size_t)(NW * RT + 1) * kRecordWords * 4;    // warp records / finalize staging (+ carry)
-    b += (size_t)NW * 16 * 4;                         // features, 16 words per warp
+    b += (size_t)NW * kWarpScratchWords * 4;          // second-phase scratch per warp
     b += ((size_t)clf_H * (kNFeat + 2) + 4) * 4;      // classifier parameters
     return b + 128;
 }
@@ -191,6 +195,144 @@ __device__ __forceinline__ float lane_pick(const LaneRecord& r, int lane) {
 
 __device__ __forceinline__ int ceil_log2(int n) { return n <= 1 ? 0 : 32 - __clz(n - 1); }
 
+// Result of merging the partial records of one sequence: statistics and key in every lane, the k-th
+// largest logit in lane k < 10 (-inf elsewhere).
+struct MergedPartials {
+    SoftmaxState st;
+    unsigned long long key;
+    float sel;
+};
+
+// Merge the NP partial records of one sequence (64 bytes each, consecutive) by one warp.
+// Up to 160 records take one L2 round trip, five per lane, and the ten largest logits are found by
+// selection instead of a merge tree: the tenth largest of the lanes' largest logits is a lower bound
+// on the tenth largest overall, so only the few logits at or above it are gathered (shared memory) and
+// ranked against each other.  More than 160 records, or more than kMergeCandidates candidates (many
+// equal logits), fall back to pairwise list merges.  scratch: kWarpScratchWords - 16 words of the warp.
+__device__ __forceinline__ MergedPartials warp_merge_partials(const float4* recs, int NP, float* scratch, int lane) {
+    constexpr int kPerLane = 5;
+    MergedPartials out;
+    bool fast = NP <= 32 * kPerLane;
+    if (fast) {
+        float4 q[kPerLane][4];
+#pragma unroll
+        for (int j = 0; j < kPerLane; ++j) {
+            const int c = j * 32 + lane;
+            if (c < NP) {
+                const float4* src = recs + (size_t)c * 4;
+                q[j][0] = __ldcg(src), q[j][1] = __ldcg(src + 1), q[j][2] = __ldcg(src + 2), q[j][3] = __ldcg(src + 3);
+            } else {
+                q[j][0] = q[j][1] = q[j][2] = q[j][3] = make_float4(0.f, 0.f, 0.f, 0.f);  // Z = 0: empty
+            }
+        }
+        int* cnt = reinterpret_cast<int*>(scratch);
+        float* cand = scratch + 1;
+        float* res = cand + kMergeCandidates;
+        if (lane == 0) *cnt = 0;
+        if (lane < kTopK) res[lane] = DISCO_NEG_INF;
+        // statistics and key inside the lane
+        SoftmaxState st;
+        st.init();
+        unsigned long long key = 0ull;
+        float head = DISCO_NEG_INF;  // largest logit of this lane's records
+#pragma unroll
+        for (int j = 0; j < kPerLane; ++j) {
+            st.merge(q[j][0].x, q[j][0].y, q[j][0].z);
+            if (q[j][0].y > 0.f) {
+                const unsigned long long k2 = key_from_words(q[j][3].z, q[j][3].w);
+                key = k2 > key ? k2 : key;
+                head = fmaxf(head, q[j][1].x);
+            }
+        }
+        // across the lanes: one max-reduction for the reference maximum, one exponential, shuffle sums
+        const float M = from_ordered_bits(__reduce_max_sync(kFullMask, ordered_bits(st.m)));
+        float Zc = 0.f, Sc = 0.f;
+        if (st.Z > 0.f) {
+            const float dm = st.m - M;
+            const float e = __expf(dm);
+            Zc = st.Z * e;
+            Sc = e * (st.S + dm * st.Z);
+        }
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) {
+            Zc += __shfl_xor_sync(kFullMask, Zc, off);
+            Sc += __shfl_xor_sync(kFullMask, Sc, off);
+        }
+        const uint32_t khi = __reduce_max_sync(kFullMask, static_cast<uint32_t>(key >> 32));
+        const uint32_t klo = __reduce_max_sync(
+            kFullMask, static_cast<uint32_t>(key >> 32) == khi ? static_cast<uint32_t>(key & 0xffffffffull) : 0u);
+        out.st.m = M, out.st.Z = Zc, out.st.S = Sc;
+        out.key = (static_cast<unsigned long long>(khi) << 32) | klo;
+        // threshold: the lane whose head has rank 9 among the 32 heads (ties broken by lane)
+        int rank = 0;
+#pragma unroll
+        for (int s2 = 0; s2 < 32; ++s2) {
+            const float o = __shfl_sync(kFullMask, head, s2);
+            rank += (o > head || (o == head && s2 < lane)) ? 1 : 0;
+        }
+        const unsigned who = __ballot_sync(kFullMask, rank == kTopK - 1);
+        const float theta = __shfl_sync(kFullMask, head, __ffs(who) - 1);
+        __syncwarp();
+        // gather every logit at or above the threshold (lists are descending: stop at the first below)
+#pragma unroll
+        for (int j = 0; j < kPerLane; ++j) {
+            if (q[j][0].y > 0.f && q[j][1].x >= theta) {
+                const float lv[kTopK] = {q[j][1].x, q[j][1].y, q[j][1].z, q[j][1].w, q[j][2].x,
+                                         q[j][2].y, q[j][2].z, q[j][2].w, q[j][3].x, q[j][3].y};
+#pragma unroll
+                for (int k = 0; k < kTopK; ++k) {
+                    if (lv[k] >= theta && lv[k] > DISCO_NEG_INF) {
+                        const int slot = atomicAdd(cnt, 1);
+                        if (slot < kMergeCandidates) cand[slot] = lv[k];
+                    }
+                }
+            }
+        }
+        __syncwarp();
+        const int n = *cnt;
+        fast = n <= kMergeCandidates;
+        if (fast) {
+            // rank the candidates against each other; ranks 0..9 are the result
+            for (int idx = lane; idx < n; idx += 32) {
+                const float x = cand[idx];
+                int r = 0;
+                for (int t = 0; t < n; ++t) {
+                    const float y = cand[t];
+                    r += (y > x || (y == x && t < idx)) ? 1 : 0;
+                }
+                if (r < kTopK) res[r] = x;
+            }
+            __syncwarp();
+            out.sel = lane < kTopK ? res[lane] : DISCO_NEG_INF;
+            __syncwarp();
+            return out;
+        }
+    }
+    // general case: pairwise merges of descending lists
+    LaneRecord r;
+    r.clear();
+#pragma unroll 1
+    for (int c0 = 0; c0 < NP; c0 += 32) {
+        const int c = c0 + lane;
+        if (c < NP) {
+            const float4* src = recs + (size_t)c * 4;
+            LaneRecord o;
+            o.set(__ldcg(src), __ldcg(src + 1), __ldcg(src + 2), __ldcg(src + 3));
+            r.absorb(o);
+        }
+    }
+    warp_reduce_records(r, 5);
+    out.st.m = r.m, out.st.Z = r.Z, out.st.S = r.S;
+    out.key = __shfl_sync(kFullMask, r.key, 0);
+    out.sel = DISCO_NEG_INF;
+#pragma unroll
+    for (int k = 0; k < kTopK; ++k) {
+        const float v = __shfl_sync(kFullMask, r.l[k], 0);
+        out.sel = (lane == k) ? v : out.sel;
+    }
+    return out;
+}
+
 // Lane 0 holds (m, Z, S, key); lane k < 10 holds the k-th logit: write them as one record.
 __device__ __forceinline__ void warp_store_record(float* rec, const SoftmaxState& st, unsigned long long key, float sel,
                                                   int lane) {
@@ -287,44 +429,18 @@ __device__ __forceinline__ void warp_draft_epilogue(const SoftmaxState& st, unsi
     if (o.feats && lane < kNFeat) o.feats[(size_t)b * kNFeat + lane] = x;
 }
 
-// Draft step, sequence b, in the last CTA, by ONE warp (the warps take different sequences): every lane
-// fetches its share of the per-CTA records (four per L2 round trip) and folds them lane-locally, one
-// cross-lane reduction merges the lanes, then features, classifier and stopping rule.
-// feat16: 16 words of shared memory owned by the calling warp.
+// Draft step, sequence b, in the last CTA, by ONE warp (the warps take different sequences): merge the
+// per-CTA records, then features, classifier and stopping rule.
+// feat16: kWarpScratchWords words of shared memory owned by the calling warp.
 __device__ __forceinline__ void finalize_draft_seq(const TailParams& p, int b, int grid, float* feat16, const float* clf_s,
                                                    int lane) {
     const float fpos = static_cast<float>(p.pos[b]);  // issued early: hidden behind the merge
     const int n_drafted = p.n_drafted[b];
-    const float4* recs = p.part_rec + (size_t)b * grid * 4;
-    LaneRecord r;
-    r.clear();
-    constexpr int kPerLane = 5;  // 160 records per L2 round trip: one round trip for a grid of 148 CTAs
-#pragma unroll 1
-    for (int c0 = 0; c0 < grid; c0 += 32 * kPerLane) {
-        float4 q[kPerLane][4];
-#pragma unroll
-        for (int j = 0; j < kPerLane; ++j) {
-            const int c = c0 + j * 32 + lane;
-            if (c < grid) {
-                const float4* src = recs + (size_t)c * 4;
-                q[j][0] = __ldcg(src), q[j][1] = __ldcg(src + 1), q[j][2] = __ldcg(src + 2), q[j][3] = __ldcg(src + 3);
-            } else {
-                q[j][0] = make_float4(0.f, 0.f, 0.f, 0.f);  // Z = 0: empty
-            }
-        }
-#pragma unroll
-        for (int j = 0; j < kPerLane; ++j) {
-            LaneRecord o;
-            o.set(q[j][0], q[j][1], q[j][2], q[j][3]);
-            r.absorb(o);
-        }
-    }
-    warp_reduce_records(r, 5);
+    const MergedPartials mp = warp_merge_partials(p.part_rec + (size_t)b * grid * 4, grid, feat16 + 16, lane);
     const int Hc = p.clf_H;
-    SoftmaxState st;
-    st.m = r.m, st.Z = r.Z, st.S = r.S;
+    const SoftmaxState st = mp.st;
     const DraftOutputs o{p.token, p.conf, p.halt, p.feats, p.final_stats, p.nll_sum};
-    warp_draft_epilogue(st, r.key, lane_pick(r, lane), fpos, n_drafted, p.tau, p.sl_max, feat16, clf_s, clf_s + Hc * kNFeat,
+    warp_draft_epilogue(st, mp.key, mp.sel, fpos, n_drafted, p.tau, p.sl_max, feat16, clf_s, clf_s + Hc * kNFeat,
                         clf_s + Hc * (kNFeat + 1), clf_s + Hc * (kNFeat + 2), Hc, b, o, lane);
 }
 
@@ -397,7 +513,7 @@ __global__ void __launch_bounds__((NW + 1) * 32, 1) stream_tail_kernel(const __g
     uint64_t* empty = full + p.stages;
     float* wstate = reinterpret_cast<float*>(empty + p.stages);  // 16-byte aligned
     float* feat_s = wstate + (NW * RT + 1) * kRecordWords;
-    float* clf_s = feat_s + NW * 16;
+    float* clf_s = feat_s + NW * kWarpScratchWords;
     __shared__ int s_is_last;
 
     const int v0 = blockIdx.x * p.rows_per_cta;
@@ -643,7 +759,7 @@ __global__ void __launch_bounds__((NW + 1) * 32, 1) stream_tail_kernel(const __g
         named_barrier_sync(1, BAR_THREADS);
         for (int b = warp; b < p.R; b += NW) {
             if (p.active && !p.active[b]) continue;
-            finalize_draft_seq(p, b, grid, feat_s + warp * 16, clf_s, lane);
+            finalize_draft_seq(p, b, grid, feat_s + warp * kWarpScratchWords, clf_s, lane);
         }
         named_barrier_sync(1, BAR_THREADS);
     } else {

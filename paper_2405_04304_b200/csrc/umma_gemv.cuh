@@ -41,7 +41,7 @@ inline size_t gemv_smem_bytes(int RK, int clf_H) {
     size_t b = kGemvRing + 1024;                                 // operand ring (+ alignment)
     b += 512;                                                    // barriers, TMEM address
     b += (size_t)(kGemvEpiWarps * RK + 1) * kRecordWords * 4;    // warp records / finalize staging
-    b += kGemvEpiWarps * 16 * 4;                                 // features, 16 words per warp
+    b += kGemvEpiWarps * kWarpScratchWords * 4;                  // second-phase scratch per warp
     b += ((size_t)clf_H * (kNFeat + 2) + 4) * 4;                 // classifier parameters
     return b + 128;
 }
@@ -77,7 +77,7 @@ umma_gemv_draft_kernel(const __grid_constant__ CUtensorMap tmap_W, const __grid_
     uint32_t* tmem_base_s = reinterpret_cast<uint32_t*>(tmem_empty + 2);
     float* wstate = reinterpret_cast<float*>(smem + kGemvRing + 512);
     float* feat_s = wstate + (kGemvEpiWarps * RK + 1) * kRecordWords;
-    float* clf_s = feat_s + kGemvEpiWarps * 16;
+    float* clf_s = feat_s + kGemvEpiWarps * kWarpScratchWords;
     __shared__ int s_is_last;
 
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
@@ -257,7 +257,7 @@ umma_gemv_draft_kernel(const __grid_constant__ CUtensorMap tmap_W, const __grid_
             named_barrier_sync(1, BAR_THREADS);
             for (int b = ew; b < p.R; b += kGemvEpiWarps) {
                 if (p.active && !p.active[b]) continue;
-                finalize_draft_seq(p, b, grid, feat_s + ew * 16, clf_s, lane);
+                finalize_draft_seq(p, b, grid, feat_s + ew * kWarpScratchWords, clf_s, lane);
             }
             if (tid == 0) *p.ticket = 0u;
         }

@@ -174,35 +174,10 @@ __device__ __forceinline__ void umma_finish_sequence(const DraftFinalParams& p, 
     if (p.active && !p.active[b]) return;
     const float fpos = static_cast<float>(p.pos[b]);
     const int n_drafted = p.n_drafted[b];
-    const float4* recs = part_rec + (size_t)b * NP * 4;
-    LaneRecord r;
-    r.clear();
-    constexpr int kPerLane = 5;  // 160 records per L2 round trip
-#pragma unroll 1
-    for (int c0 = 0; c0 < NP; c0 += 32 * kPerLane) {
-        float4 q[kPerLane][4];
-#pragma unroll
-        for (int j = 0; j < kPerLane; ++j) {
-            const int c = c0 + j * 32 + lane;
-            if (c < NP) {
-                const float4* src = recs + (size_t)c * 4;
-                q[j][0] = __ldcg(src), q[j][1] = __ldcg(src + 1), q[j][2] = __ldcg(src + 2), q[j][3] = __ldcg(src + 3);
-            } else {
-                q[j][0] = make_float4(0.f, 0.f, 0.f, 0.f);
-            }
-        }
-#pragma unroll
-        for (int j = 0; j < kPerLane; ++j) {
-            LaneRecord o;
-            o.set(q[j][0], q[j][1], q[j][2], q[j][3]);
-            r.absorb(o);
-        }
-    }
-    warp_reduce_records(r, 5);
-    SoftmaxState st;
-    st.m = r.m, st.Z = r.Z, st.S = r.S;
+    const MergedPartials mp = warp_merge_partials(part_rec + (size_t)b * NP * 4, NP, feat16 + 16, lane);
+    const SoftmaxState st = mp.st;
     const DraftOutputs o{p.token, p.conf, p.halt, p.feats, p.final_stats, p.nll_sum};
-    warp_draft_epilogue(st, r.key, lane_pick(r, lane), fpos, n_drafted, p.tau, p.sl_max, feat16, p.clf_W1, p.clf_b1,
+    warp_draft_epilogue(st, mp.key, mp.sel, fpos, n_drafted, p.tau, p.sl_max, feat16, p.clf_W1, p.clf_b1,
                         p.clf_w2, p.clf_b2, p.clf_H, b, o, lane);
 }
 
@@ -471,7 +446,7 @@ umma_tail_kernel(const __grid_constant__ CUtensorMap tmap_W, const __grid_consta
                 ok = __shfl_sync(kFullMask, ok, 0);
                 __threadfence();
                 if (ok) {
-                    float* feat16 = reinterpret_cast<float*>(xch) + ew * 16;  // the exchange area is free again
+                    float* feat16 = reinterpret_cast<float*>(xch) + ew * kWarpScratchWords;  // the exchange area is free again
                     for (int b = first; b < f.B; b += kUmmaEpiWarps * (int)gridDim.x)
                         umma_finish_sequence(f, p.part_rec, p.CN, b, feat16, lane);
                 }
