@@ -217,7 +217,8 @@ int launch_umma(disco_ctx* c, const void* W, const void* H, int d, int R, float*
     auto kern = umma_tail_kernel<DRAFT>;
     static int configured_dev = -1;
     if (configured_dev != c->device) {
-        if (!cuda_ok(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kUmmaSmemBytes),
+        if (!cuda_ok(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                          kUmmaSmemBytes + umma_clf_bytes(DISCO_MAX_CLF_HIDDEN)),
                      "cudaFuncSetAttribute(umma)"))
             return DISCO_ERR_CUDA;
         configured_dev = c->device;
@@ -225,7 +226,7 @@ int launch_umma(disco_ctx* c, const void* W, const void* H, int d, int R, float*
     cudaLaunchConfig_t cfg{};
     cfg.gridDim = dim3((unsigned)(p.MT * p.CN));
     cfg.blockDim = dim3(kUmmaThreads);
-    cfg.dynamicSmemBytes = kUmmaSmemBytes;
+    cfg.dynamicSmemBytes = kUmmaSmemBytes + (draft_final ? umma_clf_bytes(draft_final->clf_H) : 0);
     cfg.stream = st;
     // The draft step's second phase waits for every CTA of the grid: a cooperative launch makes the
     // driver refuse the launch unless all of them can be resident at once.

@@ -225,10 +225,8 @@ __device__ __forceinline__ MergedPartials warp_merge_partials(const float4* recs
                 q[j][0] = q[j][1] = q[j][2] = q[j][3] = make_float4(0.f, 0.f, 0.f, 0.f);  // Z = 0: empty
             }
         }
-        int* cnt = reinterpret_cast<int*>(scratch);
-        float* cand = scratch + 1;
+        float* cand = scratch;                      // 16-byte aligned
         float* res = cand + kMergeCandidates;
-        if (lane == 0) *cnt = 0;
         if (lane < kTopK) res[lane] = DISCO_NEG_INF;
         // statistics and key inside the lane
         SoftmaxState st;
@@ -272,33 +270,53 @@ __device__ __forceinline__ MergedPartials warp_merge_partials(const float4* recs
         }
         const unsigned who = __ballot_sync(kFullMask, rank == kTopK - 1);
         const float theta = __shfl_sync(kFullMask, head, __ffs(who) - 1);
-        __syncwarp();
-        // gather every logit at or above the threshold (lists are descending: stop at the first below)
+        // every logit at or above the threshold goes to the candidate list: count per lane (the lists
+        // are descending), exclusive prefix sum over the lanes, then plain stores
+        int mine = 0;
 #pragma unroll
         for (int j = 0; j < kPerLane; ++j) {
-            if (q[j][0].y > 0.f && q[j][1].x >= theta) {
-                const float lv[kTopK] = {q[j][1].x, q[j][1].y, q[j][1].z, q[j][1].w, q[j][2].x,
-                                         q[j][2].y, q[j][2].z, q[j][2].w, q[j][3].x, q[j][3].y};
+            const float lv[kTopK] = {q[j][1].x, q[j][1].y, q[j][1].z, q[j][1].w, q[j][2].x,
+                                     q[j][2].y, q[j][2].z, q[j][2].w, q[j][3].x, q[j][3].y};
+            const bool live = q[j][0].y > 0.f;
 #pragma unroll
-                for (int k = 0; k < kTopK; ++k) {
-                    if (lv[k] >= theta && lv[k] > DISCO_NEG_INF) {
-                        const int slot = atomicAdd(cnt, 1);
-                        if (slot < kMergeCandidates) cand[slot] = lv[k];
+            for (int k = 0; k < kTopK; ++k) mine += (live && lv[k] >= theta && lv[k] > DISCO_NEG_INF) ? 1 : 0;
+        }
+        int incl = mine;
+#pragma unroll
+        for (int off = 1; off < 32; off <<= 1) {
+            const int o = __shfl_up_sync(kFullMask, incl, off);
+            if (lane >= off) incl += o;
+        }
+        const int n = __shfl_sync(kFullMask, incl, 31);
+        fast = n <= kMergeCandidates;
+        if (fast) {
+            int at = incl - mine;
+            if (mine > 0) {
+#pragma unroll
+                for (int j = 0; j < kPerLane; ++j) {
+                    const float lv[kTopK] = {q[j][1].x, q[j][1].y, q[j][1].z, q[j][1].w, q[j][2].x,
+                                             q[j][2].y, q[j][2].z, q[j][2].w, q[j][3].x, q[j][3].y};
+                    if (q[j][0].y > 0.f && lv[0] >= theta) {
+#pragma unroll
+                        for (int k = 0; k < kTopK; ++k)
+                            if (lv[k] >= theta && lv[k] > DISCO_NEG_INF) cand[at++] = lv[k];
                     }
                 }
             }
-        }
-        __syncwarp();
-        const int n = *cnt;
-        fast = n <= kMergeCandidates;
-        if (fast) {
+            const int n4 = (n + 3) & ~3;
+            if (lane < n4 - n) cand[n + lane] = DISCO_NEG_INF;  // pad to whole float4s
+            __syncwarp();
             // rank the candidates against each other; ranks 0..9 are the result
             for (int idx = lane; idx < n; idx += 32) {
                 const float x = cand[idx];
                 int r = 0;
-                for (int t = 0; t < n; ++t) {
-                    const float y = cand[t];
-                    r += (y > x || (y == x && t < idx)) ? 1 : 0;
+#pragma unroll 2
+                for (int t = 0; t < n4; t += 4) {
+                    const float4 y = *reinterpret_cast<const float4*>(cand + t);
+                    r += (y.x > x || (y.x == x && t < idx)) ? 1 : 0;
+                    r += (y.y > x || (y.y == x && t + 1 < idx)) ? 1 : 0;
+                    r += (y.z > x || (y.z == x && t + 2 < idx)) ? 1 : 0;
+                    r += (y.w > x || (y.w == x && t + 3 < idx)) ? 1 : 0;
                 }
                 if (r < kTopK) res[r] = x;
             }

@@ -35,6 +35,8 @@ constexpr int kUmmaThreads = (2 + kUmmaEpiWarps) * 32;
 constexpr int kUmmaXchBytes = 14 * 1024;  // 64-byte records handed between the warps that share a hidden row
 constexpr int kUmmaSmemBytes =
     kUmmaRingBytes + 1024 /*align*/ + 512 /*barriers*/ + kUmmaXchBytes;
+// the draft step adds the classifier parameters behind the exchange area
+inline int umma_clf_bytes(int clf_H) { return (clf_H * (kNFeat + 2) + 4) * 4; }
 
 struct UmmaParams {
     int V, d, R;
@@ -168,17 +170,16 @@ __device__ __forceinline__ unsigned int load_acquire(const unsigned int* p) {
     return v;
 }
 
-// One warp finishes sequence b from its NP partial records.
+// One warp finishes sequence b from its NP partial records.  clf_s: classifier parameters in shared
+// memory (W1, b1, w2, b2 in this order); fpos and n_drafted were fetched by the caller.
 __device__ __forceinline__ void umma_finish_sequence(const DraftFinalParams& p, const float4* part_rec, int NP, int b,
-                                                     float* feat16, int lane) {
-    if (p.active && !p.active[b]) return;
-    const float fpos = static_cast<float>(p.pos[b]);
-    const int n_drafted = p.n_drafted[b];
+                                                     float fpos, int n_drafted, float* feat16, const float* clf_s,
+                                                     int lane) {
     const MergedPartials mp = warp_merge_partials(part_rec + (size_t)b * NP * 4, NP, feat16 + 16, lane);
-    const SoftmaxState st = mp.st;
+    const int Hc = p.clf_H;
     const DraftOutputs o{p.token, p.conf, p.halt, p.feats, p.final_stats, p.nll_sum};
-    warp_draft_epilogue(st, mp.key, mp.sel, fpos, n_drafted, p.tau, p.sl_max, feat16, p.clf_W1, p.clf_b1,
-                        p.clf_w2, p.clf_b2, p.clf_H, b, o, lane);
+    warp_draft_epilogue(mp.st, mp.key, mp.sel, fpos, n_drafted, p.tau, p.sl_max, feat16, clf_s, clf_s + Hc * kNFeat,
+                        clf_s + Hc * (kNFeat + 1), clf_s + Hc * (kNFeat + 2), Hc, b, o, lane);
 }
 
 // Vocabulary tile t covers rows [t * TR, min(V, (t + 1) * TR)).  The TMA box and the MMA take TRN >= TR
@@ -200,6 +201,7 @@ umma_tail_kernel(const __grid_constant__ CUtensorMap tmap_W, const __grid_consta
     uint64_t* tmem_empty = tmem_full + 2;
     uint32_t* tmem_base_s = reinterpret_cast<uint32_t*>(tmem_empty + 2);
     float4* xch = reinterpret_cast<float4*>(reinterpret_cast<uint8_t*>(full) + 512);
+    float* clf_s = reinterpret_cast<float*>(reinterpret_cast<uint8_t*>(xch) + kUmmaXchBytes);  // draft step only
 
     // the next kernel of the stream may begin its prologue; this one touches what its predecessor may
     // have written (hidden states, scratch) only after griddepcontrol.wait
@@ -314,6 +316,16 @@ umma_tail_kernel(const __grid_constant__ CUtensorMap tmap_W, const __grid_consta
         const int row = m_tile * 128 + tile_row;
         const bool warp_has_rows = (m_tile * 128 + (quad * 32) % p.rows_pad) < p.R;
         const bool valid = row < p.R;
+        if (DRAFT && (int)blockIdx.x < f.B && f.clf_H > 0) {
+            // this CTA will finish at least one sequence: stage the classifier while the first tile loads
+            const int Hc = f.clf_H, t = ew * 32 + lane, nt = kUmmaEpiWarps * 32;
+            for (int i = t; i < Hc * kNFeat; i += nt) clf_s[i] = f.clf_W1[i];
+            for (int i = t; i < Hc; i += nt) {
+                clf_s[Hc * kNFeat + i] = f.clf_b1[i];
+                clf_s[Hc * (kNFeat + 1) + i] = f.clf_w2[i];
+            }
+            if (t == 0) clf_s[Hc * (kNFeat + 2)] = f.clf_b2[0];
+        }
 
         float best_v = DISCO_NEG_INF;
         int best_i = kNoIndex;
@@ -430,6 +442,11 @@ umma_tail_kernel(const __grid_constant__ CUtensorMap tmap_W, const __grid_consta
             if (ew == 0 && lane == 0) atomicAdd(f.ticket, 1u);
             const int first = ew * (int)gridDim.x + (int)blockIdx.x;
             if (first < f.B) {
+                // what the sequence needs besides the records is fetched under the wait
+                int b = first;
+                bool act = !f.active || f.active[b];
+                float fpos = static_cast<float>(f.pos[b]);
+                int nd = f.n_drafted[b];
                 bool ok = true;
                 if (lane == 0) {
                     const long long t0 = clock64();
@@ -440,15 +457,19 @@ umma_tail_kernel(const __grid_constant__ CUtensorMap tmap_W, const __grid_consta
                             ok = false;
                             break;
                         }
-                        __nanosleep(64);
+                        __nanosleep(32);
                     }
                 }
                 ok = __shfl_sync(kFullMask, ok, 0);
                 __threadfence();
-                if (ok) {
-                    float* feat16 = reinterpret_cast<float*>(xch) + ew * kWarpScratchWords;  // the exchange area is free again
-                    for (int b = first; b < f.B; b += kUmmaEpiWarps * (int)gridDim.x)
-                        umma_finish_sequence(f, p.part_rec, p.CN, b, feat16, lane);
+                float* feat16 = reinterpret_cast<float*>(xch) + ew * kWarpScratchWords;  // the exchange area is free again
+                while (ok) {
+                    if (act) umma_finish_sequence(f, p.part_rec, p.CN, b, fpos, nd, feat16, clf_s, lane);
+                    b += kUmmaEpiWarps * (int)gridDim.x;
+                    if (b >= f.B) break;
+                    act = !f.active || f.active[b];
+                    fpos = static_cast<float>(f.pos[b]);
+                    nd = f.n_drafted[b];
                 }
                 // the last finishing warp of the grid puts the counters back to zero for the next call
                 const unsigned int nwarps = (unsigned int)min(f.B, kUmmaEpiWarps * (int)gridDim.x);
