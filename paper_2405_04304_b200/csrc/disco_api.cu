@@ -380,7 +380,7 @@ int disco_create(disco_ctx** out, int V, int d_draft, int d_target, int max_batc
     bool ok = true;
     ok = ok && cudaMalloc(&c->keys, (size_t)max_rows * sizeof(unsigned long long)) == cudaSuccess;
     ok = ok && cudaMalloc(&c->part_rec, slots * 64) == cudaSuccess;
-    ok = ok && cudaMalloc(&c->ticket, 256) == cudaSuccess;
+    ok = ok && cudaMalloc(&c->ticket, 1024) == cudaSuccess;
     ok = ok && cudaMalloc(&c->status, 256) == cudaSuccess;
     ok = ok && cudaMalloc(&c->final_stats, (size_t)max_batch * 2 * sizeof(float)) == cudaSuccess;
     ok = ok && cudaMalloc(&c->stage_hidden, hid) == cudaSuccess;
@@ -388,7 +388,8 @@ int disco_create(disco_ctx** out, int V, int d_draft, int d_target, int max_batc
     ok = ok && cudaMalloc(&c->stage_float, (size_t)max_batch * (1 + kNFeat) * sizeof(float)) == cudaSuccess;
     ok = ok && cudaMalloc(&c->stage_byte, (size_t)max_batch * 2 + 64) == cudaSuccess;
     ok = ok && cudaMemset(c->keys, 0, (size_t)max_rows * sizeof(unsigned long long)) == cudaSuccess;
-    ok = ok && cudaMemset(c->ticket, 0, 256) == cudaSuccess;
+    ok = ok && cudaMemset(c->ticket, 0, 1024) == cudaSuccess;
+    ok = ok && cudaMemset(c->part_rec, 0, slots * 64) == cudaSuccess;  // no record carries a launch stamp yet
     ok = ok && cudaMemset(c->status, 0, 256) == cudaSuccess;
     ok = ok && cudaDeviceSynchronize() == cudaSuccess;
     if (!ok) {
@@ -511,7 +512,7 @@ int draft_step_common(disco_ctx* c, const void* W_D, const void* h_D, int B, con
         f.feats = feats;
         f.final_stats = c->final_stats;
         f.nll_sum = nll_sum;
-        f.ticket = c->ticket + 48;
+        f.epoch = c->ticket + 48;
         rc = launch_umma<true>(c, W_D, h_D, c->d_draft, B, probs, &f, nullptr, st);
         if (rc) return rc;
     } else {

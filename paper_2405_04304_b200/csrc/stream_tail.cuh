@@ -203,24 +203,68 @@ struct MergedPartials {
     float sel;
 };
 
+// Stamped records: a writer stores words 4..15 of a record, then words 0..3 with a release store whose
+// fourth word is the stamp of the current launch; a reader that sees the stamp with an acquire load may
+// read the rest.  No fence, barrier or counter lies between the two sides.
+__device__ __forceinline__ void store_release_v4(float4* p, const float4& v) {
+    asm volatile("st.release.gpu.global.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(p), "f"(v.x), "f"(v.y), "f"(v.z), "f"(v.w)
+                 : "memory");
+}
+__device__ __forceinline__ float4 load_acquire_v4(const float4* p) {
+    float4 v;
+    asm volatile("ld.acquire.gpu.global.v4.f32 {%0, %1, %2, %3}, [%4];"
+                 : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w)
+                 : "l"(p)
+                 : "memory");
+    return v;
+}
+
 // Merge the NP partial records of one sequence (64 bytes each, consecutive) by one warp.
+// stamp != 0: the records are being written by other CTAs of this launch; wait (bounded, status gets
+// DISCO_ERR_TIMEOUT) until each carries the stamp.
 // Up to 160 records take one L2 round trip, five per lane, and the ten largest logits are found by
 // selection instead of a merge tree: the tenth largest of the lanes' largest logits is a lower bound
 // on the tenth largest overall, so only the few logits at or above it are gathered (shared memory) and
 // ranked against each other.  More than 160 records, or more than kMergeCandidates candidates (many
 // equal logits), fall back to pairwise list merges.  scratch: kWarpScratchWords - 16 words of the warp.
-__device__ __forceinline__ MergedPartials warp_merge_partials(const float4* recs, int NP, float* scratch, int lane) {
+__device__ __forceinline__ MergedPartials warp_merge_partials(const float4* recs, int NP, float* scratch, int lane,
+                                                              uint32_t stamp = 0u, int* status = nullptr) {
     constexpr int kPerLane = 5;
     MergedPartials out;
     bool fast = NP <= 32 * kPerLane;
     if (fast) {
         float4 q[kPerLane][4];
+        if (stamp) {
+            bool pend[kPerLane];
+#pragma unroll
+            for (int j = 0; j < kPerLane; ++j) pend[j] = j * 32 + lane < NP;
+            const long long t0 = clock64();
+            int polls = 0;
+            for (;;) {
+                bool any = false;
+#pragma unroll
+                for (int j = 0; j < kPerLane; ++j)
+                    if (pend[j]) q[j][0] = load_acquire_v4(recs + (size_t)(j * 32 + lane) * 4);
+#pragma unroll
+                for (int j = 0; j < kPerLane; ++j) {
+                    pend[j] = pend[j] && __float_as_uint(q[j][0].w) != stamp;
+                    any = any || pend[j];
+                }
+                if (!__any_sync(kFullMask, any)) break;
+                if ((++polls & 63) == 0 && (*reinterpret_cast<volatile int*>(status) == DISCO_ERR_TIMEOUT ||
+                                            clock64() - t0 > kWaitBudgetClocks)) {
+                    record_status(status, DISCO_ERR_TIMEOUT);
+                    break;
+                }
+            }
+        }
 #pragma unroll
         for (int j = 0; j < kPerLane; ++j) {
             const int c = j * 32 + lane;
             if (c < NP) {
                 const float4* src = recs + (size_t)c * 4;
-                q[j][0] = __ldcg(src), q[j][1] = __ldcg(src + 1), q[j][2] = __ldcg(src + 2), q[j][3] = __ldcg(src + 3);
+                if (!stamp) q[j][0] = __ldcg(src);
+                q[j][1] = __ldcg(src + 1), q[j][2] = __ldcg(src + 2), q[j][3] = __ldcg(src + 3);
             } else {
                 q[j][0] = q[j][1] = q[j][2] = q[j][3] = make_float4(0.f, 0.f, 0.f, 0.f);  // Z = 0: empty
             }
@@ -327,6 +371,20 @@ __device__ __forceinline__ MergedPartials warp_merge_partials(const float4* recs
         }
     }
     // general case: pairwise merges of descending lists
+    if (stamp && NP > 32 * kPerLane) {
+        const long long t0 = clock64();
+        int polls = 0;
+        for (int c = lane; c < NP; c += 32) {
+            while (__float_as_uint(load_acquire_v4(recs + (size_t)c * 4).w) != stamp) {
+                if ((++polls & 63) == 0 && (*reinterpret_cast<volatile int*>(status) == DISCO_ERR_TIMEOUT ||
+                                            clock64() - t0 > kWaitBudgetClocks)) {
+                    record_status(status, DISCO_ERR_TIMEOUT);
+                    break;
+                }
+            }
+        }
+        __syncwarp();
+    }
     LaneRecord r;
     r.clear();
 #pragma unroll 1

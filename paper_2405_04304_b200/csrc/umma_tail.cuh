@@ -161,21 +161,16 @@ struct DraftFinalParams {
     float* feats;
     float* final_stats;
     float* nll_sum;
-    unsigned int* ticket;  // [0] CTAs whose records are published, [1] finishing warps that are done
+    unsigned int* epoch;  // [0] launches completed so far (stamp of this launch = that + 1), [1] finishing warps done
 };
-
-__device__ __forceinline__ unsigned int load_acquire(const unsigned int* p) {
-    unsigned int v;
-    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
-    return v;
-}
 
 // One warp finishes sequence b from its NP partial records.  clf_s: classifier parameters in shared
 // memory (W1, b1, w2, b2 in this order); fpos and n_drafted were fetched by the caller.
 __device__ __forceinline__ void umma_finish_sequence(const DraftFinalParams& p, const float4* part_rec, int NP, int b,
-                                                     float fpos, int n_drafted, float* feat16, const float* clf_s,
-                                                     int lane) {
-    const MergedPartials mp = warp_merge_partials(part_rec + (size_t)b * NP * 4, NP, feat16 + 16, lane);
+                                                     bool active, float fpos, int n_drafted, float* feat16,
+                                                     const float* clf_s, uint32_t stamp, int* status, int lane) {
+    const MergedPartials mp = warp_merge_partials(part_rec + (size_t)b * NP * 4, NP, feat16 + 16, lane, stamp, status);
+    if (!active) return;
     const int Hc = p.clf_H;
     const DraftOutputs o{p.token, p.conf, p.halt, p.feats, p.final_stats, p.nll_sum};
     warp_draft_epilogue(mp.st, mp.key, mp.sel, fpos, n_drafted, p.tau, p.sl_max, feat16, clf_s, clf_s + Hc * kNFeat,
@@ -316,6 +311,9 @@ umma_tail_kernel(const __grid_constant__ CUtensorMap tmap_W, const __grid_consta
         const int row = m_tile * 128 + tile_row;
         const bool warp_has_rows = (m_tile * 128 + (quad * 32) % p.rows_pad) < p.R;
         const bool valid = row < p.R;
+        // stamp of this launch (the word is advanced by the last warp of the second phase)
+        uint32_t stamp = 0u;
+        if (DRAFT) stamp = *reinterpret_cast<volatile unsigned int*>(f.epoch) + 1u;
         if (DRAFT && (int)blockIdx.x < f.B && f.clf_H > 0) {
             // this CTA will finish at least one sequence: stage the classifier while the first tile loads
             const int Hc = f.clf_H, t = ew * 32 + lane, nt = kUmmaEpiWarps * 32;
@@ -428,54 +426,40 @@ umma_tail_kernel(const __grid_constant__ CUtensorMap tmap_W, const __grid_consta
                         if (lv[k] > top.t[kTopK - 1]) top.push(lv[k]);
                 }
                 float4* rec = p.part_rec + ((size_t)row * p.CN + nslot) * 4;
-                rec[0] = make_float4(st.m, st.Z, st.S, 0.f);
                 rec[1] = make_float4(top.t[0], top.t[1], top.t[2], top.t[3]);
                 rec[2] = make_float4(top.t[4], top.t[5], top.t[6], top.t[7]);
                 rec[3] = make_float4(top.t[8], top.t[9], __uint_as_float((uint32_t)(key & 0xffffffffull)),
                                      __uint_as_float((uint32_t)(key >> 32)));
+                store_release_v4(rec, make_float4(st.m, st.Z, st.S, __uint_as_float(stamp)));
             }
-            // Second phase inside the same (cooperative) launch: every CTA publishes its records and
-            // counts itself in; the sequences are then shared out, one warp each, over the CTAs, and a
-            // warp starts once all CTAs are counted.  The wait is bounded like every other one.
-            __threadfence();
-            named_barrier_sync(2, kUmmaEpiWarps * 32);
-            if (ew == 0 && lane == 0) atomicAdd(f.ticket, 1u);
+            // Second phase inside the same (cooperative) launch: the sequences are shared out, one warp
+            // each, over the CTAs; a warp reads the records of its sequence as the other CTAs publish
+            // them (stamped records, bounded waits).
+            named_barrier_sync(2, kUmmaEpiWarps * 32);  // the exchange area is free from here on
             const int first = ew * (int)gridDim.x + (int)blockIdx.x;
             if (first < f.B) {
-                // what the sequence needs besides the records is fetched under the wait
                 int b = first;
                 bool act = !f.active || f.active[b];
                 float fpos = static_cast<float>(f.pos[b]);
                 int nd = f.n_drafted[b];
-                bool ok = true;
-                if (lane == 0) {
-                    const long long t0 = clock64();
-                    while (load_acquire(f.ticket) < gridDim.x) {
-                        if (*reinterpret_cast<volatile int*>(p.status) == DISCO_ERR_TIMEOUT ||
-                            clock64() - t0 > kWaitBudgetClocks) {
-                            record_status(p.status, DISCO_ERR_TIMEOUT);
-                            ok = false;
-                            break;
-                        }
-                        __nanosleep(32);
-                    }
-                }
-                ok = __shfl_sync(kFullMask, ok, 0);
-                __threadfence();
                 float* feat16 = reinterpret_cast<float*>(xch) + ew * kWarpScratchWords;  // the exchange area is free again
-                while (ok) {
-                    if (act) umma_finish_sequence(f, p.part_rec, p.CN, b, fpos, nd, feat16, clf_s, lane);
+                for (;;) {
+                    // a masked sequence still waits for its records: the stamp may only advance once
+                    // every CTA has taken part in this launch
+                    umma_finish_sequence(f, p.part_rec, p.CN, b, act, fpos, nd, feat16, clf_s, stamp, p.status, lane);
                     b += kUmmaEpiWarps * (int)gridDim.x;
                     if (b >= f.B) break;
                     act = !f.active || f.active[b];
                     fpos = static_cast<float>(f.pos[b]);
                     nd = f.n_drafted[b];
                 }
-                // the last finishing warp of the grid puts the counters back to zero for the next call
+                // the last finishing warp of the grid advances the stamp for the next launch: by then every
+                // record of this launch has been read
                 const unsigned int nwarps = (unsigned int)min(f.B, kUmmaEpiWarps * (int)gridDim.x);
-                if (lane == 0 && atomicAdd(f.ticket + 1, 1u) == nwarps - 1) {
-                    f.ticket[0] = 0u;
-                    f.ticket[1] = 0u;
+                __syncwarp();
+                if (lane == 0 && atomicAdd(f.epoch + 1, 1u) == nwarps - 1) {
+                    f.epoch[1] = 0u;
+                    f.epoch[0] = stamp == 0xffffffffu ? 0u : stamp;   // the stamp is never zero
                 }
             }
         } else {
