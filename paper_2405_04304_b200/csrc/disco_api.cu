@@ -46,6 +46,7 @@ struct disco_ctx {
     int* status;
     float* final_stats;
     void* part_rec;                // draft step: 64-byte partial records, [sequence][CTA]
+    void* stamped_rec;             // batched draft step: stamped 80-byte records, [sequence][CTA]; written by nothing else
     int part_slots;                // partials per row the buffers can hold
     void* encode_tiled;            // cuTensorMapEncodeTiled, resolved through the runtime
     // device staging for the *_host entry points
@@ -208,7 +209,7 @@ int launch_umma(disco_ctx* c, const void* W, const void* H, int d, int R, float*
     p.stages = std::max(2, std::min(kUmmaMaxStages, kUmmaRingBytes / (p.a_bytes + p.b_bytes)));
     p.status = c->status;
     p.keys = c->keys;
-    p.part_rec = reinterpret_cast<float4*>(c->part_rec);
+    p.part_rec = reinterpret_cast<float4*>(c->stamped_rec);
     p.probs = probs;
     if (DRAFT && (p.CN > c->part_slots || R > c->part_rows)) return DISCO_ERR_WORKSPACE;
     CUtensorMap tmap_W, tmap_H;
@@ -389,7 +390,8 @@ int disco_create(disco_ctx** out, int V, int d_draft, int d_target, int max_batc
     ok = ok && cudaMalloc(&c->stage_byte, (size_t)max_batch * 2 + 64) == cudaSuccess;
     ok = ok && cudaMemset(c->keys, 0, (size_t)max_rows * sizeof(unsigned long long)) == cudaSuccess;
     ok = ok && cudaMemset(c->ticket, 0, 1024) == cudaSuccess;
-    ok = ok && cudaMemset(c->part_rec, 0, slots * 64) == cudaSuccess;  // no record carries a launch stamp yet
+    ok = ok && cudaMalloc(&c->stamped_rec, (size_t)c->part_rows * c->sm_count * 80) == cudaSuccess;
+    ok = ok && cudaMemset(c->stamped_rec, 0, (size_t)c->part_rows * c->sm_count * 80) == cudaSuccess;  // no stamp yet
     ok = ok && cudaMemset(c->status, 0, 256) == cudaSuccess;
     ok = ok && cudaDeviceSynchronize() == cudaSuccess;
     if (!ok) {
@@ -404,6 +406,7 @@ int disco_destroy(disco_ctx* c) {
     if (!c) return DISCO_ERR_INVALID_ARG;
     cudaFree(c->keys);
     cudaFree(c->part_rec);
+    cudaFree(c->stamped_rec);
     cudaFree(c->ticket);
     cudaFree(c->status);
     cudaFree(c->final_stats);

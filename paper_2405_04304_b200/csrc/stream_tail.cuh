@@ -203,25 +203,39 @@ struct MergedPartials {
     float sel;
 };
 
-// Stamped records: a writer stores words 4..15 of a record, then words 0..3 with a release store whose
-// fourth word is the stamp of the current launch; a reader that sees the stamp with an acquire load may
-// read the rest.  No fence, barrier or counter lies between the two sides.
-__device__ __forceinline__ void store_release_v4(float4* p, const float4& v) {
-    asm volatile("st.release.gpu.global.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(p), "f"(v.x), "f"(v.y), "f"(v.z), "f"(v.w)
-                 : "memory");
+// Stamped records (80 bytes): five 16-byte pieces, each three payload words and the stamp of the launch
+// that wrote it: (m, Z, S | l0 l1 l2 | l3 l4 l5 | l6 l7 l8 | l9, key lo, key hi).  A 16-byte piece is
+// written and read as one access, so a reader that finds the current stamp in a piece holds that
+// piece's payload of this launch, whatever the order in which the pieces travel: no fence, barrier or
+// counter lies between writer and reader (a fence at GPU scope costs about 1.5 us here).  The buffer is
+// written by nothing else and starts zeroed; the stamp is never zero.
+constexpr int kStampedPieces = 5;
+__device__ __forceinline__ void store_relaxed_v4(float4* p, float a, float b, float c, float d) {
+    asm volatile("st.relaxed.gpu.global.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(p), "f"(a), "f"(b), "f"(c), "f"(d) : "memory");
 }
-__device__ __forceinline__ float4 load_acquire_v4(const float4* p) {
+__device__ __forceinline__ float4 load_relaxed_v4(const float4* p) {
     float4 v;
-    asm volatile("ld.acquire.gpu.global.v4.f32 {%0, %1, %2, %3}, [%4];"
+    asm volatile("ld.relaxed.gpu.global.v4.f32 {%0, %1, %2, %3}, [%4];"
                  : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w)
                  : "l"(p)
                  : "memory");
     return v;
 }
+__device__ __forceinline__ void store_stamped_record(float4* rec, float m, float Z, float S, const float (&l)[kTopK],
+                                                     unsigned long long key, uint32_t stamp) {
+    const float sf = __uint_as_float(stamp);
+    store_relaxed_v4(rec, m, Z, S, sf);
+    store_relaxed_v4(rec + 1, l[0], l[1], l[2], sf);
+    store_relaxed_v4(rec + 2, l[3], l[4], l[5], sf);
+    store_relaxed_v4(rec + 3, l[6], l[7], l[8], sf);
+    store_relaxed_v4(rec + 4, l[9], __uint_as_float(static_cast<uint32_t>(key & 0xffffffffull)),
+                     __uint_as_float(static_cast<uint32_t>(key >> 32)), sf);
+}
 
-// Merge the NP partial records of one sequence (64 bytes each, consecutive) by one warp.
-// stamp != 0: the records are being written by other CTAs of this launch; wait (bounded, status gets
-// DISCO_ERR_TIMEOUT) until each carries the stamp.
+// Merge the NP partial records of one sequence (consecutive) by one warp.
+// stamp == 0: plain 64-byte records, complete before the call.  stamp != 0: stamped 80-byte records that
+// other CTAs of this launch are still writing; wait (bounded, status gets DISCO_ERR_TIMEOUT) until each
+// carries the stamp.
 // Up to 160 records take one L2 round trip, five per lane, and the ten largest logits are found by
 // selection instead of a merge tree: the tenth largest of the lanes' largest logits is a lower bound
 // on the tenth largest overall, so only the few logits at or above it are gathered (shared memory) and
@@ -237,17 +251,30 @@ __device__ __forceinline__ MergedPartials warp_merge_partials(const float4* recs
         if (stamp) {
             bool pend[kPerLane];
 #pragma unroll
-            for (int j = 0; j < kPerLane; ++j) pend[j] = j * 32 + lane < NP;
+            for (int j = 0; j < kPerLane; ++j) {
+                pend[j] = j * 32 + lane < NP;
+                q[j][0] = q[j][1] = q[j][2] = q[j][3] = make_float4(0.f, 0.f, 0.f, 0.f);  // Z = 0: empty
+            }
             const long long t0 = clock64();
             int polls = 0;
             for (;;) {
                 bool any = false;
 #pragma unroll
-                for (int j = 0; j < kPerLane; ++j)
-                    if (pend[j]) q[j][0] = load_acquire_v4(recs + (size_t)(j * 32 + lane) * 4);
-#pragma unroll
                 for (int j = 0; j < kPerLane; ++j) {
-                    pend[j] = pend[j] && __float_as_uint(q[j][0].w) != stamp;
+                    if (pend[j]) {
+                        const float4* src = recs + (size_t)(j * 32 + lane) * kStampedPieces;
+                        const float4 a = load_relaxed_v4(src), b = load_relaxed_v4(src + 1), c = load_relaxed_v4(src + 2),
+                                     d = load_relaxed_v4(src + 3), e = load_relaxed_v4(src + 4);
+                        if (__float_as_uint(a.w) == stamp && __float_as_uint(b.w) == stamp &&
+                            __float_as_uint(c.w) == stamp && __float_as_uint(d.w) == stamp &&
+                            __float_as_uint(e.w) == stamp) {
+                            pend[j] = false;
+                            q[j][0] = make_float4(a.x, a.y, a.z, 0.f);
+                            q[j][1] = make_float4(b.x, b.y, b.z, c.x);
+                            q[j][2] = make_float4(c.y, c.z, d.x, d.y);
+                            q[j][3] = make_float4(d.z, e.x, e.y, e.z);
+                        }
+                    }
                     any = any || pend[j];
                 }
                 if (!__any_sync(kFullMask, any)) break;
@@ -257,16 +284,16 @@ __device__ __forceinline__ MergedPartials warp_merge_partials(const float4* recs
                     break;
                 }
             }
-        }
+        } else {
 #pragma unroll
-        for (int j = 0; j < kPerLane; ++j) {
-            const int c = j * 32 + lane;
-            if (c < NP) {
-                const float4* src = recs + (size_t)c * 4;
-                if (!stamp) q[j][0] = __ldcg(src);
-                q[j][1] = __ldcg(src + 1), q[j][2] = __ldcg(src + 2), q[j][3] = __ldcg(src + 3);
-            } else {
-                q[j][0] = q[j][1] = q[j][2] = q[j][3] = make_float4(0.f, 0.f, 0.f, 0.f);  // Z = 0: empty
+            for (int j = 0; j < kPerLane; ++j) {
+                const int c = j * 32 + lane;
+                if (c < NP) {
+                    const float4* src = recs + (size_t)c * 4;
+                    q[j][0] = __ldcg(src), q[j][1] = __ldcg(src + 1), q[j][2] = __ldcg(src + 2), q[j][3] = __ldcg(src + 3);
+                } else {
+                    q[j][0] = q[j][1] = q[j][2] = q[j][3] = make_float4(0.f, 0.f, 0.f, 0.f);  // Z = 0: empty
+                }
             }
         }
         float* cand = scratch;                      // 16-byte aligned
@@ -371,29 +398,37 @@ __device__ __forceinline__ MergedPartials warp_merge_partials(const float4* recs
         }
     }
     // general case: pairwise merges of descending lists
-    if (stamp && NP > 32 * kPerLane) {
-        const long long t0 = clock64();
-        int polls = 0;
-        for (int c = lane; c < NP; c += 32) {
-            while (__float_as_uint(load_acquire_v4(recs + (size_t)c * 4).w) != stamp) {
-                if ((++polls & 63) == 0 && (*reinterpret_cast<volatile int*>(status) == DISCO_ERR_TIMEOUT ||
-                                            clock64() - t0 > kWaitBudgetClocks)) {
-                    record_status(status, DISCO_ERR_TIMEOUT);
-                    break;
-                }
-            }
-        }
-        __syncwarp();
-    }
     LaneRecord r;
     r.clear();
+    const long long t0 = clock64();
+    int polls = 0;
 #pragma unroll 1
     for (int c0 = 0; c0 < NP; c0 += 32) {
         const int c = c0 + lane;
         if (c < NP) {
-            const float4* src = recs + (size_t)c * 4;
             LaneRecord o;
-            o.set(__ldcg(src), __ldcg(src + 1), __ldcg(src + 2), __ldcg(src + 3));
+            if (stamp) {
+                const float4* src = recs + (size_t)c * kStampedPieces;
+                for (;;) {
+                    const float4 a = load_relaxed_v4(src), b = load_relaxed_v4(src + 1), c2 = load_relaxed_v4(src + 2),
+                                 d = load_relaxed_v4(src + 3), e = load_relaxed_v4(src + 4);
+                    if (__float_as_uint(a.w) == stamp && __float_as_uint(b.w) == stamp && __float_as_uint(c2.w) == stamp &&
+                        __float_as_uint(d.w) == stamp && __float_as_uint(e.w) == stamp) {
+                        o.set(make_float4(a.x, a.y, a.z, 0.f), make_float4(b.x, b.y, b.z, c2.x),
+                              make_float4(c2.y, c2.z, d.x, d.y), make_float4(d.z, e.x, e.y, e.z));
+                        break;
+                    }
+                    if ((++polls & 63) == 0 && (*reinterpret_cast<volatile int*>(status) == DISCO_ERR_TIMEOUT ||
+                                                clock64() - t0 > kWaitBudgetClocks)) {
+                        record_status(status, DISCO_ERR_TIMEOUT);
+                        o.clear();
+                        break;
+                    }
+                }
+            } else {
+                const float4* src = recs + (size_t)c * 4;
+                o.set(__ldcg(src), __ldcg(src + 1), __ldcg(src + 2), __ldcg(src + 3));
+            }
             r.absorb(o);
         }
     }

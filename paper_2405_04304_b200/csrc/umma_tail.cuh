@@ -56,7 +56,7 @@ struct UmmaParams {
     // verification
     unsigned long long* keys;  // [R]
     // draft step
-    float4* part_rec;   // [R][CN] records of 64 bytes: (m, Z, S, -), top-10 logits descending, arg-max key
+    float4* part_rec;   // [R][CN] stamped records of 80 bytes
     float* probs;       // optional [R][V]: raw logits are written here
     // verification finished inside this kernel by the last CTA (few sequences only)
     int fuse_final;
@@ -169,7 +169,8 @@ struct DraftFinalParams {
 __device__ __forceinline__ void umma_finish_sequence(const DraftFinalParams& p, const float4* part_rec, int NP, int b,
                                                      bool active, float fpos, int n_drafted, float* feat16,
                                                      const float* clf_s, uint32_t stamp, int* status, int lane) {
-    const MergedPartials mp = warp_merge_partials(part_rec + (size_t)b * NP * 4, NP, feat16 + 16, lane, stamp, status);
+    const MergedPartials mp =
+        warp_merge_partials(part_rec + (size_t)b * NP * kStampedPieces, NP, feat16 + 16, lane, stamp, status);
     if (!active) return;
     const int Hc = p.clf_H;
     const DraftOutputs o{p.token, p.conf, p.halt, p.feats, p.final_stats, p.nll_sum};
@@ -425,12 +426,8 @@ umma_tail_kernel(const __grid_constant__ CUtensorMap tmap_W, const __grid_consta
                     for (int k = 0; k < kTopK; ++k)
                         if (lv[k] > top.t[kTopK - 1]) top.push(lv[k]);
                 }
-                float4* rec = p.part_rec + ((size_t)row * p.CN + nslot) * 4;
-                rec[1] = make_float4(top.t[0], top.t[1], top.t[2], top.t[3]);
-                rec[2] = make_float4(top.t[4], top.t[5], top.t[6], top.t[7]);
-                rec[3] = make_float4(top.t[8], top.t[9], __uint_as_float((uint32_t)(key & 0xffffffffull)),
-                                     __uint_as_float((uint32_t)(key >> 32)));
-                store_release_v4(rec, make_float4(st.m, st.Z, st.S, __uint_as_float(stamp)));
+                store_stamped_record(p.part_rec + ((size_t)row * p.CN + nslot) * kStampedPieces, st.m, st.Z, st.S, top.t,
+                                     key, stamp);
             }
             // Second phase inside the same (cooperative) launch: the sequences are shared out, one warp
             // each, over the CTAs; a warp reads the records of its sequence as the other CTAs publish
