@@ -67,9 +67,10 @@ struct TailParams {
 
 constexpr int kRecordWords = 16;  // one partial record: m, Z, S, -, 10 logits, key (2 words)
 // Shared scratch owned by one warp in the second phase: 16 words for the features of Eq. 2, then the
-// candidate list of warp_merge_partials (counter, 64 candidates, 10 results).
-constexpr int kWarpScratchWords = 112;
+// work area of warp_merge_partials (a pool of whole records, the candidate list, the ten results).
+constexpr int kMergePoolRecords = 16;
 constexpr int kMergeCandidates = 64;
+constexpr int kWarpScratchWords = 16 + kMergePoolRecords * 12 + kMergeCandidates + 16;
 
 inline size_t stream_tail_smem_bytes(int RT, int NW, int d, int stages, uint32_t slot_bytes, int clf_H) {
     size_t b = (size_t)stages * slot_bytes;           // ring
@@ -238,9 +239,11 @@ __device__ __forceinline__ void store_stamped_record(float4* rec, float m, float
 // carries the stamp.
 // Up to 160 records take one L2 round trip, five per lane, and the ten largest logits are found by
 // selection instead of a merge tree: the tenth largest of the lanes' largest logits is a lower bound
-// on the tenth largest overall, so only the few logits at or above it are gathered (shared memory) and
-// ranked against each other.  More than 160 records, or more than kMergeCandidates candidates (many
-// equal logits), fall back to pairwise list merges.  scratch: kWarpScratchWords - 16 words of the warp.
+// on the tenth largest overall; the few records whose head reaches it are copied whole to a pool in
+// shared memory, the pool's values at or above the bound become candidates, and the candidates are
+// ranked against each other.  More than 160 records, more than kMergePoolRecords such records or more
+// than kMergeCandidates candidates (many equal logits) fall back to pairwise list merges.
+// scratch: kWarpScratchWords - 16 words owned by the warp, 16-byte aligned.
 __device__ __forceinline__ MergedPartials warp_merge_partials(const float4* recs, int NP, float* scratch, int lane,
                                                               uint32_t stamp = 0u, int* status = nullptr) {
     constexpr int kPerLane = 5;
@@ -258,21 +261,29 @@ __device__ __forceinline__ MergedPartials warp_merge_partials(const float4* recs
             const long long t0 = clock64();
             int polls = 0;
             for (;;) {
-                bool any = false;
+                // all pieces of all pending records are requested before any is looked at: one L2 round trip
+                float4 raw[kPerLane][kStampedPieces];
 #pragma unroll
                 for (int j = 0; j < kPerLane; ++j) {
                     if (pend[j]) {
                         const float4* src = recs + (size_t)(j * 32 + lane) * kStampedPieces;
-                        const float4 a = load_relaxed_v4(src), b = load_relaxed_v4(src + 1), c = load_relaxed_v4(src + 2),
-                                     d = load_relaxed_v4(src + 3), e = load_relaxed_v4(src + 4);
-                        if (__float_as_uint(a.w) == stamp && __float_as_uint(b.w) == stamp &&
-                            __float_as_uint(c.w) == stamp && __float_as_uint(d.w) == stamp &&
-                            __float_as_uint(e.w) == stamp) {
+#pragma unroll
+                        for (int i = 0; i < kStampedPieces; ++i) raw[j][i] = load_relaxed_v4(src + i);
+                    }
+                }
+                bool any = false;
+#pragma unroll
+                for (int j = 0; j < kPerLane; ++j) {
+                    if (pend[j]) {
+                        bool good = true;
+#pragma unroll
+                        for (int i = 0; i < kStampedPieces; ++i) good = good && __float_as_uint(raw[j][i].w) == stamp;
+                        if (good) {
                             pend[j] = false;
-                            q[j][0] = make_float4(a.x, a.y, a.z, 0.f);
-                            q[j][1] = make_float4(b.x, b.y, b.z, c.x);
-                            q[j][2] = make_float4(c.y, c.z, d.x, d.y);
-                            q[j][3] = make_float4(d.z, e.x, e.y, e.z);
+                            q[j][0] = make_float4(raw[j][0].x, raw[j][0].y, raw[j][0].z, 0.f);
+                            q[j][1] = make_float4(raw[j][1].x, raw[j][1].y, raw[j][1].z, raw[j][2].x);
+                            q[j][2] = make_float4(raw[j][2].y, raw[j][2].z, raw[j][3].x, raw[j][3].y);
+                            q[j][3] = make_float4(raw[j][3].z, raw[j][4].x, raw[j][4].y, raw[j][4].z);
                         }
                     }
                     any = any || pend[j];
@@ -296,31 +307,33 @@ __device__ __forceinline__ MergedPartials warp_merge_partials(const float4* recs
                 }
             }
         }
-        float* cand = scratch;                      // 16-byte aligned
-        float* res = cand + kMergeCandidates;
+        float4* pool = reinterpret_cast<float4*>(scratch);                  // kMergePoolRecords x 3 float4
+        float* cand = scratch + kMergePoolRecords * 12;                     // kMergeCandidates
+        float* res = cand + kMergeCandidates;                               // kTopK
         if (lane < kTopK) res[lane] = DISCO_NEG_INF;
-        // statistics and key inside the lane
-        SoftmaxState st;
-        st.init();
+        // reference maximum, key and largest logit of the lane's records
+        float lm = DISCO_NEG_INF, head = DISCO_NEG_INF;
         unsigned long long key = 0ull;
-        float head = DISCO_NEG_INF;  // largest logit of this lane's records
 #pragma unroll
         for (int j = 0; j < kPerLane; ++j) {
-            st.merge(q[j][0].x, q[j][0].y, q[j][0].z);
             if (q[j][0].y > 0.f) {
+                lm = fmaxf(lm, q[j][0].x);
+                head = fmaxf(head, q[j][1].x);
                 const unsigned long long k2 = key_from_words(q[j][3].z, q[j][3].w);
                 key = k2 > key ? k2 : key;
-                head = fmaxf(head, q[j][1].x);
             }
         }
-        // across the lanes: one max-reduction for the reference maximum, one exponential, shuffle sums
-        const float M = from_ordered_bits(__reduce_max_sync(kFullMask, ordered_bits(st.m)));
+        // statistics: one max-reduction, the exponentials of all records side by side, shuffle sums
+        const float M = from_ordered_bits(__reduce_max_sync(kFullMask, ordered_bits(lm)));
         float Zc = 0.f, Sc = 0.f;
-        if (st.Z > 0.f) {
-            const float dm = st.m - M;
-            const float e = __expf(dm);
-            Zc = st.Z * e;
-            Sc = e * (st.S + dm * st.Z);
+#pragma unroll
+        for (int j = 0; j < kPerLane; ++j) {
+            if (q[j][0].y > 0.f) {
+                const float dm = q[j][0].x - M;
+                const float e = __expf(dm);
+                Zc = fmaf(q[j][0].y, e, Zc);
+                Sc = fmaf(e, fmaf(dm, q[j][0].y, q[j][0].z), Sc);
+            }
         }
 #pragma unroll
         for (int off = 16; off > 0; off >>= 1) {
@@ -332,7 +345,7 @@ __device__ __forceinline__ MergedPartials warp_merge_partials(const float4* recs
             kFullMask, static_cast<uint32_t>(key >> 32) == khi ? static_cast<uint32_t>(key & 0xffffffffull) : 0u);
         out.st.m = M, out.st.Z = Zc, out.st.S = Sc;
         out.key = (static_cast<unsigned long long>(khi) << 32) | klo;
-        // threshold: the lane whose head has rank 9 among the 32 heads (ties broken by lane)
+        // threshold: the head of rank 9 among the 32 lanes' heads (ties broken by lane)
         int rank = 0;
 #pragma unroll
         for (int s2 = 0; s2 < 32; ++s2) {
@@ -341,39 +354,39 @@ __device__ __forceinline__ MergedPartials warp_merge_partials(const float4* recs
         }
         const unsigned who = __ballot_sync(kFullMask, rank == kTopK - 1);
         const float theta = __shfl_sync(kFullMask, head, __ffs(who) - 1);
-        // every logit at or above the threshold goes to the candidate list: count per lane (the lists
-        // are descending), exclusive prefix sum over the lanes, then plain stores
-        int mine = 0;
+        // records whose largest logit reaches the threshold go to the pool, whole
+        const unsigned lt = (1u << lane) - 1u;
+        int nrec = 0;
 #pragma unroll
         for (int j = 0; j < kPerLane; ++j) {
-            const float lv[kTopK] = {q[j][1].x, q[j][1].y, q[j][1].z, q[j][1].w, q[j][2].x,
-                                     q[j][2].y, q[j][2].z, q[j][2].w, q[j][3].x, q[j][3].y};
-            const bool live = q[j][0].y > 0.f;
-#pragma unroll
-            for (int k = 0; k < kTopK; ++k) mine += (live && lv[k] >= theta && lv[k] > DISCO_NEG_INF) ? 1 : 0;
-        }
-        int incl = mine;
-#pragma unroll
-        for (int off = 1; off < 32; off <<= 1) {
-            const int o = __shfl_up_sync(kFullMask, incl, off);
-            if (lane >= off) incl += o;
-        }
-        const int n = __shfl_sync(kFullMask, incl, 31);
-        fast = n <= kMergeCandidates;
-        if (fast) {
-            int at = incl - mine;
-            if (mine > 0) {
-#pragma unroll
-                for (int j = 0; j < kPerLane; ++j) {
-                    const float lv[kTopK] = {q[j][1].x, q[j][1].y, q[j][1].z, q[j][1].w, q[j][2].x,
-                                             q[j][2].y, q[j][2].z, q[j][2].w, q[j][3].x, q[j][3].y};
-                    if (q[j][0].y > 0.f && lv[0] >= theta) {
-#pragma unroll
-                        for (int k = 0; k < kTopK; ++k)
-                            if (lv[k] >= theta && lv[k] > DISCO_NEG_INF) cand[at++] = lv[k];
-                    }
-                }
+            const bool qual = q[j][0].y > 0.f && q[j][1].x >= theta && q[j][1].x > DISCO_NEG_INF;
+            const unsigned mask = __ballot_sync(kFullMask, qual);
+            const int slot = nrec + __popc(mask & lt);
+            if (qual && slot < kMergePoolRecords) {
+                pool[slot * 3] = q[j][1];
+                pool[slot * 3 + 1] = q[j][2];
+                pool[slot * 3 + 2] = make_float4(q[j][3].x, q[j][3].y, DISCO_NEG_INF, DISCO_NEG_INF);
             }
+            nrec += __popc(mask);
+        }
+        fast = nrec <= kMergePoolRecords;
+        int n = 0;
+        if (fast) {
+            __syncwarp();
+            // pool values at or above the threshold become candidates (the pool's padding is -inf)
+            const float* pv = reinterpret_cast<const float*>(pool);
+            for (int i0 = 0; i0 < nrec * 12; i0 += 32) {
+                const int i = i0 + lane;
+                const float v = i < nrec * 12 ? pv[i] : DISCO_NEG_INF;
+                const bool qual = v >= theta && v > DISCO_NEG_INF;
+                const unsigned mask = __ballot_sync(kFullMask, qual);
+                const int slot = n + __popc(mask & lt);
+                if (qual && slot < kMergeCandidates) cand[slot] = v;
+                n += __popc(mask);
+            }
+            fast = n <= kMergeCandidates;
+        }
+        if (fast) {
             const int n4 = (n + 3) & ~3;
             if (lane < n4 - n) cand[n + lane] = DISCO_NEG_INF;  // pad to whole float4s
             __syncwarp();
@@ -381,7 +394,6 @@ __device__ __forceinline__ MergedPartials warp_merge_partials(const float4* recs
             for (int idx = lane; idx < n; idx += 32) {
                 const float x = cand[idx];
                 int r = 0;
-#pragma unroll 2
                 for (int t = 0; t < n4; t += 4) {
                     const float4 y = *reinterpret_cast<const float4*>(cand + t);
                     r += (y.x > x || (y.x == x && t < idx)) ? 1 : 0;
@@ -396,6 +408,7 @@ __device__ __forceinline__ MergedPartials warp_merge_partials(const float4* recs
             __syncwarp();
             return out;
         }
+        __syncwarp();
     }
     // general case: pairwise merges of descending lists
     LaneRecord r;
