@@ -261,32 +261,41 @@ __device__ __forceinline__ MergedPartials warp_merge_partials(const float4* recs
             const long long t0 = clock64();
             int polls = 0;
             for (;;) {
-                // all pieces of all pending records are requested before any is looked at: one L2 round trip
-                float4 raw[kPerLane][kStampedPieces];
-#pragma unroll
-                for (int j = 0; j < kPerLane; ++j) {
-                    if (pend[j]) {
-                        const float4* src = recs + (size_t)(j * 32 + lane) * kStampedPieces;
-#pragma unroll
-                        for (int i = 0; i < kStampedPieces; ++i) raw[j][i] = load_relaxed_v4(src + i);
-                    }
-                }
+                // the pieces of up to three pending records are requested before any is looked at (more in
+                // flight would not fit the registers): two L2 round trips per poll of the lane's five records
                 bool any = false;
 #pragma unroll
-                for (int j = 0; j < kPerLane; ++j) {
-                    if (pend[j]) {
-                        bool good = true;
+                for (int j0 = 0; j0 < kPerLane; j0 += 3) {
+                    float4 raw[3][kStampedPieces];
 #pragma unroll
-                        for (int i = 0; i < kStampedPieces; ++i) good = good && __float_as_uint(raw[j][i].w) == stamp;
-                        if (good) {
-                            pend[j] = false;
-                            q[j][0] = make_float4(raw[j][0].x, raw[j][0].y, raw[j][0].z, 0.f);
-                            q[j][1] = make_float4(raw[j][1].x, raw[j][1].y, raw[j][1].z, raw[j][2].x);
-                            q[j][2] = make_float4(raw[j][2].y, raw[j][2].z, raw[j][3].x, raw[j][3].y);
-                            q[j][3] = make_float4(raw[j][3].z, raw[j][4].x, raw[j][4].y, raw[j][4].z);
+                    for (int jj = 0; jj < 3; ++jj) {
+                        const int j = j0 + jj;
+                        if (j < kPerLane && pend[j]) {
+                            const float4* src = recs + (size_t)(j * 32 + lane) * kStampedPieces;
+#pragma unroll
+                            for (int i = 0; i < kStampedPieces; ++i) raw[jj][i] = load_relaxed_v4(src + i);
                         }
                     }
-                    any = any || pend[j];
+#pragma unroll
+                    for (int jj = 0; jj < 3; ++jj) {
+                        const int j = j0 + jj;
+                        if (j < kPerLane) {
+                            if (pend[j]) {
+                                bool good = true;
+#pragma unroll
+                                for (int i = 0; i < kStampedPieces; ++i)
+                                    good = good && __float_as_uint(raw[jj][i].w) == stamp;
+                                if (good) {
+                                    pend[j] = false;
+                                    q[j][0] = make_float4(raw[jj][0].x, raw[jj][0].y, raw[jj][0].z, 0.f);
+                                    q[j][1] = make_float4(raw[jj][1].x, raw[jj][1].y, raw[jj][1].z, raw[jj][2].x);
+                                    q[j][2] = make_float4(raw[jj][2].y, raw[jj][2].z, raw[jj][3].x, raw[jj][3].y);
+                                    q[j][3] = make_float4(raw[jj][3].z, raw[jj][4].x, raw[jj][4].y, raw[jj][4].z);
+                                }
+                            }
+                            any = any || pend[j];
+                        }
+                    }
                 }
                 if (!__any_sync(kFullMask, any)) break;
                 if ((++polls & 63) == 0 && (*reinterpret_cast<volatile int*>(status) == DISCO_ERR_TIMEOUT ||
