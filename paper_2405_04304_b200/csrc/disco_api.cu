@@ -191,7 +191,7 @@ int launch_umma(disco_ctx* c, const void* W, const void* H, int d, int R, float*
     // Vocabulary rows per tile: up to 256 for verification (its epilogue is a compare per logit); the
     // draft step's epilogue is heavy (soft-max, top-10), so it gets several small tiles per CTA and
     // the epilogue of one tile runs under the loads of the next.
-    const int tile_target = DRAFT ? (getenv_int("DISCO_DRAFT_TILE", 64)) : 256;
+    const int tile_target = DRAFT ? getenv_int("DISCO_DRAFT_TILE", R <= 128 ? 128 : 256) : 256;
     p.TPC = std::max(1, (c->V + tile_target * p.CN - 1) / (tile_target * p.CN));
     p.TR = (c->V + p.CN * p.TPC - 1) / (p.CN * p.TPC);
     p.TRN = std::max(16, (p.TR + 15) / 16 * 16);
