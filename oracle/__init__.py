@@ -268,3 +268,109 @@ def verify(W_T, H_T, draft_ids, B: int, SL: int, nthreads: int = 1) -> VerifyRes
         _p(n, ctypes.c_int32), _p(bonus, ctypes.c_int32), _p(tid, ctypes.c_int32),
         _p(gap, ctypes.c_double), nthreads), "verify")
     return VerifyResult(n, bonus, tid, gap)
+
+
+# --------------------------------------------------------------------------- sampling at temperature 1
+def sample_cdf(w, u: float):
+    """Inverse-CDF draw from non-negative weights.  Returns (token, total weight)."""
+    w = np.ascontiguousarray(w, dtype=np.float64)
+    tok = ctypes.c_int32(-2)
+    total = ctypes.c_double(0.0)
+    _check(lib().oracle_sample_cdf(_p(w, ctypes.c_double), w.shape[0], ctypes.c_double(u), ctypes.byref(tok),
+                                   ctypes.byref(total)), "sample_cdf")
+    return int(tok.value), float(total.value)
+
+
+@dataclass
+class DraftSampleResult:
+    token: np.ndarray      # [B] int32, drawn from y^D
+    p_token: np.ndarray    # [B] float64, y^D(token)
+    conf: np.ndarray       # [B] float64
+    halt: np.ndarray       # [B] uint8
+    feats: np.ndarray      # [B, k+2] float64
+    probs: np.ndarray      # [B, V] float64
+
+
+def draft_step_sample(W_D, h_D, pos, n_drafted, clf: Classifier, tau: float, sl_max: int, u,
+                      active=None, k: int = K_TOP, nthreads: int = 1) -> DraftSampleResult:
+    W_D, h_D = _u16(W_D), _u16(h_D)
+    V, d = W_D.shape
+    B = h_D.shape[0]
+    pos = np.ascontiguousarray(pos, dtype=np.int32)
+    n_drafted = np.ascontiguousarray(n_drafted, dtype=np.int32)
+    u = np.ascontiguousarray(u, dtype=np.float64)
+    assert u.shape[0] == B
+    act = None if active is None else np.ascontiguousarray(active, dtype=np.uint8)
+    token = np.full(B, -1, dtype=np.int32)
+    p_token = np.full(B, np.nan)
+    conf = np.full(B, np.nan)
+    halt = np.full(B, 255, dtype=np.uint8)
+    feats = np.full((B, k + 2), np.nan)
+    probs = np.full((B, V), np.nan)
+    ctypes_f = ctypes.c_float
+    fn = lib().oracle_draft_step_sample
+    fn.restype = ctypes.c_int
+    _check(fn(
+        _p(W_D, ctypes.c_uint16), _p(h_D, ctypes.c_uint16), V, d, B,
+        _p(pos, ctypes.c_int32), _p(n_drafted, ctypes.c_int32), _p(act, ctypes.c_uint8),
+        _p(clf.W1, ctypes_f), _p(clf.b1, ctypes_f), _p(clf.w2, ctypes_f), _p(clf.b2, ctypes_f), clf.H, k,
+        ctypes_f(tau), int(sl_max), _p(u, ctypes.c_double),
+        _p(token, ctypes.c_int32), _p(p_token, ctypes.c_double), _p(conf, ctypes.c_double),
+        _p(halt, ctypes.c_uint8), _p(feats, ctypes.c_double), _p(probs, ctypes.c_double), nthreads),
+        "draft_step_sample")
+    return DraftSampleResult(token, p_token, conf, halt, feats, probs)
+
+
+def speculative_sample(yT, yD, tokens, ua, us: float):
+    """One sequence of speculative sampling on given distributions.  yT [(SL+1), V], yD [SL, V].
+    Returns (n_accept, next_token)."""
+    yT = np.ascontiguousarray(yT, dtype=np.float64)
+    SL = yT.shape[0] - 1
+    V = yT.shape[1]
+    yD = np.ascontiguousarray(yD, dtype=np.float64).reshape(SL, V)
+    tokens = np.ascontiguousarray(tokens, dtype=np.int32)
+    ua = np.ascontiguousarray(ua, dtype=np.float64)
+    assert tokens.shape[0] == SL and ua.shape[0] == SL
+    n = ctypes.c_int32(-1)
+    nxt = ctypes.c_int32(-1)
+    _check(lib().oracle_speculative_sample(
+        _p(yT, ctypes.c_double), _p(yD, ctypes.c_double) if SL else None,
+        _p(tokens, ctypes.c_int32) if SL else None, SL, V, _p(ua, ctypes.c_double) if SL else None,
+        ctypes.c_double(us), ctypes.byref(n), ctypes.byref(nxt)), "speculative_sample")
+    return int(n.value), int(nxt.value)
+
+
+@dataclass
+class VerifySampleResult:
+    n_accept: np.ndarray    # [B] int32
+    next_token: np.ndarray  # [B] int32
+    y_T: np.ndarray         # [R, V] float64 target distributions
+
+
+def verify_sample(W_T, H_T, draft_ids, draft_probs, row_off, ua, us, nthreads: int = 1) -> VerifySampleResult:
+    """Stochastic verification.  draft_probs: float32 [steps, B, V] (step-major); ua packed like draft_ids; us [B]."""
+    W_T, H_T = _u16(W_T), _u16(H_T)
+    V, d = W_T.shape
+    row_off = np.ascontiguousarray(row_off, dtype=np.int32)
+    B = row_off.shape[0] - 1
+    R = int(row_off[-1])
+    assert H_T.shape[0] == R
+    draft_ids = np.ascontiguousarray(draft_ids, dtype=np.int32)
+    assert draft_ids.shape[0] == R - B
+    ua = np.ascontiguousarray(ua, dtype=np.float64)
+    us = np.ascontiguousarray(us, dtype=np.float64)
+    assert ua.shape[0] == R - B and us.shape[0] == B
+    dp = np.ascontiguousarray(draft_probs, dtype=np.float32)
+    if R - B:
+        max_sl = int(np.max(np.diff(row_off))) - 1
+        assert dp.shape[0] >= max_sl and dp.shape[1] == B and dp.shape[2] == V
+    n = np.full(B, -1, dtype=np.int32)
+    nxt = np.full(B, -1, dtype=np.int32)
+    yT = np.full((R, V), np.nan)
+    _check(lib().oracle_verify_sample(
+        _p(W_T, ctypes.c_uint16), _p(H_T, ctypes.c_uint16), V, d,
+        _p(draft_ids, ctypes.c_int32) if draft_ids.size else None,
+        _p(dp, ctypes.c_float) if draft_ids.size else None, _p(row_off, ctypes.c_int32), B,
+        _p(ua, ctypes.c_double) if ua.size else None, _p(us, ctypes.c_double),
+        _p(n, ctypes.c_int32), _p(nxt, ctypes.c_int32), _p(yT, ctypes.c_double), nthreads), "verify_sample")
+    return VerifySampleResult(n, nxt, yT)

@@ -287,6 +287,147 @@ int oracle_verify(const uint16_t* W_T, const uint16_t* H_T, int V, int d,
                                 target_ids, gap, nthreads);
 }
 
+// ---------------------------------------------------------------------------
+// Sampling at temperature 1 (the paper's second evaluated mode, Table 6;
+// speculative sampling of Leviathan et al., which Sec. 3 names as the
+// verification scheme).  Random numbers are inputs: the caller passes uniforms.
+// ---------------------------------------------------------------------------
+
+// Inverse-CDF draw from non-negative weights w[V] with a uniform u in [0, 1):
+// the smallest v whose running sum w_0 + .. + w_v exceeds u * (w_0 + .. + w_{V-1}).
+// Rounding can leave no such v for u next to 1: then the last v with w_v > 0.
+// total (optional) receives the sum.  All weights zero: *token = -1.
+int oracle_sample_cdf(const double* w, int V, double u, int32_t* token, double* total) {
+    if (!w || !token || V <= 0) return ORACLE_BAD_ARG;
+    double sum = 0.0;
+    for (int v = 0; v < V; ++v) sum += w[v];
+    if (total) *total = sum;
+    const double target = u * sum;
+    double run = 0.0;
+    int last = -1;
+    for (int v = 0; v < V; ++v) {
+        run += w[v];
+        if (w[v] > 0.0) last = v;
+        if (run > target) {
+            *token = v;
+            return ORACLE_OK;
+        }
+    }
+    *token = last;
+    return ORACLE_OK;
+}
+
+// Draft step with a sampled token: as oracle_draft_step, except that the token
+// is drawn from y^D = softmax(W_D h) with u[b] instead of being the arg-max.
+// Features, classifier and stopping rule are unchanged (they look at y^D, not
+// at the token).  p_token[b] = y^D(token); probs[B,V] = y^D (needed later by the
+// verification's residual distribution).
+int oracle_draft_step_sample(const uint16_t* W_D, const uint16_t* h_D, int V, int d, int B,
+                             const int32_t* pos, const int32_t* n_drafted, const uint8_t* active,
+                             const float* W1, const float* b1, const float* w2, const float* b2, int H,
+                             int k, float tau, int sl_max, const double* u,
+                             int32_t* token, double* p_token, double* conf, uint8_t* halt, double* feats,
+                             double* probs, int nthreads) {
+    if (!W_D || !h_D || !pos || !n_drafted || !token || !u || V <= 0 || d <= 0 || B < 0 || k <= 0)
+        return ORACLE_BAD_ARG;
+    std::vector<double> z(V), y(V), x(k + 2);
+    for (int b = 0; b < B; ++b) {
+        if (active && !active[b]) continue;
+        int rc = oracle_project(W_D, h_D + (size_t)b * d, V, d, 1, z.data(), nthreads);
+        if (rc) return rc;
+        rc = oracle_softmax(z.data(), V, y.data());
+        if (rc) return rc;
+        rc = oracle_sample_cdf(y.data(), V, u[b], &token[b], nullptr);
+        if (rc) return rc;
+        if (p_token) p_token[b] = y[token[b]];
+        rc = oracle_features(y.data(), V, k, pos[b], x.data());
+        if (rc) return rc;
+        double C = 0.0;
+        rc = oracle_classifier(x.data(), k + 2, W1, b1, w2, b2, H, &C);
+        if (rc) return rc;
+        if (conf) conf[b] = C;
+        if (halt) halt[b] = (static_cast<float>(C) < tau) || (n_drafted[b] >= sl_max) ? 1 : 0;
+        if (feats) std::copy(x.begin(), x.end(), feats + (size_t)b * (k + 2));
+        if (probs) std::copy(y.begin(), y.end(), probs + (size_t)b * V);
+    }
+    return ORACLE_OK;
+}
+
+// One sequence of speculative sampling, given the distributions themselves:
+// yT[(SL+1), V] target rows, yD[SL, V] draft rows, draft tokens t[SL], uniforms
+// ua[SL] (one per draft token) and us (one for the token that ends the
+// iteration).  Draft token i is accepted iff ua_i * yD_i(t_i) < yT_i(t_i), i.e.
+// with probability min(1, yT_i(t_i) / yD_i(t_i)); n = number accepted before the
+// first rejection.  The next token is drawn with us from
+//     norm(max(0, yT_n - yD_n))   if n < SL (a rejection at position n),
+//     yT_SL                       if every draft token was accepted;
+// a residual that is zero everywhere (yT_n == yD_n, where a rejection cannot
+// happen except through rounding) falls back to yT_n.
+int oracle_speculative_sample(const double* yT, const double* yD, const int32_t* t, int SL, int V,
+                              const double* ua, double us, int32_t* n_accept, int32_t* next_token) {
+    if (!yT || !n_accept || !next_token || SL < 0 || V <= 0) return ORACLE_BAD_ARG;
+    if (SL > 0 && (!yD || !t || !ua)) return ORACLE_BAD_ARG;
+    int n = 0;
+    while (n < SL) {
+        const int tok = t[n];
+        if (tok < 0 || tok >= V) return ORACLE_BAD_ARG;
+        const double pT = yT[(size_t)n * V + tok], pD = yD[(size_t)n * V + tok];
+        if (!(ua[n] * pD < pT)) break;
+        ++n;
+    }
+    *n_accept = n;
+    std::vector<double> w(V);
+    const double* rowT = yT + (size_t)n * V;
+    if (n < SL) {
+        const double* rowD = yD + (size_t)n * V;
+        double mass = 0.0;
+        for (int v = 0; v < V; ++v) {
+            w[v] = std::max(0.0, rowT[v] - rowD[v]);
+            mass += w[v];
+        }
+        if (!(mass > 0.0)) std::copy(rowT, rowT + V, w.begin());
+    } else {
+        std::copy(rowT, rowT + V, w.begin());
+    }
+    return oracle_sample_cdf(w.data(), V, us, next_token, nullptr);
+}
+
+// Verification tail with sampling for B sequences with ragged look-ahead: rows
+// as in oracle_verify_ragged; the target distributions are yT_r = softmax(W_T
+// H_T[r]).  The draft distributions arrive as binary32 (what a draft step
+// hands over) in step-major order: draft_probs[(i * B + b) * V + v] is the
+// distribution from which token i of sequence b was drawn.  ua is packed like
+// draft_ids (one uniform per draft token), us[B] has one uniform per sequence.
+// y_T (optional, [R, V]) receives the target distributions.
+int oracle_verify_sample(const uint16_t* W_T, const uint16_t* H_T, int V, int d,
+                         const int32_t* draft_ids, const float* draft_probs, const int32_t* row_off, int B,
+                         const double* ua, const double* us, int32_t* n_accept, int32_t* next_token,
+                         double* y_T, int nthreads) {
+    if (!W_T || !H_T || !row_off || !us || !n_accept || !next_token || V <= 0 || d <= 0 || B < 0)
+        return ORACLE_BAD_ARG;
+    std::vector<double> z(V);
+    for (int b = 0; b < B; ++b) {
+        const int r0 = row_off[b], r1 = row_off[b + 1];
+        const int SL = r1 - r0 - 1;
+        if (SL < 0) return ORACLE_BAD_ARG;
+        if (SL > 0 && (!draft_ids || !draft_probs || !ua)) return ORACLE_BAD_ARG;
+        std::vector<double> yT((size_t)(SL + 1) * V), yD((size_t)SL * V);
+        for (int r = r0; r < r1; ++r) {
+            int rc = oracle_project(W_T, H_T + (size_t)r * d, V, d, 1, z.data(), nthreads);
+            if (rc) return rc;
+            rc = oracle_softmax(z.data(), V, yT.data() + (size_t)(r - r0) * V);
+            if (rc) return rc;
+        }
+        for (int i = 0; i < SL; ++i)
+            for (int v = 0; v < V; ++v) yD[(size_t)i * V + v] = draft_probs[((size_t)i * B + b) * V + v];
+        if (y_T) std::copy(yT.begin(), yT.end(), y_T + (size_t)r0 * V);
+        int rc = oracle_speculative_sample(yT.data(), yD.data(), draft_ids ? draft_ids + (r0 - b) : nullptr, SL, V,
+                                           ua ? ua + (r0 - b) : nullptr, us[b], &n_accept[b], &next_token[b]);
+        if (rc) return rc;
+    }
+    return ORACLE_OK;
+}
+
 int oracle_hardware_threads() { return (int)std::thread::hardware_concurrency(); }
 
 }  // extern "C"

@@ -413,3 +413,164 @@ def test_ppl_rule_halts_monotonically_in_the_bound_and_skips_inactive(oracle):
     tok, ppl, halt, gap, nll = oracle.draft_step_ppl(bits_of(W), bits_of(h), nd, np.full(3, 0.25), 20.0, 9,
                                                      active=np.array([1, 0, 1], np.uint8))
     assert tok[1] == -1 and halt[1] == 255 and nll[1] == 0.25 and nll[0] > 0.25
+
+
+# ------------------------------------------------------------------ sampling at temperature 1 (Table 6)
+def test_sample_cdf_closed_forms(oracle):
+    # uniform weights: token = floor(u * V), whatever the common scale of the weights
+    V = 8
+    for scale in (1.0, 0.125, 3.0):
+        for u in (0.0, 0.1, 0.124, 0.126, 0.5, 0.874, 0.876, 0.9999):
+            tok, total = oracle.sample_cdf(np.full(V, scale), u)
+            assert tok == int(math.floor(u * V)) and abs(total - V * scale) < 1e-12
+    # boundary convention: the running sum has to EXCEED u * total
+    assert oracle.sample_cdf([0.5, 0.25, 0.25], 0.5)[0] == 1
+    assert oracle.sample_cdf([0.5, 0.25, 0.25], 0.4999)[0] == 0
+    assert oracle.sample_cdf([0.5, 0.25, 0.25], 0.75)[0] == 2
+    # entries of weight zero are never drawn, not even at u = 0 or next to 1
+    assert oracle.sample_cdf([0.0, 1.0, 0.0], 0.0)[0] == 1
+    assert oracle.sample_cdf([0.0, 0.3, 0.0, 0.7, 0.0], 1.0 - 1e-17)[0] == 3
+    assert oracle.sample_cdf([0.0, 0.0], 0.3)[0] == -1
+
+
+def test_speculative_sampling_reproduces_the_target_distribution(oracle):
+    """Brute force over a grid of the three uniforms (draft draw, acceptance, final draw): the token
+    that position 0 ends up with is distributed as the target, which is the property the scheme is
+    built for.  A wrong ratio, a missing clamp or a swapped residual shifts the histogram by far more
+    than the grid's resolution."""
+    yD = np.array([0.70, 0.10, 0.15, 0.05])
+    yT = np.array([0.10, 0.20, 0.30, 0.40])
+    N = 40
+    grid = (np.arange(N) + 0.5) / N
+    hist = np.zeros(4)
+    accepted = 0
+    for ud in grid:
+        t, _ = oracle.sample_cdf(yD, ud)
+        for ua in grid:
+            for us in grid:
+                n, nxt = oracle.speculative_sample(np.stack([yT, yT]), yD[None, :], [t], [ua], us)
+                hist[t if n == 1 else nxt] += 1
+                accepted += n
+    hist /= N ** 3
+    assert np.max(np.abs(hist - yT)) < 2.5 / N
+    # acceptance rate = sum_v min(yD_v, yT_v) = 1 - total variation distance: computed here from the
+    # histogram of accepted events only, not from the formula the oracle uses
+    assert abs(accepted / N ** 3 - (1.0 - 0.5 * np.abs(yD - yT).sum())) < 2.5 / N
+
+
+def test_speculative_identical_distributions_accept_everything(oracle):
+    rng = np.random.default_rng(3)
+    V, SL = 11, 4
+    y = rng.dirichlet(np.ones(V), size=SL + 1)
+    toks = rng.integers(0, V, size=SL)
+    for trial in range(20):
+        ua = rng.random(SL)
+        us = float(rng.random())
+        n, nxt = oracle.speculative_sample(y, y[:SL], toks, ua, us)
+        assert n == SL
+        assert nxt == oracle.sample_cdf(y[SL], us)[0]          # the extra token comes from the last target row
+
+
+def test_speculative_residual_closed_form(oracle):
+    # draft certain of token 0, target splits between 0 and 1: accepted with probability 1/2, and a
+    # rejection can only ever be repaired with token 1
+    yD = np.array([[1.0, 0.0, 0.0]])
+    yT = np.array([[0.5, 0.5, 0.0], [0.2, 0.3, 0.5]])
+    for us in (0.0, 0.3, 0.99):
+        assert oracle.speculative_sample(yT, yD, [0], [0.6], us) == (0, 1)
+        assert oracle.speculative_sample(yT, yD, [0], [0.5], us) == (0, 1)      # u * p_D < p_T is strict
+    assert oracle.speculative_sample(yT, yD, [0], [0.4], 0.1) == (1, 0)         # accepted: next from row 1
+    assert oracle.speculative_sample(yT, yD, [0], [0.4], 0.45) == (1, 1)
+    assert oracle.speculative_sample(yT, yD, [0], [0.4], 0.55) == (1, 2)
+    # a token the target gives no mass is rejected even at u = 0
+    assert oracle.speculative_sample(yT, np.array([[0.0, 0.0, 1.0]]), [2], [0.0], 0.7)[0] == 0
+    # SL = 0: nothing to accept, one draw from the single target row
+    assert oracle.speculative_sample(yT[:1], np.zeros((0, 3)), [], [], 0.7) == (0, 1)
+
+
+def test_verify_sample_with_sharp_distributions_is_greedy_verification(oracle):
+    """As the distributions approach one-hot vectors the sampling scheme becomes the token-equality rule
+    of Sec. 3: same n_accept and the same next token as the greedy oracle, for any uniforms."""
+    rng = np.random.default_rng(9)
+    V, d, B = 60, 48, 3
+    sls = [3, 0, 4]
+    row_off = np.concatenate([[0], np.cumsum([s + 1 for s in sls])]).astype(np.int32)
+    R = int(row_off[-1])
+    Wf = rng.normal(size=(V, d)).astype(np.float32)
+    W = bits_of(torch.from_numpy(Wf))
+    # each hidden row points along the LM-head row of one token: that token's logit towers over the rest
+    H = bits_of(torch.from_numpy(20.0 * Wf[rng.integers(0, V, size=R)]))
+    z = oracle.project(W, H)
+    top = z.argmax(axis=1)
+    srt = np.sort(z, axis=1)
+    assert np.all(srt[:, -1] - srt[:, -2] > 40.0)             # softmax is one-hot to 1e-17
+    ids = []
+    for b in range(B):
+        want = top[row_off[b]: row_off[b + 1] - 1].copy()
+        if len(want) > 1:
+            want[len(want) // 2] = (want[len(want) // 2] + 1) % V   # one mismatch in the middle
+        ids.extend(want.tolist())
+    ids = np.array(ids, dtype=np.int32)
+    dp = np.zeros((max(sls), B, V), dtype=np.float32)
+    for b in range(B):
+        for i in range(sls[b]):
+            dp[i, b, ids[row_off[b] - b + i]] = 1.0
+    greedy = oracle.verify_ragged(W, H, ids, row_off)
+    for trial in range(5):
+        ua = rng.uniform(1e-6, 1 - 1e-6, size=R - B)
+        us = rng.uniform(1e-6, 1 - 1e-6, size=B)
+        res = oracle.verify_sample(W, H, ids, dp, row_off, ua, us)
+        np.testing.assert_array_equal(res.n_accept, greedy.n_accept)
+        np.testing.assert_array_equal(res.next_token, greedy.bonus)
+    np.testing.assert_allclose(res.y_T.sum(axis=1), 1.0, atol=1e-12)
+
+
+def test_verify_sample_is_the_per_sequence_rule_on_softmax_rows(oracle):
+    """The batched call = softmax of the projected rows, step-major draft distributions gathered per
+    sequence, and the one-sequence rule; checked with rows built here from project() and numpy."""
+    rng = np.random.default_rng(21)
+    V, d, B = 23, 8, 3
+    sls = [2, 3, 1]
+    row_off = np.concatenate([[0], np.cumsum([s + 1 for s in sls])]).astype(np.int32)
+    R = int(row_off[-1])
+    W = bits_of(torch.from_numpy(rng.normal(size=(V, d)).astype(np.float32)))
+    H = bits_of(torch.from_numpy(rng.normal(size=(R, d)).astype(np.float32)))
+    z = oracle.project(W, H)
+    e = np.exp(z - z.max(axis=1, keepdims=True))
+    yT = e / e.sum(axis=1, keepdims=True)
+    dp = rng.dirichlet(np.ones(V), size=(max(sls), B)).astype(np.float32)
+    ids = rng.integers(0, V, size=R - B).astype(np.int32)
+    ua, us = rng.random(R - B), rng.random(B)
+    res = oracle.verify_sample(W, H, ids, dp, row_off, ua, us)
+    np.testing.assert_allclose(res.y_T, yT, atol=1e-14)
+    for b in range(B):
+        r0, sl = int(row_off[b]), sls[b]
+        n, nxt = oracle.speculative_sample(yT[r0: r0 + sl + 1], dp[:sl, b].astype(np.float64),
+                                           ids[r0 - b: r0 - b + sl], ua[r0 - b: r0 - b + sl], us[b])
+        assert (res.n_accept[b], res.next_token[b]) == (n, nxt)
+
+
+def test_draft_step_sample_differs_from_greedy_step_only_in_the_token(oracle):
+    rng = np.random.default_rng(4)
+    V, d, B, Hc = 97, 24, 4, 8
+    W = bits_of(torch.from_numpy(rng.normal(size=(V, d)).astype(np.float32)))
+    h = bits_of(torch.from_numpy(rng.normal(size=(B, d)).astype(np.float32)))
+    clf = oracle.Classifier(rng.normal(size=(Hc, 12)).astype(np.float32), rng.normal(size=Hc).astype(np.float32),
+                            rng.normal(size=Hc).astype(np.float32), np.array([0.1], dtype=np.float32))
+    pos, nd = np.arange(B) + 5, np.array([1, 2, 3, 9])
+    u = np.array([0.0, 0.3, 0.77, 0.999])
+    act = np.array([1, 1, 0, 1], dtype=np.uint8)
+    g = oracle.draft_step(W, h, pos, nd, clf, 0.5, 9, active=act, want_probs=True)
+    s = oracle.draft_step_sample(W, h, pos, nd, clf, 0.5, 9, u, active=act)
+    for b in range(B):
+        if not act[b]:
+            assert s.token[b] == -1 and np.isnan(s.p_token[b])
+            continue
+        np.testing.assert_array_equal(s.probs[b], g.probs[b])
+        np.testing.assert_array_equal(s.feats[b], g.feats[b])
+        assert s.conf[b] == g.conf[b] and s.halt[b] == g.halt[b]
+        assert s.token[b] == oracle.sample_cdf(g.probs[b], u[b])[0]
+        assert s.p_token[b] == g.probs[b, s.token[b]]
+        cdf = np.cumsum(g.probs[b])
+        assert cdf[s.token[b]] > u[b] * cdf[-1] - 1e-15 and (s.token[b] == 0 or cdf[s.token[b] - 1] <= u[b] * cdf[-1] + 1e-15)
+    assert s.token[0] == int(np.argmax(g.probs[0] > 0))           # u = 0 draws the first token with mass
