@@ -135,6 +135,53 @@ int disco_draft_step_ppl(disco_ctx* ctx, const void* W_D, const void* h_D, int B
                          void* stream);
 
 /*
+ * Draft step with a sampled token (decoding at temperature 1, the mode of Table 6): everything as in
+ * disco_draft_step, except that the token is drawn from y^D = softmax(W_D h) instead of being its
+ * arg-max.  The draw is by inverse CDF with the caller's uniform:
+ *     token = min { v : y^D_0 + .. + y^D_v > u * sum_w y^D_w }.
+ * Features, classifier and stopping rule do not depend on the token and are unchanged.
+ *   u        float [B], device   uniforms in [0, 1), one per sequence
+ *   p_token  float [B] or NULL   y^D(token)
+ *   probs    float [B, V], device, REQUIRED: receives y^D; the verification needs these rows (hand the
+ *            rows of step i in as draft_probs[i] of disco_verify_sample_ragged)
+ * Other arguments, layouts, ownership and errors as in disco_draft_step.
+ */
+int disco_draft_step_sample(disco_ctx* ctx, const void* W_D, const void* h_D, int B,
+                            const int32_t* pos, const int32_t* n_drafted, const uint8_t* active,
+                            const disco_clf* clf, float tau, int sl_max, const float* u,
+                            int32_t* token, float* p_token, float* conf, uint8_t* halt, float* feats,
+                            float* probs, void* stream);
+
+/*
+ * Verification with sampling (temperature 1; Table 6): the rejection-sampling scheme of Leviathan et al.
+ * that Sec. 3 names, of which disco_verify_ragged is the zero-temperature case.  Rows and row_off as in
+ * disco_verify_ragged.  With y^T_r = softmax(W_T H_T[r]) and y^D_i the distribution draft token t_i was
+ * drawn from, token i of a sequence is accepted iff
+ *     u_accept_i * y^D_i(t_i) < y^T_i(t_i)        (probability min(1, y^T_i(t_i) / y^D_i(t_i))),
+ * n_accept is the number accepted before the first rejection, and next_token is drawn by inverse CDF with
+ * u_sample[b] from norm(max(0, y^T_n - y^D_n)) after a rejection at position n, from y^T_SL if all were
+ * accepted (a residual without mass falls back to y^T_n).
+ *   draft_ids    int32 [R - B], device   packed as in disco_verify_ragged
+ *   draft_probs  float [steps, B, V], device, steps >= max SL_b: draft_probs[i, b, :] = y^D of token i of
+ *                sequence b (the probs output of draft step i); NULL allowed iff R == B
+ *   row_off      int32 [B + 1], device, or NULL for a uniform SL = R / B - 1
+ *   u_accept     float [R - B], device   uniforms in [0, 1), packed like draft_ids
+ *   u_sample     float [B], device       uniforms in [0, 1)
+ * Outputs (device):
+ *   n_accept [B], next_token [B]
+ *   y_T         float [R, V], REQUIRED: receives the target distributions (also the call's work space)
+ *   target_ids  int32 [R] or NULL: arg-max of every target row
+ * Errors as in disco_verify_ragged; a draft id outside [0, V) sets the device status to
+ * DISCO_ERR_INVALID_ARG and ends that sequence's acceptance there.
+ */
+int disco_verify_sample_ragged(disco_ctx* ctx, const void* W_T, const void* H_T,
+                               const int32_t* draft_ids, const float* draft_probs,
+                               const int32_t* row_off, int B, int R,
+                               const float* u_accept, const float* u_sample,
+                               int32_t* n_accept, int32_t* next_token, float* y_T, int32_t* target_ids,
+                               void* stream);
+
+/*
  * Verification with the same look-ahead SL for all B sequences (Sec. 2; Fig. 1).
  *   W_T        bf16 [V, d_target]          target LM head
  *   H_T        bf16 [B*(SL+1), d_target]   row b*(SL+1)+j is the target hidden state whose

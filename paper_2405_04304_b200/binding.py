@@ -30,6 +30,7 @@ EXPORTS = [
     "disco_create", "disco_destroy", "disco_strerror", "disco_last_device_status", "disco_launch_count",
     "disco_set_kernel_path", "disco_draft_step", "disco_verify", "disco_verify_ragged",
     "disco_draft_step_host", "disco_verify_ragged_host", "disco_draft_step_static", "disco_draft_step_ppl",
+    "disco_draft_step_sample", "disco_verify_sample_ragged",
 ]
 
 
@@ -67,6 +68,9 @@ def load() -> ctypes.CDLL:
     lib.disco_draft_step.argtypes = [vp, vp, vp, ci, vp, vp, vp, ctypes.POINTER(_Clf), cf, ci,
                                      vp, vp, vp, vp, vp, vp]
     lib.disco_draft_step_ppl.argtypes = [vp, vp, vp, ci, vp, vp, vp, cf, ci, vp, vp, vp, vp]
+    lib.disco_draft_step_sample.argtypes = [vp, vp, vp, ci, vp, vp, vp, ctypes.POINTER(_Clf), cf, ci, vp,
+                                            vp, vp, vp, vp, vp, vp, vp]
+    lib.disco_verify_sample_ragged.argtypes = [vp, vp, vp, vp, vp, vp, ci, ci, vp, vp, vp, vp, vp, vp, vp]
     lib.disco_verify.argtypes = [vp, vp, vp, vp, ci, ci, vp, vp, vp, vp]
     lib.disco_verify_ragged.argtypes = [vp, vp, vp, vp, vp, ci, ci, vp, vp, vp, vp]
     lib.disco_draft_step_host.argtypes = [vp, vp, vp, ci, vp, vp, vp, ctypes.POINTER(_Clf), cf, ci,
@@ -197,6 +201,29 @@ class Context:
             _ptr(token, torch.int32), _ptr(ppl, torch.float32), _ptr(halt, torch.uint8), _stream(stream))
         if rc != OK:
             raise DiscoError(rc, "disco_draft_step_ppl")
+
+    def draft_step_sample(self, W_D, h_D, pos, n_drafted, clf: Classifier, tau: float, sl_max: int, u,
+                          token, conf, halt, probs, p_token=None, active=None, feats=None, stream=None) -> None:
+        B = int(h_D.shape[0])
+        rc = self._lib.disco_draft_step_sample(
+            self._h, _ptr(W_D, torch.bfloat16), _ptr(h_D, torch.bfloat16), B, _ptr(pos, torch.int32),
+            _ptr(n_drafted, torch.int32), _ptr(active, torch.uint8), ctypes.byref(clf._c), float(tau),
+            int(sl_max), _ptr(u, torch.float32), _ptr(token, torch.int32), _ptr(p_token, torch.float32),
+            _ptr(conf, torch.float32), _ptr(halt, torch.uint8), _ptr(feats, torch.float32),
+            _ptr(probs, torch.float32), _stream(stream))
+        if rc != OK:
+            raise DiscoError(rc, "disco_draft_step_sample")
+
+    def verify_sample_ragged(self, W_T, H_T, draft_ids, draft_probs, row_off, B: int, R: int, u_accept,
+                             u_sample, n_accept, next_token, y_T, target_ids=None, stream=None) -> None:
+        rc = self._lib.disco_verify_sample_ragged(
+            self._h, _ptr(W_T, torch.bfloat16), _ptr(H_T, torch.bfloat16), _ptr(draft_ids, torch.int32),
+            _ptr(draft_probs, torch.float32), _ptr(row_off, torch.int32), int(B), int(R),
+            _ptr(u_accept, torch.float32), _ptr(u_sample, torch.float32), _ptr(n_accept, torch.int32),
+            _ptr(next_token, torch.int32), _ptr(y_T, torch.float32), _ptr(target_ids, torch.int32),
+            _stream(stream))
+        if rc != OK:
+            raise DiscoError(rc, "disco_verify_sample_ragged")
 
     def verify(self, W_T, H_T, draft_ids, B: int, SL: int, n_accept, bonus, target_ids=None,
                stream=None) -> None:

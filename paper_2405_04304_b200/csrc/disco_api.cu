@@ -11,6 +11,7 @@
 #include "disco.h"
 #include "stream_tail.cuh"
 #include "umma_tail.cuh"
+#include "sample.cuh"
 #include "umma_gemv.cuh"
 
 using namespace disco;
@@ -211,7 +212,7 @@ int launch_umma(disco_ctx* c, const void* W, const void* H, int d, int R, float*
     p.keys = c->keys;
     p.part_rec = reinterpret_cast<float4*>(c->stamped_rec);
     p.probs = probs;
-    if (DRAFT && (p.CN > c->part_slots || R > c->part_rows)) return DISCO_ERR_WORKSPACE;
+    if (DRAFT && ((size_t)R * p.CN > (size_t)128 * c->sm_count || R > c->part_rows)) return DISCO_ERR_WORKSPACE;
     CUtensorMap tmap_W, tmap_H;
     if (!encode_bf16_2d(c, &tmap_W, W, c->V, d, p.TRN) || !encode_bf16_2d(c, &tmap_H, H, R, d, p.a_rows))
         return DISCO_ERR_CUDA;
@@ -365,7 +366,7 @@ int disco_create(disco_ctx** out, int V, int d_draft, int d_target, int max_batc
 
     const int rpc = std::max(1, std::min((V + c->sm_count - 1) / c->sm_count, 2048));
     c->max_grid = (V + rpc - 1) / rpc;
-    c->part_rows = max_batch;
+    c->part_rows = std::max(max_batch, max_rows);  // the target rows of a verification with sampling go the same way
     c->part_slots = std::max(c->max_grid, 2 * c->sm_count);
     const size_t slots = (size_t)c->part_rows * c->part_slots;
     {
@@ -383,15 +384,16 @@ int disco_create(disco_ctx** out, int V, int d_draft, int d_target, int max_batc
     ok = ok && cudaMalloc(&c->part_rec, slots * 64) == cudaSuccess;
     ok = ok && cudaMalloc(&c->ticket, 1024) == cudaSuccess;
     ok = ok && cudaMalloc(&c->status, 256) == cudaSuccess;
-    ok = ok && cudaMalloc(&c->final_stats, (size_t)max_batch * 2 * sizeof(float)) == cudaSuccess;
+    ok = ok && cudaMalloc(&c->final_stats, (size_t)c->part_rows * 2 * sizeof(float)) == cudaSuccess;
     ok = ok && cudaMalloc(&c->stage_hidden, hid) == cudaSuccess;
     ok = ok && cudaMalloc(&c->stage_int, n_int * sizeof(int32_t)) == cudaSuccess;
     ok = ok && cudaMalloc(&c->stage_float, (size_t)max_batch * (1 + kNFeat) * sizeof(float)) == cudaSuccess;
     ok = ok && cudaMalloc(&c->stage_byte, (size_t)max_batch * 2 + 64) == cudaSuccess;
     ok = ok && cudaMemset(c->keys, 0, (size_t)max_rows * sizeof(unsigned long long)) == cudaSuccess;
     ok = ok && cudaMemset(c->ticket, 0, 1024) == cudaSuccess;
-    ok = ok && cudaMalloc(&c->stamped_rec, (size_t)c->part_rows * c->sm_count * 80) == cudaSuccess;
-    ok = ok && cudaMemset(c->stamped_rec, 0, (size_t)c->part_rows * c->sm_count * 80) == cudaSuccess;  // no stamp yet
+    // R rows take R * (sm_count / ceil(R / 128)) <= 128 * sm_count records
+    ok = ok && cudaMalloc(&c->stamped_rec, (size_t)128 * c->sm_count * 80) == cudaSuccess;
+    ok = ok && cudaMemset(c->stamped_rec, 0, (size_t)128 * c->sm_count * 80) == cudaSuccess;  // no stamp yet
     ok = ok && cudaMemset(c->status, 0, 256) == cudaSuccess;
     ok = ok && cudaDeviceSynchronize() == cudaSuccess;
     if (!ok) {
@@ -443,19 +445,22 @@ int disco_set_kernel_path(disco_ctx* c, int which) {
 }  // extern "C"
 
 namespace {
-// Shared body of the two draft-step entry points.  nll_sum != null selects the perplexity rule (no
-// classifier; tau is the perplexity bound).
-int draft_step_common(disco_ctx* c, const void* W_D, const void* h_D, int B, const int32_t* pos,
+// Shared body of the LM-head + soft-max passes: B rows of hidden size d against the head W.
+//   * nll_sum != null selects the perplexity rule (no classifier; tau is the perplexity bound);
+//   * stats_only: arg-max (token, optional) and soft-max statistics only, no classifier: the target
+//     rows of a verification with sampling (pos, n_drafted, conf, halt unused).
+int draft_step_common(disco_ctx* c, const void* W_D, const void* h_D, int d, int B, int max_rows, const int32_t* pos,
                       const int32_t* n_drafted, const uint8_t* active, const disco_clf* clf, float tau,
                       int sl_max, int32_t* token, float* conf, uint8_t* halt, float* feats, float* probs,
-                      float* nll_sum, void* stream) {
-    if (!c || !W_D || !h_D || !pos || !n_drafted || !token || !conf || !halt) return DISCO_ERR_INVALID_ARG;
+                      float* nll_sum, bool stats_only, void* stream) {
+    if (!c || !W_D || !h_D) return DISCO_ERR_INVALID_ARG;
+    if (!stats_only && (!pos || !n_drafted || !token || !conf || !halt)) return DISCO_ERR_INVALID_ARG;
     if (!aligned16(W_D) || !aligned16(h_D)) return DISCO_ERR_INVALID_ARG;
     if (B < 1 || sl_max < 1) return DISCO_ERR_INVALID_ARG;
-    if (B > c->max_batch) return DISCO_ERR_WORKSPACE;
+    if (B > max_rows) return DISCO_ERR_WORKSPACE;
     static const disco_clf no_clf = {nullptr, nullptr, nullptr, nullptr, 0};
     int rc = DISCO_OK;
-    if (nll_sum) {
+    if (nll_sum || stats_only) {
         clf = &no_clf;
     } else {
         rc = check_clf(c, clf);
@@ -467,10 +472,11 @@ int draft_step_common(disco_ctx* c, const void* W_D, const void* h_D, int B, con
     p.W = static_cast<const uint16_t*>(W_D);
     p.H = static_cast<const uint16_t*>(h_D);
     p.V = c->V;
-    p.d = c->d_draft;
+    p.d = d;
     p.R = B;
     p.B = B;
     fill_scratch(c, p);
+    p.stats_only = stats_only ? 1 : 0;
     p.pos = pos;
     p.n_drafted = n_drafted;
     p.active = active;
@@ -490,7 +496,7 @@ int draft_step_common(disco_ctx* c, const void* W_D, const void* h_D, int B, con
     // Measured on B200 (Vicuna head): up to 6 sequences are fastest on the tensor-core kernel with the
     // vocabulary on the TMEM lanes, more on the one with the hidden rows on the lanes; the CUDA-core
     // streaming kernel is within 10 % for one sequence and serves as the path without tensor maps.
-    const bool gemv_ok = c->encode_tiled != nullptr && B <= kGemvMaxRows;
+    const bool gemv_ok = c->encode_tiled != nullptr && B <= kGemvMaxRows && !stats_only;
     const bool use_gemv = gemv_ok && (c->path == 3 || (c->path == 0 && B <= 6));
     const bool use_umma = !use_gemv && umma_possible(c, B) && (c->path == 2 || c->path == 3 || (c->path == 0 && B >= 2));
     if (use_gemv) {
@@ -515,8 +521,9 @@ int draft_step_common(disco_ctx* c, const void* W_D, const void* h_D, int B, con
         f.feats = feats;
         f.final_stats = c->final_stats;
         f.nll_sum = nll_sum;
+        f.stats_only = stats_only ? 1 : 0;
         f.epoch = c->ticket + 48;
-        rc = launch_umma<true>(c, W_D, h_D, c->d_draft, B, probs, &f, nullptr, st);
+        rc = launch_umma<true>(c, W_D, h_D, d, B, probs, &f, nullptr, st);
         if (rc) return rc;
     } else {
         rc = run_stream<true>(c, p, clf->H, st);
@@ -539,16 +546,65 @@ int disco_draft_step(disco_ctx* c, const void* W_D, const void* h_D, int B, cons
                      const int32_t* n_drafted, const uint8_t* active, const disco_clf* clf, float tau,
                      int sl_max, int32_t* token, float* conf, uint8_t* halt, float* feats, float* probs,
                      void* stream) {
-    return draft_step_common(c, W_D, h_D, B, pos, n_drafted, active, clf, tau, sl_max, token, conf, halt, feats,
-                             probs, nullptr, stream);
+    if (!c) return DISCO_ERR_INVALID_ARG;
+    return draft_step_common(c, W_D, h_D, c->d_draft, B, c->max_batch, pos, n_drafted, active, clf, tau, sl_max, token,
+                             conf, halt, feats, probs, nullptr, false, stream);
 }
 
 int disco_draft_step_ppl(disco_ctx* c, const void* W_D, const void* h_D, int B, const int32_t* n_drafted,
                          const uint8_t* active, float* nll_sum, float ppl_max, int sl_max, int32_t* token,
                          float* ppl, uint8_t* halt, void* stream) {
     if (!nll_sum) return DISCO_ERR_INVALID_ARG;
-    return draft_step_common(c, W_D, h_D, B, n_drafted, n_drafted, active, nullptr, ppl_max, sl_max, token, ppl,
-                             halt, nullptr, nullptr, nll_sum, stream);
+    if (!c) return DISCO_ERR_INVALID_ARG;
+    return draft_step_common(c, W_D, h_D, c->d_draft, B, c->max_batch, n_drafted, n_drafted, active, nullptr, ppl_max,
+                             sl_max, token, ppl, halt, nullptr, nullptr, nll_sum, false, stream);
+}
+
+int disco_draft_step_sample(disco_ctx* c, const void* W_D, const void* h_D, int B, const int32_t* pos,
+                            const int32_t* n_drafted, const uint8_t* active, const disco_clf* clf, float tau,
+                            int sl_max, const float* u, int32_t* token, float* p_token, float* conf, uint8_t* halt,
+                            float* feats, float* probs, void* stream) {
+    if (!c || !u || !probs) return DISCO_ERR_INVALID_ARG;
+    int rc = draft_step_common(c, W_D, h_D, c->d_draft, B, c->max_batch, pos, n_drafted, active, clf, tau, sl_max,
+                               token, conf, halt, feats, probs, nullptr, false, stream);
+    if (rc) return rc;
+    // probs now holds y^D; the greedy token is replaced by the draw
+    sample_rows_kernel<<<B, kSampleThreads, 0, static_cast<cudaStream_t>(stream)>>>(probs, u, active, c->V, token,
+                                                                                   p_token);
+    c->launches += 1;
+    return cuda_ok(cudaGetLastError(), "sample_rows_kernel launch") ? DISCO_OK : DISCO_ERR_CUDA;
+}
+
+int disco_verify_sample_ragged(disco_ctx* c, const void* W_T, const void* H_T, const int32_t* draft_ids,
+                               const float* draft_probs, const int32_t* row_off, int B, int R,
+                               const float* u_accept, const float* u_sample, int32_t* n_accept,
+                               int32_t* next_token, float* y_T, int32_t* target_ids, void* stream) {
+    if (!c || !W_T || !H_T || !u_sample || !n_accept || !next_token || !y_T) return DISCO_ERR_INVALID_ARG;
+    if (B < 1 || R < B) return DISCO_ERR_INVALID_ARG;
+    if (R > B && (!draft_ids || !draft_probs || !u_accept)) return DISCO_ERR_INVALID_ARG;
+    if (B > c->max_batch || R > c->max_rows) return DISCO_ERR_WORKSPACE;
+    // target distributions of all rows: LM head, soft-max statistics, normalised rows in y_T
+    int rc = draft_step_common(c, W_T, H_T, c->d_target, R, c->max_rows, nullptr, nullptr, nullptr, nullptr, 0.f, 1,
+                               target_ids, nullptr, nullptr, nullptr, y_T, nullptr, true, stream);
+    if (rc) return rc;
+    SpecSampleParams sp{};
+    sp.y_T = y_T;
+    sp.draft_probs = draft_probs;
+    sp.draft_ids = draft_ids;
+    sp.row_off = row_off;
+    sp.u_accept = u_accept;
+    sp.u_sample = u_sample;
+    sp.B = B;
+    sp.SL = row_off ? 0 : (R / B - 1);
+    sp.R = R;
+    sp.V = c->V;
+    sp.n_accept = n_accept;
+    sp.next_token = next_token;
+    sp.status = c->status;
+    if (!row_off && R % B != 0) return DISCO_ERR_INVALID_ARG;
+    speculative_sample_kernel<<<B, kSampleThreads, 0, static_cast<cudaStream_t>(stream)>>>(sp);
+    c->launches += 1;
+    return cuda_ok(cudaGetLastError(), "speculative_sample_kernel launch") ? DISCO_OK : DISCO_ERR_CUDA;
 }
 
 int disco_verify_ragged(disco_ctx* c, const void* W_T, const void* H_T, const int32_t* draft_ids,

@@ -56,6 +56,7 @@ struct TailParams {
     float* feats;
     float* probs;
     float* nll_sum;      // non-null: perplexity rule instead of the classifier (tau is then the perplexity bound)
+    int stats_only;      // non-zero: arg-max and soft-max statistics only; pos, n_drafted and the classifier are unused
     // verification
     const int32_t* draft_ids;
     const int32_t* row_off;  // null: uniform SL
@@ -526,11 +527,20 @@ struct DraftOutputs {
     float* feats;
     float* final_stats;
     float* nll_sum;  // non-null: perplexity rule (App. F) instead of the classifier
+    int stats_only;  // non-zero: arg-max and soft-max statistics only (rows of a verification with sampling)
 };
 __device__ __forceinline__ void warp_draft_epilogue(const SoftmaxState& st, unsigned long long key, float sel, float fpos,
                                                     int n_drafted, float tau, int sl_max, float* feat_s, const float* W1,
                                                     const float* b1, const float* w2, const float* b2, int Hc, int b,
                                                     const DraftOutputs& o, int lane) {
+    if (o.stats_only) {
+        if (lane == 0) {
+            if (o.token) o.token[b] = key_index(key);
+            o.final_stats[2 * b] = st.m;
+            o.final_stats[2 * b + 1] = st.Z;
+        }
+        return;
+    }
     if (o.nll_sum) {
         // Perplexity rule: the greedy token attains the largest logit, so -ln y(token) = ln Z.  The caller
         // keeps the running sum over the tokens drafted in this iteration; halt when the perplexity of
@@ -567,12 +577,12 @@ __device__ __forceinline__ void warp_draft_epilogue(const SoftmaxState& st, unsi
 // feat16: kWarpScratchWords words of shared memory owned by the calling warp.
 __device__ __forceinline__ void finalize_draft_seq(const TailParams& p, int b, int grid, float* feat16, const float* clf_s,
                                                    int lane) {
-    const float fpos = static_cast<float>(p.pos[b]);  // issued early: hidden behind the merge
-    const int n_drafted = p.n_drafted[b];
+    const float fpos = p.pos ? static_cast<float>(p.pos[b]) : 0.f;  // issued early: hidden behind the merge
+    const int n_drafted = p.n_drafted ? p.n_drafted[b] : 0;
     const MergedPartials mp = warp_merge_partials(p.part_rec + (size_t)b * grid * 4, grid, feat16 + 16, lane);
     const int Hc = p.clf_H;
     const SoftmaxState st = mp.st;
-    const DraftOutputs o{p.token, p.conf, p.halt, p.feats, p.final_stats, p.nll_sum};
+    const DraftOutputs o{p.token, p.conf, p.halt, p.feats, p.final_stats, p.nll_sum, p.stats_only};
     warp_draft_epilogue(st, mp.key, mp.sel, fpos, n_drafted, p.tau, p.sl_max, feat16, clf_s, clf_s + Hc * kNFeat,
                         clf_s + Hc * (kNFeat + 1), clf_s + Hc * (kNFeat + 2), Hc, b, o, lane);
 }

@@ -161,6 +161,7 @@ struct DraftFinalParams {
     float* feats;
     float* final_stats;
     float* nll_sum;
+    int stats_only;
     unsigned int* epoch;  // [0] launches completed so far (stamp of this launch = that + 1), [1] finishing warps done
 };
 
@@ -173,7 +174,7 @@ __device__ __forceinline__ void umma_finish_sequence(const DraftFinalParams& p, 
         warp_merge_partials(part_rec + (size_t)b * NP * kStampedPieces, NP, feat16 + 16, lane, stamp, status);
     if (!active) return;
     const int Hc = p.clf_H;
-    const DraftOutputs o{p.token, p.conf, p.halt, p.feats, p.final_stats, p.nll_sum};
+    const DraftOutputs o{p.token, p.conf, p.halt, p.feats, p.final_stats, p.nll_sum, p.stats_only};
     warp_draft_epilogue(mp.st, mp.key, mp.sel, fpos, n_drafted, p.tau, p.sl_max, feat16, clf_s, clf_s + Hc * kNFeat,
                         clf_s + Hc * (kNFeat + 1), clf_s + Hc * (kNFeat + 2), Hc, b, o, lane);
 }
@@ -437,8 +438,8 @@ umma_tail_kernel(const __grid_constant__ CUtensorMap tmap_W, const __grid_consta
             if (first < f.B) {
                 int b = first;
                 bool act = !f.active || f.active[b];
-                float fpos = static_cast<float>(f.pos[b]);
-                int nd = f.n_drafted[b];
+                float fpos = f.pos ? static_cast<float>(f.pos[b]) : 0.f;
+                int nd = f.n_drafted ? f.n_drafted[b] : 0;
                 float* feat16 = reinterpret_cast<float*>(xch) + ew * kWarpScratchWords;  // the exchange area is free again
                 for (;;) {
                     // a masked sequence still waits for its records: the stamp may only advance once
@@ -447,8 +448,8 @@ umma_tail_kernel(const __grid_constant__ CUtensorMap tmap_W, const __grid_consta
                     b += kUmmaEpiWarps * (int)gridDim.x;
                     if (b >= f.B) break;
                     act = !f.active || f.active[b];
-                    fpos = static_cast<float>(f.pos[b]);
-                    nd = f.n_drafted[b];
+                    fpos = f.pos ? static_cast<float>(f.pos[b]) : 0.f;
+                    nd = f.n_drafted ? f.n_drafted[b] : 0;
                 }
                 // the last finishing warp of the grid advances the stamp for the next launch: by then every
                 // record of this launch has been read

@@ -417,3 +417,159 @@ def test_draft_step_with_perplexity_rule(oracle, path, V, d, B):
         np.testing.assert_allclose(nll_gpu.cpu().numpy(), nll_ref, rtol=1e-4, atol=1e-4)
     assert ctx.device_status() == 0
     ctx.close()
+
+
+# ---------------------------------------------------------------------------------- sampling at temperature 1
+CDF_TOL = 2e-5      # slack on a running sum of fp32 probabilities against the fp64 ones
+RATIO_TOL = 1e-4    # an acceptance test whose two sides are closer than this (relative) may go either way
+
+
+def _valid_draw(weights, u, tok, tol=CDF_TOL):
+    """Is tok an inverse-CDF draw from the (fp64) weights for u, up to tol of the total on the running sums?"""
+    cdf = np.cumsum(np.asarray(weights, dtype=np.float64))
+    target = float(u) * cdf[-1]
+    slack = tol * cdf[-1]
+    if tok < 0 or tok >= len(cdf) or weights[tok] <= 0:
+        return False
+    return cdf[tok] > target - slack and (tok == 0 or cdf[tok - 1] <= target + slack)
+
+
+@pytest.mark.parametrize("path", [0, 1, 2, 3])
+@pytest.mark.parametrize("V,d,B", [(11, 8, 2), (1000, 72, 5), (4099, 264, 7), (32000, 768, 1), (5000, 128, 40)])
+def test_draft_step_sample(oracle, path, V, d, B):
+    if path == 3 and B > 16:
+        pytest.skip("the kernel with the vocabulary on the TMEM lanes takes up to 16 sequences")
+    W = inputs.lm_head(V, d, seed=V + 2 * d, std=0.25)
+    h = inputs.hidden(B, d, seed=V * 5 + B)
+    params = make_clf(32, seed=V + 3)
+    pos = np.arange(1, B + 1, dtype=np.int32) * 2
+    nd = (np.arange(B, dtype=np.int32) % 5) + 1
+    g = torch.Generator().manual_seed(V + B)
+    u = torch.rand(B, generator=g, dtype=torch.float32)
+    u[0] = 0.0
+    if B > 1:
+        u[1] = float(np.nextafter(np.float32(1.0), np.float32(0.0)))
+    active = np.ones(B, dtype=np.uint8)
+    if B > 2:
+        active[2] = 0
+    ctx = _ctx(V, d, 8, max_batch=max(8, B), H=32)
+    ctx.set_kernel_path(path)
+    token = torch.full((B,), -7, dtype=torch.int32, device="cuda")
+    p_tok = torch.full((B,), -7.0, dtype=torch.float32, device="cuda")
+    conf = torch.full((B,), -7.0, dtype=torch.float32, device="cuda")
+    halt = torch.full((B,), 77, dtype=torch.uint8, device="cuda")
+    feats = torch.full((B, binding.NFEAT), -7.0, dtype=torch.float32, device="cuda")
+    probs = torch.full((B, V), -7.0, dtype=torch.float32, device="cuda")
+    ctx.draft_step_sample(W.cuda(), h.cuda(), torch.from_numpy(pos).cuda(), torch.from_numpy(nd).cuda(),
+                          to_gpu_clf(params), 0.5, 4, u.cuda(), token, conf, halt, probs, p_token=p_tok,
+                          active=torch.from_numpy(active).cuda(), feats=feats)
+    torch.cuda.synchronize()
+    ref = oracle.draft_step_sample(_bits(W), _bits(h), pos, nd, to_oracle_clf(oracle, params), 0.5, 4,
+                                   u.numpy().astype(np.float64), active=active)
+    got = dict(token=token.cpu().numpy(), conf=conf.cpu().numpy(), halt=halt.cpu().numpy(),
+               feats=feats.cpu().numpy(), probs=probs.cpu().numpy())
+    pt = p_tok.cpu().numpy()
+    for b in range(B):
+        if not active[b]:
+            assert got["token"][b] == -7 and pt[b] == -7.0 and got["halt"][b] == 77
+            continue
+        np.testing.assert_allclose(got["probs"][b], ref.probs[b], rtol=0, atol=2e-3)
+        np.testing.assert_allclose(got["feats"][b], ref.feats[b], rtol=0, atol=2e-3)
+        assert abs(float(got["conf"][b]) - ref.conf[b]) <= 2e-3
+        if abs(ref.conf[b] - 0.5) >= 1e-4:
+            assert got["halt"][b] == ref.halt[b]
+        tok = int(got["token"][b])
+        assert tok == ref.token[b] or _valid_draw(ref.probs[b], float(u[b]), tok), f"seq {b}: token {tok}"
+        assert abs(pt[b] - ref.probs[b, tok]) <= 2e-3
+    assert int(got["token"][0]) == int(ref.token[0])            # u = 0: the first token with mass
+    assert ctx.device_status() == 0
+    ctx.close()
+
+
+def _verify_sample_case(oracle, V, d, sls, seed, path=0, uniform=False, noise=0.6):
+    B = len(sls)
+    row_off = np.concatenate([[0], np.cumsum([s + 1 for s in sls])]).astype(np.int32)
+    R = int(row_off[-1])
+    W = inputs.lm_head(V, d, seed=seed, std=0.25)
+    H = inputs.hidden(R, d, seed=seed + 1)
+    rng = np.random.default_rng(seed)
+    steps = max(max(sls), 1)
+    # draft distributions near the target's (so that a good share of the tokens is accepted): soft-max of
+    # the oracle's target logits plus noise, in binary32; tokens drawn from them
+    z = oracle.project(_bits(W), _bits(H), nthreads=8)
+    dp = np.zeros((steps, B, V), dtype=np.float32)
+    ids = np.zeros(R - B, dtype=np.int32)
+    for b in range(B):
+        for i in range(sls[b]):
+            zz = z[row_off[b] + i] + noise * rng.normal(size=V)
+            e = np.exp(zz - zz.max())
+            dp[i, b] = (e / e.sum()).astype(np.float32)
+            ids[row_off[b] - b + i] = rng.choice(V, p=dp[i, b].astype(np.float64) / dp[i, b].astype(np.float64).sum())
+    ua = rng.random(R - B).astype(np.float32)
+    us = rng.random(B).astype(np.float32)
+    ctx = _ctx(V, 8, d, max_batch=max(8, B), max_rows=max(64, R))
+    ctx.set_kernel_path(path)
+    n_acc = torch.full((B,), -7, dtype=torch.int32, device="cuda")
+    nxt = torch.full((B,), -7, dtype=torch.int32, device="cuda")
+    yT = torch.full((R, V), -7.0, dtype=torch.float32, device="cuda")
+    tids = torch.full((R,), -7, dtype=torch.int32, device="cuda")
+    ctx.verify_sample_ragged(W.cuda(), H.cuda(), torch.from_numpy(ids).cuda() if R > B else None,
+                             torch.from_numpy(dp).cuda() if R > B else None,
+                             None if uniform else torch.from_numpy(row_off).cuda(), B, R,
+                             torch.from_numpy(ua).cuda() if R > B else None, torch.from_numpy(us).cuda(),
+                             n_acc, nxt, yT, target_ids=tids)
+    torch.cuda.synchronize()
+    assert ctx.device_status() == 0
+    ctx.close()
+    ref = oracle.verify_sample(_bits(W), _bits(H), ids, dp, row_off, ua.astype(np.float64), us.astype(np.float64),
+                               nthreads=8)
+    n_g, x_g, y_g = n_acc.cpu().numpy(), nxt.cpu().numpy(), yT.cpu().numpy()
+    np.testing.assert_allclose(y_g, ref.y_T, rtol=0, atol=2e-3)
+    np.testing.assert_allclose(y_g.astype(np.float64).sum(axis=1), 1.0, atol=1e-4)
+    srt = np.sort(z, axis=1)
+    tied = srt[:, -1] - srt[:, -2] < 1e-3
+    assert np.all((tids.cpu().numpy() == z.argmax(axis=1)) | tied)
+    accepted_total = 0
+    for b in range(B):
+        r0, sl = int(row_off[b]), sls[b]
+        n_o = int(ref.n_accept[b])
+        # acceptance tests that are decided by less than RATIO_TOL may go either way
+        close = []
+        for i in range(sl):
+            t = ids[r0 - b + i]
+            pT, pD = ref.y_T[r0 + i, t], float(dp[i, b, t])
+            close.append(abs(float(ua[r0 - b + i]) * pD - pT) <= RATIO_TOL * max(pT, 1e-30))
+        n = int(n_g[b])
+        assert 0 <= n <= sl
+        if n != n_o:
+            assert close[min(n, n_o)], f"seq {b}: n_accept {n} != {n_o}"
+        if n < sl:
+            w = np.maximum(0.0, ref.y_T[r0 + n] - dp[n, b].astype(np.float64))
+            if not w.sum() > 0:
+                w = ref.y_T[r0 + n]
+        else:
+            w = ref.y_T[r0 + sl]
+        tok = int(x_g[b])
+        assert (n == n_o and tok == ref.next_token[b]) or _valid_draw(w, float(us[b]), tok), f"seq {b}: next {tok}"
+        accepted_total += n
+    return accepted_total, R - B
+
+
+@pytest.mark.parametrize("path", [0, 1])
+@pytest.mark.parametrize("V,d,sls", [(7, 8, [0]), (64, 16, [5]), (1000, 136, [3, 0, 5, 1]),
+                                     (4099, 72, [1, 2, 3, 4, 5, 6]), (5000, 64, [7] * 20)])
+def test_verify_sample_small_shapes(oracle, path, V, d, sls):
+    _verify_sample_case(oracle, V, d, sls, seed=V + len(sls), path=path)
+
+
+def test_verify_sample_uniform_look_ahead_and_acceptance_range(oracle):
+    acc, tot = _verify_sample_case(oracle, 2000, 64, [4] * 12, seed=77, uniform=True, noise=0.3)
+    assert 0.3 * tot < acc <= tot                # close distributions: most tokens pass
+    acc2, tot2 = _verify_sample_case(oracle, 2000, 64, [4] * 12, seed=78, uniform=True, noise=6.0)
+    assert acc2 < 0.6 * tot2                     # distant distributions: early rejections
+
+
+@pytest.mark.parametrize("name,SL", [("vicuna_b1", 10), ("starcoder_b1", 10)])
+def test_verify_sample_full_size_heads(oracle, name, SL):
+    wl = inputs.WORKLOADS[name]
+    _verify_sample_case(oracle, wl.V, wl.d_T, [SL], seed=wl.seed + 40)
