@@ -452,7 +452,7 @@ namespace {
 int draft_step_common(disco_ctx* c, const void* W_D, const void* h_D, int d, int B, int max_rows, const int32_t* pos,
                       const int32_t* n_drafted, const uint8_t* active, const disco_clf* clf, float tau,
                       int sl_max, int32_t* token, float* conf, uint8_t* halt, float* feats, float* probs,
-                      float* nll_sum, bool stats_only, void* stream) {
+                      float* nll_sum, bool stats_only, void* stream, bool normalize = true) {
     if (!c || !W_D || !h_D) return DISCO_ERR_INVALID_ARG;
     if (!stats_only && (!pos || !n_drafted || !token || !conf || !halt)) return DISCO_ERR_INVALID_ARG;
     if (!aligned16(W_D) || !aligned16(h_D)) return DISCO_ERR_INVALID_ARG;
@@ -529,7 +529,7 @@ int draft_step_common(disco_ctx* c, const void* W_D, const void* h_D, int d, int
         rc = run_stream<true>(c, p, clf->H, st);
         if (rc) return rc;
     }
-    if (probs) {
+    if (probs && normalize) {
         dim3 grid((unsigned)std::min(64, (c->V + 255) / 256), (unsigned)B);
         normalize_probs_kernel<<<grid, 256, 0, st>>>(probs, c->final_stats, active, c->V);
         c->launches += 1;
@@ -566,11 +566,11 @@ int disco_draft_step_sample(disco_ctx* c, const void* W_D, const void* h_D, int 
                             float* feats, float* probs, void* stream) {
     if (!c || !u || !probs) return DISCO_ERR_INVALID_ARG;
     int rc = draft_step_common(c, W_D, h_D, c->d_draft, B, c->max_batch, pos, n_drafted, active, clf, tau, sl_max,
-                               token, conf, halt, feats, probs, nullptr, false, stream);
+                               token, conf, halt, feats, probs, nullptr, false, stream, false);
     if (rc) return rc;
-    // probs now holds y^D; the greedy token is replaced by the draw
-    sample_rows_kernel<<<B, kSampleThreads, 0, static_cast<cudaStream_t>(stream)>>>(probs, u, active, c->V, token,
-                                                                                   p_token);
+    // probs holds the logits: the kernel turns them into y^D and replaces the greedy token by the draw
+    sample_rows_kernel<<<B, kSampleThreads, 0, static_cast<cudaStream_t>(stream)>>>(probs, c->final_stats, u, active,
+                                                                                   c->V, token, p_token);
     c->launches += 1;
     return cuda_ok(cudaGetLastError(), "sample_rows_kernel launch") ? DISCO_OK : DISCO_ERR_CUDA;
 }

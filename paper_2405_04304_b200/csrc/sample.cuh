@@ -11,70 +11,93 @@
 
 namespace disco {
 
-constexpr int kSampleThreads = 256;
+constexpr int kSampleThreads = 512;
+constexpr int kSampleWarps = kSampleThreads / 32;
 
-// Inverse-CDF draw by one CTA of kSampleThreads threads: the smallest v whose running sum
-// w(0) + .. + w(v) exceeds u * (w(0) + .. + w(V-1)); if rounding leaves none, the last v with w(v) > 0;
-// -1 if every weight is zero.  w(v) >= 0 is a callable.  Every thread returns the token.
-// sh: kSampleThreads / 32 + 2 doubles of shared memory; total (optional) receives the sum.
+// Inverse-CDF draw by one CTA of kSampleThreads threads from weights w(v) >= 0, v < V (a callable that
+// returns the same value whenever it is asked again): the smallest v whose running sum w(0) + .. + w(v)
+// exceeds u * (sum of all); if rounding leaves none, the last v with w(v) > 0; -1 if every weight is zero.
+// Every thread returns the token.  Three steps, each warp owning one contiguous segment of the row:
+//   A  segment totals (coalesced reads, lane-strided partial sums);
+//   B  the segment that holds the crossing, from the 16 totals;
+//   C  inside that segment only: each lane sums a contiguous piece, a warp scan finds the lane, and the
+//      lane walks its piece in vocabulary order.
+// sh: 24 doubles of shared memory; total (optional) receives the sum.
 template <typename WeightFn>
 __device__ __forceinline__ int block_sample_cdf(WeightFn w, int V, double u, double* sh, double* total_out) {
     const int t = threadIdx.x, lane = t & 31, warp = t >> 5;
-    const int chunk = (V + kSampleThreads - 1) / kSampleThreads;
-    const int v0 = min(V, t * chunk), v1 = min(V, v0 + chunk);
-    double mine = 0.0;
-    for (int v = v0; v < v1; ++v) mine += w(v);
-    // inclusive scan of the per-thread sums: inside each warp, then over the warp totals
-    double incl = mine;
-#pragma unroll
-    for (int off = 1; off < 32; off <<= 1) {
-        const double o = __shfl_up_sync(kFullMask, incl, off);
-        if (lane >= off) incl += o;
-    }
-    double* warp_tot = sh;                        // [8]
-    int* found = reinterpret_cast<int*>(sh + 8);  // [2]: token, last index with positive weight
-    if (lane == 31) warp_tot[warp] = incl;
+    const int seg = ((V + kSampleWarps - 1) / kSampleWarps + 31) & ~31;  // entries per warp, whole 32s
+    const int s0 = min(V, warp * seg), s1 = min(V, s0 + seg);
+    double* warp_tot = sh;                                     // [kSampleWarps]
+    int* found = reinterpret_cast<int*>(sh + kSampleWarps);    // [2]: token, last index with positive weight
     if (t == 0) {
         found[0] = -1;
         found[1] = -1;
     }
+    // A
+    double part = 0.0;
+    int last = -1;
+#pragma unroll 4
+    for (int v = s0 + lane; v < s1; v += 32) {
+        const float x = w(v);
+        part += static_cast<double>(x);
+        if (x > 0.f) last = v;
+    }
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) {
+        part += __shfl_xor_sync(kFullMask, part, off);
+        last = max(last, __shfl_xor_sync(kFullMask, last, off));
+    }
+    if (lane == 0) warp_tot[warp] = part;
     __syncthreads();
+    if (lane == 0 && last >= 0) atomicMax(&found[1], last);
+    // B
     double before = 0.0, total = 0.0;
 #pragma unroll
-    for (int k = 0; k < kSampleThreads / 32; ++k) {
+    for (int k = 0; k < kSampleWarps; ++k) {
         const double wt = warp_tot[k];
         if (k < warp) before += wt;
         total += wt;
     }
-    incl += before;
-    const double excl = incl - mine;
     const double target = u * total;
-    // exactly one thread holds the crossing (its chunk starts at or below the target and ends above it)
-    if (excl <= target && incl > target) {
-        double run = excl;
-        int tok = -1;
-        for (int v = v0; v < v1; ++v) {
-            run += w(v);
-            if (run > target) {
-                tok = v;
-                break;
+    // C: exactly one segment starts at or below the target and ends above it
+    if (before <= target && before + part > target) {
+        const int piece = (seg / 32 + 3) & ~3;      // consecutive entries per lane
+        const int p0 = min(s1, s0 + lane * piece), p1 = min(s1, p0 + piece);
+        double mine = 0.0;
+        int mylast = -1;
+#pragma unroll 4
+        for (int v = p0; v < p1; ++v) {
+            const float x = w(v);
+            mine += static_cast<double>(x);
+            if (x > 0.f) mylast = v;
+        }
+        double incl = mine;
+#pragma unroll
+        for (int off = 1; off < 32; off <<= 1) {
+            const double o = __shfl_up_sync(kFullMask, incl, off);
+            if (lane >= off) incl += o;
+        }
+        incl += before;
+        const bool cross = (incl - mine) <= target && incl > target;
+        const unsigned who = __ballot_sync(kFullMask, cross);
+        if (who == 0u) {
+            // the scan adds in another order than step A: if its last bit falls short, the crossing is the
+            // segment's last entry with weight
+            if (lane == 0) found[0] = last;
+        } else if (lane == __ffs(who) - 1) {
+            double run = incl - mine;
+            int tok = -1;
+            for (int v = p0; v < p1; ++v) {
+                run += static_cast<double>(w(v));
+                if (run > target) {
+                    tok = v;
+                    break;
+                }
             }
-        }
-        // the re-walk adds in a different order than the scan: if its last bit falls short, the crossing
-        // is the chunk's last entry with weight
-        for (int v = v1 - 1; tok < 0 && v >= v0; --v)
-            if (w(v) > 0.0) tok = v;
-        if (tok >= 0) found[0] = tok;
-    }
-    // fallback for u next to 1: the last index with positive weight
-    int last = -1;
-    for (int v = v1 - 1; v >= v0; --v) {
-        if (w(v) > 0.0) {
-            last = v;
-            break;
+            found[0] = tok >= 0 ? tok : mylast;
         }
     }
-    if (last >= 0) atomicMax(&found[1], last);
     __syncthreads();
     const int tok = found[0] >= 0 ? found[0] : found[1];
     if (total_out) *total_out = total;
@@ -82,17 +105,21 @@ __device__ __forceinline__ int block_sample_cdf(WeightFn w, int V, double u, dou
     return tok;
 }
 
-// Draft side: token[b] drawn from probs[b, :] with u[b]; p_token[b] = its probability.
-// One CTA per sequence; sequences with active[b] == 0 are left untouched.
+// Draft side: the row probs[b, :] arrives holding the raw logits left by the LM-head pass; it is turned
+// into the distribution y = exp(z - m) / Z in place (m, Z from stats[2b], stats[2b + 1]), then token[b]
+// is drawn from it with u[b]; p_token[b] = its probability.  One CTA per sequence; sequences with
+// active[b] == 0 are left untouched.
 static __global__ void __launch_bounds__(kSampleThreads)
-sample_rows_kernel(const float* __restrict__ probs, const float* __restrict__ u, const uint8_t* __restrict__ active,
-                   int V, int32_t* token, float* p_token) {
-    __shared__ double sh[kSampleThreads / 32 + 2];
+sample_rows_kernel(float* __restrict__ probs, const float* __restrict__ stats, const float* __restrict__ u,
+                   const uint8_t* __restrict__ active, int V, int32_t* token, float* p_token) {
+    __shared__ double sh[24];
     const int b = blockIdx.x;
     if (active && !active[b]) return;
-    const float* y = probs + (size_t)b * V;
-    const int tok = block_sample_cdf([&](int v) { return static_cast<double>(__ldcg(y + v)); }, V,
-                                     static_cast<double>(u[b]), sh, nullptr);
+    float* y = probs + (size_t)b * V;
+    const float m = stats[2 * b], inv_Z = 1.f / stats[2 * b + 1];
+    for (int v = threadIdx.x; v < V; v += kSampleThreads) y[v] = __expf(y[v] - m) * inv_Z;
+    __syncthreads();
+    const int tok = block_sample_cdf([&](int v) { return y[v]; }, V, static_cast<double>(u[b]), sh, nullptr);
     if (threadIdx.x == 0) {
         token[b] = tok;
         if (p_token) p_token[b] = tok >= 0 ? y[tok] : 0.f;
@@ -118,7 +145,7 @@ struct SpecSampleParams {
 };
 
 static __global__ void __launch_bounds__(kSampleThreads) speculative_sample_kernel(const SpecSampleParams p) {
-    __shared__ double sh[kSampleThreads / 32 + 2];
+    __shared__ double sh[24];
     __shared__ int s_n;
     const int b = blockIdx.x;
     int r0, r1;
@@ -139,20 +166,20 @@ static __global__ void __launch_bounds__(kSampleThreads) speculative_sample_kern
         return;
     }
     const int sl = r1 - r0 - 1;
-    if (threadIdx.x == 0) {
-        int n = 0;
-        while (n < sl) {
-            const int tok = p.draft_ids[r0 - b + n];
-            if (tok < 0 || tok >= p.V) {
-                record_status(p.status, DISCO_ERR_INVALID_ARG);
-                break;
-            }
-            const double pT = p.y_T[(size_t)(r0 + n) * p.V + tok];
-            const double pD = p.draft_probs[((size_t)n * p.B + b) * p.V + tok];
-            if (!(static_cast<double>(p.u_accept[r0 - b + n]) * pD < pT)) break;
-            ++n;
+    // acceptance tests of all positions side by side (one thread each), then the first that fails
+    if (threadIdx.x == 0) s_n = sl;
+    __syncthreads();
+    for (int i = threadIdx.x; i < sl; i += kSampleThreads) {
+        const int tok = p.draft_ids[r0 - b + i];
+        bool pass = false;
+        if (tok < 0 || tok >= p.V) {
+            record_status(p.status, DISCO_ERR_INVALID_ARG);
+        } else {
+            const double pT = p.y_T[(size_t)(r0 + i) * p.V + tok];
+            const double pD = p.draft_probs[((size_t)i * p.B + b) * p.V + tok];
+            pass = static_cast<double>(p.u_accept[r0 - b + i]) * pD < pT;
         }
-        s_n = n;
+        if (!pass) atomicMin(&s_n, i);
     }
     __syncthreads();
     const int n = s_n;
@@ -162,13 +189,11 @@ static __global__ void __launch_bounds__(kSampleThreads) speculative_sample_kern
     if (n < sl) {
         const float* yD = p.draft_probs + ((size_t)n * p.B + b) * p.V;
         double mass = 0.0;
-        tok = block_sample_cdf(
-            [&](int v) { return fmax(0.0, static_cast<double>(__ldcg(yT + v)) - static_cast<double>(__ldcg(yD + v))); },
-            p.V, us, sh, &mass);
-        if (!(mass > 0.0))
-            tok = block_sample_cdf([&](int v) { return static_cast<double>(__ldcg(yT + v)); }, p.V, us, sh, nullptr);
+        // the residual is rounded to binary32 (relative error 6e-8, far inside what the draw can resolve)
+        tok = block_sample_cdf([&](int v) { return fmaxf(0.f, yT[v] - yD[v]); }, p.V, us, sh, &mass);
+        if (!(mass > 0.0)) tok = block_sample_cdf([&](int v) { return yT[v]; }, p.V, us, sh, nullptr);
     } else {
-        tok = block_sample_cdf([&](int v) { return static_cast<double>(__ldcg(yT + v)); }, p.V, us, sh, nullptr);
+        tok = block_sample_cdf([&](int v) { return yT[v]; }, p.V, us, sh, nullptr);
     }
     if (threadIdx.x == 0) {
         p.n_accept[b] = n;
