@@ -445,6 +445,20 @@ int disco_set_kernel_path(disco_ctx* c, int which) {
 }  // extern "C"
 
 namespace {
+// The sampling kernels stage one row of V floats in dynamic shared memory: raise their limit once per device.
+bool configure_sampling(disco_ctx* c) {
+    static int configured_dev = -1;
+    if (configured_dev == c->device) return true;
+    const int bytes = kSampleSmemFloats * (int)sizeof(float);
+    if (!cuda_ok(cudaFuncSetAttribute(sample_rows_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes),
+                 "cudaFuncSetAttribute(sample_rows)") ||
+        !cuda_ok(cudaFuncSetAttribute(speculative_sample_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes),
+                 "cudaFuncSetAttribute(speculative_sample)"))
+        return false;
+    configured_dev = c->device;
+    return true;
+}
+
 // Shared body of the LM-head + soft-max passes: B rows of hidden size d against the head W.
 //   * nll_sum != null selects the perplexity rule (no classifier; tau is the perplexity bound);
 //   * stats_only: arg-max (token, optional) and soft-max statistics only, no classifier: the target
@@ -569,8 +583,10 @@ int disco_draft_step_sample(disco_ctx* c, const void* W_D, const void* h_D, int 
                                token, conf, halt, feats, probs, nullptr, false, stream, false);
     if (rc) return rc;
     // probs holds the logits: the kernel turns them into y^D and replaces the greedy token by the draw
-    sample_rows_kernel<<<B, kSampleThreads, 0, static_cast<cudaStream_t>(stream)>>>(probs, c->final_stats, u, active,
-                                                                                   c->V, token, p_token);
+    const size_t smem = sample_smem_bytes(c->V);
+    if (!configure_sampling(c)) return DISCO_ERR_CUDA;
+    sample_rows_kernel<<<B, kSampleThreads, smem, static_cast<cudaStream_t>(stream)>>>(
+        probs, c->final_stats, u, active, c->V, smem ? 1 : 0, token, p_token);
     c->launches += 1;
     return cuda_ok(cudaGetLastError(), "sample_rows_kernel launch") ? DISCO_OK : DISCO_ERR_CUDA;
 }
@@ -602,7 +618,10 @@ int disco_verify_sample_ragged(disco_ctx* c, const void* W_T, const void* H_T, c
     sp.next_token = next_token;
     sp.status = c->status;
     if (!row_off && R % B != 0) return DISCO_ERR_INVALID_ARG;
-    speculative_sample_kernel<<<B, kSampleThreads, 0, static_cast<cudaStream_t>(stream)>>>(sp);
+    const size_t smem = sample_smem_bytes(c->V);
+    sp.use_smem = smem ? 1 : 0;
+    if (!configure_sampling(c)) return DISCO_ERR_CUDA;
+    speculative_sample_kernel<<<B, kSampleThreads, smem, static_cast<cudaStream_t>(stream)>>>(sp);
     c->launches += 1;
     return cuda_ok(cudaGetLastError(), "speculative_sample_kernel launch") ? DISCO_OK : DISCO_ERR_CUDA;
 }

@@ -105,21 +105,48 @@ __device__ __forceinline__ int block_sample_cdf(WeightFn w, int V, double u, dou
     return tok;
 }
 
+// Rows of up to kSampleSmemFloats entries are staged in shared memory (one pass over global memory, eight
+// loads in flight per thread); longer rows are read from global memory by every step of the draw.
+constexpr int kSampleSmemFloats = 50 * 1024;
+constexpr int kSampleBatch = 8;
+inline size_t sample_smem_bytes(int V) { return V <= kSampleSmemFloats ? (size_t)V * sizeof(float) : 0; }
+
 // Draft side: the row probs[b, :] arrives holding the raw logits left by the LM-head pass; it is turned
 // into the distribution y = exp(z - m) / Z in place (m, Z from stats[2b], stats[2b + 1]), then token[b]
 // is drawn from it with u[b]; p_token[b] = its probability.  One CTA per sequence; sequences with
-// active[b] == 0 are left untouched.
+// active[b] == 0 are left untouched.  Dynamic shared memory: sample_smem_bytes(V).
 static __global__ void __launch_bounds__(kSampleThreads)
 sample_rows_kernel(float* __restrict__ probs, const float* __restrict__ stats, const float* __restrict__ u,
-                   const uint8_t* __restrict__ active, int V, int32_t* token, float* p_token) {
+                   const uint8_t* __restrict__ active, int V, int use_smem, int32_t* token, float* p_token) {
+    extern __shared__ float row_s[];
     __shared__ double sh[24];
     const int b = blockIdx.x;
     if (active && !active[b]) return;
     float* y = probs + (size_t)b * V;
     const float m = stats[2 * b], inv_Z = 1.f / stats[2 * b + 1];
-    for (int v = threadIdx.x; v < V; v += kSampleThreads) y[v] = __expf(y[v] - m) * inv_Z;
+    for (int v0 = threadIdx.x; v0 < V; v0 += kSampleBatch * kSampleThreads) {
+        float z[kSampleBatch];
+#pragma unroll
+        for (int k = 0; k < kSampleBatch; ++k) {
+            const int v = v0 + k * kSampleThreads;
+            z[k] = v < V ? __ldcg(y + v) : 0.f;
+        }
+#pragma unroll
+        for (int k = 0; k < kSampleBatch; ++k) {
+            const int v = v0 + k * kSampleThreads;
+            if (v < V) {
+                const float pv = __expf(z[k] - m) * inv_Z;
+                y[v] = pv;
+                if (use_smem) row_s[v] = pv;
+            }
+        }
+    }
     __syncthreads();
-    const int tok = block_sample_cdf([&](int v) { return y[v]; }, V, static_cast<double>(u[b]), sh, nullptr);
+    int tok;
+    if (use_smem)
+        tok = block_sample_cdf([&](int v) { return row_s[v]; }, V, static_cast<double>(u[b]), sh, nullptr);
+    else
+        tok = block_sample_cdf([&](int v) { return y[v]; }, V, static_cast<double>(u[b]), sh, nullptr);
     if (threadIdx.x == 0) {
         token[b] = tok;
         if (p_token) p_token[b] = tok >= 0 ? y[tok] : 0.f;
@@ -130,7 +157,7 @@ sample_rows_kernel(float* __restrict__ probs, const float* __restrict__ stats, c
 // sequence (SL + 1 of them); draft token i was drawn from draft_probs[(i * B + b), :].  Token i is
 // accepted iff u_accept * y_D(t_i) < y_T(t_i); n = number accepted before the first rejection.  The next
 // token is drawn with u_sample[b] from norm(max(0, y_T[n] - y_D[n])) after a rejection, from y_T[SL]
-// otherwise; a residual without mass falls back to y_T[n].
+// otherwise; a residual without mass falls back to y_T[n].  Dynamic shared memory: sample_smem_bytes(V).
 struct SpecSampleParams {
     const float* y_T;          // [R, V]
     const float* draft_probs;  // [steps, B, V]
@@ -139,12 +166,14 @@ struct SpecSampleParams {
     const float* u_accept;     // [R - B]
     const float* u_sample;     // [B]
     int B, SL, R, V;
+    int use_smem;
     int32_t* n_accept;
     int32_t* next_token;
     int* status;
 };
 
 static __global__ void __launch_bounds__(kSampleThreads) speculative_sample_kernel(const SpecSampleParams p) {
+    extern __shared__ float row_s[];
     __shared__ double sh[24];
     __shared__ int s_n;
     const int b = blockIdx.x;
@@ -184,17 +213,37 @@ static __global__ void __launch_bounds__(kSampleThreads) speculative_sample_kern
     __syncthreads();
     const int n = s_n;
     const float* yT = p.y_T + (size_t)(r0 + n) * p.V;
+    const float* yD = n < sl ? p.draft_probs + ((size_t)n * p.B + b) * p.V : nullptr;
     const double us = static_cast<double>(p.u_sample[b]);
-    int tok;
-    if (n < sl) {
-        const float* yD = p.draft_probs + ((size_t)n * p.B + b) * p.V;
-        double mass = 0.0;
-        // the residual is rounded to binary32 (relative error 6e-8, far inside what the draw can resolve)
-        tok = block_sample_cdf([&](int v) { return fmaxf(0.f, yT[v] - yD[v]); }, p.V, us, sh, &mass);
-        if (!(mass > 0.0)) tok = block_sample_cdf([&](int v) { return yT[v]; }, p.V, us, sh, nullptr);
-    } else {
-        tok = block_sample_cdf([&](int v) { return yT[v]; }, p.V, us, sh, nullptr);
+    const int V = p.V;
+    // weights of the draw: the residual max(0, y_T - y_D) after a rejection, y_T itself otherwise.  The
+    // residual is rounded to binary32 (relative error 6e-8, far inside what the draw can resolve).
+    if (p.use_smem) {
+        for (int v0 = threadIdx.x; v0 < V; v0 += kSampleBatch * kSampleThreads) {
+            float a[kSampleBatch], d[kSampleBatch];
+#pragma unroll
+            for (int k = 0; k < kSampleBatch; ++k) {
+                const int v = v0 + k * kSampleThreads;
+                a[k] = v < V ? __ldcg(yT + v) : 0.f;
+                d[k] = (yD && v < V) ? __ldcg(yD + v) : 0.f;
+            }
+#pragma unroll
+            for (int k = 0; k < kSampleBatch; ++k) {
+                const int v = v0 + k * kSampleThreads;
+                if (v < V) row_s[v] = yD ? fmaxf(0.f, a[k] - d[k]) : a[k];
+            }
+        }
+        __syncthreads();
     }
+    int tok;
+    double mass = 0.0;
+    if (p.use_smem)
+        tok = block_sample_cdf([&](int v) { return row_s[v]; }, V, us, sh, &mass);
+    else if (yD)
+        tok = block_sample_cdf([&](int v) { return fmaxf(0.f, yT[v] - yD[v]); }, V, us, sh, &mass);
+    else
+        tok = block_sample_cdf([&](int v) { return yT[v]; }, V, us, sh, &mass);
+    if (yD && !(mass > 0.0)) tok = block_sample_cdf([&](int v) { return yT[v]; }, V, us, sh, nullptr);
     if (threadIdx.x == 0) {
         p.n_accept[b] = n;
         p.next_token[b] = tok;
