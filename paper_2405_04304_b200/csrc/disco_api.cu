@@ -490,11 +490,6 @@ int draft_step_common(disco_ctx* c, const void* W_D, const void* h_D, int d, int
     p.R = B;
     p.B = B;
     fill_scratch(c, p);
-    // Stamped records (no fence before the ticket) when the stamped buffer holds a record per row and CTA
-    if (getenv_int("DISCO_STAMPED", 1) && (size_t)B * std::max(c->max_grid, c->sm_count) <= (size_t)128 * c->sm_count) {
-        p.epoch = c->ticket + 48;
-        p.stamped_rec = reinterpret_cast<float4*>(c->stamped_rec);
-    }
     p.stats_only = stats_only ? 1 : 0;
     p.pos = pos;
     p.n_drafted = n_drafted;

@@ -57,10 +57,6 @@ struct TailParams {
     float* probs;
     float* nll_sum;      // non-null: perplexity rule instead of the classifier (tau is then the perplexity bound)
     int stats_only;      // non-zero: arg-max and soft-max statistics only; pos, n_drafted and the classifier are unused
-    // draft step with stamped records (non-null epoch): the CTAs' records go to stamped_rec, 80 bytes each,
-    // and no fence precedes the ticket; epoch[0] counts completed launches (stamp = that + 1)
-    unsigned int* epoch;
-    float4* stamped_rec;
     // verification
     const int32_t* draft_ids;
     const int32_t* row_off;  // null: uniform SL
@@ -236,14 +232,6 @@ __device__ __forceinline__ void store_stamped_record(float4* rec, float m, float
     store_relaxed_v4(rec + 3, l[6], l[7], l[8], sf);
     store_relaxed_v4(rec + 4, l[9], __uint_as_float(static_cast<uint32_t>(key & 0xffffffffull)),
                      __uint_as_float(static_cast<uint32_t>(key >> 32)), sf);
-}
-
-// The reduced record that lane 0 holds, as a stamped record.
-__device__ __forceinline__ void warp_store_stamped(float4* rec, const LaneRecord& r, uint32_t stamp, int lane) {
-    if (lane == 0) {
-        const float l[kTopK] = {r.l[0], r.l[1], r.l[2], r.l[3], r.l[4], r.l[5], r.l[6], r.l[7], r.l[8], r.l[9]};
-        store_stamped_record(rec, r.m, r.Z, r.S, l, r.key, stamp);
-    }
 }
 
 // Merge the NP partial records of one sequence (consecutive) by one warp.
@@ -588,13 +576,10 @@ __device__ __forceinline__ void warp_draft_epilogue(const SoftmaxState& st, unsi
 // per-CTA records, then features, classifier and stopping rule.
 // feat16: kWarpScratchWords words of shared memory owned by the calling warp.
 __device__ __forceinline__ void finalize_draft_seq(const TailParams& p, int b, int grid, float* feat16, const float* clf_s,
-                                                   int lane, uint32_t stamp = 0u) {
+                                                   int lane) {
     const float fpos = p.pos ? static_cast<float>(p.pos[b]) : 0.f;  // issued early: hidden behind the merge
     const int n_drafted = p.n_drafted ? p.n_drafted[b] : 0;
-    const MergedPartials mp =
-        stamp ? warp_merge_partials(p.stamped_rec + (size_t)b * grid * kStampedPieces, grid, feat16 + 16, lane, stamp,
-                                    p.status)
-              : warp_merge_partials(p.part_rec + (size_t)b * grid * 4, grid, feat16 + 16, lane);
+    const MergedPartials mp = warp_merge_partials(p.part_rec + (size_t)b * grid * 4, grid, feat16 + 16, lane);
     const int Hc = p.clf_H;
     const SoftmaxState st = mp.st;
     const DraftOutputs o{p.token, p.conf, p.halt, p.feats, p.final_stats, p.nll_sum, p.stats_only};
@@ -728,8 +713,6 @@ __global__ void __launch_bounds__((NW + 1) * 32, 1) stream_tail_kernel(const __g
     // from here on the kernel reads the hidden states and writes scratch and outputs: the preceding
     // kernel of the stream must have finished
     asm volatile("griddepcontrol.wait;" ::: "memory");
-    // stamped records: the stamp of this launch (the word is advanced by the last CTA at its end)
-    const uint32_t stamp = (DRAFT && p.epoch) ? *reinterpret_cast<volatile unsigned int*>(p.epoch) + 1u : 0u;
 
     const int n16 = (int)(row_bytes >> 4);  // 16-byte pieces per row
     for (int chunk = 0; chunk < nchunks; ++chunk) {
@@ -886,10 +869,7 @@ __global__ void __launch_bounds__((NW + 1) * 32, 1) stream_tail_kernel(const __g
                     rec.set(sr[0], sr[1], sr[2], sr[3]);
                 }
                 warp_reduce_records(rec, ceil_log2(NW));
-                if (stamp)
-                    warp_store_stamped(p.stamped_rec + ((size_t)row * grid + blockIdx.x) * kStampedPieces, rec, stamp, lane);
-                else
-                    warp_store_record(reinterpret_cast<float*>(p.part_rec + ((size_t)row * grid + blockIdx.x) * 4), rec, lane);
+                warp_store_record(reinterpret_cast<float*>(p.part_rec + ((size_t)row * grid + blockIdx.x) * 4), rec, lane);
             }
         } else {
             unsigned long long* keys_s = reinterpret_cast<unsigned long long*>(wstate);
@@ -907,9 +887,7 @@ __global__ void __launch_bounds__((NW + 1) * 32, 1) stream_tail_kernel(const __g
     }
 
     // -------------------- ticket: the last CTA runs the fused epilogue --------------------
-    // Stamped records need no fence: the barrier below orders every warp's record stores before the
-    // ticket is taken, and the last CTA polls the records until they carry this launch's stamp.
-    if (!stamp) __threadfence();
+    __threadfence();
     named_barrier_sync(1, BAR_THREADS);
     if (tid == 0) {
         const unsigned t = atomicAdd(p.ticket, 1u);
@@ -918,16 +896,15 @@ __global__ void __launch_bounds__((NW + 1) * 32, 1) stream_tail_kernel(const __g
     named_barrier_sync(1, BAR_THREADS);
     if (DRAFT) cp_async_wait_all();
     if (!s_is_last) return;
-    if (!stamp) __threadfence();
+    __threadfence();
 
     if (DRAFT) {
         named_barrier_sync(1, BAR_THREADS);
         for (int b = warp; b < p.R; b += NW) {
             if (p.active && !p.active[b]) continue;
-            finalize_draft_seq(p, b, grid, feat_s + warp * kWarpScratchWords, clf_s, lane, stamp);
+            finalize_draft_seq(p, b, grid, feat_s + warp * kWarpScratchWords, clf_s, lane);
         }
         named_barrier_sync(1, BAR_THREADS);
-        if (stamp && tid == 0) *p.epoch = stamp == 0xffffffffu ? 0u : stamp;   // the stamp is never zero
     } else {
         for (int b = warp; b < p.B; b += NW)
             verify_one_sequence(p.keys, p.draft_ids, p.row_off, p.B, p.SL, p.R, b, p.n_accept, p.bonus,

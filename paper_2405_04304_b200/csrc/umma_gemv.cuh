@@ -190,8 +190,6 @@ umma_gemv_draft_kernel(const __grid_constant__ CUtensorMap tmap_W, const __grid_
             cp_async_commit();
         }
         asm volatile("griddepcontrol.wait;" ::: "memory");  // scratch and outputs belong to the predecessor until now
-        // stamped records: the stamp of this launch (the word is advanced by the last CTA at its end)
-        const uint32_t stamp = p.epoch ? *reinterpret_cast<volatile unsigned int*>(p.epoch) + 1u : 0u;
 
         SoftmaxState st[RK];
         float top_v[RK], best_v[RK];
@@ -245,32 +243,23 @@ umma_gemv_draft_kernel(const __grid_constant__ CUtensorMap tmap_W, const __grid_
                 rec.set(sr[0], sr[1], sr[2], sr[3]);
             }
             warp_reduce_records(rec, 2);
-            if (stamp)
-                warp_store_stamped(p.stamped_rec + ((size_t)r * grid + blockIdx.x) * kStampedPieces, rec, stamp, lane);
-            else
-                warp_store_record(reinterpret_cast<float*>(p.part_rec + ((size_t)r * grid + blockIdx.x) * 4), rec, lane);
+            warp_store_record(reinterpret_cast<float*>(p.part_rec + ((size_t)r * grid + blockIdx.x) * 4), rec, lane);
         }
 
         // ---- ticket: the last CTA reduces the records of all CTAs and runs the fused epilogue ----
-        // Stamped records need no fence: the barrier orders every warp's record stores before the ticket
-        // is taken, and the last CTA polls the records until they carry this launch's stamp.
-        if (!stamp) __threadfence();
+        __threadfence();
         named_barrier_sync(1, BAR_THREADS);
         if (tid == 0) s_is_last = atomicAdd(p.ticket, 1u) == (unsigned)grid - 1u;
         named_barrier_sync(1, BAR_THREADS);
         cp_async_wait_all();
         if (s_is_last) {
-            if (!stamp) __threadfence();
+            __threadfence();
             named_barrier_sync(1, BAR_THREADS);
             for (int b = ew; b < p.R; b += kGemvEpiWarps) {
                 if (p.active && !p.active[b]) continue;
-                finalize_draft_seq(p, b, grid, feat_s + ew * kWarpScratchWords, clf_s, lane, stamp);
+                finalize_draft_seq(p, b, grid, feat_s + ew * kWarpScratchWords, clf_s, lane);
             }
-            if (stamp) named_barrier_sync(1, BAR_THREADS);
-            if (tid == 0) {
-                *p.ticket = 0u;
-                if (stamp) *p.epoch = stamp == 0xffffffffu ? 0u : stamp;   // the stamp is never zero
-            }
+            if (tid == 0) *p.ticket = 0u;
         }
     }
 
