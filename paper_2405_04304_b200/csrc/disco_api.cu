@@ -258,16 +258,22 @@ template <int RK>
 int launch_gemv_rk(disco_ctx* c, GemvParams& g, const CUtensorMap& mW, const CUtensorMap& mWt, const CUtensorMap& mH,
                    cudaStream_t st) {
     auto kern = umma_gemv_draft_kernel<RK>;
-    const size_t smem = gemv_smem_bytes(RK, g.t.clf_H);
     static int configured_dev = -1;
-    static size_t configured_smem = 0;
-    if (configured_dev != c->device || configured_smem < smem) {
-        if (!cuda_ok(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem),
+    static size_t dyn_limit = 0;
+    if (configured_dev != c->device) {
+        cudaFuncAttributes fa;
+        if (!cuda_ok(cudaFuncGetAttributes(&fa, kern), "cudaFuncGetAttributes(gemv)")) return DISCO_ERR_CUDA;
+        dyn_limit = c->smem_optin - fa.sharedSizeBytes;
+        if (!cuda_ok(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn_limit),
                      "cudaFuncSetAttribute(gemv)"))
             return DISCO_ERR_CUDA;
         configured_dev = c->device;
-        configured_smem = smem;
     }
+    // the ring takes what the fixed part leaves: as many 16 KB stages as fit
+    const size_t fixed = gemv_fixed_smem_bytes(RK, g.t.clf_H, g.t.d, g.h_rows);
+    if (dyn_limit < fixed + 2 * (size_t)kGemvATile) return DISCO_ERR_UNSUPPORTED_SHAPE;
+    g.stages = (int)std::min<size_t>(kGemvMaxStages, (dyn_limit - fixed) / kGemvATile);
+    const size_t smem = gemv_smem_bytes(RK, g.t.clf_H, g.t.d, g.h_rows, g.stages);
     cudaLaunchConfig_t cfg{};
     cfg.gridDim = dim3((unsigned)c->sm_count);
     cfg.blockDim = dim3(kGemvThreads);
@@ -510,7 +516,9 @@ int draft_step_common(disco_ctx* c, const void* W_D, const void* h_D, int d, int
     // Measured on B200 (Vicuna head): up to 6 sequences are fastest on the tensor-core kernel with the
     // vocabulary on the TMEM lanes, more on the one with the hidden rows on the lanes; the CUDA-core
     // streaming kernel is within 10 % for one sequence and serves as the path without tensor maps.
-    const bool gemv_ok = c->encode_tiled != nullptr && B <= kGemvMaxRows && !stats_only;
+    // (its hidden rows stay in shared memory: up to 48 KB of them, so that the ring keeps at least 8 stages)
+    const bool gemv_ok = c->encode_tiled != nullptr && B <= kGemvMaxRows && !stats_only &&
+                         (size_t)((d + kUmmaBK - 1) / kUmmaBK) * (B <= 8 ? 8 : 16) * 128 <= 48 * 1024;
     const bool use_gemv = gemv_ok && (c->path == 3 || (c->path == 0 && B <= 6));
     const bool use_umma = !use_gemv && umma_possible(c, B) && (c->path == 2 || c->path == 3 || (c->path == 0 && B >= 2));
     if (use_gemv) {

@@ -12,8 +12,12 @@
 //
 //   * one CTA per SM and slab of ceil(V / #SM) vocabulary rows, cut into tiles of 128 rows (the last
 //     one shorter: its own TMA box, so nothing beyond the slab is fetched);
-//   * warp 0 producer (TMA, 128-byte swizzle, ring of 18 KB stages), warp 1 MMA issuer (M = 128,
-//     N = 16, K = 16, two 16-column TMEM buffers), warps 2-5 epilogue (one TMEM lane quadrant each);
+//   * warp 0 producer (TMA, 128-byte swizzle, ring of 16 KB stages for the LM head; the hidden rows are
+//     loaded once, after the dependency wait, and stay), warp 1 MMA issuer (M = 128, N = 16, K = 16, two
+//     16-column TMEM buffers), warps 2-5 epilogue (one TMEM lane quadrant each);
+//   * the ring is as deep as shared memory allows (12 stages = one whole tile of the 768-wide heads) and
+//     is filled before the dependency wait, so that after the wait the first tile needs nothing but the
+//     hidden rows;
 //   * per-CTA records, ticket, last-CTA reduction and classifier exactly as in the streaming kernel.
 #pragma once
 
@@ -25,25 +29,31 @@ constexpr int kGemvEpiWarps = 4;
 constexpr int kGemvThreads = (2 + kGemvEpiWarps) * 32;
 constexpr int kGemvMaxRows = 16;
 constexpr int kGemvATile = 128 * 128;   // 128 vocabulary rows x 128 B
-constexpr int kGemvBTile = 16 * 128;    // 16 hidden rows x 128 B
-constexpr int kGemvStages = 10;
-constexpr int kGemvRing = kGemvStages * (kGemvATile + kGemvBTile);
+constexpr int kGemvMaxStages = 16;
 
 struct GemvParams {
     TailParams t;     // V, d, R and everything the fused epilogue needs (scratch, classifier, outputs)
     int TR;           // vocabulary rows per CTA
     int tiles;        // ceil(TR / 128)
     int tail_rows;    // rows of the last tile's TMA box (multiple of 8)
-    int h_rows;       // rows of the hidden-state box (multiple of 8, <= 16)
+    int h_rows;       // rows of the hidden-state box (8 or 16)
+    int stages;       // ring depth (2 .. kGemvMaxStages)
 };
 
-inline size_t gemv_smem_bytes(int RK, int clf_H) {
-    size_t b = kGemvRing + 1024;                                 // operand ring (+ alignment)
+// Shared memory besides the ring: the resident hidden rows (one k-block of h_rows x 128 B per 64 hidden
+// units; the MMA reads 16 rows from each, the surplus lands in columns nobody reads), barriers, records,
+// second-phase scratch, classifier.
+inline size_t gemv_fixed_smem_bytes(int RK, int clf_H, int d, int h_rows) {
+    size_t b = 1024;                                             // alignment
+    b += (size_t)((d + kUmmaBK - 1) / kUmmaBK) * h_rows * 128 + 1024;  // hidden rows (+ the 16-row overhang)
     b += 512;                                                    // barriers, TMEM address
     b += (size_t)(kGemvEpiWarps * RK + 1) * kRecordWords * 4;    // warp records / finalize staging
     b += kGemvEpiWarps * kWarpScratchWords * 4;                  // second-phase scratch per warp
     b += ((size_t)clf_H * (kNFeat + 2) + 4) * 4;                 // classifier parameters
     return b + 128;
+}
+inline size_t gemv_smem_bytes(int RK, int clf_H, int d, int h_rows, int stages) {
+    return gemv_fixed_smem_bytes(RK, clf_H, d, h_rows) + (size_t)stages * kGemvATile;
 }
 
 __device__ __forceinline__ void tmem_ld16(uint32_t taddr, float (&v)[16]) {
@@ -68,14 +78,18 @@ umma_gemv_draft_kernel(const __grid_constant__ CUtensorMap tmap_W, const __grid_
     extern __shared__ uint8_t smem_dyn[];
     const TailParams& p = g.t;
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~uintptr_t(1023));
+    const int KBs = (p.d + kUmmaBK - 1) / kUmmaBK;
+    const int b_stride = g.h_rows * 128;   // bytes between the k-blocks of the resident hidden rows
     uint8_t* a_tiles = smem;
-    uint8_t* b_tiles = smem + kGemvStages * kGemvATile;
-    uint64_t* full = reinterpret_cast<uint64_t*>(smem + kGemvRing);
-    uint64_t* empty = full + kGemvStages;
-    uint64_t* tmem_full = empty + kGemvStages;
+    uint8_t* b_tiles = smem + g.stages * kGemvATile;
+    uint8_t* after_b = b_tiles + KBs * b_stride + 1024;
+    uint64_t* full = reinterpret_cast<uint64_t*>(after_b);
+    uint64_t* empty = full + kGemvMaxStages;
+    uint64_t* tmem_full = empty + kGemvMaxStages;
     uint64_t* tmem_empty = tmem_full + 2;
-    uint32_t* tmem_base_s = reinterpret_cast<uint32_t*>(tmem_empty + 2);
-    float* wstate = reinterpret_cast<float*>(smem + kGemvRing + 512);
+    uint64_t* h_full = tmem_empty + 2;
+    uint32_t* tmem_base_s = reinterpret_cast<uint32_t*>(h_full + 1);
+    float* wstate = reinterpret_cast<float*>(after_b + 512);
     float* feat_s = wstate + (kGemvEpiWarps * RK + 1) * kRecordWords;
     float* clf_s = feat_s + kGemvEpiWarps * kWarpScratchWords;
     __shared__ int s_is_last;
@@ -91,10 +105,11 @@ umma_gemv_draft_kernel(const __grid_constant__ CUtensorMap tmap_W, const __grid_
     const int tiles = v_begin < p.V ? g.tiles : 0;
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < kGemvStages; ++s) {
+        for (int s = 0; s < g.stages; ++s) {
             mbar_init(&full[s], 1);
             mbar_init(&empty[s], 1);
         }
+        mbar_init(h_full, 1);
         for (int b = 0; b < 2; ++b) {
             mbar_init(&tmem_full[b], 1);
             mbar_init(&tmem_empty[b], kGemvEpiWarps);
@@ -117,29 +132,30 @@ umma_gemv_draft_kernel(const __grid_constant__ CUtensorMap tmap_W, const __grid_
         // ------------------------------ producer ------------------------------
         if (lane == 0) {
             const int total = tiles * KB;
-            const uint32_t h_bytes = (uint32_t)g.h_rows * 128u;
-            // the LM head does not depend on the preceding kernel: its first tiles are requested at once
-            const int pre = min(kGemvStages, total);
+            // the LM head does not depend on the preceding kernel: the whole ring is requested at once
+            const int pre = min(g.stages, total);
             for (int n = 0; n < pre; ++n) {
                 const int tile = n / KB, kb = n - tile * KB;
                 const bool last = tile == g.tiles - 1;
-                mbar_arrive_expect_tx(&full[n], (uint32_t)(last ? g.tail_rows : 128) * 128u + h_bytes);
+                mbar_arrive_expect_tx(&full[n], (uint32_t)(last ? g.tail_rows : 128) * 128u);
                 tma_load_2d(a_tiles + n * kGemvATile, last ? &tmap_Wtail : &tmap_W, kb * kUmmaBK, v_begin + tile * 128,
                             &full[n]);
             }
             asm volatile("griddepcontrol.wait;" ::: "memory");
-            int stage = 0, phase = 0;
-            for (int n = 0; n < total; ++n) {
+            // the hidden rows, all k-blocks on one barrier; they stay for the whole kernel
+            if (total > 0) {
+                mbar_arrive_expect_tx(h_full, (uint32_t)(KB * b_stride));
+                for (int kb = 0; kb < KB; ++kb) tma_load_2d(b_tiles + kb * b_stride, &tmap_H, kb * kUmmaBK, 0, h_full);
+            }
+            int stage = pre == g.stages ? 0 : pre, phase = pre == g.stages ? 1 : 0;
+            for (int n = pre; n < total; ++n) {
                 const int tile = n / KB, kb = n - tile * KB;
-                if (n >= pre) {
-                    const bool last = tile == g.tiles - 1;
-                    mbar_wait(&empty[stage], phase ^ 1, p.status);
-                    mbar_arrive_expect_tx(&full[stage], (uint32_t)(last ? g.tail_rows : 128) * 128u + h_bytes);
-                    tma_load_2d(a_tiles + stage * kGemvATile, last ? &tmap_Wtail : &tmap_W, kb * kUmmaBK,
-                                v_begin + tile * 128, &full[stage]);
-                }
-                tma_load_2d(b_tiles + stage * kGemvBTile, &tmap_H, kb * kUmmaBK, 0, &full[stage]);
-                if (++stage == kGemvStages) {
+                const bool last = tile == g.tiles - 1;
+                mbar_wait(&empty[stage], phase ^ 1, p.status);
+                mbar_arrive_expect_tx(&full[stage], (uint32_t)(last ? g.tail_rows : 128) * 128u);
+                tma_load_2d(a_tiles + stage * kGemvATile, last ? &tmap_Wtail : &tmap_W, kb * kUmmaBK,
+                            v_begin + tile * 128, &full[stage]);
+                if (++stage == g.stages) {
                     stage = 0;
                     phase ^= 1;
                 }
@@ -150,6 +166,10 @@ umma_gemv_draft_kernel(const __grid_constant__ CUtensorMap tmap_W, const __grid_
         if (lane == 0) {
             int stage = 0, phase = 0;
             const uint32_t idesc = umma_idesc(16);
+            if (tiles > 0) {
+                mbar_wait(h_full, 0, p.status);
+                tc_fence_after();
+            }
             for (int tile = 0; tile < tiles; ++tile) {
                 const int buf = tile & 1;
                 mbar_wait(&tmem_empty[buf], ((tile >> 1) & 1) ^ 1, p.status);
@@ -159,12 +179,12 @@ umma_gemv_draft_kernel(const __grid_constant__ CUtensorMap tmap_W, const __grid_
                     mbar_wait(&full[stage], phase, p.status);
                     tc_fence_after();
                     const uint64_t a_desc = umma_smem_desc(a_tiles + stage * kGemvATile);
-                    const uint64_t b_desc = umma_smem_desc(b_tiles + stage * kGemvBTile);
+                    const uint64_t b_desc = umma_smem_desc(b_tiles + kb * b_stride);
 #pragma unroll
                     for (int k = 0; k < kUmmaBK / 16; ++k)
                         tc_mma_bf16(d_tmem, a_desc + 2 * k, b_desc + 2 * k, idesc, (kb | k) != 0);
                     tc_commit(&empty[stage]);
-                    if (++stage == kGemvStages) {
+                    if (++stage == g.stages) {
                         stage = 0;
                         phase ^= 1;
                     }
