@@ -179,7 +179,7 @@ bool umma_possible(const disco_ctx* c, int R) {
 }
 
 // Launch the tcgen05 kernel for R hidden rows of width d against the LM head W [V, d].
-template <bool DRAFT>
+template <bool DRAFT, bool STATS = false>
 int launch_umma(disco_ctx* c, const void* W, const void* H, int d, int R, float* probs,
                 const DraftFinalParams* draft_final, const UmmaParams* fused, cudaStream_t st) {
     UmmaParams p{};
@@ -216,7 +216,7 @@ int launch_umma(disco_ctx* c, const void* W, const void* H, int d, int R, float*
     CUtensorMap tmap_W, tmap_H;
     if (!encode_bf16_2d(c, &tmap_W, W, c->V, d, p.TRN) || !encode_bf16_2d(c, &tmap_H, H, R, d, p.a_rows))
         return DISCO_ERR_CUDA;
-    auto kern = umma_tail_kernel<DRAFT>;
+    auto kern = umma_tail_kernel<DRAFT, STATS>;
     static int configured_dev = -1;
     if (configured_dev != c->device) {
         if (!cuda_ok(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -545,7 +545,8 @@ int draft_step_common(disco_ctx* c, const void* W_D, const void* h_D, int d, int
         f.nll_sum = nll_sum;
         f.stats_only = stats_only ? 1 : 0;
         f.epoch = c->ticket + 48;
-        rc = launch_umma<true>(c, W_D, h_D, d, B, probs, &f, nullptr, st);
+        rc = stats_only ? launch_umma<true, true>(c, W_D, h_D, d, B, probs, &f, nullptr, st)
+                        : launch_umma<true>(c, W_D, h_D, d, B, probs, &f, nullptr, st);
         if (rc) return rc;
     } else {
         rc = run_stream<true>(c, p, clf->H, st);

@@ -184,7 +184,10 @@ __device__ __forceinline__ void umma_finish_sequence(const DraftFinalParams& p, 
 // ---------------------------------------------------------------------------------------------
 // main kernel
 // ---------------------------------------------------------------------------------------------
-template <bool DRAFT>
+// DRAFT: soft-max statistics, top-10 and arg-max per row (draft step) instead of the arg-max alone
+// (verification).  STATS (with DRAFT): no top-10 -- the target rows of a verification with sampling, whose
+// second phase wants the statistics and the arg-max only.
+template <bool DRAFT, bool STATS = false>
 __global__ void __launch_bounds__(kUmmaThreads, 1)
 umma_tail_kernel(const __grid_constant__ CUtensorMap tmap_W, const __grid_constant__ CUtensorMap tmap_H,
                  const UmmaParams p, const DraftFinalParams f) {
@@ -372,16 +375,23 @@ umma_tail_kernel(const __grid_constant__ CUtensorMap tmap_W, const __grid_consta
                             const float e = __expf(t);
                             st.Z += e;
                             st.S = (cbase + j < ncols) ? fmaf(e, t, st.S) : st.S;
-                            top.push(z[j]);
+                            if (!STATS) top.push(z[j]);
                             if (z[j] > best_v) {
                                 best_v = z[j];
                                 best_i = v0 + cbase + j;
                             }
                         }
                         if (p.probs && valid) {
+                            float* dst = p.probs + (size_t)row * p.V + v0 + cbase;
+                            if ((((uintptr_t)p.probs & 15) | ((p.V | (v0 + cbase)) & 3)) == 0 && cbase + 32 <= ncols) {  // 16-byte stores
 #pragma unroll
-                            for (int j = 0; j < 32; ++j)
-                                if (cbase + j < ncols) p.probs[(size_t)row * p.V + v0 + cbase + j] = z[j];
+                                for (int j = 0; j < 32; j += 4)
+                                    *reinterpret_cast<float4*>(dst + j) = make_float4(z[j], z[j + 1], z[j + 2], z[j + 3]);
+                            } else {
+#pragma unroll
+                                for (int j = 0; j < 32; ++j)
+                                    if (cbase + j < ncols) dst[j] = z[j];
+                            }
                         }
                     } else {
 #pragma unroll
