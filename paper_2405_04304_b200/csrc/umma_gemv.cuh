@@ -18,6 +18,9 @@
 //   * the ring is as deep as shared memory allows (12 stages = one whole tile of the 768-wide heads) and
 //     is filled before the dependency wait, so that after the wait the first tile needs nothing but the
 //     hidden rows;
+//   * MMAs into one accumulator form a dependent chain (about 130 cycles each, measured), and a tile of a
+//     768-wide head would be 48 of them: the four K = 16 steps of a k-block go to four accumulators
+//     instead (16 TMEM columns each), which the epilogue adds up;
 //   * per-CTA records, ticket, last-CTA reduction and classifier exactly as in the streaming kernel.
 #pragma once
 
@@ -30,6 +33,8 @@ constexpr int kGemvThreads = (2 + kGemvEpiWarps) * 32;
 constexpr int kGemvMaxRows = 16;
 constexpr int kGemvATile = 128 * 128;   // 128 vocabulary rows x 128 B
 constexpr int kGemvMaxStages = 16;
+constexpr int kGemvAcc = kUmmaBK / 16;          // independent accumulators per TMEM buffer (4)
+constexpr int kGemvBufCols = kGemvAcc * 16;     // TMEM columns per buffer
 
 struct GemvParams {
     TailParams t;     // V, d, R and everything the fused epilogue needs (scratch, classifier, outputs)
@@ -120,7 +125,7 @@ umma_gemv_draft_kernel(const __grid_constant__ CUtensorMap tmap_W, const __grid_
         prefetch_tensormap(&tmap_H);
     }
     if (warp == 1) {
-        tmem_alloc(tmem_base_s, 32);
+        tmem_alloc(tmem_base_s, 2 * kGemvBufCols);
         tmem_relinquish();
     }
     tc_fence_before();
@@ -174,15 +179,15 @@ umma_gemv_draft_kernel(const __grid_constant__ CUtensorMap tmap_W, const __grid_
                 const int buf = tile & 1;
                 mbar_wait(&tmem_empty[buf], ((tile >> 1) & 1) ^ 1, p.status);
                 tc_fence_after();
-                const uint32_t d_tmem = tmem_base + buf * 16;
+                const uint32_t d_tmem = tmem_base + buf * kGemvBufCols;
                 for (int kb = 0; kb < KB; ++kb) {
                     mbar_wait(&full[stage], phase, p.status);
                     tc_fence_after();
                     const uint64_t a_desc = umma_smem_desc(a_tiles + stage * kGemvATile);
                     const uint64_t b_desc = umma_smem_desc(b_tiles + kb * b_stride);
 #pragma unroll
-                    for (int k = 0; k < kUmmaBK / 16; ++k)
-                        tc_mma_bf16(d_tmem, a_desc + 2 * k, b_desc + 2 * k, idesc, (kb | k) != 0);
+                    for (int k = 0; k < kGemvAcc; ++k)  // step k of every k-block accumulates into accumulator k
+                        tc_mma_bf16(d_tmem + k * 16, a_desc + 2 * k, b_desc + 2 * k, idesc, kb != 0);
                     tc_commit(&empty[stage]);
                     if (++stage == g.stages) {
                         stage = 0;
@@ -230,7 +235,14 @@ umma_gemv_draft_kernel(const __grid_constant__ CUtensorMap tmap_W, const __grid_
             const int v_lane0 = v_begin + tile * 128 + quad * 32;  // vocabulary row of lane 0 of this warp
             const int n = max(0, min(32, v_end - v_lane0));        // rows of the slab in this warp's quadrant
             float z[16];
-            tmem_ld16(tmem_base + buf * 16 + (static_cast<uint32_t>(quad * 32) << 16), z);
+            tmem_ld16(tmem_base + buf * kGemvBufCols + (static_cast<uint32_t>(quad * 32) << 16), z);
+#pragma unroll
+            for (int a = 1; a < kGemvAcc; ++a) {
+                float za[16];
+                tmem_ld16(tmem_base + buf * kGemvBufCols + a * 16 + (static_cast<uint32_t>(quad * 32) << 16), za);
+#pragma unroll
+                for (int r = 0; r < 16; ++r) z[r] += za[r];
+            }
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(&tmem_empty[buf]);  // the values are in registers: the buffer is free
@@ -287,7 +299,7 @@ umma_gemv_draft_kernel(const __grid_constant__ CUtensorMap tmap_W, const __grid_
     __syncthreads();
     if (warp == 1) {
         tc_fence_after();
-        tmem_dealloc(tmem_base, 32);
+        tmem_dealloc(tmem_base, 2 * kGemvBufCols);
     }
 }
 
