@@ -255,8 +255,7 @@ int launch_umma(disco_ctx* c, const void* W, const void* H, int d, int R, float*
 
 // Launch the tensor-core GEMV-shaped draft step (1..16 sequences).
 template <int RK>
-int launch_gemv_rk(disco_ctx* c, GemvParams& g, const CUtensorMap& mW, const CUtensorMap& mWt, const CUtensorMap& mH,
-                   cudaStream_t st) {
+int launch_gemv_rk(disco_ctx* c, GemvParams& g, const CUtensorMap& mW, const CUtensorMap& mH, cudaStream_t st) {
     auto kern = umma_gemv_draft_kernel<RK>;
     static int configured_dev = -1;
     static size_t dyn_limit = 0;
@@ -269,11 +268,13 @@ int launch_gemv_rk(disco_ctx* c, GemvParams& g, const CUtensorMap& mW, const CUt
             return DISCO_ERR_CUDA;
         configured_dev = c->device;
     }
-    // the ring takes what the fixed part leaves: as many 16 KB stages as fit
+    // the ring takes what the fixed part leaves; it must hold at least two stages and the 16 KB that the
+    // MMA reads behind the last box of hidden rows
     const size_t fixed = gemv_fixed_smem_bytes(RK, g.t.clf_H, g.t.d, g.h_rows);
-    if (dyn_limit < fixed + 2 * (size_t)kGemvATile) return DISCO_ERR_UNSUPPORTED_SHAPE;
-    g.stages = (int)std::min<size_t>(kGemvMaxStages, (dyn_limit - fixed) / kGemvATile);
-    const size_t smem = gemv_smem_bytes(RK, g.t.clf_H, g.t.d, g.h_rows, g.stages);
+    if (dyn_limit < fixed + 2 * (size_t)g.b_bytes) return DISCO_ERR_UNSUPPORTED_SHAPE;
+    g.stages = (int)std::min<size_t>(kGemvMaxStages, (dyn_limit - fixed) / g.b_bytes);
+    if ((size_t)g.stages * g.b_bytes < 16384) return DISCO_ERR_UNSUPPORTED_SHAPE;
+    const size_t smem = gemv_smem_bytes(RK, g.t.clf_H, g.t.d, g.h_rows, g.stages, g.b_bytes);
     cudaLaunchConfig_t cfg{};
     cfg.gridDim = dim3((unsigned)c->sm_count);
     cfg.blockDim = dim3(kGemvThreads);
@@ -284,7 +285,7 @@ int launch_gemv_rk(disco_ctx* c, GemvParams& g, const CUtensorMap& mW, const CUt
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = c->pdl ? 1 : 0;
-    const cudaError_t e = cudaLaunchKernelEx(&cfg, kern, mW, mWt, mH, g);
+    const cudaError_t e = cudaLaunchKernelEx(&cfg, kern, mW, mH, g);
     c->launches += 1;
     return cuda_ok(e, "umma_gemv_draft_kernel launch") ? DISCO_OK : DISCO_ERR_CUDA;
 }
@@ -295,18 +296,19 @@ int launch_gemv(disco_ctx* c, const TailParams& t, cudaStream_t st) {
     const int grid = c->sm_count;
     if (grid > c->part_slots || t.R > c->part_rows) return DISCO_ERR_WORKSPACE;
     g.TR = (t.V + grid - 1) / grid;
-    g.tiles = (g.TR + 127) / 128;
-    g.tail_rows = std::max(8, (g.TR - 128 * (g.tiles - 1) + 7) / 8 * 8);
+    g.tiles = (g.TR + 255) / 256;
+    g.TRt = (g.TR + g.tiles - 1) / g.tiles;
+    g.TRN = (g.TRt + 15) / 16 * 16;
+    g.b_bytes = (g.TRN * 128 + 1023) / 1024 * 1024;
     g.h_rows = t.R <= 8 ? 8 : 16;
-    CUtensorMap mW, mWt, mH;
-    if (!encode_bf16_2d(c, &mW, t.W, t.V, t.d, 128) || !encode_bf16_2d(c, &mWt, t.W, t.V, t.d, g.tail_rows) ||
-        !encode_bf16_2d(c, &mH, t.H, t.R, t.d, g.h_rows))
+    CUtensorMap mW, mH;
+    if (!encode_bf16_2d(c, &mW, t.W, t.V, t.d, g.TRN) || !encode_bf16_2d(c, &mH, t.H, t.R, t.d, g.h_rows))
         return DISCO_ERR_CUDA;
-    if (t.R == 1) return launch_gemv_rk<1>(c, g, mW, mWt, mH, st);
-    if (t.R == 2) return launch_gemv_rk<2>(c, g, mW, mWt, mH, st);
-    if (t.R <= 4) return launch_gemv_rk<4>(c, g, mW, mWt, mH, st);
-    if (t.R <= 8) return launch_gemv_rk<8>(c, g, mW, mWt, mH, st);
-    return launch_gemv_rk<16>(c, g, mW, mWt, mH, st);
+    if (t.R == 1) return launch_gemv_rk<1>(c, g, mW, mH, st);
+    if (t.R == 2) return launch_gemv_rk<2>(c, g, mW, mH, st);
+    if (t.R <= 4) return launch_gemv_rk<4>(c, g, mW, mH, st);
+    if (t.R <= 8) return launch_gemv_rk<8>(c, g, mW, mH, st);
+    return launch_gemv_rk<16>(c, g, mW, mH, st);
 }
 
 void fill_scratch(const disco_ctx* c, TailParams& p) {

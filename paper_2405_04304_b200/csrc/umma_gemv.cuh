@@ -1,27 +1,25 @@
 // Tensor-core draft step for a handful of sequences (1..16 hidden rows): the GEMV-shaped case.
 //
-// Here the LM head is the 128-row operand of tcgen05.mma and the hidden rows are the narrow one:
+//   D[r, v] = sum_k H[r, k] * W[v, k]       r (hidden rows) on the TMEM lanes 0 .. R-1,
+//                                           v (up to 256 vocabulary rows of a tile) on the TMEM columns
 //
-//   D[v, r] = sum_k W[v, k] * H[r, k]       v (128 vocabulary rows of a tile) on the TMEM lanes,
-//                                           r (hidden rows, padded to N = 16) on the TMEM columns
+// One tcgen05.mma costs about 128 cycles whatever its N (measured: the same for N = 16 and N = 224), so
+// the vocabulary has to be the wide operand: a CTA's whole slab of ceil(V / #SM) rows is one or two MMAs
+// wide, 4 * d / 64 MMAs deep, a few microseconds that hide under the HBM stream.  (With the vocabulary on
+// the lanes and N = 16 the MMAs alone took as long as HBM needs for the slab.)
 //
-// so after tcgen05.ld every lane of an epilogue warp holds the logit of "its" vocabulary row: one
-// logit per lane, exactly the block that warp_fold_block folds into soft-max statistics, top-10 and
-// arg-max in parallel.  The dot products cost the SM a few hundred instructions instead of the
-// ~14 k of the CUDA-core kernel, so what is left is HBM streaming plus the fixed reduction tail.
-//
-//   * one CTA per SM and slab of ceil(V / #SM) vocabulary rows, cut into tiles of 128 rows (the last
-//     one shorter: its own TMA box, so nothing beyond the slab is fetched);
-//   * warp 0 producer (TMA, 128-byte swizzle, ring of 16 KB stages for the LM head; the hidden rows are
-//     loaded once, after the dependency wait, and stay), warp 1 MMA issuer (M = 128, N = 16, K = 16, two
-//     16-column TMEM buffers), warps 2-5 epilogue (one TMEM lane quadrant each);
-//   * the ring is as deep as shared memory allows (12 stages = one whole tile of the 768-wide heads) and
-//     is filled before the dependency wait, so that after the wait the first tile needs nothing but the
-//     hidden rows;
-//   * MMAs into one accumulator form a dependent chain (about 130 cycles each, measured), and a tile of a
-//     768-wide head would be 48 of them: the four K = 16 steps of a k-block go to four accumulators
-//     instead (16 TMEM columns each), which the epilogue adds up;
-//   * per-CTA records, ticket, last-CTA reduction and classifier exactly as in the streaming kernel.
+//   * one CTA per SM and slab; the slab is cut into tiles of up to 256 rows (one for the 32000-row
+//     head, two for the 49152-row one);
+//   * the hidden rows are the A operand: loaded once after the dependency wait, one 8- or 16-row box per
+//     k-block, and they stay.  The MMA reads 128 rows from each box's start: what lies behind (further
+//     boxes, the ring) only feeds accumulator lanes nobody reads;
+//   * warp 0 producer (TMA, 128-byte swizzle; ring of LM-head stages as deep as shared memory allows,
+//     filled before the dependency wait), warp 1 MMA issuer (M = 128, N = tile rows, K = 16, two
+//     256-column TMEM buffers), warps 2-5 epilogue;
+//   * epilogue: all hidden rows sit in TMEM lane quadrant 0, which one warp may read: it copies the
+//     tile's logits to shared memory (row r by lane r), then all four warps fold them 32 at a time, one
+//     logit per lane (soft-max statistics, top-10 and arg-max in parallel, warp_fold_block);
+//   * per-CTA records, ticket, last-CTA second phase and classifier exactly as in the streaming kernel.
 #pragma once
 
 #include "umma_tail.cuh"
@@ -31,70 +29,57 @@ namespace disco {
 constexpr int kGemvEpiWarps = 4;
 constexpr int kGemvThreads = (2 + kGemvEpiWarps) * 32;
 constexpr int kGemvMaxRows = 16;
-constexpr int kGemvATile = 128 * 128;   // 128 vocabulary rows x 128 B
 constexpr int kGemvMaxStages = 16;
-constexpr int kGemvAcc = kUmmaBK / 16;          // independent accumulators per TMEM buffer (4)
-constexpr int kGemvBufCols = kGemvAcc * 16;     // TMEM columns per buffer
+constexpr int kGemvRowStride = 256 + 4;   // floats per hidden row in the logit staging area (padded: no bank conflicts)
 
 struct GemvParams {
     TailParams t;     // V, d, R and everything the fused epilogue needs (scratch, classifier, outputs)
-    int TR;           // vocabulary rows per CTA
-    int tiles;        // ceil(TR / 128)
-    int tail_rows;    // rows of the last tile's TMA box (multiple of 8)
+    int TR;           // vocabulary rows per CTA (slab)
+    int tiles;        // ceil(TR / 256)
+    int TRt;          // vocabulary rows per tile
+    int TRN;          // rows of the LM-head box = N of the MMA (TRt rounded up to 16, <= 256)
+    int b_bytes;      // bytes of one ring stage (TRN * 128, a multiple of 1024)
     int h_rows;       // rows of the hidden-state box (8 or 16)
     int stages;       // ring depth (2 .. kGemvMaxStages)
 };
 
-// Shared memory besides the ring: the resident hidden rows (one k-block of h_rows x 128 B per 64 hidden
-// units; the MMA reads 16 rows from each, the surplus lands in columns nobody reads), barriers, records,
+// Shared memory besides the ring: the resident hidden rows, barriers, the logit staging area, records,
 // second-phase scratch, classifier.
 inline size_t gemv_fixed_smem_bytes(int RK, int clf_H, int d, int h_rows) {
     size_t b = 1024;                                             // alignment
-    b += (size_t)((d + kUmmaBK - 1) / kUmmaBK) * h_rows * 128 + 1024;  // hidden rows (+ the 16-row overhang)
+    b += (size_t)((d + kUmmaBK - 1) / kUmmaBK) * h_rows * 128;   // hidden rows
     b += 512;                                                    // barriers, TMEM address
+    b += (size_t)RK * kGemvRowStride * 4;                        // logits of one tile
     b += (size_t)(kGemvEpiWarps * RK + 1) * kRecordWords * 4;    // warp records / finalize staging
     b += kGemvEpiWarps * kWarpScratchWords * 4;                  // second-phase scratch per warp
     b += ((size_t)clf_H * (kNFeat + 2) + 4) * 4;                 // classifier parameters
     return b + 128;
 }
-inline size_t gemv_smem_bytes(int RK, int clf_H, int d, int h_rows, int stages) {
-    return gemv_fixed_smem_bytes(RK, clf_H, d, h_rows) + (size_t)stages * kGemvATile;
-}
-
-__device__ __forceinline__ void tmem_ld16(uint32_t taddr, float (&v)[16]) {
-    uint32_t r[16];
-    asm volatile(
-        "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
-        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
-        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
-          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
-        : "r"(taddr)
-        : "memory");
-    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-#pragma unroll
-    for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
+inline size_t gemv_smem_bytes(int RK, int clf_H, int d, int h_rows, int stages, int b_bytes) {
+    return gemv_fixed_smem_bytes(RK, clf_H, d, h_rows) + (size_t)stages * b_bytes;
 }
 
 // RK: compile-time bound on the hidden rows (1, 2, 4, 8 or 16)
 template <int RK>
 __global__ void __launch_bounds__(kGemvThreads, 1)
-umma_gemv_draft_kernel(const __grid_constant__ CUtensorMap tmap_W, const __grid_constant__ CUtensorMap tmap_Wtail,
-                       const __grid_constant__ CUtensorMap tmap_H, const GemvParams g) {
+umma_gemv_draft_kernel(const __grid_constant__ CUtensorMap tmap_W, const __grid_constant__ CUtensorMap tmap_H,
+                       const GemvParams g) {
     extern __shared__ uint8_t smem_dyn[];
     const TailParams& p = g.t;
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~uintptr_t(1023));
-    const int KBs = (p.d + kUmmaBK - 1) / kUmmaBK;
-    const int b_stride = g.h_rows * 128;   // bytes between the k-blocks of the resident hidden rows
-    uint8_t* a_tiles = smem;
-    uint8_t* b_tiles = smem + g.stages * kGemvATile;
-    uint8_t* after_b = b_tiles + KBs * b_stride + 1024;
-    uint64_t* full = reinterpret_cast<uint64_t*>(after_b);
+    const int KB = (p.d + kUmmaBK - 1) / kUmmaBK;
+    const int h_stride = g.h_rows * 128;   // bytes between the k-blocks of the resident hidden rows
+    uint8_t* h_tiles = smem;
+    uint8_t* w_tiles = smem + KB * h_stride;          // 1024-aligned; at least 16 KB long (host check)
+    uint8_t* after = w_tiles + g.stages * g.b_bytes;
+    uint64_t* full = reinterpret_cast<uint64_t*>(after);
     uint64_t* empty = full + kGemvMaxStages;
     uint64_t* tmem_full = empty + kGemvMaxStages;
     uint64_t* tmem_empty = tmem_full + 2;
     uint64_t* h_full = tmem_empty + 2;
     uint32_t* tmem_base_s = reinterpret_cast<uint32_t*>(h_full + 1);
-    float* wstate = reinterpret_cast<float*>(after_b + 512);
+    float* lg_s = reinterpret_cast<float*>(after + 512);
+    float* wstate = lg_s + RK * kGemvRowStride;
     float* feat_s = wstate + (kGemvEpiWarps * RK + 1) * kRecordWords;
     float* clf_s = feat_s + kGemvEpiWarps * kWarpScratchWords;
     __shared__ int s_is_last;
@@ -104,28 +89,26 @@ umma_gemv_draft_kernel(const __grid_constant__ CUtensorMap tmap_W, const __grid_
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
     const int grid = gridDim.x;
-    const int KB = (p.d + kUmmaBK - 1) / kUmmaBK;
     const int v_begin = blockIdx.x * g.TR;
     const int v_end = min(p.V, v_begin + g.TR);
-    const int tiles = v_begin < p.V ? g.tiles : 0;
+    const int tiles = v_begin < p.V ? (v_end - v_begin + g.TRt - 1) / g.TRt : 0;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < g.stages; ++s) {
             mbar_init(&full[s], 1);
             mbar_init(&empty[s], 1);
         }
-        mbar_init(h_full, 1);
         for (int b = 0; b < 2; ++b) {
             mbar_init(&tmem_full[b], 1);
-            mbar_init(&tmem_empty[b], kGemvEpiWarps);
+            mbar_init(&tmem_empty[b], 1);
         }
+        mbar_init(h_full, 1);
         fence_mbar_init();
         prefetch_tensormap(&tmap_W);
-        prefetch_tensormap(&tmap_Wtail);
         prefetch_tensormap(&tmap_H);
     }
     if (warp == 1) {
-        tmem_alloc(tmem_base_s, 2 * kGemvBufCols);
+        tmem_alloc(tmem_base_s, 512);
         tmem_relinquish();
     }
     tc_fence_before();
@@ -137,29 +120,26 @@ umma_gemv_draft_kernel(const __grid_constant__ CUtensorMap tmap_W, const __grid_
         // ------------------------------ producer ------------------------------
         if (lane == 0) {
             const int total = tiles * KB;
+            const uint32_t w_bytes = (uint32_t)g.TRN * 128u;
             // the LM head does not depend on the preceding kernel: the whole ring is requested at once
             const int pre = min(g.stages, total);
             for (int n = 0; n < pre; ++n) {
                 const int tile = n / KB, kb = n - tile * KB;
-                const bool last = tile == g.tiles - 1;
-                mbar_arrive_expect_tx(&full[n], (uint32_t)(last ? g.tail_rows : 128) * 128u);
-                tma_load_2d(a_tiles + n * kGemvATile, last ? &tmap_Wtail : &tmap_W, kb * kUmmaBK, v_begin + tile * 128,
-                            &full[n]);
+                mbar_arrive_expect_tx(&full[n], w_bytes);
+                tma_load_2d(w_tiles + n * g.b_bytes, &tmap_W, kb * kUmmaBK, v_begin + tile * g.TRt, &full[n]);
             }
             asm volatile("griddepcontrol.wait;" ::: "memory");
             // the hidden rows, all k-blocks on one barrier; they stay for the whole kernel
             if (total > 0) {
-                mbar_arrive_expect_tx(h_full, (uint32_t)(KB * b_stride));
-                for (int kb = 0; kb < KB; ++kb) tma_load_2d(b_tiles + kb * b_stride, &tmap_H, kb * kUmmaBK, 0, h_full);
+                mbar_arrive_expect_tx(h_full, (uint32_t)(KB * h_stride));
+                for (int kb = 0; kb < KB; ++kb) tma_load_2d(h_tiles + kb * h_stride, &tmap_H, kb * kUmmaBK, 0, h_full);
             }
             int stage = pre == g.stages ? 0 : pre, phase = pre == g.stages ? 1 : 0;
             for (int n = pre; n < total; ++n) {
                 const int tile = n / KB, kb = n - tile * KB;
-                const bool last = tile == g.tiles - 1;
                 mbar_wait(&empty[stage], phase ^ 1, p.status);
-                mbar_arrive_expect_tx(&full[stage], (uint32_t)(last ? g.tail_rows : 128) * 128u);
-                tma_load_2d(a_tiles + stage * kGemvATile, last ? &tmap_Wtail : &tmap_W, kb * kUmmaBK,
-                            v_begin + tile * 128, &full[stage]);
+                mbar_arrive_expect_tx(&full[stage], w_bytes);
+                tma_load_2d(w_tiles + stage * g.b_bytes, &tmap_W, kb * kUmmaBK, v_begin + tile * g.TRt, &full[stage]);
                 if (++stage == g.stages) {
                     stage = 0;
                     phase ^= 1;
@@ -170,7 +150,7 @@ umma_gemv_draft_kernel(const __grid_constant__ CUtensorMap tmap_W, const __grid_
         // ------------------------------ MMA issuer ------------------------------
         if (lane == 0) {
             int stage = 0, phase = 0;
-            const uint32_t idesc = umma_idesc(16);
+            const uint32_t idesc = umma_idesc(g.TRN);
             if (tiles > 0) {
                 mbar_wait(h_full, 0, p.status);
                 tc_fence_after();
@@ -179,15 +159,15 @@ umma_gemv_draft_kernel(const __grid_constant__ CUtensorMap tmap_W, const __grid_
                 const int buf = tile & 1;
                 mbar_wait(&tmem_empty[buf], ((tile >> 1) & 1) ^ 1, p.status);
                 tc_fence_after();
-                const uint32_t d_tmem = tmem_base + buf * kGemvBufCols;
+                const uint32_t d_tmem = tmem_base + buf * 256;
                 for (int kb = 0; kb < KB; ++kb) {
                     mbar_wait(&full[stage], phase, p.status);
                     tc_fence_after();
-                    const uint64_t a_desc = umma_smem_desc(a_tiles + stage * kGemvATile);
-                    const uint64_t b_desc = umma_smem_desc(b_tiles + kb * b_stride);
+                    const uint64_t a_desc = umma_smem_desc(h_tiles + kb * h_stride);
+                    const uint64_t b_desc = umma_smem_desc(w_tiles + stage * g.b_bytes);
 #pragma unroll
-                    for (int k = 0; k < kGemvAcc; ++k)  // step k of every k-block accumulates into accumulator k
-                        tc_mma_bf16(d_tmem + k * 16, a_desc + 2 * k, b_desc + 2 * k, idesc, kb != 0);
+                    for (int k = 0; k < kUmmaBK / 16; ++k)  // 16 k-elements = 32 bytes = 2 descriptor units
+                        tc_mma_bf16(d_tmem, a_desc + 2 * k, b_desc + 2 * k, idesc, (kb | k) != 0);
                     tc_commit(&empty[stage]);
                     if (++stage == g.stages) {
                         stage = 0;
@@ -230,34 +210,44 @@ umma_gemv_draft_kernel(const __grid_constant__ CUtensorMap tmap_W, const __grid_
 
         for (int tile = 0; tile < tiles; ++tile) {
             const int buf = tile & 1;
-            mbar_wait(&tmem_full[buf], (tile >> 1) & 1, p.status);
-            tc_fence_after();
-            const int v_lane0 = v_begin + tile * 128 + quad * 32;  // vocabulary row of lane 0 of this warp
-            const int n = max(0, min(32, v_end - v_lane0));        // rows of the slab in this warp's quadrant
-            float z[16];
-            tmem_ld16(tmem_base + buf * kGemvBufCols + (static_cast<uint32_t>(quad * 32) << 16), z);
+            const int v0 = v_begin + tile * g.TRt;
+            const int ncols = min(g.TRt, v_end - v0);   // further columns belong to the next tile or lie past the slab
+            const int nblocks = (ncols + 31) >> 5;
+            if (quad == 0) {
+                // the one warp that may read lane quadrant 0: row r of the tile's logits goes to shared memory
+                mbar_wait(&tmem_full[buf], (tile >> 1) & 1, p.status);
+                tc_fence_after();
+                for (int c = 0; c < nblocks; ++c) {
+                    float z[32];
+                    tmem_ld32(tmem_base + buf * 256 + c * 32, z);
+                    if (lane < p.R) {
+                        float4* dst = reinterpret_cast<float4*>(lg_s + lane * kGemvRowStride + c * 32);
 #pragma unroll
-            for (int a = 1; a < kGemvAcc; ++a) {
-                float za[16];
-                tmem_ld16(tmem_base + buf * kGemvBufCols + a * 16 + (static_cast<uint32_t>(quad * 32) << 16), za);
-#pragma unroll
-                for (int r = 0; r < 16; ++r) z[r] += za[r];
+                        for (int j = 0; j < 32; j += 4)
+                            dst[j >> 2] = make_float4(__fadd_rn(z[j], 0.f), __fadd_rn(z[j + 1], 0.f),
+                                                      __fadd_rn(z[j + 2], 0.f), __fadd_rn(z[j + 3], 0.f));
+                    }
+                }
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&tmem_empty[buf]);  // the values are in shared memory: the buffer is free
             }
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&tmem_empty[buf]);  // the values are in registers: the buffer is free
-            if (n > 0) {
-                const int idx = v_lane0 + lane;
+            named_barrier_sync(1, BAR_THREADS);
+            // blocks of 32 logits, one per lane, dealt round-robin to the four warps
+            for (int c = ew; c < nblocks; c += kGemvEpiWarps) {
+                const int n = min(32, ncols - c * 32);
+                const int idx = v0 + c * 32 + lane;
 #pragma unroll
                 for (int r = 0; r < RK; ++r) {
                     if (r < p.R) {
-                        const float val = lane < n ? __fadd_rn(z[r], 0.f) : DISCO_NEG_INF;
+                        const float val = lane < n ? lg_s[r * kGemvRowStride + c * 32 + lane] : DISCO_NEG_INF;
                         if (p.probs && lane < n) p.probs[(size_t)r * p.V + idx] = val;
                         warp_fold_block(val, idx, n, lane, st[r], best_v[r], best_i[r], top_v[r],
                                         fold_scratch + r * kRecordWords);
                     }
                 }
             }
+            if (tile + 1 < tiles) named_barrier_sync(1, BAR_THREADS);  // the staging area is overwritten next
         }
 
         // ---- merge the four warps of this CTA, publish the CTA's record for each hidden row ----
@@ -299,7 +289,7 @@ umma_gemv_draft_kernel(const __grid_constant__ CUtensorMap tmap_W, const __grid_
     __syncthreads();
     if (warp == 1) {
         tc_fence_after();
-        tmem_dealloc(tmem_base, 2 * kGemvBufCols);
+        tmem_dealloc(tmem_base, 512);
     }
 }
 
