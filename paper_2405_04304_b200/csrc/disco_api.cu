@@ -515,13 +515,14 @@ int draft_step_common(disco_ctx* c, const void* W_D, const void* h_D, int d, int
     p.feats = feats;
     p.probs = probs;
     p.nll_sum = nll_sum;
-    // Measured on B200 (Vicuna head): up to 6 sequences are fastest on the tensor-core kernel with the
-    // vocabulary on the TMEM lanes, more on the one with the hidden rows on the lanes; the CUDA-core
-    // streaming kernel is within 10 % for one sequence and serves as the path without tensor maps.
+    // Measured on B200 (Vicuna head, us per step for 1 / 2 / 3 / 4 / 6 / 8 sequences): the tensor-core kernel
+    // that folds the logits a block at a time 15.0 / 18.6 / 21.2 / 23.7 / 30.7 / 34.0, the one with a thread
+    // per hidden row 22.9 / 23.3 / 23.4 / 23.0 / 23.3 / 23.5: the first up to 3 sequences, the second beyond.
+    // The CUDA-core streaming kernel is within 5 % for one sequence and serves as the path without tensor maps.
     // (its hidden rows stay in shared memory: up to 48 KB of them, so that the ring keeps at least 8 stages)
     const bool gemv_ok = c->encode_tiled != nullptr && B <= kGemvMaxRows && !stats_only &&
                          (size_t)((d + kUmmaBK - 1) / kUmmaBK) * (B <= 8 ? 8 : 16) * 128 <= 48 * 1024;
-    const bool use_gemv = gemv_ok && (c->path == 3 || (c->path == 0 && B <= 6));
+    const bool use_gemv = gemv_ok && (c->path == 3 || (c->path == 0 && B <= 3));
     const bool use_umma = !use_gemv && umma_possible(c, B) && (c->path == 2 || c->path == 3 || (c->path == 0 && B >= 2));
     if (use_gemv) {
         rc = launch_gemv(c, p, st);
