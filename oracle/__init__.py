@@ -374,3 +374,50 @@ def verify_sample(W_T, H_T, draft_ids, draft_probs, row_off, ua, us, nthreads: i
         _p(ua, ctypes.c_double) if ua.size else None, _p(us, ctypes.c_double),
         _p(n, ctypes.c_int32), _p(nxt, ctypes.c_int32), _p(yT, ctypes.c_double), nthreads), "verify_sample")
     return VerifySampleResult(n, nxt, yT)
+
+
+# --------------------------------------------------------------------------- bulk feature extraction (App. D)
+def total_variation(p, q) -> float:
+    p = np.ascontiguousarray(p, dtype=np.float64)
+    q = np.ascontiguousarray(q, dtype=np.float64)
+    assert p.shape == q.shape and p.ndim == 1
+    tv = ctypes.c_double(-1.0)
+    _check(lib().oracle_total_variation(_p(p, ctypes.c_double), _p(q, ctypes.c_double), p.shape[0], ctypes.byref(tv)),
+           "total_variation")
+    return float(tv.value)
+
+
+@dataclass
+class FeatureRows:
+    feats_D: np.ndarray   # [N, k+2] float64
+    feats_T: np.ndarray   # [N, k+2] float64
+    tv: np.ndarray        # [N] float64
+    label: np.ndarray     # [N] uint8, 1 = accepted
+    token_D: np.ndarray   # [N] int32
+    token_T: np.ndarray   # [N] int32
+    gap_D: np.ndarray     # [N] float64, top-2 logit gaps
+    gap_T: np.ndarray
+
+
+def extract_features(W_D, H_D, W_T, H_T, pos, k: int = K_TOP, nthreads: int = 1) -> FeatureRows:
+    W_D, H_D, W_T, H_T = _u16(W_D), _u16(H_D), _u16(W_T), _u16(H_T)
+    V, d_D = W_D.shape
+    V2, d_T = W_T.shape
+    N = H_D.shape[0]
+    assert V == V2 and H_T.shape[0] == N and H_D.shape[1] == d_D and H_T.shape[1] == d_T
+    pos = np.ascontiguousarray(pos, dtype=np.int32)
+    assert pos.shape[0] == N
+    fD = np.full((N, k + 2), np.nan)
+    fT = np.full((N, k + 2), np.nan)
+    tv = np.full(N, np.nan)
+    label = np.full(N, 255, dtype=np.uint8)
+    tD = np.full(N, -1, dtype=np.int32)
+    tT = np.full(N, -1, dtype=np.int32)
+    gD = np.full(N, np.nan)
+    gT = np.full(N, np.nan)
+    _check(lib().oracle_extract_features(
+        _p(W_D, ctypes.c_uint16), _p(H_D, ctypes.c_uint16), d_D, _p(W_T, ctypes.c_uint16), _p(H_T, ctypes.c_uint16),
+        d_T, V, N, _p(pos, ctypes.c_int32), k, _p(fD, ctypes.c_double), _p(fT, ctypes.c_double),
+        _p(tv, ctypes.c_double), _p(label, ctypes.c_uint8), _p(tD, ctypes.c_int32), _p(tT, ctypes.c_int32),
+        _p(gD, ctypes.c_double), _p(gT, ctypes.c_double), nthreads), "extract_features")
+    return FeatureRows(fD, fT, tv, label, tD, tT, gD, gT)

@@ -428,6 +428,66 @@ int oracle_verify_sample(const uint16_t* W_T, const uint16_t* H_T, int V, int d,
     return ORACLE_OK;
 }
 
+// ---------------------------------------------------------------------------
+// Bulk feature extraction for classifier training (App. D, Sec. 4 "SL classifier
+// training"): for N positions at once, the features of Eq. 2 of the draft AND of
+// the target distribution, the accepted/rejected label and the total-variation
+// distance between the two distributions.
+// ---------------------------------------------------------------------------
+
+// Total variation distance TV(p, q) = (1/2) * sum_v |p_v - q_v|.
+int oracle_total_variation(const double* p, const double* q, int V, double* tv) {
+    if (!p || !q || !tv || V <= 0) return ORACLE_BAD_ARG;
+    double s = 0.0;
+    for (int v = 0; v < V; ++v) s += std::fabs(p[v] - q[v]);
+    *tv = 0.5 * s;
+    return ORACLE_OK;
+}
+
+// Position n (0 <= n < N) has a draft hidden state H_D[n] and a target hidden state H_T[n] (both models
+// have seen the same prefix: the prompt plus the target's own tokens) and the position counter pos[n].
+//   y^D = softmax(W_D H_D[n]),  y^T = softmax(W_T H_T[n])
+//   feats_D[n] = Concat(Top_k(y^D), Ent(y^D), pos[n]),  feats_T[n] likewise from y^T
+//   label[n]   = 1 iff arg-max y^D == arg-max y^T        (the draft token "resembles" the target token:
+//                token equality, the criterion of greedy verification)
+//   tv[n]      = TV(y^D, y^T)
+// token_D, token_T, gap_D, gap_T (top-2 logit gaps) are optional.
+int oracle_extract_features(const uint16_t* W_D, const uint16_t* H_D, int d_D,
+                            const uint16_t* W_T, const uint16_t* H_T, int d_T, int V, int N,
+                            const int32_t* pos, int k,
+                            double* feats_D, double* feats_T, double* tv, uint8_t* label,
+                            int32_t* token_D, int32_t* token_T, double* gap_D, double* gap_T, int nthreads) {
+    if (!W_D || !H_D || !W_T || !H_T || !pos || !feats_D || !feats_T || !tv || !label || V <= 0 || d_D <= 0 ||
+        d_T <= 0 || N < 0 || k <= 0)
+        return ORACLE_BAD_ARG;
+    std::vector<double> z(V), yD(V), yT(V);
+    for (int n = 0; n < N; ++n) {
+        int32_t tD = -1, tT = -1;
+        int rc = oracle_project(W_D, H_D + (size_t)n * d_D, V, d_D, 1, z.data(), nthreads);
+        if (rc) return rc;
+        rc = oracle_argmax(z.data(), V, &tD, gap_D ? &gap_D[n] : nullptr);
+        if (rc) return rc;
+        rc = oracle_softmax(z.data(), V, yD.data());
+        if (rc) return rc;
+        rc = oracle_project(W_T, H_T + (size_t)n * d_T, V, d_T, 1, z.data(), nthreads);
+        if (rc) return rc;
+        rc = oracle_argmax(z.data(), V, &tT, gap_T ? &gap_T[n] : nullptr);
+        if (rc) return rc;
+        rc = oracle_softmax(z.data(), V, yT.data());
+        if (rc) return rc;
+        rc = oracle_features(yD.data(), V, k, pos[n], feats_D + (size_t)n * (k + 2));
+        if (rc) return rc;
+        rc = oracle_features(yT.data(), V, k, pos[n], feats_T + (size_t)n * (k + 2));
+        if (rc) return rc;
+        rc = oracle_total_variation(yD.data(), yT.data(), V, &tv[n]);
+        if (rc) return rc;
+        label[n] = tD == tT ? 1 : 0;
+        if (token_D) token_D[n] = tD;
+        if (token_T) token_T[n] = tT;
+    }
+    return ORACLE_OK;
+}
+
 int oracle_hardware_threads() { return (int)std::thread::hardware_concurrency(); }
 
 }  // extern "C"

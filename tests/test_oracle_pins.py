@@ -574,3 +574,57 @@ def test_draft_step_sample_differs_from_greedy_step_only_in_the_token(oracle):
         cdf = np.cumsum(g.probs[b])
         assert cdf[s.token[b]] > u[b] * cdf[-1] - 1e-15 and (s.token[b] == 0 or cdf[s.token[b] - 1] <= u[b] * cdf[-1] + 1e-15)
     assert s.token[0] == int(np.argmax(g.probs[0] > 0))           # u = 0 draws the first token with mass
+
+
+# ------------------------------------------------------------------ bulk feature extraction (App. D)
+def test_total_variation_closed_forms_and_event_characterisation(oracle):
+    assert oracle.total_variation([0.5, 0.5], [0.9, 0.1]) == pytest.approx(0.4, abs=1e-15)
+    assert oracle.total_variation([0.2, 0.3, 0.5], [0.2, 0.3, 0.5]) == 0.0
+    assert oracle.total_variation([1.0, 0.0, 0.0], [0.0, 0.0, 1.0]) == 1.0          # disjoint supports
+    rng = np.random.default_rng(8)
+    p, q = rng.dirichlet(np.ones(7)), rng.dirichlet(np.ones(7))
+    tv = oracle.total_variation(p, q)
+    assert tv == pytest.approx(oracle.total_variation(q, p), abs=1e-15)             # symmetric
+    # TV is the largest difference in probability that the two distributions give to any event:
+    # brute force over all 2^7 subsets of the vocabulary
+    best = 0.0
+    for mask in range(1 << 7):
+        sel = [(mask >> v) & 1 == 1 for v in range(7)]
+        best = max(best, abs(p[sel].sum() - q[sel].sum()))
+    assert tv == pytest.approx(best, abs=1e-14)
+    # and one minus the mass the two distributions share: checked against the acceptance rate that
+    # the brute-force pin of speculative sampling measured for these two vectors
+    yD, yT = np.array([0.70, 0.10, 0.15, 0.05]), np.array([0.10, 0.20, 0.30, 0.40])
+    assert oracle.total_variation(yD, yT) == pytest.approx(0.6, abs=1e-15)
+
+
+def test_extract_features_is_two_draft_steps_a_label_and_a_distance(oracle):
+    rng = np.random.default_rng(12)
+    V, dD, dT, N = 83, 16, 40, 6
+    WD = bits_of(torch.from_numpy(rng.normal(size=(V, dD)).astype(np.float32)))
+    WT = bits_of(torch.from_numpy(rng.normal(size=(V, dT)).astype(np.float32)))
+    HD = bits_of(torch.from_numpy(rng.normal(size=(N, dD)).astype(np.float32)))
+    HT = bits_of(torch.from_numpy(rng.normal(size=(N, dT)).astype(np.float32)))
+    # make two positions agree by construction: both hidden states point along their head's row of one token
+    for n, tok in ((1, 17), (4, 60)):
+        HD[n] = bits_of(torch.tensor([6.0 * py_bf16(b) for b in WD[tok]], dtype=torch.float32))
+        HT[n] = bits_of(torch.tensor([6.0 * py_bf16(b) for b in WT[tok]], dtype=torch.float32))
+    pos = np.arange(N, dtype=np.int32) + 3
+    res = oracle.extract_features(WD, HD, WT, HT, pos)
+    clf = oracle.Classifier(np.zeros((4, 12), np.float32), np.zeros(4, np.float32), np.zeros(4, np.float32),
+                            np.zeros(1, np.float32))
+    dD_ = oracle.draft_step(WD, HD, pos, np.ones(N, np.int32), clf, 0.5, 9, want_probs=True)
+    dT_ = oracle.draft_step(WT, HT, pos, np.ones(N, np.int32), clf, 0.5, 9, want_probs=True)
+    np.testing.assert_array_equal(res.feats_D, dD_.feats)
+    np.testing.assert_array_equal(res.feats_T, dT_.feats)
+    np.testing.assert_array_equal(res.token_D, dD_.token)
+    np.testing.assert_array_equal(res.token_T, dT_.token)
+    np.testing.assert_array_equal(res.label, (dD_.token == dT_.token).astype(np.uint8))
+    assert res.label[1] == 1 and res.label[4] == 1 and res.token_D[1] == 17 and res.token_T[4] == 60
+    for n in range(N):
+        assert res.tv[n] == pytest.approx(0.5 * np.abs(dD_.probs[n] - dT_.probs[n]).sum(), abs=1e-14)
+        assert 0.0 <= res.tv[n] <= 1.0
+    # the label is what greedy verification would decide for a one-token look-ahead at that position
+    for n in range(N):
+        v = oracle.verify_ragged(WT, HT[n:n + 1], np.zeros(0, np.int32), np.array([0, 1], np.int32))
+        assert (v.bonus[0] == res.token_D[n]) == bool(res.label[n])
