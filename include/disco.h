@@ -182,6 +182,26 @@ int disco_verify_sample_ragged(disco_ctx* ctx, const void* W_T, const void* H_T,
                                void* stream);
 
 /*
+ * Bulk feature extraction for classifier training (App. D; Sec. 4 "SL classifier training"): N positions
+ * at once, each with the draft model's and the target model's hidden state for the same prefix.
+ *   y^D = softmax(W_D H_D[n]),  y^T = softmax(W_T H_T[n])
+ *   feats_D[n] = Concat(Top_10(y^D), Ent(y^D), pos[n]);  feats_T[n] the same from y^T   (Eq. 2's features)
+ *   label[n]   = 1 ("accepted") iff arg-max y^D == arg-max y^T, else 0
+ *   tv[n]      = TV(y^D, y^T) = (1/2) sum_v |y^D_v - y^T_v|   (the distance named for the training loss)
+ * Arguments (device pointers):
+ *   W_D bf16 [V, d_draft], H_D bf16 [N, d_draft], W_T bf16 [V, d_target], H_T bf16 [N, d_target],
+ *   pos int32 [N]; 1 <= N <= max_rows of disco_create
+ * Outputs (device): feats_D, feats_T float [N, 12]; tv float [N]; label uint8 [N];
+ *   token_D, token_T int32 [N] (the arg-max ids); y_D, y_T float [N, V]: the two distributions (also
+ *   the call's work space).  All REQUIRED.
+ * Errors as in disco_draft_step.
+ */
+int disco_extract_features(disco_ctx* ctx, const void* W_D, const void* H_D, const void* W_T, const void* H_T,
+                           const int32_t* pos, int N, float* feats_D, float* feats_T, float* tv,
+                           uint8_t* label, int32_t* token_D, int32_t* token_T, float* y_D, float* y_T,
+                           void* stream);
+
+/*
  * Verification with the same look-ahead SL for all B sequences (Sec. 2; Fig. 1).
  *   W_T        bf16 [V, d_target]          target LM head
  *   H_T        bf16 [B*(SL+1), d_target]   row b*(SL+1)+j is the target hidden state whose

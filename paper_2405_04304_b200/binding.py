@@ -30,7 +30,7 @@ EXPORTS = [
     "disco_create", "disco_destroy", "disco_strerror", "disco_last_device_status", "disco_launch_count",
     "disco_set_kernel_path", "disco_draft_step", "disco_verify", "disco_verify_ragged",
     "disco_draft_step_host", "disco_verify_ragged_host", "disco_draft_step_static", "disco_draft_step_ppl",
-    "disco_draft_step_sample", "disco_verify_sample_ragged",
+    "disco_draft_step_sample", "disco_verify_sample_ragged", "disco_extract_features",
 ]
 
 
@@ -71,6 +71,7 @@ def load() -> ctypes.CDLL:
     lib.disco_draft_step_sample.argtypes = [vp, vp, vp, ci, vp, vp, vp, ctypes.POINTER(_Clf), cf, ci, vp,
                                             vp, vp, vp, vp, vp, vp, vp]
     lib.disco_verify_sample_ragged.argtypes = [vp, vp, vp, vp, vp, vp, ci, ci, vp, vp, vp, vp, vp, vp, vp]
+    lib.disco_extract_features.argtypes = [vp, vp, vp, vp, vp, vp, ci, vp, vp, vp, vp, vp, vp, vp, vp, vp]
     lib.disco_verify.argtypes = [vp, vp, vp, vp, ci, ci, vp, vp, vp, vp]
     lib.disco_verify_ragged.argtypes = [vp, vp, vp, vp, vp, ci, ci, vp, vp, vp, vp]
     lib.disco_draft_step_host.argtypes = [vp, vp, vp, ci, vp, vp, vp, ctypes.POINTER(_Clf), cf, ci,
@@ -224,6 +225,18 @@ class Context:
             _stream(stream))
         if rc != OK:
             raise DiscoError(rc, "disco_verify_sample_ragged")
+
+    def extract_features(self, W_D, H_D, W_T, H_T, pos, feats_D, feats_T, tv, label, token_D, token_T, y_D, y_T,
+                         stream=None) -> None:
+        N = int(H_D.shape[0])
+        rc = self._lib.disco_extract_features(
+            self._h, _ptr(W_D, torch.bfloat16), _ptr(H_D, torch.bfloat16), _ptr(W_T, torch.bfloat16),
+            _ptr(H_T, torch.bfloat16), _ptr(pos, torch.int32), N, _ptr(feats_D, torch.float32),
+            _ptr(feats_T, torch.float32), _ptr(tv, torch.float32), _ptr(label, torch.uint8),
+            _ptr(token_D, torch.int32), _ptr(token_T, torch.int32), _ptr(y_D, torch.float32),
+            _ptr(y_T, torch.float32), _stream(stream))
+        if rc != OK:
+            raise DiscoError(rc, "disco_extract_features")
 
     def verify(self, W_T, H_T, draft_ids, B: int, SL: int, n_accept, bonus, target_ids=None,
                stream=None) -> None:

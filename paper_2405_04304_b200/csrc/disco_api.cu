@@ -469,14 +469,16 @@ bool configure_sampling(disco_ctx* c) {
 
 // Shared body of the LM-head + soft-max passes: B rows of hidden size d against the head W.
 //   * nll_sum != null selects the perplexity rule (no classifier; tau is the perplexity bound);
-//   * stats_only: arg-max (token, optional) and soft-max statistics only, no classifier: the target
-//     rows of a verification with sampling (pos, n_drafted, conf, halt unused).
+//   * stats_only = 1: arg-max (token, optional) and soft-max statistics only, no classifier: the target
+//     rows of a verification with sampling (pos, n_drafted, conf, halt unused);
+//   * stats_only = 2: token and features, no classifier: bulk feature extraction (n_drafted, conf, halt unused).
 int draft_step_common(disco_ctx* c, const void* W_D, const void* h_D, int d, int B, int max_rows, const int32_t* pos,
                       const int32_t* n_drafted, const uint8_t* active, const disco_clf* clf, float tau,
                       int sl_max, int32_t* token, float* conf, uint8_t* halt, float* feats, float* probs,
-                      float* nll_sum, bool stats_only, void* stream, bool normalize = true) {
+                      float* nll_sum, int stats_only, void* stream, bool normalize = true) {
     if (!c || !W_D || !h_D) return DISCO_ERR_INVALID_ARG;
     if (!stats_only && (!pos || !n_drafted || !token || !conf || !halt)) return DISCO_ERR_INVALID_ARG;
+    if (stats_only == 2 && (!pos || !feats)) return DISCO_ERR_INVALID_ARG;
     if (!aligned16(W_D) || !aligned16(h_D)) return DISCO_ERR_INVALID_ARG;
     if (B < 1 || sl_max < 1) return DISCO_ERR_INVALID_ARG;
     if (B > max_rows) return DISCO_ERR_WORKSPACE;
@@ -498,7 +500,7 @@ int draft_step_common(disco_ctx* c, const void* W_D, const void* h_D, int d, int
     p.R = B;
     p.B = B;
     fill_scratch(c, p);
-    p.stats_only = stats_only ? 1 : 0;
+    p.stats_only = stats_only;
     p.pos = pos;
     p.n_drafted = n_drafted;
     p.active = active;
@@ -546,9 +548,9 @@ int draft_step_common(disco_ctx* c, const void* W_D, const void* h_D, int d, int
         f.feats = feats;
         f.final_stats = c->final_stats;
         f.nll_sum = nll_sum;
-        f.stats_only = stats_only ? 1 : 0;
+        f.stats_only = stats_only;
         f.epoch = c->ticket + 48;
-        rc = stats_only ? launch_umma<true, true>(c, W_D, h_D, d, B, probs, &f, nullptr, st)
+        rc = stats_only == 1 ? launch_umma<true, true>(c, W_D, h_D, d, B, probs, &f, nullptr, st)
                         : launch_umma<true>(c, W_D, h_D, d, B, probs, &f, nullptr, st);
         if (rc) return rc;
     } else {
@@ -574,7 +576,7 @@ int disco_draft_step(disco_ctx* c, const void* W_D, const void* h_D, int B, cons
                      void* stream) {
     if (!c) return DISCO_ERR_INVALID_ARG;
     return draft_step_common(c, W_D, h_D, c->d_draft, B, c->max_batch, pos, n_drafted, active, clf, tau, sl_max, token,
-                             conf, halt, feats, probs, nullptr, false, stream);
+                             conf, halt, feats, probs, nullptr, 0, stream);
 }
 
 int disco_draft_step_ppl(disco_ctx* c, const void* W_D, const void* h_D, int B, const int32_t* n_drafted,
@@ -583,7 +585,7 @@ int disco_draft_step_ppl(disco_ctx* c, const void* W_D, const void* h_D, int B, 
     if (!nll_sum) return DISCO_ERR_INVALID_ARG;
     if (!c) return DISCO_ERR_INVALID_ARG;
     return draft_step_common(c, W_D, h_D, c->d_draft, B, c->max_batch, n_drafted, n_drafted, active, nullptr, ppl_max,
-                             sl_max, token, ppl, halt, nullptr, nullptr, nll_sum, false, stream);
+                             sl_max, token, ppl, halt, nullptr, nullptr, nll_sum, 0, stream);
 }
 
 int disco_draft_step_sample(disco_ctx* c, const void* W_D, const void* h_D, int B, const int32_t* pos,
@@ -592,7 +594,7 @@ int disco_draft_step_sample(disco_ctx* c, const void* W_D, const void* h_D, int 
                             float* feats, float* probs, void* stream) {
     if (!c || !u || !probs) return DISCO_ERR_INVALID_ARG;
     int rc = draft_step_common(c, W_D, h_D, c->d_draft, B, c->max_batch, pos, n_drafted, active, clf, tau, sl_max,
-                               token, conf, halt, feats, probs, nullptr, false, stream, false);
+                               token, conf, halt, feats, probs, nullptr, 0, stream, false);
     if (rc) return rc;
     // probs holds the logits: the kernel turns them into y^D and replaces the greedy token by the draw
     const size_t smem = sample_smem_bytes(c->V);
@@ -613,7 +615,7 @@ int disco_verify_sample_ragged(disco_ctx* c, const void* W_T, const void* H_T, c
     if (B > c->max_batch || R > c->max_rows) return DISCO_ERR_WORKSPACE;
     // target distributions of all rows: LM head, soft-max statistics, normalised rows in y_T
     int rc = draft_step_common(c, W_T, H_T, c->d_target, R, c->max_rows, nullptr, nullptr, nullptr, nullptr, 0.f, 1,
-                               target_ids, nullptr, nullptr, nullptr, y_T, nullptr, true, stream);
+                               target_ids, nullptr, nullptr, nullptr, y_T, nullptr, 1, stream);
     if (rc) return rc;
     SpecSampleParams sp{};
     sp.y_T = y_T;
@@ -636,6 +638,25 @@ int disco_verify_sample_ragged(disco_ctx* c, const void* W_T, const void* H_T, c
     speculative_sample_kernel<<<B, kSampleThreads, smem, static_cast<cudaStream_t>(stream)>>>(sp);
     c->launches += 1;
     return cuda_ok(cudaGetLastError(), "speculative_sample_kernel launch") ? DISCO_OK : DISCO_ERR_CUDA;
+}
+
+int disco_extract_features(disco_ctx* c, const void* W_D, const void* H_D, const void* W_T, const void* H_T,
+                           const int32_t* pos, int N, float* feats_D, float* feats_T, float* tv, uint8_t* label,
+                           int32_t* token_D, int32_t* token_T, float* y_D, float* y_T, void* stream) {
+    if (!c || !pos || !feats_D || !feats_T || !tv || !label || !token_D || !token_T || !y_D || !y_T)
+        return DISCO_ERR_INVALID_ARG;
+    if (N < 1) return DISCO_ERR_INVALID_ARG;
+    if (N > c->max_rows) return DISCO_ERR_WORKSPACE;
+    // the same LM-head pass as a draft step, once per model, without the classifier
+    int rc = draft_step_common(c, W_D, H_D, c->d_draft, N, c->max_rows, pos, nullptr, nullptr, nullptr, 0.f, 1, token_D,
+                               nullptr, nullptr, feats_D, y_D, nullptr, 2, stream);
+    if (rc) return rc;
+    rc = draft_step_common(c, W_T, H_T, c->d_target, N, c->max_rows, pos, nullptr, nullptr, nullptr, 0.f, 1, token_T,
+                           nullptr, nullptr, feats_T, y_T, nullptr, 2, stream);
+    if (rc) return rc;
+    tv_label_kernel<<<N, 256, 0, static_cast<cudaStream_t>(stream)>>>(y_D, y_T, token_D, token_T, c->V, tv, label);
+    c->launches += 1;
+    return cuda_ok(cudaGetLastError(), "tv_label_kernel launch") ? DISCO_OK : DISCO_ERR_CUDA;
 }
 
 int disco_verify_ragged(disco_ctx* c, const void* W_T, const void* H_T, const int32_t* draft_ids,

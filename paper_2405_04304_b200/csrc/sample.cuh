@@ -250,4 +250,38 @@ static __global__ void __launch_bounds__(kSampleThreads) speculative_sample_kern
     }
 }
 
+// Bulk feature extraction (App. D): per position the total-variation distance TV(y^D, y^T) =
+// (1/2) sum_v |y^D_v - y^T_v| of the two distributions (rows of y_D and y_T) and the accepted label
+// (draft arg-max equals target arg-max).  One CTA per position.
+static __global__ void __launch_bounds__(256)
+tv_label_kernel(const float* __restrict__ y_D, const float* __restrict__ y_T, const int32_t* __restrict__ token_D,
+                const int32_t* __restrict__ token_T, int V, float* tv, uint8_t* label) {
+    __shared__ double part[8];
+    const int n = blockIdx.x;
+    const float* a = y_D + (size_t)n * V;
+    const float* b = y_T + (size_t)n * V;
+    double s = 0.0;
+    for (int v0 = threadIdx.x; v0 < V; v0 += kSampleBatch * 256) {
+        float x[kSampleBatch], y[kSampleBatch];
+#pragma unroll
+        for (int k = 0; k < kSampleBatch; ++k) {
+            const int v = v0 + k * 256;
+            x[k] = v < V ? __ldcg(a + v) : 0.f;
+            y[k] = v < V ? __ldcg(b + v) : 0.f;
+        }
+#pragma unroll
+        for (int k = 0; k < kSampleBatch; ++k) s += static_cast<double>(fabsf(x[k] - y[k]));
+    }
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) s += __shfl_xor_sync(kFullMask, s, off);
+    if ((threadIdx.x & 31) == 0) part[threadIdx.x >> 5] = s;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        double t = 0.0;
+        for (int w = 0; w < 8; ++w) t += part[w];
+        tv[n] = static_cast<float>(0.5 * t);
+        label[n] = token_D[n] == token_T[n] ? 1 : 0;
+    }
+}
+
 }  // namespace disco

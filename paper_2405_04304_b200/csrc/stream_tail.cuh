@@ -56,7 +56,8 @@ struct TailParams {
     float* feats;
     float* probs;
     float* nll_sum;      // non-null: perplexity rule instead of the classifier (tau is then the perplexity bound)
-    int stats_only;      // non-zero: arg-max and soft-max statistics only; pos, n_drafted and the classifier are unused
+    int stats_only;      // 1: arg-max and soft-max statistics only (pos, n_drafted, classifier unused); 2: token and
+                         // features only (classifier, n_drafted unused)
     // verification
     const int32_t* draft_ids;
     const int32_t* row_off;  // null: uniform SL
@@ -527,13 +528,14 @@ struct DraftOutputs {
     float* feats;
     float* final_stats;
     float* nll_sum;  // non-null: perplexity rule (App. F) instead of the classifier
-    int stats_only;  // non-zero: arg-max and soft-max statistics only (rows of a verification with sampling)
+    int stats_only;  // 1: arg-max and soft-max statistics only (rows of a verification with sampling);
+                     // 2: token and features, no classifier (bulk feature extraction)
 };
 __device__ __forceinline__ void warp_draft_epilogue(const SoftmaxState& st, unsigned long long key, float sel, float fpos,
                                                     int n_drafted, float tau, int sl_max, float* feat_s, const float* W1,
                                                     const float* b1, const float* w2, const float* b2, int Hc, int b,
                                                     const DraftOutputs& o, int lane) {
-    if (o.stats_only) {
+    if (o.stats_only == 1) {
         if (lane == 0) {
             if (o.token) o.token[b] = key_index(key);
             o.final_stats[2 * b] = st.m;
@@ -561,6 +563,15 @@ __device__ __forceinline__ void warp_draft_epilogue(const SoftmaxState& st, unsi
     const float prob = (lane < kTopK && sel > DISCO_NEG_INF) ? __expf(sel - st.m) * inv_Z : 0.f;
     const float ent = __logf(st.Z) - st.S * inv_Z;
     const float x = lane < kTopK ? prob : (lane == kTopK ? ent : (lane == kTopK + 1 ? fpos : 0.f));
+    if (o.stats_only == 2) {
+        if (lane == 0) {
+            if (o.token) o.token[b] = key_index(key);
+            o.final_stats[2 * b] = st.m;
+            o.final_stats[2 * b + 1] = st.Z;
+        }
+        if (o.feats && lane < kNFeat) o.feats[(size_t)b * kNFeat + lane] = x;
+        return;
+    }
     const float C = warp_halt_classifier(x, feat_s, W1, b1, w2, b2, Hc, lane);
     if (lane == 0) {
         o.token[b] = key_index(key);

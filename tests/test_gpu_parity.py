@@ -573,3 +573,56 @@ def test_verify_sample_uniform_look_ahead_and_acceptance_range(oracle):
 def test_verify_sample_full_size_heads(oracle, name, SL):
     wl = inputs.WORKLOADS[name]
     _verify_sample_case(oracle, wl.V, wl.d_T, [SL], seed=wl.seed + 40)
+
+
+# ---------------------------------------------------------------------------------- bulk feature extraction (App. D)
+def _extract_case(oracle, V, dD, dT, N, seed, path=0):
+    WD = inputs.lm_head(V, dD, seed=seed, std=0.25)
+    WT = inputs.lm_head(V, dT, seed=seed + 1, std=0.25)
+    HD = inputs.hidden(N, dD, seed=seed + 2)
+    HT = inputs.hidden(N, dT, seed=seed + 3)
+    # a share of the positions agrees by construction: both hidden states point along their head's row of one token
+    g = torch.Generator().manual_seed(seed)
+    toks = torch.randint(0, V, (N,), generator=g)
+    for n in range(0, N, 3):
+        HD[n] = (8.0 / 0.25 ** 2 / dD) * WD[toks[n]].float()
+        HT[n] = (8.0 / 0.25 ** 2 / dT) * WT[toks[n]].float()
+    HD, HT = HD.to(torch.bfloat16), HT.to(torch.bfloat16)
+    pos = np.arange(N, dtype=np.int32) * 2 + 1
+    ctx = _ctx(V, dD, dT, max_batch=8, max_rows=max(64, N))
+    ctx.set_kernel_path(path)
+    dev = "cuda"
+    fD = torch.full((N, binding.NFEAT), -7.0, device=dev); fT = torch.full((N, binding.NFEAT), -7.0, device=dev)
+    tv = torch.full((N,), -7.0, device=dev); label = torch.full((N,), 77, dtype=torch.uint8, device=dev)
+    tD = torch.full((N,), -7, dtype=torch.int32, device=dev); tT = torch.full((N,), -7, dtype=torch.int32, device=dev)
+    yD = torch.full((N, V), -7.0, device=dev); yT = torch.full((N, V), -7.0, device=dev)
+    ctx.extract_features(WD.cuda(), HD.cuda(), WT.cuda(), HT.cuda(), torch.from_numpy(pos).cuda(), fD, fT, tv, label,
+                         tD, tT, yD, yT)
+    torch.cuda.synchronize()
+    assert ctx.device_status() == 0
+    ctx.close()
+    ref = oracle.extract_features(_bits(WD), _bits(HD), _bits(WT), _bits(HT), pos, nthreads=8)
+    np.testing.assert_allclose(fD.cpu().numpy(), ref.feats_D, rtol=0, atol=2e-3)
+    np.testing.assert_allclose(fT.cpu().numpy(), ref.feats_T, rtol=0, atol=2e-3)
+    np.testing.assert_allclose(tv.cpu().numpy(), ref.tv, rtol=0, atol=2e-3)
+    np.testing.assert_allclose(yD.cpu().numpy().astype(np.float64).sum(axis=1), 1.0, atol=1e-4)
+    tDg, tTg, lab = tD.cpu().numpy(), tT.cpu().numpy(), label.cpu().numpy()
+    tiedD, tiedT = ref.gap_D < 1e-3, ref.gap_T < 1e-3
+    assert np.all((tDg == ref.token_D) | tiedD) and np.all((tTg == ref.token_T) | tiedT)
+    np.testing.assert_array_equal(lab, (tDg == tTg).astype(np.uint8))          # the rule, on the ids it reported
+    ok = ~(tiedD | tiedT)
+    np.testing.assert_array_equal(lab[ok], ref.label[ok])
+    assert ref.label[::3].all() and lab[::3].all()                              # the constructed agreements
+    return ref
+
+
+@pytest.mark.parametrize("path", [0, 1])
+@pytest.mark.parametrize("V,dD,dT,N", [(50, 16, 24, 1), (1000, 64, 136, 5), (4099, 72, 264, 19), (5000, 128, 64, 150)])
+def test_extract_features_small_shapes(oracle, path, V, dD, dT, N):
+    _extract_case(oracle, V, dD, dT, N, seed=V + N, path=path)
+
+
+def test_extract_features_full_size_heads(oracle):
+    wl = inputs.WORKLOADS["vicuna_b1"]
+    ref = _extract_case(oracle, wl.V, wl.d_D, wl.d_T, 12, seed=wl.seed + 60)
+    assert 0.0 < ref.tv.min() and ref.tv.max() <= 1.0
