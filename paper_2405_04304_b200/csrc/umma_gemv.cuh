@@ -15,9 +15,9 @@
 //     boxes, the ring) only feeds accumulator lanes nobody reads;
 //   * warp 0 producer (TMA, 128-byte swizzle; ring of LM-head stages as deep as shared memory allows,
 //     filled before the dependency wait), warp 1 MMA issuer (M = 128, N = tile rows, K = 16, two
-//     256-column TMEM buffers), warps 2-5 epilogue;
-//   * epilogue: all hidden rows sit in TMEM lane quadrant 0, which one warp may read: it copies the
-//     tile's logits to shared memory (row r by lane r), then all four warps fold them 32 at a time, one
+//     256-column TMEM buffers), warps 2-9 epilogue;
+//   * epilogue: all hidden rows sit in TMEM lane quadrant 0, which two of the eight warps may read: they
+//     copy the tile's logits to shared memory (row r by lane r), then all eight warps fold them 32 at a time, one
 //     logit per lane (soft-max statistics, top-10 and arg-max in parallel, warp_fold_block);
 //   * per-CTA records, ticket, last-CTA second phase and classifier exactly as in the streaming kernel.
 #pragma once
@@ -26,7 +26,8 @@
 
 namespace disco {
 
-constexpr int kGemvEpiWarps = 4;
+constexpr int kGemvEpiWarps = 8;
+constexpr int kGemvDumpWarps = kGemvEpiWarps / 4;   // epilogue warps that may read TMEM lane quadrant 0
 constexpr int kGemvThreads = (2 + kGemvEpiWarps) * 32;
 constexpr int kGemvMaxRows = 16;
 constexpr int kGemvMaxStages = 16;
@@ -100,7 +101,7 @@ umma_gemv_draft_kernel(const __grid_constant__ CUtensorMap tmap_W, const __grid_
         }
         for (int b = 0; b < 2; ++b) {
             mbar_init(&tmem_full[b], 1);
-            mbar_init(&tmem_empty[b], 1);
+            mbar_init(&tmem_empty[b], kGemvDumpWarps);
         }
         mbar_init(h_full, 1);
         fence_mbar_init();
@@ -180,7 +181,7 @@ umma_gemv_draft_kernel(const __grid_constant__ CUtensorMap tmap_W, const __grid_
     } else {
         // ------------------------------ epilogue ------------------------------
         constexpr int BAR_THREADS = kGemvEpiWarps * 32;
-        const int ew = warp - 2;    // 0..3: role in the reductions
+        const int ew = warp - 2;    // 0..7: role in the reductions
         const int quad = warp & 3;  // TMEM lane quadrant this warp may read
         const int tid = ew * 32 + lane;
         if (p.clf_H > 0) {  // classifier parameters -> shared, asynchronously; only the last CTA reads them
@@ -217,7 +218,7 @@ umma_gemv_draft_kernel(const __grid_constant__ CUtensorMap tmap_W, const __grid_
                 // the one warp that may read lane quadrant 0: row r of the tile's logits goes to shared memory
                 mbar_wait(&tmem_full[buf], (tile >> 1) & 1, p.status);
                 tc_fence_after();
-                for (int c = 0; c < nblocks; ++c) {
+                for (int c = ew >> 2; c < nblocks; c += kGemvDumpWarps) {   // the quadrant-0 warps share the blocks
                     float z[32];
                     tmem_ld32(tmem_base + buf * 256 + c * 32, z);
                     if (lane < p.R) {
@@ -264,7 +265,7 @@ umma_gemv_draft_kernel(const __grid_constant__ CUtensorMap tmap_W, const __grid_
                 const float4* sr = reinterpret_cast<const float4*>(wstate + (lane * RK + r) * kRecordWords);
                 rec.set(sr[0], sr[1], sr[2], sr[3]);
             }
-            warp_reduce_records(rec, 2);
+            warp_reduce_records(rec, ceil_log2(kGemvEpiWarps));
             warp_store_record(reinterpret_cast<float*>(p.part_rec + ((size_t)r * grid + blockIdx.x) * 4), rec, lane);
         }
 
