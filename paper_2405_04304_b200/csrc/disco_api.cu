@@ -518,13 +518,13 @@ int draft_step_common(disco_ctx* c, const void* W_D, const void* h_D, int d, int
     p.probs = probs;
     p.nll_sum = nll_sum;
     // Measured on B200 (Vicuna head, us per step for 1 / 2 / 3 / 4 / 6 / 8 sequences): the tensor-core kernel
-    // that folds the logits a block at a time 15.0 / 18.6 / 21.2 / 23.7 / 30.7 / 34.0, the one with a thread
-    // per hidden row 22.9 / 23.3 / 23.4 / 23.0 / 23.3 / 23.5: the first up to 3 sequences, the second beyond.
+    // that folds the logits a block at a time 14.8 / 17.0 / 19.4 / 21.3 / 24.8 / 26.8, the one with a thread
+    // per hidden row 22.9 / 23.3 / 23.4 / 23.0 / 23.3 / 23.5: the first up to 4 sequences, the second beyond.
     // The CUDA-core streaming kernel is within 5 % for one sequence and serves as the path without tensor maps.
     // (its hidden rows stay in shared memory: up to 48 KB of them, so that the ring keeps at least 8 stages)
     const bool gemv_ok = c->encode_tiled != nullptr && B <= kGemvMaxRows && !stats_only &&
                          (size_t)((d + kUmmaBK - 1) / kUmmaBK) * (B <= 8 ? 8 : 16) * 128 <= 48 * 1024;
-    const bool use_gemv = gemv_ok && (c->path == 3 || (c->path == 0 && B <= 3));
+    const bool use_gemv = gemv_ok && (c->path == 3 || (c->path == 0 && B <= 4));
     const bool use_umma = !use_gemv && umma_possible(c, B) && (c->path == 2 || c->path == 3 || (c->path == 0 && B >= 2));
     if (use_gemv) {
         rc = launch_gemv(c, p, st);
