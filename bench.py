@@ -418,9 +418,87 @@ def run_ours(args, rank: int, world: int):
     }
     if static is not None:
         out["static_sl_max"] = static
+    if wl.B == 1 and not args.no_static:
+        out["other_modes"] = other_modes(ctx, data, clf, wl, stream, device)
+        if ctx.device_status() != 0:
+            raise RuntimeError(f"device status {ctx.device_status()} after the other modes")
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         out["cpu_baseline"] = cpu_baseline(data, wl, budget_s=args.cpu_seconds)
     ctx.close()
+    return out
+
+
+def other_modes(ctx, data: Data, clf, wl, stream, device) -> dict:
+    """Average device time of the further entry points on the same inputs (one sequence, look-ahead
+    SL_max), each as a CUDA-graph replay of 20 calls with the draft LM head rotating: the draft step with
+    the perplexity rule, the sampled draft step, verification with sampling, and bulk feature extraction."""
+    B, S, V = wl.B, wl.sl_max, wl.V
+    R = B * (S + 1)
+    g = torch.Generator(device=device).manual_seed(12345)
+    u = torch.rand(B, generator=g, device=device)
+    ua = torch.rand(B * S, generator=g, device=device)
+    us = torch.rand(B, generator=g, device=device)
+    pos = torch.ones(B, dtype=torch.int32, device=device)
+    nd = torch.ones(B, dtype=torch.int32, device=device)
+    tok = torch.zeros(B, dtype=torch.int32, device=device)
+    conf = torch.zeros(B, device=device)
+    halt = torch.zeros(B, dtype=torch.uint8, device=device)
+    nll = torch.zeros(B, device=device)
+    ptok = torch.zeros(B, device=device)
+    dprobs = torch.zeros(S, B, V, device=device)
+    yT = torch.zeros(R, V, device=device)
+    ids = data.draft_full[0].reshape(-1).to(device)
+    na = torch.zeros(B, dtype=torch.int32, device=device)
+    nx = torch.zeros(B, dtype=torch.int32, device=device)
+    N = 256                                        # positions of the feature-extraction pass
+    HD = data.h_D.reshape(-1, wl.d_D)
+    HT = data.H_T.reshape(-1, wl.d_T)
+    N = min(N, HD.shape[0], HT.shape[0])
+    from paper_2405_04304_b200 import binding
+    fx = binding.Context(wl.V, wl.d_D, wl.d_T, max_batch=B, max_rows=N, clf_hidden=wl.H)   # scratch for N rows
+    fD = torch.zeros(N, 12, device=device); fT = torch.zeros(N, 12, device=device)
+    tv = torch.zeros(N, device=device); lab = torch.zeros(N, dtype=torch.uint8, device=device)
+    tD = torch.zeros(N, dtype=torch.int32, device=device); tT = torch.zeros(N, dtype=torch.int32, device=device)
+    yDn = torch.zeros(N, V, device=device); yTn = torch.zeros(N, V, device=device)
+    posN = torch.arange(N, dtype=torch.int32, device=device)
+    h = data.h_D[0, 0]
+    H_T = data.H_T[0]
+    calls = {
+        "draft_step_ppl": lambda i: ctx.draft_step_ppl(data.W_D[i % data.n_rot], h, nd, nll, 1e9, S, tok, conf, halt,
+                                                       stream=stream),
+        "draft_step_sample": lambda i: ctx.draft_step_sample(data.W_D[i % data.n_rot], h, pos, nd, clf, wl.tau, S, u,
+                                                             tok, conf, halt, dprobs[i % S], p_token=ptok,
+                                                             stream=stream),
+        "verify_sample": lambda i: ctx.verify_sample_ragged(data.W_T, H_T, ids, dprobs, None, B, R, ua, us, na, nx, yT,
+                                                            stream=stream),
+        "extract_features": lambda i: fx.extract_features(data.W_D[i % data.n_rot], HD[:N], data.W_T, HT[:N], posN,
+                                                           fD, fT, tv, lab, tD, tT, yDn, yTn, stream=stream),
+    }
+    out = {}
+    reps = 20
+    e0 = torch.cuda.Event(enable_timing=True)
+    e1 = torch.cuda.Event(enable_timing=True)
+    with torch.cuda.stream(stream):
+        for name, fn in calls.items():
+            for i in range(3):
+                fn(i)
+            stream.synchronize()
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph, stream=stream):
+                for i in range(reps):
+                    fn(i)
+            graph.replay()
+            stream.synchronize()
+            e0.record(stream)
+            graph.replay()
+            e1.record(stream)
+            stream.synchronize()
+            out[name + "_us"] = e0.elapsed_time(e1) * 1e3 / reps
+    if fx.device_status() != 0:
+        raise RuntimeError(f"device status {fx.device_status()} after feature extraction")
+    fx.close()
+    out["extract_features_positions"] = N
+    out["look_ahead"] = S
     return out
 
 
