@@ -17,56 +17,70 @@ constexpr int kSampleWarps = kSampleThreads / 32;
 // Inverse-CDF draw by one CTA of kSampleThreads threads from weights w(v) >= 0, v < V (a callable that
 // returns the same value whenever it is asked again): the smallest v whose running sum w(0) + .. + w(v)
 // exceeds u * (sum of all); if rounding leaves none, the last v with w(v) > 0; -1 if every weight is zero.
-// Every thread returns the token.  Three steps, each warp owning one contiguous segment of the row:
-//   A  segment totals (coalesced reads, lane-strided partial sums);
-//   B  the segment that holds the crossing, from the 16 totals;
-//   C  inside that segment only: each lane sums a contiguous piece, a warp scan finds the lane, and the
-//      lane walks its piece in vocabulary order.
-// sh: 24 doubles of shared memory; total (optional) receives the sum.
+// Every thread returns the token.  Three steps:
+//   A  each warp sums one contiguous segment of the row (coalesced reads, four partial sums per lane);
+//   B  every thread finds, from the 16 totals, the segment that holds u * total;
+//   C  that segment is dealt out again, a few consecutive entries per thread of the whole CTA: sums in
+//      vocabulary order, a scan over the CTA, and the thread that holds the crossing walks its entries.
+// sh: 40 doubles of shared memory; total (optional) receives the sum.
 template <typename WeightFn>
 __device__ __forceinline__ int block_sample_cdf(WeightFn w, int V, double u, double* sh, double* total_out) {
     const int t = threadIdx.x, lane = t & 31, warp = t >> 5;
     const int seg = ((V + kSampleWarps - 1) / kSampleWarps + 31) & ~31;  // entries per warp, whole 32s
     const int s0 = min(V, warp * seg), s1 = min(V, s0 + seg);
-    double* warp_tot = sh;                                     // [kSampleWarps]
-    int* found = reinterpret_cast<int*>(sh + kSampleWarps);    // [2]: token, last index with positive weight
+    double* warp_tot = sh;                                        // [kSampleWarps] segment totals
+    double* piece_tot = sh + kSampleWarps;                        // [kSampleWarps] step C: per-warp sums
+    int* found = reinterpret_cast<int*>(sh + 2 * kSampleWarps);   // [2]: token, last index with positive weight
     if (t == 0) {
         found[0] = -1;
         found[1] = -1;
     }
     // A
-    double part = 0.0;
+    double part[4] = {0.0, 0.0, 0.0, 0.0};
     int last = -1;
-#pragma unroll 4
-    for (int v = s0 + lane; v < s1; v += 32) {
-        const float x = w(v);
-        part += static_cast<double>(x);
-        if (x > 0.f) last = v;
+    for (int v0 = s0 + lane; v0 < s1; v0 += 128) {
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            const int v = v0 + 32 * k;
+            if (v < s1) {
+                const float x = w(v);
+                part[k] += static_cast<double>(x);
+                if (x > 0.f) last = max(last, v);
+            }
+        }
     }
+    double tot = (part[0] + part[1]) + (part[2] + part[3]);
 #pragma unroll
     for (int off = 16; off > 0; off >>= 1) {
-        part += __shfl_xor_sync(kFullMask, part, off);
+        tot += __shfl_xor_sync(kFullMask, tot, off);
         last = max(last, __shfl_xor_sync(kFullMask, last, off));
     }
-    if (lane == 0) warp_tot[warp] = part;
+    if (lane == 0) warp_tot[warp] = tot;
     __syncthreads();
     if (lane == 0 && last >= 0) atomicMax(&found[1], last);
-    // B
-    double before = 0.0, total = 0.0;
+    // B: the first segment whose running total exceeds the target (the same for every thread)
+    double total = 0.0;
+#pragma unroll
+    for (int k = 0; k < kSampleWarps; ++k) total += warp_tot[k];
+    const double target = u * total;
+    int win = -1;
+    double before = 0.0, run = 0.0;
 #pragma unroll
     for (int k = 0; k < kSampleWarps; ++k) {
-        const double wt = warp_tot[k];
-        if (k < warp) before += wt;
-        total += wt;
+        const double nxt = run + warp_tot[k];
+        if (win < 0 && nxt > target) {
+            win = k;
+            before = run;
+        }
+        run = nxt;
     }
-    const double target = u * total;
-    // C: exactly one segment starts at or below the target and ends above it
-    if (before <= target && before + part > target) {
-        const int piece = (seg / 32 + 3) & ~3;      // consecutive entries per lane
-        const int p0 = min(s1, s0 + lane * piece), p1 = min(s1, p0 + piece);
+    // C
+    if (win >= 0) {
+        const int c0 = min(V, win * seg), c1 = min(V, c0 + seg);
+        const int q = (c1 - c0 + kSampleThreads - 1) / kSampleThreads;   // consecutive entries per thread
+        const int p0 = min(c1, c0 + t * q), p1 = min(c1, p0 + q);
         double mine = 0.0;
         int mylast = -1;
-#pragma unroll 4
         for (int v = p0; v < p1; ++v) {
             const float x = w(v);
             mine += static_cast<double>(x);
@@ -78,24 +92,33 @@ __device__ __forceinline__ int block_sample_cdf(WeightFn w, int V, double u, dou
             const double o = __shfl_up_sync(kFullMask, incl, off);
             if (lane >= off) incl += o;
         }
-        incl += before;
-        const bool cross = (incl - mine) <= target && incl > target;
-        const unsigned who = __ballot_sync(kFullMask, cross);
-        if (who == 0u) {
-            // the scan adds in another order than step A: if its last bit falls short, the crossing is the
-            // segment's last entry with weight
-            if (lane == 0) found[0] = last;
-        } else if (lane == __ffs(who) - 1) {
-            double run = incl - mine;
+        if (lane == 31) piece_tot[warp] = incl;
+        __syncthreads();
+        double pre = before;
+#pragma unroll
+        for (int k = 0; k < kSampleWarps; ++k)
+            if (k < warp) pre += piece_tot[k];
+        incl += pre;
+        const double excl = incl - mine;
+        if (excl <= target && incl > target) {   // at most one thread
+            double r2 = excl;
             int tok = -1;
             for (int v = p0; v < p1; ++v) {
-                run += static_cast<double>(w(v));
-                if (run > target) {
+                r2 += static_cast<double>(w(v));
+                if (r2 > target) {
                     tok = v;
                     break;
                 }
             }
             found[0] = tok >= 0 ? tok : mylast;
+        }
+        // the scan adds in another order than step A: if its last bit falls short of the target, the
+        // crossing is the segment's last entry with weight
+        if (t == kSampleThreads - 1 && !(incl > target)) {
+            int sl = -1;
+            for (int v = c1 - 1; v >= c0 && sl < 0; --v)
+                if (w(v) > 0.f) sl = v;
+            found[0] = sl;
         }
     }
     __syncthreads();
@@ -108,7 +131,7 @@ __device__ __forceinline__ int block_sample_cdf(WeightFn w, int V, double u, dou
 // Rows of up to kSampleSmemFloats entries are staged in shared memory (one pass over global memory, eight
 // loads in flight per thread); longer rows are read from global memory by every step of the draw.
 constexpr int kSampleSmemFloats = 50 * 1024;
-constexpr int kSampleBatch = 8;
+constexpr int kSampleBatch = 16;
 inline size_t sample_smem_bytes(int V) { return V <= kSampleSmemFloats ? (size_t)V * sizeof(float) : 0; }
 
 // Draft side: the row probs[b, :] arrives holding the raw logits left by the LM-head pass; it is turned
@@ -119,7 +142,7 @@ static __global__ void __launch_bounds__(kSampleThreads)
 sample_rows_kernel(float* __restrict__ probs, const float* __restrict__ stats, const float* __restrict__ u,
                    const uint8_t* __restrict__ active, int V, int use_smem, int32_t* token, float* p_token) {
     extern __shared__ float row_s[];
-    __shared__ double sh[24];
+    __shared__ double sh[40];
     const int b = blockIdx.x;
     if (active && !active[b]) return;
     float* y = probs + (size_t)b * V;
@@ -174,7 +197,7 @@ struct SpecSampleParams {
 
 static __global__ void __launch_bounds__(kSampleThreads) speculative_sample_kernel(const SpecSampleParams p) {
     extern __shared__ float row_s[];
-    __shared__ double sh[24];
+    __shared__ double sh[40];
     __shared__ int s_n;
     const int b = blockIdx.x;
     int r0, r1;
