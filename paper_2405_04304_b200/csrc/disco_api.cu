@@ -453,6 +453,24 @@ int disco_set_kernel_path(disco_ctx* c, int which) {
 }  // extern "C"
 
 namespace {
+// Launch a small follow-up kernel with programmatic stream serialization (it waits with griddepcontrol.wait
+// before it reads anything), so that its launch latency hides behind the kernel before it.
+template <typename... KArgs, typename... Args>
+cudaError_t launch_after(const disco_ctx* c, void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
+                         Args... args) {
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = c->pdl ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, kern, static_cast<KArgs>(args)...);
+}
+
 // The sampling kernels stage one row of V floats in dynamic shared memory: raise their limit once per device.
 bool configure_sampling(disco_ctx* c) {
     static int configured_dev = -1;
@@ -559,9 +577,10 @@ int draft_step_common(disco_ctx* c, const void* W_D, const void* h_D, int d, int
     }
     if (probs && normalize) {
         dim3 grid((unsigned)std::min(64, (c->V + 255) / 256), (unsigned)B);
-        normalize_probs_kernel<<<grid, 256, 0, st>>>(probs, c->final_stats, active, c->V);
+        const cudaError_t e = launch_after(c, normalize_probs_kernel, grid, dim3(256), 0, st, probs,
+                                           (const float*)c->final_stats, active, c->V);
         c->launches += 1;
-        if (cudaGetLastError() != cudaSuccess) return DISCO_ERR_CUDA;
+        if (!cuda_ok(e, "normalize_probs_kernel launch")) return DISCO_ERR_CUDA;
     }
     return DISCO_OK;
 }
@@ -599,10 +618,11 @@ int disco_draft_step_sample(disco_ctx* c, const void* W_D, const void* h_D, int 
     // probs holds the logits: the kernel turns them into y^D and replaces the greedy token by the draw
     const size_t smem = sample_smem_bytes(c->V);
     if (!configure_sampling(c)) return DISCO_ERR_CUDA;
-    sample_rows_kernel<<<B, kSampleThreads, smem, static_cast<cudaStream_t>(stream)>>>(
-        probs, c->final_stats, u, active, c->V, smem ? 1 : 0, token, p_token);
+    const cudaError_t e = launch_after(c, sample_rows_kernel, dim3(B), dim3(kSampleThreads), smem,
+                                       static_cast<cudaStream_t>(stream), probs, (const float*)c->final_stats, u, active,
+                                       c->V, smem ? 1 : 0, token, p_token);
     c->launches += 1;
-    return cuda_ok(cudaGetLastError(), "sample_rows_kernel launch") ? DISCO_OK : DISCO_ERR_CUDA;
+    return cuda_ok(e, "sample_rows_kernel launch") ? DISCO_OK : DISCO_ERR_CUDA;
 }
 
 int disco_verify_sample_ragged(disco_ctx* c, const void* W_T, const void* H_T, const int32_t* draft_ids,
@@ -635,9 +655,10 @@ int disco_verify_sample_ragged(disco_ctx* c, const void* W_T, const void* H_T, c
     const size_t smem = sample_smem_bytes(c->V);
     sp.use_smem = smem ? 1 : 0;
     if (!configure_sampling(c)) return DISCO_ERR_CUDA;
-    speculative_sample_kernel<<<B, kSampleThreads, smem, static_cast<cudaStream_t>(stream)>>>(sp);
+    const cudaError_t e = launch_after(c, speculative_sample_kernel, dim3(B), dim3(kSampleThreads), smem,
+                                       static_cast<cudaStream_t>(stream), sp);
     c->launches += 1;
-    return cuda_ok(cudaGetLastError(), "speculative_sample_kernel launch") ? DISCO_OK : DISCO_ERR_CUDA;
+    return cuda_ok(e, "speculative_sample_kernel launch") ? DISCO_OK : DISCO_ERR_CUDA;
 }
 
 int disco_extract_features(disco_ctx* c, const void* W_D, const void* H_D, const void* W_T, const void* H_T,

@@ -143,6 +143,10 @@ sample_rows_kernel(float* __restrict__ probs, const float* __restrict__ stats, c
                    const uint8_t* __restrict__ active, int V, int use_smem, int32_t* token, float* p_token) {
     extern __shared__ float row_s[];
     __shared__ double sh[40];
+    // launched with programmatic stream serialization: resident early, reading only once the LM-head
+    // kernel before it has completed
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     const int b = blockIdx.x;
     if (active && !active[b]) return;
     float* y = probs + (size_t)b * V;
@@ -199,6 +203,8 @@ static __global__ void __launch_bounds__(kSampleThreads) speculative_sample_kern
     extern __shared__ float row_s[];
     __shared__ double sh[40];
     __shared__ int s_n;
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     const int b = blockIdx.x;
     int r0, r1;
     if (p.row_off) {

@@ -928,6 +928,8 @@ __global__ void __launch_bounds__((NW + 1) * 32, 1) stream_tail_kernel(const __g
 
 // probs[b, v] currently holds the raw logit; turn it into the soft-max probability.
 static __global__ void normalize_probs_kernel(float* probs, const float* final_stats, const uint8_t* active, int V) {
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     const int b = blockIdx.y;
     if (active && !active[b]) return;
     const float m = final_stats[2 * b], inv_Z = 1.f / final_stats[2 * b + 1];
