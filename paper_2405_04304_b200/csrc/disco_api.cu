@@ -192,7 +192,7 @@ int launch_umma(disco_ctx* c, const void* W, const void* H, int d, int R, float*
     // Vocabulary rows per tile: up to 256 for verification (its epilogue is a compare per logit); the
     // draft step's epilogue is heavy (soft-max, top-10), so it gets several small tiles per CTA and
     // the epilogue of one tile runs under the loads of the next.
-    const int tile_target = DRAFT ? getenv_int("DISCO_DRAFT_TILE", R <= 128 ? 128 : 256) : 256;
+    const int tile_target = (DRAFT && !STATS) ? getenv_int("DISCO_DRAFT_TILE", R <= 128 ? 128 : 256) : 256;
     p.TPC = std::max(1, (c->V + tile_target * p.CN - 1) / (tile_target * p.CN));
     p.TR = (c->V + p.CN * p.TPC - 1) / (p.CN * p.TPC);
     p.TRN = std::max(16, (p.TR + 15) / 16 * 16);
@@ -200,7 +200,7 @@ int launch_umma(disco_ctx* c, const void* W, const void* H, int d, int R, float*
     // Draft step with few rows: copies of the rows fill the other TMEM lane quadrants, so that the
     // epilogue (heavy there) runs on every warp scheduler.  Verification's epilogue is a compare per
     // logit and keeps the smaller stage instead.
-    p.rep = (DRAFT && R <= 64) ? (R <= 32 ? 4 : 2) : 1;
+    p.rep = (DRAFT && !STATS && R <= 64) ? (R <= 32 ? 4 : 2) : 1;   // the statistics-only epilogue is light too
     p.rows_pad = 128 / p.rep;
     // The A stage holds a_rows rows (rep copies, rows_pad rows apart).  The MMA still reads 128 rows from
     // its start: what lies behind the tile (other stages of the ring, always inside it) or between the
