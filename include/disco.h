@@ -47,7 +47,8 @@ enum {
     DISCO_ERR_UNSUPPORTED_SHAPE = -2, /* shape outside what the kernels handle */
     DISCO_ERR_WORKSPACE = -3,         /* batch or row count beyond what the context was created for */
     DISCO_ERR_CUDA = -4,              /* a CUDA runtime call failed */
-    DISCO_ERR_TIMEOUT = -5,           /* a bounded device-side wait ran out (device status word only) */
+    DISCO_ERR_TIMEOUT = -5,           /* a bounded device-side wait ran out (device status word only); the
+                                         context's counters are then undefined: destroy it */
     DISCO_ERR_STATIC_LIMIT = -6       /* size beyond the fixed scratch of disco_draft_step_static */
 };
 
