@@ -626,3 +626,49 @@ def test_extract_features_full_size_heads(oracle):
     wl = inputs.WORKLOADS["vicuna_b1"]
     ref = _extract_case(oracle, wl.V, wl.d_D, wl.d_T, 12, seed=wl.seed + 60)
     assert 0.0 < ref.tv.min() and ref.tv.max() <= 1.0
+
+
+def test_verify_sample_edge_cases(oracle):
+    """Identical distributions accept everything; draws at u = 0 and next to 1; a draft id outside the
+    vocabulary is reported through the status word and ends that sequence's acceptance, nothing else."""
+    V, d, B, SL = 3000, 64, 3, 4
+    R = B * (SL + 1)
+    W = inputs.lm_head(V, d, seed=5, std=0.25)
+    H = inputs.hidden(R, d, seed=6)
+    z = oracle.project(_bits(W), _bits(H), nthreads=8)
+    e = np.exp(z - z.max(axis=1, keepdims=True))
+    yT = e / e.sum(axis=1, keepdims=True)                                   # oracle's target rows
+    dp = np.zeros((SL, B, V), dtype=np.float32)
+    for b in range(B):
+        dp[:, b] = yT[b * (SL + 1): b * (SL + 1) + SL].astype(np.float32)   # draft distributions = target's
+    rng = np.random.default_rng(3)
+    ids = np.array([rng.choice(V, p=yT[b * (SL + 1) + i]) for b in range(B) for i in range(SL)], dtype=np.int32)
+    ua = rng.uniform(0.0, 0.99, size=B * SL).astype(np.float32)
+    us = np.array([0.0, float(np.nextafter(np.float32(1.0), np.float32(0.0))), 0.5], dtype=np.float32)
+
+    def run(ids_):
+        ctx = _ctx(V, 8, d, max_batch=8, max_rows=64)
+        n_acc = torch.full((B,), -7, dtype=torch.int32, device="cuda")
+        nxt = torch.full((B,), -7, dtype=torch.int32, device="cuda")
+        y = torch.zeros((R, V), dtype=torch.float32, device="cuda")
+        ctx.verify_sample_ragged(W.cuda(), H.cuda(), torch.from_numpy(ids_).cuda(), torch.from_numpy(dp).cuda(), None, B, R,
+                                 torch.from_numpy(ua).cuda(), torch.from_numpy(us).cuda(), n_acc, nxt, y)
+        torch.cuda.synchronize()
+        st = ctx.device_status()
+        ctx.close()
+        return n_acc.cpu().numpy(), nxt.cpu().numpy(), st
+
+    n, x, st = run(ids)
+    assert st == 0
+    np.testing.assert_array_equal(n, SL)                                     # ratio ~ 1 > u: everything passes
+    last = yT[np.arange(B) * (SL + 1) + SL]
+    for b in range(B):
+        assert _valid_draw(last[b], float(us[b]), int(x[b]))
+    assert x[0] == int(np.argmax(last[0] > 0))                               # u = 0: first entry with mass
+    assert last[1][x[1] + 1:].sum() < 1e-4                                   # u next to 1: only crumbs lie beyond
+
+    bad = ids.copy()
+    bad[SL + 2] = V                                                          # sequence 1, position 2
+    n, x, st = run(bad)
+    assert st == binding.ERR_INVALID_ARG
+    assert n[0] == SL and n[2] == SL and n[1] == 2
