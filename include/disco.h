@@ -237,9 +237,10 @@ int disco_verify_ragged(disco_ctx* ctx, const void* W_T, const void* H_T, const 
 /*
  * The same two operations for a caller whose per-step data lives in HOST memory (pinned memory
  * makes the copies asynchronous).  The LM heads and classifier parameters stay on the device;
- * the hidden states, integer inputs and every output are host pointers.  Each call copies its
- * inputs to staging owned by the context, runs the kernels, copies the results back and
- * synchronises the stream before returning.  feats / target_ids may be NULL.
+ * the hidden states, integer inputs and every output are host pointers.  Each call copies the
+ * hidden states to device staging owned by the context, passes the small inputs and outputs through
+ * pinned host memory that the GPU maps (the kernels read and write it in place), runs the kernels
+ * and synchronises the stream before returning.  feats / target_ids may be NULL.
  */
 int disco_draft_step_host(disco_ctx* ctx, const void* W_D /*device*/, const void* h_D_host, int B,
                           const int32_t* pos_host, const int32_t* n_drafted_host,

@@ -52,9 +52,12 @@ struct disco_ctx {
     void* encode_tiled;            // cuTensorMapEncodeTiled, resolved through the runtime
     // device staging for the *_host entry points
     void* stage_hidden;
-    int32_t* stage_int;   // pos | n_drafted | draft_ids | row_off | token | n_accept | bonus | target_ids
-    float* stage_float;   // conf | feats
-    uint8_t* stage_byte;  // active | halt
+    // Small inputs and outputs of the *_host entry points live in pinned host memory that the GPU maps:
+    // the kernels read and write it in place, so a host call costs one copy (the hidden states), one
+    // launch and one synchronisation.  *_h: host address, *_d: the same memory as the device sees it.
+    int32_t *stage_int_h, *stage_int_d;    // pos | n_drafted | token | draft_ids | row_off | n_accept | bonus | target_ids
+    float *stage_float_h, *stage_float_d;  // conf | feats
+    uint8_t *stage_byte_h, *stage_byte_d;  // active | halt
 };
 
 namespace {
@@ -394,9 +397,12 @@ int disco_create(disco_ctx** out, int V, int d_draft, int d_target, int max_batc
     ok = ok && cudaMalloc(&c->status, 256) == cudaSuccess;
     ok = ok && cudaMalloc(&c->final_stats, (size_t)c->part_rows * 2 * sizeof(float)) == cudaSuccess;
     ok = ok && cudaMalloc(&c->stage_hidden, hid) == cudaSuccess;
-    ok = ok && cudaMalloc(&c->stage_int, n_int * sizeof(int32_t)) == cudaSuccess;
-    ok = ok && cudaMalloc(&c->stage_float, (size_t)max_batch * (1 + kNFeat) * sizeof(float)) == cudaSuccess;
-    ok = ok && cudaMalloc(&c->stage_byte, (size_t)max_batch * 2 + 64) == cudaSuccess;
+    ok = ok && cudaHostAlloc(&c->stage_int_h, n_int * sizeof(int32_t), cudaHostAllocMapped) == cudaSuccess;
+    ok = ok && cudaHostAlloc(&c->stage_float_h, (size_t)max_batch * (1 + kNFeat) * sizeof(float), cudaHostAllocMapped) == cudaSuccess;
+    ok = ok && cudaHostAlloc(&c->stage_byte_h, (size_t)max_batch * 2 + 64, cudaHostAllocMapped) == cudaSuccess;
+    ok = ok && cudaHostGetDevicePointer(&c->stage_int_d, c->stage_int_h, 0) == cudaSuccess;
+    ok = ok && cudaHostGetDevicePointer(&c->stage_float_d, c->stage_float_h, 0) == cudaSuccess;
+    ok = ok && cudaHostGetDevicePointer(&c->stage_byte_d, c->stage_byte_h, 0) == cudaSuccess;
     ok = ok && cudaMemset(c->keys, 0, (size_t)max_rows * sizeof(unsigned long long)) == cudaSuccess;
     ok = ok && cudaMemset(c->ticket, 0, 1024) == cudaSuccess;
     // R rows take R * (sm_count / ceil(R / 128)) <= 128 * sm_count records
@@ -421,9 +427,9 @@ int disco_destroy(disco_ctx* c) {
     cudaFree(c->status);
     cudaFree(c->final_stats);
     cudaFree(c->stage_hidden);
-    cudaFree(c->stage_int);
-    cudaFree(c->stage_float);
-    cudaFree(c->stage_byte);
+    cudaFreeHost(c->stage_int_h);
+    cudaFreeHost(c->stage_float_h);
+    cudaFreeHost(c->stage_byte_h);
     delete c;
     return DISCO_OK;
 }
@@ -756,42 +762,36 @@ int disco_draft_step_host(disco_ctx* c, const void* W_D, const void* h_D_host, i
     if (B > c->max_batch) return DISCO_ERR_WORKSPACE;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const int mb = c->max_batch;
-    int32_t* d_pos = c->stage_int;
-    int32_t* d_nd = d_pos + mb;
-    int32_t* d_tok = d_nd + mb;
-    float* d_conf = c->stage_float;
-    float* d_feats = d_conf + mb;
-    uint8_t* d_act = c->stage_byte;
-    uint8_t* d_halt = d_act + mb;
-    bool ok = true;
-    ok = ok && cudaMemcpyAsync(c->stage_hidden, h_D_host, (size_t)B * c->d_draft * 2, cudaMemcpyHostToDevice, st) == cudaSuccess;
-    ok = ok && cudaMemcpyAsync(d_pos, pos_host, (size_t)B * 4, cudaMemcpyHostToDevice, st) == cudaSuccess;
-    ok = ok && cudaMemcpyAsync(d_nd, n_drafted_host, (size_t)B * 4, cudaMemcpyHostToDevice, st) == cudaSuccess;
-    if (active_host) ok = ok && cudaMemcpyAsync(d_act, active_host, (size_t)B, cudaMemcpyHostToDevice, st) == cudaSuccess;
-    if (!ok) return DISCO_ERR_CUDA;
-    int rc = disco_draft_step(c, W_D, c->stage_hidden, B, d_pos, d_nd, active_host ? d_act : nullptr, clf, tau,
-                              sl_max, d_tok, d_conf, d_halt, feats_host ? d_feats : nullptr, nullptr, stream);
+    int32_t* h_pos = c->stage_int_h;
+    int32_t* h_nd = h_pos + mb;
+    int32_t* h_tok = h_nd + mb;
+    float* h_conf = c->stage_float_h;
+    float* h_feats = h_conf + mb;
+    uint8_t* h_act = c->stage_byte_h;
+    uint8_t* h_halt = h_act + mb;
+    // host -> device view of the same words
+    auto dev_i = [c](int32_t* h) { return c->stage_int_d + (h - c->stage_int_h); };
+    auto dev_f = [c](float* h) { return c->stage_float_d + (h - c->stage_float_h); };
+    auto dev_b = [c](uint8_t* h) { return c->stage_byte_d + (h - c->stage_byte_h); };
+    std::memcpy(h_pos, pos_host, (size_t)B * 4);
+    std::memcpy(h_nd, n_drafted_host, (size_t)B * 4);
+    if (active_host) std::memcpy(h_act, active_host, (size_t)B);
+    if (cudaMemcpyAsync(c->stage_hidden, h_D_host, (size_t)B * c->d_draft * 2, cudaMemcpyHostToDevice, st) != cudaSuccess)
+        return DISCO_ERR_CUDA;
+    int rc = disco_draft_step(c, W_D, c->stage_hidden, B, dev_i(h_pos), dev_i(h_nd), active_host ? dev_b(h_act) : nullptr,
+                              clf, tau, sl_max, dev_i(h_tok), dev_f(h_conf), dev_b(h_halt),
+                              feats_host ? dev_f(h_feats) : nullptr, nullptr, stream);
     if (rc) return rc;
-    if (active_host) {
-        // inactive sequences keep the caller's values: copy back only what the kernel wrote
-        for (int b = 0; b < B; ++b) {
-            if (!active_host[b]) continue;
-            ok = ok && cudaMemcpyAsync(token_host + b, d_tok + b, 4, cudaMemcpyDeviceToHost, st) == cudaSuccess;
-            ok = ok && cudaMemcpyAsync(conf_host + b, d_conf + b, 4, cudaMemcpyDeviceToHost, st) == cudaSuccess;
-            ok = ok && cudaMemcpyAsync(halt_host + b, d_halt + b, 1, cudaMemcpyDeviceToHost, st) == cudaSuccess;
-            if (feats_host)
-                ok = ok && cudaMemcpyAsync(feats_host + (size_t)b * kNFeat, d_feats + (size_t)b * kNFeat,
-                                           kNFeat * 4, cudaMemcpyDeviceToHost, st) == cudaSuccess;
-        }
-    } else {
-        ok = ok && cudaMemcpyAsync(token_host, d_tok, (size_t)B * 4, cudaMemcpyDeviceToHost, st) == cudaSuccess;
-        ok = ok && cudaMemcpyAsync(conf_host, d_conf, (size_t)B * 4, cudaMemcpyDeviceToHost, st) == cudaSuccess;
-        ok = ok && cudaMemcpyAsync(halt_host, d_halt, (size_t)B, cudaMemcpyDeviceToHost, st) == cudaSuccess;
-        if (feats_host)
-            ok = ok && cudaMemcpyAsync(feats_host, d_feats, (size_t)B * kNFeat * 4, cudaMemcpyDeviceToHost, st) == cudaSuccess;
+    if (cudaStreamSynchronize(st) != cudaSuccess) return DISCO_ERR_CUDA;
+    // inactive sequences keep the caller's values: hand back only what the kernel wrote
+    for (int b = 0; b < B; ++b) {
+        if (active_host && !active_host[b]) continue;
+        token_host[b] = h_tok[b];
+        conf_host[b] = h_conf[b];
+        halt_host[b] = h_halt[b];
+        if (feats_host) std::memcpy(feats_host + (size_t)b * kNFeat, h_feats + (size_t)b * kNFeat, kNFeat * 4);
     }
-    ok = ok && cudaStreamSynchronize(st) == cudaSuccess;
-    return ok ? DISCO_OK : DISCO_ERR_CUDA;
+    return DISCO_OK;
 }
 
 int disco_verify_ragged_host(disco_ctx* c, const void* W_T, const void* H_T_host, const int32_t* draft_ids_host,
@@ -807,25 +807,24 @@ int disco_verify_ragged_host(disco_ctx* c, const void* W_T, const void* H_T_host
         if (row_off_host[b + 1] <= row_off_host[b]) return DISCO_ERR_INVALID_ARG;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const int mb = c->max_batch, mr = c->max_rows;
-    int32_t* d_ids = c->stage_int + 3 * (size_t)mb;
-    int32_t* d_off = d_ids + mr;
-    int32_t* d_nacc = d_off + mb + 1;
-    int32_t* d_bonus = d_nacc + mb;
-    int32_t* d_tids = d_bonus + mb;
-    bool ok = true;
-    ok = ok && cudaMemcpyAsync(c->stage_hidden, H_T_host, (size_t)R * c->d_target * 2, cudaMemcpyHostToDevice, st) == cudaSuccess;
-    if (R > B) ok = ok && cudaMemcpyAsync(d_ids, draft_ids_host, (size_t)(R - B) * 4, cudaMemcpyHostToDevice, st) == cudaSuccess;
-    ok = ok && cudaMemcpyAsync(d_off, row_off_host, (size_t)(B + 1) * 4, cudaMemcpyHostToDevice, st) == cudaSuccess;
-    if (!ok) return DISCO_ERR_CUDA;
-    int rc = disco_verify_ragged(c, W_T, c->stage_hidden, d_ids, d_off, B, R, d_nacc, d_bonus,
-                                 target_ids_host ? d_tids : nullptr, stream);
+    int32_t* h_ids = c->stage_int_h + 3 * (size_t)mb;
+    int32_t* h_off = h_ids + mr;
+    int32_t* h_nacc = h_off + mb + 1;
+    int32_t* h_bonus = h_nacc + mb;
+    int32_t* h_tids = h_bonus + mb;
+    auto dev_i = [c](int32_t* h) { return c->stage_int_d + (h - c->stage_int_h); };   // device view of the same words
+    if (R > B) std::memcpy(h_ids, draft_ids_host, (size_t)(R - B) * 4);
+    std::memcpy(h_off, row_off_host, (size_t)(B + 1) * 4);
+    if (cudaMemcpyAsync(c->stage_hidden, H_T_host, (size_t)R * c->d_target * 2, cudaMemcpyHostToDevice, st) != cudaSuccess)
+        return DISCO_ERR_CUDA;
+    int rc = disco_verify_ragged(c, W_T, c->stage_hidden, dev_i(h_ids), dev_i(h_off), B, R, dev_i(h_nacc), dev_i(h_bonus),
+                                 target_ids_host ? dev_i(h_tids) : nullptr, stream);
     if (rc) return rc;
-    ok = ok && cudaMemcpyAsync(n_accept_host, d_nacc, (size_t)B * 4, cudaMemcpyDeviceToHost, st) == cudaSuccess;
-    ok = ok && cudaMemcpyAsync(bonus_host, d_bonus, (size_t)B * 4, cudaMemcpyDeviceToHost, st) == cudaSuccess;
-    if (target_ids_host)
-        ok = ok && cudaMemcpyAsync(target_ids_host, d_tids, (size_t)R * 4, cudaMemcpyDeviceToHost, st) == cudaSuccess;
-    ok = ok && cudaStreamSynchronize(st) == cudaSuccess;
-    return ok ? DISCO_OK : DISCO_ERR_CUDA;
+    if (cudaStreamSynchronize(st) != cudaSuccess) return DISCO_ERR_CUDA;
+    std::memcpy(n_accept_host, h_nacc, (size_t)B * 4);
+    std::memcpy(bonus_host, h_bonus, (size_t)B * 4);
+    if (target_ids_host) std::memcpy(target_ids_host, h_tids, (size_t)R * 4);
+    return DISCO_OK;
 }
 
 }  // extern "C"
