@@ -182,17 +182,6 @@ struct SoftmaxState {
     }
 };
 
-// Butterfly merge of one SoftmaxState per lane; every lane ends with the merged state.
-__device__ __forceinline__ void warp_merge_softmax(SoftmaxState& st) {
-#pragma unroll
-    for (int off = 16; off > 0; off >>= 1) {
-        const float m2 = __shfl_xor_sync(kFullMask, st.m, off);
-        const float Z2 = __shfl_xor_sync(kFullMask, st.Z, off);
-        const float S2 = __shfl_xor_sync(kFullMask, st.S, off);
-        st.merge(m2, Z2, S2);
-    }
-}
-
 // A block of up to 32 logits of one hidden row, one per lane (lanes >= n hold -inf), folded into the
 // warp's running state in one go: soft-max statistics by an integer max-reduction, one exponential per
 // lane and shuffle sums; arg-max by a ballot (lanes hold ascending vocabulary indices, so the lowest
@@ -264,24 +253,5 @@ struct RegTop10 {
         }
     }
 };
-
-// Every lane holds a descending list l[0..9] (values only, -inf = empty).  Lane k < 10 returns the k-th
-// largest of all 320 values; the lists are consumed.  Equal values are interchangeable here.
-__device__ __forceinline__ float warp_select_sorted(float (&l)[kTopK], int lane) {
-    float out = DISCO_NEG_INF;
-#pragma unroll 1
-    for (int r = 0; r < kTopK; ++r) {
-        const uint32_t mine = ordered_bits(l[0]);
-        const uint32_t best = __reduce_max_sync(kFullMask, mine);
-        const unsigned who = __ballot_sync(kFullMask, mine == best);
-        if (lane == r) out = from_ordered_bits(best);
-        if (lane == __ffs(who) - 1) {  // the owner of the winner moves its list up by one
-#pragma unroll
-            for (int k = 0; k + 1 < kTopK; ++k) l[k] = l[k + 1];
-            l[kTopK - 1] = DISCO_NEG_INF;
-        }
-    }
-    return out;
-}
 
 }  // namespace disco

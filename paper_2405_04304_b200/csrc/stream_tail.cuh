@@ -188,14 +188,6 @@ __device__ __forceinline__ void warp_reduce_records(LaneRecord& r, int levels) {
     r.S = Sc;
 }
 
-// The k-th largest logit for lane k < 10 (others: -inf) out of a reduced record.
-__device__ __forceinline__ float lane_pick(const LaneRecord& r, int lane) {
-    float sel = DISCO_NEG_INF;
-#pragma unroll
-    for (int k = 0; k < kTopK; ++k) sel = (lane == k) ? r.l[k] : sel;
-    return sel;
-}
-
 __device__ __forceinline__ int ceil_log2(int n) { return n <= 1 ? 0 : 32 - __clz(n - 1); }
 
 // Result of merging the partial records of one sequence: statistics and key in every lane, the k-th
