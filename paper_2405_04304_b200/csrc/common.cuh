@@ -252,6 +252,22 @@ struct RegTop10 {
             t[k] = hi;
         }
     }
+    // Two values at once.  With a >= b the (k+1)-th largest of the list and {a, b} is
+    //     max(t[k], min(t[k-1], a), min(t[k-2], b))          (t[-1] = t[-2] = +inf),
+    // the merge rule of two descending lists: three min/max per slot for two values instead of four, no
+    // carry chain, and the outer maximum is one three-input instruction.
+    __device__ __forceinline__ void push2(float z0, float z1) {
+        const float a = fmaxf(z0, z1), b = fminf(z0, z1);
+#pragma unroll
+        for (int k = kTopK - 1; k >= 2; --k) t[k] = max3(t[k], fminf(t[k - 1], a), fminf(t[k - 2], b));
+        t[1] = max3(t[1], fminf(t[0], a), b);
+        t[0] = fmaxf(t[0], a);
+    }
+    static __device__ __forceinline__ float max3(float x, float y, float z) {
+        float d;
+        asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(x), "f"(y), "f"(z));
+        return d;
+    }
 };
 
 }  // namespace disco

@@ -375,11 +375,14 @@ umma_tail_kernel(const __grid_constant__ CUtensorMap tmap_W, const __grid_consta
                             const float e = __expf(t);
                             st.Z += e;
                             st.S = (cbase + j < ncols) ? fmaf(e, t, st.S) : st.S;
-                            if (!STATS) top.push(z[j]);
                             if (z[j] > best_v) {
                                 best_v = z[j];
                                 best_i = v0 + cbase + j;
                             }
+                        }
+                        if (!STATS) {
+#pragma unroll
+                            for (int j = 0; j < 32; j += 2) top.push2(z[j], z[j + 1]);
                         }
                         if (p.probs && valid) {
                             float* dst = p.probs + (size_t)row * p.V + v0 + cbase;
