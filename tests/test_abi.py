@@ -51,6 +51,16 @@ def test_strerror_and_argument_checks_need_no_gpu(lib):
     assert lib.disco_create(ctypes.byref(h), 100, 8, 1 << 20, 1, 2, 10, 8) == binding.ERR_UNSUPPORTED_SHAPE
     assert lib.disco_destroy(None) == binding.ERR_INVALID_ARG
     assert h.value is None
+    # every per-step entry point refuses a null context before it touches the GPU
+    z = ctypes.c_void_p(None)
+    assert lib.disco_draft_step(None, z, z, 1, z, z, z, None, 0.5, 1, z, z, z, z, z, z) == binding.ERR_INVALID_ARG
+    assert lib.disco_draft_step_ppl(None, z, z, 1, z, z, z, 1.0, 1, z, z, z, z) == binding.ERR_INVALID_ARG
+    assert lib.disco_draft_step_sample(None, z, z, 1, z, z, z, None, 0.5, 1, z, z, z, z, z, z, z, z) == binding.ERR_INVALID_ARG
+    assert lib.disco_verify_ragged(None, z, z, z, z, 1, 1, z, z, z, z) == binding.ERR_INVALID_ARG
+    assert lib.disco_verify_sample_ragged(None, z, z, z, z, z, 1, 1, z, z, z, z, z, z, z) == binding.ERR_INVALID_ARG
+    assert lib.disco_extract_features(None, z, z, z, z, z, 1, z, z, z, z, z, z, z, z, z) == binding.ERR_INVALID_ARG
+    assert lib.disco_draft_step_host(None, z, z, 1, z, z, z, None, 0.5, 1, z, z, z, z, z) == binding.ERR_INVALID_ARG
+    assert lib.disco_verify_ragged_host(None, z, z, z, z, 1, 1, z, z, z, z) == binding.ERR_INVALID_ARG
 
 
 def test_oracle_and_library_share_no_code():
