@@ -521,6 +521,11 @@ def run_e2e(ctx, data: Data, clf, wl, Wm: int, K: int, stream, world: int):
     emitted = np.zeros(B, dtype=np.int64)
     trace = []
     rot = 0
+    # numpy views of the pinned buffers: the loop's own bookkeeping stays off torch's dispatcher
+    pos_np, nd_np, act_np, halt_np, nacc_np = pos.numpy(), nd.numpy(), act.numpy(), halt.numpy(), n_acc.numpy()
+    forced = None if data.forced_sl is None else data.forced_sl.numpy()
+    off = torch.zeros(B + 1, dtype=torch.int32).pin_memory()
+    off_np = off.numpy()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     for it in range(Wm + K):
         if it == Wm:
@@ -530,37 +535,36 @@ def run_e2e(ctx, data: Data, clf, wl, Wm: int, K: int, stream, world: int):
             e0.record(stream)
             h2d = d2h = 0
         d = data.idx(it)
-        act.fill_(1)
+        act_np[:] = 1
         sl = np.zeros(B, dtype=np.int64)
         for j in range(S):
-            pos.copy_(torch.from_numpy((emitted + j + 1).astype(np.int32)))
-            nd.fill_(j + 1)
+            pos_np[:] = emitted + (j + 1)
+            nd_np[:] = j + 1
             ctx.draft_step_host(data.W_D[rot % data.n_rot], h_D_host[d, j], pos, nd, clf, wl.tau, S, token, conf,
                                 halt, active=act if B > 1 else None, stream=stream)
             rot += 1
             h2d += B * (wl.d_D * 2 + 4 + 4 + 1)
-            n_act = int(act.sum())
-            d2h += n_act * (4 + 4 + 1)
-            a = act.numpy().astype(bool)
+            a = act_np.astype(bool)
+            d2h += int(a.sum()) * (4 + 4 + 1)
             sl[a] = j + 1
-            stop = (data.forced_sl[d].numpy() <= j + 1) if data.forced_sl is not None else halt.numpy().astype(bool)
-            act.copy_(torch.from_numpy((a & ~stop).astype(np.uint8)))
-            if not act.any():
+            stop = (forced[d] <= j + 1) if forced is not None else halt_np.astype(bool)
+            act_np[:] = a & ~stop
+            if not act_np.any():
                 break
         sl_t = torch.as_tensor(sl, dtype=torch.int32)
-        off = inputs.row_offsets(sl_t).pin_memory()
+        off_np[1:] = np.cumsum(sl + 1)
         if B == 1:
             H = H_T_host[d, : int(sl[0]) + 1]
             ids = data.draft_full[d, 0, : int(sl[0])].contiguous()
         else:
             H = inputs.pack_rows(H_T_host[d], sl_t, S)
             ids = inputs.pack_ids(data.draft_full[d].reshape(-1), sl_t, S)
-        R = int(off[-1])
+        R = int(off_np[-1])
         ctx.verify_ragged_host(data.W_T, H, ids if ids.numel() else None, off, B, R, n_acc, bonus, stream=stream)
         h2d += R * wl.d_T * 2 + (R - B) * 4 + (B + 1) * 4
         d2h += B * 8
-        emitted += n_acc.numpy().astype(np.int64) + 1
-        trace.append((sl.copy(), n_acc.numpy().copy()))
+        emitted += nacc_np.astype(np.int64) + 1
+        trace.append((sl.copy(), nacc_np.copy()))
     e1.record(stream)
     torch.cuda.synchronize()
     if world > 1:
