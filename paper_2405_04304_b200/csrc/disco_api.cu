@@ -141,6 +141,7 @@ int run_stream(disco_ctx* c, TailParams& p, int clf_H, cudaStream_t st) {
     if (!pl.ok) return DISCO_ERR_UNSUPPORTED_SHAPE;
     if (DRAFT && (pl.grid > c->max_grid || p.R > c->part_rows)) return DISCO_ERR_WORKSPACE;
     p.rows_per_cta = pl.rows_per_cta;
+    p.slab_rows = pl.rows_per_cta;
     p.rps = pl.rps;
     p.stages = pl.stages;
     p.slot_bytes = pl.slot_bytes;
@@ -299,6 +300,7 @@ int launch_gemv(disco_ctx* c, const TailParams& t, cudaStream_t st) {
     const int grid = c->sm_count;
     if (grid > c->part_slots || t.R > c->part_rows) return DISCO_ERR_WORKSPACE;
     g.TR = (t.V + grid - 1) / grid;
+    g.t.slab_rows = g.TR;
     g.tiles = (g.TR + 255) / 256;
     g.TRt = (g.TR + g.tiles - 1) / g.tiles;
     g.TRN = (g.TRt + 15) / 16 * 16;
@@ -499,7 +501,8 @@ bool configure_sampling(disco_ctx* c) {
 int draft_step_common(disco_ctx* c, const void* W_D, const void* h_D, int d, int B, int max_rows, const int32_t* pos,
                       const int32_t* n_drafted, const uint8_t* active, const disco_clf* clf, float tau,
                       int sl_max, int32_t* token, float* conf, uint8_t* halt, float* feats, float* probs,
-                      float* nll_sum, int stats_only, void* stream, bool normalize = true) {
+                      float* nll_sum, int stats_only, void* stream, bool normalize = true,
+                      const float* u_draw = nullptr, float* p_token = nullptr, bool* drew = nullptr) {
     if (!c || !W_D || !h_D) return DISCO_ERR_INVALID_ARG;
     if (!stats_only && (!pos || !n_drafted || !token || !conf || !halt)) return DISCO_ERR_INVALID_ARG;
     if (stats_only == 2 && (!pos || !feats)) return DISCO_ERR_INVALID_ARG;
@@ -550,6 +553,15 @@ int draft_step_common(disco_ctx* c, const void* W_D, const void* h_D, int d, int
                          (size_t)((d + kUmmaBK - 1) / kUmmaBK) * (B <= 8 ? 8 : 16) * 128 <= 48 * 1024;
     const bool use_gemv = gemv_ok && (c->path == 3 || (c->path == 0 && B <= 4));
     const bool use_umma = !use_gemv && umma_possible(c, B) && (c->path == 2 || c->path == 3 || (c->path == 0 && B >= 2));
+    // Sampled step: the kernels that end in a last-CTA second phase draw the token there (their records are
+    // at most 160 and in vocabulary order); the batched kernel leaves the draw to a follow-up kernel.
+    const bool fused_draw = u_draw && probs && !use_umma && (use_gemv || c->max_grid <= 160);
+    if (fused_draw) {
+        p.u_draw = u_draw;
+        p.p_token = p_token;
+        normalize = true;
+    }
+    if (drew) *drew = fused_draw;
     if (use_gemv) {
         rc = launch_gemv(c, p, st);
         if (rc) return rc;
@@ -618,9 +630,11 @@ int disco_draft_step_sample(disco_ctx* c, const void* W_D, const void* h_D, int 
                             int sl_max, const float* u, int32_t* token, float* p_token, float* conf, uint8_t* halt,
                             float* feats, float* probs, void* stream) {
     if (!c || !u || !probs) return DISCO_ERR_INVALID_ARG;
+    bool drew = false;
     int rc = draft_step_common(c, W_D, h_D, c->d_draft, B, c->max_batch, pos, n_drafted, active, clf, tau, sl_max,
-                               token, conf, halt, feats, probs, nullptr, 0, stream, false);
+                               token, conf, halt, feats, probs, nullptr, 0, stream, false, u, p_token, &drew);
     if (rc) return rc;
+    if (drew) return DISCO_OK;   // token drawn by the LM-head kernel's second phase, probs normalised
     // probs holds the logits: the kernel turns them into y^D and replaces the greedy token by the draw
     const size_t smem = sample_smem_bytes(c->V);
     if (!configure_sampling(c)) return DISCO_ERR_CUDA;

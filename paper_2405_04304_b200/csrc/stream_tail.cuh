@@ -58,6 +58,11 @@ struct TailParams {
     float* nll_sum;      // non-null: perplexity rule instead of the classifier (tau is then the perplexity bound)
     int stats_only;      // 1: arg-max and soft-max statistics only (pos, n_drafted, classifier unused); 2: token and
                          // features only (classifier, n_drafted unused)
+    // sampled draft step (non-null u_draw): the token is drawn from the soft-max by the second phase, from the
+    // per-CTA sums and the one slab of logits (in probs) that holds u * total; at most 160 CTAs
+    const float* u_draw;  // [B] uniforms in [0, 1)
+    float* p_token;       // [B] or null: probability of the drawn token
+    int slab_rows;        // vocabulary rows per CTA (the slab of record c starts at c * slab_rows)
     // verification
     const int32_t* draft_ids;
     const int32_t* row_off;  // null: uniform SL
@@ -196,6 +201,7 @@ struct MergedPartials {
     SoftmaxState st;
     unsigned long long key;
     float sel;
+    float zs[5];   // up to 160 records: sum of e^(z - m) over the slab of record j * 32 + lane (0 if none)
 };
 
 // Stamped records (80 bytes): five 16-byte pieces, each three payload words and the stamp of the launch
@@ -331,10 +337,12 @@ __device__ __forceinline__ MergedPartials warp_merge_partials(const float4* recs
         float Zc = 0.f, Sc = 0.f;
 #pragma unroll
         for (int j = 0; j < kPerLane; ++j) {
+            out.zs[j] = 0.f;
             if (q[j][0].y > 0.f) {
                 const float dm = q[j][0].x - M;
                 const float e = __expf(dm);
-                Zc = fmaf(q[j][0].y, e, Zc);
+                out.zs[j] = q[j][0].y * e;
+                Zc += out.zs[j];
                 Sc = fmaf(e, fmaf(dm, q[j][0].y, q[j][0].z), Sc);
             }
         }
@@ -575,6 +583,92 @@ __device__ __forceinline__ void warp_draft_epilogue(const SoftmaxState& st, unsi
     if (o.feats && lane < kNFeat) o.feats[(size_t)b * kNFeat + lane] = x;
 }
 
+// Inverse-CDF draw of one token by one warp, after warp_merge_partials: the records are in vocabulary
+// order (record c = the slab of rows [c * slab_rows, (c + 1) * slab_rows)), so the running sums of their
+// scaled Z locate the slab that holds u * Z; inside it the logits (row `logits` of the probs buffer, still
+// unnormalised) are exponentiated again, summed a contiguous piece per lane, scanned, and the lane that
+// holds the crossing walks its piece.  Returns the token (every lane) and its probability.
+__device__ __forceinline__ int warp_draw_token(const MergedPartials& mp, int NP, int slab_rows, int V,
+                                               const float* logits, float u, int lane, float* p_out) {
+    const float target = u * mp.st.Z;
+    // inclusive running sums in record order: a scan per group of 32 records, groups in sequence
+    float base = 0.f, my_before = 0.f;
+    int my_c = -1, last_c = -1;
+#pragma unroll
+    for (int j = 0; j < 5; ++j) {
+        float incl = mp.zs[j];
+#pragma unroll
+        for (int off = 1; off < 32; off <<= 1) {
+            const float o = __shfl_up_sync(kFullMask, incl, off);
+            if (lane >= off) incl += o;
+        }
+        incl += base;
+        const float excl = incl - mp.zs[j];
+        if (my_c < 0 && mp.zs[j] > 0.f && excl <= target && incl > target) {
+            my_c = j * 32 + lane;
+            my_before = excl;
+        }
+        if (mp.zs[j] > 0.f) last_c = j * 32 + lane;
+        base = __shfl_sync(kFullMask, incl, 31);
+    }
+    // the first record that crosses; rounding next to u = 1: the last record with mass
+    const unsigned who = __ballot_sync(kFullMask, my_c >= 0);
+    int c;
+    float before;
+    if (who) {
+        const int src = __ffs(who) - 1;
+        c = __shfl_sync(kFullMask, my_c, src);
+        before = __shfl_sync(kFullMask, my_before, src);
+    } else {
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) last_c = max(last_c, __shfl_xor_sync(kFullMask, last_c, off));
+        c = last_c;
+        before = DISCO_NEG_INF;   // nothing crosses: the walk below ends at the slab's last entry with mass
+    }
+    if (c < 0 || c >= NP) {
+        if (p_out) *p_out = 0.f;
+        return -1;
+    }
+    const int v0 = c * slab_rows, v1 = min(V, v0 + slab_rows);
+    const int piece = (v1 - v0 + 31) / 32;
+    const int p0 = min(v1, v0 + lane * piece), p1 = min(v1, p0 + piece);
+    float mine = 0.f;
+    for (int v = p0; v < p1; ++v) mine += __expf(__ldcg(logits + v) - mp.st.m);
+    float incl = mine;
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+        const float o = __shfl_up_sync(kFullMask, incl, off);
+        if (lane >= off) incl += o;
+    }
+    incl += before;
+    const bool cross = (incl - mine) <= target && incl > target;
+    unsigned w2 = __ballot_sync(kFullMask, cross);
+    // the re-summed slab may fall short of the record's sum in its last bit: then the last lane with mass
+    if (!w2) {
+        const unsigned has = __ballot_sync(kFullMask, mine > 0.f);
+        w2 = has ? (1u << (31 - __clz(has))) : 1u;
+    }
+    const int owner = __ffs(w2) - 1;
+    int tok = -1;
+    float pe = 0.f;
+    if (lane == owner) {
+        float run = incl - mine;
+        for (int v = p0; v < p1; ++v) {
+            const float e = __expf(__ldcg(logits + v) - mp.st.m);
+            if (e > 0.f) {   // remember the last entry with mass in case the sum never crosses
+                tok = v;
+                pe = e;
+            }
+            run += e;
+            if (run > target) break;
+        }
+    }
+    tok = __shfl_sync(kFullMask, tok, owner);
+    pe = __shfl_sync(kFullMask, pe, owner);
+    if (p_out) *p_out = pe / mp.st.Z;
+    return tok;
+}
+
 // Draft step, sequence b, in the last CTA, by ONE warp (the warps take different sequences): merge the
 // per-CTA records, then features, classifier and stopping rule.
 // feat16: kWarpScratchWords words of shared memory owned by the calling warp.
@@ -588,6 +682,14 @@ __device__ __forceinline__ void finalize_draft_seq(const TailParams& p, int b, i
     const DraftOutputs o{p.token, p.conf, p.halt, p.feats, p.final_stats, p.nll_sum, p.stats_only};
     warp_draft_epilogue(st, mp.key, mp.sel, fpos, n_drafted, p.tau, p.sl_max, feat16, clf_s, clf_s + Hc * kNFeat,
                         clf_s + Hc * (kNFeat + 1), clf_s + Hc * (kNFeat + 2), Hc, b, o, lane);
+    if (p.u_draw) {   // the greedy token is replaced by a draw from the distribution
+        float pt = 0.f;
+        const int tok = warp_draw_token(mp, grid, p.slab_rows, p.V, p.probs + (size_t)b * p.V, p.u_draw[b], lane, &pt);
+        if (lane == 0) {
+            p.token[b] = tok;
+            if (p.p_token) p.p_token[b] = pt;
+        }
+    }
 }
 
 // Verification: decode the arg-max keys, match the draft prefix, pick the bonus token.
