@@ -244,8 +244,10 @@ __device__ __forceinline__ void store_stamped_record(float4* rec, float m, float
 // ranked against each other.  More than 160 records, more than kMergePoolRecords such records or more
 // than kMergeCandidates candidates (many equal logits) fall back to pairwise list merges.
 // scratch: kWarpScratchWords - 16 words owned by the warp, 16-byte aligned.
+// want_top10 = false: statistics and key only (sel = -inf).
 __device__ __forceinline__ MergedPartials warp_merge_partials(const float4* recs, int NP, float* scratch, int lane,
-                                                              uint32_t stamp = 0u, int* status = nullptr) {
+                                                              uint32_t stamp = 0u, int* status = nullptr,
+                                                              bool want_top10 = true) {
     constexpr int kPerLane = 5;
     MergedPartials out;
     bool fast = NP <= 32 * kPerLane;
@@ -356,6 +358,10 @@ __device__ __forceinline__ MergedPartials warp_merge_partials(const float4* recs
             kFullMask, static_cast<uint32_t>(key >> 32) == khi ? static_cast<uint32_t>(key & 0xffffffffull) : 0u);
         out.st.m = M, out.st.Z = Zc, out.st.S = Sc;
         out.key = (static_cast<unsigned long long>(khi) << 32) | klo;
+        if (!want_top10) {
+            out.sel = DISCO_NEG_INF;
+            return out;
+        }
         // threshold: the head of rank 9 among the 32 lanes' heads (ties broken by lane)
         int rank = 0;
 #pragma unroll
@@ -676,7 +682,8 @@ __device__ __forceinline__ void finalize_draft_seq(const TailParams& p, int b, i
                                                    int lane) {
     const float fpos = p.pos ? static_cast<float>(p.pos[b]) : 0.f;  // issued early: hidden behind the merge
     const int n_drafted = p.n_drafted ? p.n_drafted[b] : 0;
-    const MergedPartials mp = warp_merge_partials(p.part_rec + (size_t)b * grid * 4, grid, feat16 + 16, lane);
+    const MergedPartials mp =
+        warp_merge_partials(p.part_rec + (size_t)b * grid * 4, grid, feat16 + 16, lane, 0u, nullptr, p.stats_only != 1);
     const int Hc = p.clf_H;
     const SoftmaxState st = mp.st;
     const DraftOutputs o{p.token, p.conf, p.halt, p.feats, p.final_stats, p.nll_sum, p.stats_only};

@@ -171,7 +171,8 @@ __device__ __forceinline__ void umma_finish_sequence(const DraftFinalParams& p, 
                                                      bool active, float fpos, int n_drafted, float* feat16,
                                                      const float* clf_s, uint32_t stamp, int* status, int lane) {
     const MergedPartials mp =
-        warp_merge_partials(part_rec + (size_t)b * NP * kStampedPieces, NP, feat16 + 16, lane, stamp, status);
+        warp_merge_partials(part_rec + (size_t)b * NP * kStampedPieces, NP, feat16 + 16, lane, stamp, status,
+                            p.stats_only != 1);
     if (!active) return;
     const int Hc = p.clf_H;
     const DraftOutputs o{p.token, p.conf, p.halt, p.feats, p.final_stats, p.nll_sum, p.stats_only};
