@@ -672,3 +672,51 @@ def test_verify_sample_edge_cases(oracle):
     n, x, st = run(bad)
     assert st == binding.ERR_INVALID_ARG
     assert n[0] == SL and n[2] == SL and n[1] == 2
+
+
+def test_look_ahead_is_monotone_in_the_threshold_at_full_size():
+    """Batched Starcoder shapes, no oracle needed: on the same stream of hidden states the look-ahead that the
+    stopping rule produces cannot grow with the threshold, the cap ends every sequence, and tau <= 0 never
+    halts before the cap (the static policy)."""
+    wl = inputs.WORKLOADS["starcoder_b256"]
+    B, S = wl.B, wl.sl_max
+    W = inputs.lm_head(wl.V, wl.d_D, seed=wl.seed, device="cuda")
+    params = make_clf(wl.H, seed=wl.seed + 3)
+    clf = to_gpu_clf(params)
+    hs = [inputs.hidden(B, wl.d_D, seed=wl.seed * 100 + j, device="cuda") for j in range(S)]
+    ctx = binding.Context(wl.V, wl.d_D, wl.d_T, max_batch=B, max_rows=B * (S + 1), clf_hidden=wl.H)
+    pos = torch.arange(B, dtype=torch.int32, device="cuda")
+    token = torch.zeros(B, dtype=torch.int32, device="cuda")
+    conf = torch.zeros(B, dtype=torch.float32, device="cuda")
+    halt = torch.zeros(B, dtype=torch.uint8, device="cuda")
+    sl, confs = {}, {}
+    for tau in (0.0, 0.3, 0.5, 0.7):
+        active = torch.ones(B, dtype=torch.uint8, device="cuda")
+        n = torch.zeros(B, dtype=torch.int64, device="cuda")
+        cs = []
+        for j in range(S):
+            nd = torch.full((B,), j + 1, dtype=torch.int32, device="cuda")
+            ctx.draft_step(W, hs[j], pos + j, nd, clf, tau, S, token, conf, halt, active=active)
+            torch.cuda.synchronize()
+            n += active.to(torch.int64)
+            cs.append(torch.where(active.bool(), conf, torch.full_like(conf, float("nan"))).cpu().numpy())
+            active = active & (1 - halt) if j + 1 < S else torch.zeros_like(active)
+            if not bool(active.any()):
+                break
+        sl[tau] = n.cpu().numpy()
+        confs[tau] = np.stack(cs)
+    assert ctx.device_status() == 0
+    ctx.close()
+    assert np.all(sl[0.0] == S)                                       # tau = 0: only the cap halts
+    assert np.all((sl[0.3] >= sl[0.5]) & (sl[0.5] >= sl[0.7]))
+    assert np.all((sl[0.7] >= 1) & (sl[0.3] <= S))
+    # the confidences do not depend on the threshold: wherever two runs both computed one, they agree bit for bit
+    a, b = confs[0.0][: confs[0.7].shape[0]], confs[0.7]
+    both = ~np.isnan(a) & ~np.isnan(b)
+    assert both.any() and np.array_equal(a[both], b[both])
+    # and each look-ahead is the first step whose confidence falls below the threshold
+    c0 = confs[0.0]
+    for tau in (0.3, 0.5, 0.7):
+        below = c0 < np.float32(tau)
+        first = np.where(below.any(axis=0), below.argmax(axis=0) + 1, S)
+        np.testing.assert_array_equal(sl[tau], np.minimum(first, S))
