@@ -18,6 +18,10 @@
  *     aborts.  Argument errors are detected on the host before anything is enqueued.
  *   - Unless a parameter says "host", data pointers are DEVICE pointers owned by the caller,
  *     16-byte aligned, and must stay valid until the stream has run the call.
+ *   - The LM heads and the classifier arrays are read-only inputs that the kernels start to read
+ *     BEFORE the preceding kernel of the stream has finished (programmatic dependent launch; everything
+ *     else is touched only after it has).  The work enqueued immediately before a call must therefore
+ *     not write them.
  *   - bf16 matrices are row-major with the hidden dimension contiguous; hidden widths are
  *     multiples of 8.
  *   - The library owns only the opaque context: scratch for cross-block reductions, a device
@@ -272,7 +276,8 @@ int disco_verify_ragged_host(disco_ctx* ctx, const void* W_T /*device*/, const v
  * returns DISCO_ERR_STATIC_LIMIT and does nothing.
  *
  * The first call on each device resolves the array's device address and raises the kernel's
- * shared-memory limit (with that device current); make that first call before any stream capture.
+ * shared-memory limit (with that device current; host threads that race to it take turns behind a
+ * lock); make that first call before any stream capture.
  * All calls on a device share the one array: it keeps the previous call's contents (the call clears
  * the words that must start at zero), and two calls that overlap on the GPU - different streams, or a
  * context-free call racing another - corrupt each other's results.  Issue them on one stream, or

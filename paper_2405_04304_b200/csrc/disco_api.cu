@@ -6,6 +6,7 @@
 #include <cstdio>
 #include <cstdlib>
 #include <cstring>
+#include <mutex>
 #include <new>
 
 #include "disco.h"
@@ -21,6 +22,17 @@ namespace {
 constexpr int kStreamWarps = 16;     // consumer warps of the streaming kernel
 constexpr int kMaxHidden = 16384;    // widest hidden dimension the kernels accept
 constexpr int kSlotTargetBytes = 6144;
+
+constexpr int kMaxDevices = 64;
+
+// One-time, per-device configuration of one kernel (its dynamic shared-memory limit).  Every template
+// instance of a launcher owns one of these; the lock makes first calls from several host threads, and
+// contexts on several devices, safe.
+struct KernelSetup {
+    std::mutex mu;
+    bool done[kMaxDevices] = {};
+    size_t dyn_limit[kMaxDevices] = {};
+};
 
 struct StreamPlan {
     int rows_per_cta, grid, rps, stages;
@@ -39,6 +51,7 @@ struct disco_ctx {
     int path;
     int pdl;  // launch the streaming kernel with programmatic stream serialization (DISCO_PDL=0 turns it off)
     long long launches;
+    cudaStream_t last_stream;  // stream of the most recent enqueue (disco_last_device_status waits for it only)
     // scratch for cross-block reductions
     int part_rows;  // rows the partial buffers can hold
     int max_grid;
@@ -70,12 +83,30 @@ inline bool cuda_ok(cudaError_t e, const char* what) {
     return false;
 }
 
-inline int getenv_int(const char* name, int dflt) {
-    const char* e = std::getenv(name);
-    return e ? std::atoi(e) : dflt;
-}
-
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+// Raise a kernel's dynamic shared-memory limit once per device: to `bytes`, or (bytes == 0) to all that the
+// device allows beside the kernel's static shared memory.  *limit receives the value in force.
+template <typename Kern>
+bool raise_smem_limit(const disco_ctx* c, KernelSetup& ks, Kern kern, size_t bytes, size_t* limit) {
+    if (c->device < 0 || c->device >= kMaxDevices) return false;
+    std::lock_guard<std::mutex> lock(ks.mu);
+    if (!ks.done[c->device]) {
+        size_t want = bytes;
+        if (want == 0) {
+            cudaFuncAttributes fa;
+            if (!cuda_ok(cudaFuncGetAttributes(&fa, kern), "cudaFuncGetAttributes")) return false;
+            want = c->smem_optin - fa.sharedSizeBytes;
+        }
+        if (!cuda_ok(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)want),
+                     "cudaFuncSetAttribute"))
+            return false;
+        ks.dyn_limit[c->device] = want;
+        ks.done[c->device] = true;
+    }
+    if (limit) *limit = ks.dyn_limit[c->device];
+    return true;
+}
 
 StreamPlan plan_stream(const disco_ctx* c, int V, int d, int RT, int clf_H) {
     StreamPlan pl{};
@@ -104,17 +135,9 @@ StreamPlan plan_stream(const disco_ctx* c, int V, int d, int RT, int clf_H) {
 template <int RT, bool DRAFT, int KC>
 int launch_stream(disco_ctx* c, TailParams& p, const StreamPlan& pl, cudaStream_t st) {
     auto kern = stream_tail_kernel<RT, DRAFT, kStreamWarps, KC>;
-    static int configured_dev = -1;
-    static size_t dyn_limit = 0;
-    if (configured_dev != c->device) {
-        cudaFuncAttributes fa;
-        if (!cuda_ok(cudaFuncGetAttributes(&fa, kern), "cudaFuncGetAttributes")) return DISCO_ERR_CUDA;
-        dyn_limit = c->smem_optin - fa.sharedSizeBytes;
-        if (!cuda_ok(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn_limit),
-                     "cudaFuncSetAttribute"))
-            return DISCO_ERR_CUDA;
-        configured_dev = c->device;
-    }
+    static KernelSetup setup;
+    size_t dyn_limit = 0;
+    if (!raise_smem_limit(c, setup, kern, 0, &dyn_limit)) return DISCO_ERR_CUDA;
     if (pl.smem > dyn_limit) return DISCO_ERR_UNSUPPORTED_SHAPE;
     // Programmatic dependent launch: the kernel may start while the preceding kernel of the stream is
     // still in its tail; it streams the LM head (never written by this library) and waits with
@@ -196,7 +219,7 @@ int launch_umma(disco_ctx* c, const void* W, const void* H, int d, int R, float*
     // Vocabulary rows per tile: up to 256 for verification (its epilogue is a compare per logit); the
     // draft step's epilogue is heavy (soft-max, top-10), so it gets several small tiles per CTA and
     // the epilogue of one tile runs under the loads of the next.
-    const int tile_target = (DRAFT && !STATS) ? getenv_int("DISCO_DRAFT_TILE", R <= 128 ? 128 : 256) : 256;
+    const int tile_target = (DRAFT && !STATS) ? (R <= 128 ? 128 : 256) : 256;
     p.TPC = std::max(1, (c->V + tile_target * p.CN - 1) / (tile_target * p.CN));
     p.TR = (c->V + p.CN * p.TPC - 1) / (p.CN * p.TPC);
     p.TRN = std::max(16, (p.TR + 15) / 16 * 16);
@@ -221,14 +244,9 @@ int launch_umma(disco_ctx* c, const void* W, const void* H, int d, int R, float*
     if (!encode_bf16_2d(c, &tmap_W, W, c->V, d, p.TRN) || !encode_bf16_2d(c, &tmap_H, H, R, d, p.a_rows))
         return DISCO_ERR_CUDA;
     auto kern = umma_tail_kernel<DRAFT, STATS>;
-    static int configured_dev = -1;
-    if (configured_dev != c->device) {
-        if (!cuda_ok(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                          kUmmaSmemBytes + umma_clf_bytes(DISCO_MAX_CLF_HIDDEN)),
-                     "cudaFuncSetAttribute(umma)"))
-            return DISCO_ERR_CUDA;
-        configured_dev = c->device;
-    }
+    static KernelSetup setup;
+    if (!raise_smem_limit(c, setup, kern, (size_t)kUmmaSmemBytes + umma_clf_bytes(DISCO_MAX_CLF_HIDDEN), nullptr))
+        return DISCO_ERR_CUDA;
     cudaLaunchConfig_t cfg{};
     cfg.gridDim = dim3((unsigned)(p.MT * p.CN));
     cfg.blockDim = dim3(kUmmaThreads);
@@ -261,17 +279,9 @@ int launch_umma(disco_ctx* c, const void* W, const void* H, int d, int R, float*
 template <int RK>
 int launch_gemv_rk(disco_ctx* c, GemvParams& g, const CUtensorMap& mW, const CUtensorMap& mH, cudaStream_t st) {
     auto kern = umma_gemv_draft_kernel<RK>;
-    static int configured_dev = -1;
-    static size_t dyn_limit = 0;
-    if (configured_dev != c->device) {
-        cudaFuncAttributes fa;
-        if (!cuda_ok(cudaFuncGetAttributes(&fa, kern), "cudaFuncGetAttributes(gemv)")) return DISCO_ERR_CUDA;
-        dyn_limit = c->smem_optin - fa.sharedSizeBytes;
-        if (!cuda_ok(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn_limit),
-                     "cudaFuncSetAttribute(gemv)"))
-            return DISCO_ERR_CUDA;
-        configured_dev = c->device;
-    }
+    static KernelSetup setup;
+    size_t dyn_limit = 0;
+    if (!raise_smem_limit(c, setup, kern, 0, &dyn_limit)) return DISCO_ERR_CUDA;
     // the ring takes what the fixed part leaves; it must hold at least two stages and the 16 KB that the
     // MMA reads behind the last box of hidden rows
     const size_t fixed = gemv_fixed_smem_bytes(RK, g.t.clf_H, g.t.d, g.h_rows);
@@ -438,10 +448,12 @@ int disco_destroy(disco_ctx* c) {
 
 int disco_last_device_status(disco_ctx* c, int* out) {
     if (!c || !out) return DISCO_ERR_INVALID_ARG;
+    // read and clear on the stream the context was last used on: nothing else on the device is waited for
     int v = 0;
-    if (cudaDeviceSynchronize() != cudaSuccess) return DISCO_ERR_CUDA;
-    if (cudaMemcpy(&v, c->status, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) return DISCO_ERR_CUDA;
-    if (cudaMemset(c->status, 0, sizeof(int)) != cudaSuccess) return DISCO_ERR_CUDA;
+    if (cudaMemcpyAsync(&v, c->status, sizeof(int), cudaMemcpyDeviceToHost, c->last_stream) != cudaSuccess ||
+        cudaMemsetAsync(c->status, 0, sizeof(int), c->last_stream) != cudaSuccess ||
+        cudaStreamSynchronize(c->last_stream) != cudaSuccess)
+        return DISCO_ERR_CUDA;
     *out = v;
     return DISCO_OK;
 }
@@ -481,16 +493,10 @@ cudaError_t launch_after(const disco_ctx* c, void (*kern)(KArgs...), dim3 grid, 
 
 // The sampling kernels stage one row of V floats in dynamic shared memory: raise their limit once per device.
 bool configure_sampling(disco_ctx* c) {
-    static int configured_dev = -1;
-    if (configured_dev == c->device) return true;
-    const int bytes = kSampleSmemFloats * (int)sizeof(float);
-    if (!cuda_ok(cudaFuncSetAttribute(sample_rows_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes),
-                 "cudaFuncSetAttribute(sample_rows)") ||
-        !cuda_ok(cudaFuncSetAttribute(speculative_sample_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes),
-                 "cudaFuncSetAttribute(speculative_sample)"))
-        return false;
-    configured_dev = c->device;
-    return true;
+    static KernelSetup rows_setup, spec_setup;
+    const size_t bytes = (size_t)kSampleSmemFloats * sizeof(float);
+    return raise_smem_limit(c, rows_setup, sample_rows_kernel, bytes, nullptr) &&
+           raise_smem_limit(c, spec_setup, speculative_sample_kernel, bytes, nullptr);
 }
 
 // Shared body of the LM-head + soft-max passes: B rows of hidden size d against the head W.
@@ -518,6 +524,7 @@ int draft_step_common(disco_ctx* c, const void* W_D, const void* h_D, int d, int
         if (rc) return rc;
     }
     cudaStream_t st = static_cast<cudaStream_t>(stream);
+    c->last_stream = st;
 
     TailParams p{};
     p.W = static_cast<const uint16_t*>(W_D);
@@ -653,6 +660,8 @@ int disco_verify_sample_ragged(disco_ctx* c, const void* W_T, const void* H_T, c
     if (B < 1 || R < B) return DISCO_ERR_INVALID_ARG;
     if (R > B && (!draft_ids || !draft_probs || !u_accept)) return DISCO_ERR_INVALID_ARG;
     if (B > c->max_batch || R > c->max_rows) return DISCO_ERR_WORKSPACE;
+    if (!row_off && R % B != 0) return DISCO_ERR_INVALID_ARG;
+    if (!aligned16(W_T) || !aligned16(H_T)) return DISCO_ERR_INVALID_ARG;
     // target distributions of all rows: LM head, soft-max statistics, normalised rows in y_T
     int rc = draft_step_common(c, W_T, H_T, c->d_target, R, c->max_rows, nullptr, nullptr, nullptr, nullptr, 0.f, 1,
                                target_ids, nullptr, nullptr, nullptr, y_T, nullptr, 1, stream);
@@ -671,7 +680,6 @@ int disco_verify_sample_ragged(disco_ctx* c, const void* W_T, const void* H_T, c
     sp.n_accept = n_accept;
     sp.next_token = next_token;
     sp.status = c->status;
-    if (!row_off && R % B != 0) return DISCO_ERR_INVALID_ARG;
     const size_t smem = sample_smem_bytes(c->V);
     sp.use_smem = smem ? 1 : 0;
     if (!configure_sampling(c)) return DISCO_ERR_CUDA;
@@ -688,6 +696,9 @@ int disco_extract_features(disco_ctx* c, const void* W_D, const void* H_D, const
         return DISCO_ERR_INVALID_ARG;
     if (N < 1) return DISCO_ERR_INVALID_ARG;
     if (N > c->max_rows) return DISCO_ERR_WORKSPACE;
+    // everything both passes will check, before the first of them is enqueued
+    if (!W_D || !H_D || !W_T || !H_T) return DISCO_ERR_INVALID_ARG;
+    if (!aligned16(W_D) || !aligned16(H_D) || !aligned16(W_T) || !aligned16(H_T)) return DISCO_ERR_INVALID_ARG;
     // the same LM-head pass as a draft step, once per model, without the classifier
     int rc = draft_step_common(c, W_D, H_D, c->d_draft, N, c->max_rows, pos, nullptr, nullptr, nullptr, 0.f, 1, token_D,
                                nullptr, nullptr, feats_D, y_D, nullptr, 2, stream);
@@ -709,6 +720,7 @@ int disco_verify_ragged(disco_ctx* c, const void* W_T, const void* H_T, const in
     if (R > B && !draft_ids) return DISCO_ERR_INVALID_ARG;
     if (R > c->max_rows) return DISCO_ERR_WORKSPACE;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
+    c->last_stream = st;
 
     TailParams p{};
     p.W = static_cast<const uint16_t*>(W_T);

@@ -13,6 +13,7 @@
 #include <cuda_runtime.h>
 
 #include <algorithm>
+#include <mutex>
 
 #include "disco.h"
 #include "stream_tail.cuh"
@@ -41,6 +42,7 @@ struct DeviceSetup {
     size_t dyn_limit[3];
 };
 DeviceSetup g_setup[kMaxDevices];
+std::mutex g_setup_mu;   // first calls from several host threads take turns at the set-up
 
 template <int RT, int KC>
 bool configure(DeviceSetup& s, int slot) {
@@ -50,13 +52,14 @@ bool configure(DeviceSetup& s, int slot) {
     const size_t limit = s.smem_optin - fa.sharedSizeBytes;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)limit) != cudaSuccess)
         return false;
-    s.dyn_limit[slot] = std::min(slot == 0 ? limit : s.dyn_limit[slot], limit);
+    s.dyn_limit[slot] = std::min(s.dyn_limit[slot], limit);   // the slot starts at the device's opt-in maximum
     return true;
 }
 
 // Once per device, with that device current: resolve the device address of the scratch array and
 // raise the shared-memory limit of the kernels.
 int setup_device(int dev) {
+    std::lock_guard<std::mutex> lock(g_setup_mu);
     DeviceSetup& s = g_setup[dev];
     if (s.ready) return DISCO_OK;
     void* ptr = nullptr;

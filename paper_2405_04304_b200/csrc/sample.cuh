@@ -214,7 +214,7 @@ static __global__ void __launch_bounds__(kSampleThreads) speculative_sample_kern
         r0 = b * (p.SL + 1);
         r1 = r0 + p.SL + 1;
     }
-    const bool bad = r0 < 0 || r1 <= r0 || r1 > p.R || (b == 0 && r0 != 0) || (b == p.B - 1 && r1 != p.R);
+    const bool bad = r0 < b || r1 <= r0 || r1 > p.R - (p.B - 1 - b) || (b == 0 && r0 != 0) || (b == p.B - 1 && r1 != p.R);
     if (bad) {
         if (threadIdx.x == 0) {
             record_status(p.status, DISCO_ERR_INVALID_ARG);

@@ -713,7 +713,9 @@ __device__ __forceinline__ void verify_one_sequence(const unsigned long long* ke
         r0 = b * (SL + 1);
         r1 = r0 + SL + 1;
     }
-    const bool bad = r0 < 0 || r1 <= r0 || r1 > R || (b == 0 && r0 != 0) || (b == B - 1 && r1 != R);
+    // every sequence owns at least one row, so row_off[b] >= b and R - row_off[b+1] >= B - 1 - b: offsets that
+    // break this would put the sequence's draft ids (which start at r0 - b) outside the [R - B] array
+    const bool bad = r0 < b || r1 <= r0 || r1 > R - (B - 1 - b) || (b == 0 && r0 != 0) || (b == B - 1 && r1 != R);
     if (bad) {
         if (lane == 0) {
             record_status(status, DISCO_ERR_INVALID_ARG);
@@ -854,6 +856,13 @@ __global__ void __launch_bounds__((NW + 1) * 32, 1) stream_tail_kernel(const __g
         }
         // scratch for the rank scatter: the warp's record slots (written for good only after the loop)
         float* fold_scratch = wstate + (warp * RT) * kRecordWords + 4;
+        // rows whose logits go to the optional probs output: none of a masked sequence's outputs is written
+        bool keep_logits[RT];
+#pragma unroll
+        for (int r = 0; r < RT; ++r) {
+            const int row = chunk * RT + r;
+            keep_logits[r] = DRAFT && p.probs && row < p.R && (!p.active || p.active[row]);
+        }
 
         // With one hidden row and a narrow head the warp keeps its share of h in registers.
         float hreg[KC > 0 ? KC : 1][8];
@@ -937,8 +946,7 @@ __global__ void __launch_bounds__((NW + 1) * 32, 1) stream_tail_kernel(const __g
                         for (int r = 0; r < RT; ++r) {
                             const float z = __fadd_rn(acc[g][r], 0.f);  // folds -0 into +0
                             if (mine) blk_v[r] = z;
-                            if (DRAFT && p.probs && lane == 0 && chunk * RT + r < p.R)
-                                p.probs[(size_t)(chunk * RT + r) * p.V + v] = z;
+                            if (keep_logits[r] && lane == 0) p.probs[(size_t)(chunk * RT + r) * p.V + v] = z;
                         }
                         if ((++cnt & 31) == 0) {  // 32 logits parked: fold them
 #pragma unroll

@@ -208,6 +208,9 @@ umma_gemv_draft_kernel(const __grid_constant__ CUtensorMap tmap_W, const __grid_
             best_i[r] = kNoIndex;
         }
         float* fold_scratch = wstate + (ew * RK) * kRecordWords + 4;
+        bool keep_logits[RK];   // rows whose logits go to the optional probs output (never a masked sequence's)
+#pragma unroll
+        for (int r = 0; r < RK; ++r) keep_logits[r] = p.probs && r < p.R && (!p.active || p.active[r]);
 
         for (int tile = 0; tile < tiles; ++tile) {
             const int buf = tile & 1;
@@ -242,7 +245,7 @@ umma_gemv_draft_kernel(const __grid_constant__ CUtensorMap tmap_W, const __grid_
                 for (int r = 0; r < RK; ++r) {
                     if (r < p.R) {
                         const float val = lane < n ? lg_s[r * kGemvRowStride + c * 32 + lane] : DISCO_NEG_INF;
-                        if (p.probs && lane < n) p.probs[(size_t)r * p.V + idx] = val;
+                        if (keep_logits[r] && lane < n) p.probs[(size_t)r * p.V + idx] = val;
                         warp_fold_block(val, idx, n, lane, st[r], best_v[r], best_i[r], top_v[r],
                                         fold_scratch + r * kRecordWords);
                     }

@@ -317,6 +317,8 @@ umma_tail_kernel(const __grid_constant__ CUtensorMap tmap_W, const __grid_consta
         const int row = m_tile * 128 + tile_row;
         const bool warp_has_rows = (m_tile * 128 + (quad * 32) % p.rows_pad) < p.R;
         const bool valid = row < p.R;
+        // the optional probs output receives the raw logits of this row, unless the sequence is masked
+        const bool keep_logits = DRAFT && p.probs && valid && (!f.active || f.active[row]);
         // stamp of this launch (the word is advanced by the last warp of the second phase)
         uint32_t stamp = 0u;
         if (DRAFT) stamp = *reinterpret_cast<volatile unsigned int*>(f.epoch) + 1u;
@@ -385,7 +387,7 @@ umma_tail_kernel(const __grid_constant__ CUtensorMap tmap_W, const __grid_consta
 #pragma unroll
                             for (int j = 0; j < 32; j += 2) top.push2(z[j], z[j + 1]);
                         }
-                        if (p.probs && valid) {
+                        if (keep_logits) {
                             float* dst = p.probs + (size_t)row * p.V + v0 + cbase;
                             if ((((uintptr_t)p.probs & 15) | ((p.V | (v0 + cbase)) & 3)) == 0 && cbase + 32 <= ncols) {  // 16-byte stores
 #pragma unroll

@@ -6,7 +6,8 @@ Tolerances
     whose two largest oracle logits are closer than GAP_EXEMPT may return either of the two;
   * probabilities, features and the classifier output agree within PROB_TOL absolute (fp32 accumulation
     over bf16 inputs against the fp64 oracle);
-  * a halt flag may differ only if the oracle's C lies within HALT_MARGIN of tau.
+  * a halt flag may differ only if the oracle's C lies within HALT_MARGIN of tau; every such case is counted
+    in COUNTS (printed at the end of the run by conftest.py), never passed over silently.
 """
 from __future__ import annotations
 
@@ -17,7 +18,31 @@ from paper_2405_04304_b200 import binding, inputs
 
 GAP_EXEMPT = 1e-3
 PROB_TOL = 2e-3
-HALT_MARGIN = 1e-4
+HALT_MARGIN = 1e-5
+
+# What the tolerances let through, summed over the whole run: halt flags compared / exempted (|C - tau| below
+# HALT_MARGIN) / exempted and actually different; arg-max positions exempted as near-ties; the largest
+# |C_gpu - C_oracle| seen.
+COUNTS = {"halt_checked": 0, "halt_exempt": 0, "halt_exempt_differs": 0, "argmax_near_tie": 0,
+          "verify_rows_near_tie": 0, "max_conf_err": 0.0}
+
+
+def top2_ids(oracle, W_bits, H_bits, rows, nthreads=8):
+    """{row: (best id, runner-up id)} from the oracle's logits of just these hidden rows."""
+    rows = [int(r) for r in rows]
+    if not rows:
+        return {}
+    z = oracle.project(W_bits, np.ascontiguousarray(H_bits[rows]), nthreads=nthreads)
+    out = {}
+    for i, r in enumerate(rows):
+        order = np.argsort(-z[i], kind="stable")[:2]
+        out[r] = (int(order[0]), int(order[-1]))
+    return out
+
+
+def near_tie_ids(oracle, W_bits, H_bits, gap):
+    """The two ids a near-tie row may return, for every row whose top-2 logit gap is below GAP_EXEMPT."""
+    return top2_ids(oracle, W_bits, H_bits, np.nonzero(np.asarray(gap) < GAP_EXEMPT)[0])
 
 
 def make_clf(H: int, seed: int, b2=None, zero_head: bool = False):
@@ -76,9 +101,12 @@ def check_draft(got, ref, tau, active=None):
             assert got["token"][b] == -7 and got["halt"][b] == 77 and got["conf"][b] == -7.0, \
                 f"inactive sequence {b} was written"
             assert np.all(got["feats"][b] == -7.0)
+            if got["probs"] is not None:
+                assert np.all(got["probs"][b] == -7.0), f"probs row of inactive sequence {b} was written"
             continue
         if ref.gap[b] < GAP_EXEMPT:
             exempt += 1
+            COUNTS["argmax_near_tie"] += 1
             assert got["token"][b] in ref.topk_ids[b, :2], f"seq {b}: token not among the tied top-2"
         else:
             assert got["token"][b] == ref.token[b], f"seq {b}: token {got['token'][b]} != {ref.token[b]}"
@@ -86,8 +114,14 @@ def check_draft(got, ref, tau, active=None):
                                    err_msg=f"features of sequence {b}")
         assert got["feats"][b, 11] == ref.feats[b, 11]          # the position is copied exactly
         assert abs(float(got["conf"][b]) - ref.conf[b]) <= PROB_TOL, f"seq {b}: conf"
+        COUNTS["max_conf_err"] = max(COUNTS["max_conf_err"], abs(float(got["conf"][b]) - ref.conf[b]))
+        COUNTS["halt_checked"] += 1
         if abs(ref.conf[b] - tau) >= HALT_MARGIN:
             assert got["halt"][b] == ref.halt[b], f"seq {b}: halt {got['halt'][b]} != {ref.halt[b]}"
+        else:
+            COUNTS["halt_exempt"] += 1
+            COUNTS["halt_exempt_differs"] += int(got["halt"][b] != ref.halt[b])
+            assert got["halt"][b] in (0, 1)
         if got["probs"] is not None:
             np.testing.assert_allclose(got["probs"][b], ref.probs[b], rtol=0, atol=PROB_TOL)
             assert abs(float(got["probs"][b].astype(np.float64).sum()) - 1.0) < 1e-4
@@ -121,9 +155,11 @@ def gpu_verify(ctx, W, H, draft_ids, B=None, SL=None, row_off=None, host=False, 
                 target_ids=None if tids is None else tids.cpu().numpy())
 
 
-def check_verify(got, ref, row_off, draft_ids):
-    """Compare with the oracle's VerifyResult.  Rows whose top-2 gap is below GAP_EXEMPT may differ; a
-    sequence with such a row at or before min(n_oracle, n_gpu) is checked for self-consistency only."""
+def check_verify(got, ref, row_off, draft_ids, tie_ids):
+    """Compare with the oracle's VerifyResult.  A row whose top-2 gap is below GAP_EXEMPT may return the
+    oracle's best id or its runner-up, nothing else (tie_ids: {row: (best, runner-up)} for every such row,
+    from near_tie_ids); a sequence with such a row at or before min(n_oracle, n_gpu) is checked against the
+    prefix rule applied to the ids the library reported."""
     row_off = np.asarray(row_off)
     draft_ids = np.asarray(draft_ids)
     B = row_off.shape[0] - 1
@@ -133,9 +169,13 @@ def check_verify(got, ref, row_off, draft_ids):
         r0, r1 = int(row_off[b]), int(row_off[b + 1])
         sl = r1 - r0 - 1
         tied = ref.gap[r0:r1] < GAP_EXEMPT
+        COUNTS["verify_rows_near_tie"] += int(tied.sum())
         if tid is not None:
             same = tid[r0:r1] == ref.target_ids[r0:r1]
             assert np.all(same | tied), f"seq {b}: target ids differ on rows that are not near-ties"
+            for r in np.nonzero(tied)[0] + r0:
+                assert int(tid[r]) in tie_ids[int(r)], f"row {r}: id {tid[r]} is neither of the tied top-2"
+
         n_g, n_o = int(got["n_accept"][b]), int(ref.n_accept[b])
         assert 0 <= n_g <= sl
         lim = min(n_g, n_o)
