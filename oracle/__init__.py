@@ -421,3 +421,98 @@ def extract_features(W_D, H_D, W_T, H_T, pos, k: int = K_TOP, nthreads: int = 1)
         _p(tv, ctypes.c_double), _p(label, ctypes.c_uint8), _p(tD, ctypes.c_int32), _p(tT, ctypes.c_int32),
         _p(gD, ctypes.c_double), _p(gT, ctypes.c_double), nthreads), "extract_features")
     return FeatureRows(fD, fT, tv, label, tD, tT, gD, gT)
+
+
+# --------------------------------------------------------------------------- whole iteration (Sec. 3)
+@dataclass
+class IterationResult:
+    token: np.ndarray       # [sl_max, B] int32, -1 where the sequence had stopped
+    conf: np.ndarray        # [sl_max, B] float64 (nan where not taken)
+    halt: np.ndarray        # [sl_max, B] uint8 (255 where not taken)
+    feats: np.ndarray       # [sl_max, B, k+2]
+    gap_D: np.ndarray       # [sl_max, B] top-2 logit gap of each draft step
+    sl: np.ndarray          # [B] int32 tokens drafted
+    n_accept: np.ndarray | None   # [B]
+    bonus: np.ndarray | None      # [B]
+    target_ids: np.ndarray | None  # [B, sl_max+1], -1 beyond sl[b]
+    gap_T: np.ndarray | None       # [B, sl_max+1]
+
+
+def _clf_args(clf: Classifier):
+    f = ctypes.c_float
+    return _p(clf.W1, f), _p(clf.b1, f), _p(clf.w2, f), _p(clf.b2, f), clf.H
+
+
+def draft_loop(W_D, h_D, pos0, clf: Classifier, tau: float, sl_max: int, sl_forced=None, k: int = K_TOP,
+               nthreads: int = 1) -> IterationResult:
+    """Draft phase of one iteration.  h_D: bf16 bits [sl_max, B, d]."""
+    W_D, h_D = _u16(W_D), _u16(h_D)
+    V, d = W_D.shape
+    S, B = h_D.shape[0], h_D.shape[1]
+    assert S == sl_max and h_D.shape[2] == d
+    pos0 = np.ascontiguousarray(pos0, dtype=np.int32)
+    forced = None if sl_forced is None else np.ascontiguousarray(sl_forced, dtype=np.int32)
+    token = np.full((S, B), -1, dtype=np.int32)
+    conf = np.full((S, B), np.nan)
+    halt = np.full((S, B), 255, dtype=np.uint8)
+    feats = np.full((S, B, k + 2), np.nan)
+    gap = np.full((S, B), np.nan)
+    sl = np.full(B, -1, dtype=np.int32)
+    _check(lib().oracle_draft_loop(
+        _p(W_D, ctypes.c_uint16), _p(h_D, ctypes.c_uint16), V, d, B, _p(pos0, ctypes.c_int32), *_clf_args(clf), k,
+        ctypes.c_float(tau), int(sl_max), _p(forced, ctypes.c_int32), _p(token, ctypes.c_int32),
+        _p(conf, ctypes.c_double), _p(halt, ctypes.c_uint8), _p(feats, ctypes.c_double), _p(gap, ctypes.c_double),
+        _p(sl, ctypes.c_int32), nthreads), "draft_loop")
+    return IterationResult(token, conf, halt, feats, gap, sl, None, None, None, None)
+
+
+def verify_padded(W_T, H_T, sl, draft, stride_b: int, stride_j: int, nthreads: int = 1):
+    """Verification in the fixed-shape layout.  H_T: bf16 bits [B, sl_max+1, d]; draft: int32, token j of
+    sequence b at draft.flat[b * stride_b + j * stride_j].  Returns (n_accept, bonus, target_ids, gap)."""
+    W_T, H_T = _u16(W_T), _u16(H_T)
+    V, d = W_T.shape
+    B, S1 = H_T.shape[0], H_T.shape[1]
+    sl = np.ascontiguousarray(sl, dtype=np.int32)
+    draft = None if draft is None else np.ascontiguousarray(draft, dtype=np.int32)
+    n = np.full(B, -1, dtype=np.int32)
+    bonus = np.full(B, -1, dtype=np.int32)
+    tid = np.full((B, S1), -1, dtype=np.int32)
+    gap = np.full((B, S1), np.nan)
+    _check(lib().oracle_verify_padded(
+        _p(W_T, ctypes.c_uint16), _p(H_T, ctypes.c_uint16), V, d, B, S1 - 1, _p(sl, ctypes.c_int32),
+        _p(draft, ctypes.c_int32), ctypes.c_longlong(stride_b), ctypes.c_longlong(stride_j), _p(n, ctypes.c_int32),
+        _p(bonus, ctypes.c_int32), _p(tid, ctypes.c_int32), _p(gap, ctypes.c_double), nthreads), "verify_padded")
+    return n, bonus, tid, gap
+
+
+def iteration(W_D, h_D, W_T, H_T, pos0, clf: Classifier, tau: float, sl_max: int, sl_forced=None, draft_ids=None,
+              k: int = K_TOP, nthreads: int = 1) -> IterationResult:
+    """One whole iteration: draft phase, then verification of what it drafted (draft_ids None) or of the
+    ids given ([B, sl_max])."""
+    W_D, h_D, W_T, H_T = _u16(W_D), _u16(h_D), _u16(W_T), _u16(H_T)
+    V, d_D = W_D.shape
+    d_T = W_T.shape[1]
+    S, B = h_D.shape[0], h_D.shape[1]
+    assert S == sl_max and H_T.shape == (B, S + 1, d_T) and W_T.shape[0] == V
+    pos0 = np.ascontiguousarray(pos0, dtype=np.int32)
+    forced = None if sl_forced is None else np.ascontiguousarray(sl_forced, dtype=np.int32)
+    ids = None if draft_ids is None else np.ascontiguousarray(draft_ids, dtype=np.int32)
+    assert ids is None or ids.shape == (B, S)
+    token = np.full((S, B), -1, dtype=np.int32)
+    conf = np.full((S, B), np.nan)
+    halt = np.full((S, B), 255, dtype=np.uint8)
+    feats = np.full((S, B, k + 2), np.nan)
+    gapD = np.full((S, B), np.nan)
+    sl = np.full(B, -1, dtype=np.int32)
+    n = np.full(B, -1, dtype=np.int32)
+    bonus = np.full(B, -1, dtype=np.int32)
+    tid = np.full((B, S + 1), -1, dtype=np.int32)
+    gapT = np.full((B, S + 1), np.nan)
+    _check(lib().oracle_iteration(
+        _p(W_D, ctypes.c_uint16), _p(h_D, ctypes.c_uint16), d_D, _p(W_T, ctypes.c_uint16), _p(H_T, ctypes.c_uint16),
+        d_T, V, B, _p(pos0, ctypes.c_int32), *_clf_args(clf), k, ctypes.c_float(tau), int(sl_max),
+        _p(forced, ctypes.c_int32), _p(ids, ctypes.c_int32), _p(token, ctypes.c_int32), _p(conf, ctypes.c_double),
+        _p(halt, ctypes.c_uint8), _p(feats, ctypes.c_double), _p(gapD, ctypes.c_double), _p(sl, ctypes.c_int32),
+        _p(n, ctypes.c_int32), _p(bonus, ctypes.c_int32), _p(tid, ctypes.c_int32), _p(gapT, ctypes.c_double),
+        nthreads), "iteration")
+    return IterationResult(token, conf, halt, feats, gapD, sl, n, bonus, tid, gapT)

@@ -488,6 +488,109 @@ int oracle_extract_features(const uint16_t* W_D, const uint16_t* H_D, int d_D,
     return ORACLE_OK;
 }
 
+// ---------------------------------------------------------------------------
+// One whole speculative iteration with the look-ahead decided on the fly (Sec. 3:
+// "immediately after generating any draft token" the classifier decides whether
+// the draft model generates the next token or the target takes over; never more
+// than SL_max draft tokens).
+// ---------------------------------------------------------------------------
+
+// Draft phase.  Sequence b drafts token i = 1, 2, ... from the hidden state
+// h_D[i-1, b] (h_D is [SL_max, B, d]: the draft model's body is not part of this
+// path, its outputs are given).  The token's position feature is pos0[b] + i,
+// where pos0[b] counts the tokens generated before this iteration, and its
+// n_drafted is i.  After token i:
+//   * sl_forced == null: the stopping rule of oracle_draft_step decides
+//     (classifier below tau, or i == SL_max);
+//   * sl_forced != null: the policy is overruled and sequence b drafts exactly
+//     min(sl_forced[b], SL_max) tokens (sl_forced[b] >= 1); the classifier still
+//     runs and its outputs are reported.
+// tau <= 0 is the static policy (SL = SL_max); tau > 1 gives SL = 1.
+// Outputs are step-major [SL_max, B] (feats [SL_max, B, k+2]); entries of steps a
+// sequence did not take are left untouched.  sl[b] = tokens drafted.
+int oracle_draft_loop(const uint16_t* W_D, const uint16_t* h_D, int V, int d, int B,
+                      const int32_t* pos0, const float* W1, const float* b1, const float* w2,
+                      const float* b2, int H, int k, float tau, int sl_max, const int32_t* sl_forced,
+                      int32_t* token, double* conf, uint8_t* halt, double* feats, double* gap,
+                      int32_t* sl, int nthreads) {
+    if (!W_D || !h_D || !pos0 || !token || !sl || V <= 0 || d <= 0 || B < 0 || sl_max < 1 || k <= 0)
+        return ORACLE_BAD_ARG;
+    for (int b = 0; b < B; ++b) {
+        if (sl_forced && sl_forced[b] < 1) return ORACLE_BAD_ARG;
+        sl[b] = 0;
+        for (int i = 1; i <= sl_max; ++i) {
+            const size_t at = (size_t)(i - 1) * B + b;   // step-major slot of (step i, sequence b)
+            const int32_t pos = pos0[b] + i, n_drafted = i;
+            uint8_t stop = 0;
+            int rc = oracle_draft_step(W_D, h_D + at * d, V, d, 1, &pos, &n_drafted, nullptr, W1, b1, w2, b2, H,
+                                       k, tau, sl_max, &token[at], conf ? &conf[at] : nullptr, &stop,
+                                       feats ? feats + at * (k + 2) : nullptr, nullptr,
+                                       gap ? &gap[at] : nullptr, nullptr, nthreads);
+            if (rc) return rc;
+            if (halt) halt[at] = stop;
+            sl[b] = i;
+            if (sl_forced ? (i >= sl_forced[b]) : (stop != 0)) break;
+        }
+    }
+    return ORACLE_OK;
+}
+
+// Verification of the tokens the draft phase produced, in the fixed-shape layout
+// the SL_max footnote of Sec. 3 points to: H_T is [B, SL_max+1, d] (row j of
+// sequence b is the target hidden state that predicts the token after draft
+// token j; only rows 0 .. sl[b] are looked at), the draft tokens are
+// draft[b * stride_b + j * stride_j], j < sl[b].  n_accept, bonus as in
+// oracle_accept_prefix.  target_ids / gap are [B, SL_max+1]; entries beyond
+// sl[b] are left untouched.
+int oracle_verify_padded(const uint16_t* W_T, const uint16_t* H_T, int V, int d, int B, int sl_max,
+                         const int32_t* sl, const int32_t* draft, long long stride_b, long long stride_j,
+                         int32_t* n_accept, int32_t* bonus, int32_t* target_ids, double* gap,
+                         int nthreads) {
+    if (!W_T || !H_T || !sl || !n_accept || !bonus || V <= 0 || d <= 0 || B < 0 || sl_max < 0)
+        return ORACLE_BAD_ARG;
+    std::vector<double> z(V);
+    for (int b = 0; b < B; ++b) {
+        const int SL = sl[b];
+        if (SL < 0 || SL > sl_max || (SL > 0 && !draft)) return ORACLE_BAD_ARG;
+        std::vector<int32_t> a(SL + 1), t(SL);
+        for (int j = 0; j < SL; ++j) t[j] = draft[(long long)b * stride_b + (long long)j * stride_j];
+        for (int j = 0; j <= SL; ++j) {
+            const size_t row = (size_t)b * (sl_max + 1) + j;
+            int rc = oracle_project(W_T, H_T + row * d, V, d, 1, z.data(), nthreads);
+            if (rc) return rc;
+            rc = oracle_argmax(z.data(), V, &a[j], gap ? &gap[row] : nullptr);
+            if (rc) return rc;
+            if (target_ids) target_ids[row] = a[j];
+        }
+        int rc = oracle_accept_prefix(SL ? t.data() : nullptr, a.data(), SL, &n_accept[b], &bonus[b]);
+        if (rc) return rc;
+    }
+    return ORACLE_OK;
+}
+
+// The iteration: draft phase, then verification of what it drafted.
+//   draft_ids == null: the target checks the tokens the draft phase produced
+//                      (token[j, b], the real loop);
+//   draft_ids != null: [B, SL_max] ids offered to the target instead (the synthetic
+//                      workloads plant the target's own tokens there, corrupted with a
+//                      given probability, to set the acceptance rate).
+int oracle_iteration(const uint16_t* W_D, const uint16_t* h_D, int d_D, const uint16_t* W_T,
+                     const uint16_t* H_T, int d_T, int V, int B, const int32_t* pos0,
+                     const float* W1, const float* b1, const float* w2, const float* b2, int H, int k,
+                     float tau, int sl_max, const int32_t* sl_forced, const int32_t* draft_ids,
+                     int32_t* token, double* conf, uint8_t* halt, double* feats, double* gap_D,
+                     int32_t* sl, int32_t* n_accept, int32_t* bonus, int32_t* target_ids, double* gap_T,
+                     int nthreads) {
+    int rc = oracle_draft_loop(W_D, h_D, V, d_D, B, pos0, W1, b1, w2, b2, H, k, tau, sl_max, sl_forced,
+                               token, conf, halt, feats, gap_D, sl, nthreads);
+    if (rc) return rc;
+    if (draft_ids)
+        return oracle_verify_padded(W_T, H_T, V, d_T, B, sl_max, sl, draft_ids, sl_max, 1, n_accept, bonus,
+                                    target_ids, gap_T, nthreads);
+    return oracle_verify_padded(W_T, H_T, V, d_T, B, sl_max, sl, token, 1, B, n_accept, bonus, target_ids,
+                                gap_T, nthreads);
+}
+
 int oracle_hardware_threads() { return (int)std::thread::hardware_concurrency(); }
 
 }  // extern "C"

@@ -628,3 +628,150 @@ def test_extract_features_is_two_draft_steps_a_label_and_a_distance(oracle):
     for n in range(N):
         v = oracle.verify_ragged(WT, HT[n:n + 1], np.zeros(0, np.int32), np.array([0, 1], np.int32))
         assert (v.bonus[0] == res.token_D[n]) == bool(res.label[n])
+
+
+# ------------------------------------------------------------------ whole iteration (Sec. 3)
+def _position_classifier(oracle, cut: float, H: int = 4):
+    """A hand-made 2-layer classifier that looks at the position feature only:
+    C = sigmoid(6 - 30 * relu(pos - cut)), i.e. about 0.998 up to pos = cut and below 1e-10 from cut + 1 on."""
+    W1 = np.zeros((H, 12), np.float32)
+    b1 = np.zeros(H, np.float32)
+    w2 = np.zeros(H, np.float32)
+    W1[0, 11] = 1.0
+    b1[0] = -cut
+    w2[0] = -30.0
+    return oracle.Classifier(W1, b1, w2, np.array([6.0], np.float32))
+
+
+def _iteration_inputs(V, dD, dT, B, S, seed):
+    g = torch.Generator().manual_seed(seed)
+    W_D = (torch.randn(V, dD, generator=g) * 0.3).to(torch.bfloat16)
+    W_T = (torch.randn(V, dT, generator=g) * 0.3).to(torch.bfloat16)
+    h_D = torch.randn(S, B, dD, generator=g).to(torch.bfloat16)
+    H_T = torch.randn(B, S + 1, dT, generator=g).to(torch.bfloat16)
+    bits = lambda t: inputs.bf16_bits(t.reshape(-1, t.shape[-1])).reshape(t.shape)
+    return bits(W_D), bits(W_T), bits(h_D), bits(H_T)
+
+
+def test_draft_loop_look_ahead_from_a_position_classifier(oracle):
+    """With a classifier that only reads the position, the look-ahead is known in closed form: drafting
+    stops at the first token whose position exceeds the cut, SL = clip(cut + 1 - pos0, 1, SL_max)."""
+    V, dD, dT, B, S = 50, 16, 24, 5, 6
+    W_D, W_T, h_D, H_T = _iteration_inputs(V, dD, dT, B, S, seed=1)
+    pos0 = np.array([0, 3, 7, 9, 20], np.int32)
+    clf = _position_classifier(oracle, cut=9.0)
+    res = oracle.draft_loop(W_D, h_D, pos0, clf, 0.5, S)
+    np.testing.assert_array_equal(res.sl, np.clip(9 + 1 - pos0, 1, S))     # [6, 6, 3, 1, 1]
+    for b in range(B):
+        n = res.sl[b]
+        assert np.all(res.halt[: n - 1, b] == 0) and res.halt[n - 1, b] == 1   # halts exactly at its last token
+        assert np.all(res.token[n:, b] == -1) and np.all(res.halt[n:, b] == 255)   # later steps never ran
+        np.testing.assert_array_equal(res.feats[:n, b, 11], pos0[b] + np.arange(1, n + 1))  # position feature
+        # each token is the plain single draft step on that hidden state
+        for i in range(n):
+            one = oracle.draft_step(W_D, h_D[i, b:b + 1], [pos0[b] + i + 1], [i + 1], clf, 0.5, S)
+            assert one.token[0] == res.token[i, b] and one.conf[0] == res.conf[i, b]
+
+
+def test_draft_loop_degenerate_policies(oracle):
+    """tau <= 0 never halts before the cap (static SL = SL_max); tau > 1 halts after the first token; a
+    forced look-ahead overrules the classifier but leaves its outputs in place."""
+    V, dD, dT, B, S = 40, 8, 8, 3, 5
+    W_D, W_T, h_D, H_T = _iteration_inputs(V, dD, dT, B, S, seed=2)
+    W1, b1, w2, b2 = inputs.classifier_params(8, 3)
+    clf = oracle.Classifier(W1.numpy(), b1.numpy(), w2.numpy(), b2.numpy())
+    pos0 = np.array([4, 0, 11], np.int32)
+    static = oracle.draft_loop(W_D, h_D, pos0, clf, 0.0, S)
+    np.testing.assert_array_equal(static.sl, [S] * B)
+    assert np.all(static.halt[: S - 1] == 0) and np.all(static.halt[S - 1] == 1)      # only the cap halts
+    np.testing.assert_array_equal(oracle.draft_loop(W_D, h_D, pos0, clf, 1.5, S).sl, [1] * B)
+    forced = oracle.draft_loop(W_D, h_D, pos0, clf, 1.5, S, sl_forced=[2, 9, 4])
+    np.testing.assert_array_equal(forced.sl, [2, S, 4])                                # capped at SL_max
+    np.testing.assert_array_equal(forced.token[:2, 0], static.token[:2, 0])            # same tokens either way
+    assert np.all(forced.halt[:2, 0] == 1)                                             # tau > 1: the classifier said halt
+    # the look-ahead cannot grow with the threshold
+    sls = [oracle.draft_loop(W_D, h_D, pos0, clf, t, S).sl for t in (0.3, 0.5, 0.7)]
+    assert np.all(sls[0] >= sls[1]) and np.all(sls[1] >= sls[2])
+
+
+def test_iteration_equals_the_host_closed_loop(oracle):
+    """The iteration is the loop a host would run with the single-step calls: draft steps until the halt
+    flag, then one ragged verification of the rows and ids kept.  Bit for bit."""
+    V, dD, dT, B, S = 64, 16, 24, 4, 5
+    W_D, W_T, h_D, H_T = _iteration_inputs(V, dD, dT, B, S, seed=3)
+    pos0 = np.array([2, 5, 6, 1], np.int32)
+    clf = _position_classifier(oracle, cut=7.0)
+    g = np.random.default_rng(3)
+    for ids in (None, g.integers(0, V, size=(B, S)).astype(np.int32)):
+        res = oracle.iteration(W_D, h_D, W_T, H_T, pos0, clf, 0.5, S, draft_ids=ids)
+        # host closed loop
+        active = np.ones(B, np.uint8)
+        sl = np.zeros(B, np.int64)
+        toks = np.full((S, B), -1, np.int32)
+        for j in range(S):
+            st = oracle.draft_step(W_D, h_D[j], pos0 + j + 1, np.full(B, j + 1, np.int32), clf, 0.5, S, active=active)
+            toks[j, active == 1] = st.token[active == 1]
+            sl[active == 1] = j + 1
+            active = (active.astype(bool) & (st.halt != 1)).astype(np.uint8)
+            if not active.any():
+                break
+        off = np.concatenate([[0], np.cumsum(sl + 1)]).astype(np.int32)
+        rows = np.concatenate([H_T[b, : sl[b] + 1] for b in range(B)])
+        offered = toks.T if ids is None else ids
+        packed = np.concatenate([offered[b, : sl[b]] for b in range(B)]).astype(np.int32)
+        v = oracle.verify_ragged(W_T, rows, packed, off)
+        np.testing.assert_array_equal(res.sl, sl)
+        np.testing.assert_array_equal(res.token, toks)
+        np.testing.assert_array_equal(res.n_accept, v.n_accept)
+        np.testing.assert_array_equal(res.bonus, v.bonus)
+        for b in range(B):
+            np.testing.assert_array_equal(res.target_ids[b, : sl[b] + 1], v.target_ids[off[b]:off[b + 1]])
+            assert np.all(res.target_ids[b, sl[b] + 1:] == -1)
+
+
+def test_iteration_reproduces_the_worked_example_of_fig1(oracle):
+    """Fig. 1 through the whole iteration: the look-ahead comes out as 5 (position classifier), the target
+    agrees with the first three offered tokens and not with the fourth: 3 accepted, 4 tokens emitted."""
+    with open(os.path.join(GOLDEN, "fig1_iteration.txt")) as f:
+        gold = dict(line.split() for line in f if line.strip() and not line.startswith("#"))
+    SL, accepted, emitted = int(gold["SL"]), int(gold["accepted"]), int(gold["emitted"])
+    V, dD, dT, S = 80, 16, 32, 8
+    W_D, W_T, h_D, H_T = _iteration_inputs(V, dD, dT, 1, S, seed=4)
+    clf = _position_classifier(oracle, cut=float(SL - 1))            # pos0 = 0: tokens 1..SL are drafted
+    free = oracle.verify_padded(W_T, H_T, [S], np.zeros((1, S), np.int32), S, 1)[2][0]    # the target's own tokens
+    ids = free[:S].copy().reshape(1, S)
+    ids[0, accepted] = (ids[0, accepted] + 1) % V                    # t4 wrong
+    ids[0, accepted + 1] = (ids[0, accepted + 1] + 1) % V            # t5 wrong
+    res = oracle.iteration(W_D, h_D, W_T, H_T, [0], clf, 0.5, S, draft_ids=ids)
+    assert res.sl[0] == SL and res.n_accept[0] == accepted and res.n_accept[0] + 1 == emitted
+    assert res.bonus[0] == free[accepted]
+    # offering the draft phase's own tokens instead: a random draft head agrees with nothing here
+    own = oracle.iteration(W_D, h_D, W_T, H_T, [0], clf, 0.5, S)
+    n = 0
+    while n < SL and own.token[n, 0] == free[n]:
+        n += 1
+    assert own.n_accept[0] == n and own.bonus[0] == free[n]
+
+
+def test_verify_padded_strides_and_unused_rows(oracle):
+    """The padded layout gives what the packed one gives; rows beyond sl[b] do not matter; the two id
+    layouts ([B, S] and step-major [S, B]) are read through their strides."""
+    V, dD, dT, B, S = 30, 8, 16, 3, 4
+    W_D, W_T, h_D, H_T = _iteration_inputs(V, dD, dT, B, S, seed=5)
+    sl = np.array([4, 0, 2], np.int32)
+    g = np.random.default_rng(5)
+    free = oracle.verify_padded(W_T, H_T, [S] * B, np.zeros((B, S), np.int32), S, 1)[2]
+    ids = free[:, :S].copy()
+    ids[0, 3] = (ids[0, 3] + 1) % V
+    n, bonus, tid, gap = oracle.verify_padded(W_T, H_T, sl, ids, S, 1)
+    np.testing.assert_array_equal(n, [3, 0, 2])
+    np.testing.assert_array_equal(bonus, [free[0, 3], free[1, 0], free[2, 2]])
+    n2, bonus2, _, _ = oracle.verify_padded(W_T, H_T, sl, np.ascontiguousarray(ids.T), 1, B)   # step-major ids
+    np.testing.assert_array_equal(n2, n)
+    np.testing.assert_array_equal(bonus2, bonus)
+    junk = H_T.copy()
+    junk[1, 1:] = g.integers(0, 65535, size=junk[1, 1:].shape).astype(np.uint16) & 0x7F7F   # rows no sequence owns
+    junk[2, 3:] = 0
+    n3, bonus3, _, _ = oracle.verify_padded(W_T, junk, sl, ids, S, 1)
+    np.testing.assert_array_equal(n3, n)
+    np.testing.assert_array_equal(bonus3, bonus)
