@@ -35,6 +35,7 @@
 #ifndef DISCO_H_
 #define DISCO_H_
 
+#include <stddef.h>
 #include <stdint.h>
 
 #ifdef __cplusplus
@@ -237,6 +238,66 @@ int disco_verify(disco_ctx* ctx, const void* W_T, const void* H_T, const int32_t
 int disco_verify_ragged(disco_ctx* ctx, const void* W_T, const void* H_T, const int32_t* draft_ids,
                         const int32_t* row_off, int B, int R,
                         int32_t* n_accept, int32_t* bonus, int32_t* target_ids, void* stream);
+
+/*
+ * The draft phase of one speculative iteration with the look-ahead decided on the device (Sec. 3: the
+ * classifier decides "immediately after generating any draft token" whether the next one is drafted; the
+ * footnote on SL_max: fixed tensor shapes).  One enqueue runs up to sl_max draft steps; step i (1-based) is
+ * disco_draft_step on the hidden states h_D[i-1] with pos = pos0 + i and n_drafted = i, for the sequences
+ * that have not stopped yet, and the halt flag it produces is consumed on the device: no host round trip
+ * between the steps.  A step that finds no sequence drafting any more returns at once.  (In this isolated
+ * tail the hidden state of every step is an input; a decoder would produce h_D[i] from token i-1.  Step i
+ * reads h_D[i-1] only after step i-1 has finished.)
+ *   W_D            bf16 [V, d_draft]            draft LM head
+ *   w_step_stride  bytes between the LM heads used by consecutive steps; 0 = the same head for every step
+ *                  (the normal case).  Non-zero lets a benchmark rotate through copies of the head so that
+ *                  no step finds it in L2; a multiple of 16
+ *   h_D            bf16 [sl_max, B, d_draft]    step-major
+ *   pos0           int32 [B]                    tokens generated before this iteration
+ *   sl_forced      int32 [B] or NULL            non-NULL overrules the stopping rule: sequence b drafts
+ *                  exactly min(sl_forced[b], sl_max) tokens (>= 1); the classifier still runs and reports
+ *   tau <= 0 is the static policy (SL = sl_max for every sequence); tau > 1 gives SL = 1.
+ * Outputs (device), step-major; entries of steps a sequence did not take are not written:
+ *   token, conf, halt [sl_max, B];  feats [sl_max, B, DISCO_NFEAT] or NULL
+ *   sl             int32 [B]                    tokens drafted by each sequence (1 .. sl_max)
+ * B <= max_batch of disco_create.  Errors as in disco_draft_step.
+ */
+int disco_draft_loop(disco_ctx* ctx, const void* W_D, size_t w_step_stride, const void* h_D, int B,
+                     const int32_t* pos0, const disco_clf* clf, float tau, int sl_max,
+                     const int32_t* sl_forced, int32_t* token, float* conf, uint8_t* halt, float* feats,
+                     int32_t* sl, void* stream);
+
+/*
+ * Verification in the fixed-shape layout, with the per-sequence look-ahead read from device memory (the sl
+ * output of disco_draft_loop): the second half of a device-resident iteration (Sec. 2, Fig. 1; Sec. 3).
+ *   H_T        bf16 [B, sl_max + 1, d_target]   row j of sequence b predicts the token after draft token j;
+ *                                               rows beyond sl[b] are projected but do not count
+ *   draft_ids  int32; draft token j of sequence b is draft_ids[b * ids_stride_b + j * ids_stride_j]
+ *              ([B, sl_max] row-major: strides (sl_max, 1); the step-major token output of disco_draft_loop:
+ *              strides (1, B)); may be NULL when sl_max == 0
+ *   sl         int32 [B], device, 0 <= sl[b] <= sl_max (outside: DISCO_ERR_INVALID_ARG in the status word,
+ *              -1 in that sequence's outputs)
+ * Outputs (device): n_accept [B], bonus [B] as in disco_verify;
+ *   target_ids int32 [B, sl_max + 1] or NULL: greedy target token of rows 0 .. sl[b] (others not written)
+ *   row_off    int32 [B + 1] or NULL: exclusive prefix sums of sl[b] + 1, the offsets of the packed rows
+ * B * (sl_max + 1) <= max_rows of disco_create.
+ */
+int disco_verify_sl(disco_ctx* ctx, const void* W_T, const void* H_T, const int32_t* draft_ids,
+                    long long ids_stride_b, long long ids_stride_j, const int32_t* sl, int B, int sl_max,
+                    int32_t* n_accept, int32_t* bonus, int32_t* target_ids, int32_t* row_off, void* stream);
+
+/*
+ * One whole iteration as one call: disco_draft_loop, then disco_verify_sl on what it drafted.
+ *   draft_ids  int32 [B, sl_max] or NULL.  NULL: the target checks the tokens the draft phase produced (the
+ *              real loop).  Non-NULL: these ids are offered to the target instead (synthetic workloads plant
+ *              the target's own tokens there, corrupted at a given rate, to set the acceptance rate).
+ * Other arguments and outputs as in the two calls above.  Nothing is read back by the host.
+ */
+int disco_iteration(disco_ctx* ctx, const void* W_D, size_t w_step_stride, const void* h_D, const void* W_T,
+                    const void* H_T, int B, const int32_t* pos0, const disco_clf* clf, float tau, int sl_max,
+                    const int32_t* sl_forced, const int32_t* draft_ids,
+                    int32_t* token, float* conf, uint8_t* halt, float* feats, int32_t* sl,
+                    int32_t* n_accept, int32_t* bonus, int32_t* target_ids, int32_t* row_off, void* stream);
 
 /*
  * The same two operations for a caller whose per-step data lives in HOST memory (pinned memory

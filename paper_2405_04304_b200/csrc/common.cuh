@@ -25,6 +25,43 @@ __device__ __forceinline__ void record_status(int* status, int code) {
 }
 
 // ------------------------------------------------------------------------------------------
+// draft steps chained on the device (the draft phase of an iteration as one enqueue, Sec. 3: after every
+// draft token the classifier decides whether the next one is drafted)
+// ------------------------------------------------------------------------------------------
+// A launch with alive != null is draft step `step` (1-based) of such a chain: the position feature of
+// sequence b is pos0[b] + step, its n_drafted is step, and it takes part iff it is still drafting (every
+// sequence at step 1; alive[b] afterwards, as the step before left it).  When a sequence has been finished
+// the launch records sl[b] = step and alive[b] = 0 if it stops here (the stopping rule, or the forced
+// look-ahead sl_forced[b] when that is given), 1 otherwise.  alive and sl are written by the predecessor
+// launch: they are read and written past L1 only, after the dependency wait.
+struct ChainLink {
+    uint8_t* alive;            // [B] library scratch; null: a plain draft step
+    int32_t* sl;               // [B] tokens drafted so far
+    const int32_t* pos0;       // [B] tokens generated before this iteration
+    const int32_t* sl_forced;  // [B] or null
+    int step;
+};
+
+__device__ __forceinline__ bool chain_seq_live(const ChainLink& c, const uint8_t* active, int b) {
+    if (c.alive) return c.step == 1 || __ldcg(c.alive + b) != 0;
+    return !active || active[b] != 0;
+}
+// Warp-collective: does any of the B sequences still draft?  (Always true outside a chain and at step 1.)
+__device__ __forceinline__ bool chain_any_live(const ChainLink& c, int B, int lane) {
+    if (!c.alive || c.step == 1) return true;
+    bool any = false;
+    for (int b = lane; b < B; b += 32) any = any || __ldcg(c.alive + b) != 0;
+    return __any_sync(0xffffffffu, any);
+}
+// By the thread that has just written sequence b's halt flag.
+__device__ __forceinline__ void chain_record(const ChainLink& c, int b, bool halt) {
+    if (!c.alive) return;
+    const bool stop = c.sl_forced ? (c.step >= c.sl_forced[b]) : halt;
+    __stcg(c.sl + b, c.step);
+    __stcg(c.alive + b, static_cast<uint8_t>(stop ? 0 : 1));
+}
+
+// ------------------------------------------------------------------------------------------
 // shared-memory barriers and bulk (TMA-unit) copies
 // ------------------------------------------------------------------------------------------
 __device__ __forceinline__ uint32_t smem_addr(const void* p) {

@@ -59,6 +59,7 @@ struct disco_ctx {
     unsigned int* ticket;
     int* status;
     float* final_stats;
+    uint8_t* chain_alive;          // [max_batch] draft phase on the device: which sequences still draft
     void* part_rec;                // draft step: 64-byte partial records, [sequence][CTA]
     void* stamped_rec;             // batched draft step: stamped 80-byte records, [sequence][CTA]; written by nothing else
     int part_slots;                // partials per row the buffers can hold
@@ -408,6 +409,7 @@ int disco_create(disco_ctx** out, int V, int d_draft, int d_target, int max_batc
     ok = ok && cudaMalloc(&c->ticket, 1024) == cudaSuccess;
     ok = ok && cudaMalloc(&c->status, 256) == cudaSuccess;
     ok = ok && cudaMalloc(&c->final_stats, (size_t)c->part_rows * 2 * sizeof(float)) == cudaSuccess;
+    ok = ok && cudaMalloc(&c->chain_alive, (size_t)max_batch + 64) == cudaSuccess;
     ok = ok && cudaMalloc(&c->stage_hidden, hid) == cudaSuccess;
     ok = ok && cudaHostAlloc(&c->stage_int_h, n_int * sizeof(int32_t), cudaHostAllocMapped) == cudaSuccess;
     ok = ok && cudaHostAlloc(&c->stage_float_h, (size_t)max_batch * (1 + kNFeat) * sizeof(float), cudaHostAllocMapped) == cudaSuccess;
@@ -438,6 +440,7 @@ int disco_destroy(disco_ctx* c) {
     cudaFree(c->ticket);
     cudaFree(c->status);
     cudaFree(c->final_stats);
+    cudaFree(c->chain_alive);
     cudaFree(c->stage_hidden);
     cudaFreeHost(c->stage_int_h);
     cudaFreeHost(c->stage_float_h);
@@ -508,9 +511,11 @@ int draft_step_common(disco_ctx* c, const void* W_D, const void* h_D, int d, int
                       const int32_t* n_drafted, const uint8_t* active, const disco_clf* clf, float tau,
                       int sl_max, int32_t* token, float* conf, uint8_t* halt, float* feats, float* probs,
                       float* nll_sum, int stats_only, void* stream, bool normalize = true,
-                      const float* u_draw = nullptr, float* p_token = nullptr, bool* drew = nullptr) {
+                      const float* u_draw = nullptr, float* p_token = nullptr, bool* drew = nullptr,
+                      const ChainLink* chain = nullptr) {
     if (!c || !W_D || !h_D) return DISCO_ERR_INVALID_ARG;
-    if (!stats_only && (!pos || !n_drafted || !token || !conf || !halt)) return DISCO_ERR_INVALID_ARG;
+    if (!stats_only && !chain && (!pos || !n_drafted)) return DISCO_ERR_INVALID_ARG;
+    if (!stats_only && (!token || !conf || !halt)) return DISCO_ERR_INVALID_ARG;
     if (stats_only == 2 && (!pos || !feats)) return DISCO_ERR_INVALID_ARG;
     if (!aligned16(W_D) || !aligned16(h_D)) return DISCO_ERR_INVALID_ARG;
     if (B < 1 || sl_max < 1) return DISCO_ERR_INVALID_ARG;
@@ -538,6 +543,7 @@ int draft_step_common(disco_ctx* c, const void* W_D, const void* h_D, int d, int
     p.pos = pos;
     p.n_drafted = n_drafted;
     p.active = active;
+    if (chain) p.chain = *chain;
     p.clf_W1 = clf->W1;
     p.clf_b1 = clf->b1;
     p.clf_w2 = clf->w2;
@@ -593,6 +599,7 @@ int draft_step_common(disco_ctx* c, const void* W_D, const void* h_D, int d, int
         f.nll_sum = nll_sum;
         f.stats_only = stats_only;
         f.epoch = c->ticket + 48;
+        if (chain) f.chain = *chain;
         rc = stats_only == 1 ? launch_umma<true, true>(c, W_D, h_D, d, B, probs, &f, nullptr, st)
                         : launch_umma<true>(c, W_D, h_D, d, B, probs, &f, nullptr, st);
         if (rc) return rc;
@@ -608,6 +615,68 @@ int draft_step_common(disco_ctx* c, const void* W_D, const void* h_D, int d, int
         if (!cuda_ok(e, "normalize_probs_kernel launch")) return DISCO_ERR_CUDA;
     }
     return DISCO_OK;
+}
+
+// Verification of R rows for B sequences.  pad == null: packed rows (row_off, or a uniform look-ahead SL);
+// pad != null: the fixed-shape layout, R = B * (SL + 1) rows of which the first sl[b] + 1 of each sequence
+// count (sl is device memory).
+int verify_common(disco_ctx* c, const void* W_T, const void* H_T, const int32_t* draft_ids, const int32_t* row_off,
+                  int B, int R, int SL, int32_t* n_accept, int32_t* bonus, int32_t* target_ids,
+                  const VerifyPadded* pad, void* stream) {
+    if (!aligned16(W_T) || !aligned16(H_T)) return DISCO_ERR_INVALID_ARG;
+    if (R > c->max_rows) return DISCO_ERR_WORKSPACE;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    c->last_stream = st;
+
+    TailParams p{};
+    p.W = static_cast<const uint16_t*>(W_T);
+    p.H = static_cast<const uint16_t*>(H_T);
+    p.V = c->V;
+    p.d = c->d_target;
+    p.R = R;
+    p.B = B;
+    p.SL = SL;
+    fill_scratch(c, p);
+    p.draft_ids = draft_ids;
+    p.row_off = row_off;
+    p.n_accept = n_accept;
+    p.bonus = bonus;
+    p.target_ids = target_ids;
+    if (pad) p.padded = *pad;
+    const bool use_umma = umma_possible(c, R) && (c->path == 2 || (c->path == 0 && R >= 2));
+    if (!use_umma) return run_stream<false>(c, p, 0, st);
+    if (B <= 16) {  // few sequences: the last CTA of the main kernel finishes the job, no second launch
+        UmmaParams fp{};
+        fp.fuse_final = 1;
+        fp.ticket = c->ticket + 32;
+        fp.draft_ids = draft_ids;
+        fp.row_off = row_off;
+        fp.B = B;
+        fp.SL = p.SL;
+        fp.n_accept = n_accept;
+        fp.bonus = bonus;
+        fp.target_ids = target_ids;
+        fp.padded = p.padded;
+        return launch_umma<false>(c, W_T, H_T, c->d_target, R, nullptr, nullptr, &fp, st);
+    }
+    int rc = launch_umma<false>(c, W_T, H_T, c->d_target, R, nullptr, nullptr, nullptr, st);
+    if (rc) return rc;
+    VerifyFinalParams f{};
+    f.keys = c->keys;
+    f.draft_ids = draft_ids;
+    f.row_off = row_off;
+    f.B = B;
+    f.SL = p.SL;
+    f.R = R;
+    f.n_accept = n_accept;
+    f.bonus = bonus;
+    f.target_ids = target_ids;
+    f.status = c->status;
+    f.ticket = c->ticket + 16;
+    f.padded = p.padded;
+    verify_finalize_kernel<<<(B + 3) / 4, 128, 0, st>>>(f);
+    c->launches += 1;
+    return cuda_ok(cudaGetLastError(), "verify_finalize_kernel launch") ? DISCO_OK : DISCO_ERR_CUDA;
 }
 
 }  // namespace
@@ -715,59 +784,10 @@ int disco_verify_ragged(disco_ctx* c, const void* W_T, const void* H_T, const in
                         const int32_t* row_off, int B, int R, int32_t* n_accept, int32_t* bonus,
                         int32_t* target_ids, void* stream) {
     if (!c || !W_T || !H_T || !n_accept || !bonus) return DISCO_ERR_INVALID_ARG;
-    if (!aligned16(W_T) || !aligned16(H_T)) return DISCO_ERR_INVALID_ARG;
     if (B < 1 || R < B) return DISCO_ERR_INVALID_ARG;
     if (R > B && !draft_ids) return DISCO_ERR_INVALID_ARG;
-    if (R > c->max_rows) return DISCO_ERR_WORKSPACE;
-    cudaStream_t st = static_cast<cudaStream_t>(stream);
-    c->last_stream = st;
-
-    TailParams p{};
-    p.W = static_cast<const uint16_t*>(W_T);
-    p.H = static_cast<const uint16_t*>(H_T);
-    p.V = c->V;
-    p.d = c->d_target;
-    p.R = R;
-    p.B = B;
-    p.SL = row_off ? 0 : (R / B - 1);
-    fill_scratch(c, p);
-    p.draft_ids = draft_ids;
-    p.row_off = row_off;
-    p.n_accept = n_accept;
-    p.bonus = bonus;
-    p.target_ids = target_ids;
-    const bool use_umma = umma_possible(c, R) && (c->path == 2 || (c->path == 0 && R >= 2));
-    if (!use_umma) return run_stream<false>(c, p, 0, st);
-    if (B <= 16) {  // few sequences: the last CTA of the main kernel finishes the job, no second launch
-        UmmaParams fp{};
-        fp.fuse_final = 1;
-        fp.ticket = c->ticket + 32;
-        fp.draft_ids = draft_ids;
-        fp.row_off = row_off;
-        fp.B = B;
-        fp.SL = p.SL;
-        fp.n_accept = n_accept;
-        fp.bonus = bonus;
-        fp.target_ids = target_ids;
-        return launch_umma<false>(c, W_T, H_T, c->d_target, R, nullptr, nullptr, &fp, st);
-    }
-    int rc = launch_umma<false>(c, W_T, H_T, c->d_target, R, nullptr, nullptr, nullptr, st);
-    if (rc) return rc;
-    VerifyFinalParams f{};
-    f.keys = c->keys;
-    f.draft_ids = draft_ids;
-    f.row_off = row_off;
-    f.B = B;
-    f.SL = p.SL;
-    f.R = R;
-    f.n_accept = n_accept;
-    f.bonus = bonus;
-    f.target_ids = target_ids;
-    f.status = c->status;
-    f.ticket = c->ticket + 16;
-    verify_finalize_kernel<<<(B + 3) / 4, 128, 0, st>>>(f);
-    c->launches += 1;
-    return cuda_ok(cudaGetLastError(), "verify_finalize_kernel launch") ? DISCO_OK : DISCO_ERR_CUDA;
+    return verify_common(c, W_T, H_T, draft_ids, row_off, B, R, row_off ? 0 : (R / B - 1), n_accept, bonus, target_ids,
+                         nullptr, stream);
 }
 
 int disco_verify(disco_ctx* c, const void* W_T, const void* H_T, const int32_t* draft_ids, int B, int SL,
@@ -776,6 +796,60 @@ int disco_verify(disco_ctx* c, const void* W_T, const void* H_T, const int32_t* 
     const long long R = (long long)B * (SL + 1);
     if (c && R > c->max_rows) return DISCO_ERR_WORKSPACE;
     return disco_verify_ragged(c, W_T, H_T, draft_ids, nullptr, B, (int)R, n_accept, bonus, target_ids, stream);
+}
+
+int disco_draft_loop(disco_ctx* c, const void* W_D, size_t w_step_stride, const void* h_D, int B, const int32_t* pos0,
+                     const disco_clf* clf, float tau, int sl_max, const int32_t* sl_forced, int32_t* token,
+                     float* conf, uint8_t* halt, float* feats, int32_t* sl, void* stream) {
+    if (!c || !W_D || !h_D || !pos0 || !token || !conf || !halt || !sl) return DISCO_ERR_INVALID_ARG;
+    if (B < 1 || sl_max < 1) return DISCO_ERR_INVALID_ARG;
+    if (!aligned16(W_D) || !aligned16(h_D) || (w_step_stride & 15u)) return DISCO_ERR_INVALID_ARG;
+    if (B > c->max_batch) return DISCO_ERR_WORKSPACE;
+    int rc = check_clf(c, clf);
+    if (rc) return rc;
+    const size_t h_step = (size_t)B * c->d_draft * 2;   // bytes of one step's hidden states
+    if (h_step & 15u) return DISCO_ERR_INVALID_ARG;
+    for (int step = 1; step <= sl_max; ++step) {
+        const size_t k = (size_t)(step - 1);
+        const ChainLink link{c->chain_alive, sl, pos0, sl_forced, step};
+        rc = draft_step_common(c, static_cast<const char*>(W_D) + k * w_step_stride,
+                               static_cast<const char*>(h_D) + k * h_step, c->d_draft, B, c->max_batch, nullptr,
+                               nullptr, nullptr, clf, tau, sl_max, token + k * B, conf + k * B, halt + k * B,
+                               feats ? feats + k * B * kNFeat : nullptr, nullptr, nullptr, 0, stream, true, nullptr,
+                               nullptr, nullptr, &link);
+        if (rc) return rc;
+    }
+    return DISCO_OK;
+}
+
+int disco_verify_sl(disco_ctx* c, const void* W_T, const void* H_T, const int32_t* draft_ids, long long ids_stride_b,
+                    long long ids_stride_j, const int32_t* sl, int B, int sl_max, int32_t* n_accept, int32_t* bonus,
+                    int32_t* target_ids, int32_t* row_off, void* stream) {
+    if (!c || !W_T || !H_T || !sl || !n_accept || !bonus) return DISCO_ERR_INVALID_ARG;
+    if (B < 1 || sl_max < 0) return DISCO_ERR_INVALID_ARG;
+    if (sl_max > 0 && !draft_ids) return DISCO_ERR_INVALID_ARG;
+    const long long R = (long long)B * (sl_max + 1);
+    if (R > c->max_rows) return DISCO_ERR_WORKSPACE;
+    const VerifyPadded pad{sl, ids_stride_b, ids_stride_j, row_off};
+    return verify_common(c, W_T, H_T, draft_ids, nullptr, B, (int)R, sl_max, n_accept, bonus, target_ids, &pad, stream);
+}
+
+int disco_iteration(disco_ctx* c, const void* W_D, size_t w_step_stride, const void* h_D, const void* W_T,
+                    const void* H_T, int B, const int32_t* pos0, const disco_clf* clf, float tau, int sl_max,
+                    const int32_t* sl_forced, const int32_t* draft_ids, int32_t* token, float* conf, uint8_t* halt,
+                    float* feats, int32_t* sl, int32_t* n_accept, int32_t* bonus, int32_t* target_ids,
+                    int32_t* row_off, void* stream) {
+    // everything the second half will check, before the first half is enqueued
+    if (!c || !W_T || !H_T || !n_accept || !bonus || !sl) return DISCO_ERR_INVALID_ARG;
+    if (!aligned16(W_T) || !aligned16(H_T)) return DISCO_ERR_INVALID_ARG;
+    if (B < 1 || sl_max < 1 || (long long)B * (sl_max + 1) > c->max_rows) return B < 1 || sl_max < 1 ? DISCO_ERR_INVALID_ARG : DISCO_ERR_WORKSPACE;
+    int rc = disco_draft_loop(c, W_D, w_step_stride, h_D, B, pos0, clf, tau, sl_max, sl_forced, token, conf, halt, feats,
+                              sl, stream);
+    if (rc) return rc;
+    if (draft_ids)
+        return disco_verify_sl(c, W_T, H_T, draft_ids, sl_max, 1, sl, B, sl_max, n_accept, bonus, target_ids, row_off,
+                               stream);
+    return disco_verify_sl(c, W_T, H_T, token, 1, B, sl, B, sl_max, n_accept, bonus, target_ids, row_off, stream);
 }
 
 int disco_draft_step_host(disco_ctx* c, const void* W_D, const void* h_D_host, int B, const int32_t* pos_host,

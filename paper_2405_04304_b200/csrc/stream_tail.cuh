@@ -24,6 +24,15 @@
 
 namespace disco {
 
+// Verification in the fixed-shape layout (the SL_max footnote of Sec. 3): every sequence owns SL + 1 rows
+// (SL = the cap), of which the first sl[b] + 1 count; sl[b] is device memory that the draft phase wrote.
+// Draft token j of sequence b is ids[b * stride_b + j * stride_j].
+struct VerifyPadded {
+    const int32_t* sl;        // [B]; null: not this mode
+    long long stride_b, stride_j;
+    int32_t* row_off_out;     // [B + 1] or null: exclusive prefix sums of sl[b] + 1 (offsets of the packed rows)
+};
+
 struct TailParams {
     // projection
     const uint16_t* W;   // bf16 [V, d]
@@ -43,6 +52,7 @@ struct TailParams {
     const int32_t* pos;
     const int32_t* n_drafted;
     const uint8_t* active;
+    ChainLink chain;     // alive != null: this launch is one step of a draft phase chained on the device
     const float* clf_W1;
     const float* clf_b1;
     const float* clf_w2;
@@ -70,6 +80,7 @@ struct TailParams {
     int32_t* n_accept;
     int32_t* bonus;
     int32_t* target_ids;
+    VerifyPadded padded;     // sl != null: fixed-shape rows, per-sequence look-ahead read from the device
 };
 
 constexpr int kRecordWords = 16;  // one partial record: m, Z, S, -, 10 logits, key (2 words)
@@ -536,6 +547,7 @@ struct DraftOutputs {
     float* nll_sum;  // non-null: perplexity rule (App. F) instead of the classifier
     int stats_only;  // 1: arg-max and soft-max statistics only (rows of a verification with sampling);
                      // 2: token and features, no classifier (bulk feature extraction)
+    ChainLink chain; // draft phase chained on the device: the look-ahead bookkeeping goes with the halt flag
 };
 __device__ __forceinline__ void warp_draft_epilogue(const SoftmaxState& st, unsigned long long key, float sel, float fpos,
                                                     int n_drafted, float tau, int sl_max, float* feat_s, const float* W1,
@@ -580,9 +592,11 @@ __device__ __forceinline__ void warp_draft_epilogue(const SoftmaxState& st, unsi
     }
     const float C = warp_halt_classifier(x, feat_s, W1, b1, w2, b2, Hc, lane);
     if (lane == 0) {
+        const bool halt = (C < tau) || (n_drafted >= sl_max);
         o.token[b] = key_index(key);
         o.conf[b] = C;
-        o.halt[b] = ((C < tau) || (n_drafted >= sl_max)) ? 1 : 0;
+        o.halt[b] = halt ? 1 : 0;
+        chain_record(o.chain, b, halt);
         o.final_stats[2 * b] = st.m;
         o.final_stats[2 * b + 1] = st.Z;
     }
@@ -680,13 +694,15 @@ __device__ __forceinline__ int warp_draw_token(const MergedPartials& mp, int NP,
 // feat16: kWarpScratchWords words of shared memory owned by the calling warp.
 __device__ __forceinline__ void finalize_draft_seq(const TailParams& p, int b, int grid, float* feat16, const float* clf_s,
                                                    int lane) {
-    const float fpos = p.pos ? static_cast<float>(p.pos[b]) : 0.f;  // issued early: hidden behind the merge
-    const int n_drafted = p.n_drafted ? p.n_drafted[b] : 0;
+    // issued early: hidden behind the merge
+    const float fpos = p.chain.alive ? static_cast<float>(p.chain.pos0[b] + p.chain.step)
+                                     : (p.pos ? static_cast<float>(p.pos[b]) : 0.f);
+    const int n_drafted = p.chain.alive ? p.chain.step : (p.n_drafted ? p.n_drafted[b] : 0);
     const MergedPartials mp =
         warp_merge_partials(p.part_rec + (size_t)b * grid * 4, grid, feat16 + 16, lane, 0u, nullptr, p.stats_only != 1);
     const int Hc = p.clf_H;
     const SoftmaxState st = mp.st;
-    const DraftOutputs o{p.token, p.conf, p.halt, p.feats, p.final_stats, p.nll_sum, p.stats_only};
+    const DraftOutputs o{p.token, p.conf, p.halt, p.feats, p.final_stats, p.nll_sum, p.stats_only, p.chain};
     warp_draft_epilogue(st, mp.key, mp.sel, fpos, n_drafted, p.tau, p.sl_max, feat16, clf_s, clf_s + Hc * kNFeat,
                         clf_s + Hc * (kNFeat + 1), clf_s + Hc * (kNFeat + 2), Hc, b, o, lane);
     if (p.u_draw) {   // the greedy token is replaced by a draw from the distribution
@@ -700,22 +716,36 @@ __device__ __forceinline__ void finalize_draft_seq(const TailParams& p, int b, i
 }
 
 // Verification: decode the arg-max keys, match the draft prefix, pick the bonus token.
-// One warp per sequence; lane j looks at row j of the sequence.
+// One warp per sequence; lane j looks at row j of the sequence.  Three row layouts: packed rows with
+// offsets (row_off), a uniform look-ahead SL, or the fixed-shape layout with the look-ahead read from
+// device memory (pad.sl).
 __device__ __forceinline__ void verify_one_sequence(const unsigned long long* keys, const int32_t* draft_ids,
                                                     const int32_t* row_off, int B, int SL, int R, int b,
                                                     int32_t* n_accept, int32_t* bonus, int32_t* target_ids,
-                                                    int* status, int lane) {
+                                                    int* status, int lane, const VerifyPadded& pad) {
     int r0, r1;
-    if (row_off) {
-        r0 = row_off[b];
-        r1 = row_off[b + 1];
-    } else {
+    long long id0, idj = 1;
+    bool bad;
+    if (pad.sl) {
+        const int s = __ldcg(pad.sl + b);
         r0 = b * (SL + 1);
-        r1 = r0 + SL + 1;
+        r1 = r0 + s + 1;
+        id0 = (long long)b * pad.stride_b;
+        idj = pad.stride_j;
+        bad = s < 0 || s > SL;
+    } else {
+        if (row_off) {
+            r0 = row_off[b];
+            r1 = row_off[b + 1];
+        } else {
+            r0 = b * (SL + 1);
+            r1 = r0 + SL + 1;
+        }
+        id0 = r0 - b;
+        // every sequence owns at least one row, so row_off[b] >= b and R - row_off[b+1] >= B - 1 - b: offsets that
+        // break this would put the sequence's draft ids (which start at r0 - b) outside the [R - B] array
+        bad = r0 < b || r1 <= r0 || r1 > R - (B - 1 - b) || (b == 0 && r0 != 0) || (b == B - 1 && r1 != R);
     }
-    // every sequence owns at least one row, so row_off[b] >= b and R - row_off[b+1] >= B - 1 - b: offsets that
-    // break this would put the sequence's draft ids (which start at r0 - b) outside the [R - B] array
-    const bool bad = r0 < b || r1 <= r0 || r1 > R - (B - 1 - b) || (b == 0 && r0 != 0) || (b == B - 1 && r1 != R);
     if (bad) {
         if (lane == 0) {
             record_status(status, DISCO_ERR_INVALID_ARG);
@@ -725,7 +755,6 @@ __device__ __forceinline__ void verify_one_sequence(const unsigned long long* ke
         return;
     }
     const int sl = r1 - r0 - 1;
-    const int32_t* draft = draft_ids + (r0 - b);
     int n_acc = -1, bonus_tok = -1;
     for (int j0 = 0; j0 <= sl; j0 += 32) {
         const int j = j0 + lane;
@@ -734,7 +763,7 @@ __device__ __forceinline__ void verify_one_sequence(const unsigned long long* ke
         if (j <= sl) {
             a = key_index(__ldcg(keys + r0 + j));
             if (target_ids) target_ids[r0 + j] = a;
-            match = (j < sl) && (draft[j] == a);
+            match = (j < sl) && (__ldcg(draft_ids + id0 + j * idj) == a);
         }
         if (n_acc < 0) {  // warp-uniform
             const unsigned miss = ~__ballot_sync(kFullMask, match);  // bit set: that row ends the prefix
@@ -749,6 +778,27 @@ __device__ __forceinline__ void verify_one_sequence(const unsigned long long* ke
         n_accept[b] = n_acc;
         bonus[b] = bonus_tok;
     }
+}
+
+// Fixed-shape verification: offsets of the packed rows, row_off[b] = sum over b' < b of (sl[b'] + 1), for the
+// caller's next stage.  One warp.
+__device__ __forceinline__ void warp_write_row_offsets(const VerifyPadded& pad, int B, int SL, int lane) {
+    if (!pad.sl || !pad.row_off_out) return;
+    int base = 0;
+    for (int b0 = 0; b0 < B; b0 += 32) {
+        const int b = b0 + lane;
+        int rows = 0;
+        if (b < B) rows = min(max(__ldcg(pad.sl + b), 0), SL) + 1;
+        int incl = rows;
+#pragma unroll
+        for (int off = 1; off < 32; off <<= 1) {
+            const int o = __shfl_up_sync(kFullMask, incl, off);
+            if (lane >= off) incl += o;
+        }
+        if (b < B) pad.row_off_out[b] = base + incl - rows;
+        base += __shfl_sync(kFullMask, incl, 31);
+    }
+    if (lane == 0) pad.row_off_out[B] = base;
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -1021,14 +1071,15 @@ __global__ void __launch_bounds__((NW + 1) * 32, 1) stream_tail_kernel(const __g
     if (DRAFT) {
         named_barrier_sync(1, BAR_THREADS);
         for (int b = warp; b < p.R; b += NW) {
-            if (p.active && !p.active[b]) continue;
+            if (!chain_seq_live(p.chain, p.active, b)) continue;
             finalize_draft_seq(p, b, grid, feat_s + warp * kWarpScratchWords, clf_s, lane);
         }
         named_barrier_sync(1, BAR_THREADS);
     } else {
         for (int b = warp; b < p.B; b += NW)
             verify_one_sequence(p.keys, p.draft_ids, p.row_off, p.B, p.SL, p.R, b, p.n_accept, p.bonus,
-                                p.target_ids, p.status, lane);
+                                p.target_ids, p.status, lane, p.padded);
+        if (warp == 0) warp_write_row_offsets(p.padded, p.B, p.SL, lane);
         named_barrier_sync(1, BAR_THREADS);
         for (int r = tid; r < p.R; r += BAR_THREADS) p.keys[r] = 0ull;
     }

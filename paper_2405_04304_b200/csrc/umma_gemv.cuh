@@ -116,20 +116,29 @@ umma_gemv_draft_kernel(const __grid_constant__ CUtensorMap tmap_W, const __grid_
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *tmem_base_s;
+    // A chained draft step (draft phase run on the device) in which no sequence drafts any more has nothing
+    // to do: every warp finds that out by itself after the dependency wait (the flags are the predecessor's
+    // output).  The LM-head stages requested before the wait are awaited, then the CTA leaves.
+    const bool chained = p.chain.alive != nullptr && p.chain.step > 1;
 
     if (warp == 0) {
         // ------------------------------ producer ------------------------------
+        const int total = tiles * KB;
+        const uint32_t w_bytes = (uint32_t)g.TRN * 128u;
+        const int pre = min(g.stages, total);
         if (lane == 0) {
-            const int total = tiles * KB;
-            const uint32_t w_bytes = (uint32_t)g.TRN * 128u;
             // the LM head does not depend on the preceding kernel: the whole ring is requested at once
-            const int pre = min(g.stages, total);
             for (int n = 0; n < pre; ++n) {
                 const int tile = n / KB, kb = n - tile * KB;
                 mbar_arrive_expect_tx(&full[n], w_bytes);
                 tma_load_2d(w_tiles + n * g.b_bytes, &tmap_W, kb * kUmmaBK, v_begin + tile * g.TRt, &full[n]);
             }
-            asm volatile("griddepcontrol.wait;" ::: "memory");
+        }
+        asm volatile("griddepcontrol.wait;" ::: "memory");
+        const bool live = !chained || chain_any_live(p.chain, p.R, lane);
+        if (lane == 0 && !live) {
+            for (int n = 0; n < pre; ++n) mbar_wait(&full[n], 0, p.status);   // nothing may still be landing at exit
+        } else if (lane == 0) {
             // the hidden rows, all k-blocks on one barrier; they stay for the whole kernel
             if (total > 0) {
                 mbar_arrive_expect_tx(h_full, (uint32_t)(KB * h_stride));
@@ -149,7 +158,12 @@ umma_gemv_draft_kernel(const __grid_constant__ CUtensorMap tmap_W, const __grid_
         }
     } else if (warp == 1) {
         // ------------------------------ MMA issuer ------------------------------
-        if (lane == 0) {
+        bool live = true;
+        if (chained) {
+            asm volatile("griddepcontrol.wait;" ::: "memory");
+            live = chain_any_live(p.chain, p.R, lane);
+        }
+        if (lane == 0 && live) {
             int stage = 0, phase = 0;
             const uint32_t idesc = umma_idesc(g.TRN);
             if (tiles > 0) {
@@ -196,6 +210,9 @@ umma_gemv_draft_kernel(const __grid_constant__ CUtensorMap tmap_W, const __grid_
             cp_async_commit();
         }
         asm volatile("griddepcontrol.wait;" ::: "memory");  // scratch and outputs belong to the predecessor until now
+        const bool live = !chained || chain_any_live(p.chain, p.R, lane);
+        if (!live) cp_async_wait_all();
+      if (live) {
 
         SoftmaxState st[RK];
         float top_v[RK], best_v[RK];
@@ -282,11 +299,12 @@ umma_gemv_draft_kernel(const __grid_constant__ CUtensorMap tmap_W, const __grid_
             __threadfence();
             named_barrier_sync(1, BAR_THREADS);
             for (int b = ew; b < p.R; b += kGemvEpiWarps) {
-                if (p.active && !p.active[b]) continue;
+                if (!chain_seq_live(p.chain, p.active, b)) continue;
                 finalize_draft_seq(p, b, grid, feat_s + ew * kWarpScratchWords, clf_s, lane);
             }
             if (tid == 0) *p.ticket = 0u;
         }
+      }  // live
     }
 
     tc_fence_before();

@@ -67,6 +67,7 @@ struct UmmaParams {
     int32_t* n_accept;
     int32_t* bonus;
     int32_t* target_ids;
+    VerifyPadded padded;   // sl != null: fixed-shape rows, per-sequence look-ahead read from the device
 };
 
 // ---------------------------------------------------------------------------------------------
@@ -163,6 +164,7 @@ struct DraftFinalParams {
     float* nll_sum;
     int stats_only;
     unsigned int* epoch;  // [0] launches completed so far (stamp of this launch = that + 1), [1] finishing warps done
+    ChainLink chain;      // alive != null: this launch is one step of a draft phase chained on the device
 };
 
 // One warp finishes sequence b from its NP partial records.  clf_s: classifier parameters in shared
@@ -175,7 +177,7 @@ __device__ __forceinline__ void umma_finish_sequence(const DraftFinalParams& p, 
                             p.stats_only != 1);
     if (!active) return;
     const int Hc = p.clf_H;
-    const DraftOutputs o{p.token, p.conf, p.halt, p.feats, p.final_stats, p.nll_sum, p.stats_only};
+    const DraftOutputs o{p.token, p.conf, p.halt, p.feats, p.final_stats, p.nll_sum, p.stats_only, p.chain};
     warp_draft_epilogue(mp.st, mp.key, mp.sel, fpos, n_drafted, p.tau, p.sl_max, feat16, clf_s, clf_s + Hc * kNFeat,
                         clf_s + Hc * (kNFeat + 1), clf_s + Hc * (kNFeat + 2), Hc, b, o, lane);
 }
@@ -236,9 +238,17 @@ umma_tail_kernel(const __grid_constant__ CUtensorMap tmap_W, const __grid_consta
     tc_fence_after();
     const uint32_t tmem_base = *tmem_base_s;
 
+    // A chained draft step in which no sequence drafts any more has nothing to do.  Every warp finds that out
+    // by itself, after the dependency wait (the flags are the predecessor's output), and goes to the exit.
+    bool live = true;
+    if (DRAFT && f.chain.alive != nullptr && f.chain.step > 1) {
+        asm volatile("griddepcontrol.wait;" ::: "memory");
+        live = chain_any_live(f.chain, f.B, lane);
+    }
+
     if (warp == 0) {
         // ------------------------------ producer ------------------------------
-        if (lane == 0) {
+        if (lane == 0 && live) {
             int stage = 0, phase = 0;
             const uint32_t bytes = (uint32_t)(p.rep * p.a_rows + p.TRN) * 128u;
             // The LM head is never written by this library: its first tiles are requested before the
@@ -277,7 +287,7 @@ umma_tail_kernel(const __grid_constant__ CUtensorMap tmap_W, const __grid_consta
         }
     } else if (warp == 1) {
         // ------------------------------ MMA issuer ------------------------------
-        if (lane == 0) {
+        if (lane == 0 && live) {
             int stage = 0, phase = 0, it = 0;
             const uint32_t idesc = umma_idesc(p.TRN);
             for (int i = 0; i < p.TPC; ++i) {
@@ -304,7 +314,7 @@ umma_tail_kernel(const __grid_constant__ CUtensorMap tmap_W, const __grid_consta
                 ++it;
             }
         }
-    } else {
+    } else if (live) {
         // ------------------------------ epilogue ------------------------------
         asm volatile("griddepcontrol.wait;" ::: "memory");  // scratch and outputs belong to the predecessor until now
         const int ew = warp - 2;            // 0 .. kUmmaEpiWarps-1
@@ -453,9 +463,11 @@ umma_tail_kernel(const __grid_constant__ CUtensorMap tmap_W, const __grid_consta
             const int first = ew * (int)gridDim.x + (int)blockIdx.x;
             if (first < f.B) {
                 int b = first;
-                bool act = !f.active || f.active[b];
-                float fpos = f.pos ? static_cast<float>(f.pos[b]) : 0.f;
-                int nd = f.n_drafted ? f.n_drafted[b] : 0;
+                const bool chain = f.chain.alive != nullptr;
+                bool act = chain_seq_live(f.chain, f.active, b);
+                float fpos = chain ? static_cast<float>(f.chain.pos0[b] + f.chain.step)
+                                   : (f.pos ? static_cast<float>(f.pos[b]) : 0.f);
+                int nd = chain ? f.chain.step : (f.n_drafted ? f.n_drafted[b] : 0);
                 float* feat16 = reinterpret_cast<float*>(xch) + ew * kWarpScratchWords;  // the exchange area is free again
                 for (;;) {
                     // a masked sequence still waits for its records: the stamp may only advance once
@@ -463,9 +475,10 @@ umma_tail_kernel(const __grid_constant__ CUtensorMap tmap_W, const __grid_consta
                     umma_finish_sequence(f, p.part_rec, p.CN, b, act, fpos, nd, feat16, clf_s, stamp, p.status, lane);
                     b += kUmmaEpiWarps * (int)gridDim.x;
                     if (b >= f.B) break;
-                    act = !f.active || f.active[b];
-                    fpos = f.pos ? static_cast<float>(f.pos[b]) : 0.f;
-                    nd = f.n_drafted ? f.n_drafted[b] : 0;
+                    act = chain_seq_live(f.chain, f.active, b);
+                    fpos = chain ? static_cast<float>(f.chain.pos0[b] + f.chain.step)
+                                 : (f.pos ? static_cast<float>(f.pos[b]) : 0.f);
+                    nd = chain ? f.chain.step : (f.n_drafted ? f.n_drafted[b] : 0);
                 }
                 // the last finishing warp of the grid advances the stamp for the next launch: by then every
                 // record of this launch has been read
@@ -489,7 +502,8 @@ umma_tail_kernel(const __grid_constant__ CUtensorMap tmap_W, const __grid_consta
                     __threadfence();
                     for (int b = ew; b < p.B; b += kUmmaEpiWarps)
                         verify_one_sequence(p.keys, p.draft_ids, p.row_off, p.B, p.SL, p.R, b, p.n_accept, p.bonus,
-                                            p.target_ids, p.status, lane);
+                                            p.target_ids, p.status, lane, p.padded);
+                    if (ew == 0) warp_write_row_offsets(p.padded, p.B, p.SL, lane);
                     named_barrier_sync(2, kUmmaEpiWarps * 32);
                     for (int r = ew * 32 + lane; r < p.R; r += kUmmaEpiWarps * 32) p.keys[r] = 0ull;
                     if (ew == 0 && lane == 0) *p.ticket = 0u;
@@ -522,6 +536,7 @@ struct VerifyFinalParams {
     int32_t* target_ids;
     int* status;
     unsigned int* ticket;
+    VerifyPadded padded;
 };
 
 __global__ void __launch_bounds__(128) verify_finalize_kernel(const VerifyFinalParams p) {
@@ -530,7 +545,8 @@ __global__ void __launch_bounds__(128) verify_finalize_kernel(const VerifyFinalP
     const int b = blockIdx.x * (blockDim.x >> 5) + warp;
     if (b < p.B)
         verify_one_sequence(p.keys, p.draft_ids, p.row_off, p.B, p.SL, p.R, b, p.n_accept, p.bonus, p.target_ids,
-                            p.status, lane);
+                            p.status, lane, p.padded);
+    if (blockIdx.x == gridDim.x - 1 && warp == (blockDim.x >> 5) - 1) warp_write_row_offsets(p.padded, p.B, p.SL, lane);
     __syncthreads();
     if (threadIdx.x == 0) {
         __threadfence();
