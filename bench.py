@@ -1,9 +1,10 @@
 #!/usr/bin/env python
 """Benchmark of the DISCO logit tails on B200.
 
-A step is one speculative iteration of the hot path: draft steps (LM head, soft-max statistics,
-top-10 / entropy / position features, halt classifier, stopping rule) until the classifier or SL_max
-stops the drafting, then one verification (LM head on SL+1 rows, greedy tokens, accepted prefix, bonus).
+A step is one speculative iteration of the hot path, run through disco_iteration: draft steps (LM head,
+soft-max statistics, top-10 / entropy / position features, halt classifier, stopping rule) chained on the
+device until the classifier or SL_max stops the drafting, then one verification (LM head on the target rows,
+greedy tokens, accepted prefix, bonus token).  Nothing is read back by the host between the kernels.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--workload vicuna_b1] [--impl ours|reference]
 
@@ -47,11 +48,8 @@ def measured_peaks():
 # dram__bytes_read.sum + dram__bytes_write.sum per launch, from the ncu captures summarised under
 # profiles/.  Valid only for the kernel sources they were taken on: reported as null once csrc/ changes.
 NCU_TRAFFIC = {
-    "sources": "347370975812aea5",
-    "bytes_per_launch": {
-        ("vicuna_b1", "verification tail"): 327.77e6 + 4.34e6,
-        ("vicuna_b1", "draft-step tail"): 49.23e6 + 0.02e6,
-    },
+    "sources": "",
+    "bytes_per_launch": {},
 }
 
 
@@ -68,7 +66,7 @@ def kernel_sources_hash() -> str:
 def ncu_traffic(workload: str, kernel: str):
     if kernel_sources_hash() != NCU_TRAFFIC["sources"]:
         return None
-    return NCU_TRAFFIC["bytes_per_launch"].get((workload, kernel))
+    return NCU_TRAFFIC["bytes_per_launch"].get(f"{workload}/{kernel}")
 
 
 # ------------------------------------------------------------------------------------------ ranks
@@ -96,7 +94,7 @@ def whole_job_value(steps_per_rank: int, world: int, seconds: float) -> float:
 class ClockSampler:
     """Polls SM clock and throttle reasons through NVML while the timed region runs (read-only)."""
 
-    def __init__(self, index: int, period_s: float = 0.004):
+    def __init__(self, index: int, period_s: float = 0.002):
         self.samples, self.reasons = [], set()
         self.max_mhz = None
         self._stop = threading.Event()
@@ -147,217 +145,279 @@ class ClockSampler:
     def summary(self):
         med = int(np.median(self.samples)) if self.samples else None
         return {"sm_mhz": med, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons),
-                "samples": len(self.samples)}
+                "samples": len(self.samples), "sm_mhz_min": min(self.samples) if self.samples else None}
 
 
 # ------------------------------------------------------------------------------------------ workload
-class Data:
-    """All seeded inputs of T iterations of a workload, resident on the device (and, for the
-    end-to-end leg, in pinned host memory)."""
+def calibrate_b2(W_D, clf_params, d_D: int, positions: int, seed: int, device: str) -> float:
+    """Random-initialised classifier parameters leave the score far from zero on these inputs, so the loop
+    would never or always halt.  The output bias is set to minus the median pre-sigmoid score over a seeded
+    calibration draw (hidden states of the workload's law, positions uniform in 1..positions), so that the
+    confidence straddles 0.5 and both branches of the stopping rule occur.  Harness-side plain torch; the
+    result is an input like any other."""
+    W1, b1, w2, _ = (t.to(device) for t in clf_params)
+    n = 256
+    h = inputs.hidden(n, d_D, inputs.sub_seed(seed, 11), device=device).float()
+    g = torch.Generator(device="cpu").manual_seed(int(inputs.sub_seed(seed, 12)) & 0x7FFFFFFF)
+    pos = torch.randint(1, max(2, positions + 1), (n,), generator=g).to(device).float()
+    y = torch.softmax(h @ W_D.float().T, dim=-1)
+    top = torch.topk(y, 10, dim=-1).values
+    ent = -(y * torch.log(y.clamp_min(1e-38))).sum(-1)
+    x = torch.cat([top, ent[:, None], pos[:, None]], dim=1)
+    s = torch.relu(x @ W1.T + b1) @ w2
+    return -float(s.median())
 
-    def __init__(self, wl: inputs.Workload, T: int, seed: int, device: str):
+
+class Data:
+    """All seeded inputs of D distinct iterations of a workload, resident on the device."""
+
+    def __init__(self, wl: inputs.Workload, T: int, seed: int, device: str, calibrate: bool = True):
         self.wl, self.T = wl, T
         B, S = wl.B, wl.sl_max
-        self.n_rot = max(2, -(-2 * L2_BYTES // (wl.V * wl.d_D * 2)) + 1)   # copies of W_D: > 2x L2 in total
+        # copies of the draft LM head: consecutive draft steps read consecutive copies, and the window of copies
+        # moves on from iteration to iteration, so that no step finds its head in L2 (n_rot copies > 2x L2)
+        self.n_rot = max(2, -(-2 * L2_BYTES // (wl.V * wl.d_D * 2)) + 1)
+        n_copies = self.n_rot + S
         W_D = inputs.lm_head(wl.V, wl.d_D, inputs.sub_seed(seed, 1), device=device)
-        self.W_D = [W_D] + [W_D.clone() for _ in range(self.n_rot - 1)]
+        self.W_D_ring = W_D.unsqueeze(0).repeat(n_copies, 1, 1).contiguous()
+        self.w_stride = wl.V * wl.d_D * 2
         self.W_T = inputs.lm_head(wl.V, wl.d_T, inputs.sub_seed(seed, 2), device=device)
-        self.clf_params = inputs.classifier_params(wl.H, inputs.sub_seed(seed, 3))
+        W1, b1, w2, b2 = inputs.classifier_params(wl.H, inputs.sub_seed(seed, 3))
+        self.b2_random_init = float(b2[0])
+        self.calibration_positions = 4 * T
+        if calibrate:
+            b2 = torch.tensor([calibrate_b2(W_D, (W1, b1, w2, b2), wl.d_D, self.calibration_positions, seed, device)])
+        self.clf_params = (W1, b1, w2, b2)
         # distinct iterations held in memory (cycled if T is larger)
         per_it = B * (S * wl.d_D + (S + 1) * wl.d_T) * 2
         self.n_distinct = int(max(1, min(T, (3 << 30) // per_it)))
         D = self.n_distinct
         self.h_D = inputs.hidden(D * S * B, wl.d_D, inputs.sub_seed(seed, 4), device=device).view(D, S, B, wl.d_D)
         self.H_T = inputs.hidden(D * B * (S + 1), wl.d_T, inputs.sub_seed(seed, 5), device=device).view(
-            D, B * (S + 1), wl.d_T)
+            D, B, S + 1, wl.d_T)
         # draft ids offered to verification: the target's greedy tokens, corrupted per position.
         # (Harness-side fp32 matmul; any ids are valid inputs, the kernels are timed on whatever they get.)
         Wf = self.W_T.float()
-        tgt = torch.empty((D, B * (S + 1)), dtype=torch.int32)
         rows = self.H_T.view(-1, wl.d_T)
         flat = torch.empty(rows.shape[0], dtype=torch.int64, device=device)
         for r0 in range(0, rows.shape[0], 2048):
             flat[r0:r0 + 2048] = (rows[r0:r0 + 2048].float() @ Wf.T).argmax(-1)
         del Wf
-        tgt.copy_(flat.view(D, B * (S + 1)).to(torch.int32).cpu())
-        clean = tgt.view(D, B, S + 1)[:, :, :S].contiguous()
+        clean = flat.view(D, B, S + 1)[:, :, :S].to(torch.int32).cpu().contiguous()
         if wl.accept_beta is not None:
             alpha = inputs.beta_rates(B, wl.accept_beta[0], wl.accept_beta[1], inputs.sub_seed(seed, 6))
             p = (1.0 - alpha).view(1, B, 1).expand(D, B, S)
+            self.alpha = alpha.numpy().astype(np.float64)
         else:
             p = wl.p_corrupt
-        self.draft_full = inputs.corrupt_ids(clean, p, wl.V, inputs.sub_seed(seed, 7))      # [D, B, S] cpu
-        if wl.sl_mode == "uniform":
-            self.forced_sl = inputs.uniform_sl(D * B, 1, S, inputs.sub_seed(seed, 8)).view(D, B)
-        else:
-            self.forced_sl = None
+            self.alpha = np.full(B, 1.0 - wl.p_corrupt * (1.0 - 1.0 / wl.V))
+        self.draft_cpu = inputs.corrupt_ids(clean, p, wl.V, inputs.sub_seed(seed, 7)).contiguous()   # [D, B, S]
+        self.draft_dev = self.draft_cpu.to(device)
+        self.uniform_sl_cpu = inputs.uniform_sl(D * B, 1, S, inputs.sub_seed(seed, 8)).view(D, B).contiguous()
+        self.uniform_sl_dev = self.uniform_sl_cpu.to(device)
 
     def idx(self, it: int) -> int:
         return it % self.n_distinct
 
 
-def pack_iteration(data: Data, it: int, sl: np.ndarray):
-    """Rows and draft ids of one verification for per-sequence look-aheads sl [B]."""
-    wl = data.wl
-    d = data.idx(it)
-    sl_t = torch.as_tensor(sl, dtype=torch.int32)
-    off = inputs.row_offsets(sl_t)
-    if wl.B == 1:
-        H = data.H_T[d, : int(sl[0]) + 1]
-        ids = data.draft_full[d, 0, : int(sl[0])].contiguous()
-    else:
-        H = inputs.pack_rows(data.H_T[d], sl_t, wl.sl_max)
-        ids = inputs.pack_ids(data.draft_full[d].reshape(-1), sl_t, wl.sl_max)
-    return H, ids, off
-
-
 # ------------------------------------------------------------------------------------------ our arm
-def device_pass(ctx, data: Data, clf, wl, tau: float, Wm: int, K: int, stream, world: int, device, sampler=None):
-    """Closed loop once (discovery + warm-up), then the same launches captured in CUDA graphs and timed.
+def time_replays(graph, stream, reps: int, world: int, warm: int = 3, sampler=None):
+    """Replay a captured graph `warm` times untimed, then `reps` times, each between its own pair of events on
+    the launching stream.  Returns the per-replay seconds."""
+    with torch.cuda.stream(stream):
+        for _ in range(warm):
+            graph.replay()
+        stream.synchronize()
+        if world > 1:
+            torch.distributed.barrier()
+        torch.cuda.synchronize()
+        ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(reps)]
+        if sampler is not None:
+            sampler.__enter__()
+        for e0, e1 in ev:
+            e0.record(stream)
+            graph.replay()
+            e1.record(stream)
+        stream.synchronize()
+        torch.cuda.synchronize()
+        if sampler is not None:
+            sampler.__exit__()
+        if world > 1:
+            torch.distributed.barrier()
+    return [e0.elapsed_time(e1) * 1e-3 for e0, e1 in ev]
 
-    Returns the time of the K timed iterations, the times of graphs holding only their draft-step or
-    only their verification launches, and the closed-loop trace."""
+
+def stats(ts):
+    a = np.asarray(ts, dtype=np.float64)
+    return {"median": float(np.median(a)), "min": float(a.min()), "max": float(a.max()), "replays": int(a.size)}
+
+
+def device_pass(ctx, data: Data, clf, wl, tau: float, forced, Wm: int, K: int, reps: int, stream, world: int, device,
+                sampler=None, check_iterations: int = 0):
+    """The device-resident loop.  All Wm + K iterations are run once eagerly (warm-up; it also yields the
+    look-aheads, from which the rotation of the draft LM-head copies is laid out), then the K timed
+    iterations are captured in CUDA graphs -- the whole iteration, its draft phases only, its verifications
+    only -- and each graph is replayed `reps` times.  forced: None (the classifier decides) or "uniform"."""
     B, S = wl.B, wl.sl_max
     T = Wm + K
-    token = torch.zeros((T, S, B), dtype=torch.int32, device=device)
+    i32 = dict(dtype=torch.int32, device=device)
+    token = torch.zeros((T, S, B), **i32)
     conf = torch.zeros((T, S, B), dtype=torch.float32, device=device)
     halt = torch.zeros((T, S, B), dtype=torch.uint8, device=device)
-    n_acc = torch.zeros((T, B), dtype=torch.int32, device=device)
-    bonus = torch.zeros((T, B), dtype=torch.int32, device=device)
-    pos_all = torch.zeros((T, S, B), dtype=torch.int32)
-    act_all = torch.zeros((T, S, B), dtype=torch.uint8)
-    nd_all = torch.arange(1, S + 1, dtype=torch.int32).view(S, 1).expand(S, B).contiguous().to(device)
-    sl_all = np.zeros((T, B), dtype=np.int64)
-    steps_all = np.zeros(T, dtype=np.int64)
-    emitted = np.zeros(B, dtype=np.int64)
-    packed = []
-    rot = 0
-    # ---------------- discovery: the closed loop, the host reads the halt flags ----------------
+    sl = torch.zeros((T, B), **i32)
+    n_acc = torch.zeros((T, B), **i32)
+    bonus = torch.zeros((T, B), **i32)
+    pos = torch.zeros((T + 1, B), **i32)          # pos[t]: tokens generated before iteration t; row 0 stays zero
+    scratch_n, scratch_b = torch.zeros((B,), **i32), torch.zeros((B,), **i32)
+
+    def forced_of(it):
+        return data.uniform_sl_dev[data.idx(it)] if forced == "uniform" else None
+
+    def iteration(it, base, st):
+        d = data.idx(it)
+        ctx.iteration(data.W_D_ring[base], data.h_D[d], data.W_T, data.H_T[d], pos[it], clf, tau, S, token[it], conf[it],
+                      halt[it], sl[it], n_acc[it], bonus[it], sl_forced=forced_of(it), draft_ids=data.draft_dev[d],
+                      pos_next=pos[it + 1], w_step_stride=data.w_stride, stream=st)
+
     with torch.cuda.stream(stream):
         for it in range(T):
-            d = data.idx(it)
-            active = np.ones(B, dtype=np.uint8)
-            sl = np.zeros(B, dtype=np.int64)
-            for j in range(S):
-                pos_all[it, j] = torch.from_numpy((emitted + j + 1).astype(np.int32))
-                act_all[it, j] = torch.from_numpy(active)
-                pos_d = pos_all[it, j].to(device, non_blocking=False)
-                act_d = act_all[it, j].to(device)
-                ctx.draft_step(data.W_D[rot % data.n_rot], data.h_D[d, j], pos_d, nd_all[j], clf, tau, S,
-                               token[it, j], conf[it, j], halt[it, j], active=act_d, stream=stream)
-                rot += 1
-                stream.synchronize()
-                h = halt[it, j].cpu().numpy()
-                sl[active == 1] = j + 1
-                if data.forced_sl is not None:
-                    stop = (data.forced_sl[d].numpy() <= j + 1)
-                else:
-                    stop = h.astype(bool)
-                active = (active.astype(bool) & ~stop).astype(np.uint8)
-                steps_all[it] = j + 1
-                if not active.any():
-                    break
-            sl_all[it] = sl
-            H, ids, off = pack_iteration(data, it, sl)
-            ids_d, off_d = ids.to(device), off.to(device)
-            packed.append((H, ids_d, off_d, int(off[-1])))
-            ctx.verify_ragged(data.W_T, H, ids_d, off_d, B, int(off[-1]), n_acc[it], bonus[it], stream=stream)
-            stream.synchronize()
-            emitted += n_acc[it].cpu().numpy().astype(np.int64) + 1
-    status = ctx.device_status()
-    if status != 0:
-        raise RuntimeError(f"device status {status} after the discovery pass")
-    pos_dev, act_dev = pos_all.to(device), act_all.to(device)
-    ref_token, ref_halt = token.clone(), halt.clone()
-    ref_nacc, ref_bonus = n_acc.clone(), bonus.clone()
+            iteration(it, 0, stream)
+        stream.synchronize()
+    if ctx.device_status() != 0:
+        raise RuntimeError("device status after the eager pass")
+    sl_all = sl.cpu().numpy().astype(np.int64)
+    ref = [t.clone() for t in (token, halt, sl, n_acc, bonus, pos)]
+    bases = np.zeros(T, dtype=np.int64)
+    for it in range(1, T):
+        bases[it] = (bases[it - 1] + int(sl_all[it - 1].max())) % data.n_rot
 
-    # ---------------- the same launch sequence, captured in CUDA graphs ----------------
     timed = range(Wm, T)
-
-    def enqueue(which: str):
-        r = 0
-        for it in timed:
-            d = data.idx(it)
-            if which in ("all", "draft"):
-                for j in range(int(steps_all[it])):
-                    ctx.draft_step(data.W_D[r % data.n_rot], data.h_D[d, j], pos_dev[it, j], nd_all[j], clf, tau,
-                                   S, token[it, j], conf[it, j], halt[it, j], active=act_dev[it, j])
-                    r += 1
-            if which in ("all", "verify"):
-                H, ids_d, off_d, R = packed[it]
-                ctx.verify_ragged(data.W_T, H, ids_d, off_d, B, R, n_acc[it], bonus[it])
-
-    graphs = {}
-    launches = {}
+    graphs, launches = {}, {}
     for which in ("all", "draft", "verify"):
-        token.zero_(); halt.zero_(); n_acc.zero_(); bonus.zero_()
         torch.cuda.synchronize()
         g = torch.cuda.CUDAGraph()
         c0 = ctx.launch_count()
         with torch.cuda.graph(g, stream=stream):
-            enqueue(which)
+            for it in timed:
+                d = data.idx(it)
+                if which == "all":
+                    iteration(it, int(bases[it]), None)
+                elif which == "draft":
+                    ctx.draft_loop(data.W_D_ring[int(bases[it])], data.h_D[d], pos[it], clf, tau, S, token[it], conf[it],
+                                   halt[it], sl[it], sl_forced=forced_of(it), w_step_stride=data.w_stride)
+                else:
+                    ctx.verify_sl(data.W_T, data.H_T[d], data.draft_dev[d], S, 1, sl[it], B, S, scratch_n, scratch_b)
         launches[which] = ctx.launch_count() - c0
         graphs[which] = g
 
-    def time_graph(g, smp=None):
-        with torch.cuda.stream(stream):
-            g.replay()                               # untimed replay (graph upload, caches, clocks)
-            stream.synchronize()
-            if world > 1:
-                torch.distributed.barrier()
-            torch.cuda.synchronize()
-            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            if smp is not None:
-                smp.__enter__()
-            e0.record(stream)
-            g.replay()
-            e1.record(stream)
-            stream.synchronize()
-            torch.cuda.synchronize()
-            if smp is not None:
-                smp.__exit__()
-            if world > 1:
-                torch.distributed.barrier()
-        return e0.elapsed_time(e1) * 1e-3
-
-    t_all = time_graph(graphs["all"], sampler)
-    # results of the replay must be those of the closed loop
-    same = (torch.equal(token[Wm:], ref_token[Wm:]) and torch.equal(halt[Wm:], ref_halt[Wm:]) and
-            torch.equal(n_acc[Wm:], ref_nacc[Wm:]) and torch.equal(bonus[Wm:], ref_bonus[Wm:]))
+    t_all = time_replays(graphs["all"], stream, reps, world, sampler=sampler)
+    same = all(torch.equal(a[Wm:], b[Wm:]) for a, b in zip((token, halt, sl, n_acc, bonus, pos), ref))
     if not same or ctx.device_status() != 0:
-        raise RuntimeError("graph replay did not reproduce the closed-loop results")
-    t_draft = time_graph(graphs["draft"])
-    t_verify = time_graph(graphs["verify"])
+        raise RuntimeError("graph replay did not reproduce the eager results")
+    t_draft = time_replays(graphs["draft"], stream, max(5, reps // 2), world)
+    t_verify = time_replays(graphs["verify"], stream, max(5, reps // 2), world)
     del graphs
-    n_draft = int(steps_all[Wm:].sum())
-    rows_total = int(sum(packed[it][3] for it in timed))
-    return {"t_all": t_all, "t_draft": t_draft, "t_verify": t_verify, "n_draft": n_draft, "rows_total": rows_total,
-            "sl_all": sl_all, "n_acc": ref_nacc.cpu().numpy(), "launches": launches["all"]}
+    if ctx.device_status() != 0:
+        raise RuntimeError("device status after the timed replays")
+
+    checked = 0
+    if check_iterations:
+        checked = closed_loop_check(ctx, data, clf, wl, tau, forced, range(Wm, Wm + min(K, check_iterations)),
+                                    ref, stream, device)
+    n_live = int(sl_all[Wm:].max(axis=1).sum())      # draft launches that had work (per iteration: the longest look-ahead)
+    return {"t_all": t_all, "t_draft": t_draft, "t_verify": t_verify, "n_live_steps": n_live, "sl_all": sl_all,
+            "rows_counted": int((sl_all[Wm:] + 1).sum()),
+            "n_acc": ref[3].cpu().numpy(), "launches": launches, "closed_loop_checked": checked}
+
+
+def closed_loop_check(ctx, data: Data, clf, wl, tau, forced, its, ref, stream, device) -> int:
+    """The same iterations driven by the host, one call per draft step with the halt flags read back, then one
+    ragged verification: must give what the device-resident loop gave."""
+    B, S = wl.B, wl.sl_max
+    r_token, r_halt, r_sl, r_nacc, r_bonus, r_pos = (t.cpu().numpy() for t in ref)
+    tok = torch.zeros(B, dtype=torch.int32, device=device)
+    cf = torch.zeros(B, dtype=torch.float32, device=device)
+    hl = torch.zeros(B, dtype=torch.uint8, device=device)
+    na = torch.zeros(B, dtype=torch.int32, device=device)
+    bo = torch.zeros(B, dtype=torch.int32, device=device)
+    with torch.cuda.stream(stream):
+        for it in its:
+            d = data.idx(it)
+            active = np.ones(B, dtype=bool)
+            sl = np.zeros(B, dtype=np.int64)
+            for j in range(S):
+                p = torch.from_numpy((r_pos[it] + j + 1).astype(np.int32)).to(device)
+                nd = torch.full((B,), j + 1, dtype=torch.int32, device=device)
+                act = torch.from_numpy(active.astype(np.uint8)).to(device)
+                ctx.draft_step(data.W_D_ring[0], data.h_D[d, j], p, nd, clf, tau, S, tok, cf, hl, active=act, stream=stream)
+                stream.synchronize()
+                sl[active] = j + 1
+                if not np.array_equal(tok.cpu().numpy()[active], r_token[it, j][active]):
+                    raise RuntimeError("closed loop: tokens differ from the device-resident loop")
+                stop = (data.uniform_sl_cpu[d].numpy() <= j + 1) if forced == "uniform" else hl.cpu().numpy().astype(bool)
+                active = active & ~stop
+                if not active.any():
+                    break
+            sl_t = torch.as_tensor(sl, dtype=torch.int32)
+            off = inputs.row_offsets(sl_t)
+            H = inputs.pack_rows(data.H_T[d].reshape(B * (S + 1), -1), sl_t, S)
+            ids = inputs.pack_ids(data.draft_cpu[d].reshape(-1), sl_t, S).to(device)
+            ctx.verify_ragged(data.W_T, H, ids if ids.numel() else None, off.to(device), B, int(off[-1]), na, bo,
+                              stream=stream)
+            stream.synchronize()
+            if not (np.array_equal(sl, r_sl[it]) and np.array_equal(na.cpu().numpy(), r_nacc[it]) and
+                    np.array_equal(bo.cpu().numpy(), r_bonus[it])):
+                raise RuntimeError("closed loop: look-ahead, accepted length or bonus differ from the device-resident loop")
+    return len(its)
 
 
 def rooflines(wl, K: int, res: dict, hbm_peak: float, tensor_peak: float, peak_kind: str):
     """Achieved algorithmic GB/s (or, beyond the machine balance, TFLOP/s) of the two kernels against the
-    measured peaks.  Returns (dominant kernel, other kernel)."""
-    draft_bytes = res["n_draft"] * (wl.V * wl.d_D * 2 + wl.B * wl.d_D * 2)
-    verify_bytes = K * wl.V * wl.d_T * 2 + res["rows_total"] * wl.d_T * 2
-    verify_flops = 2.0 * res["rows_total"] * wl.V * wl.d_T
-    roof_verify = {"kernel": "verification tail", "bound": "hbm", "achieved": verify_bytes / res["t_verify"] / 1e9,
+    measured peaks, from the median replay of the graphs that hold only that kernel.  A verification launch
+    reads the LM head and all B * (SL_max + 1) fixed-shape rows; a draft step that has work reads its LM head
+    and B hidden rows.  Returns (dominant kernel, other kernel)."""
+    B, S = wl.B, wl.sl_max
+    R = B * (S + 1)
+    t_v, t_d = float(np.median(res["t_verify"])), float(np.median(res["t_draft"]))
+    n_live = max(res["n_live_steps"], 1)
+    rows = res["rows_counted"]          # over the K launches: rows that count, sum of SL_b + 1 (the padding rows do not)
+    draft_bytes = n_live * (wl.V * wl.d_D * 2 + B * wl.d_D * 2)
+    verify_bytes = K * wl.V * wl.d_T * 2 + rows * wl.d_T * 2
+    verify_flops = 2.0 * rows * wl.V * wl.d_T
+    roof_verify = {"kernel": "verification tail", "bound": "hbm", "achieved": verify_bytes / t_v / 1e9,
                    "peak": hbm_peak, "peak_kind": peak_kind, "unit": "GB/s", "launches": K,
-                   "avg_launch_us": res["t_verify"] / K * 1e6, "traffic": None,
-                   "tensor_tflops": verify_flops / res["t_verify"] / 1e12}
-    roof_draft = {"kernel": "draft-step tail", "bound": "hbm", "achieved": draft_bytes / res["t_draft"] / 1e9,
-                  "peak": hbm_peak, "peak_kind": peak_kind, "unit": "GB/s", "launches": res["n_draft"],
-                  "avg_launch_us": res["t_draft"] / max(res["n_draft"], 1) * 1e6, "traffic": None}
+                   "avg_launch_us": t_v / K * 1e6, "rows_per_launch": R, "rows_counted_per_launch": rows / K,
+                   "traffic": None,
+                   "tensor_tflops": verify_flops / t_v / 1e12}
+    roof_draft = {"kernel": "draft-step tail", "bound": "hbm", "achieved": draft_bytes / t_d / 1e9,
+                  "peak": hbm_peak, "peak_kind": peak_kind, "unit": "GB/s", "launches": n_live,
+                  "launches_without_work": K * S - n_live, "avg_launch_us": t_d / n_live * 1e6, "traffic": None,
+                  "note": "time of the draft phases (launches without work included) over the steps that had work"}
     for r in (roof_verify, roof_draft):
         r["traffic"] = ncu_traffic(wl.name, r["kernel"])
         r["frac"] = r["achieved"] / r["peak"]
         r["frac_of_nominal_8TBs"] = r["achieved"] / 8000.0
-    if res["rows_total"] / K > tensor_peak * 1e12 / (hbm_peak * 1e9):   # rows per call beyond the machine balance
+    if rows / K > tensor_peak * 1e12 / (hbm_peak * 1e9):   # rows per call beyond the machine balance
         roof_verify.update({"bound": "tensor", "hbm_gbs": roof_verify["achieved"],
                             "achieved": roof_verify["tensor_tflops"], "peak": tensor_peak, "unit": "TFLOP/s",
                             "frac": roof_verify["tensor_tflops"] / tensor_peak})
         roof_verify.pop("frac_of_nominal_8TBs")
-    return (roof_verify, roof_draft) if res["t_verify"] >= res["t_draft"] else (roof_draft, roof_verify)
+    return (roof_verify, roof_draft) if t_v >= t_d else (roof_draft, roof_verify)
+
+
+def summarise(wl, data: Data, res: dict, K: int, Wm: int, world: int):
+    """Throughput and look-ahead statistics of one device pass."""
+    sl = res["sl_all"][Wm:]
+    n_acc = res["n_acc"][Wm:]
+    hist = np.bincount(sl.reshape(-1), minlength=wl.sl_max + 1)[1:]
+    # Eq. 1's numerator: expected tokens per iteration under i.i.d. acceptance, for the look-aheads that occurred
+    a = data.alpha.reshape(1, -1)
+    expected = float(np.mean((1.0 - a ** (sl + 1)) / (1.0 - a)))
+    t = stats(res["t_all"])
+    return {"value": whole_job_value(K, world, t["median"]), "unit": UNIT, "steps": K, "ms_per_step": t["median"] / K * 1e3,
+            "replay_seconds": t, "mean_sl": float(sl.mean()), "sl_histogram_1_to_max": hist.tolist(),
+            "mean_tokens_per_iteration": float((n_acc + 1).mean()), "eq1_expected_tokens_per_iteration": expected,
+            "draft_steps_with_work_per_iteration": res["n_live_steps"] / K}
 
 
 def run_ours(args, rank: int, world: int):
@@ -371,60 +431,108 @@ def run_ours(args, rank: int, world: int):
     T = Wm + K
     data = Data(wl, T, replica_seed(wl.seed, rank), device)
     B, S = wl.B, wl.sl_max
-    max_rows = B * (S + 1)
-    ctx = binding.Context(wl.V, wl.d_D, wl.d_T, max_batch=B, max_rows=max_rows, clf_hidden=wl.H)
+    ctx = binding.Context(wl.V, wl.d_D, wl.d_T, max_batch=B, max_rows=B * (S + 1), clf_hidden=wl.H)
     ctx.set_kernel_path(args.kernel_path)
     clf = binding.Classifier(*(t.to(device) for t in data.clf_params))
     stream = torch.cuda.Stream()
     hbm_peak, tensor_peak, peak_kind = measured_peaks()
+    forced = "uniform" if wl.sl_mode == "uniform" else None
 
     sampler = ClockSampler(dev_index)
-    res = device_pass(ctx, data, clf, wl, wl.tau, Wm, K, stream, world, device, sampler)
+    res = device_pass(ctx, data, clf, wl, wl.tau, forced, Wm, K, args.replays, stream, world, device, sampler,
+                      check_iterations=8)
     dominant, other = rooflines(wl, K, res, hbm_peak, tensor_peak, peak_kind)
-    t_all = res["t_all"]
+    main = summarise(wl, data, res, K, Wm, world)
 
-    # the same workload with the classifier overruled: tau = 0 never halts before SL_max (static SL)
-    static = None
-    if data.forced_sl is None and not args.no_static:
-        Ks = min(K, 256)
-        rs = device_pass(ctx, data, clf, wl, 0.0, Wm, Ks, stream, world, device)
-        sd, so = rooflines(wl, Ks, rs, hbm_peak, tensor_peak, peak_kind)
-        static = {"value": Ks * world / rs["t_all"], "unit": UNIT, "steps": Ks,
-                  "mean_sl": float(rs["sl_all"][Wm:].mean()), "ms_per_step": rs["t_all"] / Ks * 1e3,
-                  "roofline": sd, "roofline_other_kernel": so}
+    # the same workload under the two degenerate policies: tau = 0 never halts before SL_max (static SL), and a
+    # forced look-ahead drawn uniformly from 1..SL_max per iteration
+    extra = {}
+    if not args.no_static:
+        Ks = min(K, 128)
+        for name, (tau_x, forced_x) in {"static_sl_max": (0.0, None), "uniform_sl": (wl.tau, "uniform")}.items():
+            if forced_x == forced and tau_x == wl.tau:
+                continue
+            rs = device_pass(ctx, data, clf, wl, tau_x, forced_x, Wm, Ks, max(5, args.replays // 2), stream, world, device)
+            sd, so = rooflines(wl, Ks, rs, hbm_peak, tensor_peak, peak_kind)
+            extra[name] = dict(summarise(wl, data, rs, Ks, Wm, world), roofline=sd, roofline_other_kernel=so)
 
-    # ---------------- end to end: host buffers through the *_host entry points, closed loop ----------
-    e2e = run_e2e(ctx, data, clf, wl, Wm, K, stream, world)
-    e2e["matches"] = all(np.array_equal(sl, res["sl_all"][it]) and np.array_equal(na, res["n_acc"][it])
-                         for it, (sl, na) in enumerate(e2e["trace"]))
+    # ---------------- end to end: host buffers through disco_iteration_host ----------
+    e2e = run_e2e(ctx, data, clf, wl, forced, Wm, K, stream, world)
+    e2e["matches"] = bool(np.array_equal(e2e["sl"], res["sl_all"][Wm:]) and np.array_equal(e2e["n_acc"], res["n_acc"][Wm:]))
 
-    t_all, e2e["seconds"] = max_over_ranks([t_all, e2e["seconds"]], device)
+    t_med = main["replay_seconds"]["median"]
+    t_med, e2e["seconds"] = max_over_ranks([t_med, e2e["seconds"]], device)
 
     out = {
-        "metric": METRIC, "value": whole_job_value(K, world, t_all), "unit": UNIT, "n_gpus": world, "steps": K, "warmup": Wm,
-        "ms_per_step": t_all / K * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "metric": METRIC, "value": whole_job_value(K, world, t_med), "unit": UNIT, "n_gpus": world, "steps": K, "warmup": Wm,
+        "ms_per_step": t_med / K * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "bf16 inputs, fp32 accumulate", "data": "synthetic (seeded Gaussian LM heads and hidden states)",
         "config": {"workload": wl.name, "V": wl.V, "d_draft": wl.d_D, "d_target": wl.d_T, "batch": B,
                    "sl_max": S, "tau": wl.tau, "clf_hidden": wl.H, "p_corrupt": wl.p_corrupt,
-                   "sl_source": wl.sl_mode, "mean_sl": float(res["sl_all"][Wm:].mean()),
-                   "mean_accepted": float(res["n_acc"][Wm:].mean()),
-                   "draft_steps_per_iteration": res["n_draft"] / K, "replicas": world,
-                   "l2": f"draft LM head rotates through {data.n_rot} copies (> 2x L2); the target LM head alone "
-                         "exceeds L2", "launch": "CUDA graph of the K iterations' kernels"},
+                   "sl_source": "forced uniform 1..SL_max" if forced else "halt classifier, consumed on the device",
+                   "classifier": {"init": "U(-1/sqrt(fan_in), 1/sqrt(fan_in))", "b2_random_init": data.b2_random_init,
+                                  "b2_calibrated": float(data.clf_params[3][0]),
+                                  "calibration": f"b2 = -median(score) over 256 seeded draft steps, positions uniform in "
+                                                 f"1..{data.calibration_positions}"},
+                   "mean_sl": main["mean_sl"], "sl_histogram_1_to_max": main["sl_histogram_1_to_max"],
+                   "mean_tokens_per_iteration": main["mean_tokens_per_iteration"],
+                   "eq1_expected_tokens_per_iteration": main["eq1_expected_tokens_per_iteration"],
+                   "draft_steps_with_work_per_iteration": main["draft_steps_with_work_per_iteration"], "replicas": world,
+                   "l2": f"every draft step reads its own copy of the draft LM head ({data.n_rot + S} copies, the window "
+                         f"moves on by the look-ahead each iteration: > 2x L2 between reuses); the target LM head alone "
+                         "exceeds L2",
+                   "launch": "one disco_iteration call per iteration, K of them in a CUDA graph; median of the replays",
+                   "closed_loop_checked_iterations": res["closed_loop_checked"]},
+        "replay_seconds": main["replay_seconds"],
         "roofline": dominant, "roofline_other_kernel": other,
         "e2e": {"value": whole_job_value(K, world, e2e["seconds"]), "unit": UNIT, "h2d_bytes_per_step": e2e["h2d"] / K,
-                "d2h_bytes_per_step": e2e["d2h"] / K, "matches_device_run": e2e["matches"]},
-        "gpu_launches": res["launches"], "clocks": sampler.summary(),
+                "d2h_bytes_per_step": e2e["d2h"] / K, "matches_device_run": e2e["matches"],
+                "call": "disco_iteration_host, one call per iteration, pinned host buffers",
+                "us_per_call": e2e["seconds"] / K * 1e6, "us_on_the_device_per_call": t_med / K * 1e6,
+                "us_of_copies_at_25GBs_per_call": (e2e["h2d"] + e2e["d2h"]) / K / 25e3},
+        "gpu_launches": res["launches"]["all"], "clocks": sampler.summary(),
     }
-    if static is not None:
-        out["static_sl_max"] = static
-    if wl.B == 1 and not args.no_static:
-        out["other_modes"] = other_modes(ctx, data, clf, wl, stream, device)
-        if ctx.device_status() != 0:
-            raise RuntimeError(f"device status {ctx.device_status()} after the other modes")
-    if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        out["cpu_baseline"] = cpu_baseline(data, wl, budget_s=args.cpu_seconds)
+    out.update(extra)
+    if rank == 0 and world == 1:
+        if not args.no_other_workloads:
+            out["other_workloads"] = other_workloads(binding, wl.name, args, hbm_peak, tensor_peak, peak_kind, device)
+        if wl.B == 1 and not args.no_static:
+            out["other_modes"] = other_modes(ctx, data, clf, wl, stream, device)
+            if ctx.device_status() != 0:
+                raise RuntimeError("device status after the other modes")
+        if not args.no_cpu_baseline:
+            out["cpu_baseline"] = cpu_baseline(data, wl, forced, budget_s=args.cpu_seconds)
     ctx.close()
+    return out
+
+
+def other_workloads(binding, skip: str, args, hbm_peak, tensor_peak, peak_kind, device) -> dict:
+    """The remaining configurations, a handful of iterations each: device-resident iterations/s, look-ahead
+    histogram, accepted length next to Eq. 1's closed form, and the dominant kernel's time against the
+    measured peak.  The batched Starcoder shapes are run at the three thresholds of its sweep."""
+    plan = {"tiny": 16, "vicuna_b1": 16, "starcoder_b1": 16, "vicuna_b64": 8, "starcoder_b256": 4}
+    out = {}
+    stream = torch.cuda.Stream()
+    for name, K in plan.items():
+        if name == skip:
+            continue
+        wl = inputs.WORKLOADS[name]
+        Wm = 3
+        data = Data(wl, Wm + K, wl.seed, device)
+        B, S = wl.B, wl.sl_max
+        ctx = binding.Context(wl.V, wl.d_D, wl.d_T, max_batch=B, max_rows=B * (S + 1), clf_hidden=wl.H)
+        clf = binding.Classifier(*(t.to(device) for t in data.clf_params))
+        forced = "uniform" if wl.sl_mode == "uniform" else None
+        taus = (0.3, 0.5, 0.7) if name == "starcoder_b256" else (wl.tau,)
+        for tau in taus:
+            res = device_pass(ctx, data, clf, wl, tau, forced, Wm, K, 5, stream, 1, device, check_iterations=1)
+            dom, oth = rooflines(wl, K, res, hbm_peak, tensor_peak, peak_kind)
+            key = name if len(taus) == 1 else f"{name}@tau={tau}"
+            out[key] = dict(summarise(wl, data, res, K, Wm, 1), tau=tau, roofline=dom, roofline_other_kernel=oth,
+                            sl_source="forced uniform 1..SL_max" if forced else "halt classifier")
+        ctx.close()
+        del data, ctx, clf
+        torch.cuda.empty_cache()
     return out
 
 
@@ -447,7 +555,7 @@ def other_modes(ctx, data: Data, clf, wl, stream, device) -> dict:
     ptok = torch.zeros(B, device=device)
     dprobs = torch.zeros(S, B, V, device=device)
     yT = torch.zeros(R, V, device=device)
-    ids = data.draft_full[0].reshape(-1).to(device)
+    ids = data.draft_dev[0].reshape(-1)
     na = torch.zeros(B, dtype=torch.int32, device=device)
     nx = torch.zeros(B, dtype=torch.int32, device=device)
     N = 256                                        # positions of the feature-extraction pass
@@ -462,22 +570,24 @@ def other_modes(ctx, data: Data, clf, wl, stream, device) -> dict:
     yDn = torch.zeros(N, V, device=device); yTn = torch.zeros(N, V, device=device)
     posN = torch.arange(N, dtype=torch.int32, device=device)
     h = data.h_D[0, 0]
-    H_T = data.H_T[0]
+    H_T = data.H_T[0].reshape(R, wl.d_T)
+    n_w = data.W_D_ring.shape[0]
     calls = {
-        "draft_step_ppl": lambda i: ctx.draft_step_ppl(data.W_D[i % data.n_rot], h, nd, nll, 1e9, S, tok, conf, halt,
+        "draft_step": lambda i: ctx.draft_step(data.W_D_ring[i % n_w], h, pos, nd, clf, wl.tau, S, tok, conf, halt,
+                                               stream=stream),
+        "verify": lambda i: ctx.verify(data.W_T, H_T, ids, B, S, na, nx, stream=stream),
+        "draft_step_ppl": lambda i: ctx.draft_step_ppl(data.W_D_ring[i % n_w], h, nd, nll, 1e9, S, tok, conf, halt,
                                                        stream=stream),
-        "draft_step_sample": lambda i: ctx.draft_step_sample(data.W_D[i % data.n_rot], h, pos, nd, clf, wl.tau, S, u,
+        "draft_step_sample": lambda i: ctx.draft_step_sample(data.W_D_ring[i % n_w], h, pos, nd, clf, wl.tau, S, u,
                                                              tok, conf, halt, dprobs[i % S], p_token=ptok,
                                                              stream=stream),
         "verify_sample": lambda i: ctx.verify_sample_ragged(data.W_T, H_T, ids, dprobs, None, B, R, ua, us, na, nx, yT,
                                                             stream=stream),
-        "extract_features": lambda i: fx.extract_features(data.W_D[i % data.n_rot], HD[:N], data.W_T, HT[:N], posN,
+        "extract_features": lambda i: fx.extract_features(data.W_D_ring[i % n_w], HD[:N], data.W_T, HT[:N], posN,
                                                            fD, fT, tv, lab, tD, tT, yDn, yTn, stream=stream),
     }
     out = {}
     reps = 20
-    e0 = torch.cuda.Event(enable_timing=True)
-    e1 = torch.cuda.Event(enable_timing=True)
     with torch.cuda.stream(stream):
         for name, fn in calls.items():
             for i in range(3):
@@ -487,135 +597,89 @@ def other_modes(ctx, data: Data, clf, wl, stream, device) -> dict:
             with torch.cuda.graph(graph, stream=stream):
                 for i in range(reps):
                     fn(i)
-            graph.replay()
-            stream.synchronize()
-            e0.record(stream)
-            graph.replay()
-            e1.record(stream)
-            stream.synchronize()
-            out[name + "_us"] = e0.elapsed_time(e1) * 1e3 / reps
+            ts = time_replays(graph, stream, 5, 1)
+            out[name + "_us"] = float(np.median(ts)) * 1e6 / reps
     if fx.device_status() != 0:
-        raise RuntimeError(f"device status {fx.device_status()} after feature extraction")
+        raise RuntimeError("device status after feature extraction")
     fx.close()
     out["extract_features_positions"] = N
     out["look_ahead"] = S
+    out["note"] = "stand-alone calls, 20 in a row in a CUDA graph, draft LM head rotating through its copies"
     return out
 
 
-def run_e2e(ctx, data: Data, clf, wl, Wm: int, K: int, stream, world: int):
-    """Closed loop through the host-buffer entry points: per-step inputs start in pinned host memory,
-    every result (halt flag, token, accepted length, bonus) is read back by the host."""
+def run_e2e(ctx, data: Data, clf, wl, forced, Wm: int, K: int, stream, world: int):
+    """One disco_iteration_host call per iteration: every per-iteration input starts in pinned host memory,
+    every result is in host memory when the call returns.  The position base is carried by the call itself."""
     B, S = wl.B, wl.sl_max
-    D = data.n_distinct
     h_D_host = data.h_D.cpu().pin_memory()
     H_T_host = data.H_T.cpu().pin_memory()
-    token = torch.zeros(B, dtype=torch.int32).pin_memory()
-    conf = torch.zeros(B, dtype=torch.float32).pin_memory()
-    halt = torch.zeros(B, dtype=torch.uint8).pin_memory()
-    n_acc = torch.zeros(B, dtype=torch.int32).pin_memory()
-    bonus = torch.zeros(B, dtype=torch.int32).pin_memory()
-    pos = torch.zeros(B, dtype=torch.int32).pin_memory()
-    nd = torch.zeros(B, dtype=torch.int32).pin_memory()
-    act = torch.ones(B, dtype=torch.uint8).pin_memory()
-    h2d = d2h = 0
-    emitted = np.zeros(B, dtype=np.int64)
-    trace = []
-    rot = 0
-    # numpy views of the pinned buffers: the loop's own bookkeeping stays off torch's dispatcher
-    pos_np, nd_np, act_np, halt_np, nacc_np = pos.numpy(), nd.numpy(), act.numpy(), halt.numpy(), n_acc.numpy()
-    forced = None if data.forced_sl is None else data.forced_sl.numpy()
-    off = torch.zeros(B + 1, dtype=torch.int32).pin_memory()
-    off_np = off.numpy()
+    ids_host = data.draft_cpu.pin_memory()
+    forced_host = data.uniform_sl_cpu.pin_memory() if forced == "uniform" else None
+    pin = lambda *shape, dtype: torch.zeros(shape, dtype=dtype).pin_memory()
+    token, conf, halt = pin(S, B, dtype=torch.int32), pin(S, B, dtype=torch.float32), pin(S, B, dtype=torch.uint8)
+    sl, n_acc, bonus, pos = (pin(B, dtype=torch.int32) for _ in range(4))
+    sl_np, nacc_np = sl.numpy(), n_acc.numpy()
+    T = Wm + K
+    sl_hist = np.zeros((T, B), dtype=np.int64)
+    nacc_hist = np.zeros((T, B), dtype=np.int64)
+    per_call_h2d = B * (S * wl.d_D + (S + 1) * wl.d_T) * 2 + B * 4 + B * S * 4 + (B * 4 if forced else 0) + S * B * 9
+    per_call_d2h = S * B * 9 + 4 * B * 4
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    for it in range(Wm + K):
+    ring = data.W_D_ring
+    for it in range(T):
         if it == Wm:
             torch.cuda.synchronize()
             if world > 1:
                 torch.distributed.barrier()
             e0.record(stream)
-            h2d = d2h = 0
-        d = data.idx(it)
-        act_np[:] = 1
-        sl = np.zeros(B, dtype=np.int64)
-        for j in range(S):
-            pos_np[:] = emitted + (j + 1)
-            nd_np[:] = j + 1
-            ctx.draft_step_host(data.W_D[rot % data.n_rot], h_D_host[d, j], pos, nd, clf, wl.tau, S, token, conf,
-                                halt, active=act if B > 1 else None, stream=stream)
-            rot += 1
-            h2d += B * (wl.d_D * 2 + 4 + 4 + 1)
-            a = act_np.astype(bool)
-            d2h += int(a.sum()) * (4 + 4 + 1)
-            sl[a] = j + 1
-            stop = (forced[d] <= j + 1) if forced is not None else halt_np.astype(bool)
-            act_np[:] = a & ~stop
-            if not act_np.any():
-                break
-        sl_t = torch.as_tensor(sl, dtype=torch.int32)
-        off_np[1:] = np.cumsum(sl + 1)
-        if B == 1:
-            H = H_T_host[d, : int(sl[0]) + 1]
-            ids = data.draft_full[d, 0, : int(sl[0])].contiguous()
-        else:
-            H = inputs.pack_rows(H_T_host[d], sl_t, S)
-            ids = inputs.pack_ids(data.draft_full[d].reshape(-1), sl_t, S)
-        R = int(off_np[-1])
-        ctx.verify_ragged_host(data.W_T, H, ids if ids.numel() else None, off, B, R, n_acc, bonus, stream=stream)
-        h2d += R * wl.d_T * 2 + (R - B) * 4 + (B + 1) * 4
-        d2h += B * 8
-        emitted += nacc_np.astype(np.int64) + 1
-        trace.append((sl.copy(), nacc_np.copy()))
+        d = it % data.n_distinct
+        ctx.iteration_host(ring[(it * S) % data.n_rot], h_D_host[d], data.W_T, H_T_host[d], pos, clf, wl.tau, S, token, conf,
+                           halt, sl, n_acc, bonus, sl_forced=None if forced_host is None else forced_host[d],
+                           draft_ids=ids_host[d], pos_next=pos, w_step_stride=data.w_stride, stream=stream)
+        sl_hist[it] = sl_np
+        nacc_hist[it] = nacc_np
     e1.record(stream)
     torch.cuda.synchronize()
     if world > 1:
         torch.distributed.barrier()
-    return {"seconds": e0.elapsed_time(e1) * 1e-3, "h2d": h2d, "d2h": d2h, "matches": True, "trace": trace}
+    seconds = e0.elapsed_time(e1) * 1e-3
+    return {"seconds": seconds, "h2d": per_call_h2d * K, "d2h": per_call_d2h * K, "sl": sl_hist[Wm:], "n_acc": nacc_hist[Wm:]}
 
 
 # ------------------------------------------------------------------------------------------ CPU legs
-def oracle_iteration(oracle, wl, W_D, W_T, clf, h_D, H_T, draft, emitted, nthreads, forced_sl=None):
-    """One iteration with the CPU oracle (closed loop on its own halt flags).  Arrays are numpy."""
+def oracle_iterations(oracle, wl, W_D, W_T, clf, data: Data, forced, nthreads: int, budget_s: float, at_least: int):
+    """Whole iterations of the workload with the CPU oracle (oracle.iteration: its own loop on its own halt
+    flags) until the time budget is used.  Returns (iterations, seconds)."""
     B, S = wl.B, wl.sl_max
-    active = np.ones(B, dtype=np.uint8)
-    sl = np.zeros(B, dtype=np.int64)
-    for j in range(S):
-        res = oracle.draft_step(W_D, h_D[j], (emitted + j + 1).astype(np.int32), np.full(B, j + 1, np.int32), clf,
-                                wl.tau, S, active=active, nthreads=nthreads)
-        sl[active == 1] = j + 1
-        stop = (forced_sl <= j + 1) if forced_sl is not None else (res.halt == 1)
-        active = (active.astype(bool) & ~stop).astype(np.uint8)
-        if not active.any():
-            break
-    sl_t = torch.as_tensor(sl, dtype=torch.int32)
-    off = inputs.row_offsets(sl_t).numpy()
-    rows = np.concatenate([H_T[b * (S + 1): b * (S + 1) + sl[b] + 1] for b in range(B)])
-    ids = np.concatenate([draft[b, : sl[b]] for b in range(B)]).astype(np.int32)
-    v = oracle.verify_ragged(W_T, rows, ids, off, nthreads=nthreads)
-    return emitted + v.n_accept + 1
+    pos = np.zeros(B, dtype=np.int32)
+    n, t0 = 0, time.perf_counter()
+    while n < at_least or (time.perf_counter() - t0 < budget_s and n < data.n_distinct):
+        d = data.idx(n)
+        h_D = inputs.bf16_bits(data.h_D[d].reshape(-1, wl.d_D)).reshape(S, B, wl.d_D)
+        H_T = inputs.bf16_bits(data.H_T[d].reshape(-1, wl.d_T)).reshape(B, S + 1, wl.d_T)
+        f = data.uniform_sl_cpu[d].numpy() if forced == "uniform" else None
+        r = oracle.iteration(W_D, h_D, W_T, H_T, pos, clf, wl.tau, S, sl_forced=f, draft_ids=data.draft_cpu[d].numpy(),
+                             nthreads=nthreads)
+        pos = (pos + r.n_accept + 1).astype(np.int32)
+        n += 1
+    return n, time.perf_counter() - t0
 
 
-def cpu_baseline(data: Data, wl, budget_s: float):
-    """The oracle, as it stands, on the host cores: whole iterations of the same workload until the
-    time budget is used (at least two)."""
+def cpu_baseline(data: Data, wl, forced, budget_s: float):
+    """The oracle, as it stands, on the host cores: whole iterations of the same workload until the time
+    budget is used, on all hardware threads and on one."""
     import oracle
     oracle.build()
     cores = oracle.hardware_threads()
-    W_D, W_T = inputs.bf16_bits(data.W_D[0]), inputs.bf16_bits(data.W_T)
+    W_D, W_T = inputs.bf16_bits(data.W_D_ring[0]), inputs.bf16_bits(data.W_T)
     W1, b1, w2, b2 = data.clf_params
     clf = oracle.Classifier(W1.numpy(), b1.numpy(), w2.numpy(), b2.numpy())
-    emitted = np.zeros(wl.B, dtype=np.int64)
-    n, t0 = 0, time.perf_counter()
-    while n < 2 or (time.perf_counter() - t0 < budget_s and n < data.n_distinct):
-        d = data.idx(n)
-        h_D = inputs.bf16_bits(data.h_D[d].reshape(-1, wl.d_D)).reshape(wl.sl_max, wl.B, wl.d_D)
-        H_T = inputs.bf16_bits(data.H_T[d])
-        forced = data.forced_sl[d].numpy() if data.forced_sl is not None else None
-        emitted = oracle_iteration(oracle, wl, W_D, W_T, clf, h_D, H_T, data.draft_full[d].numpy(), emitted, cores,
-                                   forced)
-        n += 1
-    dt = time.perf_counter() - t0
+    n, dt = oracle_iterations(oracle, wl, W_D, W_T, clf, data, forced, cores, budget_s, 2)
+    n1, dt1 = oracle_iterations(oracle, wl, W_D, W_T, clf, data, forced, 1, budget_s / 2, 1)
     return {"value": n / dt, "unit": UNIT, "cores": cores, "kind": "oracle",
-            "sample": f"first {n} iterations of {wl.name} (all vocabulary rows), {dt:.1f} s"}
+            "sample": f"first {n} iterations of {wl.name} (all vocabulary rows), {dt:.1f} s",
+            "value_1_thread": n1 / dt1, "sample_1_thread": f"first {n1} iterations, {dt1:.1f} s"}
 
 
 def run_reference(args):
@@ -626,13 +690,14 @@ def run_reference(args):
     oracle.build()
     wl = inputs.WORKLOADS[args.workload]
     K, Wm = args.steps, args.warmup
+    B, S = wl.B, wl.sl_max
     cores = oracle.hardware_threads()
     W1, b1, w2, b2 = inputs.classifier_params(wl.H, inputs.sub_seed(wl.seed, 3))
     clf = oracle.Classifier(W1.numpy(), b1.numpy(), w2.numpy(), b2.numpy())
     # calibrate on 1024 rows
     Vc = min(wl.V, 1024)
     Wc = inputs.bf16_bits(inputs.lm_head(Vc, wl.d_T, 1))
-    Hc = inputs.bf16_bits(inputs.hidden(wl.B * (wl.sl_max + 1), wl.d_T, 2))
+    Hc = inputs.bf16_bits(inputs.hidden(B * (S + 1), wl.d_T, 2))
     t0 = time.perf_counter()
     oracle.project(Wc, Hc, nthreads=cores)
     per_row = (time.perf_counter() - t0) / Vc * 1.5          # + draft steps
@@ -640,20 +705,20 @@ def run_reference(args):
     Vs = int(max(64, min(wl.V, budget / per_row)))
     W_D = inputs.bf16_bits(inputs.lm_head(Vs, wl.d_D, inputs.sub_seed(wl.seed, 1)))
     W_T = inputs.bf16_bits(inputs.lm_head(Vs, wl.d_T, inputs.sub_seed(wl.seed, 2)))
-    sub = wl.with_(V=Vs)
-    emitted = np.zeros(wl.B, dtype=np.int64)
+    pos = np.zeros(B, dtype=np.int32)
     total = 0.0
     rng = np.random.default_rng(wl.seed)
     for it in range(Wm + K):
-        h_D = inputs.bf16_bits(inputs.hidden(wl.sl_max * wl.B, wl.d_D, inputs.sub_seed(wl.seed, 4, it))).reshape(
-            wl.sl_max, wl.B, wl.d_D)
-        H_T = inputs.bf16_bits(inputs.hidden(wl.B * (wl.sl_max + 1), wl.d_T, inputs.sub_seed(wl.seed, 5, it)))
-        draft = rng.integers(0, Vs, size=(wl.B, wl.sl_max)).astype(np.int32)
+        h_D = inputs.bf16_bits(inputs.hidden(S * B, wl.d_D, inputs.sub_seed(wl.seed, 4, it))).reshape(S, B, wl.d_D)
+        H_T = inputs.bf16_bits(inputs.hidden(B * (S + 1), wl.d_T, inputs.sub_seed(wl.seed, 5, it))).reshape(
+            B, S + 1, wl.d_T)
+        draft = rng.integers(0, Vs, size=(B, S)).astype(np.int32)
         forced = None
         if wl.sl_mode == "uniform":
-            forced = inputs.uniform_sl(wl.B, 1, wl.sl_max, inputs.sub_seed(wl.seed, 8, it)).numpy()
+            forced = inputs.uniform_sl(B, 1, S, inputs.sub_seed(wl.seed, 8, it)).numpy()
         t0 = time.perf_counter()
-        emitted = oracle_iteration(oracle, sub, W_D, W_T, clf, h_D, H_T, draft, emitted, cores, forced)
+        r = oracle.iteration(W_D, h_D, W_T, H_T, pos, clf, wl.tau, S, sl_forced=forced, draft_ids=draft, nthreads=cores)
+        pos = (pos + r.n_accept + 1).astype(np.int32)
         if it >= Wm:
             total += time.perf_counter() - t0
     scaled = total * (wl.V / Vs)
@@ -672,17 +737,20 @@ def run_reference(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=1024)
+    ap.add_argument("--steps", type=int, default=256)
     ap.add_argument("--warmup", type=int, default=8)
+    ap.add_argument("--replays", type=int, default=24, help="timed replays of the graph of --steps iterations")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="vicuna_b1", choices=sorted(inputs.WORKLOADS))
-    ap.add_argument("--cpu-seconds", type=float, default=15.0)
+    ap.add_argument("--cpu-seconds", type=float, default=12.0)
     ap.add_argument("--reference-seconds", type=float, default=120.0)
     ap.add_argument("--kernel-path", type=int, default=0, help="0 automatic; 1..3 force a kernel family (tuning)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--no-static", action="store_true", help="skip the extra pass with SL forced to SL_max")
+    ap.add_argument("--no-static", action="store_true", help="skip the passes with other stopping policies and modes")
+    ap.add_argument("--no-other-workloads", action="store_true")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
+    args.replays = max(args.replays, 20)
     rank = int(os.environ.get("RANK", 0))
     world = int(os.environ.get("WORLD_SIZE", 1))
 

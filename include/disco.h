@@ -280,11 +280,15 @@ int disco_draft_loop(disco_ctx* ctx, const void* W_D, size_t w_step_stride, cons
  * Outputs (device): n_accept [B], bonus [B] as in disco_verify;
  *   target_ids int32 [B, sl_max + 1] or NULL: greedy target token of rows 0 .. sl[b] (others not written)
  *   row_off    int32 [B + 1] or NULL: exclusive prefix sums of sl[b] + 1, the offsets of the packed rows
+ *   pos_next   int32 [B] or NULL: pos0[b] + n_accept[b] + 1, the token count after this iteration (its
+ *              accepted tokens and the bonus token), i.e. the next iteration's pos0; may be pos0 itself
+ *              (pos0 int32 [B], device, is read only for this and may be NULL when pos_next is)
  * B * (sl_max + 1) <= max_rows of disco_create.
  */
 int disco_verify_sl(disco_ctx* ctx, const void* W_T, const void* H_T, const int32_t* draft_ids,
                     long long ids_stride_b, long long ids_stride_j, const int32_t* sl, int B, int sl_max,
-                    int32_t* n_accept, int32_t* bonus, int32_t* target_ids, int32_t* row_off, void* stream);
+                    int32_t* n_accept, int32_t* bonus, int32_t* target_ids, int32_t* row_off,
+                    const int32_t* pos0, int32_t* pos_next, void* stream);
 
 /*
  * One whole iteration as one call: disco_draft_loop, then disco_verify_sl on what it drafted.
@@ -297,7 +301,8 @@ int disco_iteration(disco_ctx* ctx, const void* W_D, size_t w_step_stride, const
                     const void* H_T, int B, const int32_t* pos0, const disco_clf* clf, float tau, int sl_max,
                     const int32_t* sl_forced, const int32_t* draft_ids,
                     int32_t* token, float* conf, uint8_t* halt, float* feats, int32_t* sl,
-                    int32_t* n_accept, int32_t* bonus, int32_t* target_ids, int32_t* row_off, void* stream);
+                    int32_t* n_accept, int32_t* bonus, int32_t* target_ids, int32_t* row_off,
+                    int32_t* pos_next, void* stream);
 
 /*
  * The same two operations for a caller whose per-step data lives in HOST memory (pinned memory
@@ -317,6 +322,21 @@ int disco_verify_ragged_host(disco_ctx* ctx, const void* W_T /*device*/, const v
                              const int32_t* draft_ids_host, const int32_t* row_off_host, int B, int R,
                              int32_t* n_accept_host, int32_t* bonus_host, int32_t* target_ids_host,
                              void* stream);
+
+/*
+ * disco_iteration for a caller whose per-iteration data lives in HOST memory: the hidden states of all steps,
+ * the target rows, pos0, sl_forced and draft_ids (either may be NULL) are host pointers, and so are the
+ * outputs token, conf, halt [sl_max, B], sl, n_accept, bonus [B] and pos_next [B] (or NULL; may be pos0_host
+ * itself).  One copy of each hidden-state block to device staging, the small arrays through pinned memory
+ * that the GPU maps, the whole iteration on the device, one synchronisation.  The LM heads and the classifier
+ * stay on the device.  Entries of steps a sequence did not take keep the caller's values.
+ */
+int disco_iteration_host(disco_ctx* ctx, const void* W_D /*device*/, size_t w_step_stride, const void* h_D_host,
+                         const void* W_T /*device*/, const void* H_T_host, int B, const int32_t* pos0_host,
+                         const disco_clf* clf /*device arrays*/, float tau, int sl_max,
+                         const int32_t* sl_forced_host, const int32_t* draft_ids_host,
+                         int32_t* token_host, float* conf_host, uint8_t* halt_host, int32_t* sl_host,
+                         int32_t* n_accept_host, int32_t* bonus_host, int32_t* pos_next_host, void* stream);
 
 /*
  * Draft step without any allocation.  (The paper has no counterpart: this is a packaging variant of

@@ -31,7 +31,7 @@ EXPORTS = [
     "disco_set_kernel_path", "disco_draft_step", "disco_verify", "disco_verify_ragged",
     "disco_draft_step_host", "disco_verify_ragged_host", "disco_draft_step_static", "disco_draft_step_ppl",
     "disco_draft_step_sample", "disco_verify_sample_ragged", "disco_extract_features",
-    "disco_draft_loop", "disco_verify_sl", "disco_iteration",
+    "disco_draft_loop", "disco_verify_sl", "disco_iteration", "disco_iteration_host",
 ]
 
 
@@ -82,9 +82,11 @@ def load() -> ctypes.CDLL:
                                             vp, vp, vp, vp, vp]
     sz, ll = ctypes.c_size_t, ctypes.c_longlong
     lib.disco_draft_loop.argtypes = [vp, vp, sz, vp, ci, vp, ctypes.POINTER(_Clf), cf, ci, vp, vp, vp, vp, vp, vp, vp]
-    lib.disco_verify_sl.argtypes = [vp, vp, vp, vp, ll, ll, vp, ci, ci, vp, vp, vp, vp, vp]
+    lib.disco_verify_sl.argtypes = [vp, vp, vp, vp, ll, ll, vp, ci, ci, vp, vp, vp, vp, vp, vp, vp]
     lib.disco_iteration.argtypes = [vp, vp, sz, vp, vp, vp, ci, vp, ctypes.POINTER(_Clf), cf, ci, vp, vp,
-                                    vp, vp, vp, vp, vp, vp, vp, vp, vp, vp]
+                                    vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp]
+    lib.disco_iteration_host.argtypes = [vp, vp, sz, vp, vp, vp, ci, vp, ctypes.POINTER(_Clf), cf, ci, vp, vp,
+                                         vp, vp, vp, vp, vp, vp, vp, vp]
     _lib = lib
     return lib
 
@@ -276,19 +278,19 @@ class Context:
             raise DiscoError(rc, "disco_draft_loop")
 
     def verify_sl(self, W_T, H_T, draft_ids, ids_stride_b: int, ids_stride_j: int, sl, B: int, sl_max: int,
-                  n_accept, bonus, target_ids=None, row_off=None, stream=None) -> None:
+                  n_accept, bonus, target_ids=None, row_off=None, pos0=None, pos_next=None, stream=None) -> None:
         """disco_verify_sl: H_T [B, sl_max + 1, d]; sl [B] on the device."""
         rc = self._lib.disco_verify_sl(
             self._h, _ptr(W_T, torch.bfloat16), _ptr(H_T, torch.bfloat16), _ptr(draft_ids, torch.int32),
             int(ids_stride_b), int(ids_stride_j), _ptr(sl, torch.int32), int(B), int(sl_max),
             _ptr(n_accept, torch.int32), _ptr(bonus, torch.int32), _ptr(target_ids, torch.int32),
-            _ptr(row_off, torch.int32), _stream(stream))
+            _ptr(row_off, torch.int32), _ptr(pos0, torch.int32), _ptr(pos_next, torch.int32), _stream(stream))
         if rc != OK:
             raise DiscoError(rc, "disco_verify_sl")
 
     def iteration(self, W_D, h_D, W_T, H_T, pos0, clf: Classifier, tau: float, sl_max: int, token, conf, halt, sl,
                   n_accept, bonus, sl_forced=None, draft_ids=None, feats=None, target_ids=None, row_off=None,
-                  w_step_stride: int = 0, stream=None) -> None:
+                  pos_next=None, w_step_stride: int = 0, stream=None) -> None:
         """disco_iteration: the draft phase and the verification of one iteration in one call."""
         B = int(h_D.shape[1])
         rc = self._lib.disco_iteration(
@@ -297,9 +299,24 @@ class Context:
             float(tau), int(sl_max), _ptr(sl_forced, torch.int32), _ptr(draft_ids, torch.int32),
             _ptr(token, torch.int32), _ptr(conf, torch.float32), _ptr(halt, torch.uint8), _ptr(feats, torch.float32),
             _ptr(sl, torch.int32), _ptr(n_accept, torch.int32), _ptr(bonus, torch.int32),
-            _ptr(target_ids, torch.int32), _ptr(row_off, torch.int32), _stream(stream))
+            _ptr(target_ids, torch.int32), _ptr(row_off, torch.int32), _ptr(pos_next, torch.int32), _stream(stream))
         if rc != OK:
             raise DiscoError(rc, "disco_iteration")
+
+    def iteration_host(self, W_D, h_D, W_T, H_T, pos0, clf: Classifier, tau: float, sl_max: int, token, conf, halt,
+                       sl, n_accept, bonus, sl_forced=None, draft_ids=None, pos_next=None, w_step_stride: int = 0,
+                       stream=None) -> None:
+        """disco_iteration_host: LM heads on the device, everything else CPU tensors."""
+        B = int(h_D.shape[1])
+        h = lambda t, dt: _ptr(t, dt, cuda=False)
+        rc = self._lib.disco_iteration_host(
+            self._h, _ptr(W_D, torch.bfloat16), int(w_step_stride), h(h_D, torch.bfloat16), _ptr(W_T, torch.bfloat16),
+            h(H_T, torch.bfloat16), B, h(pos0, torch.int32), ctypes.byref(clf._c), float(tau), int(sl_max),
+            h(sl_forced, torch.int32), h(draft_ids, torch.int32), h(token, torch.int32), h(conf, torch.float32),
+            h(halt, torch.uint8), h(sl, torch.int32), h(n_accept, torch.int32), h(bonus, torch.int32),
+            h(pos_next, torch.int32), _stream(stream))
+        if rc != OK:
+            raise DiscoError(rc, "disco_iteration_host")
 
     # ---------------------------------------------------------------- host-buffer calls
     def draft_step_host(self, W_D, h_D, pos, n_drafted, clf: Classifier, tau: float, sl_max: int,

@@ -66,6 +66,7 @@ struct disco_ctx {
     void* encode_tiled;            // cuTensorMapEncodeTiled, resolved through the runtime
     // device staging for the *_host entry points
     void* stage_hidden;
+    void* stage_hidden_draft;      // disco_iteration_host: the draft hidden states of all steps
     // Small inputs and outputs of the *_host entry points live in pinned host memory that the GPU maps:
     // the kernels read and write it in place, so a host call costs one copy (the hidden states), one
     // launch and one synchronisation.  *_h: host address, *_d: the same memory as the device sees it.
@@ -400,8 +401,8 @@ int disco_create(disco_ctx** out, int V, int d_draft, int d_target, int max_batc
             qres == cudaDriverEntryPointSuccess)
             c->encode_tiled = fn;
     }
-    const size_t n_int = (size_t)2 * max_batch + (size_t)max_rows + (max_batch + 1) + max_batch + 2 * (size_t)max_batch +
-                         (size_t)max_rows + 64;
+    // the largest layout is disco_iteration_host's: 6 arrays of max_batch words and 2 of max_rows
+    const size_t n_int = (size_t)8 * max_batch + (size_t)3 * max_rows + 64;
     const size_t hid = std::max((size_t)max_batch * d_draft, (size_t)max_rows * d_target) * 2;
     bool ok = true;
     ok = ok && cudaMalloc(&c->keys, (size_t)max_rows * sizeof(unsigned long long)) == cudaSuccess;
@@ -411,9 +412,10 @@ int disco_create(disco_ctx** out, int V, int d_draft, int d_target, int max_batc
     ok = ok && cudaMalloc(&c->final_stats, (size_t)c->part_rows * 2 * sizeof(float)) == cudaSuccess;
     ok = ok && cudaMalloc(&c->chain_alive, (size_t)max_batch + 64) == cudaSuccess;
     ok = ok && cudaMalloc(&c->stage_hidden, hid) == cudaSuccess;
+    ok = ok && cudaMalloc(&c->stage_hidden_draft, (size_t)max_rows * d_draft * 2) == cudaSuccess;
     ok = ok && cudaHostAlloc(&c->stage_int_h, n_int * sizeof(int32_t), cudaHostAllocMapped) == cudaSuccess;
-    ok = ok && cudaHostAlloc(&c->stage_float_h, (size_t)max_batch * (1 + kNFeat) * sizeof(float), cudaHostAllocMapped) == cudaSuccess;
-    ok = ok && cudaHostAlloc(&c->stage_byte_h, (size_t)max_batch * 2 + 64, cudaHostAllocMapped) == cudaSuccess;
+    ok = ok && cudaHostAlloc(&c->stage_float_h, ((size_t)max_batch * (1 + kNFeat) + max_rows) * sizeof(float), cudaHostAllocMapped) == cudaSuccess;
+    ok = ok && cudaHostAlloc(&c->stage_byte_h, (size_t)max_batch * 2 + max_rows + 64, cudaHostAllocMapped) == cudaSuccess;
     ok = ok && cudaHostGetDevicePointer(&c->stage_int_d, c->stage_int_h, 0) == cudaSuccess;
     ok = ok && cudaHostGetDevicePointer(&c->stage_float_d, c->stage_float_h, 0) == cudaSuccess;
     ok = ok && cudaHostGetDevicePointer(&c->stage_byte_d, c->stage_byte_h, 0) == cudaSuccess;
@@ -442,6 +444,7 @@ int disco_destroy(disco_ctx* c) {
     cudaFree(c->final_stats);
     cudaFree(c->chain_alive);
     cudaFree(c->stage_hidden);
+    cudaFree(c->stage_hidden_draft);
     cudaFreeHost(c->stage_int_h);
     cudaFreeHost(c->stage_float_h);
     cudaFreeHost(c->stage_byte_h);
@@ -824,13 +827,14 @@ int disco_draft_loop(disco_ctx* c, const void* W_D, size_t w_step_stride, const 
 
 int disco_verify_sl(disco_ctx* c, const void* W_T, const void* H_T, const int32_t* draft_ids, long long ids_stride_b,
                     long long ids_stride_j, const int32_t* sl, int B, int sl_max, int32_t* n_accept, int32_t* bonus,
-                    int32_t* target_ids, int32_t* row_off, void* stream) {
+                    int32_t* target_ids, int32_t* row_off, const int32_t* pos0, int32_t* pos_next, void* stream) {
     if (!c || !W_T || !H_T || !sl || !n_accept || !bonus) return DISCO_ERR_INVALID_ARG;
     if (B < 1 || sl_max < 0) return DISCO_ERR_INVALID_ARG;
     if (sl_max > 0 && !draft_ids) return DISCO_ERR_INVALID_ARG;
+    if (pos_next && !pos0) return DISCO_ERR_INVALID_ARG;
     const long long R = (long long)B * (sl_max + 1);
     if (R > c->max_rows) return DISCO_ERR_WORKSPACE;
-    const VerifyPadded pad{sl, ids_stride_b, ids_stride_j, row_off};
+    const VerifyPadded pad{sl, ids_stride_b, ids_stride_j, row_off, pos0, pos_next};
     return verify_common(c, W_T, H_T, draft_ids, nullptr, B, (int)R, sl_max, n_accept, bonus, target_ids, &pad, stream);
 }
 
@@ -838,7 +842,7 @@ int disco_iteration(disco_ctx* c, const void* W_D, size_t w_step_stride, const v
                     const void* H_T, int B, const int32_t* pos0, const disco_clf* clf, float tau, int sl_max,
                     const int32_t* sl_forced, const int32_t* draft_ids, int32_t* token, float* conf, uint8_t* halt,
                     float* feats, int32_t* sl, int32_t* n_accept, int32_t* bonus, int32_t* target_ids,
-                    int32_t* row_off, void* stream) {
+                    int32_t* row_off, int32_t* pos_next, void* stream) {
     // everything the second half will check, before the first half is enqueued
     if (!c || !W_T || !H_T || !n_accept || !bonus || !sl) return DISCO_ERR_INVALID_ARG;
     if (!aligned16(W_T) || !aligned16(H_T)) return DISCO_ERR_INVALID_ARG;
@@ -848,8 +852,9 @@ int disco_iteration(disco_ctx* c, const void* W_D, size_t w_step_stride, const v
     if (rc) return rc;
     if (draft_ids)
         return disco_verify_sl(c, W_T, H_T, draft_ids, sl_max, 1, sl, B, sl_max, n_accept, bonus, target_ids, row_off,
-                               stream);
-    return disco_verify_sl(c, W_T, H_T, token, 1, B, sl, B, sl_max, n_accept, bonus, target_ids, row_off, stream);
+                               pos0, pos_next, stream);
+    return disco_verify_sl(c, W_T, H_T, token, 1, B, sl, B, sl_max, n_accept, bonus, target_ids, row_off, pos0,
+                           pos_next, stream);
 }
 
 int disco_draft_step_host(disco_ctx* c, const void* W_D, const void* h_D_host, int B, const int32_t* pos_host,
@@ -924,6 +929,58 @@ int disco_verify_ragged_host(disco_ctx* c, const void* W_T, const void* H_T_host
     std::memcpy(n_accept_host, h_nacc, (size_t)B * 4);
     std::memcpy(bonus_host, h_bonus, (size_t)B * 4);
     if (target_ids_host) std::memcpy(target_ids_host, h_tids, (size_t)R * 4);
+    return DISCO_OK;
+}
+
+int disco_iteration_host(disco_ctx* c, const void* W_D, size_t w_step_stride, const void* h_D_host, const void* W_T,
+                         const void* H_T_host, int B, const int32_t* pos0_host, const disco_clf* clf, float tau,
+                         int sl_max, const int32_t* sl_forced_host, const int32_t* draft_ids_host,
+                         int32_t* token_host, float* conf_host, uint8_t* halt_host, int32_t* sl_host,
+                         int32_t* n_accept_host, int32_t* bonus_host, int32_t* pos_next_host, void* stream) {
+    if (!c || !h_D_host || !H_T_host || !pos0_host || !token_host || !conf_host || !halt_host || !sl_host ||
+        !n_accept_host || !bonus_host)
+        return DISCO_ERR_INVALID_ARG;
+    if (B < 1 || sl_max < 1) return DISCO_ERR_INVALID_ARG;
+    const size_t SB = (size_t)sl_max * B, R = (size_t)B * (sl_max + 1);
+    if (B > c->max_batch || R > (size_t)c->max_rows) return DISCO_ERR_WORKSPACE;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const size_t mb = (size_t)c->max_batch, mr = (size_t)c->max_rows;
+    // pinned, device-mapped staging: pos0 | forced | sl | n_accept | bonus | pos_next (max_batch each), ids | token
+    // (max_rows each); conf; halt
+    int32_t* h_pos = c->stage_int_h;
+    int32_t* h_forced = h_pos + mb;
+    int32_t* h_sl = h_forced + mb;
+    int32_t* h_nacc = h_sl + mb;
+    int32_t* h_bonus = h_nacc + mb;
+    int32_t* h_next = h_bonus + mb;
+    int32_t* h_ids = h_next + mb;
+    int32_t* h_tok = h_ids + mr;
+    float* h_conf = c->stage_float_h;
+    uint8_t* h_halt = c->stage_byte_h;
+    auto dev_i = [c](int32_t* h) { return c->stage_int_d + (h - c->stage_int_h); };
+    std::memcpy(h_pos, pos0_host, (size_t)B * 4);
+    if (sl_forced_host) std::memcpy(h_forced, sl_forced_host, (size_t)B * 4);
+    if (draft_ids_host) std::memcpy(h_ids, draft_ids_host, SB * 4);
+    // entries of steps a sequence does not take are not written by the kernels: hand the caller's values back
+    std::memcpy(h_tok, token_host, SB * 4);
+    std::memcpy(h_conf, conf_host, SB * 4);
+    std::memcpy(h_halt, halt_host, SB);
+    if (cudaMemcpyAsync(c->stage_hidden_draft, h_D_host, SB * c->d_draft * 2, cudaMemcpyHostToDevice, st) != cudaSuccess ||
+        cudaMemcpyAsync(c->stage_hidden, H_T_host, R * c->d_target * 2, cudaMemcpyHostToDevice, st) != cudaSuccess)
+        return DISCO_ERR_CUDA;
+    int rc = disco_iteration(c, W_D, w_step_stride, c->stage_hidden_draft, W_T, c->stage_hidden, B, dev_i(h_pos), clf, tau,
+                             sl_max, sl_forced_host ? dev_i(h_forced) : nullptr, draft_ids_host ? dev_i(h_ids) : nullptr,
+                             dev_i(h_tok), c->stage_float_d, c->stage_byte_d, nullptr, dev_i(h_sl), dev_i(h_nacc),
+                             dev_i(h_bonus), nullptr, nullptr, pos_next_host ? dev_i(h_next) : nullptr, stream);
+    if (rc) return rc;
+    if (cudaStreamSynchronize(st) != cudaSuccess) return DISCO_ERR_CUDA;
+    std::memcpy(token_host, h_tok, SB * 4);
+    std::memcpy(conf_host, h_conf, SB * 4);
+    std::memcpy(halt_host, h_halt, SB);
+    std::memcpy(sl_host, h_sl, (size_t)B * 4);
+    std::memcpy(n_accept_host, h_nacc, (size_t)B * 4);
+    std::memcpy(bonus_host, h_bonus, (size_t)B * 4);
+    if (pos_next_host) std::memcpy(pos_next_host, h_next, (size_t)B * 4);
     return DISCO_OK;
 }
 

@@ -31,6 +31,8 @@ struct VerifyPadded {
     const int32_t* sl;        // [B]; null: not this mode
     long long stride_b, stride_j;
     int32_t* row_off_out;     // [B + 1] or null: exclusive prefix sums of sl[b] + 1 (offsets of the packed rows)
+    const int32_t* pos0;      // [B] tokens generated before this iteration (with pos_next)
+    int32_t* pos_next;        // [B] or null: pos0[b] + n_accept[b] + 1, the next iteration's pos0 (may be pos0 itself)
 };
 
 struct TailParams {
@@ -777,6 +779,7 @@ __device__ __forceinline__ void verify_one_sequence(const unsigned long long* ke
     if (lane == 0) {
         n_accept[b] = n_acc;
         bonus[b] = bonus_tok;
+        if (pad.sl && pad.pos_next) pad.pos_next[b] = pad.pos0[b] + n_acc + 1;   // n_acc accepted tokens and the bonus token
     }
 }
 

@@ -60,8 +60,9 @@ def test_strerror_and_argument_checks_need_no_gpu(lib):
     assert lib.disco_verify_sample_ragged(None, z, z, z, z, z, 1, 1, z, z, z, z, z, z, z) == binding.ERR_INVALID_ARG
     assert lib.disco_extract_features(None, z, z, z, z, z, 1, z, z, z, z, z, z, z, z, z) == binding.ERR_INVALID_ARG
     assert lib.disco_draft_loop(None, z, 0, z, 1, z, None, 0.5, 1, z, z, z, z, z, z, z) == binding.ERR_INVALID_ARG
-    assert lib.disco_verify_sl(None, z, z, z, 1, 1, z, 1, 1, z, z, z, z, z) == binding.ERR_INVALID_ARG
-    assert lib.disco_iteration(None, z, 0, z, z, z, 1, z, None, 0.5, 1, z, z, z, z, z, z, z, z, z, z, z, z) == binding.ERR_INVALID_ARG
+    assert lib.disco_verify_sl(None, z, z, z, 1, 1, z, 1, 1, z, z, z, z, z, z, z) == binding.ERR_INVALID_ARG
+    assert lib.disco_iteration(None, z, 0, z, z, z, 1, z, None, 0.5, 1, z, z, z, z, z, z, z, z, z, z, z, z, z) == binding.ERR_INVALID_ARG
+    assert lib.disco_iteration_host(None, z, 0, z, z, z, 1, z, None, 0.5, 1, z, z, z, z, z, z, z, z, z, z) == binding.ERR_INVALID_ARG
     assert lib.disco_draft_step_host(None, z, z, 1, z, z, z, None, 0.5, 1, z, z, z, z, z) == binding.ERR_INVALID_ARG
     assert lib.disco_verify_ragged_host(None, z, z, z, z, 1, 1, z, z, z, z) == binding.ERR_INVALID_ARG
 

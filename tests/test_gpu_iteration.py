@@ -53,7 +53,8 @@ def gpu_iteration(ctx, W_D, W_T, h_D, H_T, pos0, clf, tau, S, sl_forced=None, dr
                n_accept=torch.full((B,), -7, dtype=torch.int32, device=dev),
                bonus=torch.full((B,), -7, dtype=torch.int32, device=dev),
                target_ids=torch.full((B, S + 1), -7, dtype=torch.int32, device=dev),
-               row_off=torch.full((B + 1,), -7, dtype=torch.int32, device=dev))
+               row_off=torch.full((B + 1,), -7, dtype=torch.int32, device=dev),
+               pos_next=torch.full((B,), -7, dtype=torch.int32, device=dev))
     p0 = torch.as_tensor(pos0, dtype=torch.int32).cuda()
     forced = None if sl_forced is None else torch.as_tensor(sl_forced, dtype=torch.int32).cuda()
     ids = None if draft_ids is None else torch.as_tensor(draft_ids, dtype=torch.int32).cuda().contiguous()
@@ -64,14 +65,17 @@ def gpu_iteration(ctx, W_D, W_T, h_D, H_T, pos0, clf, tau, S, sl_forced=None, dr
                            sl_forced=forced, feats=out["feats"], w_step_stride=stride, stream=stream)
             if ids is None:
                 ctx.verify_sl(Wt, Ht, out["token"], 1, B, out["sl"], B, S, out["n_accept"], out["bonus"],
-                              target_ids=out["target_ids"], row_off=out["row_off"], stream=stream)
+                              target_ids=out["target_ids"], row_off=out["row_off"], pos0=p0,
+                              pos_next=out["pos_next"], stream=stream)
             else:
                 ctx.verify_sl(Wt, Ht, ids, S, 1, out["sl"], B, S, out["n_accept"], out["bonus"],
-                              target_ids=out["target_ids"], row_off=out["row_off"], stream=stream)
+                              target_ids=out["target_ids"], row_off=out["row_off"], pos0=p0,
+                              pos_next=out["pos_next"], stream=stream)
         else:
             ctx.iteration(Wd, hd, Wt, Ht, p0, clf, tau, S, out["token"], out["conf"], out["halt"], out["sl"],
                           out["n_accept"], out["bonus"], sl_forced=forced, draft_ids=ids, feats=out["feats"],
-                          target_ids=out["target_ids"], row_off=out["row_off"], w_step_stride=stride, stream=stream)
+                          target_ids=out["target_ids"], row_off=out["row_off"], pos_next=out["pos_next"],
+                          w_step_stride=stride, stream=stream)
 
     if graph:
         st = torch.cuda.Stream()
@@ -89,7 +93,9 @@ def gpu_iteration(ctx, W_D, W_T, h_D, H_T, pos0, clf, tau, S, sl_forced=None, dr
     else:
         call()
     torch.cuda.synchronize()
-    return {k: v.cpu().numpy() for k, v in out.items()}
+    res = {k: v.cpu().numpy() for k, v in out.items()}
+    res["pos0"] = np.asarray(pos0, dtype=np.int32)
+    return res
 
 
 def check_iteration(oracle, got, ref, W_T, H_T, tau, S, draft_ids=None):
@@ -147,6 +153,8 @@ def check_iteration(oracle, got, ref, W_T, H_T, tau, S, draft_ids=None):
         else:
             assert got["n_accept"][b] == ref.n_accept[b] and got["bonus"][b] == ref.bonus[b]
     np.testing.assert_array_equal(got["row_off"], np.concatenate([[0], np.cumsum(ref.sl + 1)]))
+    if "pos0" in got:                                     # the next iteration's position base
+        np.testing.assert_array_equal(got["pos_next"], got["pos0"] + got["n_accept"] + 1)
     return exempt
 
 
@@ -210,6 +218,32 @@ def test_iteration_degenerate_policies(oracle):
     got = gpu_iteration(ctx, W_D, W_T, h_D, H_T, pos0, clf_g, 1.5, S, sl_forced=forced)
     assert list(got["sl"]) == list(np.minimum(forced, S))
     check_iteration(oracle, got, oracle.iteration(*args, 1.5, S, sl_forced=forced, nthreads=8), W_T, H_T, 1.5, S)
+    assert ctx.device_status() == 0
+    ctx.close()
+
+
+def test_iteration_host_entry_point_matches_the_device_one(oracle):
+    """disco_iteration_host: the same iteration with every per-iteration array in host memory; the position
+    base is advanced in place, as a host loop would carry it from one iteration to the next."""
+    V, dD, dT, B, S = 3000, 72, 136, 5, 6
+    W_D, W_T, h_D, H_T = make_inputs(V, dD, dT, B, S, seed=91)
+    pos0 = np.array([0, 2, 4, 6, 8], np.int32)
+    params = position_clf(cut=6.0)
+    rng = np.random.default_rng(9)
+    ids = rng.integers(0, V, size=(B, S)).astype(np.int32)
+    ctx = binding.Context(V, dD, dT, max_batch=B, max_rows=B * (S + 1), clf_hidden=8)
+    clf = to_gpu_clf(params)
+    dev = gpu_iteration(ctx, W_D, W_T, h_D, H_T, pos0, clf, 0.5, S, draft_ids=ids)
+    pin = lambda t: t.contiguous().pin_memory()
+    token, conf = pin(torch.full((S, B), -7, dtype=torch.int32)), pin(torch.full((S, B), -7.0))
+    halt = pin(torch.full((S, B), 77, dtype=torch.uint8))
+    sl, n_acc, bonus = (pin(torch.full((B,), -7, dtype=torch.int32)) for _ in range(3))
+    pos = pin(torch.from_numpy(pos0.copy()))
+    ctx.iteration_host(W_D.cuda(), pin(h_D), W_T.cuda(), pin(H_T), pos, clf, 0.5, S, token, conf, halt, sl, n_acc,
+                       bonus, draft_ids=pin(torch.from_numpy(ids)), pos_next=pos)
+    for k, t in (("token", token), ("conf", conf), ("halt", halt), ("sl", sl), ("n_accept", n_acc), ("bonus", bonus)):
+        np.testing.assert_array_equal(t.numpy(), dev[k])
+    np.testing.assert_array_equal(pos.numpy(), pos0 + dev["n_accept"] + 1)
     assert ctx.device_status() == 0
     ctx.close()
 
