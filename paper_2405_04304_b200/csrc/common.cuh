@@ -53,12 +53,13 @@ __device__ __forceinline__ bool chain_any_live(const ChainLink& c, int B, int la
     for (int b = lane; b < B; b += 32) any = any || __ldcg(c.alive + b) != 0;
     return __any_sync(0xffffffffu, any);
 }
-// By the thread that has just written sequence b's halt flag.
-__device__ __forceinline__ void chain_record(const ChainLink& c, int b, bool halt) {
-    if (!c.alive) return;
+// By the thread that has just written sequence b's halt flag.  Returns whether the sequence drafts on.
+__device__ __forceinline__ bool chain_record(const ChainLink& c, int b, bool halt) {
+    if (!c.alive) return !halt;
     const bool stop = c.sl_forced ? (c.step >= c.sl_forced[b]) : halt;
     __stcg(c.sl + b, c.step);
     __stcg(c.alive + b, static_cast<uint8_t>(stop ? 0 : 1));
+    return !stop;
 }
 
 // ------------------------------------------------------------------------------------------

@@ -14,6 +14,7 @@
 #include "umma_tail.cuh"
 #include "sample.cuh"
 #include "umma_gemv.cuh"
+#include "umma_gemv_loop.cuh"
 
 using namespace disco;
 
@@ -60,6 +61,7 @@ struct disco_ctx {
     int* status;
     float* final_stats;
     uint8_t* chain_alive;          // [max_batch] draft phase on the device: which sequences still draft
+    void* loop_rec;                // persistent draft-phase kernel: stamped 80-byte records, [4][CTA]; written by nothing else
     void* part_rec;                // draft step: 64-byte partial records, [sequence][CTA]
     void* stamped_rec;             // batched draft step: stamped 80-byte records, [sequence][CTA]; written by nothing else
     int part_slots;                // partials per row the buffers can hold
@@ -328,6 +330,70 @@ int launch_gemv(disco_ctx* c, const TailParams& t, cudaStream_t st) {
     return launch_gemv_rk<16>(c, g, mW, mH, st);
 }
 
+// The draft phase as one persistent kernel (1..4 sequences): see umma_gemv_loop.cuh.
+template <int RK>
+int launch_gemv_loop_rk(disco_ctx* c, GemvLoopParams& lp, const CUtensorMap& mW, const CUtensorMap& mH, cudaStream_t st) {
+    auto kern = umma_gemv_loop_kernel<RK>;
+    static KernelSetup setup;
+    size_t dyn_limit = 0;
+    if (!raise_smem_limit(c, setup, kern, 0, &dyn_limit)) return DISCO_ERR_CUDA;
+    GemvParams& g = lp.g;
+    const size_t fixed = gemv_loop_fixed_smem_bytes(RK, g.t.clf_H, g.t.d, g.h_rows);
+    if (dyn_limit < fixed + 2 * (size_t)g.b_bytes) return DISCO_ERR_UNSUPPORTED_SHAPE;
+    g.stages = (int)std::min<size_t>(kGemvMaxStages, (dyn_limit - fixed) / g.b_bytes);
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3((unsigned)c->sm_count);
+    cfg.blockDim = dim3(kGemvThreads);
+    cfg.dynamicSmemBytes = fixed + (size_t)g.stages * g.b_bytes;
+    cfg.stream = st;
+    // the steps hand over through global memory: every CTA has to be running, which a cooperative launch checks
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeCooperative;
+    attr[0].val.cooperative = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = c->pdl ? 2 : 1;
+    const cudaError_t e = cudaLaunchKernelEx(&cfg, kern, mW, mH, lp);
+    c->launches += 1;
+    return cuda_ok(e, "umma_gemv_loop_kernel launch") ? DISCO_OK : DISCO_ERR_CUDA;
+}
+
+bool gemv_loop_possible(const disco_ctx* c, int B, int sl_max, size_t w_step_stride) {
+    if (!c->encode_tiled || B > 4 || sl_max > kLoopMaxSteps) return false;
+    if (c->path != 0 && c->path != 3) return false;
+    if (w_step_stride != 0 && w_step_stride != (size_t)c->V * c->d_draft * 2) return false;   // one tensor map over all copies
+    if ((long long)c->V * sl_max > 0x7fffffffll) return false;
+    return (size_t)((c->d_draft + kUmmaBK - 1) / kUmmaBK) * 8 * 128 <= 48 * 1024;
+}
+
+int launch_gemv_loop(disco_ctx* c, const TailParams& t, int steps, size_t w_step_stride, cudaStream_t st) {
+    GemvLoopParams lp{};
+    GemvParams& g = lp.g;
+    g.t = t;
+    const int grid = c->sm_count;
+    if (grid > kGroupMaxRecords) return DISCO_ERR_UNSUPPORTED_SHAPE;
+    g.TR = (t.V + grid - 1) / grid;
+    g.t.slab_rows = g.TR;
+    g.tiles = (g.TR + 255) / 256;
+    g.TRt = (g.TR + g.tiles - 1) / g.tiles;
+    g.TRN = (g.TRt + 15) / 16 * 16;
+    g.b_bytes = (g.TRN * 128 + 1023) / 1024 * 1024;
+    g.h_rows = 8;
+    lp.steps = steps;
+    lp.w_rows_per_step = w_step_stride ? t.V : 0;
+    lp.flags = c->ticket + 64;
+    lp.epoch = c->ticket + 128;
+    lp.records = reinterpret_cast<float4*>(c->loop_rec);
+    CUtensorMap mW, mH;
+    if (!encode_bf16_2d(c, &mW, t.W, t.V * (w_step_stride ? steps : 1), t.d, g.TRN) ||
+        !encode_bf16_2d(c, &mH, t.H, t.R * steps, t.d, g.h_rows))
+        return DISCO_ERR_CUDA;
+    if (t.R == 1) return launch_gemv_loop_rk<1>(c, lp, mW, mH, st);
+    if (t.R == 2) return launch_gemv_loop_rk<2>(c, lp, mW, mH, st);
+    return launch_gemv_loop_rk<4>(c, lp, mW, mH, st);
+}
+
 void fill_scratch(const disco_ctx* c, TailParams& p) {
     p.part_rec = reinterpret_cast<float4*>(c->part_rec);
     p.keys = c->keys;
@@ -411,6 +477,8 @@ int disco_create(disco_ctx** out, int V, int d_draft, int d_target, int max_batc
     ok = ok && cudaMalloc(&c->status, 256) == cudaSuccess;
     ok = ok && cudaMalloc(&c->final_stats, (size_t)c->part_rows * 2 * sizeof(float)) == cudaSuccess;
     ok = ok && cudaMalloc(&c->chain_alive, (size_t)max_batch + 64) == cudaSuccess;
+    ok = ok && cudaMalloc(&c->loop_rec, (size_t)4 * c->sm_count * 80) == cudaSuccess;
+    ok = ok && cudaMemset(c->loop_rec, 0, (size_t)4 * c->sm_count * 80) == cudaSuccess;   // no stamp yet
     ok = ok && cudaMalloc(&c->stage_hidden, hid) == cudaSuccess;
     ok = ok && cudaMalloc(&c->stage_hidden_draft, (size_t)max_rows * d_draft * 2) == cudaSuccess;
     ok = ok && cudaHostAlloc(&c->stage_int_h, n_int * sizeof(int32_t), cudaHostAllocMapped) == cudaSuccess;
@@ -443,6 +511,7 @@ int disco_destroy(disco_ctx* c) {
     cudaFree(c->status);
     cudaFree(c->final_stats);
     cudaFree(c->chain_alive);
+    cudaFree(c->loop_rec);
     cudaFree(c->stage_hidden);
     cudaFree(c->stage_hidden_draft);
     cudaFreeHost(c->stage_int_h);
@@ -812,6 +881,32 @@ int disco_draft_loop(disco_ctx* c, const void* W_D, size_t w_step_stride, const 
     if (rc) return rc;
     const size_t h_step = (size_t)B * c->d_draft * 2;   // bytes of one step's hidden states
     if (h_step & 15u) return DISCO_ERR_INVALID_ARG;
+    if (gemv_loop_possible(c, B, sl_max, w_step_stride)) {
+        // a handful of sequences: all steps in one persistent kernel
+        cudaStream_t st = static_cast<cudaStream_t>(stream);
+        c->last_stream = st;
+        TailParams p{};
+        p.W = static_cast<const uint16_t*>(W_D);
+        p.H = static_cast<const uint16_t*>(h_D);
+        p.V = c->V;
+        p.d = c->d_draft;
+        p.R = B;
+        p.B = B;
+        fill_scratch(c, p);
+        p.chain = ChainLink{c->chain_alive, sl, pos0, sl_forced, 1};
+        p.clf_W1 = clf->W1;
+        p.clf_b1 = clf->b1;
+        p.clf_w2 = clf->w2;
+        p.clf_b2 = clf->b2;
+        p.clf_H = clf->H;
+        p.tau = tau;
+        p.sl_max = sl_max;
+        p.token = token;
+        p.conf = conf;
+        p.halt = halt;
+        p.feats = feats;
+        return launch_gemv_loop(c, p, sl_max, w_step_stride, st);
+    }
     for (int step = 1; step <= sl_max; ++step) {
         const size_t k = (size_t)(step - 1);
         const ChainLink link{c->chain_alive, sl, pos0, sl_forced, step};

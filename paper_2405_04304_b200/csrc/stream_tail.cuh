@@ -539,7 +539,7 @@ __device__ __forceinline__ float warp_halt_classifier(float x, float* feat_s, co
 }
 
 // Features of Eq. 2 from merged statistics, then classifier and stopping rule; one warp.
-// sel: lane k < 10 holds the k-th largest logit.
+// sel: lane k < 10 holds the k-th largest logit.  Returns (lane 0) whether the sequence drafts on.
 struct DraftOutputs {
     int32_t* token;
     float* conf;
@@ -551,7 +551,7 @@ struct DraftOutputs {
                      // 2: token and features, no classifier (bulk feature extraction)
     ChainLink chain; // draft phase chained on the device: the look-ahead bookkeeping goes with the halt flag
 };
-__device__ __forceinline__ void warp_draft_epilogue(const SoftmaxState& st, unsigned long long key, float sel, float fpos,
+__device__ __forceinline__ bool warp_draft_epilogue(const SoftmaxState& st, unsigned long long key, float sel, float fpos,
                                                     int n_drafted, float tau, int sl_max, float* feat_s, const float* W1,
                                                     const float* b1, const float* w2, const float* b2, int Hc, int b,
                                                     const DraftOutputs& o, int lane) {
@@ -561,7 +561,7 @@ __device__ __forceinline__ void warp_draft_epilogue(const SoftmaxState& st, unsi
             o.final_stats[2 * b] = st.m;
             o.final_stats[2 * b + 1] = st.Z;
         }
-        return;
+        return false;
     }
     if (o.nll_sum) {
         // Perplexity rule: the greedy token attains the largest logit, so -ln y(token) = ln Z.  The caller
@@ -577,7 +577,7 @@ __device__ __forceinline__ void warp_draft_epilogue(const SoftmaxState& st, unsi
             o.final_stats[2 * b] = st.m;
             o.final_stats[2 * b + 1] = st.Z;
         }
-        return;
+        return false;
     }
     const float inv_Z = 1.f / st.Z;
     const float prob = (lane < kTopK && sel > DISCO_NEG_INF) ? __expf(sel - st.m) * inv_Z : 0.f;
@@ -590,19 +590,21 @@ __device__ __forceinline__ void warp_draft_epilogue(const SoftmaxState& st, unsi
             o.final_stats[2 * b + 1] = st.Z;
         }
         if (o.feats && lane < kNFeat) o.feats[(size_t)b * kNFeat + lane] = x;
-        return;
+        return false;
     }
     const float C = warp_halt_classifier(x, feat_s, W1, b1, w2, b2, Hc, lane);
+    bool goes_on = false;
     if (lane == 0) {
         const bool halt = (C < tau) || (n_drafted >= sl_max);
         o.token[b] = key_index(key);
         o.conf[b] = C;
         o.halt[b] = halt ? 1 : 0;
-        chain_record(o.chain, b, halt);
+        goes_on = chain_record(o.chain, b, halt);
         o.final_stats[2 * b] = st.m;
         o.final_stats[2 * b + 1] = st.Z;
     }
     if (o.feats && lane < kNFeat) o.feats[(size_t)b * kNFeat + lane] = x;
+    return goes_on;   // lane 0: the sequence drafts another token after this one
 }
 
 // Inverse-CDF draw of one token by one warp, after warp_merge_partials: the records are in vocabulary

@@ -80,6 +80,10 @@ __device__ __forceinline__ void tma_load_2d(void* dst_smem, const CUtensorMap* t
         "l"(tmap), "r"(c0), "r"(c1), "r"(smem_addr(bar))
         : "memory");
 }
+// Bring one box of a tensor map into L2 (no shared-memory destination, nothing to wait for).
+__device__ __forceinline__ void tma_prefetch_l2_2d(const CUtensorMap* tmap, int c0, int c1) {
+    asm volatile("cp.async.bulk.prefetch.tensor.2d.L2.global.tile [%0, {%1, %2}];" ::"l"(tmap), "r"(c0), "r"(c1) : "memory");
+}
 __device__ __forceinline__ void prefetch_tensormap(const CUtensorMap* tmap) {
     asm volatile("prefetch.tensormap [%0];" ::"l"(tmap) : "memory");
 }
