@@ -398,8 +398,13 @@ umma_tail_kernel(const __grid_constant__ CUtensorMap tmap_W, const __grid_consta
                             }
                         }
                         if (!STATS) {
+                            // A logit enters a row's ten largest with probability about 10 / (columns seen so far): the
+                            // insertion network runs only for the pairs that some lane's row needs (a warp-wide vote,
+                            // so the branch does not diverge).
 #pragma unroll
-                            for (int j = 0; j < 32; j += 2) top.push2(z[j], z[j + 1]);
+                            for (int j = 0; j < 32; j += 2) {
+                                if (__any_sync(kFullMask, fmaxf(z[j], z[j + 1]) > top.t[kTopK - 1])) top.push2(z[j], z[j + 1]);
+                            }
                         }
                         if (keep_logits) {
                             float* dst = p.probs + (size_t)row * p.V + v0 + cbase;
