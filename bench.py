@@ -389,10 +389,14 @@ def rooflines(wl, K: int, res: dict, hbm_peak: float, tensor_peak: float, peak_k
                    "avg_launch_us": t_v / K * 1e6, "rows_per_launch": R, "rows_counted_per_launch": rows / K,
                    "traffic": None,
                    "tensor_tflops": verify_flops / t_v / 1e12}
+    draft_launches = res["launches"]["draft"]
     roof_draft = {"kernel": "draft-step tail", "bound": "hbm", "achieved": draft_bytes / t_d / 1e9,
-                  "peak": hbm_peak, "peak_kind": peak_kind, "unit": "GB/s", "launches": n_live,
-                  "launches_without_work": K * S - n_live, "avg_launch_us": t_d / n_live * 1e6, "traffic": None,
-                  "note": "time of the draft phases (launches without work included) over the steps that had work"}
+                  "peak": hbm_peak, "peak_kind": peak_kind, "unit": "GB/s", "steps": n_live,
+                  "kernel_launches": draft_launches, "avg_step_us": t_d / n_live * 1e6,
+                  "avg_launch_us": t_d / max(draft_launches, 1) * 1e6, "traffic": None,
+                  "note": ("one persistent kernel per iteration runs all its draft steps" if draft_launches == K else
+                           "one launch per draft step of the cap; launches that find no sequence drafting return at once") +
+                          "; achieved = algorithmic bytes of the steps that had work over the time of all draft launches"}
     for r in (roof_verify, roof_draft):
         r["traffic"] = ncu_traffic(wl.name, r["kernel"])
         r["frac"] = r["achieved"] / r["peak"]

@@ -97,6 +97,17 @@ int disco_launch_count(disco_ctx* ctx, long long* out);
  * tcgen05 kernel with the vocabulary on the TMEM lanes (draft step, up to 16 sequences). */
 int disco_set_kernel_path(disco_ctx* ctx, int which);
 
+/* For the test-suite: how the bounded device-side waits behave when what they wait for never comes.
+ *   wait_budget_clocks  SM clock ticks after which a wait gives up and records DISCO_ERR_TIMEOUT in the device
+ *                       status word (0 restores the default of about 0.05 s); applies to every context of the
+ *                       process
+ *   withhold_records    non-zero: the batched draft step (the tensor-core kernel for five sequences and more)
+ *                       makes its finishing warps look for per-CTA records that no CTA publishes, so that
+ *                       their wait runs out.  The kernel still returns by itself; its outputs are then
+ *                       meaningless and the context must be destroyed (see DISCO_ERR_TIMEOUT).
+ * Nothing traps, faults or waits without bound in either setting. */
+int disco_test_hooks(disco_ctx* ctx, long long wait_budget_clocks, int withhold_records);
+
 /*
  * One draft step for B sequences (Sec. 3, Eq. 2).  B = 1 is the single-sequence call.
  *   W_D        bf16 [V, d_draft]   draft LM head

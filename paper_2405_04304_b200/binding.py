@@ -31,7 +31,7 @@ EXPORTS = [
     "disco_set_kernel_path", "disco_draft_step", "disco_verify", "disco_verify_ragged",
     "disco_draft_step_host", "disco_verify_ragged_host", "disco_draft_step_static", "disco_draft_step_ppl",
     "disco_draft_step_sample", "disco_verify_sample_ragged", "disco_extract_features",
-    "disco_draft_loop", "disco_verify_sl", "disco_iteration", "disco_iteration_host",
+    "disco_draft_loop", "disco_verify_sl", "disco_iteration", "disco_iteration_host", "disco_test_hooks",
 ]
 
 
@@ -66,6 +66,7 @@ def load() -> ctypes.CDLL:
     lib.disco_last_device_status.argtypes = [vp, ctypes.POINTER(ci)]
     lib.disco_launch_count.argtypes = [vp, ctypes.POINTER(ctypes.c_longlong)]
     lib.disco_set_kernel_path.argtypes = [vp, ci]
+    lib.disco_test_hooks.argtypes = [vp, ctypes.c_longlong, ci]
     lib.disco_draft_step.argtypes = [vp, vp, vp, ci, vp, vp, vp, ctypes.POINTER(_Clf), cf, ci,
                                      vp, vp, vp, vp, vp, vp]
     lib.disco_draft_step_ppl.argtypes = [vp, vp, vp, ci, vp, vp, vp, cf, ci, vp, vp, vp, vp]
@@ -183,6 +184,11 @@ class Context:
         out = ctypes.c_longlong()
         self._lib.disco_launch_count(self._h, ctypes.byref(out))
         return int(out.value)
+
+    def test_hooks(self, wait_budget_clocks: int = 0, withhold_records: bool = False) -> None:
+        rc = self._lib.disco_test_hooks(self._h, int(wait_budget_clocks), int(bool(withhold_records)))
+        if rc != OK:
+            raise DiscoError(rc, "disco_test_hooks")
 
     def set_kernel_path(self, which: int) -> None:
         rc = self._lib.disco_set_kernel_path(self._h, int(which))

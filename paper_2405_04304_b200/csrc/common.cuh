@@ -14,8 +14,12 @@ constexpr int kNFeat = DISCO_NFEAT;
 constexpr unsigned kFullMask = 0xffffffffu;
 constexpr int kNoIndex = 0x7fffffff;
 
-// Bounded-wait budget: a barrier wait gives up after this many clock ticks (about 0.05 s).
-constexpr long long kWaitBudgetClocks = 100000000ll;
+// Bounded-wait budget: a wait gives up after this many clock ticks (about 0.05 s by default).  A device
+// variable, one copy per translation unit, so that a test can shorten it (disco_test_hooks) and make a wait
+// run out without anything hanging.
+constexpr long long kDefaultWaitBudgetClocks = 100000000ll;
+static __device__ long long g_wait_budget_clocks = kDefaultWaitBudgetClocks;
+#define kWaitBudgetClocks (*reinterpret_cast<volatile long long*>(&g_wait_budget_clocks))
 
 // ------------------------------------------------------------------------------------------
 // status word

@@ -53,6 +53,7 @@ struct disco_ctx {
     int pdl;  // launch the streaming kernel with programmatic stream serialization (DISCO_PDL=0 turns it off)
     long long launches;
     cudaStream_t last_stream;  // stream of the most recent enqueue (disco_last_device_status waits for it only)
+    unsigned int test_stamp_skew;  // disco_test_hooks
     // scratch for cross-block reductions
     int part_rows;  // rows the partial buffers can hold
     int max_grid;
@@ -539,6 +540,14 @@ int disco_launch_count(disco_ctx* c, long long* out) {
     return DISCO_OK;
 }
 
+int disco_test_hooks(disco_ctx* c, long long wait_budget_clocks, int withhold_records) {
+    if (!c || wait_budget_clocks < 0) return DISCO_ERR_INVALID_ARG;
+    const long long budget = wait_budget_clocks ? wait_budget_clocks : kDefaultWaitBudgetClocks;
+    if (cudaMemcpyToSymbol(g_wait_budget_clocks, &budget, sizeof(budget)) != cudaSuccess) return DISCO_ERR_CUDA;
+    c->test_stamp_skew = withhold_records ? 0x40000000u : 0u;
+    return DISCO_OK;
+}
+
 int disco_set_kernel_path(disco_ctx* c, int which) {
     if (!c || which < 0 || which > 3) return DISCO_ERR_INVALID_ARG;
     c->path = which;
@@ -671,6 +680,7 @@ int draft_step_common(disco_ctx* c, const void* W_D, const void* h_D, int d, int
         f.nll_sum = nll_sum;
         f.stats_only = stats_only;
         f.epoch = c->ticket + 48;
+        f.test_stamp_skew = c->test_stamp_skew;
         if (chain) f.chain = *chain;
         rc = stats_only == 1 ? launch_umma<true, true>(c, W_D, h_D, d, B, probs, &f, nullptr, st)
                         : launch_umma<true>(c, W_D, h_D, d, B, probs, &f, nullptr, st);

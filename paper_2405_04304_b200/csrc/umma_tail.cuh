@@ -169,6 +169,7 @@ struct DraftFinalParams {
     int stats_only;
     unsigned int* epoch;  // [0] launches completed so far (stamp of this launch = that + 1), [1] finishing warps done
     ChainLink chain;      // alive != null: this launch is one step of a draft phase chained on the device
+    unsigned int test_stamp_skew;   // 0.  Tests: the finishing warps expect a stamp that no CTA writes, so their wait runs out
 };
 
 // One warp finishes sequence b from its NP partial records.  clf_s: classifier parameters in shared
@@ -481,7 +482,8 @@ umma_tail_kernel(const __grid_constant__ CUtensorMap tmap_W, const __grid_consta
                 for (;;) {
                     // a masked sequence still waits for its records: the stamp may only advance once
                     // every CTA has taken part in this launch
-                    umma_finish_sequence(f, p.part_rec, p.CN, b, act, fpos, nd, feat16, clf_s, stamp, p.status, lane);
+                    umma_finish_sequence(f, p.part_rec, p.CN, b, act, fpos, nd, feat16, clf_s, stamp + f.test_stamp_skew,
+                                         p.status, lane);
                     b += kUmmaEpiWarps * (int)gridDim.x;
                     if (b >= f.B) break;
                     act = chain_seq_live(f.chain, f.active, b);

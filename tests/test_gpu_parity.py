@@ -806,3 +806,37 @@ def test_look_ahead_is_monotone_in_the_threshold_at_full_size():
         below = c0 < np.float32(tau)
         first = np.where(below.any(axis=0), below.argmax(axis=0) + 1, S)
         np.testing.assert_array_equal(sl[tau], np.minimum(first, S))
+
+
+# ---------------------------------------------------------------------------------- bounded waits
+def test_a_wait_that_runs_out_is_reported_and_nothing_hangs():
+    """The finishing warps of the batched draft step wait (bounded) for the per-CTA records of their sequence.
+    With the test hook set those records never come: the wait must give up within the (shortened) budget, the
+    kernel must return by itself, the status word must say DISCO_ERR_TIMEOUT, and after the context has been
+    thrown away a fresh one must work as before."""
+    V, d, B = 5000, 128, 12
+    W = inputs.lm_head(V, d, seed=31, std=0.2).cuda()
+    h = inputs.hidden(B, d, seed=32)
+    clf = to_gpu_clf(make_clf(16, seed=33))
+    pos, nd = np.arange(1, B + 1, dtype=np.int32), np.ones(B, np.int32)
+    good_ctx = _ctx(V, d, 8, max_batch=B, H=16)
+    good = gpu_draft_step(good_ctx, W, h, pos, nd, clf, 0.5, 4)
+    assert good_ctx.device_status() == 0
+    ctx = _ctx(V, d, 8, max_batch=B, H=16)
+    ctx.test_hooks(wait_budget_clocks=2_000_000, withhold_records=True)      # about a millisecond
+    try:
+        gpu_draft_step(ctx, W, h, pos, nd, clf, 0.5, 4)                       # returns: the kernel ended by itself
+        assert ctx.device_status() == binding.ERR_TIMEOUT
+        assert ctx.device_status() == 0                                       # the word is cleared by the query
+    finally:
+        ctx.test_hooks(0, False)                                              # default budget again
+        ctx.close()
+    again = gpu_draft_step(good_ctx, W, h, pos, nd, clf, 0.5, 4)              # other contexts are not affected
+    fresh = _ctx(V, d, 8, max_batch=B, H=16)
+    new = gpu_draft_step(fresh, W, h, pos, nd, clf, 0.5, 4)
+    for k in ("token", "conf", "halt", "feats"):
+        np.testing.assert_array_equal(good[k], again[k])
+        np.testing.assert_array_equal(good[k], new[k])
+    assert fresh.device_status() == 0 and good_ctx.device_status() == 0
+    fresh.close()
+    good_ctx.close()
