@@ -62,6 +62,8 @@ struct disco_ctx {
     int* status;
     float* final_stats;
     uint8_t* chain_alive;          // [max_batch] draft phase on the device: which sequences still draft
+    void* pack_rows;               // fixed-shape verification with many rows: the rows that count, packed
+    int32_t* pack_off;             // [max_batch + 1] their offsets; the last entry is the row count
     void* loop_rec;                // persistent draft-phase kernel: stamped 80-byte records, [4][CTA]; written by nothing else
     void* part_rec;                // draft step: 64-byte partial records, [sequence][CTA]
     void* stamped_rec;             // batched draft step: stamped 80-byte records, [sequence][CTA]; written by nothing else
@@ -213,7 +215,8 @@ bool umma_possible(const disco_ctx* c, int R) {
 // Launch the tcgen05 kernel for R hidden rows of width d against the LM head W [V, d].
 template <bool DRAFT, bool STATS = false>
 int launch_umma(disco_ctx* c, const void* W, const void* H, int d, int R, float* probs,
-                const DraftFinalParams* draft_final, const UmmaParams* fused, cudaStream_t st) {
+                const DraftFinalParams* draft_final, const UmmaParams* fused, cudaStream_t st,
+                const int32_t* dev_R = nullptr) {
     UmmaParams p{};
     if (fused) p = *fused;  // verification finished by the main kernel's last CTA
     p.V = c->V;
@@ -228,6 +231,8 @@ int launch_umma(disco_ctx* c, const void* W, const void* H, int d, int R, float*
     p.TPC = std::max(1, (c->V + tile_target * p.CN - 1) / (tile_target * p.CN));
     p.TR = (c->V + p.CN * p.TPC - 1) / (p.CN * p.TPC);
     p.TRN = std::max(16, (p.TR + 15) / 16 * 16);
+    p.dev_R = dev_R;
+    if (dev_R) p.TRN = 256;   // the kernel derives the tiling from the device-side row count; the box is the largest tile
     p.a_rows = p.MT > 1 ? 128 : std::max(8, (R + 7) / 8 * 8);
     // Draft step with few rows: copies of the rows fill the other TMEM lane quadrants, so that the
     // epilogue (heavy there) runs on every warp scheduler.  Verification's epilogue is a compare per
@@ -253,7 +258,7 @@ int launch_umma(disco_ctx* c, const void* W, const void* H, int d, int R, float*
     if (!raise_smem_limit(c, setup, kern, (size_t)kUmmaSmemBytes + umma_clf_bytes(DISCO_MAX_CLF_HIDDEN), nullptr))
         return DISCO_ERR_CUDA;
     cudaLaunchConfig_t cfg{};
-    cfg.gridDim = dim3((unsigned)(p.MT * p.CN));
+    cfg.gridDim = dim3((unsigned)(dev_R ? c->sm_count : p.MT * p.CN));
     cfg.blockDim = dim3(kUmmaThreads);
     cfg.dynamicSmemBytes = kUmmaSmemBytes + (draft_final ? umma_clf_bytes(draft_final->clf_H) : 0);
     cfg.stream = st;
@@ -478,6 +483,8 @@ int disco_create(disco_ctx** out, int V, int d_draft, int d_target, int max_batc
     ok = ok && cudaMalloc(&c->status, 256) == cudaSuccess;
     ok = ok && cudaMalloc(&c->final_stats, (size_t)c->part_rows * 2 * sizeof(float)) == cudaSuccess;
     ok = ok && cudaMalloc(&c->chain_alive, (size_t)max_batch + 64) == cudaSuccess;
+    ok = ok && cudaMalloc(&c->pack_rows, (size_t)max_rows * d_target * 2) == cudaSuccess;
+    ok = ok && cudaMalloc(&c->pack_off, ((size_t)max_batch + 2) * sizeof(int32_t)) == cudaSuccess;
     ok = ok && cudaMalloc(&c->loop_rec, (size_t)4 * c->sm_count * 80) == cudaSuccess;
     ok = ok && cudaMemset(c->loop_rec, 0, (size_t)4 * c->sm_count * 80) == cudaSuccess;   // no stamp yet
     ok = ok && cudaMalloc(&c->stage_hidden, hid) == cudaSuccess;
@@ -513,6 +520,8 @@ int disco_destroy(disco_ctx* c) {
     cudaFree(c->final_stats);
     cudaFree(c->chain_alive);
     cudaFree(c->loop_rec);
+    cudaFree(c->pack_rows);
+    cudaFree(c->pack_off);
     cudaFree(c->stage_hidden);
     cudaFree(c->stage_hidden_draft);
     cudaFreeHost(c->stage_int_h);
@@ -727,6 +736,27 @@ int verify_common(disco_ctx* c, const void* W_T, const void* H_T, const int32_t*
     if (pad) p.padded = *pad;
     const bool use_umma = umma_possible(c, R) && (c->path == 2 || (c->path == 0 && R >= 2));
     if (!use_umma) return run_stream<false>(c, p, 0, st);
+    // Fixed-shape rows beyond one tile of 128: the projection is no longer free of charge for the rows that do not
+    // count, so they are packed first and the tensor-core kernel tiles for the row count it finds on the device.
+    const int32_t* dev_R = nullptr;
+    if (pad && R > 128) {
+        PackParams pk{};
+        pk.H = static_cast<const uint16_t*>(H_T);
+        pk.packed = static_cast<uint16_t*>(c->pack_rows);
+        pk.sl = pad->sl;
+        pk.off = c->pack_off;
+        pk.off_user = pad->row_off_out;
+        pk.B = B;
+        pk.SL = SL;
+        pk.d = c->d_target;
+        const cudaError_t e = launch_after(c, pack_rows_kernel, dim3((unsigned)(SL + 1), (unsigned)B), dim3(128), 0, st, pk);
+        c->launches += 1;
+        if (!cuda_ok(e, "pack_rows_kernel launch")) return DISCO_ERR_CUDA;
+        H_T = c->pack_rows;
+        p.padded.packed_off = c->pack_off;
+        p.padded.row_off_out = nullptr;
+        dev_R = c->pack_off + B;
+    }
     if (B <= 16) {  // few sequences: the last CTA of the main kernel finishes the job, no second launch
         UmmaParams fp{};
         fp.fuse_final = 1;
@@ -739,9 +769,9 @@ int verify_common(disco_ctx* c, const void* W_T, const void* H_T, const int32_t*
         fp.bonus = bonus;
         fp.target_ids = target_ids;
         fp.padded = p.padded;
-        return launch_umma<false>(c, W_T, H_T, c->d_target, R, nullptr, nullptr, &fp, st);
+        return launch_umma<false>(c, W_T, H_T, c->d_target, R, nullptr, nullptr, &fp, st, dev_R);
     }
-    int rc = launch_umma<false>(c, W_T, H_T, c->d_target, R, nullptr, nullptr, nullptr, st);
+    int rc = launch_umma<false>(c, W_T, H_T, c->d_target, R, nullptr, nullptr, nullptr, st, dev_R);
     if (rc) return rc;
     VerifyFinalParams f{};
     f.keys = c->keys;
@@ -756,6 +786,7 @@ int verify_common(disco_ctx* c, const void* W_T, const void* H_T, const int32_t*
     f.status = c->status;
     f.ticket = c->ticket + 16;
     f.padded = p.padded;
+    f.dev_R = dev_R;
     verify_finalize_kernel<<<(B + 3) / 4, 128, 0, st>>>(f);
     c->launches += 1;
     return cuda_ok(cudaGetLastError(), "verify_finalize_kernel launch") ? DISCO_OK : DISCO_ERR_CUDA;

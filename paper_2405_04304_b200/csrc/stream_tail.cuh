@@ -33,6 +33,9 @@ struct VerifyPadded {
     int32_t* row_off_out;     // [B + 1] or null: exclusive prefix sums of sl[b] + 1 (offsets of the packed rows)
     const int32_t* pos0;      // [B] tokens generated before this iteration (with pos_next)
     int32_t* pos_next;        // [B] or null: pos0[b] + n_accept[b] + 1, the next iteration's pos0 (may be pos0 itself)
+    const int32_t* packed_off;  // [B + 1] or null.  Non-null: the hidden rows were packed before the projection (row_off of
+                                // the packed rows, computed on the device): the keys of sequence b start at packed_off[b],
+                                // while its outputs keep the fixed-shape layout
 };
 
 struct TailParams {
@@ -728,15 +731,17 @@ __device__ __forceinline__ void verify_one_sequence(const unsigned long long* ke
                                                     int32_t* n_accept, int32_t* bonus, int32_t* target_ids,
                                                     int* status, int lane, const VerifyPadded& pad) {
     int r0, r1;
+    int out0 = -1;            // first row of the sequence in target_ids when that differs from its first key row
     long long id0, idj = 1;
     bool bad;
     if (pad.sl) {
         const int s = __ldcg(pad.sl + b);
-        r0 = b * (SL + 1);
+        out0 = b * (SL + 1);
+        r0 = pad.packed_off ? __ldcg(pad.packed_off + b) : out0;
         r1 = r0 + s + 1;
         id0 = (long long)b * pad.stride_b;
         idj = pad.stride_j;
-        bad = s < 0 || s > SL;
+        bad = s < 0 || s > SL || r0 < 0 || r1 > R;
     } else {
         if (row_off) {
             r0 = row_off[b];
@@ -766,7 +771,7 @@ __device__ __forceinline__ void verify_one_sequence(const unsigned long long* ke
         bool match = false;
         if (j <= sl) {
             a = key_index(__ldcg(keys + r0 + j));
-            if (target_ids) target_ids[r0 + j] = a;
+            if (target_ids) target_ids[(out0 >= 0 ? out0 : r0) + j] = a;
             match = (j < sl) && (__ldcg(draft_ids + id0 + j * idj) == a);
         }
         if (n_acc < 0) {  // warp-uniform
@@ -1089,6 +1094,63 @@ __global__ void __launch_bounds__((NW + 1) * 32, 1) stream_tail_kernel(const __g
         for (int r = tid; r < p.R; r += BAR_THREADS) p.keys[r] = 0ull;
     }
     if (tid == 0) *p.ticket = 0u;
+}
+
+// Fixed-shape verification with many rows: the rows that count (the first sl[b] + 1 of each sequence's SL + 1) are
+// copied next to each other, so that the projection does not pay for the padding.  Block (b, j) copies row j of
+// sequence b to packed row off[b] + j, where off[b] = sum over b' < b of (sl[b'] + 1) (every block sums what it
+// needs itself; block (0, 0) also writes all B + 1 offsets, off[B] = the number of packed rows).
+// grid = (SL + 1, B), 128 threads.
+struct PackParams {
+    const uint16_t* H;    // bf16 [B, SL + 1, d]
+    uint16_t* packed;     // bf16 [<= B * (SL + 1), d]
+    const int32_t* sl;    // [B]
+    int32_t* off;         // [B + 1]
+    int32_t* off_user;    // [B + 1] or null: a second copy for the caller
+    int B, SL, d;
+};
+static __global__ void __launch_bounds__(128) pack_rows_kernel(const PackParams p) {
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    __shared__ int s_part[4];
+    const int j = blockIdx.x, b = blockIdx.y;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    auto rows_of = [&](int q) { return min(max(__ldcg(p.sl + q), 0), p.SL) + 1; };
+    if (j == 0 && b == 0) {   // all offsets, by one warp
+        if (warp == 0) {
+            int base = 0;
+            for (int q0 = 0; q0 < p.B; q0 += 32) {
+                const int q = q0 + lane;
+                const int rows = q < p.B ? rows_of(q) : 0;
+                int incl = rows;
+#pragma unroll
+                for (int o = 1; o < 32; o <<= 1) {
+                    const int t = __shfl_up_sync(kFullMask, incl, o);
+                    if (lane >= o) incl += t;
+                }
+                if (q < p.B) {
+                    p.off[q] = base + incl - rows;
+                    if (p.off_user) p.off_user[q] = base + incl - rows;
+                }
+                base += __shfl_sync(kFullMask, incl, 31);
+            }
+            if (lane == 0) {
+                p.off[p.B] = base;
+                if (p.off_user) p.off_user[p.B] = base;
+            }
+        }
+    }
+    if (j >= rows_of(b)) return;   // a padding row (uniform over the block)
+    int part = 0;
+    for (int q = threadIdx.x; q < b; q += blockDim.x) part += rows_of(q);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) part += __shfl_xor_sync(kFullMask, part, o);
+    if (lane == 0) s_part[warp] = part;
+    __syncthreads();
+    const int dst = s_part[0] + s_part[1] + s_part[2] + s_part[3] + j;
+    const uint4* src = reinterpret_cast<const uint4*>(p.H + ((size_t)b * (p.SL + 1) + j) * p.d);
+    uint4* out = reinterpret_cast<uint4*>(p.packed + (size_t)dst * p.d);
+    for (int c = threadIdx.x; c < p.d / 8; c += blockDim.x) out[c] = __ldg(src + c);
 }
 
 // probs[b, v] currently holds the raw logit; turn it into the soft-max probability.

@@ -68,6 +68,10 @@ struct UmmaParams {
     int32_t* bonus;
     int32_t* target_ids;
     VerifyPadded padded;   // sl != null: fixed-shape rows, per-sequence look-ahead read from the device
+    // Verification whose row count is device memory (rows packed by the kernel before this one): R, MT, CN, TPC, TR
+    // above are then upper bounds / unused, the kernel derives the tiling from *dev_R; TRN stays the box height of
+    // the LM-head tensor map (256) and the MMAs take the tile height rounded up to 16.
+    const int32_t* dev_R;
 };
 
 // ---------------------------------------------------------------------------------------------
@@ -217,9 +221,22 @@ umma_tail_kernel(const __grid_constant__ CUtensorMap tmap_W, const __grid_consta
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
-    const int m_tile = blockIdx.x % p.MT;
-    const int nslot = blockIdx.x / p.MT;
     const int KB = (p.d + kUmmaBK - 1) / kUmmaBK;
+    // tiling: from the host, or (row count in device memory) derived here by the same rule
+    int gR = p.R, gMT = p.MT, gCN = p.CN, gTPC = p.TPC, gTR = p.TR, gTRN = p.TRN;
+    bool idle = false;
+    if (!DRAFT && p.dev_R) {
+        asm volatile("griddepcontrol.wait;" ::: "memory");   // the count is the predecessor's output
+        gR = min(max(__ldcg(p.dev_R), 1), p.R);
+        gMT = (gR + 127) / 128;
+        gCN = (int)gridDim.x / gMT;
+        gTPC = max(1, (p.V + 256 * gCN - 1) / (256 * gCN));
+        gTR = (p.V + gCN * gTPC - 1) / (gCN * gTPC);
+        gTRN = max(16, (gTR + 15) / 16 * 16);
+        idle = (int)blockIdx.x >= gMT * gCN;
+    }
+    const int m_tile = blockIdx.x % gMT;
+    const int nslot = blockIdx.x / gMT;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < p.stages; ++s) {
@@ -245,7 +262,7 @@ umma_tail_kernel(const __grid_constant__ CUtensorMap tmap_W, const __grid_consta
 
     // A chained draft step in which no sequence drafts any more has nothing to do.  Every warp finds that out
     // by itself, after the dependency wait (the flags are the predecessor's output), and goes to the exit.
-    bool live = true;
+    bool live = !idle;   // (a CTA beyond the tiling derived from the device-side row count has nothing to do either)
     if (DRAFT && f.chain.alive != nullptr && f.chain.step > 1) {
         asm volatile("griddepcontrol.wait;" ::: "memory");
         live = chain_any_live(f.chain, f.B, lane);
@@ -255,12 +272,12 @@ umma_tail_kernel(const __grid_constant__ CUtensorMap tmap_W, const __grid_consta
         // ------------------------------ producer ------------------------------
         if (lane == 0 && live) {
             int stage = 0, phase = 0;
-            const uint32_t bytes = (uint32_t)(p.rep * p.a_rows + p.TRN) * 128u;
+            const uint32_t bytes = (uint32_t)(p.rep * p.a_rows + p.TRN) * 128u;   // the boxes of the two tensor maps
             // The LM head is never written by this library: its first tiles are requested before the
             // dependency wait, the hidden-state tiles of the same stages right after it.
             int pre = 0;
             {
-                const int v0 = nslot * p.TPC * p.TR;
+                const int v0 = nslot * gTPC * gTR;
                 if (v0 < p.V) {
                     pre = min(p.stages, KB);
                     for (int kb = 0; kb < pre; ++kb) {
@@ -271,8 +288,8 @@ umma_tail_kernel(const __grid_constant__ CUtensorMap tmap_W, const __grid_consta
             }
             asm volatile("griddepcontrol.wait;" ::: "memory");
             int n = 0;
-            for (int i = 0; i < p.TPC; ++i) {
-                const int v0 = (nslot * p.TPC + i) * p.TR;
+            for (int i = 0; i < gTPC; ++i) {
+                const int v0 = (nslot * gTPC + i) * gTR;
                 if (v0 >= p.V) break;
                 for (int kb = 0; kb < KB; ++kb, ++n) {
                     if (n >= pre) {
@@ -294,9 +311,9 @@ umma_tail_kernel(const __grid_constant__ CUtensorMap tmap_W, const __grid_consta
         // ------------------------------ MMA issuer ------------------------------
         if (lane == 0 && live) {
             int stage = 0, phase = 0, it = 0;
-            const uint32_t idesc = umma_idesc(p.TRN);
-            for (int i = 0; i < p.TPC; ++i) {
-                if ((nslot * p.TPC + i) * p.TR >= p.V) break;
+            const uint32_t idesc = umma_idesc(gTRN);
+            for (int i = 0; i < gTPC; ++i) {
+                if ((nslot * gTPC + i) * gTR >= p.V) break;
                 const int buf = it & 1;
                 mbar_wait(&tmem_empty[buf], ((it >> 1) & 1) ^ 1, p.status);
                 tc_fence_after();
@@ -330,8 +347,8 @@ umma_tail_kernel(const __grid_constant__ CUtensorMap tmap_W, const __grid_consta
         const int share = (ew >> 2) * p.rep + (quad * 32) / p.rows_pad;
         const int nshare = 2 * p.rep;
         const int row = m_tile * 128 + tile_row;
-        const bool warp_has_rows = (m_tile * 128 + (quad * 32) % p.rows_pad) < p.R;
-        const bool valid = row < p.R;
+        const bool warp_has_rows = (m_tile * 128 + (quad * 32) % p.rows_pad) < gR;
+        const bool valid = row < gR;
         // the optional probs output receives the raw logits of this row, unless the sequence is masked
         const bool keep_logits = DRAFT && p.probs && valid && (!f.active || f.active[row]);
         // stamp of this launch (the word is advanced by the last warp of the second phase)
@@ -356,13 +373,13 @@ umma_tail_kernel(const __grid_constant__ CUtensorMap tmap_W, const __grid_consta
         top.init();
 
         int it = 0;
-        for (int i = 0; i < p.TPC; ++i) {
-            const int v0 = (nslot * p.TPC + i) * p.TR;
+        for (int i = 0; i < gTPC; ++i) {
+            const int v0 = (nslot * gTPC + i) * gTR;
             if (v0 >= p.V) break;
             const int buf = it & 1;
             mbar_wait(&tmem_full[buf], (it >> 1) & 1, p.status);
             tc_fence_after();
-            const int ncols = min(p.TR, p.V - v0);  // further columns belong to the next tile or lie past V
+            const int ncols = min(gTR, p.V - v0);  // further columns belong to the next tile or lie past V
             if (warp_has_rows) {
                 const int nchunks = (ncols + 31) >> 5;
                 const int c_lo = (nchunks * share + nshare - 1) / nshare;
@@ -507,12 +524,12 @@ umma_tail_kernel(const __grid_constant__ CUtensorMap tmap_W, const __grid_consta
                 __shared__ int s_last;
                 __threadfence();
                 named_barrier_sync(2, kUmmaEpiWarps * 32);
-                if (ew == 0 && lane == 0) s_last = atomicAdd(p.ticket, 1u) == gridDim.x - 1;
+                if (ew == 0 && lane == 0) s_last = atomicAdd(p.ticket, 1u) == (unsigned)(gMT * gCN) - 1u;   // idle CTAs take none
                 named_barrier_sync(2, kUmmaEpiWarps * 32);
                 if (s_last) {
                     __threadfence();
                     for (int b = ew; b < p.B; b += kUmmaEpiWarps)
-                        verify_one_sequence(p.keys, p.draft_ids, p.row_off, p.B, p.SL, p.R, b, p.n_accept, p.bonus,
+                        verify_one_sequence(p.keys, p.draft_ids, p.row_off, p.B, p.SL, gR, b, p.n_accept, p.bonus,
                                             p.target_ids, p.status, lane, p.padded);
                     if (ew == 0) warp_write_row_offsets(p.padded, p.B, p.SL, lane);
                     named_barrier_sync(2, kUmmaEpiWarps * 32);
@@ -548,14 +565,16 @@ struct VerifyFinalParams {
     int* status;
     unsigned int* ticket;
     VerifyPadded padded;
+    const int32_t* dev_R;   // non-null: the row count is device memory (R is then the upper bound)
 };
 
 __global__ void __launch_bounds__(128) verify_finalize_kernel(const VerifyFinalParams p) {
     __shared__ int s_last;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int b = blockIdx.x * (blockDim.x >> 5) + warp;
+    const int R = p.dev_R ? min(max(__ldcg(p.dev_R), 1), p.R) : p.R;
     if (b < p.B)
-        verify_one_sequence(p.keys, p.draft_ids, p.row_off, p.B, p.SL, p.R, b, p.n_accept, p.bonus, p.target_ids,
+        verify_one_sequence(p.keys, p.draft_ids, p.row_off, p.B, p.SL, R, b, p.n_accept, p.bonus, p.target_ids,
                             p.status, lane, p.padded);
     if (blockIdx.x == gridDim.x - 1 && warp == (blockDim.x >> 5) - 1) warp_write_row_offsets(p.padded, p.B, p.SL, lane);
     __syncthreads();

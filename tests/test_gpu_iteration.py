@@ -160,7 +160,7 @@ def check_iteration(oracle, got, ref, W_T, H_T, tau, S, draft_ids=None):
 
 @pytest.mark.parametrize("split,graph", [(False, False), (True, False), (False, True)])
 @pytest.mark.parametrize("V,dD,dT,B,S", [(50, 16, 24, 1, 4), (1000, 72, 136, 3, 6), (4099, 264, 72, 7, 5),
-                                         (3000, 128, 64, 20, 9)])
+                                         (3000, 128, 64, 20, 9), (2000, 64, 72, 12, 11), (1500, 64, 136, 40, 16)])
 def test_iteration_small_shapes(oracle, V, dD, dT, B, S, split, graph):
     W_D, W_T, h_D, H_T = make_inputs(V, dD, dT, B, S, seed=V + B)
     pos0 = (np.arange(B, dtype=np.int32) * 3) % 11
