@@ -49,7 +49,13 @@ def measured_peaks():
 # profiles/.  Valid only for the kernel sources they were taken on: reported as null once csrc/ changes.
 NCU_TRAFFIC = {
     "sources": "",
-    "bytes_per_launch": {},
+    "bytes_per_launch": {
+        # verification: the LM head once (327.87 MB read) + write-backs of lines other kernels left dirty
+        "vicuna_b1/verification tail": 327.87e6 + 4.6e6,
+        # persistent draft-phase kernel: the LM head once per step, plus per launch the stages requested ahead for
+        # the step that does not take place (58 % of a slab, thrown away) and a few MB of foreign write-backs
+        "vicuna_b1/draft-step tail": {"per_step": 49.2e6, "per_launch": 33.0e6 + 4.0e6},
+    },
 }
 
 
@@ -63,10 +69,14 @@ def kernel_sources_hash() -> str:
     return h.hexdigest()[:16]
 
 
-def ncu_traffic(workload: str, kernel: str):
+def ncu_traffic(workload: str, kernel: str, steps_per_launch: float = 1.0):
+    """DRAM bytes per launch of that kernel as ncu counted them, or None if the kernels have changed since."""
     if kernel_sources_hash() != NCU_TRAFFIC["sources"]:
         return None
-    return NCU_TRAFFIC["bytes_per_launch"].get(f"{workload}/{kernel}")
+    t = NCU_TRAFFIC["bytes_per_launch"].get(f"{workload}/{kernel}")
+    if isinstance(t, dict):
+        return t["per_launch"] + t["per_step"] * steps_per_launch
+    return t
 
 
 # ------------------------------------------------------------------------------------------ ranks
@@ -398,7 +408,8 @@ def rooflines(wl, K: int, res: dict, hbm_peak: float, tensor_peak: float, peak_k
                            "one launch per draft step of the cap; launches that find no sequence drafting return at once") +
                           "; achieved = algorithmic bytes of the steps that had work over the time of all draft launches"}
     for r in (roof_verify, roof_draft):
-        r["traffic"] = ncu_traffic(wl.name, r["kernel"])
+        per_launch = n_live / max(draft_launches, 1) if r is roof_draft and draft_launches == K else 1.0
+        r["traffic"] = ncu_traffic(wl.name, r["kernel"], per_launch)
         r["frac"] = r["achieved"] / r["peak"]
         r["frac_of_nominal_8TBs"] = r["achieved"] / 8000.0
     if rows / K > tensor_peak * 1e12 / (hbm_peak * 1e9):   # rows per call beyond the machine balance

@@ -110,11 +110,13 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, int* s
     if (mbar_try_wait(bar, parity)) return true;
     const long long t0 = clock64();
     for (;;) {
-        // once any wait in the grid has run out, all others give up at once
-        if (status && *reinterpret_cast<volatile int*>(status) == DISCO_ERR_TIMEOUT) return false;
 #pragma unroll 1
         for (int i = 0; i < 64; ++i)
             if (mbar_try_wait(bar, parity)) return true;
+        // Once any wait in the grid has run out, all others give up at once.  (The status word is global
+        // memory, a round trip of about a thousand cycles: it is looked at between batches of polls, never
+        // ahead of a poll that may succeed.)
+        if (status && *reinterpret_cast<volatile int*>(status) == DISCO_ERR_TIMEOUT) return false;
         if (clock64() - t0 > kWaitBudgetClocks) {
             record_status(status, DISCO_ERR_TIMEOUT);
             return false;

@@ -24,6 +24,7 @@
 
 #include "common.cuh"
 #include "stream_tail.cuh"  // verify_one_sequence, warp_halt_classifier
+#include "group_merge.cuh"
 
 namespace disco {
 
@@ -483,38 +484,77 @@ umma_tail_kernel(const __grid_constant__ CUtensorMap tmap_W, const __grid_consta
                 store_stamped_record(p.part_rec + ((size_t)row * p.CN + nslot) * kStampedPieces, st.m, st.Z, st.S, top.t,
                                      key, stamp);
             }
-            // Second phase inside the same (cooperative) launch: the sequences are shared out, one warp
-            // each, over the CTAs; a warp reads the records of its sequence as the other CTAs publish
-            // them (stamped records, bounded waits).
+            // Second phase inside the same (cooperative) launch: a CTA reads the records of its sequences
+            // as the other CTAs publish them (stamped records, bounded waits).  Up to two sequences per CTA
+            // are finished by groups of warps (all eight for one sequence, four each for two); beyond that,
+            // and for statistics-only rows, the sequences are shared out one warp each.
             named_barrier_sync(2, kUmmaEpiWarps * 32);  // the exchange area is free from here on
-            const int first = ew * (int)gridDim.x + (int)blockIdx.x;
-            if (first < f.B) {
-                int b = first;
-                const bool chain = f.chain.alive != nullptr;
-                bool act = chain_seq_live(f.chain, f.active, b);
-                float fpos = chain ? static_cast<float>(f.chain.pos0[b] + f.chain.step)
-                                   : (f.pos ? static_cast<float>(f.pos[b]) : 0.f);
-                int nd = chain ? f.chain.step : (f.n_drafted ? f.n_drafted[b] : 0);
-                float* feat16 = reinterpret_cast<float*>(xch) + ew * kWarpScratchWords;  // the exchange area is free again
-                for (;;) {
-                    // a masked sequence still waits for its records: the stamp may only advance once
-                    // every CTA has taken part in this launch
-                    umma_finish_sequence(f, p.part_rec, p.CN, b, act, fpos, nd, feat16, clf_s, stamp + f.test_stamp_skew,
-                                         p.status, lane);
-                    b += kUmmaEpiWarps * (int)gridDim.x;
-                    if (b >= f.B) break;
-                    act = chain_seq_live(f.chain, f.active, b);
-                    fpos = chain ? static_cast<float>(f.chain.pos0[b] + f.chain.step)
-                                 : (f.pos ? static_cast<float>(f.pos[b]) : 0.f);
-                    nd = chain ? f.chain.step : (f.n_drafted ? f.n_drafted[b] : 0);
+            const int grid = (int)gridDim.x;
+            if (!STATS && f.B <= 2 * grid) {
+                const bool two = f.B > grid;
+                const int g = two ? ew >> 2 : 0;
+                const int gt = two ? (ew & 3) * 32 + lane : ew * 32 + lane;
+                const int b = (int)blockIdx.x + g * grid;
+                if (b < f.B) {
+                    float* group_s = reinterpret_cast<float*>(xch) + g * kGroupScratchWords;
+                    const float4* recs = p.part_rec + (size_t)b * p.CN * kStampedPieces;
+                    const uint32_t want = stamp + f.test_stamp_skew;
+                    // a masked sequence still waits for its records: the stamp may only advance once every
+                    // CTA has taken part in this launch
+                    const MergedPartials mp = two ? group_merge_partials<4>(recs, p.CN, want, p.status, group_s, 3 + g, gt)
+                                                  : group_merge_partials<8>(recs, p.CN, want, p.status, group_s, 3, gt);
+                    if (gt < 32) {
+                        const bool chain = f.chain.alive != nullptr;
+                        if (chain_seq_live(f.chain, f.active, b)) {
+                            const float fpos = chain ? static_cast<float>(f.chain.pos0[b] + f.chain.step)
+                                                     : (f.pos ? static_cast<float>(f.pos[b]) : 0.f);
+                            const int nd = chain ? f.chain.step : (f.n_drafted ? f.n_drafted[b] : 0);
+                            const int Hc = f.clf_H;
+                            const DraftOutputs o{f.token, f.conf, f.halt, f.feats, f.final_stats, f.nll_sum,
+                                                 f.stats_only, f.chain};
+                            warp_draft_epilogue(mp.st, mp.key, mp.sel, fpos, nd, f.tau, f.sl_max, group_s, clf_s,
+                                                clf_s + Hc * kNFeat, clf_s + Hc * (kNFeat + 1), clf_s + Hc * (kNFeat + 2),
+                                                Hc, b, o, lane);
+                        }
+                        // the last finished sequence of the grid advances the stamp for the next launch: by
+                        // then every record of this launch has been read
+                        __syncwarp();
+                        if (lane == 0 && atomicAdd(f.epoch + 1, 1u) == (unsigned int)f.B - 1u) {
+                            f.epoch[1] = 0u;
+                            f.epoch[0] = stamp == 0xffffffffu ? 0u : stamp;   // the stamp is never zero
+                        }
+                    }
                 }
-                // the last finishing warp of the grid advances the stamp for the next launch: by then every
-                // record of this launch has been read
-                const unsigned int nwarps = (unsigned int)min(f.B, kUmmaEpiWarps * (int)gridDim.x);
-                __syncwarp();
-                if (lane == 0 && atomicAdd(f.epoch + 1, 1u) == nwarps - 1) {
-                    f.epoch[1] = 0u;
-                    f.epoch[0] = stamp == 0xffffffffu ? 0u : stamp;   // the stamp is never zero
+            } else {
+                const int first = ew * (int)gridDim.x + (int)blockIdx.x;
+                if (first < f.B) {
+                    int b = first;
+                    const bool chain = f.chain.alive != nullptr;
+                    bool act = chain_seq_live(f.chain, f.active, b);
+                    float fpos = chain ? static_cast<float>(f.chain.pos0[b] + f.chain.step)
+                                       : (f.pos ? static_cast<float>(f.pos[b]) : 0.f);
+                    int nd = chain ? f.chain.step : (f.n_drafted ? f.n_drafted[b] : 0);
+                    float* feat16 = reinterpret_cast<float*>(xch) + ew * kWarpScratchWords;  // the exchange area is free again
+                    for (;;) {
+                        // a masked sequence still waits for its records: the stamp may only advance once
+                        // every CTA has taken part in this launch
+                        umma_finish_sequence(f, p.part_rec, p.CN, b, act, fpos, nd, feat16, clf_s, stamp + f.test_stamp_skew,
+                                             p.status, lane);
+                        b += kUmmaEpiWarps * (int)gridDim.x;
+                        if (b >= f.B) break;
+                        act = chain_seq_live(f.chain, f.active, b);
+                        fpos = chain ? static_cast<float>(f.chain.pos0[b] + f.chain.step)
+                                     : (f.pos ? static_cast<float>(f.pos[b]) : 0.f);
+                        nd = chain ? f.chain.step : (f.n_drafted ? f.n_drafted[b] : 0);
+                    }
+                    // the last finishing warp of the grid advances the stamp for the next launch: by then every
+                    // record of this launch has been read
+                    const unsigned int nwarps = (unsigned int)min(f.B, kUmmaEpiWarps * (int)gridDim.x);
+                    __syncwarp();
+                    if (lane == 0 && atomicAdd(f.epoch + 1, 1u) == nwarps - 1) {
+                        f.epoch[1] = 0u;
+                        f.epoch[0] = stamp == 0xffffffffu ? 0u : stamp;   // the stamp is never zero
+                    }
                 }
             }
         } else {
