@@ -244,7 +244,9 @@ int launch_umma(disco_ctx* c, const void* W, const void* H, int d, int R, float*
     // copies only feeds accumulator lanes nobody reads.
     p.a_bytes = p.rep > 1 ? 128 * 128 : (p.a_rows * 128 + 1023) / 1024 * 1024;
     p.b_bytes = (p.TRN * 128 + 1023) / 1024 * 1024;
-    p.stages = std::max(2, std::min(kUmmaMaxStages, kUmmaRingBytes / (p.a_bytes + p.b_bytes)));
+    // (the draft step's epilogue keeps its candidate queues in the last bytes of the ring)
+    const int ring_bytes = kUmmaRingBytes - ((DRAFT && !STATS) ? kUmmaQueueBytes : 0);
+    p.stages = std::max(2, std::min(kUmmaMaxStages, ring_bytes / (p.a_bytes + p.b_bytes)));
     p.status = c->status;
     p.keys = c->keys;
     p.part_rec = reinterpret_cast<float4*>(c->stamped_rec);

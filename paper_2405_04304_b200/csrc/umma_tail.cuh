@@ -34,6 +34,9 @@ constexpr int kUmmaRingBytes = 192 * 1024;  // shared memory for the operand sta
 constexpr int kUmmaEpiWarps = 8;
 constexpr int kUmmaThreads = (2 + kUmmaEpiWarps) * 32;
 constexpr int kUmmaXchBytes = 14 * 1024;  // 64-byte records handed between the warps that share a hidden row
+// Draft step: the last bytes of the ring are left to the epilogue warps' candidate queues (16 entries per lane)
+constexpr int kUmmaQueueEntries = 16;
+constexpr int kUmmaQueueBytes = kUmmaEpiWarps * kUmmaQueueEntries * 32 * 4;
 constexpr int kUmmaSmemBytes =
     kUmmaRingBytes + 1024 /*align*/ + 512 /*barriers*/ + kUmmaXchBytes;
 // the draft step adds the classifier parameters behind the exchange area
@@ -372,6 +375,8 @@ umma_tail_kernel(const __grid_constant__ CUtensorMap tmap_W, const __grid_consta
         st.init();
         RegTop10 top;
         top.init();
+        // this lane's candidate queue (draft step): entry i at queue[32 i]
+        float* queue = reinterpret_cast<float*>(smem + kUmmaRingBytes - kUmmaQueueBytes) + ew * (kUmmaQueueEntries * 32) + lane;
 
         int it = 0;
         for (int i = 0; i < gTPC; ++i) {
@@ -390,11 +395,20 @@ umma_tail_kernel(const __grid_constant__ CUtensorMap tmap_W, const __grid_consta
                     tmem_ld32(tmem_base + buf * 256 + c * 32 + (static_cast<uint32_t>(quad * 32) << 16), z);
                     const int cbase = c * 32;
                     if (DRAFT) {
+                        const bool whole = cbase + 32 <= ncols;   // (warp-uniform) no column of the chunk is masked
                         float cmax = DISCO_NEG_INF;
+                        if (whole) {
 #pragma unroll
-                        for (int j = 0; j < 32; ++j) {
-                            z[j] = (cbase + j < ncols) ? __fadd_rn(z[j], 0.f) : DISCO_NEG_INF;
-                            cmax = fmaxf(cmax, z[j]);
+                            for (int j = 0; j < 32; ++j) {
+                                z[j] = __fadd_rn(z[j], 0.f);
+                                cmax = fmaxf(cmax, z[j]);
+                            }
+                        } else {
+#pragma unroll
+                            for (int j = 0; j < 32; ++j) {
+                                z[j] = (cbase + j < ncols) ? __fadd_rn(z[j], 0.f) : DISCO_NEG_INF;
+                                cmax = fmaxf(cmax, z[j]);
+                            }
                         }
                         if (cmax > st.m) {  // move the reference maximum first, then add the chunk
                             if (st.Z > 0.f) {
@@ -405,24 +419,56 @@ umma_tail_kernel(const __grid_constant__ CUtensorMap tmap_W, const __grid_consta
                             }
                             st.m = cmax;
                         }
+                        if (whole) {
 #pragma unroll
-                        for (int j = 0; j < 32; ++j) {
-                            const float t = z[j] - st.m;       // -inf for masked columns: e = 0
-                            const float e = __expf(t);
-                            st.Z += e;
-                            st.S = (cbase + j < ncols) ? fmaf(e, t, st.S) : st.S;
-                            if (z[j] > best_v) {
-                                best_v = z[j];
-                                best_i = v0 + cbase + j;
+                            for (int j = 0; j < 32; ++j) {
+                                const float t = z[j] - st.m;
+                                const float e = __expf(t);
+                                st.Z += e;
+                                st.S = fmaf(e, t, st.S);
+                                if (z[j] > best_v) {
+                                    best_v = z[j];
+                                    best_i = v0 + cbase + j;
+                                }
+                            }
+                        } else {
+#pragma unroll
+                            for (int j = 0; j < 32; ++j) {
+                                const float t = z[j] - st.m;       // -inf for masked columns: e = 0
+                                const float e = __expf(t);
+                                st.Z += e;
+                                st.S = (cbase + j < ncols) ? fmaf(e, t, st.S) : st.S;
+                                if (z[j] > best_v) {
+                                    best_v = z[j];
+                                    best_i = v0 + cbase + j;
+                                }
                             }
                         }
                         if (!STATS) {
-                            // A logit enters a row's ten largest with probability about 10 / (columns seen so far): the
-                            // insertion network runs only for the pairs that some lane's row needs (a warp-wide vote,
-                            // so the branch does not diverge).
+                            // The ten largest per row.  A logit enters a row's list with probability about
+                            // 10 / (columns seen so far), but in a warp of 32 rows some lane nearly always needs the
+                            // insertion network, so running it per logit costs 32 rows' worth for one row's need.
+                            // Instead each lane queues the logits above its row's 10th largest (its own slots of
+                            // shared memory, 16 logits at a time), and the network then runs as often as the
+                            // longest queue of the warp is deep: two or three times per 16 logits, not eight.
 #pragma unroll
-                            for (int j = 0; j < 32; j += 2) {
-                                if (__any_sync(kFullMask, fmaxf(z[j], z[j + 1]) > top.t[kTopK - 1])) top.push2(z[j], z[j + 1]);
+                            for (int h = 0; h < 32; h += kUmmaQueueEntries) {
+                                const float thr = top.t[kTopK - 1];
+                                float* qp = queue;
+#pragma unroll
+                                for (int j = 0; j < kUmmaQueueEntries; ++j) {
+                                    if (z[h + j] > thr) {
+                                        *qp = z[h + j];
+                                        qp += 32;
+                                    }
+                                }
+                                const int cnt = static_cast<int>(qp - queue) >> 5;
+                                const int deepest = __reduce_max_sync(kFullMask, cnt);
+                                for (int i = 0; i < deepest; i += 2) {
+                                    const float a = i < cnt ? queue[i * 32] : DISCO_NEG_INF;
+                                    const float b = i + 1 < cnt ? queue[(i + 1) * 32] : DISCO_NEG_INF;
+                                    top.push2(a, b);
+                                }
                             }
                         }
                         if (keep_logits) {
