@@ -642,16 +642,21 @@ def run_e2e(ctx, data: Data, clf, wl, forced, Wm: int, K: int, stream, world: in
     per_call_d2h = S * B * 9 + 4 * B * 4
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     ring = data.W_D_ring
+    # the buffers of each iteration, as the caller of the library would hold them (views, made once)
+    args = []
+    for it in range(T):
+        d = it % data.n_distinct
+        args.append((ring[(it * S) % data.n_rot], h_D_host[d], H_T_host[d], None if forced_host is None else forced_host[d],
+                     ids_host[d]))
     for it in range(T):
         if it == Wm:
             torch.cuda.synchronize()
             if world > 1:
                 torch.distributed.barrier()
             e0.record(stream)
-        d = it % data.n_distinct
-        ctx.iteration_host(ring[(it * S) % data.n_rot], h_D_host[d], data.W_T, H_T_host[d], pos, clf, wl.tau, S, token, conf,
-                           halt, sl, n_acc, bonus, sl_forced=None if forced_host is None else forced_host[d],
-                           draft_ids=ids_host[d], pos_next=pos, w_step_stride=data.w_stride, stream=stream)
+        W_D_it, h_D_it, H_T_it, forced_it, ids_it = args[it]
+        ctx.iteration_host(W_D_it, h_D_it, data.W_T, H_T_it, pos, clf, wl.tau, S, token, conf, halt, sl, n_acc, bonus,
+                           sl_forced=forced_it, draft_ids=ids_it, pos_next=pos, w_step_stride=data.w_stride, stream=stream)
         sl_hist[it] = sl_np
         nacc_hist[it] = nacc_np
     e1.record(stream)

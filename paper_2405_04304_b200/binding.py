@@ -97,20 +97,21 @@ def strerror(code: int) -> str:
 
 
 def _ptr(t, dtype=None, cuda=True):
+    """Address of a contiguous tensor of the expected dtype and device kind (None -> NULL), as an integer."""
     if t is None:
         return None
-    if dtype is not None and t.dtype != dtype:
-        raise TypeError(f"expected {dtype}, got {t.dtype}")
-    if t.is_cuda != cuda:
-        raise ValueError("tensor is on the wrong device kind for this call")
-    if not t.is_contiguous():
+    if (dtype is not None and t.dtype is not dtype) or t.is_cuda is not cuda or not t.is_contiguous():
+        if dtype is not None and t.dtype != dtype:
+            raise TypeError(f"expected {dtype}, got {t.dtype}")
+        if t.is_cuda != cuda:
+            raise ValueError("tensor is on the wrong device kind for this call")
         raise ValueError("tensor must be contiguous")
-    return ctypes.c_void_p(t.data_ptr())
+    return t.data_ptr()
 
 
-def _stream(stream) -> ctypes.c_void_p:
+def _stream(stream) -> int:
     s = stream if stream is not None else torch.cuda.current_stream()
-    return ctypes.c_void_p(s.cuda_stream)
+    return s.cuda_stream
 
 
 class Classifier:

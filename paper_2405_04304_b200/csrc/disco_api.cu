@@ -62,6 +62,9 @@ struct disco_ctx {
     int* status;
     float* final_stats;
     uint8_t* chain_alive;          // [max_batch] draft phase on the device: which sequences still draft
+    double* sample_seg_tot;        // verification with sampling: [max_batch][kSampleMaxSegments][2] sums of weights
+    int32_t* sample_seg_last;      //   the same shape: last index with positive weight
+    unsigned int* sample_tickets;  //   [max_batch]
     void* pack_rows;               // fixed-shape verification with many rows: the rows that count, packed
     int32_t* pack_off;             // [max_batch + 1] their offsets; the last entry is the row count
     void* loop_rec;                // persistent draft-phase kernel: stamped 80-byte records, [4][CTA]; written by nothing else
@@ -237,7 +240,7 @@ int launch_umma(disco_ctx* c, const void* W, const void* H, int d, int R, float*
     // Draft step with few rows: copies of the rows fill the other TMEM lane quadrants, so that the
     // epilogue (heavy there) runs on every warp scheduler.  Verification's epilogue is a compare per
     // logit and keeps the smaller stage instead.
-    p.rep = (DRAFT && !STATS && R <= 64) ? (R <= 32 ? 4 : 2) : 1;   // the statistics-only epilogue is light too
+    p.rep = (DRAFT && !STATS && R <= 64) ? (R <= 32 ? 4 : 2) : 1;   // (measured: no gain for the statistics-only epilogue)
     p.rows_pad = 128 / p.rep;
     // The A stage holds a_rows rows (rep copies, rows_pad rows apart).  The MMA still reads 128 rows from
     // its start: what lies behind the tile (other stages of the ring, always inside it) or between the
@@ -485,6 +488,9 @@ int disco_create(disco_ctx** out, int V, int d_draft, int d_target, int max_batc
     ok = ok && cudaMalloc(&c->status, 256) == cudaSuccess;
     ok = ok && cudaMalloc(&c->final_stats, (size_t)c->part_rows * 2 * sizeof(float)) == cudaSuccess;
     ok = ok && cudaMalloc(&c->chain_alive, (size_t)max_batch + 64) == cudaSuccess;
+    ok = ok && cudaMalloc(&c->sample_seg_tot, (size_t)max_batch * kSampleMaxSegments * 2 * sizeof(double)) == cudaSuccess;
+    ok = ok && cudaMalloc(&c->sample_seg_last, (size_t)max_batch * kSampleMaxSegments * 2 * sizeof(int32_t)) == cudaSuccess;
+    ok = ok && cudaMalloc(&c->sample_tickets, (size_t)max_batch * sizeof(unsigned int)) == cudaSuccess;
     ok = ok && cudaMalloc(&c->pack_rows, (size_t)max_rows * d_target * 2) == cudaSuccess;
     ok = ok && cudaMalloc(&c->pack_off, ((size_t)max_batch + 2) * sizeof(int32_t)) == cudaSuccess;
     ok = ok && cudaMalloc(&c->loop_rec, (size_t)4 * c->sm_count * 80) == cudaSuccess;
@@ -521,6 +527,9 @@ int disco_destroy(disco_ctx* c) {
     cudaFree(c->status);
     cudaFree(c->final_stats);
     cudaFree(c->chain_alive);
+    cudaFree(c->sample_seg_tot);
+    cudaFree(c->sample_seg_last);
+    cudaFree(c->sample_tickets);
     cudaFree(c->loop_rec);
     cudaFree(c->pack_rows);
     cudaFree(c->pack_off);
@@ -588,10 +597,9 @@ cudaError_t launch_after(const disco_ctx* c, void (*kern)(KArgs...), dim3 grid, 
 
 // The sampling kernels stage one row of V floats in dynamic shared memory: raise their limit once per device.
 bool configure_sampling(disco_ctx* c) {
-    static KernelSetup rows_setup, spec_setup;
+    static KernelSetup rows_setup;
     const size_t bytes = (size_t)kSampleSmemFloats * sizeof(float);
-    return raise_smem_limit(c, rows_setup, sample_rows_kernel, bytes, nullptr) &&
-           raise_smem_limit(c, spec_setup, speculative_sample_kernel, bytes, nullptr);
+    return raise_smem_limit(c, rows_setup, sample_rows_kernel, bytes, nullptr);
 }
 
 // Shared body of the LM-head + soft-max passes: B rows of hidden size d against the head W.
@@ -604,7 +612,7 @@ int draft_step_common(disco_ctx* c, const void* W_D, const void* h_D, int d, int
                       int sl_max, int32_t* token, float* conf, uint8_t* halt, float* feats, float* probs,
                       float* nll_sum, int stats_only, void* stream, bool normalize = true,
                       const float* u_draw = nullptr, float* p_token = nullptr, bool* drew = nullptr,
-                      const ChainLink* chain = nullptr) {
+                      const ChainLink* chain = nullptr, unsigned int* clear_words = nullptr, int clear_n = 0) {
     if (!c || !W_D || !h_D) return DISCO_ERR_INVALID_ARG;
     if (!stats_only && !chain && (!pos || !n_drafted)) return DISCO_ERR_INVALID_ARG;
     if (!stats_only && (!token || !conf || !halt)) return DISCO_ERR_INVALID_ARG;
@@ -636,6 +644,8 @@ int draft_step_common(disco_ctx* c, const void* W_D, const void* h_D, int d, int
     p.n_drafted = n_drafted;
     p.active = active;
     if (chain) p.chain = *chain;
+    p.clear_words = clear_words;
+    p.clear_n = clear_n;
     p.clf_W1 = clf->W1;
     p.clf_b1 = clf->b1;
     p.clf_w2 = clf->w2;
@@ -692,6 +702,8 @@ int draft_step_common(disco_ctx* c, const void* W_D, const void* h_D, int d, int
         f.stats_only = stats_only;
         f.epoch = c->ticket + 48;
         f.test_stamp_skew = c->test_stamp_skew;
+        f.clear_words = clear_words;
+        f.clear_n = clear_n;
         if (chain) f.chain = *chain;
         rc = stats_only == 1 ? launch_umma<true, true>(c, W_D, h_D, d, B, probs, &f, nullptr, st)
                         : launch_umma<true>(c, W_D, h_D, d, B, probs, &f, nullptr, st);
@@ -846,12 +858,16 @@ int disco_verify_sample_ragged(disco_ctx* c, const void* W_T, const void* H_T, c
     if (B > c->max_batch || R > c->max_rows) return DISCO_ERR_WORKSPACE;
     if (!row_off && R % B != 0) return DISCO_ERR_INVALID_ARG;
     if (!aligned16(W_T) || !aligned16(H_T)) return DISCO_ERR_INVALID_ARG;
-    // target distributions of all rows: LM head, soft-max statistics, normalised rows in y_T
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    // logits and soft-max statistics of all rows by the LM-head pass (which also clears the tickets); one more
+    // launch normalises the rows, counts the accepted tokens and draws the next one
     int rc = draft_step_common(c, W_T, H_T, c->d_target, R, c->max_rows, nullptr, nullptr, nullptr, nullptr, 0.f, 1,
-                               target_ids, nullptr, nullptr, nullptr, y_T, nullptr, 1, stream);
+                               target_ids, nullptr, nullptr, nullptr, y_T, nullptr, 1, stream, false, nullptr, nullptr,
+                               nullptr, nullptr, c->sample_tickets, B);
     if (rc) return rc;
-    SpecSampleParams sp{};
+    SampleRowsParams sp{};
     sp.y_T = y_T;
+    sp.stats = c->final_stats;
     sp.draft_probs = draft_probs;
     sp.draft_ids = draft_ids;
     sp.row_off = row_off;
@@ -861,16 +877,18 @@ int disco_verify_sample_ragged(disco_ctx* c, const void* W_T, const void* H_T, c
     sp.SL = row_off ? 0 : (R / B - 1);
     sp.R = R;
     sp.V = c->V;
+    // about two CTAs per SM; a row is cut into at most kSampleMaxSegments segments
+    sp.SEG = std::max(1, std::min(kSampleMaxSegments, (2 * c->sm_count + R - 1) / R));
+    sp.seg_len = ((c->V + sp.SEG - 1) / sp.SEG + 3) & ~3;
     sp.n_accept = n_accept;
     sp.next_token = next_token;
+    sp.seg_tot = c->sample_seg_tot;
+    sp.seg_last = c->sample_seg_last;
+    sp.tickets = c->sample_tickets;
     sp.status = c->status;
-    const size_t smem = sample_smem_bytes(c->V);
-    sp.use_smem = smem ? 1 : 0;
-    if (!configure_sampling(c)) return DISCO_ERR_CUDA;
-    const cudaError_t e = launch_after(c, speculative_sample_kernel, dim3(B), dim3(kSampleThreads), smem,
-                                       static_cast<cudaStream_t>(stream), sp);
+    const cudaError_t e = launch_after(c, sample_rows_fused_kernel, dim3((unsigned)R * sp.SEG), dim3(kSampleThreads), 0, st, sp);
     c->launches += 1;
-    return cuda_ok(e, "speculative_sample_kernel launch") ? DISCO_OK : DISCO_ERR_CUDA;
+    return cuda_ok(e, "sample_rows_fused_kernel launch") ? DISCO_OK : DISCO_ERR_CUDA;
 }
 
 int disco_extract_features(disco_ctx* c, const void* W_D, const void* H_D, const void* W_T, const void* H_T,

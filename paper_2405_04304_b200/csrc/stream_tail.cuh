@@ -77,6 +77,9 @@ struct TailParams {
     // per-CTA sums and the one slab of logits (in probs) that holds u * total; at most 160 CTAs
     const float* u_draw;  // [B] uniforms in [0, 1)
     float* p_token;       // [B] or null: probability of the drawn token
+    // words that the kernel after this one counts in (the tickets of a verification with sampling): cleared here
+    unsigned int* clear_words;
+    int clear_n;
     int slab_rows;        // vocabulary rows per CTA (the slab of record c starts at c * slab_rows)
     // verification
     const int32_t* draft_ids;
@@ -887,6 +890,8 @@ __global__ void __launch_bounds__((NW + 1) * 32, 1) stream_tail_kernel(const __g
     // from here on the kernel reads the hidden states and writes scratch and outputs: the preceding
     // kernel of the stream must have finished
     asm volatile("griddepcontrol.wait;" ::: "memory");
+    if (blockIdx.x == 0)
+        for (int i = tid; i < p.clear_n; i += BAR_THREADS) p.clear_words[i] = 0u;
 
     const int n16 = (int)(row_bytes >> 4);  // 16-byte pieces per row
     for (int chunk = 0; chunk < nchunks; ++chunk) {

@@ -178,6 +178,9 @@ struct DraftFinalParams {
     unsigned int* epoch;  // [0] launches completed so far (stamp of this launch = that + 1), [1] finishing warps done
     ChainLink chain;      // alive != null: this launch is one step of a draft phase chained on the device
     unsigned int test_stamp_skew;   // 0.  Tests: the finishing warps expect a stamp that no CTA writes, so their wait runs out
+    // words that the kernel after this one counts in (the tickets of a verification with sampling): cleared here
+    unsigned int* clear_words;
+    int clear_n;
 };
 
 // One warp finishes sequence b from its NP partial records.  clf_s: classifier parameters in shared
@@ -344,6 +347,8 @@ umma_tail_kernel(const __grid_constant__ CUtensorMap tmap_W, const __grid_consta
         // ------------------------------ epilogue ------------------------------
         asm volatile("griddepcontrol.wait;" ::: "memory");  // scratch and outputs belong to the predecessor until now
         const int ew = warp - 2;            // 0 .. kUmmaEpiWarps-1
+        if (DRAFT && blockIdx.x == 0)
+            for (int i = ew * 32 + lane; i < f.clear_n; i += kUmmaEpiWarps * 32) f.clear_words[i] = 0u;
         const int quad = warp & 3;          // TMEM lane quadrant this warp may read
         // The warps that hold the same hidden rows (two per quadrant, times the copies of the rows in
         // other quadrants) split the columns of a tile into `nshare` shares.
