@@ -504,7 +504,13 @@ def run_ours(args, rank: int, world: int):
                 "d2h_bytes_per_step": e2e["d2h"] / K, "matches_device_run": e2e["matches"],
                 "call": "disco_iteration_host, one call per iteration, pinned host buffers",
                 "us_per_call": e2e["seconds"] / K * 1e6, "us_on_the_device_per_call": t_med / K * 1e6,
-                "us_of_copies_at_25GBs_per_call": (e2e["h2d"] + e2e["d2h"]) / K / 25e3},
+                "us_of_copies_at_25GBs_per_call": (e2e["h2d"] + e2e["d2h"]) / K / 25e3,
+                "breakdown_us_per_call": {
+                    "kernels (the graph replay)": t_med / K * 1e6,
+                    "one call and one synchronisation per iteration, buffers on the device":
+                        e2e["resident_seconds"] / K * 1e6 - t_med / K * 1e6,
+                    "host buffers (staging, two host-to-device copies ahead of the kernels)":
+                        e2e["seconds"] / K * 1e6 - e2e["resident_seconds"] / K * 1e6}},
         "gpu_launches": res["launches"]["all"], "clocks": sampler.summary(),
     }
     out.update(extra)
@@ -664,7 +670,30 @@ def run_e2e(ctx, data: Data, clf, wl, forced, Wm: int, K: int, stream, world: in
     if world > 1:
         torch.distributed.barrier()
     seconds = e0.elapsed_time(e1) * 1e-3
-    return {"seconds": seconds, "h2d": per_call_h2d * K, "d2h": per_call_d2h * K, "sl": sl_hist[Wm:], "n_acc": nacc_hist[Wm:]}
+    # For the breakdown: the same iterations with every buffer already on the device, still one call and one
+    # synchronisation per iteration (what is left of the host's share once the copies are gone).
+    dev = data.W_T.device
+    i32 = dict(dtype=torch.int32, device=dev)
+    tok_d, conf_d = torch.zeros((S, B), **i32), torch.zeros((S, B), dtype=torch.float32, device=dev)
+    halt_d = torch.zeros((S, B), dtype=torch.uint8, device=dev)
+    sl_d, nacc_d, bonus_d, pos_d = (torch.zeros((B,), **i32) for _ in range(4))
+    dargs = []
+    for it in range(T):
+        d = it % data.n_distinct
+        dargs.append((ring[(it * S) % data.n_rot], data.h_D[d], data.H_T[d],
+                      None if forced_host is None else data.uniform_sl_dev[d], data.draft_dev[d]))
+    t0 = 0.0
+    for it in range(T):
+        if it == Wm:
+            torch.cuda.synchronize()
+            t0 = time.perf_counter()
+        W_D_it, h_D_it, H_T_it, forced_it, ids_it = dargs[it]
+        ctx.iteration(W_D_it, h_D_it, data.W_T, H_T_it, pos_d, clf, wl.tau, S, tok_d, conf_d, halt_d, sl_d, nacc_d, bonus_d,
+                      sl_forced=forced_it, draft_ids=ids_it, pos_next=pos_d, w_step_stride=data.w_stride, stream=stream)
+        stream.synchronize()
+    resident_seconds = time.perf_counter() - t0
+    return {"seconds": seconds, "h2d": per_call_h2d * K, "d2h": per_call_d2h * K, "sl": sl_hist[Wm:], "n_acc": nacc_hist[Wm:],
+            "resident_seconds": resident_seconds}
 
 
 # ------------------------------------------------------------------------------------------ CPU legs

@@ -307,6 +307,36 @@ struct RegTop10 {
         t[1] = max3(t[1], fminf(t[0], a), b);
         t[0] = fmaxf(t[0], a);
     }
+    // Merge with another descending list of ten: both lists laid end to end, the other one reversed, fall
+    // then rise (a bitonic sequence of 32 with -inf in the middle); the half-cleaner of distance 16 leaves the 16
+    // largest in 16 slots, four of them by a comparison and the rest by position, and four more distances sort
+    // them.  A chain of five min/max instead of the hundred of ten insertions; what only feeds slots 10 .. 15 of
+    // the result is dead code.
+    __device__ __forceinline__ void merge(const float (&o)[kTopK]) {
+        static_assert(kTopK == 10, "the network below is written for lists of ten");
+        float L[16];
+#pragma unroll
+        for (int i = 0; i < 6; ++i) L[i] = t[i];
+        L[6] = fmaxf(t[6], o[9]);
+        L[7] = fmaxf(t[7], o[8]);
+        L[8] = fmaxf(t[8], o[7]);
+        L[9] = fmaxf(t[9], o[6]);
+#pragma unroll
+        for (int i = 10; i < 16; ++i) L[i] = o[15 - i];
+#pragma unroll
+        for (int s = 8; s >= 1; s >>= 1) {
+#pragma unroll
+            for (int i = 0; i < 16; ++i) {
+                if ((i & s) == 0) {
+                    const float hi = fmaxf(L[i], L[i + s]), lo = fminf(L[i], L[i + s]);
+                    L[i] = hi;
+                    L[i + s] = lo;
+                }
+            }
+        }
+#pragma unroll
+        for (int k = 0; k < kTopK; ++k) t[k] = L[k];
+    }
     static __device__ __forceinline__ float max3(float x, float y, float z) {
         float d;
         asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(x), "f"(y), "f"(z));

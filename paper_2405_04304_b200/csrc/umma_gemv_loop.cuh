@@ -397,6 +397,7 @@ umma_gemv_loop_kernel(const __grid_constant__ CUtensorMap tmap_W, const __grid_c
         }
         cp_async_wait_all();
         int t_global = 0, fold_calls = 0;
+        int h_ahead_step = -1;     // (thread 0) step whose hidden rows were requested and not yet used
 
         for (int step0 = 0; step0 < lp.steps; ++step0) {
             // stamp of this step's records: unique among everything a reader can still find in the buffer
@@ -441,6 +442,13 @@ umma_gemv_loop_kernel(const __grid_constant__ CUtensorMap tmap_W, const __grid_c
                 named_barrier_sync(1, BAR_THREADS);   // the staging area is overwritten by the next tile
             }
             if (tiles == 0) named_barrier_sync(1, BAR_THREADS);   // the cleared row states are visible
+            // The MMAs of this step are done with the hidden rows: those of the next step are requested now, ahead
+            // of the decision (if the phase stops here they are awaited before the CTA leaves).
+            h_ahead_step = -1;
+            if (tid == 0 && step0 + 1 < lp.steps && total > 0) {
+                loop_issue_hidden(h_tiles, h_stride, KB, &tmap_H, (step0 + 1) * B, h_full);
+                h_ahead_step = step0 + 1;
+            }
             // ---- the CTA's record of this step for each sequence, in stamped pieces ----
             if (tid < B * kStampedPieces) {
                 const int r = tid / kStampedPieces, piece = tid - r * kStampedPieces;
@@ -513,8 +521,6 @@ umma_gemv_loop_kernel(const __grid_constant__ CUtensorMap tmap_W, const __grid_c
                         break;
                     }
                 }
-                // the hidden rows of the next step are requested here, by the first thread to know that it takes place
-                if (code == kLoopContinue && total > 0) loop_issue_hidden(h_tiles, h_stride, KB, &tmap_H, (step0 + 1) * B, h_full);
                 s_code[step0] = code;
                 __threadfence_block();
                 mbar_arrive(go_bar);                // the producer and the MMA issuer go on (or leave)
@@ -522,6 +528,8 @@ umma_gemv_loop_kernel(const __grid_constant__ CUtensorMap tmap_W, const __grid_c
             named_barrier_sync(1, BAR_THREADS);
             if (s_code[step0] != kLoopContinue) break;
         }
+        // rows requested for a step that does not take place: their copy must land before the CTA leaves
+        if (h_ahead_step >= 0) mbar_wait(h_full, h_ahead_step & 1, p.status);
     }
 
     tc_fence_before();

@@ -528,9 +528,7 @@ umma_tail_kernel(const __grid_constant__ CUtensorMap tmap_W, const __grid_consta
                         (static_cast<unsigned long long>(__float_as_uint(cq.w)) << 32) | __float_as_uint(cq.z);
                     key = k2 > key ? k2 : key;
                     const float lv[kTopK] = {a.x, a.y, a.z, a.w, bq.x, bq.y, bq.z, bq.w, cq.x, cq.y};
-#pragma unroll
-                    for (int k = 0; k < kTopK; ++k)
-                        if (lv[k] > top.t[kTopK - 1]) top.push(lv[k]);
+                    top.merge(lv);
                 }
                 store_stamped_record(p.part_rec + ((size_t)row * p.CN + nslot) * kStampedPieces, st.m, st.Z, st.S, top.t,
                                      key, stamp);
