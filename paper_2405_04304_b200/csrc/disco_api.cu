@@ -75,6 +75,8 @@ struct disco_ctx {
     // device staging for the *_host entry points
     void* stage_hidden;
     void* stage_hidden_draft;      // disco_iteration_host: the draft hidden states of all steps
+    cudaStream_t copy_stream;      // disco_iteration_host: the target hidden states travel beside the draft phase
+    cudaEvent_t copy_done;
     // Small inputs and outputs of the *_host entry points live in pinned host memory that the GPU maps:
     // the kernels read and write it in place, so a host call costs one copy (the hidden states), one
     // launch and one synchronisation.  *_h: host address, *_d: the same memory as the device sees it.
@@ -497,6 +499,8 @@ int disco_create(disco_ctx** out, int V, int d_draft, int d_target, int max_batc
     ok = ok && cudaMemset(c->loop_rec, 0, (size_t)4 * c->sm_count * 80) == cudaSuccess;   // no stamp yet
     ok = ok && cudaMalloc(&c->stage_hidden, hid) == cudaSuccess;
     ok = ok && cudaMalloc(&c->stage_hidden_draft, (size_t)max_rows * d_draft * 2) == cudaSuccess;
+    ok = ok && cudaStreamCreateWithFlags(&c->copy_stream, cudaStreamNonBlocking) == cudaSuccess;
+    ok = ok && cudaEventCreateWithFlags(&c->copy_done, cudaEventDisableTiming) == cudaSuccess;
     ok = ok && cudaHostAlloc(&c->stage_int_h, n_int * sizeof(int32_t), cudaHostAllocMapped) == cudaSuccess;
     ok = ok && cudaHostAlloc(&c->stage_float_h, ((size_t)max_batch * (1 + kNFeat) + max_rows) * sizeof(float), cudaHostAllocMapped) == cudaSuccess;
     ok = ok && cudaHostAlloc(&c->stage_byte_h, (size_t)max_batch * 2 + max_rows + 64, cudaHostAllocMapped) == cudaSuccess;
@@ -535,6 +539,8 @@ int disco_destroy(disco_ctx* c) {
     cudaFree(c->pack_off);
     cudaFree(c->stage_hidden);
     cudaFree(c->stage_hidden_draft);
+    if (c->copy_stream) cudaStreamDestroy(c->copy_stream);
+    if (c->copy_done) cudaEventDestroy(c->copy_done);
     cudaFreeHost(c->stage_int_h);
     cudaFreeHost(c->stage_float_h);
     cudaFreeHost(c->stage_byte_h);
@@ -994,11 +1000,13 @@ int disco_verify_sl(disco_ctx* c, const void* W_T, const void* H_T, const int32_
     return verify_common(c, W_T, H_T, draft_ids, nullptr, B, (int)R, sl_max, n_accept, bonus, target_ids, &pad, stream);
 }
 
-int disco_iteration(disco_ctx* c, const void* W_D, size_t w_step_stride, const void* h_D, const void* W_T,
-                    const void* H_T, int B, const int32_t* pos0, const disco_clf* clf, float tau, int sl_max,
-                    const int32_t* sl_forced, const int32_t* draft_ids, int32_t* token, float* conf, uint8_t* halt,
-                    float* feats, int32_t* sl, int32_t* n_accept, int32_t* bonus, int32_t* target_ids,
-                    int32_t* row_off, int32_t* pos_next, void* stream) {
+// late_src (optional): host memory to copy to H_T (late_bytes bytes) on the context's copy stream once the draft
+// phase has been enqueued; the verification waits for it.
+static int iteration_impl(disco_ctx* c, const void* W_D, size_t w_step_stride, const void* h_D, const void* W_T,
+                          const void* H_T, int B, const int32_t* pos0, const disco_clf* clf, float tau, int sl_max,
+                          const int32_t* sl_forced, const int32_t* draft_ids, int32_t* token, float* conf, uint8_t* halt,
+                          float* feats, int32_t* sl, int32_t* n_accept, int32_t* bonus, int32_t* target_ids,
+                          int32_t* row_off, int32_t* pos_next, void* stream, const void* late_src, size_t late_bytes) {
     // everything the second half will check, before the first half is enqueued
     if (!c || !W_T || !H_T || !n_accept || !bonus || !sl) return DISCO_ERR_INVALID_ARG;
     if (!aligned16(W_T) || !aligned16(H_T)) return DISCO_ERR_INVALID_ARG;
@@ -1006,11 +1014,26 @@ int disco_iteration(disco_ctx* c, const void* W_D, size_t w_step_stride, const v
     int rc = disco_draft_loop(c, W_D, w_step_stride, h_D, B, pos0, clf, tau, sl_max, sl_forced, token, conf, halt, feats,
                               sl, stream);
     if (rc) return rc;
+    if (late_src &&
+        (!cuda_ok(cudaMemcpyAsync(const_cast<void*>(H_T), late_src, late_bytes, cudaMemcpyHostToDevice, c->copy_stream),
+                  "cudaMemcpyAsync") ||
+         !cuda_ok(cudaEventRecord(c->copy_done, c->copy_stream), "cudaEventRecord") ||
+         !cuda_ok(cudaStreamWaitEvent(static_cast<cudaStream_t>(stream), c->copy_done, 0), "cudaStreamWaitEvent")))
+        return DISCO_ERR_CUDA;
     if (draft_ids)
         return disco_verify_sl(c, W_T, H_T, draft_ids, sl_max, 1, sl, B, sl_max, n_accept, bonus, target_ids, row_off,
                                pos0, pos_next, stream);
     return disco_verify_sl(c, W_T, H_T, token, 1, B, sl, B, sl_max, n_accept, bonus, target_ids, row_off, pos0,
                            pos_next, stream);
+}
+
+int disco_iteration(disco_ctx* c, const void* W_D, size_t w_step_stride, const void* h_D, const void* W_T,
+                    const void* H_T, int B, const int32_t* pos0, const disco_clf* clf, float tau, int sl_max,
+                    const int32_t* sl_forced, const int32_t* draft_ids, int32_t* token, float* conf, uint8_t* halt,
+                    float* feats, int32_t* sl, int32_t* n_accept, int32_t* bonus, int32_t* target_ids,
+                    int32_t* row_off, int32_t* pos_next, void* stream) {
+    return iteration_impl(c, W_D, w_step_stride, h_D, W_T, H_T, B, pos0, clf, tau, sl_max, sl_forced, draft_ids, token, conf,
+                          halt, feats, sl, n_accept, bonus, target_ids, row_off, pos_next, stream, nullptr, 0);
 }
 
 int disco_draft_step_host(disco_ctx* c, const void* W_D, const void* h_D_host, int B, const int32_t* pos_host,
@@ -1121,14 +1144,20 @@ int disco_iteration_host(disco_ctx* c, const void* W_D, size_t w_step_stride, co
     std::memcpy(h_tok, token_host, SB * 4);
     std::memcpy(h_conf, conf_host, SB * 4);
     std::memcpy(h_halt, halt_host, SB);
-    if (cudaMemcpyAsync(c->stage_hidden_draft, h_D_host, SB * c->d_draft * 2, cudaMemcpyHostToDevice, st) != cudaSuccess ||
-        cudaMemcpyAsync(c->stage_hidden, H_T_host, R * c->d_target * 2, cudaMemcpyHostToDevice, st) != cudaSuccess)
+    // The draft phase needs the draft hidden states only: the (larger) target hidden states are sent once it is
+    // enqueued, on a stream of their own, and the verification waits for them.  (Every host entry point returns with its
+    // work done, so nothing earlier still reads the staging buffers.)
+    if (cudaMemcpyAsync(c->stage_hidden_draft, h_D_host, SB * c->d_draft * 2, cudaMemcpyHostToDevice, st) != cudaSuccess)
         return DISCO_ERR_CUDA;
-    int rc = disco_iteration(c, W_D, w_step_stride, c->stage_hidden_draft, W_T, c->stage_hidden, B, dev_i(h_pos), clf, tau,
-                             sl_max, sl_forced_host ? dev_i(h_forced) : nullptr, draft_ids_host ? dev_i(h_ids) : nullptr,
-                             dev_i(h_tok), c->stage_float_d, c->stage_byte_d, nullptr, dev_i(h_sl), dev_i(h_nacc),
-                             dev_i(h_bonus), nullptr, nullptr, pos_next_host ? dev_i(h_next) : nullptr, stream);
-    if (rc) return rc;
+    int rc = iteration_impl(c, W_D, w_step_stride, c->stage_hidden_draft, W_T, c->stage_hidden, B, dev_i(h_pos), clf, tau,
+                            sl_max, sl_forced_host ? dev_i(h_forced) : nullptr, draft_ids_host ? dev_i(h_ids) : nullptr,
+                            dev_i(h_tok), c->stage_float_d, c->stage_byte_d, nullptr, dev_i(h_sl), dev_i(h_nacc),
+                            dev_i(h_bonus), nullptr, nullptr, pos_next_host ? dev_i(h_next) : nullptr, stream, H_T_host,
+                            R * c->d_target * 2);
+    if (rc) {
+        cudaStreamSynchronize(c->copy_stream);   // the copy must not outlive the call
+        return rc;
+    }
     if (cudaStreamSynchronize(st) != cudaSuccess) return DISCO_ERR_CUDA;
     std::memcpy(token_host, h_tok, SB * 4);
     std::memcpy(conf_host, h_conf, SB * 4);
