@@ -180,7 +180,9 @@ int disco_draft_step_sample(disco_ctx* ctx, const void* W_D, const void* h_D, in
  * accepted (a residual without mass falls back to y^T_n).
  *   draft_ids    int32 [R - B], device   packed as in disco_verify_ragged
  *   draft_probs  float [steps, B, V], device, steps >= max SL_b: draft_probs[i, b, :] = y^D of token i of
- *                sequence b (the probs output of draft step i); NULL allowed iff R == B
+ *                sequence b (the probs output of draft step i); NULL allowed iff R == B.  The kernel cannot see
+ *                `steps`: it reads draft_probs[i] for every i below the look-ahead that row_off gives a sequence
+ *                (at most R - B), so a caller that cannot vouch for row_off sizes the array for R - B steps
  *   row_off      int32 [B + 1], device, or NULL for a uniform SL = R / B - 1
  *   u_accept     float [R - B], device   uniforms in [0, 1), packed like draft_ids
  *   u_sample     float [B], device       uniforms in [0, 1)

@@ -760,6 +760,63 @@ def test_verify_sample_edge_cases(oracle):
     assert n[0] == SL and n[2] == SL and n[1] == 2
 
 
+def test_verify_sample_context_is_reusable_after_malformed_offsets(oracle):
+    """The per-sequence tickets of the sampling kernel live in the context.  A call with overlapping row offsets
+    (reported as an invalid argument) may leave them half counted; the next call must not inherit that: the same
+    well-formed call before and after gives the same answer, and the answer matches the oracle."""
+    V, d, sls = 1500, 72, [3, 0, 5, 2]
+    B, R = len(sls), sum(sls) + len(sls)
+    row_off = np.concatenate([[0], np.cumsum(np.array(sls) + 1)]).astype(np.int32)
+    W = inputs.lm_head(V, d, seed=31, std=0.25)
+    H = inputs.hidden(R, d, seed=32)
+    rng = np.random.default_rng(33)
+    z = oracle.project(_bits(W), _bits(H), nthreads=8)
+    S = R - B          # as many steps as any look-ahead that fits the rows: whatever offsets arrive, reads stay inside
+    dp = np.full((S, B, V), 1.0 / V, dtype=np.float32)
+    ids = np.zeros(R - B, dtype=np.int32)
+    for b in range(B):
+        for i in range(sls[b]):
+            zz = z[row_off[b] + i] + rng.normal(0.0, 1.0, V)
+            e = np.exp(zz - zz.max())
+            dp[i, b] = (e / e.sum()).astype(np.float32)
+            ids[row_off[b] - b + i] = rng.choice(V, p=dp[i, b].astype(np.float64) / dp[i, b].astype(np.float64).sum())
+    ua = rng.uniform(0.0, 1.0, R - B).astype(np.float32)
+    us = rng.uniform(0.0, 1.0, B).astype(np.float32)
+    ctx = _ctx(V, 8, d, max_batch=8, max_rows=64)
+    Wc, Hc = W.cuda(), H.cuda()
+    dev = lambda a: torch.from_numpy(a).cuda()
+
+    def run(off):
+        n_acc = torch.full((B,), -7, dtype=torch.int32, device="cuda")
+        nxt = torch.full((B,), -7, dtype=torch.int32, device="cuda")
+        y = torch.zeros((R, V), dtype=torch.float32, device="cuda")
+        ctx.verify_sample_ragged(Wc, Hc, dev(ids), dev(dp), dev(off), B, R, dev(ua), dev(us), n_acc, nxt, y)
+        torch.cuda.synchronize()
+        return n_acc.cpu().numpy(), nxt.cpu().numpy(), y.cpu().numpy(), ctx.device_status()
+
+    n1, x1, y1, st1 = run(row_off)
+    assert st1 == 0
+    bad = row_off.copy()
+    bad[2] = bad[1] - 1          # sequence 1 ends before it starts; sequence 2 overlaps sequence 0
+    _, _, _, st_bad = run(bad)
+    assert st_bad == binding.ERR_INVALID_ARG
+    n2, x2, y2, st2 = run(row_off)
+    assert st2 == 0
+    np.testing.assert_array_equal(n1, n2)
+    np.testing.assert_array_equal(x1, x2)
+    np.testing.assert_array_equal(y1, y2)
+    ctx.close()
+    ref = oracle.verify_sample(_bits(W), _bits(H), ids, dp, row_off, ua.astype(np.float64), us.astype(np.float64), nthreads=8)
+    np.testing.assert_allclose(y1, ref.y_T, rtol=0, atol=2e-3)
+    for b in range(B):
+        if int(n1[b]) == int(ref.n_accept[b]):
+            n = int(n1[b])
+            r0 = int(row_off[b])
+            w = np.maximum(0.0, ref.y_T[r0 + n] - dp[n, b].astype(np.float64)) if n < sls[b] else ref.y_T[r0 + sls[b]]
+            assert x1[b] == ref.next_token[b] or _valid_draw(w, float(us[b]), int(x1[b]))
+    assert (n1 == ref.n_accept).sum() >= B - 1      # an acceptance decided in the last bits may go either way
+
+
 def test_look_ahead_is_monotone_in_the_threshold_at_full_size():
     """Batched Starcoder shapes, no oracle needed: on the same stream of hidden states the look-ahead that the
     stopping rule produces cannot grow with the threshold, the cap ends every sequence, and tau <= 0 never
