@@ -340,9 +340,11 @@ int disco_verify_ragged_host(disco_ctx* ctx, const void* W_T /*device*/, const v
  * disco_iteration for a caller whose per-iteration data lives in HOST memory: the hidden states of all steps,
  * the target rows, pos0, sl_forced and draft_ids (either may be NULL) are host pointers, and so are the
  * outputs token, conf, halt [sl_max, B], sl, n_accept, bonus [B] and pos_next [B] (or NULL; may be pos0_host
- * itself).  One copy of each hidden-state block to device staging, the small arrays through pinned memory
- * that the GPU maps, the whole iteration on the device, one synchronisation.  The LM heads and the classifier
- * stay on the device.  Entries of steps a sequence did not take keep the caller's values.
+ * itself).  One copy of each hidden-state block to device staging (the target rows travel on a stream the
+ * context owns while the draft phase runs on the caller's; the verification waits for them), the small arrays
+ * through pinned memory that the GPU maps, the whole iteration on the device, one synchronisation.  The LM
+ * heads and the classifier stay on the device.  Entries of steps a sequence did not take keep the caller's
+ * values.  Like every *_host entry point it returns with its work done, and it cannot be captured in a graph.
  */
 int disco_iteration_host(disco_ctx* ctx, const void* W_D /*device*/, size_t w_step_stride, const void* h_D_host,
                          const void* W_T /*device*/, const void* H_T_host, int B, const int32_t* pos0_host,
