@@ -37,6 +37,35 @@ def test_draft_step_small_shapes(oracle, V, d, B):
     ctx.close()
 
 
+@pytest.mark.parametrize("path", [0, 1, 2, 3])
+def test_every_small_vocabulary(oracle, path):
+    """V = 1 .. 64 without a gap (fewer than ten logits, one CTA with rows and 147 without, ragged last tile), two
+    sequences, both tails, on each kernel family."""
+    d, B, SL = 16, 2, 3
+    params = make_clf(8, seed=5)
+    clf_g, clf_o = to_gpu_clf(params), to_oracle_clf(oracle, params)
+    pos, nd = np.array([4, 9], np.int32), np.array([1, 2], np.int32)
+    for V in range(1, 65):
+        W = inputs.lm_head(V, d, seed=1000 + V, std=0.3)
+        h = inputs.hidden(B, d, seed=2000 + V)
+        ctx = _ctx(V, d, d, max_batch=8, max_rows=64, H=8)
+        ctx.set_kernel_path(path)
+        got = gpu_draft_step(ctx, W.cuda(), h, pos, nd, clf_g, 0.5, 3, want_probs=True)
+        ref = oracle.draft_step(_bits(W), _bits(h), pos, nd, clf_o, 0.5, 3, want_probs=True)
+        check_draft(got, ref, 0.5)
+        R = B * (SL + 1)
+        H = inputs.hidden(R, d, seed=3000 + V)
+        off = np.arange(B + 1, dtype=np.int32) * (SL + 1)
+        free = oracle.verify_ragged(_bits(W), _bits(H), np.zeros(R - B, np.int32), off)
+        clean = np.concatenate([free.target_ids[off[b]:off[b + 1] - 1] for b in range(B)]).astype(np.int32)
+        draft = inputs.corrupt_ids(torch.from_numpy(clean), 0.3, V, seed=V).numpy()
+        refv = oracle.verify_ragged(_bits(W), _bits(H), draft, off)
+        gotv = gpu_verify(ctx, W.cuda(), H, draft, row_off=off)
+        check_verify(gotv, refv, off, draft, near_tie_ids(oracle, _bits(W), _bits(H), refv.gap))
+        assert ctx.device_status() == 0, f"V = {V}"
+        ctx.close()
+
+
 def test_draft_step_tiny_workload_shapes(oracle):
     wl = inputs.WORKLOADS["tiny"]
     W = inputs.lm_head(wl.V, wl.d_D, seed=inputs.sub_seed(wl.seed, 1))
