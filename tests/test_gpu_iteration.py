@@ -181,6 +181,24 @@ def test_iteration_small_shapes(oracle, V, dD, dT, B, S, split, graph):
     ctx.close()
 
 
+@pytest.mark.parametrize("B", [1, 2, 4, 5])
+def test_iteration_every_small_vocabulary(oracle, B):
+    """V = 1 .. 48 without a gap through the whole iteration: the persistent draft-phase kernel for up to four
+    sequences (147 CTAs without a vocabulary row, fewer than ten logits), the chained per-step launches for five."""
+    dD, dT, S = 16, 24, 4
+    params = position_clf(cut=6.0)
+    clf_g, clf_o = to_gpu_clf(params), to_oracle_clf(oracle, params)
+    pos0 = (np.arange(B, dtype=np.int32) * 2 + 3) % 8
+    for V in range(1, 49):
+        W_D, W_T, h_D, H_T = make_inputs(V, dD, dT, B, S, seed=500 + V)
+        ctx = binding.Context(V, dD, dT, max_batch=B, max_rows=B * (S + 1), clf_hidden=8)
+        got = gpu_iteration(ctx, W_D, W_T, h_D, H_T, pos0, clf_g, 0.5, S)
+        ref = oracle.iteration(_bits(W_D), _bits(h_D), _bits(W_T), _bits(H_T), pos0, clf_o, 0.5, S, nthreads=4)
+        check_iteration(oracle, got, ref, W_T, H_T, 0.5, S)
+        assert ctx.device_status() == 0, f"V = {V}"
+        ctx.close()
+
+
 @pytest.mark.parametrize("path", [1, 2, 3])
 @pytest.mark.parametrize("B", [2, 12])
 def test_iteration_on_each_kernel_path(oracle, path, B):
