@@ -37,14 +37,15 @@ def test_draft_step_small_shapes(oracle, V, d, B):
     ctx.close()
 
 
+@pytest.mark.parametrize("B", [1, 2, 3])
 @pytest.mark.parametrize("path", [0, 1, 2, 3])
-def test_every_small_vocabulary(oracle, path):
-    """V = 1 .. 64 without a gap (fewer than ten logits, one CTA with rows and 147 without, ragged last tile), two
-    sequences, both tails, on each kernel family."""
-    d, B, SL = 16, 2, 3
+def test_every_small_vocabulary(oracle, path, B):
+    """V = 1 .. 64 without a gap (fewer than ten logits, one CTA with rows and 147 without, ragged last tile), the
+    narrowest hidden state, one to three sequences, both tails, on each kernel family."""
+    d, SL = 8, 3
     params = make_clf(8, seed=5)
     clf_g, clf_o = to_gpu_clf(params), to_oracle_clf(oracle, params)
-    pos, nd = np.array([4, 9], np.int32), np.array([1, 2], np.int32)
+    pos, nd = np.array([4, 9, 2][:B], np.int32), np.array([1, 2, 3][:B], np.int32)
     for V in range(1, 65):
         W = inputs.lm_head(V, d, seed=1000 + V, std=0.3)
         h = inputs.hidden(B, d, seed=2000 + V)
